@@ -1,0 +1,384 @@
+"""CPU oracle for the GRAM training step.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain statement of what the CUDA library must compute.
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+it; the product path never does, and it shares no code with the CUDA sources.
+
+What it states, and from where in the paper:
+
+* `e2e_step`: standard end-to-end training (Section 3.3): the content encoder
+  CE runs once per *interaction* (every occurrence of an item, duplicates
+  included), the task module CF consumes the encodings, and the loss is
+  back-propagated through every one of those encoder calls; parameter gradients
+  sum over occurrences.  Single-step GRAM reaches exactly this gradient by a
+  cheaper route (Proposition, Section 4.1), so this definition is its oracle.
+* `gram_single_step`: the route itself (Algorithm 1 with N = 1): encode the
+  unique items once (Eq. 4), task forward/backward (Eq. 5), sum dL/dh over the
+  occurrences of each item (Eq. 6 with SGD of learning rate 1 makes
+  h - h~ equal to that sum), and one encoder VJP per unique item (Eq. 7).
+  It exists to check the Proposition on the oracle itself.
+* `multistep_window`: Algorithm 1 with N = K > 1, step by step.  The paper
+  states that this is not equivalent to end-to-end training, so there is no
+  plain definition to reduce to; the readings taken where the algorithm is
+  silent are listed in the function's docstring.
+* `unique_inverse_bruteforce`, `unique_inverse`, `segment_sum`,
+  `table_accumulate`: the index work and the per-item sums on their own.
+* `boost_ratio`: the speed-boost ratio R (Section 4.4).
+
+Arithmetic is float64 throughout unless a caller passes another dtype: the
+paper never fixes a precision.  Derivatives of the end-to-end definition come
+from torch's autograd over the plain forward written here; the tests pin that
+combination with central finite differences and closed forms.
+
+Pins (tests/test_oracle_*.py): brute force on tiny inputs, the worked count
+of Fig. 1, finite differences on a 1-layer encoder, closed forms of softmax /
+LayerNorm / GELU / BCE, the Proposition (e2e == single-step), the pseudo-loss
+identity (Eqs. 1-3), K = 1 reducing to single-step, and conservation of
+column sums.  The Multi-step *trajectory* beyond those is pinned only by the
+readings below: parity unpinned by the paper for that part.
+"""
+from __future__ import annotations
+
+import math
+from collections import OrderedDict
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+import torch
+
+LN_EPS = 1e-5
+
+
+# ---------------------------------------------------------------------------
+# index work: the unique-item set B_I of a mini-batch (Table 1) and the map
+# from occurrences to items that Fig. 1 draws
+# ---------------------------------------------------------------------------
+
+def unique_inverse_bruteforce(ids) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """O(P*U) scan, for tiny inputs.  Returns
+    unique   ascending distinct IDs                                  [U]
+    inverse  unique[inverse[p]] == ids[p]                            [P]
+    perm     positions grouped by item, ascending inside each group  [P]
+    seg_off  group u is perm[seg_off[u]:seg_off[u+1]]                [U+1]
+    """
+    ids = [int(v) for v in np.asarray(ids).ravel()]
+    unique: List[int] = []
+    for v in ids:
+        if v not in unique:
+            unique.append(v)
+    # ascending order by repeated minimum selection
+    ordered: List[int] = []
+    rest = list(unique)
+    while rest:
+        m = min(rest)
+        ordered.append(m)
+        rest.remove(m)
+    inverse = [ordered.index(v) for v in ids]
+    perm: List[int] = []
+    seg_off = [0]
+    for u in range(len(ordered)):
+        for p, v in enumerate(ids):
+            if v == ordered[u]:
+                perm.append(p)
+        seg_off.append(len(perm))
+    i32 = np.int32
+    return (np.array(ordered, i32), np.array(inverse, i32), np.array(perm, i32), np.array(seg_off, i32))
+
+
+def unique_inverse(ids) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Same result at any size: a library stable sort, then one scan."""
+    ids = np.asarray(ids).ravel().astype(np.int64)
+    P = ids.size
+    perm = np.argsort(ids, kind="stable")
+    sk = ids[perm]
+    head = np.ones(P, dtype=bool)
+    head[1:] = sk[1:] != sk[:-1]
+    starts = np.nonzero(head)[0]
+    unique = sk[starts]
+    seg_off = np.concatenate([starts, [P]])
+    seg_of_sorted = np.cumsum(head) - 1
+    inverse = np.empty(P, dtype=np.int64)
+    inverse[perm] = seg_of_sorted
+    i32 = np.int32
+    return unique.astype(i32), inverse.astype(i32), perm.astype(i32), seg_off.astype(i32)
+
+
+def boost_ratio(n_interactions: int, n_items: int) -> float:
+    """R = #interactions / #items (Section 4.4)."""
+    return float(n_interactions) / float(n_items)
+
+
+def segment_sum(dE, perm, seg_off) -> np.ndarray:
+    """G[u, :] = sum of dE[perm[j], :] over j in [seg_off[u], seg_off[u+1]), in
+    float64, rows added in ascending j (Eq. 6: every occurrence of item u
+    contributes its gradient to the one pseudo-target of u)."""
+    dE = np.asarray(dE, dtype=np.float64)
+    U = len(seg_off) - 1
+    G = np.zeros((U, dE.shape[1]), dtype=np.float64)
+    for u in range(U):
+        for j in range(int(seg_off[u]), int(seg_off[u + 1])):
+            G[u, :] += dE[int(perm[j]), :]
+    return G
+
+
+def table_accumulate(table, touched, dE, ids) -> None:
+    """Multi-step accumulation in place: table[ids[p], :] += dE[p, :] for p in
+    ascending order, touched[ids[p]] = True (Section 4.2: gradient buffers are
+    kept per item across several mini-batches)."""
+    dE = np.asarray(dE, dtype=np.float64)
+    for p, i in enumerate(np.asarray(ids).ravel()):
+        table[int(i), :] += dE[p, :]
+        touched[int(i)] = True
+
+
+# ---------------------------------------------------------------------------
+# the two modules.  CE: a BERT-shaped post-LayerNorm transformer over one
+# item's tokens (Appendix D: MHSA layers of width 768; mean pooling for KT).
+# CF: the task module over a history of encodings (Section 3.1).
+# ---------------------------------------------------------------------------
+
+def layer_norm(x: torch.Tensor, g: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    mu = x.mean(dim=-1, keepdim=True)
+    var = ((x - mu) ** 2).mean(dim=-1, keepdim=True)
+    return (x - mu) / torch.sqrt(var + LN_EPS) * g + b
+
+
+def gelu(x: torch.Tensor) -> torch.Tensor:
+    return 0.5 * x * (1.0 + torch.erf(x / math.sqrt(2.0)))
+
+
+def softmax_rows(s: torch.Tensor) -> torch.Tensor:
+    e = torch.exp(s - s.max(dim=-1, keepdim=True).values)
+    return e / e.sum(dim=-1, keepdim=True)
+
+
+def attention(x: torch.Tensor, th: Dict[str, torch.Tensor], pre: str, n_heads: int, causal: bool) -> torch.Tensor:
+    """Multi-head self-attention over one sequence x [S, d], output projection
+    included.  Rows 0..d-1 of wqkv give Q, d..2d-1 K, 2d..3d-1 V; head h owns
+    columns h*d_h..(h+1)*d_h of each."""
+    S, d = x.shape
+    dh = d // n_heads
+    qkv = x @ th[pre + "wqkv"].T + th[pre + "bqkv"]
+    q, k, v = qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:]
+    heads = []
+    for h in range(n_heads):
+        sl = slice(h * dh, (h + 1) * dh)
+        s = (q[:, sl] @ k[:, sl].T) / math.sqrt(dh)
+        if causal:
+            mask = torch.ones(S, S, dtype=torch.bool).tril()
+            s = torch.where(mask, s, torch.full_like(s, -float("inf")))
+        heads.append(softmax_rows(s) @ v[:, sl])
+    ctx = torch.cat(heads, dim=1)
+    return ctx @ th[pre + "wo"].T + th[pre + "bo"]
+
+
+def transformer_layer(x, th, pre, n_heads, causal, attn_only=False):
+    a = attention(x, th, pre, n_heads, causal)
+    if attn_only:
+        return x + a
+    h1 = layer_norm(x + a, th[pre + "ln1_g"], th[pre + "ln1_b"])
+    f = gelu(h1 @ th[pre + "w1"].T + th[pre + "b1"]) @ th[pre + "w2"].T + th[pre + "b2"]
+    return layer_norm(h1 + f, th[pre + "ln2_g"], th[pre + "ln2_b"])
+
+
+def ce_forward(th: Dict[str, torch.Tensor], tokens, shape) -> torch.Tensor:
+    """h = CE(c; theta_CE) for ONE item: tokens [l_t] -> encoding [d]."""
+    tok = torch.as_tensor(np.asarray(tokens), dtype=torch.long)
+    x = th["tok_emb"][tok] + th["pos_emb"]
+    x = layer_norm(x, th["emb_ln_g"], th["emb_ln_b"])
+    for l in range(shape.n_layers):
+        x = transformer_layer(x, th, f"l{l}.", shape.n_heads, causal=False)
+    if shape.pooling == "mean":
+        return x.mean(dim=0)
+    if shape.pooling == "cls":
+        return x[0]
+    raise KeyError(shape.pooling)
+
+
+def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> torch.Tensor:
+    """The CF objective (Eq. 8) over a mini-batch: E [B, L, d] -> scalar.
+
+    kt: the model sees interactions (e_1, r_1) .. (e_{n-1}, r_{n-1}) and the
+        next item e_n, and predicts r_n (Section 3.1): input
+        x_n = E[b, n] + pos[n] + resp[r_{n-1}] (resp row 2 marks "no previous
+        response" at n = 0), causal attention, logit_n = head_w . y_n + head_b,
+        binary cross-entropy, averaged over all B*L predictions.
+    nr: additive attention over the first L - n_cand encodings gives the user
+        vector, dot products with the n_cand candidate encodings give scores,
+        loss = -log softmax(scores)[0] (the first candidate is the click),
+        averaged over the B users.
+    """
+    B, L, d = E.shape
+    lab = torch.as_tensor(np.asarray(labels), dtype=torch.long)
+    if shape.task == "kt":
+        total = E.new_zeros(())
+        for b in range(B):
+            prev = torch.cat([torch.full((1,), 2, dtype=torch.long), lab[b, :-1]])
+            x = E[b] + th["pos"] + th["resp"][prev]
+            for l in range(shape.task_layers):
+                x = transformer_layer(x, th, f"t{l}.", shape.task_heads, causal=True,
+                                      attn_only=shape.task_attn_only)
+            z = x @ th["head_w"] + th["head_b"]
+            y = lab[b].to(E.dtype)
+            # BCE with logits: softplus(z) - y*z, written with a stable softplus
+            total = total + (torch.clamp(z, min=0) + torch.log1p(torch.exp(-z.abs())) - y * z).sum()
+        return total / (B * L)
+    if shape.task == "nr":
+        n_hist = L - shape.n_cand
+        total = E.new_zeros(())
+        for b in range(B):
+            hist, cand = E[b, :n_hist], E[b, n_hist:]
+            a = torch.tanh(hist @ th["wa"].T + th["ba"]) @ th["qa"]
+            alpha = softmax_rows(a[None, :])[0]
+            u = alpha @ hist
+            s = cand @ u
+            total = total - (s[0] - s.max() - torch.log(torch.exp(s - s.max()).sum()))
+        return total / B
+    raise KeyError(shape.task)
+
+
+# ---------------------------------------------------------------------------
+# helpers
+# ---------------------------------------------------------------------------
+
+def as_torch(params: Dict[str, np.ndarray], dtype=torch.float64, requires_grad=True) -> "OrderedDict[str, torch.Tensor]":
+    out: "OrderedDict[str, torch.Tensor]" = OrderedDict()
+    for k, v in params.items():
+        t = torch.tensor(np.asarray(v), dtype=dtype)
+        t.requires_grad_(requires_grad)
+        out[k] = t
+    return out
+
+
+def _grads(th: Dict[str, torch.Tensor]) -> "OrderedDict[str, np.ndarray]":
+    out: "OrderedDict[str, np.ndarray]" = OrderedDict()
+    for k, t in th.items():
+        out[k] = (t.grad if t.grad is not None else torch.zeros_like(t)).detach().numpy().copy()
+    return out
+
+
+# ---------------------------------------------------------------------------
+# standard end-to-end training: the definition (Section 3.3)
+# ---------------------------------------------------------------------------
+
+def e2e_step(shape, ce_params, task_params, item_tokens, ids, labels, dtype=torch.float64):
+    """One end-to-end gradient evaluation.  The encoder is called afresh for
+    every occurrence; nothing is shared between two occurrences of an item.
+    Returns dict(loss, grad_ce, grad_task, E)."""
+    ids = np.asarray(ids)
+    B, L = ids.shape
+    th_ce = as_torch(ce_params, dtype)
+    th_cf = as_torch(task_params, dtype)
+    rows = []
+    for b in range(B):
+        rows.append(torch.stack([ce_forward(th_ce, item_tokens[int(ids[b, n])], shape) for n in range(L)]))
+    E = torch.stack(rows)
+    loss = task_loss(th_cf, E, labels, shape)
+    loss.backward()
+    return dict(loss=float(loss.detach()), grad_ce=_grads(th_ce), grad_task=_grads(th_cf),
+                E=E.detach().numpy().copy())
+
+
+# ---------------------------------------------------------------------------
+# Single-step GRAM (Algorithm 1, N = 1), used to check the Proposition
+# ---------------------------------------------------------------------------
+
+def gram_single_step(shape, ce_params, task_params, item_tokens, ids, labels, dtype=torch.float64):
+    """Returns dict(loss, grad_ce, grad_task, H, G, dE, unique, inverse)."""
+    ids = np.asarray(ids)
+    B, L = ids.shape
+    unique, inverse, perm, seg_off = unique_inverse(ids)
+    th_ce = as_torch(ce_params, dtype)
+    th_cf = as_torch(task_params, dtype)
+    # Eq. 4: one encoding per unique item
+    H = torch.stack([ce_forward(th_ce, item_tokens[int(i)], shape) for i in unique])
+    # the task module sees the encodings as leaves ("trainable embeddings")
+    E = H.detach()[torch.as_tensor(inverse.astype(np.int64))].reshape(B, L, -1).clone().requires_grad_(True)
+    loss = task_loss(th_cf, E, labels, shape)
+    loss.backward()                                  # Eq. 5 gradients, and dL/dE
+    dE = E.grad.reshape(B * L, -1).numpy()
+    # Eq. 6: h~_i = h_i - sum over occurrences of dL/dE, so h_i - h~_i = G_i
+    G = segment_sum(dE, perm, seg_off)
+    # Eq. 7 / Eq. 9: gradient of 1/2 sum_i (h~_i - CE(c_i))^2 at the current
+    # parameters is the VJP of CE with cotangent (h_i - h~_i) = G_i
+    H.backward(torch.tensor(G, dtype=dtype))
+    return dict(loss=float(loss.detach()), grad_ce=_grads(th_ce), grad_task=_grads(th_cf),
+                H=H.detach().numpy().copy(), G=G, dE=dE.copy(), unique=unique, inverse=inverse)
+
+
+def pseudo_loss_grad(shape, ce_params, item_tokens, items, h_tilde, dtype=torch.float64):
+    """Gradient of the pseudo-loss 1/2 sum_i (h~_i - CE(c_i; theta'))^2 (Eq. 9)
+    with respect to theta' at the given parameters; h_tilde is a constant."""
+    th = as_torch(ce_params, dtype)
+    H = torch.stack([ce_forward(th, item_tokens[int(i)], shape) for i in items])
+    lt = 0.5 * ((torch.tensor(np.asarray(h_tilde), dtype=dtype) - H) ** 2).sum()
+    lt.backward()
+    return float(lt.detach()), _grads(th)
+
+
+# ---------------------------------------------------------------------------
+# Multi-step GRAM (Algorithm 1, N = K > 1)
+# ---------------------------------------------------------------------------
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even to bfloat16, returned in float64."""
+    return torch.tensor(np.asarray(a), dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def encode_all(shape, ce_params, item_tokens, items, dtype=torch.float64) -> np.ndarray:
+    th = as_torch(ce_params, dtype, requires_grad=False)
+    with torch.no_grad():
+        return torch.stack([ce_forward(th, item_tokens[int(i)], shape) for i in items]).numpy()
+
+
+def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache, lr_task: float,
+                     cache_bf16: bool = False, dtype=torch.float64):
+    """One window of K = len(batches) steps of Algorithm 1, then the encoder
+    pass.  Readings where the algorithm is silent or ambiguous:
+
+    * Step 1 (Eq. 4) inside a window reads the per-item encoding from `cache`
+      [n_items, d] (values computed before the window) instead of re-running
+      CE, since CE's parameters do not change inside a window.
+    * Step 2 (Eq. 5): `opt` is plain SGD with learning rate lr_task, applied
+      after every step, so later steps of the window see updated task
+      parameters.
+    * Step 3 (Eq. 6): the per-item modification h_i - h~_i accumulates in a
+      separate table (the cache itself stays unchanged during the window):
+      table[i] += dL/dE[p] for every occurrence p of item i, in position order.
+    * Step 4 fires after the K-th step of the window (the printed test
+      `t mod N = 0` with t counted from 1), over ALL items touched in the
+      window, with cotangent table[i]; its forward uses the current encoder
+      parameters, and that forward value replaces cache[i].
+
+    Returns dict(losses [K], grad_ce (sum over touched items in ascending item
+    order), grad_task_last, task_params (after K SGD steps), table, touched,
+    cache (updated))."""
+    n_items, d = cache.shape
+    cache = np.array(cache, dtype=np.float64)
+    if cache_bf16:
+        cache = round_to_bf16(cache)
+    table = np.zeros((n_items, d), dtype=np.float64)
+    touched = np.zeros(n_items, dtype=bool)
+    cur_task = OrderedDict((k, np.array(v, dtype=np.float64)) for k, v in task_params.items())
+    losses = []
+    grad_task_last = None
+    for ids, labels in batches:
+        ids = np.asarray(ids)
+        B, L = ids.shape
+        th_cf = as_torch(cur_task, dtype)
+        E = torch.tensor(cache[ids.ravel()], dtype=dtype).reshape(B, L, d).requires_grad_(True)
+        loss = task_loss(th_cf, E, labels, shape)
+        loss.backward()
+        losses.append(float(loss.detach()))
+        grad_task_last = _grads(th_cf)
+        for k in cur_task:
+            cur_task[k] = cur_task[k] - lr_task * grad_task_last[k]
+        table_accumulate(table, touched, E.grad.reshape(B * L, d).numpy(), ids)
+    items = np.nonzero(touched)[0]
+    th_ce = as_torch(ce_params, dtype)
+    H = torch.stack([ce_forward(th_ce, item_tokens[int(i)], shape) for i in items])
+    H.backward(torch.tensor(table[items], dtype=dtype))
+    newc = H.detach().numpy()
+    cache[items] = round_to_bf16(newc) if cache_bf16 else newc
+    return dict(losses=losses, grad_ce=_grads(th_ce), grad_task_last=grad_task_last, task_params=cur_task,
+                table=table, touched=touched, cache=cache, items=items.astype(np.int32))

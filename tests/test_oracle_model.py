@@ -1,0 +1,253 @@
+"""Pins for the oracle's encoder / task module and for the training schemes (CPU only)."""
+import math
+from collections import OrderedDict
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gram_oracle as orc
+from paper_2204_04179_b200 import synth
+
+T64 = torch.float64
+
+
+def small_shape(**kw):
+    base = dict(name="s", n_items=7, l_t=4, vocab=20, d=16, n_heads=2, d_ff=32, n_layers=1, pooling="mean",
+                task="kt", task_layers=1, task_heads=2, task_d_ff=32, task_attn_only=True, B=2, L=5, zipf_s=1.1)
+    base.update(kw)
+    return synth.GramShape(**base)
+
+
+def make(shape, seed=0, sigma=0.3):
+    ce = synth.encoder_params(shape, seed, sigma=sigma, plain=False)
+    tk = synth.task_params(shape, seed, sigma=sigma, plain=False)
+    toks = synth.item_tokens(seed, shape.n_items, shape.l_t, shape.vocab)
+    ids, lab = synth.batch(shape, seed)
+    return ce, tk, toks, ids, lab
+
+
+# ---- closed forms and library routines ------------------------------------
+
+def test_gelu_and_layernorm_closed_forms():
+    x = torch.tensor([0.0, 1.0, -1.0, 3.0], dtype=T64)
+    phi = lambda v: 0.5 * (1 + math.erf(v / math.sqrt(2)))
+    np.testing.assert_allclose(orc.gelu(x).numpy(), [0.0, phi(1.0), -phi(-1.0), 3 * phi(3.0)], rtol=1e-14)
+    assert abs(float(orc.gelu(x)[1]) - 0.8413447460685429) < 1e-15
+    r = torch.randn(5, 12, dtype=T64, generator=torch.Generator().manual_seed(0)) * 3 + 1
+    y = orc.layer_norm(r, torch.ones(12, dtype=T64), torch.zeros(12, dtype=T64))
+    np.testing.assert_allclose(y.mean(-1).numpy(), 0, atol=1e-14)
+    var = r.var(-1, unbiased=False)
+    np.testing.assert_allclose((y ** 2).mean(-1).numpy(), (var / (var + orc.LN_EPS)).numpy(), rtol=1e-12)
+    g, b = torch.randn(12, dtype=T64), torch.randn(12, dtype=T64)
+    np.testing.assert_allclose(orc.layer_norm(r, g, b).numpy(),
+                               torch.nn.functional.layer_norm(r, (12,), g, b, eps=orc.LN_EPS).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_attention_uniform_scores_is_running_mean():
+    # Q = 0 makes every score equal, so causal attention returns the running mean of V
+    S, d = 6, 8
+    th = {"a.wqkv": torch.zeros(3 * d, d, dtype=T64), "a.bqkv": torch.zeros(3 * d, dtype=T64),
+          "a.wo": torch.eye(d, dtype=T64), "a.bo": torch.zeros(d, dtype=T64)}
+    th["a.wqkv"][2 * d:] = torch.eye(d, dtype=T64)          # V = x
+    x = torch.randn(S, d, dtype=T64, generator=torch.Generator().manual_seed(1))
+    out = orc.attention(x, th, "a.", 2, causal=True)
+    run = torch.cumsum(x, 0) / torch.arange(1, S + 1, dtype=T64)[:, None]
+    np.testing.assert_allclose(out.numpy(), run.numpy(), rtol=1e-13, atol=1e-13)
+    out = orc.attention(x, th, "a.", 2, causal=False)
+    np.testing.assert_allclose(out.numpy(), x.mean(0, keepdim=True).expand(S, d).numpy(), rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_layer_matches_library_transformer_layer(causal):
+    # the post-LayerNorm layer is the textbook one: torch's own encoder layer with the same weights
+    shape = small_shape(d=16, n_heads=4, d_ff=24)
+    p = synth._draw_params(synth._layer_spec("x.", 16, 24, False), np.random.default_rng(3), 0.4, False)
+    th = orc.as_torch(p, T64, requires_grad=False)
+    lib = torch.nn.TransformerEncoderLayer(16, 4, 24, dropout=0.0, activation="gelu", layer_norm_eps=orc.LN_EPS,
+                                           batch_first=True, norm_first=False, dtype=T64)
+    with torch.no_grad():
+        lib.self_attn.in_proj_weight.copy_(th["x.wqkv"]); lib.self_attn.in_proj_bias.copy_(th["x.bqkv"])
+        lib.self_attn.out_proj.weight.copy_(th["x.wo"]); lib.self_attn.out_proj.bias.copy_(th["x.bo"])
+        lib.linear1.weight.copy_(th["x.w1"]); lib.linear1.bias.copy_(th["x.b1"])
+        lib.linear2.weight.copy_(th["x.w2"]); lib.linear2.bias.copy_(th["x.b2"])
+        lib.norm1.weight.copy_(th["x.ln1_g"]); lib.norm1.bias.copy_(th["x.ln1_b"])
+        lib.norm2.weight.copy_(th["x.ln2_g"]); lib.norm2.bias.copy_(th["x.ln2_b"])
+    lib.train()                                        # keep the plain (non-fused) code path
+    x = torch.randn(9, 16, dtype=T64, generator=torch.Generator().manual_seed(2))
+    mask = torch.triu(torch.full((9, 9), float("-inf"), dtype=T64), diagonal=1) if causal else None
+    with torch.no_grad():
+        want = lib(x[None], src_mask=mask)[0]
+        got = orc.transformer_layer(x, th, "x.", 4, causal)
+    np.testing.assert_allclose(got.numpy(), want.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_losses_at_zero_parameters():
+    # all-zero task parameters: every logit is 0 -> BCE = ln 2; every score equal -> CE = ln(n_cand)
+    kt = small_shape()
+    z = OrderedDict((k, np.zeros(s, np.float32)) for k, s in synth.task_param_spec(kt))
+    E = torch.randn(kt.B, kt.L, kt.d, dtype=T64)
+    lab = synth.labels(0, kt.B, kt.L, 0.6)
+    assert float(orc.task_loss(orc.as_torch(z, T64, False), E, lab, kt)) == pytest.approx(math.log(2), rel=1e-14)
+    nr = small_shape(task="nr", n_cand=5, L=8, d_a=6, task_layers=0)
+    z = OrderedDict((k, np.zeros(s, np.float32)) for k, s in synth.task_param_spec(nr))
+    E = torch.zeros(nr.B, nr.L, nr.d, dtype=T64)
+    assert float(orc.task_loss(orc.as_torch(z, T64, False), E, lab, nr)) == pytest.approx(math.log(5), rel=1e-14)
+
+
+def test_kt_task_does_not_see_the_label_it_predicts():
+    # prediction n may depend on responses 0..n-1 only (Section 3.1)
+    shape = small_shape(task_attn_only=False)
+    ce, tk, toks, ids, lab = make(shape)
+    th = orc.as_torch(tk, T64, False)
+    E = torch.randn(1, shape.L, shape.d, dtype=T64, generator=torch.Generator().manual_seed(0))
+
+    def logits(labels):
+        prev = torch.cat([torch.full((1,), 2, dtype=torch.long), torch.as_tensor(labels[0, :-1], dtype=torch.long)])
+        x = E[0] + th["pos"] + th["resp"][prev]
+        for l in range(shape.task_layers):
+            x = orc.transformer_layer(x, th, f"t{l}.", shape.task_heads, True, shape.task_attn_only)
+        return x @ th["head_w"] + th["head_b"]
+    a = np.array([[1, 0, 1, 1, 0]]); b = a.copy(); b[0, 3] = 0
+    la, lb = logits(a), logits(b)
+    np.testing.assert_allclose(la[:4].numpy(), lb[:4].numpy(), rtol=0, atol=0)      # logits 0..3 unchanged
+    assert abs(float(la[4] - lb[4])) > 1e-9                                         # logit 4 sees response 3
+
+
+# ---- derivatives: central finite differences on a 1-layer encoder ----------
+
+def _loss_only(shape, ce, tk, toks, ids, lab):
+    th_ce, th_cf = orc.as_torch(ce, T64, False), orc.as_torch(tk, T64, False)
+    with torch.no_grad():
+        E = torch.stack([torch.stack([orc.ce_forward(th_ce, toks[int(i)], shape) for i in row]) for row in ids])
+        return float(orc.task_loss(th_cf, E, lab, shape))
+
+
+@pytest.mark.parametrize("variant", ["kt_attn_mean", "kt_full_cls", "nr_cls"])
+def test_e2e_gradients_match_finite_differences(variant):
+    if variant == "kt_attn_mean":
+        shape = small_shape()
+    elif variant == "kt_full_cls":
+        shape = small_shape(pooling="cls", task_attn_only=False)
+    else:
+        shape = small_shape(pooling="cls", task="nr", n_cand=3, L=6, d_a=5, task_layers=0)
+    ce, tk, toks, ids, lab = make(shape, seed=4)
+    ce = OrderedDict((k, v.astype(np.float64)) for k, v in ce.items())
+    tk = OrderedDict((k, v.astype(np.float64)) for k, v in tk.items())
+    out = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    rng = np.random.default_rng(0)
+    eps = 1e-5
+    for params, grads, which in ((ce, out["grad_ce"], "ce"), (tk, out["grad_task"], "task")):
+        for name, arr in params.items():
+            if name == "tok_emb":        # only rows of tokens that occur carry gradient: sample among them
+                used = np.unique(toks[np.unique(ids)])
+                cand = [(int(r), int(c)) for r in used[:3] for c in (0, 5)]
+            else:
+                flat = rng.choice(arr.size, size=min(3, arr.size), replace=False)
+                cand = [np.unravel_index(int(f), arr.shape) for f in flat]
+            for idx in cand:
+                old = arr[idx]
+                arr[idx] = old + eps
+                lp = _loss_only(shape, ce, tk, toks, ids, lab)
+                arr[idx] = old - eps
+                lm = _loss_only(shape, ce, tk, toks, ids, lab)
+                arr[idx] = old
+                fd = (lp - lm) / (2 * eps)
+                an = grads[name][idx]
+                assert abs(fd - an) <= 1e-6 * max(1.0, abs(fd)) + 1e-8, (which, name, idx, fd, an)
+
+
+# ---- the Proposition: Single-step GRAM's gradients equal end-to-end's -------
+
+@pytest.mark.parametrize("variant", ["tiny_cfg", "kt_full_cls", "nr_cls"])
+def test_single_step_equals_e2e(variant):
+    if variant == "tiny_cfg":
+        shape = synth.config("tiny").replace(B=3, L=8, n_items=10)      # heavy reuse: 24 occurrences of <= 10 items
+    elif variant == "kt_full_cls":
+        shape = small_shape(pooling="cls", task_attn_only=False, B=3, L=6)
+    else:
+        shape = small_shape(pooling="cls", task="nr", n_cand=3, L=7, d_a=5, task_layers=0, B=3)
+    ce, tk, toks, ids, lab = make(shape, seed=7)
+    a = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    b = orc.gram_single_step(shape, ce, tk, toks, ids, lab)
+    assert len(b["unique"]) < ids.size                                    # duplicates really occur
+    assert a["loss"] == pytest.approx(b["loss"], rel=1e-13)
+    for key in ("grad_ce", "grad_task"):
+        for name in a[key]:
+            scale = np.abs(a[key][name]).max() + 1e-30
+            assert np.abs(a[key][name] - b[key][name]).max() <= 1e-11 * scale + 1e-15, (key, name)
+    # and a planted mistake (one occurrence dropped from an item's sum) is seen
+    unique, inverse, perm, seg_off = orc.unique_inverse(ids)
+    u = int(np.argmax(np.diff(seg_off)))                                  # the most repeated item
+    drop = int(np.argmax(np.abs(b["dE"][perm[seg_off[u]:seg_off[u + 1]]]).max(1))) + int(seg_off[u])
+    so_bad = seg_off.copy(); so_bad[u + 1:] -= 1
+    G_bad = orc.segment_sum(b["dE"], np.delete(perm, drop), so_bad)
+    assert np.abs(G_bad - b["G"]).max() > 1e-6
+
+
+def test_pseudo_loss_identity_and_lr1_sgd():
+    # Eqs. 1-3: with h~ = h - dL/dh, the gradient of 1/2 (h~ - f(x; theta'))^2 at theta' = theta is dL/dtheta
+    shape = small_shape(B=2, L=6)
+    ce, tk, toks, ids, lab = make(shape, seed=9)
+    s = orc.gram_single_step(shape, ce, tk, toks, ids, lab)
+    h_tilde = s["H"] - s["G"]                          # Eq. 6: SGD with learning rate 1 on the embedding
+    np.testing.assert_allclose(s["H"] - h_tilde, s["G"], rtol=1e-9, atol=1e-12)
+    lt, g = orc.pseudo_loss_grad(shape, ce, toks, s["unique"], h_tilde)
+    assert lt == pytest.approx(0.5 * (s["G"] ** 2).sum(), rel=1e-9)
+    for name in g:
+        scale = np.abs(s["grad_ce"][name]).max() + 1e-30
+        assert np.abs(g[name] - s["grad_ce"][name]).max() <= 1e-9 * scale + 1e-14, name
+    # a learning rate other than 1 in Eq. 6 breaks the identity
+    _, g2 = orc.pseudo_loss_grad(shape, ce, toks, s["unique"], s["H"] - 0.5 * s["G"])
+    assert np.abs(g2["l0.wqkv"] - s["grad_ce"]["l0.wqkv"]).max() > 1e-3 * np.abs(s["grad_ce"]["l0.wqkv"]).max()
+
+
+# ---- Multi-step -------------------------------------------------------------
+
+def test_multistep_k1_reduces_to_single_step():
+    # Section 4.3: the algorithm is Single-step GRAM for N = 1 (given a cache that holds CE's current outputs)
+    shape = small_shape(B=2, L=6)
+    ce, tk, toks, ids, lab = make(shape, seed=11)
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    m = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.1)
+    s = orc.gram_single_step(shape, ce, tk, toks, ids, lab)
+    assert m["losses"][0] == pytest.approx(s["loss"], rel=1e-13)
+    assert np.array_equal(m["items"], s["unique"])
+    for name in s["grad_ce"]:
+        scale = np.abs(s["grad_ce"][name]).max() + 1e-30
+        assert np.abs(m["grad_ce"][name] - s["grad_ce"][name]).max() <= 1e-11 * scale, name
+    for name in s["grad_task"]:
+        np.testing.assert_allclose(m["task_params"][name], tk[name] - 0.1 * s["grad_task"][name], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(m["cache"], cache, rtol=1e-12, atol=1e-14)     # encoder unchanged -> same values
+
+
+def test_multistep_table_and_touched_over_k_steps():
+    shape = small_shape(B=2, L=6, K=3)
+    ce, tk, toks, _, _ = make(shape, seed=13)
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    batches = [synth.batch(shape, 13, step=k) for k in range(3)]
+    m = orc.multistep_window(shape, ce, tk, toks, batches, cache, lr_task=0.0)
+    # with lr_task = 0 the task module is frozen, so each step's dE is the single-step dE on the cached encodings
+    expect = np.zeros_like(m["table"]); union = set()
+    for ids, lab in batches:
+        s = orc.gram_single_step(shape, ce, tk, toks, ids, lab)
+        expect[s["unique"]] += s["G"]
+        union |= set(int(i) for i in s["unique"])
+    np.testing.assert_allclose(m["table"], expect, rtol=1e-10, atol=1e-13)
+    assert set(int(i) for i in m["items"]) == union
+    # the encoder gradient is the VJP with the table rows: linear in the table
+    th = orc.as_torch(ce, T64)
+    H = torch.stack([orc.ce_forward(th, toks[int(i)], shape) for i in m["items"]])
+    H.backward(torch.tensor(expect[m["items"]]))
+    np.testing.assert_allclose(m["grad_ce"]["l0.w1"], th["l0.w1"].grad.numpy(), rtol=1e-9, atol=1e-13)
+
+
+def test_multistep_later_steps_see_updated_task_parameters():
+    shape = small_shape(B=2, L=6, K=2)
+    ce, tk, toks, _, _ = make(shape, seed=15)
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    batches = [synth.batch(shape, 15, step=k) for k in range(2)]
+    a = orc.multistep_window(shape, ce, tk, toks, batches, cache, lr_task=0.5)
+    b = orc.multistep_window(shape, ce, tk, toks, batches, cache, lr_task=0.0)
+    assert a["losses"][0] == pytest.approx(b["losses"][0], rel=1e-13)
+    assert abs(a["losses"][1] - b["losses"][1]) > 1e-6
