@@ -1,0 +1,218 @@
+/* gram.h - C ABI of the GRAM deduplicated encode/accumulate training step (CUDA, sm_100a).
+ *
+ * GRAM (gradient accumulation for content-based collaborative filtering) trains
+ * a content encoder CE and a task module CF (Section 3) without running CE once
+ * per interaction: per mini-batch it encodes every *unique* item once, sums the
+ * task module's gradients over the occurrences of each item, and runs CE's
+ * backward once per unique item (Section 4.1, Fig. 1, Algorithm 1).
+ *
+ * Conventions for every call
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
+ *     owns every buffer it passes; the context owns parameters, gradients,
+ *     workspaces, the Multi-step table and cache.  Nothing passed in is kept
+ *     after the call returns unless stated.
+ *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = the default
+ *     stream).  Work is stream-ordered; calls return without synchronising
+ *     unless stated.  A context is not thread-safe.
+ *   - Item IDs are int32 in [0, n_items).  Matrices are row-major.
+ *   - Every call returns a gram_status and never throws, aborts or traps.  An
+ *     error found on the device (an ID out of range) is recorded in the context
+ *     and returned by the next synchronising call (gram_sync, gram_step*).
+ *   - Outputs are fully overwritten, except the Multi-step table, which
+ *     accumulates by definition until gram_window_reset.
+ */
+#ifndef GRAM_H_
+#define GRAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gram_ctx gram_ctx;
+typedef void* gram_stream;              /* a cudaStream_t */
+
+typedef enum gram_status {
+  GRAM_OK = 0,
+  GRAM_ERR_ARG = 1,                     /* null pointer, negative or inconsistent size */
+  GRAM_ERR_ID_RANGE = 2,                /* an item or token ID outside its range */
+  GRAM_ERR_WORKSPACE = 3,               /* sizes exceed what the context was created for */
+  GRAM_ERR_UNSUPPORTED = 4,             /* a shape the kernels do not cover */
+  GRAM_ERR_CUDA = 5,                    /* a CUDA runtime call failed; see gram_last_error */
+  GRAM_ERR_TIMEOUT = 6                  /* a bounded device-side wait ran out */
+} gram_status;
+
+enum { GRAM_F32 = 0, GRAM_BF16 = 1 };                 /* element types */
+enum { GRAM_POOL_MEAN = 0, GRAM_POOL_CLS = 1 };       /* item pooling */
+enum { GRAM_TASK_NONE = 0, GRAM_TASK_KT = 1, GRAM_TASK_NR = 2 };
+enum { GRAM_MODULE_CE = 0, GRAM_MODULE_TASK = 1 };
+
+/* Shapes of the two modules and of the batches a context serves.
+ * CE (Section 3.2; Appendix D: attention layers of width 768): token + position
+ * embedding, LayerNorm, n_layers post-LayerNorm transformer layers (multi-head
+ * attention, erf-GELU feed-forward), pooled to one d-vector per item.
+ * CF (Section 3.1): task = KT: x_n = E[b,n] + pos[n] + resp[r_{n-1}], task_layers
+ * causal layers (attention only when task_attn_only != 0), a linear head and
+ * binary cross-entropy averaged over B*L predictions; task = NR: additive
+ * attention (width d_a) over the first L - n_cand encodings, dot-product scores
+ * with the n_cand candidates, softmax cross-entropy on candidate 0 averaged
+ * over B.  A context with n_layers == 0 and task == GRAM_TASK_NONE serves only
+ * the index and accumulation calls.
+ * dtype = GRAM_BF16: matrix products take bf16 operands with fp32 accumulation,
+ * activations are stored as bf16, parameters and their gradients stay fp32. */
+typedef struct gram_config {
+  int32_t dtype;
+  int32_t n_items, l_t, vocab;
+  int32_t d, n_heads, d_ff, n_layers, pooling;
+  int32_t task, task_layers, task_heads, task_d_ff, task_attn_only, d_a, n_cand;
+  int32_t B_max, L;            /* largest batch: B_max histories of L positions */
+  int64_t P_max;               /* largest number of positions for the index/accumulate calls (0 = B_max*L) */
+  int32_t d_max;               /* widest row for gather/accumulate (0 = d) */
+  int32_t K;                   /* Multi-step window length (Section 4.2); 1 = Single-step */
+  int32_t ce_micro_batch;      /* items per encoder pass, bounds activation memory (Section 6.3); 0 = all at once */
+  float lr_task;               /* SGD step applied to the task parameters after every gram_step (0 = none) */
+  float lr_ce;                 /* SGD step applied to the encoder parameters after an encoder pass (0 = none) */
+} gram_config;
+
+typedef struct gram_step_report {
+  float loss;                  /* task loss of this step (Eq. 8) */
+  int32_t n_positions;         /* P = B*L interactions in the batch */
+  int32_t n_unique;            /* |B_I|, unique items in the batch */
+  float boost_ratio;           /* R = P / n_unique (Section 4.4) */
+  int32_t n_touched;           /* Multi-step: items touched so far in the window (Single-step: n_unique) */
+  int32_t encoder_pass;        /* 1 if this step ran the encoder backward (always for K = 1, every K-th step else) */
+  int32_t n_encoded;           /* items the encoder ran on in this step */
+  float ms_dedup, ms_encode, ms_gather, ms_task, ms_accumulate, ms_backward, ms_total;  /* device time per stage */
+} gram_step_report;
+
+/* --- life cycle ---------------------------------------------------------- */
+
+/* Allocates everything a context will ever need (parameters, gradients,
+ * activations for one micro-batch, workspaces, Multi-step table / bitmap /
+ * cache when K > 1); no later call allocates.  *out is NULL on failure. */
+gram_status gram_create(const gram_config* cfg, gram_ctx** out);
+gram_status gram_destroy(gram_ctx* ctx);
+/* Waits for the stream and returns any error recorded on the device. */
+gram_status gram_sync(gram_ctx* ctx, gram_stream stream);
+/* Text of the last error of this context (valid until the next call on it). */
+const char* gram_last_error(const gram_ctx* ctx);
+
+/* Number of fp32 parameters of a module.  The flat layout is, for CE:
+ * tok_emb[vocab,d] pos_emb[l_t,d] emb_ln_g[d] emb_ln_b[d], then per layer
+ * wqkv[3d,d] bqkv[3d] wo[d,d] bo[d] ln1_g ln1_b w1[d_ff,d] b1[d_ff] w2[d,d_ff]
+ * b2[d] ln2_g ln2_b; for KT: pos[L,d] resp[3,d], the layers (attention-only
+ * layers hold wqkv bqkv wo bo), head_w[d] head_b[1]; for NR: wa[d_a,d] ba[d_a]
+ * qa[d_a].  Rows 0..d-1 of wqkv produce Q, the next d K, the last d V; head h
+ * owns columns h*d/n_heads .. of each. */
+gram_status gram_param_count(const gram_ctx* ctx, int module, size_t* n);
+gram_status gram_set_params(gram_ctx* ctx, int module, const float* h_params, size_t n);
+gram_status gram_get_params(gram_ctx* ctx, int module, float* h_params, size_t n);
+/* Gradients of the last gram_step / gram_encoder_backward / gram_task, same layout (synchronises). */
+gram_status gram_get_grads(gram_ctx* ctx, int module, float* h_grads, size_t n);
+gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream);
+/* Token IDs c_i of every item (Table 1), int32 [n_items, l_t], copied to the device. */
+gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens);
+
+/* --- the five stages (Algorithm 1; Fig. 1) -------------------------------- */
+
+/* Stage 1, the unique-item set B_I of a mini-batch (Table 1) and the map from
+ * occurrences to items (Fig. 1).  d_ids int32 [P].  Outputs:
+ *   d_unique  [>= min(P, n_items)]  distinct IDs, ascending (first U valid)
+ *   d_inverse [P]   d_unique[d_inverse[p]] == d_ids[p]
+ *   d_perm    [P]   positions grouped by item, ascending inside a group (stable sort order)
+ *   d_seg_off [>= min(P, n_items) + 1]  group u is d_perm[d_seg_off[u] .. d_seg_off[u+1])
+ *   d_n_unique [1]  U
+ * Radix sort on the low ceil(log2 n_items) key bits, then a run-length pass.
+ * An ID outside [0, n_items) records GRAM_ERR_ID_RANGE (outputs then unspecified). */
+gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n_items,
+                       int32_t* d_unique, int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off,
+                       int32_t* d_n_unique, gram_stream stream);
+
+/* Stage 2, Eq. 4: d_H[u, :] = CE(tokens of item d_items[u]) for u < U, once per
+ * unique item.  d_item_tokens int32 [n_items, l_t] (NULL = the context's copy).
+ * d_H is [U, d] of the context's dtype.  save_activations != 0 keeps what
+ * gram_encoder_backward needs (U must then fit one micro-batch). */
+gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
+                               void* d_H, int save_activations, gram_stream stream);
+
+/* Stage 3: d_E[p, :] = d_src[d_index[p], :] for p < P.  Single-step: src = H,
+ * index = inverse.  Multi-step: src = the encoding cache, index = ids.
+ * Rows are d elements of `dtype`; n_src_rows bounds the index (ID_RANGE else). */
+gram_status gram_gather(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                        int32_t d, int dtype, void* d_E, gram_stream stream);
+
+/* Stage 4, Single-step (Eq. 6: with SGD of rate 1 the change of an item's
+ * encoding is the sum of dL/dE over its occurrences):
+ *   d_G[u, :] = sum over j in [d_seg_off[u], d_seg_off[u+1]) of d_dE[d_perm[j], :]
+ * fp32 [P, d] -> fp32 [U, d].  The order of additions is fixed by (P, U,
+ * d_seg_off) alone, so repeated calls give bit-identical results. */
+gram_status gram_accumulate(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm, const int32_t* d_seg_off,
+                            int64_t P, int32_t U, int32_t d, float* d_G, gram_stream stream);
+
+/* Stage 4, Multi-step (Section 4.2): the same sums are added into the per-item
+ * table, d_table[d_unique[u], :] += sum, fp32 [n_items, d], and bit d_unique[u]
+ * of d_touched_bits (uint32 [ceil(n_items/32)]) is set.  NULL table/bits select
+ * the context's own (K > 1). */
+gram_status gram_accumulate_multistep(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm,
+                                      const int32_t* d_seg_off, const int32_t* d_unique, int64_t P, int32_t U,
+                                      int32_t d, int32_t n_items, float* d_table, uint32_t* d_touched_bits,
+                                      gram_stream stream);
+/* Ascending list of the set bits: d_list [>= n_items], d_count [1]. */
+gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int32_t n_items, int32_t* d_list,
+                              int32_t* d_count, gram_stream stream);
+
+/* Task module forward and backward (Eq. 5 and the gradient of Eq. 8 with
+ * respect to the encodings): d_E [B, L, d] of the context's dtype, d_labels
+ * int32 [B, L] -> d_dE fp32 [B*L, d], d_loss fp32 [1]; task parameter
+ * gradients are overwritten in the context. */
+gram_status gram_task(gram_ctx* ctx, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE,
+                      float* d_loss, gram_stream stream);
+
+/* Stage 5, Eq. 7: encoder parameter gradients += sum over u of J_u^T d_G[u, :],
+ * one VJP per unique item, using the activations saved by the last
+ * gram_encode_unique(save_activations = 1) over the same items. */
+gram_status gram_encoder_backward(gram_ctx* ctx, const float* d_G, const int32_t* d_items, int32_t U,
+                                  gram_stream stream);
+
+/* --- the whole step -------------------------------------------------------- */
+
+/* One training step (Algorithm 1) on a batch of B histories: d_ids, d_labels
+ * int32 [B, L].  K = 1: dedup, encode unique, gather, task forward/backward,
+ * accumulate, encoder backward; gradients of both modules are left in the
+ * context.  K > 1: encodings come from the cache (gram_cache_fill first), the
+ * sums go to the table, and every K-th call runs the encoder forward and
+ * backward over the touched items in micro-batches, refreshes their cache
+ * rows and clears the window.  Task parameters take an SGD step of lr_task,
+ * encoder parameters one of lr_ce after an encoder pass.  Synchronises; fills
+ * *report (may be NULL). */
+gram_status gram_step(gram_ctx* ctx, const int32_t* d_ids, const int32_t* d_labels, int32_t B,
+                      gram_step_report* report, gram_stream stream);
+/* The same with HOST buffers: copies ids and labels to the device, runs the
+ * step, copies the loss back. */
+gram_status gram_step_host(gram_ctx* ctx, const int32_t* h_ids, const int32_t* h_labels, int32_t B,
+                           gram_step_report* report, gram_stream stream);
+
+/* Multi-step: encode every item with the current parameters into the cache. */
+gram_status gram_cache_fill(gram_ctx* ctx, gram_stream stream);
+/* Multi-step: zero the table and the touched bitmap, restart the window. */
+gram_status gram_window_reset(gram_ctx* ctx, gram_stream stream);
+/* Multi-step state, copied to host: table fp32 [n_items, d], touched uint32
+ * [ceil(n_items/32)], cache fp32 [n_items, d] (converted).  NULL skips one. */
+gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache);
+
+/* --- a building block, exported so that it can be tested on its own --------
+ * C[M, N] = A x B with bf16 operands and fp32 accumulation on the tensor cores.
+ * a_kmajor != 0: A is [M, K] row-major, else [K, M] row-major; b_kmajor != 0:
+ * B is [N, K] row-major, else [K, N] row-major.  C is fp32 [M, N] when
+ * c_f32 != 0, else bf16.  d_bias (fp32 [N]) may be NULL.  accumulate != 0
+ * adds to C instead of overwriting (fp32 C only).  M, N, K multiples of 8. */
+gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
+                           int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
+                           gram_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRAM_H_ */

@@ -1,0 +1,224 @@
+// The C ABI of libgram: context life cycle, argument checks, and the calls of include/gram.h.
+#include <stdarg.h>
+
+#include <new>
+
+#include "gram_internal.h"
+#include "model.h"
+
+struct gram_ctx {
+  gram_config cfg;
+  char err[512];
+  int32_t* d_status = nullptr;      // device status word (first device-side error)
+  IndexWorkspace iws;
+  Model* model = nullptr;           // encoder + task module state (null for an index-only context)
+};
+
+void gram_set_error(gram_ctx* ctx, const char* fmt, ...) {
+  if (!ctx) return;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+  va_end(ap);
+}
+
+int32_t* gram_status_word(gram_ctx* ctx) { return ctx->d_status; }
+IndexWorkspace* gram_index_ws(gram_ctx* ctx) { return &ctx->iws; }
+const gram_config* gram_cfg(const gram_ctx* ctx) { return &ctx->cfg; }
+
+static cudaStream_t S(gram_stream s) { return reinterpret_cast<cudaStream_t>(s); }
+
+static gram_status check_device_status(gram_ctx* ctx) {
+  int32_t h = 0;
+  GRAM_CUDA(ctx, cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
+  if (h != 0) {
+    GRAM_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    gram_set_error(ctx, h == GRAM_ERR_ID_RANGE ? "an ID outside its range was met on the device"
+                                               : (h == GRAM_ERR_TIMEOUT ? "a bounded device-side wait ran out" : "device-side error"));
+    return (gram_status)h;
+  }
+  return GRAM_OK;
+}
+
+extern "C" {
+
+gram_status gram_create(const gram_config* cfg, gram_ctx** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !out) return GRAM_ERR_ARG;
+  if (cfg->n_items <= 0 || cfg->B_max < 0 || cfg->L < 0 || cfg->P_max < 0 || cfg->K < 0 || cfg->n_layers < 0) return GRAM_ERR_ARG;
+  gram_ctx* ctx = new (std::nothrow) gram_ctx();
+  if (!ctx) return GRAM_ERR_CUDA;
+  ctx->cfg = *cfg;
+  ctx->err[0] = 0;
+  if (ctx->cfg.K == 0) ctx->cfg.K = 1;
+  int64_t P_max = cfg->P_max > 0 ? cfg->P_max : (int64_t)cfg->B_max * cfg->L;
+  if (ctx->cfg.n_layers > 0) {       // the token-embedding gradient reuses the index kernels over token positions
+    int64_t mb = cfg->ce_micro_batch > 0 ? cfg->ce_micro_batch : cfg->n_items;
+    if (mb > cfg->n_items) mb = cfg->n_items;
+    if (mb > P_max && P_max > 0 && cfg->K <= 1) mb = P_max;
+    int64_t tok = mb * cfg->l_t;
+    if (tok > P_max) P_max = tok;
+  }
+  ctx->cfg.P_max = P_max;
+  int32_t d_max = cfg->d_max > 0 ? cfg->d_max : cfg->d;
+  if (d_max < cfg->d) d_max = cfg->d;
+  ctx->cfg.d_max = d_max;
+  gram_status s = GRAM_OK;
+  do {
+    if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess) {
+      s = GRAM_ERR_CUDA;
+      break;
+    }
+    int32_t n_keys = cfg->n_items > cfg->vocab ? cfg->n_items : cfg->vocab;
+    s = index_ws_alloc(ctx, &ctx->iws, P_max, n_keys, d_max);
+    if (s != GRAM_OK) break;
+    if (ctx->cfg.n_layers > 0 || ctx->cfg.task != GRAM_TASK_NONE) {
+      s = model_create(ctx, &ctx->cfg, &ctx->model);
+      if (s != GRAM_OK) break;
+    }
+  } while (0);
+  if (s != GRAM_OK) {
+    fprintf(stderr, "gram_create failed: %s\n", ctx->err);
+    gram_destroy(ctx);
+    return s;
+  }
+  *out = ctx;
+  return GRAM_OK;
+}
+
+gram_status gram_destroy(gram_ctx* ctx) {
+  if (!ctx) return GRAM_OK;
+  cudaDeviceSynchronize();
+  if (ctx->model) model_destroy(ctx->model);
+  index_ws_free(&ctx->iws);
+  cudaFree(ctx->d_status);
+  delete ctx;
+  return GRAM_OK;
+}
+
+gram_status gram_sync(gram_ctx* ctx, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  GRAM_CUDA(ctx, cudaStreamSynchronize(S(stream)));
+  return check_device_status(ctx);
+}
+
+const char* gram_last_error(const gram_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n_items, int32_t* d_unique,
+                       int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off, int32_t* d_n_unique,
+                       gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  return dedup_launch(ctx, &ctx->iws, d_ids, P, n_items, d_unique, d_inverse, d_perm, d_seg_off, d_n_unique, S(stream));
+}
+
+gram_status gram_gather(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                        int32_t d, int dtype, void* d_E, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  if (dtype != GRAM_F32 && dtype != GRAM_BF16) return gram_set_error(ctx, "gram_gather: unknown dtype"), GRAM_ERR_ARG;
+  return gather_launch(ctx, d_src, n_src_rows, d_index, P, d, dtype == GRAM_F32 ? 4 : 2, d_E, S(stream));
+}
+
+gram_status gram_accumulate(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm, const int32_t* d_seg_off,
+                            int64_t P, int32_t U, int32_t d, float* d_G, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  return accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, d, nullptr, 0, d_G, S(stream));
+}
+
+gram_status gram_accumulate_multistep(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm,
+                                      const int32_t* d_seg_off, const int32_t* d_unique, int64_t P, int32_t U,
+                                      int32_t d, int32_t n_items, float* d_table, uint32_t* d_touched_bits,
+                                      gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  if (!d_unique && U > 0) return gram_set_error(ctx, "gram_accumulate_multistep: null d_unique"), GRAM_ERR_ARG;
+  if (!d_table || !d_touched_bits) {
+    if (!ctx->model || !model_table(ctx->model) || n_items != ctx->cfg.n_items || d != ctx->cfg.d)
+      return gram_set_error(ctx, "gram_accumulate_multistep: no table given and the context holds none of this shape"), GRAM_ERR_ARG;
+    if (!d_table) d_table = model_table(ctx->model);
+    if (!d_touched_bits) d_touched_bits = model_touched(ctx->model);
+  }
+  GRAM_TRY(accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, d, d_unique, 1, d_table, S(stream)));
+  return touched_mark_launch(ctx, d_unique, U, n_items, d_touched_bits, S(stream));
+}
+
+gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int32_t n_items, int32_t* d_list,
+                              int32_t* d_count, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  return touched_list_launch(ctx, d_touched_bits, n_items, d_list, d_count, S(stream));
+}
+
+// ---- calls that need the modules -----------------------------------------------------------
+#define NEED_MODEL(name)                                                                                  \
+  if (!ctx) return GRAM_ERR_ARG;                                                                          \
+  if (!ctx->model) return gram_set_error(ctx, name ": the context was created without modules"), GRAM_ERR_ARG;
+
+gram_status gram_param_count(const gram_ctx* ctx, int module, size_t* n) {
+  if (!ctx || !n || !ctx->model) return GRAM_ERR_ARG;
+  return model_param_count(ctx->model, module, n);
+}
+gram_status gram_set_params(gram_ctx* ctx, int module, const float* h, size_t n) {
+  NEED_MODEL("gram_set_params");
+  return model_set_params(ctx->model, module, h, n);
+}
+gram_status gram_get_params(gram_ctx* ctx, int module, float* h, size_t n) {
+  NEED_MODEL("gram_get_params");
+  return model_get_params(ctx->model, module, h, n, 0);
+}
+gram_status gram_get_grads(gram_ctx* ctx, int module, float* h, size_t n) {
+  NEED_MODEL("gram_get_grads");
+  return model_get_params(ctx->model, module, h, n, 1);
+}
+gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream) {
+  NEED_MODEL("gram_zero_grads");
+  return model_zero_grads(ctx->model, module, S(stream));
+}
+gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens) {
+  NEED_MODEL("gram_set_item_tokens");
+  return model_set_item_tokens(ctx->model, h_tokens);
+}
+gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
+                               void* d_H, int save_activations, gram_stream stream) {
+  NEED_MODEL("gram_encode_unique");
+  return model_encode(ctx->model, d_item_tokens, d_items, U, d_H, save_activations, S(stream));
+}
+gram_status gram_task(gram_ctx* ctx, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
+                      gram_stream stream) {
+  NEED_MODEL("gram_task");
+  return model_task(ctx->model, d_E, d_labels, B, d_dE, d_loss, S(stream));
+}
+gram_status gram_encoder_backward(gram_ctx* ctx, const float* d_G, const int32_t* d_items, int32_t U,
+                                  gram_stream stream) {
+  NEED_MODEL("gram_encoder_backward");
+  return model_encoder_backward(ctx->model, d_G, d_items, U, S(stream));
+}
+gram_status gram_step(gram_ctx* ctx, const int32_t* d_ids, const int32_t* d_labels, int32_t B,
+                      gram_step_report* report, gram_stream stream) {
+  NEED_MODEL("gram_step");
+  GRAM_TRY(model_step(ctx->model, d_ids, d_labels, B, 0, report, S(stream)));
+  return check_device_status(ctx);
+}
+gram_status gram_step_host(gram_ctx* ctx, const int32_t* h_ids, const int32_t* h_labels, int32_t B,
+                           gram_step_report* report, gram_stream stream) {
+  NEED_MODEL("gram_step_host");
+  GRAM_TRY(model_step(ctx->model, h_ids, h_labels, B, 1, report, S(stream)));
+  return check_device_status(ctx);
+}
+gram_status gram_cache_fill(gram_ctx* ctx, gram_stream stream) {
+  NEED_MODEL("gram_cache_fill");
+  return model_cache_fill(ctx->model, S(stream));
+}
+gram_status gram_window_reset(gram_ctx* ctx, gram_stream stream) {
+  NEED_MODEL("gram_window_reset");
+  return model_window_reset(ctx->model, S(stream));
+}
+gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache) {
+  NEED_MODEL("gram_get_window");
+  return model_get_window(ctx->model, h_table, h_touched, h_cache);
+}
+gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
+                           int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
+                           gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  return gemm_bf16_public(ctx, d_A, a_kmajor, d_B, b_kmajor, d_C, c_f32, d_bias, accumulate, M, N, K, S(stream));
+}
+
+}  // extern "C"

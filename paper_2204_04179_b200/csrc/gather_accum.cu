@@ -1,0 +1,364 @@
+// Stage 3 (gather encodings into sequence positions) and stage 4 (sum the per-position
+// gradients of each item, Eq. 6; Multi-step: add them into the per-item table, Section 4.2).
+// Both are HBM-bound: 128-bit accesses, a warp per row, several rows in flight per warp.
+#include "gram_internal.h"
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// gather: E[p, :] = src[index[p], :]
+// Algorithmic bytes: P*row written + (distinct rows)*row read + 4P index.
+// ---------------------------------------------------------------------------
+template <int ROWS>   // rows a warp keeps in flight
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ src, int64_t n_src_rows,
+                                                          const int32_t* __restrict__ index, int64_t P, int nvec,
+                                                          uint4* __restrict__ dst, int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t p0 = warp * ROWS; p0 < P; p0 += nwarps * ROWS) {
+    int64_t row[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      int64_t p = p0 + r;
+      int32_t i = (p < P) ? index[p] : 0;
+      if (i < 0 || i >= n_src_rows) {
+        gram_device_fail(status, GRAM_ERR_ID_RANGE);
+        i = 0;
+      }
+      row[r] = i;
+    }
+    for (int c = lane; c < nvec; c += 32) {
+      uint4 v[ROWS];
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) v[r] = __ldg(src + row[r] * nvec + c);
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r)
+        if (p0 + r < P) __stcs(dst + (p0 + r) * nvec + c, v[r]);
+    }
+  }
+}
+
+// rows whose byte length is not a multiple of 16: element-wise copy of 2- or 4-byte elements
+template <typename T>
+__global__ void gather_scalar_kernel(const T* __restrict__ src, int64_t n_src_rows, const int32_t* __restrict__ index,
+                                     int64_t P, int d, T* __restrict__ dst, int32_t* status) {
+  const int64_t n = P * d;
+  for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += (int64_t)gridDim.x * blockDim.x) {
+    int64_t p = k / d;
+    int c = (int)(k - p * d);
+    int32_t i = index[p];
+    if (i < 0 || i >= n_src_rows) {
+      gram_device_fail(status, GRAM_ERR_ID_RANGE);
+      i = 0;
+    }
+    dst[k] = src[(int64_t)i * d + c];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// segmented sum.  The sorted order j in [0, P) is cut into nchunks equal chunks of R rows; the
+// columns into slabs of VPL*128 floats.  One warp owns one (chunk, slab): it walks its rows in
+// order, adding into registers, and closes a sum whenever the item changes.
+//   - an item whose rows all lie inside the chunk is written to its output row directly;
+//   - the item that entered the chunk from the left leaves its part in partial[chunk][0];
+//   - the item that leaves the chunk to the right leaves its part in partial[chunk][1].
+// A second launch adds, for every item that spans chunks, partial[first][1] and then
+// partial[c][0] for the following chunks in ascending c.  The order of additions depends only
+// on (P, U, seg_off), never on scheduling: repeated runs are bit-identical.
+// Algorithmic bytes: 4*P*d read + 4*U*d written + 4P (perm) + 4(U+1) (seg_off).
+// ---------------------------------------------------------------------------
+template <typename InT> struct Row4;
+template <> struct Row4<float> {
+  typedef float4 vec;
+  static __device__ __forceinline__ float4 load(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+};
+template <> struct Row4<bf16> {
+  typedef uint2 vec;
+  static __device__ __forceinline__ float4 load(const bf16* p) {
+    uint2 u = __ldcs(reinterpret_cast<const uint2*>(p));
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x), b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+    float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+    return make_float4(fa.x, fa.y, fb.x, fb.y);
+  }
+};
+
+__device__ __forceinline__ int32_t find_segment(const int32_t* __restrict__ seg_off, int32_t U, int64_t j) {
+  // largest u in [0, U) with seg_off[u] <= j
+  int32_t lo = 0, hi = U - 1;
+  while (lo < hi) {
+    int32_t mid = (lo + hi + 1) >> 1;
+    if (seg_off[mid] <= j) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+template <int VPL>
+__device__ __forceinline__ void store_row(float* __restrict__ out, int64_t row, int d, int col0, int lane,
+                                          const float4 (&acc)[VPL], bool add) {
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) {
+    int c = col0 + (v * 32 + lane) * 4;
+    if (c < d) {
+      float4* q = reinterpret_cast<float4*>(out + row * d + c);
+      float4 a = acc[v];
+      if (add) {
+        float4 o = *q;
+        a.x += o.x; a.y += o.y; a.z += o.z; a.w += o.w;
+      }
+      *q = a;
+    }
+  }
+}
+
+template <typename InT, int VPL, int UNROLL>
+__global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restrict__ in, const int32_t* __restrict__ perm,
+                                                            const int32_t* __restrict__ seg_off, int64_t P, int32_t U,
+                                                            int d, int64_t R, int nchunks, int nslabs,
+                                                            const int32_t* __restrict__ rows, int add,
+                                                            float* __restrict__ out, float* __restrict__ partial,
+                                                            int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= (int64_t)nchunks * nslabs) return;
+  const int chunk = (int)(w / nslabs), slab = (int)(w - (int64_t)chunk * nslabs);
+  const int col0 = slab * (VPL * 128);
+  const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
+  if (c0 >= c1) return;
+
+  int32_t u = find_segment(seg_off, U, c0);
+  int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
+  float4 acc[VPL];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  for (int64_t j0 = c0; j0 < c1; j0 += 32) {
+    const int nrow = (int)min((int64_t)32, c1 - j0);
+    int32_t my = (lane < nrow) ? perm[j0 + lane] : 0;
+    if ((uint32_t)my >= (uint32_t)P) {       // a position outside the batch: record it, read row 0 instead
+      gram_device_fail(status, GRAM_ERR_ID_RANGE);
+      my = 0;
+    }
+    for (int b = 0; b < nrow; b += UNROLL) {
+      float4 x[UNROLL][VPL];
+#pragma unroll
+      for (int r = 0; r < UNROLL; ++r) {
+        const int32_t p = __shfl_sync(0xffffffffu, my, (b + r) & 31);
+        const bool live = (b + r) < nrow;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+          int c = col0 + (v * 32 + lane) * 4;
+          x[r][v] = (live && c < d) ? Row4<InT>::load(in + (int64_t)p * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < UNROLL; ++r) {
+        const int64_t j = j0 + b + r;
+        if (j < c1) {
+          while (j == seg_end && u + 1 < U) {   // item u is complete (its end lies inside this chunk)
+            if (seg_begin >= c0) store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
+            else store_row<VPL>(partial, (int64_t)chunk * 2 + 0, d, col0, lane, acc, false);
+            ++u;
+            seg_begin = seg_end;
+            seg_end = seg_off[u + 1];
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int v = 0; v < VPL; ++v) {
+            acc[v].x += x[r][v].x; acc[v].y += x[r][v].y; acc[v].z += x[r][v].z; acc[v].w += x[r][v].w;
+          }
+        }
+      }
+    }
+  }
+  // the item still open at the end of the chunk
+  if (seg_end <= c1) {             // it ends exactly at the chunk end
+    if (seg_begin >= c0) store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
+    else store_row<VPL>(partial, (int64_t)chunk * 2 + 0, d, col0, lane, acc, false);
+  } else {                         // it continues to the right
+    store_row<VPL>(partial, (int64_t)chunk * 2 + (seg_begin >= c0 ? 1 : 0), d, col0, lane, acc, false);
+  }
+}
+
+// one warp per (chunk, slab): if an item starts in this chunk and runs past its end, add its parts
+template <int VPL>
+__global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __restrict__ seg_off, int64_t P, int32_t U,
+                                                           int d, int64_t R, int nchunks, int nslabs,
+                                                           const int32_t* __restrict__ rows, int add,
+                                                           float* __restrict__ out, const float* __restrict__ partial) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= (int64_t)nchunks * nslabs) return;
+  const int chunk = (int)(w / nslabs), slab = (int)(w - (int64_t)chunk * nslabs);
+  const int col0 = slab * (VPL * 128);
+  const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
+  if (c0 >= c1 || c1 >= P) return;
+  const int32_t u = find_segment(seg_off, U, c1 - 1);
+  const int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
+  if (seg_begin < c0 || seg_end <= c1) return;      // not the first chunk of a spanning item
+  const int last = (int)((seg_end - 1) / R);
+  float4 acc[VPL];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) {
+    int c = col0 + (v * 32 + lane) * 4;
+    acc[v] = (c < d) ? *reinterpret_cast<const float4*>(partial + ((int64_t)chunk * 2 + 1) * d + c)
+                     : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int c = chunk + 1; c <= last; ++c) {
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      int cc = col0 + (v * 32 + lane) * 4;
+      if (cc < d) {
+        float4 x = *reinterpret_cast<const float4*>(partial + ((int64_t)c * 2 + 0) * d + cc);
+        acc[v].x += x.x; acc[v].y += x.y; acc[v].z += x.z; acc[v].w += x.w;
+      }
+    }
+  }
+  store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
+}
+
+__global__ void touched_mark_kernel(const int32_t* __restrict__ unique, int32_t U, int32_t n_items,
+                                    uint32_t* __restrict__ bits, int32_t* status) {
+  int32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= U) return;
+  int32_t i = unique[u];
+  if (i < 0 || i >= n_items) {
+    gram_device_fail(status, GRAM_ERR_ID_RANGE);
+    return;
+  }
+  atomicOr(&bits[i >> 5], 1u << (i & 31));
+}
+
+// ascending list of set bits, one block
+__global__ void __launch_bounds__(1024) touched_list_kernel(const uint32_t* __restrict__ bits, int32_t n_items,
+                                                            int32_t* __restrict__ list, int32_t* __restrict__ count) {
+  __shared__ int32_t sw[33];
+  const int nwords = (n_items + 31) >> 5;
+  const int per = (nwords + 1023) / 1024;
+  const int w0 = threadIdx.x * per, w1 = min(w0 + per, nwords);
+  int32_t c = 0;
+  for (int w = w0; w < w1; ++w) {
+    uint32_t b = bits[w];
+    if (w == nwords - 1 && (n_items & 31)) b &= (1u << (n_items & 31)) - 1u;
+    c += __popc(b);
+  }
+  // exclusive scan over the 1024 threads
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int32_t incl = c;
+  for (int o = 1; o < 32; o <<= 1) {
+    int32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) sw[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int32_t x = sw[lane], xi = x;
+    for (int o = 1; o < 32; o <<= 1) {
+      int32_t t = __shfl_up_sync(0xffffffffu, xi, o);
+      if (lane >= o) xi += t;
+    }
+    sw[lane] = xi - x;
+    if (lane == 31) sw[32] = xi;
+  }
+  __syncthreads();
+  int32_t pos = sw[warp] + incl - c;
+  for (int w = w0; w < w1; ++w) {
+    uint32_t b = bits[w];
+    if (w == nwords - 1 && (n_items & 31)) b &= (1u << (n_items & 31)) - 1u;
+    while (b) {
+      int bit = __ffs(b) - 1;
+      list[pos++] = w * 32 + bit;
+      b &= b - 1;
+    }
+  }
+  if (threadIdx.x == 0) *count = sw[32];
+}
+
+}  // namespace
+
+gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                          int32_t d, int elem_bytes, void* d_E, cudaStream_t st) {
+  if (P < 0 || d <= 0 || n_src_rows < 0 || (elem_bytes != 2 && elem_bytes != 4))
+    return gram_set_error(ctx, "gram_gather: bad argument"), GRAM_ERR_ARG;
+  if (P == 0) return GRAM_OK;
+  if (!d_src || !d_index || !d_E || n_src_rows == 0)
+    return gram_set_error(ctx, "gram_gather: null buffer"), GRAM_ERR_ARG;
+  int32_t* status = gram_status_word(ctx);
+  const int64_t row_bytes = (int64_t)d * elem_bytes;
+  const bool vec_ok = (row_bytes % 16 == 0) && ((uintptr_t)d_src % 16 == 0) && ((uintptr_t)d_E % 16 == 0);
+  if (vec_ok) {
+    const int nvec = (int)(row_bytes / 16);
+    constexpr int ROWS = 4;
+    int64_t warps = ceil_div64(P, ROWS);
+    int blocks = (int)ceil_div64(warps, 8);
+    const int cap = kNumSMs * 8;
+    if (blocks > cap) blocks = cap;
+    gather_rows_kernel<ROWS><<<blocks, 256, 0, st>>>((const uint4*)d_src, n_src_rows, d_index, P, nvec, (uint4*)d_E,
+                                                     status);
+  } else {
+    int64_t n = P * d;
+    int blocks = (int)ceil_div64(n, 256);
+    if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
+    if (elem_bytes == 4)
+      gather_scalar_kernel<float><<<blocks, 256, 0, st>>>((const float*)d_src, n_src_rows, d_index, P, d, (float*)d_E, status);
+    else
+      gather_scalar_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)d_src, n_src_rows, d_index, P, d, (bf16*)d_E, status);
+  }
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+template <typename InT, int VPL>
+static void segsum_run(const void* d_in, const int32_t* d_perm, const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d,
+                       int64_t R, int nchunks, const int32_t* d_rows, int add, float* d_out, float* partial,
+                       int32_t* status, cudaStream_t st) {
+  const int nslabs = ceil_div(d, VPL * 128);
+  const int64_t warps = (int64_t)nchunks * nslabs;
+  const int blocks = (int)ceil_div64(warps, 8);
+  segsum_chunks_kernel<InT, VPL, 8><<<blocks, 256, 0, st>>>((const InT*)d_in, d_perm, d_seg_off, P, U, d, R, nchunks, nslabs,
+                                                            d_rows, add, d_out, partial, status);
+  if (nchunks > 1)
+    segsum_fixup_kernel<VPL><<<blocks, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial);
+}
+
+gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
+                              const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d, const int32_t* d_rows,
+                              int add, float* d_out, cudaStream_t st) {
+  if (P < 0 || U < 0 || d <= 0 || U > P) return gram_set_error(ctx, "gram_accumulate: bad argument"), GRAM_ERR_ARG;
+  if (P == 0 || U == 0) return GRAM_OK;
+  if (!d_in || !d_perm || !d_seg_off || !d_out) return gram_set_error(ctx, "gram_accumulate: null buffer"), GRAM_ERR_ARG;
+  if (d % 4 != 0 || ((uintptr_t)d_in % (in_bf16 ? 8 : 16)) || ((uintptr_t)d_out % 16))
+    return gram_set_error(ctx, "gram_accumulate: d must be a multiple of 4 and buffers 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
+  if (d > ws->d_max) return gram_set_error(ctx, "gram_accumulate: d=%d exceeds the context's d_max=%d", d, ws->d_max), GRAM_ERR_WORKSPACE;
+  // chunks: at least 16 rows each, at most kAccMaxChunks
+  int64_t nchunks = ceil_div64(P, 16);
+  if (nchunks > kAccMaxChunks) nchunks = kAccMaxChunks;
+  const int64_t R = ceil_div64(P, nchunks);
+  nchunks = ceil_div64(P, R);
+  if (d >= 256) {
+    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+  } else {
+    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+  }
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items, uint32_t* d_bits,
+                                cudaStream_t st) {
+  if (U <= 0) return GRAM_OK;
+  touched_mark_kernel<<<ceil_div(U, 256), 256, 0, st>>>(d_unique, U, n_items, d_bits, gram_status_word(ctx));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n_items, int32_t* d_list,
+                                int32_t* d_count, cudaStream_t st) {
+  if (n_items <= 0 || !d_bits || !d_list || !d_count) return gram_set_error(ctx, "gram_touched_list: bad argument"), GRAM_ERR_ARG;
+  touched_list_kernel<<<1, 1024, 0, st>>>(d_bits, n_items, d_list, d_count);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}

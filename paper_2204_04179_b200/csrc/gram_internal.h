@@ -1,0 +1,80 @@
+// Internal declarations shared by the CUDA translation units of libgram.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "gram.h"
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------------------
+// error plumbing
+// ---------------------------------------------------------------------------
+struct gram_ctx;
+void gram_set_error(gram_ctx* ctx, const char* fmt, ...);
+
+#define GRAM_CUDA(ctx, expr)                                                              \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess) {                                                             \
+      gram_set_error((ctx), "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+      return GRAM_ERR_CUDA;                                                               \
+    }                                                                                     \
+  } while (0)
+
+#define GRAM_TRY(expr)                        \
+  do {                                        \
+    gram_status s__ = (expr);                 \
+    if (s__ != GRAM_OK) return s__;           \
+  } while (0)
+
+#define GRAM_LAUNCH_CHECK(ctx) GRAM_CUDA(ctx, cudaGetLastError())
+
+static inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------
+// index / accumulation workspaces (dedup.cu, gather_accum.cu)
+// ---------------------------------------------------------------------------
+constexpr int kAccMaxChunks = 148 * 16;   // work units of the segmented sum
+constexpr int kNumSMs = 148;
+
+struct IndexWorkspace {
+  int64_t P_max = 0;
+  int32_t n_items_max = 0;
+  int32_t d_max = 0;
+  int32_t *keys0 = nullptr, *keys1 = nullptr, *vals0 = nullptr, *vals1 = nullptr;  // [P_max] radix ping-pong
+  int32_t* hist = nullptr;        // [256 * n_sort_blocks] digit-major block histograms
+  int32_t* block_sums = nullptr;  // scan scratch
+  int32_t* rank_table = nullptr;  // [n_items_max] item ID -> index in unique
+  float* partial = nullptr;       // [kAccMaxChunks * 2 * d_max] chunk-boundary partial sums
+  int32_t n_sort_blocks = 0;
+};
+
+gram_status index_ws_alloc(gram_ctx* ctx, IndexWorkspace* ws, int64_t P_max, int32_t n_items_max, int32_t d_max);
+void index_ws_free(IndexWorkspace* ws);
+
+gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids, int64_t P, int32_t n_items,
+                         int32_t* d_unique, int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off,
+                         int32_t* d_n_unique, cudaStream_t st);
+
+gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                          int32_t d, int elem_bytes, void* d_E, cudaStream_t st);
+
+// in_bf16: rows of d_in are bf16 instead of fp32.  d_rows (may be NULL): output row of segment u is
+// d_rows[u] instead of u.  add != 0: out[row] += sum instead of out[row] = sum.
+gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
+                              const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d, const int32_t* d_rows,
+                              int add, float* d_out, cudaStream_t st);
+
+gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items,
+                                uint32_t* d_bits, cudaStream_t st);
+gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n_items, int32_t* d_list,
+                                int32_t* d_count, cudaStream_t st);
+
+// the device status word: kernels record the first error kind they meet
+__device__ __forceinline__ void gram_device_fail(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+int32_t* gram_status_word(gram_ctx* ctx);

@@ -1,0 +1,187 @@
+"""Parity of the index and accumulation kernels (stages 1, 3, 4) with the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gram_oracle as orc
+from paper_2204_04179_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def index_ctx(P_max, n_items, d_max=1024):
+    cfg = binding.GramConfig()
+    cfg.n_items = n_items
+    cfg.P_max = P_max
+    cfg.d_max = d_max
+    cfg.d = d_max
+    return binding.Gram(cfg)
+
+
+def run_dedup(g, ids_np, n_items):
+    P = ids_np.size
+    cap = max(1, min(P, n_items))
+    ids = torch.from_numpy(ids_np).to(DEV)
+    unique = torch.full((cap,), -7, dtype=torch.int32, device=DEV)
+    inverse = torch.full((max(P, 1),), -7, dtype=torch.int32, device=DEV)
+    perm = torch.full((max(P, 1),), -7, dtype=torch.int32, device=DEV)
+    seg_off = torch.full((cap + 1,), -7, dtype=torch.int32, device=DEV)
+    nu = torch.full((1,), -7, dtype=torch.int32, device=DEV)
+    g.dedup(ids, n_items, unique, inverse, perm, seg_off, nu)
+    g.sync()
+    U = int(nu.item())
+    return U, unique[:U].cpu().numpy(), inverse[:P].cpu().numpy(), perm[:P].cpu().numpy(), seg_off[:U + 1].cpu().numpy()
+
+
+@pytest.mark.parametrize("P,N,s", [(1, 1, 1.0), (1, 5, 1.0), (160, 200, 1.1), (4096, 1000, 1.0), (4097, 255, 1.5),
+                                  (25_600, 10_000, 1.0), (3520, 100_000, 1.1), (100_003, 1_000_000, 0.8),
+                                  (300_000, 70_000, 1.5), (65_536, 257, 1.1)])
+def test_dedup_bit_exact(P, N, s):
+    ids = synth.zipf_ids(11, N, s, P)
+    g = index_ctx(P, N)
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, N)
+    want = orc.unique_inverse(ids)
+    assert U == len(want[0])
+    for got, w, name in zip((unique, inverse, perm, seg_off), want, ("unique", "inverse", "perm", "seg_off")):
+        assert np.array_equal(got, w), name
+    g.close()
+
+
+def test_dedup_tiny_against_bruteforce_and_fig1():
+    g = index_ctx(64, 16)
+    ids = np.array([3, 7, 3, 9, 7, 7, 1, 3, 9, 4, 1, 3], np.int32)      # Fig. 1: 12 interactions, 5 items
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, 16)
+    want = orc.unique_inverse_bruteforce(ids)
+    assert U == 5
+    for got, w in zip((unique, inverse, perm, seg_off), want):
+        assert np.array_equal(got, w)
+    g.close()
+
+
+def test_dedup_edge_cases():
+    g = index_ctx(5000, 300)
+    # empty batch
+    U, unique, inverse, perm, seg_off = run_dedup(g, np.zeros(0, np.int32), 300)
+    assert U == 0 and list(seg_off) == [0]
+    # all equal, all distinct, maximum ID
+    for ids in (np.full(5000, 299, np.int32), np.arange(300, dtype=np.int32)[::-1].copy(), np.array([299, 0, 299], np.int32)):
+        U, unique, inverse, perm, seg_off = run_dedup(g, ids, 300)
+        want = orc.unique_inverse(ids)
+        for got, w in zip((unique, inverse, perm, seg_off), want):
+            assert np.array_equal(got, w)
+    # out-of-range ID is reported, not a fault
+    bad = np.array([1, 2, 300, 4], np.int32)
+    with pytest.raises(binding.GramError) as e:
+        run_dedup(g, bad, 300)
+    assert e.value.status == 2
+    # the context is still usable
+    U, *_ = run_dedup(g, np.array([5, 5, 6], np.int32), 300)
+    assert U == 2
+    # too large for the context
+    with pytest.raises(binding.GramError) as e:
+        run_dedup(g, np.zeros(5001, np.int32), 300)
+    assert e.value.status == 3
+    g.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,U,d", [(160, 60, 64), (1000, 37, 768), (5001, 1234, 256), (300, 50, 1024), (77, 9, 6)])
+def test_gather_exact(P, U, d, dtype):
+    g = index_ctx(P, 10)
+    rng = np.random.default_rng(0)
+    H = torch.from_numpy(rng.standard_normal((U, d)).astype(np.float32)).to(DEV).to(dtype)
+    idx = torch.from_numpy(rng.integers(0, U, P).astype(np.int32)).to(DEV)
+    E = torch.zeros(P, d, dtype=dtype, device=DEV)
+    g.gather(H, idx, E)
+    g.sync()
+    assert torch.equal(E, H[idx.long()])
+    # an index past the source rows is reported
+    idx[P // 2] = U
+    g.gather(H, idx, E)
+    with pytest.raises(binding.GramError) as e:
+        g.sync()
+    assert e.value.status == 2
+    g.close()
+
+
+@pytest.mark.parametrize("P,N,s,d", [(160, 200, 1.1, 64), (25_600, 10_000, 1.0, 768), (50_000, 1000, 1.5, 256),
+                                    (40_000, 100_000, 0.8, 1024), (3000, 1, 1.0, 128), (2000, 5000, 1.1, 4),
+                                    (70_001, 3, 1.1, 768)])
+def test_accumulate_matches_fp64_segment_sum(P, N, s, d):
+    ids = synth.zipf_ids(5, N, s, P)
+    dE_np = synth.position_gradients(5, P, d)
+    g = index_ctx(P, N)
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, N)
+    # vectorised float64 statement of the oracle's loop (np.add.at adds rows in ascending position)
+    want = np.zeros((U, d))
+    np.add.at(want, inverse, dE_np.astype(np.float64))
+    if P <= 3000:
+        np.testing.assert_allclose(want, orc.segment_sum(dE_np, perm, seg_off), rtol=1e-12, atol=1e-12)
+    dE = torch.from_numpy(dE_np).to(DEV)
+    perm_d, so_d = torch.from_numpy(perm).to(DEV), torch.from_numpy(seg_off).to(DEV)
+    G = torch.full((U, d), float("nan"), device=DEV)
+    g.accumulate(dE, perm_d, so_d, U, G)
+    g.sync()
+    got = G.cpu().numpy().astype(np.float64)
+    # fp32 sums of n terms of magnitude <= 1: error <= n * 2^-24 * sum|x| bound; use a per-row bound
+    counts = np.diff(seg_off).astype(np.float64)[:, None]
+    bound = (counts * 2.0 ** -24) * counts + 1e-6
+    assert np.all(np.abs(got - want) <= bound)
+    assert np.abs(got.sum(0) - dE_np.astype(np.float64).sum(0)).max() <= 1e-3 * max(1.0, np.sqrt(P))
+    # bit-identical on a second run (fixed order of additions)
+    G2 = torch.full((U, d), float("nan"), device=DEV)
+    g.accumulate(dE, perm_d, so_d, U, G2)
+    g.sync()
+    assert torch.equal(G, G2)
+    g.close()
+
+
+def test_accumulate_special_cases():
+    P, d = 4100, 256
+    dE_np = synth.position_gradients(1, P, d)
+    dE = torch.from_numpy(dE_np).to(DEV)
+    g = index_ctx(P, P)
+    # all-distinct IDs: G is dE reordered, exactly
+    ids = np.random.default_rng(3).permutation(P).astype(np.int32)
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, P)
+    G = torch.empty(U, d, device=DEV)
+    g.accumulate(dE, torch.from_numpy(perm).to(DEV), torch.from_numpy(seg_off).to(DEV), U, G)
+    g.sync()
+    assert np.array_equal(G.cpu().numpy(), dE_np[perm])
+    g.close()
+
+
+def test_multistep_table_and_touched():
+    N, d, P = 1000, 768, 6000
+    g = index_ctx(P, N)
+    table = torch.zeros(N, d, device=DEV)
+    bits = torch.zeros((N + 31) // 32, dtype=torch.int32, device=DEV)
+    want = np.zeros((N, d))
+    touched = np.zeros(N, bool)
+    for step in range(3):
+        ids = synth.zipf_ids(9, N, 1.1, P, step=step)
+        dE_np = synth.position_gradients(9 + step, P, d)
+        U, unique, inverse, perm, seg_off = run_dedup(g, ids, N)
+        g.accumulate_multistep(torch.from_numpy(dE_np).to(DEV), torch.from_numpy(perm).to(DEV),
+                               torch.from_numpy(seg_off).to(DEV), torch.from_numpy(unique).to(DEV), U, N, table, bits)
+        np.add.at(want, ids, dE_np.astype(np.float64))
+        touched[ids] = True
+    g.sync()
+    got = table.cpu().numpy()
+    assert np.abs(got - want).max() <= 1e-3
+    assert np.all(got[~touched] == 0)
+    lst = torch.full((N,), -1, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    g.touched_list(bits, N, lst, cnt)
+    g.sync()
+    c = int(cnt.item())
+    assert np.array_equal(lst[:c].cpu().numpy(), np.nonzero(touched)[0].astype(np.int32))
+    # the oracle's own loop on a small slice of the same data
+    t2 = np.zeros((N, d)); tt = np.zeros(N, bool)
+    ids = synth.zipf_ids(9, N, 1.1, P, step=0)[:300]
+    dE_np = synth.position_gradients(9, P, d)[:300]
+    orc.table_accumulate(t2, tt, dE_np, ids)
+    chk = np.zeros((N, d)); np.add.at(chk, ids, dE_np.astype(np.float64))
+    np.testing.assert_allclose(t2, chk, rtol=1e-12, atol=1e-12)
+    g.close()
