@@ -3,6 +3,7 @@
 
 #include <new>
 
+#include "gemm.h"
 #include "gram_internal.h"
 #include "model.h"
 
@@ -11,6 +12,7 @@ struct gram_ctx {
   char err[512];
   int32_t* d_status = nullptr;      // device status word (first device-side error)
   IndexWorkspace iws;
+  GemmWorkspace gws;
   Model* model = nullptr;           // encoder + task module state (null for an index-only context)
 };
 
@@ -24,6 +26,7 @@ void gram_set_error(gram_ctx* ctx, const char* fmt, ...) {
 
 int32_t* gram_status_word(gram_ctx* ctx) { return ctx->d_status; }
 IndexWorkspace* gram_index_ws(gram_ctx* ctx) { return &ctx->iws; }
+GemmWorkspace* gram_gemm_ws(gram_ctx* ctx) { return &ctx->gws; }
 const gram_config* gram_cfg(const gram_ctx* ctx) { return &ctx->cfg; }
 
 static cudaStream_t S(gram_stream s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -72,6 +75,13 @@ gram_status gram_create(const gram_config* cfg, gram_ctx** out) {
     int32_t n_keys = cfg->n_items > cfg->vocab ? cfg->n_items : cfg->vocab;
     s = index_ws_alloc(ctx, &ctx->iws, P_max, n_keys, d_max);
     if (s != GRAM_OK) break;
+    {  // split-K partial products: up to 16 parts of the largest weight matrix, within 32..256 MB
+      size_t w = (size_t)(cfg->d_ff > cfg->task_d_ff ? cfg->d_ff : cfg->task_d_ff) * (size_t)cfg->d * sizeof(float) * 16;
+      if (w < ((size_t)32 << 20)) w = (size_t)32 << 20;
+      if (w > ((size_t)256 << 20)) w = (size_t)256 << 20;
+      s = gemm_ws_alloc(ctx, &ctx->gws, w);
+      if (s != GRAM_OK) break;
+    }
     if (ctx->cfg.n_layers > 0 || ctx->cfg.task != GRAM_TASK_NONE) {
       s = model_create(ctx, &ctx->cfg, &ctx->model);
       if (s != GRAM_OK) break;
@@ -91,6 +101,7 @@ gram_status gram_destroy(gram_ctx* ctx) {
   cudaDeviceSynchronize();
   if (ctx->model) model_destroy(ctx->model);
   index_ws_free(&ctx->iws);
+  gemm_ws_free(&ctx->gws);
   cudaFree(ctx->d_status);
   delete ctx;
   return GRAM_OK;
@@ -218,7 +229,13 @@ gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const v
                            int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
                            gram_stream stream) {
   if (!ctx) return GRAM_ERR_ARG;
-  return gemm_bf16_public(ctx, d_A, a_kmajor, d_B, b_kmajor, d_C, c_f32, d_bias, accumulate, M, N, K, S(stream));
+  if (M < 0 || N < 0 || K <= 0 || (M % 8) || (N % 8) || (K % 8))
+    return gram_set_error(ctx, "gram_gemm_bf16: M, N, K must be positive multiples of 8"), GRAM_ERR_ARG;
+  GemmEpilogue e;
+  e.bias = d_bias;
+  e.accumulate = accumulate;
+  return gemm_launch(ctx, &ctx->gws, GRAM_BF16, d_A, a_kmajor, a_kmajor ? K : M, d_B, b_kmajor, b_kmajor ? K : N, d_C,
+                     c_f32, N, M, N, K, e, 1, S(stream));
 }
 
 }  // extern "C"

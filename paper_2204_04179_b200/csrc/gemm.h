@@ -1,0 +1,46 @@
+// Matrix products of the encoder and task module.
+#pragma once
+#include "gram_internal.h"
+
+// What happens to an accumulator element acc(m, n) before it is stored to C(m, n):
+//   v = acc + bias[n]
+//   gelu:       pre(m, n) = v (if pre != null);  v = gelu(v)          (forward of the feed-forward layer)
+//   dgelu_pre:  v = v * gelu'(dgelu_pre(m, n))                        (backward through the GELU)
+//   residual:   v += residual(m, n)
+//   accumulate: v += C(m, n)                                          (fp32 C only)
+// pre, dgelu_pre and residual have C's element type and leading dimension.
+struct GemmEpilogue {
+  const float* bias = nullptr;
+  const void* residual = nullptr;
+  void* pre = nullptr;
+  const void* dgelu_pre = nullptr;
+  int gelu = 0;
+  int accumulate = 0;
+};
+
+struct GemmWorkspace {
+  float* splitk = nullptr;      // partial products of split-K launches
+  size_t splitk_bytes = 0;
+};
+
+// C[M, N] = op(A) x op(B)^T with fp32 accumulation.
+//   a_kmajor: A is [M, K] (lda elements between rows), else [K, M].
+//   b_kmajor: B is [N, K] (ldb), else [K, N].
+//   dtype GRAM_F32: A, B float (plain CUDA cores).  GRAM_BF16: A, B bf16 on the tensor cores
+//   (tcgen05 with TMA-fed shared-memory operands and the accumulator in tensor memory).
+//   c_f32: C (and the epilogue's matrices) float, else bf16.  For GRAM_F32, c_f32 must be 1.
+//   allow_splitk: the K range may be cut into parts that are added in a fixed order.
+gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void* A, int a_kmajor, int64_t lda,
+                        const void* B, int b_kmajor, int64_t ldb, void* C, int c_f32, int64_t ldc, int64_t M, int N,
+                        int64_t K, const GemmEpilogue& epi, int allow_splitk, cudaStream_t st);
+
+gram_status gemm_ws_alloc(gram_ctx* ctx, GemmWorkspace* ws, size_t splitk_bytes);
+void gemm_ws_free(GemmWorkspace* ws);
+
+__host__ __device__ inline float gelu_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+__host__ __device__ inline float gelu_grad_f(float x) {
+  // d/dx [x * Phi(x)] = Phi(x) + x * phi(x)
+  const float cdf = 0.5f * (1.0f + erff(x * 0.70710678118654752f));
+  const float pdf = 0.39894228040143268f * expf(-0.5f * x * x);
+  return cdf + x * pdf;
+}

@@ -27,6 +27,5 @@ gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, floa
 float* model_table(Model* m);
 uint32_t* model_touched(Model* m);
 
-gram_status gemm_bf16_public(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
-                             int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
-                             cudaStream_t st);
+struct GemmWorkspace;
+GemmWorkspace* gram_gemm_ws(gram_ctx* ctx);

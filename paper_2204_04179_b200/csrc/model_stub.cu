@@ -16,4 +16,3 @@ gram_status model_window_reset(Model*, cudaStream_t) { return GRAM_ERR_UNSUPPORT
 gram_status model_get_window(Model*, float*, uint32_t*, float*) { return GRAM_ERR_UNSUPPORTED; }
 float* model_table(Model*) { return nullptr; }
 uint32_t* model_touched(Model*) { return nullptr; }
-gram_status gemm_bf16_public(gram_ctx*, const void*, int, const void*, int, void*, int, const float*, int, int64_t, int32_t, int64_t, cudaStream_t) { return GRAM_ERR_UNSUPPORTED; }
