@@ -56,10 +56,10 @@ gram_status gram_create(const gram_config* cfg, gram_ctx** out) {
   if (ctx->cfg.K == 0) ctx->cfg.K = 1;
   int64_t P_max = cfg->P_max > 0 ? cfg->P_max : (int64_t)cfg->B_max * cfg->L;
   if (ctx->cfg.n_layers > 0) {       // the token-embedding gradient reuses the index kernels over token positions
-    int64_t mb = cfg->ce_micro_batch > 0 ? cfg->ce_micro_batch : cfg->n_items;
+    const int64_t u_cap = P_max < cfg->n_items ? P_max : cfg->n_items;
+    int64_t mb = cfg->ce_micro_batch > 0 ? cfg->ce_micro_batch : (ctx->cfg.K > 1 ? cfg->n_items : u_cap);
     if (mb > cfg->n_items) mb = cfg->n_items;
-    if (mb > P_max && P_max > 0 && cfg->K <= 1) mb = P_max;
-    int64_t tok = mb * cfg->l_t;
+    const int64_t tok = mb * cfg->l_t;
     if (tok > P_max) P_max = tok;
   }
   ctx->cfg.P_max = P_max;
@@ -132,7 +132,7 @@ gram_status gram_gather(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, co
 gram_status gram_accumulate(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm, const int32_t* d_seg_off,
                             int64_t P, int32_t U, int32_t d, float* d_G, gram_stream stream) {
   if (!ctx) return GRAM_ERR_ARG;
-  return accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, d, nullptr, 0, d_G, S(stream));
+  return accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, nullptr, d, nullptr, 0, d_G, S(stream));
 }
 
 gram_status gram_accumulate_multistep(gram_ctx* ctx, const float* d_dE, const int32_t* d_perm,
@@ -147,7 +147,7 @@ gram_status gram_accumulate_multistep(gram_ctx* ctx, const float* d_dE, const in
     if (!d_table) d_table = model_table(ctx->model);
     if (!d_touched_bits) d_touched_bits = model_touched(ctx->model);
   }
-  GRAM_TRY(accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, d, d_unique, 1, d_table, S(stream)));
+  GRAM_TRY(accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, nullptr, d, d_unique, 1, d_table, S(stream)));
   return touched_mark_launch(ctx, d_unique, U, n_items, d_touched_bits, S(stream));
 }
 

@@ -117,7 +117,9 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
                                                             int d, int64_t R, int nchunks, int nslabs,
                                                             const int32_t* __restrict__ rows, int add,
                                                             float* __restrict__ out, float* __restrict__ partial,
-                                                            int32_t* status) {
+                                                            int32_t* status, const int32_t* __restrict__ d_U) {
+  if (d_U) U = *d_U;            // the number of items may live on the device
+  if (U <= 0) return;
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (w >= (int64_t)nchunks * nslabs) return;
@@ -186,7 +188,10 @@ template <int VPL>
 __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __restrict__ seg_off, int64_t P, int32_t U,
                                                            int d, int64_t R, int nchunks, int nslabs,
                                                            const int32_t* __restrict__ rows, int add,
-                                                           float* __restrict__ out, const float* __restrict__ partial) {
+                                                           float* __restrict__ out, const float* __restrict__ partial,
+                                                           const int32_t* __restrict__ d_U) {
+  if (d_U) U = *d_U;
+  if (U <= 0) return;
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (w >= (int64_t)nchunks * nslabs) return;
@@ -312,21 +317,21 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
 template <typename InT, int VPL>
 static void segsum_run(const void* d_in, const int32_t* d_perm, const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d,
                        int64_t R, int nchunks, const int32_t* d_rows, int add, float* d_out, float* partial,
-                       int32_t* status, cudaStream_t st) {
+                       int32_t* status, const int32_t* d_U, cudaStream_t st) {
   const int nslabs = ceil_div(d, VPL * 128);
   const int64_t warps = (int64_t)nchunks * nslabs;
   const int blocks = (int)ceil_div64(warps, 8);
   segsum_chunks_kernel<InT, VPL, 8><<<blocks, 256, 0, st>>>((const InT*)d_in, d_perm, d_seg_off, P, U, d, R, nchunks, nslabs,
-                                                            d_rows, add, d_out, partial, status);
+                                                            d_rows, add, d_out, partial, status, d_U);
   if (nchunks > 1)
-    segsum_fixup_kernel<VPL><<<blocks, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial);
+    segsum_fixup_kernel<VPL><<<blocks, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, d_U);
 }
 
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
-                              const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d, const int32_t* d_rows,
-                              int add, float* d_out, cudaStream_t st) {
+                              const int32_t* d_seg_off, int64_t P, int32_t U, const int32_t* d_U, int32_t d,
+                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st) {
   if (P < 0 || U < 0 || d <= 0 || U > P) return gram_set_error(ctx, "gram_accumulate: bad argument"), GRAM_ERR_ARG;
-  if (P == 0 || U == 0) return GRAM_OK;
+  if (P == 0 || (U == 0 && !d_U)) return GRAM_OK;
   if (!d_in || !d_perm || !d_seg_off || !d_out) return gram_set_error(ctx, "gram_accumulate: null buffer"), GRAM_ERR_ARG;
   if (d % 4 != 0 || ((uintptr_t)d_in % (in_bf16 ? 8 : 16)) || ((uintptr_t)d_out % 16))
     return gram_set_error(ctx, "gram_accumulate: d must be a multiple of 4 and buffers 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
@@ -337,11 +342,11 @@ gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_i
   const int64_t R = ceil_div64(P, nchunks);
   nchunks = ceil_div64(P, R);
   if (d >= 256) {
-    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
-    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
+    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
   } else {
-    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
-    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), st);
+    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
+    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
   }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;

@@ -64,11 +64,12 @@ gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids
 gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
                           int32_t d, int elem_bytes, void* d_E, cudaStream_t st);
 
-// in_bf16: rows of d_in are bf16 instead of fp32.  d_rows (may be NULL): output row of segment u is
-// d_rows[u] instead of u.  add != 0: out[row] += sum instead of out[row] = sum.
+// in_bf16: rows of d_in are bf16 instead of fp32.  d_U (may be NULL): the number of segments is read
+// from the device instead of U.  d_rows (may be NULL): output row of segment u is d_rows[u] instead
+// of u.  add != 0: out[row] += sum instead of out[row] = sum.
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
-                              const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d, const int32_t* d_rows,
-                              int add, float* d_out, cudaStream_t st);
+                              const int32_t* d_seg_off, int64_t P, int32_t U, const int32_t* d_U, int32_t d,
+                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st);
 
 gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items,
                                 uint32_t* d_bits, cudaStream_t st);

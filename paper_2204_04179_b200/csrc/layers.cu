@@ -1,0 +1,839 @@
+// Non-GEMM layers: embedding, LayerNorm, attention over short sequences, pooling, bias-gradient
+// column sums, the task heads.  All reductions that feed parameter gradients run in a fixed order
+// (per-warp registers -> ordered block sum -> ordered sum over blocks), so results are bit-stable.
+#include "gemm.h"
+#include "layers.h"
+
+namespace {
+
+__device__ __forceinline__ float ldf(const float* p) { return *p; }
+__device__ __forceinline__ float ldf(const bf16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float* p, float v) { *p = v; }
+__device__ __forceinline__ void stf(bf16* p, float v) { *p = __float2bfloat16(v); }
+__device__ __forceinline__ float2 ld2(const float* p) { return *reinterpret_cast<const float2*>(p); }
+__device__ __forceinline__ float2 ld2(const bf16* p) {
+  return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+}
+__device__ __forceinline__ void st2(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
+__device__ __forceinline__ void st2(bf16* p, float2 v) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v.x, v.y);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ---------------------------------------------------------------------------- embedding
+template <typename T>
+__global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const int32_t* __restrict__ items,
+                                 int32_t first_item, int64_t n_tok, int32_t n_items_total, int l_t, int vocab, int d,
+                                 const float* __restrict__ tok_emb, const float* __restrict__ pos_emb, T* __restrict__ z0,
+                                 int32_t* __restrict__ tok_ids, int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t t = w; t < n_tok; t += nw) {
+    const int64_t u = t / l_t;
+    const int s = (int)(t - u * l_t);
+    int32_t item = items ? items[u] : first_item + (int32_t)u;
+    if (item < 0 || item >= n_items_total) { gram_device_fail(status, GRAM_ERR_ID_RANGE); item = 0; }
+    int32_t tok = item_tokens[(int64_t)item * l_t + s];
+    if (tok < 0 || tok >= vocab) { gram_device_fail(status, GRAM_ERR_ID_RANGE); tok = 0; }
+    if (lane == 0) tok_ids[t] = tok;
+    const float* te = tok_emb + (int64_t)tok * d;
+    const float* pe = pos_emb + (int64_t)s * d;
+    for (int c = 2 * lane; c < d; c += 64) {
+      float2 a = ld2(te + c), b = ld2(pe + c);
+      st2(z0 + t * d + c, make_float2(a.x + b.x, a.y + b.y));
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------- LayerNorm
+template <typename T, int NP>   // NP pairs of columns per lane: d <= 64*NP
+__global__ void __launch_bounds__(256) ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ g,
+                                                     const float* __restrict__ b, T* __restrict__ y,
+                                                     float* __restrict__ mean, float* __restrict__ rstd, int64_t rows,
+                                                     int d) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t r = w; r < rows; r += nw) {
+    float2 v[NP];
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = 2 * (lane + 32 * i);
+      v[i] = (c < d) ? ld2(z + r * d + c) : make_float2(0.f, 0.f);
+      s += v[i].x + v[i].y;
+    }
+    const float mu = warp_sum(s) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = 2 * (lane + 32 * i);
+      if (c < d) q += (v[i].x - mu) * (v[i].x - mu) + (v[i].y - mu) * (v[i].y - mu);
+    }
+    const float rs = rsqrtf(warp_sum(q) / d + kLnEps);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = 2 * (lane + 32 * i);
+      if (c < d) {
+        float2 gg = ld2(g + c), bb = ld2(b + c);
+        st2(y + r * d + c, make_float2((v[i].x - mu) * rs * gg.x + bb.x, (v[i].y - mu) * rs * gg.y + bb.y));
+      }
+    }
+    if (lane == 0) {
+      mean[r] = mu;
+      rstd[r] = rs;
+    }
+  }
+}
+
+template <typename T, int NP>
+__global__ void __launch_bounds__(256) ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z,
+                                                     const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                     const float* __restrict__ g, T* __restrict__ dz,
+                                                     float* __restrict__ part, int64_t rows, int d) {
+  extern __shared__ float sacc[];          // [2][d]: dgamma, dbeta of this block
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
+  const int64_t w = (int64_t)blockIdx.x * nwb + warp;
+  const int64_t nw = (int64_t)gridDim.x * nwb;
+  float2 ag[NP], ab[NP], gg[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int c = 2 * (lane + 32 * i);
+    ag[i] = make_float2(0.f, 0.f);
+    ab[i] = make_float2(0.f, 0.f);
+    gg[i] = (c < d) ? ld2(g + c) : make_float2(0.f, 0.f);
+  }
+  for (int64_t r = w; r < rows; r += nw) {
+    const float mu = mean[r], rs = rstd[r];
+    float2 xh[NP], gy[NP];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = 2 * (lane + 32 * i);
+      if (c < d) {
+        float2 zz = ld2(z + r * d + c), dd = ld2(dy + r * d + c);
+        xh[i] = make_float2((zz.x - mu) * rs, (zz.y - mu) * rs);
+        gy[i] = make_float2(dd.x * gg[i].x, dd.y * gg[i].y);
+        ag[i].x += dd.x * xh[i].x; ag[i].y += dd.y * xh[i].y;
+        ab[i].x += dd.x; ab[i].y += dd.y;
+        s1 += gy[i].x + gy[i].y;
+        s2 += gy[i].x * xh[i].x + gy[i].y * xh[i].y;
+      } else {
+        xh[i] = make_float2(0.f, 0.f);
+        gy[i] = make_float2(0.f, 0.f);
+      }
+    }
+    s1 = warp_sum(s1) / d;
+    s2 = warp_sum(s2) / d;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = 2 * (lane + 32 * i);
+      if (c < d) st2(dz + r * d + c, make_float2(rs * (gy[i].x - s1 - xh[i].x * s2), rs * (gy[i].y - s1 - xh[i].y * s2)));
+    }
+  }
+  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sacc[i] = 0.f;
+  __syncthreads();
+  for (int ww = 0; ww < nwb; ++ww) {       // warps add in ascending order
+    if (warp == ww) {
+#pragma unroll
+      for (int i = 0; i < NP; ++i) {
+        const int c = 2 * (lane + 32 * i);
+        if (c < d) {
+          sacc[c] += ag[i].x; sacc[c + 1] += ag[i].y;
+          sacc[d + c] += ab[i].x; sacc[d + c + 1] += ab[i].y;
+        }
+      }
+    }
+    __syncthreads();
+  }
+  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) part[(int64_t)blockIdx.x * 2 * d + i] = sacc[i];
+}
+
+// out[c] += sum_b part[b*stride + c]   (two outputs when out2 != null: second half of each partial row)
+__global__ void reduce_partials_kernel(const float* __restrict__ part, int nblocks, int64_t stride, int n,
+                                       float* __restrict__ out, float* __restrict__ out2, float scale) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= n) return;
+  float a = 0.f, b = 0.f;
+  for (int k = 0; k < nblocks; ++k) {
+    a += part[(int64_t)k * stride + c];
+    if (out2) b += part[(int64_t)k * stride + n + c];
+  }
+  out[c] += a * scale;
+  if (out2) out2[c] += b * scale;
+}
+
+// ---------------------------------------------------------------------------- attention
+// One block per (sequence, head).  Rows of Q, K, V live in shared memory as fp32 with a padded
+// stride; a warp owns one query row at a time, with keys spread over lanes (S <= 128).
+template <typename T>
+__global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out, int S, int d,
+                                                       int n_heads, int causal, float scale) {
+  extern __shared__ float sm[];
+  const int dh = d / n_heads, ld = dh + 1;
+  float* Q = sm;
+  float* K = Q + S * ld;
+  float* V = K + S * ld;
+  const int64_t seq = blockIdx.x / n_heads;
+  const int h = blockIdx.x % n_heads;
+  const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
+  for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
+    const int s = i / dh, c = i - s * dh;
+    const T* p = base + (int64_t)s * 3 * d + c;
+    Q[s * ld + c] = ldf(p);
+    K[s * ld + c] = ldf(p + d);
+    V[s * ld + c] = ldf(p + 2 * d);
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
+  for (int i = warp; i < S; i += nwb) {
+    float p[4];
+    float m = -INFINITY;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int j = lane + 32 * jj;
+      float sc = -INFINITY;
+      if (j < S && (!causal || j <= i)) {
+        float acc = 0.f;
+        for (int c = 0; c < dh; ++c) acc += Q[i * ld + c] * K[j * ld + c];
+        sc = acc * scale;
+      }
+      p[jj] = sc;
+      m = fmaxf(m, sc);
+    }
+    m = warp_max(m);
+    float l = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      p[jj] = (p[jj] == -INFINITY) ? 0.f : __expf(p[jj] - m);
+      l += p[jj];
+    }
+    l = warp_sum(l);
+    const float inv = 1.f / l;
+    const int jmax = causal ? i + 1 : S;
+    float o0 = 0.f, o1 = 0.f;      // columns lane and lane + 32 (dh <= 64)
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      for (int l2 = 0; l2 < 32; ++l2) {
+        const int j = jj * 32 + l2;
+        if (j >= jmax) break;
+        const float pj = __shfl_sync(0xffffffffu, p[jj], l2);
+        if (lane < dh) o0 += pj * V[j * ld + lane];
+        if (lane + 32 < dh) o1 += pj * V[j * ld + lane + 32];
+      }
+    }
+    T* o = out + (seq * S + i) * (int64_t)d + h * dh;
+    if (lane < dh) stf(o + lane, o0 * inv);
+    if (lane + 32 < dh) stf(o + lane + 32, o1 * inv);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dctx,
+                                                       T* __restrict__ dqkv, int S, int d, int n_heads, int causal,
+                                                       float scale) {
+  extern __shared__ float sm[];
+  const int dh = d / n_heads, ld = dh + 1, lp = S + 1;
+  float* Q = sm;
+  float* K = Q + S * ld;
+  float* V = K + S * ld;
+  float* dO = V + S * ld;
+  float* Pm = dO + S * ld;       // [S][S+1] probabilities
+  float* dS = Pm + S * lp;       // [S][S+1] gradient of the scaled scores
+  const int64_t seq = blockIdx.x / n_heads;
+  const int h = blockIdx.x % n_heads;
+  const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
+  const T* dbase = dctx + seq * S * (int64_t)d + h * dh;
+  for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
+    const int s = i / dh, c = i - s * dh;
+    const T* p = base + (int64_t)s * 3 * d + c;
+    Q[s * ld + c] = ldf(p);
+    K[s * ld + c] = ldf(p + d);
+    V[s * ld + c] = ldf(p + 2 * d);
+    dO[s * ld + c] = ldf(dbase + (int64_t)s * d + c);
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
+  T* dbq = dqkv + seq * S * 3 * (int64_t)d + h * dh;
+  // phase 1: one query row per warp: probabilities, dS, and dQ
+  for (int i = warp; i < S; i += nwb) {
+    float p[4], dp[4];
+    float m = -INFINITY;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int j = lane + 32 * jj;
+      float sc = -INFINITY, g = 0.f;
+      if (j < S && (!causal || j <= i)) {
+        float acc = 0.f;
+        for (int c = 0; c < dh; ++c) {
+          acc += Q[i * ld + c] * K[j * ld + c];
+          g += dO[i * ld + c] * V[j * ld + c];
+        }
+        sc = acc * scale;
+      }
+      p[jj] = sc;
+      dp[jj] = g;
+      m = fmaxf(m, sc);
+    }
+    m = warp_max(m);
+    float l = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      p[jj] = (p[jj] == -INFINITY) ? 0.f : __expf(p[jj] - m);
+      l += p[jj];
+    }
+    l = warp_sum(l);
+    const float inv = 1.f / l;
+    float delta = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      p[jj] *= inv;
+      delta += p[jj] * dp[jj];
+    }
+    delta = warp_sum(delta);
+    float ds[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int j = lane + 32 * jj;
+      ds[jj] = p[jj] * (dp[jj] - delta) * scale;
+      if (j < S) {
+        Pm[i * lp + j] = p[jj];
+        dS[i * lp + j] = ds[jj];
+      }
+    }
+    const int jmax = causal ? i + 1 : S;
+    float o0 = 0.f, o1 = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      for (int l2 = 0; l2 < 32; ++l2) {
+        const int j = jj * 32 + l2;
+        if (j >= jmax) break;
+        const float dsj = __shfl_sync(0xffffffffu, ds[jj], l2);
+        if (lane < dh) o0 += dsj * K[j * ld + lane];
+        if (lane + 32 < dh) o1 += dsj * K[j * ld + lane + 32];
+      }
+    }
+    T* o = dbq + (int64_t)i * 3 * d;
+    if (lane < dh) stf(o + lane, o0);
+    if (lane + 32 < dh) stf(o + lane + 32, o1);
+  }
+  __syncthreads();
+  // phase 2: one key row per warp: dK[j] = sum_i dS[i][j] Q[i], dV[j] = sum_i P[i][j] dO[i]
+  for (int j = warp; j < S; j += nwb) {
+    float k0 = 0.f, k1 = 0.f, v0 = 0.f, v1 = 0.f;
+    const int i0 = causal ? j : 0;
+    for (int i = i0; i < S; ++i) {
+      const float a = dS[i * lp + j], b = Pm[i * lp + j];
+      if (lane < dh) { k0 += a * Q[i * ld + lane]; v0 += b * dO[i * ld + lane]; }
+      if (lane + 32 < dh) { k1 += a * Q[i * ld + lane + 32]; v1 += b * dO[i * ld + lane + 32]; }
+    }
+    T* o = dbq + (int64_t)j * 3 * d;
+    if (lane < dh) { stf(o + d + lane, k0); stf(o + 2 * d + lane, v0); }
+    if (lane + 32 < dh) { stf(o + d + lane + 32, k1); stf(o + 2 * d + lane + 32, v1); }
+  }
+}
+
+// ---------------------------------------------------------------------------- column sums
+// grid (column slabs of 64, row blocks); each warp sums rows warp, warp+8, ... of the block's range
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, int64_t rows, int N, int64_t rows_per_block,
+                                                     float* __restrict__ part) {
+  __shared__ float2 sw[8][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * 64 + 2 * lane;
+  const int64_t r0 = (int64_t)blockIdx.y * rows_per_block, r1 = min(r0 + rows_per_block, rows);
+  float2 acc = make_float2(0.f, 0.f);
+  if (c < N) {
+    for (int64_t r = r0 + warp; r < r1; r += 8) {
+      float2 v = ld2(X + r * N + c);
+      acc.x += v.x;
+      acc.y += v.y;
+    }
+  }
+  sw[warp][lane] = acc;
+  __syncthreads();
+  if (warp == 0 && c < N) {
+    float2 t = sw[0][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) { t.x += sw[w][lane].x; t.y += sw[w][lane].y; }
+    part[(int64_t)blockIdx.y * N + c] = t.x;
+    part[(int64_t)blockIdx.y * N + c + 1] = t.y;
+  }
+}
+
+template <typename T>
+__global__ void periodic_rowsum_kernel(const T* __restrict__ X, int64_t n_groups, int period, int d, float* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (int64_t)period * d) return;
+  const int s = (int)(i / d), c = (int)(i - (int64_t)s * d);
+  float acc = 0.f;
+  for (int64_t u = 0; u < n_groups; ++u) acc += ldf(X + (u * period + s) * d + c);
+  out[i] += acc;
+}
+
+// ---------------------------------------------------------------------------- pooling
+template <typename T>
+__global__ void pool_fwd_kernel(const T* __restrict__ x, T* __restrict__ H, int64_t n, int l_t, int d, int pooling) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * d) return;
+  const int64_t u = i / d;
+  const int c = (int)(i - u * d);
+  if (pooling == GRAM_POOL_CLS) {
+    H[i] = x[u * l_t * d + c];
+  } else {
+    float acc = 0.f;
+    for (int s = 0; s < l_t; ++s) acc += ldf(x + (u * l_t + s) * d + c);
+    stf(H + i, acc / l_t);
+  }
+}
+template <typename T>
+__global__ void pool_bwd_kernel(const float* __restrict__ G, T* __restrict__ dx, int64_t n, int l_t, int d, int pooling) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * l_t * d) return;
+  const int64_t t = i / d;
+  const int c = (int)(i - t * d);
+  const int64_t u = t / l_t;
+  const int s = (int)(t - u * l_t);
+  float v;
+  if (pooling == GRAM_POOL_CLS) v = (s == 0) ? G[u * d + c] : 0.f;
+  else v = G[u * d + c] / l_t;
+  stf(dx + i, v);
+}
+
+// ---------------------------------------------------------------------------- KT task input / head
+template <typename T>
+__global__ void kt_input_fwd_kernel(const T* __restrict__ E, const float* __restrict__ pos, const float* __restrict__ resp,
+                                    const int32_t* __restrict__ labels, T* __restrict__ x, int64_t P, int L, int d) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= P * d) return;
+  const int64_t p = i / d;
+  const int c = (int)(i - p * d);
+  const int n = (int)(p % L);
+  int prev = (n == 0) ? 2 : labels[p - 1];
+  prev = prev < 0 ? 0 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);
+  stf(x + i, ldf(E + i) + pos[(int64_t)n * d + c] + resp[(int64_t)prev * d + c]);
+}
+// one thread per column: dE = dx; dpos[n, c] += sum_b; dresp[r, c] += sum over positions with prev == r
+template <typename T>
+__global__ void kt_input_bwd_kernel(const T* __restrict__ dx, const int32_t* __restrict__ labels, float* __restrict__ dE,
+                                    float* __restrict__ dpos, float* __restrict__ dresp, int B, int L, int d) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = blockIdx.y;
+  if (c >= d) return;
+  float ap = 0.f, r0 = 0.f, r1 = 0.f, r2 = 0.f;
+  for (int b = 0; b < B; ++b) {
+    const int64_t p = (int64_t)b * L + n;
+    const float v = ldf(dx + p * d + c);
+    dE[p * d + c] = v;
+    ap += v;
+    int prev = (n == 0) ? 2 : labels[p - 1];
+    if (prev == 0) r0 += v; else if (prev == 1) r1 += v; else r2 += v;
+  }
+  dpos[(int64_t)n * d + c] += ap;
+  // per-position partial of dresp, reduced over n by the caller: part[n][3][d]
+  dresp[((int64_t)n * 3 + 0) * d + c] = r0;
+  dresp[((int64_t)n * 3 + 1) * d + c] = r1;
+  dresp[((int64_t)n * 3 + 2) * d + c] = r2;
+}
+
+// warp per position; per-block partials: [d] for dw, then loss and db
+template <typename T>
+__global__ void __launch_bounds__(256) kt_head_kernel(const T* __restrict__ y, const float* __restrict__ w,
+                                                      const float* __restrict__ bias, const int32_t* __restrict__ labels,
+                                                      T* __restrict__ dy, float* __restrict__ part, int64_t P, int d,
+                                                      int64_t pstride) {
+  extern __shared__ float sacc[];            // [d + 2]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
+  for (int i = threadIdx.x; i < d + 2; i += blockDim.x) sacc[i] = 0.f;
+  __syncthreads();
+  const float b0 = bias[0], invP = 1.f / (float)P;
+  // rows are dealt to blocks in contiguous ranges so that each block adds its rows in order
+  const int64_t per = (P + gridDim.x - 1) / gridDim.x;
+  const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(r0 + per, P);
+  for (int64_t rb = r0; rb < r1; rb += nwb) {
+    const int64_t r = rb + warp;
+    float dzl = 0.f, lossr = 0.f;
+    if (r < r1) {
+      float acc = 0.f;
+      for (int c = lane; c < d; c += 32) acc += ldf(y + r * d + c) * w[c];
+      const float z = warp_sum(acc) + b0;
+      const float lab = (float)labels[r];
+      lossr = fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
+      dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
+      for (int c = lane; c < d; c += 32) stf(dy + r * d + c, dzl * w[c]);
+    }
+    for (int ww = 0; ww < nwb; ++ww) {       // rows of this round add in ascending order
+      if (warp == ww && r < r1) {
+        for (int c = lane; c < d; c += 32) sacc[c] += dzl * ldf(y + r * d + c);
+        if (lane == 0) { sacc[d] += lossr; sacc[d + 1] += dzl; }
+      }
+      __syncthreads();
+    }
+  }
+  for (int i = threadIdx.x; i < d + 2; i += blockDim.x) part[(int64_t)blockIdx.x * pstride + i] = sacc[i];
+}
+
+__global__ void kt_head_reduce_kernel(const float* __restrict__ part, int nblocks, int64_t pstride, int d, float invP,
+                                      float* __restrict__ dw, float* __restrict__ db, float* __restrict__ loss) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d + 2) return;
+  float a = 0.f;
+  for (int k = 0; k < nblocks; ++k) a += part[(int64_t)k * pstride + c];
+  if (c < d) dw[c] += a;
+  else if (c == d) loss[0] = a * invP;
+  else db[0] += a;
+}
+
+// ---------------------------------------------------------------------------- NR task (per user)
+// pre[b, n, :] = E[b, n, :] wa^T + ba is given.  One block per user.
+template <typename T>
+__global__ void __launch_bounds__(256) nr_user_kernel(const T* __restrict__ E, const T* __restrict__ pre,
+                                                      const float* __restrict__ qa, float* __restrict__ dE,
+                                                      T* __restrict__ dpre, float* __restrict__ part, int L, int n_cand,
+                                                      int d, int d_a, float invB) {
+  extern __shared__ float sm[];
+  const int n_hist = L - n_cand;
+  float* a = sm;                 // [L] scores / alpha
+  float* da = a + L;             // [L]
+  float* u = da + L;             // [d]
+  float* du = u + d;             // [d]
+  float* sc = du + d;            // [n_cand] scores, then ds
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
+  const T* Eb = E + (int64_t)b * L * d;
+  const T* pb = pre + (int64_t)b * L * d_a;
+  for (int n = warp; n < n_hist; n += nwb) {
+    float acc = 0.f;
+    for (int k = lane; k < d_a; k += 32) acc += qa[k] * tanhf(ldf(pb + (int64_t)n * d_a + k));
+    acc = warp_sum(acc);
+    if (lane == 0) a[n] = acc;
+  }
+  __syncthreads();
+  if (warp == 0) {               // softmax over the history
+    float m = -INFINITY;
+    for (int n = lane; n < n_hist; n += 32) m = fmaxf(m, a[n]);
+    m = warp_max(m);
+    float l = 0.f;
+    for (int n = lane; n < n_hist; n += 32) l += __expf(a[n] - m);
+    l = warp_sum(l);
+    for (int n = lane; n < n_hist; n += 32) a[n] = __expf(a[n] - m) / l;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.f;
+    for (int n = 0; n < n_hist; ++n) acc += a[n] * ldf(Eb + (int64_t)n * d + c);
+    u[c] = acc;
+  }
+  __syncthreads();
+  for (int j = warp; j < n_cand; j += nwb) {
+    float acc = 0.f;
+    for (int c = lane; c < d; c += 32) acc += u[c] * ldf(Eb + (int64_t)(n_hist + j) * d + c);
+    acc = warp_sum(acc);
+    if (lane == 0) sc[j] = acc;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = -INFINITY;
+    for (int j = 0; j < n_cand; ++j) m = fmaxf(m, sc[j]);
+    float l = 0.f;
+    for (int j = 0; j < n_cand; ++j) l += expf(sc[j] - m);
+    part[(int64_t)b * (d_a + 1) + d_a] = -(sc[0] - m - logf(l));       // this user's loss
+    for (int j = 0; j < n_cand; ++j) sc[j] = (expf(sc[j] - m) / l - (j == 0 ? 1.f : 0.f)) * invB;   // ds
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.f;
+    for (int j = 0; j < n_cand; ++j) {
+      acc += sc[j] * ldf(Eb + (int64_t)(n_hist + j) * d + c);
+      dE[((int64_t)b * L + n_hist + j) * d + c] = sc[j] * u[c];          // gradient of the candidates
+    }
+    du[c] = acc;
+  }
+  __syncthreads();
+  for (int n = warp; n < n_hist; n += nwb) {     // d alpha_n = du . h_n
+    float acc = 0.f;
+    for (int c = lane; c < d; c += 32) acc += du[c] * ldf(Eb + (int64_t)n * d + c);
+    acc = warp_sum(acc);
+    if (lane == 0) da[n] = acc;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float s = 0.f;
+    for (int n = lane; n < n_hist; n += 32) s += a[n] * da[n];
+    s = warp_sum(s);
+    for (int n = lane; n < n_hist; n += 32) da[n] = a[n] * (da[n] - s);   // gradient of the scores a_n
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_hist * d; i += blockDim.x) {            // direct part of dh_n
+    const int n = i / d, c = i - n * d;
+    dE[((int64_t)b * L + n) * d + c] = a[n] * du[c];
+  }
+  for (int k = threadIdx.x; k < d_a; k += blockDim.x) {
+    float gq = 0.f;
+    for (int n = 0; n < L; ++n) {
+      float v = 0.f;
+      if (n < n_hist) {
+        const float t = tanhf(ldf(pb + (int64_t)n * d_a + k));
+        gq += da[n] * t;
+        v = da[n] * qa[k] * (1.f - t * t);
+      }
+      stf(dpre + ((int64_t)b * L + n) * d_a + k, v);
+    }
+    part[(int64_t)b * (d_a + 1) + k] = gq;
+  }
+}
+
+__global__ void nr_reduce_kernel(const float* __restrict__ part, int B, int d_a, float invB, float* __restrict__ dqa,
+                                 float* __restrict__ loss) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k > d_a) return;
+  float a = 0.f;
+  for (int b = 0; b < B; ++b) a += part[(int64_t)b * (d_a + 1) + k];
+  if (k < d_a) dqa[k] += a;
+  else loss[0] = a * invB;
+}
+
+// ---------------------------------------------------------------------------- element-wise
+__global__ void f32_to_bf16_kernel(const float* __restrict__ in, bf16* __restrict__ out, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    out[i] = __float2bfloat16(in[i]);
+}
+__global__ void bf16_to_f32_kernel(const bf16* __restrict__ in, float* __restrict__ out, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    out[i] = __bfloat162float(in[i]);
+}
+__global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float lr, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    w[i] -= lr * g[i];
+}
+template <typename T>
+__global__ void scatter_rows_kernel(const T* __restrict__ src, const int32_t* __restrict__ index, int64_t n, int d,
+                                    int64_t n_dst_rows, T* __restrict__ dst, int32_t* status) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * d) return;
+  const int64_t u = i / d;
+  const int c = (int)(i - u * d);
+  const int32_t r = index[u];
+  if (r < 0 || r >= n_dst_rows) { gram_device_fail(status, GRAM_ERR_ID_RANGE); return; }
+  dst[(int64_t)r * d + c] = src[i];
+}
+
+inline int grid_for(int64_t n, int threads, int cap) {
+  int64_t b = (n + threads - 1) / threads;
+  if (b > cap) b = cap;
+  if (b < 1) b = 1;
+  return (int)b;
+}
+
+template <typename F> gram_status set_smem(gram_ctx* ctx, F kern, size_t bytes) {
+  if (bytes > 227 * 1024) return gram_set_error(ctx, "a sequence is too long for the attention kernel's shared memory"), GRAM_ERR_UNSUPPORTED;
+  if (bytes > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  return GRAM_OK;
+}
+
+}  // namespace
+
+#define DISPATCH_T(dtype, ...)             \
+  if ((dtype) == GRAM_F32) { typedef float T; __VA_ARGS__; } else { typedef bf16 T; __VA_ARGS__; }
+
+#define DISPATCH_NP(d, ...)                                                    \
+  if ((d) <= 64) { constexpr int NP = 1; __VA_ARGS__; }                        \
+  else if ((d) <= 128) { constexpr int NP = 2; __VA_ARGS__; }                  \
+  else if ((d) <= 256) { constexpr int NP = 4; __VA_ARGS__; }                  \
+  else if ((d) <= 512) { constexpr int NP = 8; __VA_ARGS__; }                  \
+  else if ((d) <= 768) { constexpr int NP = 12; __VA_ARGS__; }                 \
+  else { constexpr int NP = 16; __VA_ARGS__; }
+
+gram_status embed_forward(gram_ctx* ctx, int dtype, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
+                          int32_t n_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
+                          const float* pos_emb, void* z0, int32_t* tok_ids, cudaStream_t st) {
+  const int64_t n_tok = (int64_t)n_chunk * l_t;
+  if (n_tok == 0) return GRAM_OK;
+  const int blocks = grid_for(n_tok * 32, 256, kNumSMs * 8);
+  DISPATCH_T(dtype, embed_fwd_kernel<T><<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t,
+                                                               vocab, d, tok_emb, pos_emb, (T*)z0, tok_ids,
+                                                               gram_status_word(ctx)));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status layernorm_forward(gram_ctx* ctx, int dtype, const void* z, const float* gamma, const float* beta, void* y,
+                              float* mean, float* rstd, int64_t rows, int d, cudaStream_t st) {
+  if (rows == 0) return GRAM_OK;
+  if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
+  const int blocks = grid_for(rows * 32, 256, kNumSMs * 8);
+  DISPATCH_T(dtype, DISPATCH_NP(d, ln_fwd_kernel<T, NP><<<blocks, 256, 0, st>>>((const T*)z, gamma, beta, (T*)y, mean, rstd, rows, d)));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status layernorm_backward(gram_ctx* ctx, int dtype, const void* dy, const void* z, const float* mean,
+                               const float* rstd, const float* gamma, void* dz, float* dgamma, float* dbeta,
+                               float* scratch, int64_t rows, int d, cudaStream_t st) {
+  if (rows == 0) return GRAM_OK;
+  if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
+  const int blocks = grid_for(rows * 32, 256, kRedBlocks);
+  const size_t smem = (size_t)2 * d * sizeof(float);
+  DISPATCH_T(dtype, DISPATCH_NP(d, ln_bwd_kernel<T, NP><<<blocks, 256, smem, st>>>((const T*)dy, (const T*)z, mean, rstd, gamma, (T*)dz, scratch, rows, d)));
+  reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
+                              int n_heads, int causal, cudaStream_t st) {
+  if (n_seq == 0) return GRAM_OK;
+  const int dh = d / n_heads;
+  if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
+  const float scale = 1.f / sqrtf((float)dh);
+  DISPATCH_T(dtype, {
+    GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
+    attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale);
+  });
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq,
+                               int S, int d, int n_heads, int causal, cudaStream_t st) {
+  if (n_seq == 0) return GRAM_OK;
+  const int dh = d / n_heads;
+  if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
+  const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
+  const float scale = 1.f / sqrtf((float)dh);
+  DISPATCH_T(dtype, {
+    GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
+    attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);
+  });
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t rows, int N, float* out, float* scratch,
+                              cudaStream_t st) {
+  if (rows == 0 || N == 0) return GRAM_OK;
+  if (N & 1) return gram_set_error(ctx, "column sum: N must be even"), GRAM_ERR_UNSUPPORTED;
+  int64_t rb = ceil_div64(rows, 64);
+  const int64_t cap = (int64_t)(kRedScratchBytes / sizeof(float)) / N;
+  if (rb > 256) rb = 256;
+  if (rb > cap) rb = cap;
+  const int64_t per = ceil_div64(rows, rb);
+  rb = ceil_div64(rows, per);
+  dim3 grid((unsigned)ceil_div(N, 64), (unsigned)rb);
+  DISPATCH_T(dtype, colsum_kernel<T><<<grid, 256, 0, st>>>((const T*)X, rows, N, per, scratch));
+  reduce_partials_kernel<<<ceil_div(N, 256), 256, 0, st>>>(scratch, (int)rb, (int64_t)N, N, out, nullptr, 1.f);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status periodic_rowsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t n_groups, int period, int d,
+                                       float* out, cudaStream_t st) {
+  if (n_groups == 0) return GRAM_OK;
+  const int64_t n = (int64_t)period * d;
+  DISPATCH_T(dtype, periodic_rowsum_kernel<T><<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>((const T*)X, n_groups, period, d, out));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status pool_forward(gram_ctx* ctx, int dtype, const void* x, void* H, int64_t n, int l_t, int d, int pooling,
+                         cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  DISPATCH_T(dtype, pool_fwd_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>((const T*)x, (T*)H, n, l_t, d, pooling));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status pool_backward(gram_ctx* ctx, int dtype, const float* G, void* dx, int64_t n, int l_t, int d, int pooling,
+                          cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  DISPATCH_T(dtype, pool_bwd_kernel<T><<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, (T*)dx, n, l_t, d, pooling));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status kt_input_forward(gram_ctx* ctx, int dtype, const void* E, const float* pos, const float* resp,
+                             const int32_t* labels, void* x, int B, int L, int d, cudaStream_t st) {
+  const int64_t P = (int64_t)B * L;
+  if (P == 0) return GRAM_OK;
+  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)ceil_div64(P * d, 256), 256, 0, st>>>((const T*)E, pos, resp, labels, (T*)x, P, L, d));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status kt_head(gram_ctx* ctx, int dtype, const void* y, const float* w, const float* b, const int32_t* labels,
+                    void* dy, float* dw, float* db, float* loss, float* scratch, int64_t P, int d, cudaStream_t st) {
+  if (P == 0) return GRAM_OK;
+  int blocks = (int)ceil_div64(P, 64);
+  if (blocks > kRedBlocks) blocks = kRedBlocks;
+  const int64_t pstride = d + 2;
+  const size_t smem = (size_t)(d + 2) * sizeof(float);
+  DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>((const T*)y, w, b, labels, (T*)dy, scratch, P, d, pstride));
+  kt_head_reduce_kernel<<<ceil_div(d + 2, 256), 256, 0, st>>>(scratch, blocks, pstride, d, 1.f / (float)P, dw, db, loss);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+// dE = dx, dpos += column sums over b, dresp += sums by previous response; scratch holds [L][3][d]
+gram_status kt_input_backward(gram_ctx* ctx, int dtype, const void* dx, const int32_t* labels, float* dE, float* dpos,
+                                 float* dresp, float* scratch, int B, int L, int d, cudaStream_t st) {
+  if (B == 0) return GRAM_OK;
+  if ((size_t)L * 3 * d * sizeof(float) > kRedScratchBytes) return gram_set_error(ctx, "kt task: L*d too large for the reduction scratch"), GRAM_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)ceil_div(d, 128), (unsigned)L);
+  DISPATCH_T(dtype, kt_input_bwd_kernel<T><<<grid, 128, 0, st>>>((const T*)dx, labels, dE, dpos, scratch, B, L, d));
+  reduce_partials_kernel<<<ceil_div(3 * d, 256), 256, 0, st>>>(scratch, L, (int64_t)3 * d, 3 * d, dresp, nullptr, 1.f);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status nr_user(gram_ctx* ctx, int dtype, const void* E, const void* pre, const float* qa, float* dE,
+                           void* dpre, float* dqa, float* loss, float* scratch, int B, int L, int n_cand, int d, int d_a,
+                           cudaStream_t st) {
+  if (B == 0) return GRAM_OK;
+  if (n_cand <= 0 || n_cand >= L) return gram_set_error(ctx, "nr task: need 0 < n_cand < L"), GRAM_ERR_ARG;
+  const size_t smem = ((size_t)2 * L + 2 * d + n_cand) * sizeof(float);
+  DISPATCH_T(dtype, {
+    GRAM_TRY(set_smem(ctx, nr_user_kernel<T>, smem));
+    nr_user_kernel<T><<<B, 256, smem, st>>>((const T*)E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B);
+  });
+  nr_reduce_kernel<<<ceil_div(d_a + 1, 256), 256, 0, st>>>(scratch, B, d_a, 1.f / (float)B, dqa, loss);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  f32_to_bf16_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(in, out, n);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if (dtype == GRAM_F32) GRAM_CUDA(ctx, cudaMemcpyAsync(out, in, n * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  else bf16_to_f32_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>((const bf16*)in, out, n);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st) {
+  if (n == 0 || lr == 0.f) return GRAM_OK;
+  sgd_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(w, g, lr, n);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status scatter_rows(gram_ctx* ctx, int dtype, const void* src, const int32_t* index, int64_t n, int d,
+                         int64_t n_dst_rows, void* dst, cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  DISPATCH_T(dtype, scatter_rows_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>((const T*)src, index, n, d, n_dst_rows, (T*)dst, gram_status_word(ctx)));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}

@@ -1,0 +1,722 @@
+// The two modules (content encoder CE, task module CF) and the training step that ties the five
+// stages together (Algorithm 1): parameter layout, activation arenas, forward and backward passes
+// composed from gemm.cu / layers.cu / the index kernels, Single-step and Multi-step drivers.
+#include <new>
+#include <vector>
+
+#include "gemm.h"
+#include "layers.h"
+#include "model.h"
+
+namespace {
+
+struct LayerOff {
+  size_t wqkv, bqkv, wo, bo, ln1g, ln1b, w1, b1, w2, b2, ln2g, ln2b;
+};
+
+struct Module {
+  size_t n = 0;
+  float* w = nullptr;      // fp32 parameters
+  float* g = nullptr;      // fp32 gradients
+  bf16* wb = nullptr;      // bf16 copy of the parameters (bf16 contexts), refreshed when stale
+  bool wb_stale = true;
+};
+
+struct LayerActs {
+  void *qkv, *ctx, *z1, *h1, *u, *g, *z2, *out;
+  float *mean1, *rstd1, *mean2, *rstd2;
+};
+
+// a run of post-LayerNorm transformer layers over sequences of S tokens
+struct Stack {
+  int d = 0, heads = 0, d_ff = 0, n_layers = 0, attn_only = 0, causal = 0;
+  int64_t cap = 0;                         // tokens the buffers hold
+  std::vector<LayerOff> off;
+  std::vector<LayerActs> acts;
+  void *dA = nullptr, *dB = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;   // backward scratch
+};
+
+struct Arena {
+  char* base = nullptr;
+  size_t off = 0;
+  void* take(size_t bytes) {
+    off = (off + 255) & ~(size_t)255;
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+size_t layer_layout(LayerOff* o, size_t at, int d, int d_ff, int attn_only) {
+  o->wqkv = at; at += (size_t)3 * d * d;
+  o->bqkv = at; at += (size_t)3 * d;
+  o->wo = at; at += (size_t)d * d;
+  o->bo = at; at += d;
+  if (!attn_only) {
+    o->ln1g = at; at += d;
+    o->ln1b = at; at += d;
+    o->w1 = at; at += (size_t)d_ff * d;
+    o->b1 = at; at += d_ff;
+    o->w2 = at; at += (size_t)d * d_ff;
+    o->b2 = at; at += d;
+    o->ln2g = at; at += d;
+    o->ln2b = at; at += d;
+  }
+  return at;
+}
+
+}  // namespace
+
+struct Model {
+  gram_ctx* ctx = nullptr;
+  gram_config cfg;
+  int dtype = GRAM_F32;
+  size_t esz = 4;
+  Module ce, task;
+  // encoder
+  size_t o_tok = 0, o_pos = 0, o_elng = 0, o_elnb = 0;
+  Stack enc;
+  void *z0 = nullptr, *x0 = nullptr;
+  float *mean0 = nullptr, *rstd0 = nullptr;
+  int32_t *tok_ids = nullptr, *tok_unique = nullptr, *tok_inverse = nullptr, *tok_perm = nullptr, *tok_seg = nullptr,
+          *tok_nu = nullptr;
+  int32_t mb = 0;                    // items per encoder pass
+  int32_t saved_n = -1;              // items whose activations the last encoder pass saved (-1: none)
+  // task
+  size_t t_pos = 0, t_resp = 0, t_headw = 0, t_headb = 0, t_wa = 0, t_ba = 0, t_qa = 0;
+  Stack tk;
+  void *tx = nullptr, *pre = nullptr, *dpre = nullptr;
+  // step buffers
+  int32_t* item_tokens = nullptr;
+  int32_t *ids = nullptr, *labels = nullptr, *unique = nullptr, *inverse = nullptr, *perm = nullptr, *seg_off = nullptr,
+          *n_unique = nullptr;
+  int32_t u_cap = 0;
+  void *H = nullptr, *E = nullptr;
+  float *dE = nullptr, *G = nullptr, *loss = nullptr, *red = nullptr;
+  // Multi-step window
+  float* table = nullptr;
+  uint32_t* touched = nullptr;
+  void* cache = nullptr;
+  int32_t *tlist = nullptr, *tcount = nullptr;
+  int step_in_window = 0;
+  char* arena = nullptr;
+  size_t arena_bytes = 0;
+  cudaEvent_t ev[8] = {};
+  int32_t* h_pinned = nullptr;       // [4] pinned host words for small read-backs
+};
+
+namespace {
+
+void stack_buffers(Arena& a, Stack& s, size_t esz) {
+  s.acts.resize(s.n_layers);
+  const size_t T = (size_t)s.cap, d = s.d, f = s.d_ff;
+  for (int l = 0; l < s.n_layers; ++l) {
+    LayerActs& x = s.acts[l];
+    x.qkv = a.take(T * 3 * d * esz);
+    x.ctx = a.take(T * d * esz);
+    x.out = a.take(T * d * esz);
+    if (!s.attn_only) {
+      x.z1 = a.take(T * d * esz);
+      x.h1 = a.take(T * d * esz);
+      x.u = a.take(T * f * esz);
+      x.g = a.take(T * f * esz);
+      x.z2 = a.take(T * d * esz);
+      x.mean1 = (float*)a.take(T * 4);
+      x.rstd1 = (float*)a.take(T * 4);
+      x.mean2 = (float*)a.take(T * 4);
+      x.rstd2 = (float*)a.take(T * 4);
+    }
+  }
+  s.dA = a.take(T * d * esz);
+  s.dB = a.take(T * d * esz);
+  s.dqkv = a.take(T * 3 * d * esz);
+  s.dctx = a.take(T * d * esz);
+  s.du = s.attn_only ? nullptr : a.take(T * f * esz);
+}
+
+void layout_buffers(Model* m, Arena& a) {
+  const gram_config& c = m->cfg;
+  const size_t esz = m->esz, d = c.d;
+  const int64_t P = (int64_t)c.B_max * c.L;
+  if (c.n_layers > 0) {
+    const size_t T = (size_t)m->mb * c.l_t;
+    m->z0 = a.take(T * d * esz);
+    m->x0 = a.take(T * d * esz);
+    m->mean0 = (float*)a.take(T * 4);
+    m->rstd0 = (float*)a.take(T * 4);
+    m->tok_ids = (int32_t*)a.take(T * 4);
+    const size_t tu = T < (size_t)c.vocab ? T : (size_t)c.vocab;
+    m->tok_unique = (int32_t*)a.take(tu * 4);
+    m->tok_inverse = (int32_t*)a.take(T * 4);
+    m->tok_perm = (int32_t*)a.take(T * 4);
+    m->tok_seg = (int32_t*)a.take((tu + 1) * 4);
+    m->tok_nu = (int32_t*)a.take(4);
+    stack_buffers(a, m->enc, esz);
+    m->item_tokens = (int32_t*)a.take((size_t)c.n_items * c.l_t * 4);
+  }
+  if (c.task != GRAM_TASK_NONE) {
+    if (c.task == GRAM_TASK_KT) {
+      m->tx = a.take((size_t)P * d * esz);
+      stack_buffers(a, m->tk, esz);
+    } else {
+      m->pre = a.take((size_t)P * c.d_a * esz);
+      m->dpre = a.take((size_t)P * c.d_a * esz);
+    }
+  }
+  m->ids = (int32_t*)a.take((size_t)P * 4);
+  m->labels = (int32_t*)a.take((size_t)P * 4);
+  m->unique = (int32_t*)a.take((size_t)m->u_cap * 4);
+  m->inverse = (int32_t*)a.take((size_t)P * 4);
+  m->perm = (int32_t*)a.take((size_t)P * 4);
+  m->seg_off = (int32_t*)a.take(((size_t)m->u_cap + 1) * 4);
+  m->n_unique = (int32_t*)a.take(4);
+  const size_t hrows = (size_t)(m->u_cap > m->mb ? m->u_cap : m->mb);
+  m->H = a.take(hrows * d * esz);
+  m->G = (float*)a.take(hrows * d * 4);
+  m->E = a.take((size_t)P * d * esz);
+  m->dE = (float*)a.take((size_t)P * d * 4);
+  m->loss = (float*)a.take(4);
+  m->red = (float*)a.take(kRedScratchBytes);
+  if (c.K > 1) {
+    m->table = (float*)a.take((size_t)c.n_items * d * 4);
+    m->touched = (uint32_t*)a.take((size_t)((c.n_items + 31) / 32) * 4);
+    m->cache = a.take((size_t)c.n_items * d * esz);
+    m->tlist = (int32_t*)a.take((size_t)c.n_items * 4);
+    m->tcount = (int32_t*)a.take(4);
+  }
+}
+
+gram_status module_alloc(gram_ctx* ctx, Module* mod, size_t n, bool want_bf16) {
+  mod->n = n;
+  if (n == 0) return GRAM_OK;
+  GRAM_CUDA(ctx, cudaMalloc(&mod->w, n * 4));
+  GRAM_CUDA(ctx, cudaMalloc(&mod->g, n * 4));
+  GRAM_CUDA(ctx, cudaMemset(mod->w, 0, n * 4));
+  GRAM_CUDA(ctx, cudaMemset(mod->g, 0, n * 4));
+  if (want_bf16) GRAM_CUDA(ctx, cudaMalloc(&mod->wb, n * 2));
+  mod->wb_stale = true;
+  return GRAM_OK;
+}
+
+gram_status refresh_bf16(Model* m, Module& mod, cudaStream_t st) {
+  if (m->dtype == GRAM_BF16 && mod.wb_stale && mod.n) {
+    GRAM_TRY(convert_f32_to_bf16(m->ctx, mod.w, mod.wb, mod.n, st));
+    mod.wb_stale = false;
+  }
+  return GRAM_OK;
+}
+
+// the weight matrix at `off` in the element type the matrix products take
+inline const void* W(const Model* m, const Module& mod, size_t off) {
+  return m->dtype == GRAM_BF16 ? (const void*)(mod.wb + off) : (const void*)(mod.w + off);
+}
+inline void* at(const Model* m, void* p, size_t elems) { return (char*)p + elems * m->esz; }
+
+// Y[T, N] = X[T, K] W[N, K]^T (+ epilogue), activations of type T
+gram_status mm_fwd(Model* m, const void* X, const void* Wt, void* Y, int64_t T, int N, int K, const GemmEpilogue& e,
+                   cudaStream_t st) {
+  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, X, 1, K, Wt, 1, K, Y, m->dtype == GRAM_F32, N, T, N, K, e, 0, st);
+}
+// dX[T, K] = dY[T, N] W[N, K] (+ epilogue)
+gram_status mm_dx(Model* m, const void* dY, const void* Wt, void* dX, int64_t T, int N, int K, const GemmEpilogue& e,
+                  cudaStream_t st) {
+  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 1, N, Wt, 0, K, dX, m->dtype == GRAM_F32, K, T, K, N, e, 0, st);
+}
+// dW[N, K] += dY[T, N]^T X[T, K]   (fp32 result, the token dimension may be split)
+gram_status mm_dw(Model* m, const void* dY, const void* X, float* dW, int64_t T, int N, int K, cudaStream_t st) {
+  GemmEpilogue e;
+  e.accumulate = 1;
+  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 0, N, X, 0, K, dW, 1, K, N, K, T, e, 1, st);
+}
+
+gram_status stack_forward(Model* m, Module& mod, Stack& s, const void* x_in, int64_t n_seq, int S, cudaStream_t st,
+                          const void** out) {
+  const int64_t T = n_seq * S;
+  const int d = s.d, f = s.d_ff;
+  gram_ctx* ctx = m->ctx;
+  const void* x = x_in;
+  for (int l = 0; l < s.n_layers; ++l) {
+    const LayerOff& o = s.off[l];
+    LayerActs& a = s.acts[l];
+    GemmEpilogue e;
+    e.bias = mod.w + o.bqkv;
+    GRAM_TRY(mm_fwd(m, x, W(m, mod, o.wqkv), a.qkv, T, 3 * d, d, e, st));
+    GRAM_TRY(attention_forward(ctx, m->dtype, a.qkv, a.ctx, n_seq, S, d, s.heads, s.causal, st));
+    e = GemmEpilogue();
+    e.bias = mod.w + o.bo;
+    e.residual = x;
+    if (s.attn_only) {
+      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.out, T, d, d, e, st));
+    } else {
+      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.z1, T, d, d, e, st));
+      GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z1, mod.w + o.ln1g, mod.w + o.ln1b, a.h1, a.mean1, a.rstd1, T, d, st));
+      e = GemmEpilogue();
+      e.bias = mod.w + o.b1;
+      e.gelu = 1;
+      e.pre = a.u;
+      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, T, f, d, e, st));
+      e = GemmEpilogue();
+      e.bias = mod.w + o.b2;
+      e.residual = a.h1;
+      GRAM_TRY(mm_fwd(m, a.g, W(m, mod, o.w2), a.z2, T, d, f, e, st));
+      GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z2, mod.w + o.ln2g, mod.w + o.ln2b, a.out, a.mean2, a.rstd2, T, d, st));
+    }
+    x = a.out;
+  }
+  *out = x;
+  return GRAM_OK;
+}
+
+// the incoming gradient (with respect to the stack's output) is in s.dA; *d_in points at the
+// gradient with respect to x_in when this returns
+gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in, int64_t n_seq, int S, cudaStream_t st,
+                           void** d_in) {
+  const int64_t T = n_seq * S;
+  const int d = s.d, f = s.d_ff;
+  gram_ctx* ctx = m->ctx;
+  float* red = m->red;
+  void* cur = s.dA;
+  void* oth = s.dB;
+  for (int l = s.n_layers - 1; l >= 0; --l) {
+    const LayerOff& o = s.off[l];
+    LayerActs& a = s.acts[l];
+    const void* x_l = (l == 0) ? x_in : s.acts[l - 1].out;
+    GemmEpilogue e;
+    if (!s.attn_only) {
+      // out = LN2(z2), z2 = h1 + W2 gelu(u) + b2, u = W1 h1 + b1, h1 = LN1(z1), z1 = x + Wo ctx + bo
+      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, mod.g + o.ln2g,
+                                  mod.g + o.ln2b, red, T, d, st));                       // oth = dz2
+      GRAM_TRY(colsum_accumulate(ctx, m->dtype, oth, T, d, mod.g + o.b2, red, st));
+      GRAM_TRY(mm_dw(m, oth, a.g, mod.g + o.w2, T, d, f, st));
+      e = GemmEpilogue();
+      e.dgelu_pre = a.u;
+      GRAM_TRY(mm_dx(m, oth, W(m, mod, o.w2), s.du, T, d, f, e, st));                    // du = (dz2 W2) * gelu'(u)
+      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
+      GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st));
+      e = GemmEpilogue();
+      e.residual = oth;
+      GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, T, f, d, e, st));                    // cur = dh1 = du W1 + dz2
+      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, mod.g + o.ln1g,
+                                  mod.g + o.ln1b, red, T, d, st));                       // oth = dz1
+    } else {
+      void* t = cur; cur = oth; oth = t;                                                 // oth = d(out)
+    }
+    GRAM_TRY(colsum_accumulate(ctx, m->dtype, oth, T, d, mod.g + o.bo, red, st));
+    GRAM_TRY(mm_dw(m, oth, a.ctx, mod.g + o.wo, T, d, d, st));
+    e = GemmEpilogue();
+    GRAM_TRY(mm_dx(m, oth, W(m, mod, o.wo), s.dctx, T, d, d, e, st));
+    GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, n_seq, S, d, s.heads, s.causal, st));
+    GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
+    GRAM_TRY(mm_dw(m, s.dqkv, x_l, mod.g + o.wqkv, T, 3 * d, d, st));
+    e = GemmEpilogue();
+    e.residual = oth;
+    GRAM_TRY(mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, T, 3 * d, d, e, st));              // cur = dx = dqkv Wqkv + dz1
+  }
+  *d_in = cur;
+  return GRAM_OK;
+}
+
+// encoder forward over n items (d_items, or first_item.. when null): H_out [n, d] of type T
+gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t first_item,
+                                  int32_t n, void* H_out, cudaStream_t st) {
+  const gram_config& c = m->cfg;
+  gram_ctx* ctx = m->ctx;
+  if (n > m->mb) return gram_set_error(ctx, "encoder pass over %d items exceeds the micro-batch of %d", n, m->mb), GRAM_ERR_WORKSPACE;
+  GRAM_TRY(refresh_bf16(m, m->ce, st));
+  const int64_t T = (int64_t)n * c.l_t;
+  GRAM_TRY(embed_forward(ctx, m->dtype, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items,
+                         c.l_t, c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, st));
+  GRAM_TRY(layernorm_forward(ctx, m->dtype, m->z0, m->ce.w + m->o_elng, m->ce.w + m->o_elnb, m->x0, m->mean0, m->rstd0, T,
+                             c.d, st));
+  const void* out = nullptr;
+  GRAM_TRY(stack_forward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &out));
+  GRAM_TRY(pool_forward(ctx, m->dtype, out, H_out, n, c.l_t, c.d, c.pooling, st));
+  m->saved_n = n;
+  return GRAM_OK;
+}
+
+// encoder parameter gradients += VJP of the last encoder_forward_chunk with cotangent G [n, d] (fp32)
+gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStream_t st) {
+  const gram_config& c = m->cfg;
+  gram_ctx* ctx = m->ctx;
+  if (n != m->saved_n) return gram_set_error(ctx, "encoder backward over %d items, but activations of %d are saved", n, m->saved_n), GRAM_ERR_ARG;
+  const int64_t T = (int64_t)n * c.l_t;
+  GRAM_TRY(pool_backward(ctx, m->dtype, G, m->enc.dA, n, c.l_t, c.d, c.pooling, st));
+  void* dx0 = nullptr;
+  GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
+  void* dz0 = (dx0 == m->enc.dA) ? m->enc.dB : m->enc.dA;
+  GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, m->ce.g + m->o_elng,
+                              m->ce.g + m->o_elnb, m->red, T, c.d, st));
+  GRAM_TRY(periodic_rowsum_accumulate(ctx, m->dtype, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, st));
+  // token-embedding gradient: sum dz0 over the occurrences of each token (same index kernels as stage 1 / 4)
+  IndexWorkspace* iws = gram_index_ws(ctx);
+  GRAM_TRY(dedup_launch(ctx, iws, m->tok_ids, T, c.vocab, m->tok_unique, m->tok_inverse, m->tok_perm, m->tok_seg, m->tok_nu, st));
+  GRAM_TRY(accumulate_launch(ctx, iws, dz0, m->dtype == GRAM_BF16, m->tok_perm, m->tok_seg, T, 0, m->tok_nu, c.d,
+                             m->tok_unique, 1, m->ce.g + m->o_tok, st));
+  return GRAM_OK;
+}
+
+gram_status task_forward_backward(Model* m, const void* E, const int32_t* labels, int32_t B, float* dE, float* loss,
+                                  cudaStream_t st) {
+  const gram_config& c = m->cfg;
+  gram_ctx* ctx = m->ctx;
+  const int64_t P = (int64_t)B * c.L;
+  GRAM_TRY(refresh_bf16(m, m->task, st));
+  GRAM_CUDA(ctx, cudaMemsetAsync(m->task.g, 0, m->task.n * 4, st));
+  if (c.task == GRAM_TASK_KT) {
+    GRAM_TRY(kt_input_forward(ctx, m->dtype, E, m->task.w + m->t_pos, m->task.w + m->t_resp, labels, m->tx, B, c.L, c.d, st));
+    const void* y = nullptr;
+    GRAM_TRY(stack_forward(m, m->task, m->tk, m->tx, B, c.L, st, &y));
+    GRAM_TRY(kt_head(ctx, m->dtype, y, m->task.w + m->t_headw, m->task.w + m->t_headb, labels, m->tk.dA,
+                     m->task.g + m->t_headw, m->task.g + m->t_headb, loss, m->red, P, c.d, st));
+    void* dx = nullptr;
+    GRAM_TRY(stack_backward(m, m->task, m->tk, m->tx, B, c.L, st, &dx));
+    GRAM_TRY(kt_input_backward(ctx, m->dtype, dx, labels, dE, m->task.g + m->t_pos, m->task.g + m->t_resp, m->red, B, c.L,
+                               c.d, st));
+    return GRAM_OK;
+  }
+  if (c.task == GRAM_TASK_NR) {
+    GemmEpilogue e;
+    e.bias = m->task.w + m->t_ba;
+    GRAM_TRY(mm_fwd(m, E, W(m, m->task, m->t_wa), m->pre, P, c.d_a, c.d, e, st));
+    GRAM_TRY(nr_user(ctx, m->dtype, E, m->pre, m->task.w + m->t_qa, dE, m->dpre, m->task.g + m->t_qa, loss, m->red, B, c.L,
+                     c.n_cand, c.d, c.d_a, st));
+    GRAM_TRY(colsum_accumulate(ctx, m->dtype, m->dpre, P, c.d_a, m->task.g + m->t_ba, m->red, st));
+    GRAM_TRY(mm_dw(m, m->dpre, E, m->task.g + m->t_wa, P, c.d_a, c.d, st));
+    e = GemmEpilogue();
+    e.accumulate = 1;                    // dE already holds the direct part
+    GRAM_TRY(gemm_launch(ctx, gram_gemm_ws(ctx), m->dtype, m->dpre, 1, c.d_a, W(m, m->task, m->t_wa), 0, c.d, dE, 1, c.d, P,
+                         c.d, c.d_a, e, 0, st));
+    return GRAM_OK;
+  }
+  return gram_set_error(ctx, "the context has no task module"), GRAM_ERR_ARG;
+}
+
+gram_status read_i32(Model* m, const int32_t* d_ptr, int32_t* out, cudaStream_t st) {
+  GRAM_CUDA(m->ctx, cudaMemcpyAsync(m->h_pinned, d_ptr, 4, cudaMemcpyDeviceToHost, st));
+  GRAM_CUDA(m->ctx, cudaStreamSynchronize(st));
+  *out = m->h_pinned[0];
+  return GRAM_OK;
+}
+
+gram_status apply_sgd(Model* m, Module& mod, float lr, cudaStream_t st) {
+  if (lr == 0.f || mod.n == 0) return GRAM_OK;
+  GRAM_TRY(sgd_update(m->ctx, mod.w, mod.g, lr, mod.n, st));
+  mod.wb_stale = true;
+  return GRAM_OK;
+}
+
+// encoder forward + backward over `n_total` items listed in d_items, in micro-batches; G_of(u0, n)
+// must leave the cotangent rows of items [u0, u0+n) in m->G
+template <typename GFn>
+gram_status encoder_pass(Model* m, const int32_t* d_items, int32_t n_total, bool update_cache, GFn G_of, cudaStream_t st) {
+  for (int32_t u0 = 0; u0 < n_total; u0 += m->mb) {
+    const int32_t n = (n_total - u0 < m->mb) ? n_total - u0 : m->mb;
+    GRAM_TRY(encoder_forward_chunk(m, nullptr, d_items + u0, 0, n, m->H, st));
+    if (update_cache) GRAM_TRY(scatter_rows(m->ctx, m->dtype, m->H, d_items + u0, n, m->cfg.d, m->cfg.n_items, m->cache, st));
+    const float* G = nullptr;
+    GRAM_TRY(G_of(u0, n, &G));
+    GRAM_TRY(encoder_backward_chunk(m, G, n, st));
+  }
+  return GRAM_OK;
+}
+
+}  // namespace
+
+// ===========================================================================================
+gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
+  *out = nullptr;
+  Model* m = new (std::nothrow) Model();
+  if (!m) return GRAM_ERR_CUDA;
+  *out = m;                             // destroyed by the caller on failure
+  m->ctx = ctx;
+  m->cfg = *cfg;
+  const gram_config& c = m->cfg;
+  m->dtype = c.dtype;
+  if (c.dtype != GRAM_F32 && c.dtype != GRAM_BF16) return gram_set_error(ctx, "unknown dtype %d", c.dtype), GRAM_ERR_ARG;
+  m->esz = c.dtype == GRAM_BF16 ? 2 : 4;
+  if (c.d <= 0 || (c.d & 1)) return gram_set_error(ctx, "d must be positive and even"), GRAM_ERR_ARG;
+  if (c.dtype == GRAM_BF16 && (c.d % 8 || c.d_ff % 8 || c.task_d_ff % 8 || c.d_a % 8))
+    return gram_set_error(ctx, "bf16 contexts need widths that are multiples of 8"), GRAM_ERR_UNSUPPORTED;
+  if (c.B_max <= 0 || c.L <= 0) return gram_set_error(ctx, "B_max and L must be positive"), GRAM_ERR_ARG;
+  // ---- parameter layouts (the order include/gram.h documents) ----
+  size_t at = 0;
+  if (c.n_layers > 0) {
+    if (c.n_heads <= 0 || c.d % c.n_heads || c.l_t <= 0 || c.vocab <= 0 || c.d_ff <= 0)
+      return gram_set_error(ctx, "bad encoder shape"), GRAM_ERR_ARG;
+    m->o_tok = at; at += (size_t)c.vocab * c.d;
+    m->o_pos = at; at += (size_t)c.l_t * c.d;
+    m->o_elng = at; at += c.d;
+    m->o_elnb = at; at += c.d;
+    m->enc.d = c.d; m->enc.heads = c.n_heads; m->enc.d_ff = c.d_ff; m->enc.n_layers = c.n_layers;
+    m->enc.attn_only = 0; m->enc.causal = 0;
+    m->enc.off.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) at = layer_layout(&m->enc.off[l], at, c.d, c.d_ff, 0);
+  }
+  GRAM_TRY(module_alloc(ctx, &m->ce, at, c.dtype == GRAM_BF16));
+  at = 0;
+  if (c.task == GRAM_TASK_KT) {
+    if (c.task_layers > 0 && (c.task_heads <= 0 || c.d % c.task_heads)) return gram_set_error(ctx, "bad task shape"), GRAM_ERR_ARG;
+    m->t_pos = at; at += (size_t)c.L * c.d;
+    m->t_resp = at; at += (size_t)3 * c.d;
+    m->tk.d = c.d; m->tk.heads = c.task_heads; m->tk.d_ff = c.task_d_ff; m->tk.n_layers = c.task_layers;
+    m->tk.attn_only = c.task_attn_only ? 1 : 0; m->tk.causal = 1;
+    m->tk.off.resize(c.task_layers);
+    for (int l = 0; l < c.task_layers; ++l) at = layer_layout(&m->tk.off[l], at, c.d, c.task_d_ff, m->tk.attn_only);
+    m->t_headw = at; at += c.d;
+    m->t_headb = at; at += 1;
+  } else if (c.task == GRAM_TASK_NR) {
+    if (c.d_a <= 0 || c.n_cand <= 0 || c.n_cand >= c.L) return gram_set_error(ctx, "bad task shape"), GRAM_ERR_ARG;
+    m->t_wa = at; at += (size_t)c.d_a * c.d;
+    m->t_ba = at; at += c.d_a;
+    m->t_qa = at; at += c.d_a;
+  }
+  GRAM_TRY(module_alloc(ctx, &m->task, at, c.dtype == GRAM_BF16));
+  // ---- sizes ----
+  const int64_t P = (int64_t)c.B_max * c.L;
+  m->u_cap = (int32_t)(P < c.n_items ? P : c.n_items);
+  int64_t mb = c.ce_micro_batch > 0 ? c.ce_micro_batch : (c.K > 1 ? c.n_items : m->u_cap);
+  if (mb > c.n_items) mb = c.n_items;
+  m->mb = (int32_t)mb;
+  m->enc.cap = (int64_t)m->mb * c.l_t;
+  m->tk.cap = P;
+  Arena dry;
+  layout_buffers(m, dry);
+  m->arena_bytes = dry.off + 256;
+  GRAM_CUDA(ctx, cudaMalloc(&m->arena, m->arena_bytes));
+  GRAM_CUDA(ctx, cudaMemset(m->arena, 0, m->arena_bytes));
+  Arena real;
+  real.base = m->arena;
+  layout_buffers(m, real);
+  for (int i = 0; i < 8; ++i) GRAM_CUDA(ctx, cudaEventCreate(&m->ev[i]));
+  GRAM_CUDA(ctx, cudaMallocHost(&m->h_pinned, 16));
+  return GRAM_OK;
+}
+
+void model_destroy(Model* m) {
+  if (!m) return;
+  cudaFree(m->ce.w); cudaFree(m->ce.g); cudaFree(m->ce.wb);
+  cudaFree(m->task.w); cudaFree(m->task.g); cudaFree(m->task.wb);
+  cudaFree(m->arena);
+  for (int i = 0; i < 8; ++i) if (m->ev[i]) cudaEventDestroy(m->ev[i]);
+  if (m->h_pinned) cudaFreeHost(m->h_pinned);
+  delete m;
+}
+
+static Module* pick(Model* m, int module) {
+  return module == GRAM_MODULE_CE ? &m->ce : (module == GRAM_MODULE_TASK ? &m->task : nullptr);
+}
+
+gram_status model_param_count(const Model* m, int module, size_t* n) {
+  const Module* mod = pick(const_cast<Model*>(m), module);
+  if (!mod) return GRAM_ERR_ARG;
+  *n = mod->n;
+  return GRAM_OK;
+}
+
+gram_status model_set_params(Model* m, int module, const float* h, size_t n) {
+  Module* mod = pick(m, module);
+  if (!mod || !h || n != mod->n) return gram_set_error(m->ctx, "gram_set_params: module or count mismatch (%zu given)", n), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  GRAM_CUDA(m->ctx, cudaMemcpy(mod->w, h, n * 4, cudaMemcpyHostToDevice));
+  mod->wb_stale = true;
+  m->saved_n = -1;
+  return GRAM_OK;
+}
+
+gram_status model_get_params(Model* m, int module, float* h, size_t n, int grads) {
+  Module* mod = pick(m, module);
+  if (!mod || !h || n != mod->n) return gram_set_error(m->ctx, "gram_get_params/grads: module or count mismatch"), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  GRAM_CUDA(m->ctx, cudaMemcpy(h, grads ? mod->g : mod->w, n * 4, cudaMemcpyDeviceToHost));
+  return GRAM_OK;
+}
+
+gram_status model_zero_grads(Model* m, int module, cudaStream_t st) {
+  Module* mod = pick(m, module);
+  if (!mod) return GRAM_ERR_ARG;
+  if (mod->n) GRAM_CUDA(m->ctx, cudaMemsetAsync(mod->g, 0, mod->n * 4, st));
+  return GRAM_OK;
+}
+
+gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens) {
+  if (!h_tokens || !m->item_tokens) return gram_set_error(m->ctx, "gram_set_item_tokens: no encoder or null tokens"), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  GRAM_CUDA(m->ctx, cudaMemcpy(m->item_tokens, h_tokens, (size_t)m->cfg.n_items * m->cfg.l_t * 4, cudaMemcpyHostToDevice));
+  return GRAM_OK;
+}
+
+gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, void* d_H, int save,
+                         cudaStream_t st) {
+  if (m->cfg.n_layers <= 0) return gram_set_error(m->ctx, "the context has no encoder"), GRAM_ERR_ARG;
+  if (U < 0 || (U > 0 && (!d_items || !d_H))) return gram_set_error(m->ctx, "gram_encode_unique: bad argument"), GRAM_ERR_ARG;
+  if (save && U > m->mb)
+    return gram_set_error(m->ctx, "gram_encode_unique: %d items do not fit the micro-batch of %d when activations are kept", U, m->mb), GRAM_ERR_WORKSPACE;
+  for (int32_t u0 = 0; u0 < U; u0 += m->mb) {
+    const int32_t n = (U - u0 < m->mb) ? U - u0 : m->mb;
+    GRAM_TRY(encoder_forward_chunk(m, d_item_tokens, d_items + u0, 0, n, (char*)d_H + (size_t)u0 * m->cfg.d * m->esz, st));
+  }
+  if (!save || U == 0) m->saved_n = save ? 0 : -1;
+  return GRAM_OK;
+}
+
+gram_status model_task(Model* m, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
+                       cudaStream_t st) {
+  if (B < 0 || B > m->cfg.B_max) return gram_set_error(m->ctx, "gram_task: B=%d exceeds B_max=%d", B, m->cfg.B_max), GRAM_ERR_WORKSPACE;
+  if (B == 0) return GRAM_OK;
+  if (!d_E || !d_labels || !d_dE || !d_loss) return gram_set_error(m->ctx, "gram_task: null buffer"), GRAM_ERR_ARG;
+  return task_forward_backward(m, d_E, d_labels, B, d_dE, d_loss, st);
+}
+
+gram_status model_encoder_backward(Model* m, const float* d_G, const int32_t* d_items, int32_t U, cudaStream_t st) {
+  (void)d_items;
+  if (m->cfg.n_layers <= 0) return gram_set_error(m->ctx, "the context has no encoder"), GRAM_ERR_ARG;
+  if (U == 0) return GRAM_OK;
+  if (!d_G) return gram_set_error(m->ctx, "gram_encoder_backward: null buffer"), GRAM_ERR_ARG;
+  return encoder_backward_chunk(m, d_G, U, st);
+}
+
+float* model_table(Model* m) { return m->table; }
+uint32_t* model_touched(Model* m) { return m->touched; }
+
+gram_status model_window_reset(Model* m, cudaStream_t st) {
+  if (!m->table) return gram_set_error(m->ctx, "the context was created with K <= 1"), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaMemsetAsync(m->table, 0, (size_t)m->cfg.n_items * m->cfg.d * 4, st));
+  GRAM_CUDA(m->ctx, cudaMemsetAsync(m->touched, 0, (size_t)((m->cfg.n_items + 31) / 32) * 4, st));
+  m->step_in_window = 0;
+  return GRAM_OK;
+}
+
+gram_status model_cache_fill(Model* m, cudaStream_t st) {
+  if (!m->cache) return gram_set_error(m->ctx, "the context was created with K <= 1"), GRAM_ERR_ARG;
+  const gram_config& c = m->cfg;
+  for (int32_t u0 = 0; u0 < c.n_items; u0 += m->mb) {
+    const int32_t n = (c.n_items - u0 < m->mb) ? c.n_items - u0 : m->mb;
+    GRAM_TRY(encoder_forward_chunk(m, nullptr, nullptr, u0, n, (char*)m->cache + (size_t)u0 * c.d * m->esz, st));
+  }
+  m->saved_n = -1;
+  return GRAM_OK;
+}
+
+gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, float* h_cache) {
+  if (!m->table) return gram_set_error(m->ctx, "the context was created with K <= 1"), GRAM_ERR_ARG;
+  const gram_config& c = m->cfg;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  if (h_table) GRAM_CUDA(m->ctx, cudaMemcpy(h_table, m->table, (size_t)c.n_items * c.d * 4, cudaMemcpyDeviceToHost));
+  if (h_touched) GRAM_CUDA(m->ctx, cudaMemcpy(h_touched, m->touched, (size_t)((c.n_items + 31) / 32) * 4, cudaMemcpyDeviceToHost));
+  if (h_cache) {
+    // convert through the gradient buffer G is too small in general: stage through dE-sized chunks
+    const size_t rows_per = (size_t)((int64_t)c.B_max * c.L);
+    for (size_t r0 = 0; r0 < (size_t)c.n_items; r0 += rows_per) {
+      const size_t nr = ((size_t)c.n_items - r0 < rows_per) ? (size_t)c.n_items - r0 : rows_per;
+      GRAM_TRY(convert_to_f32(m->ctx, m->dtype, (char*)m->cache + r0 * c.d * m->esz, m->dE, nr * c.d, 0));
+      GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+      GRAM_CUDA(m->ctx, cudaMemcpy(h_cache + r0 * c.d, m->dE, nr * c.d * 4, cudaMemcpyDeviceToHost));
+    }
+  }
+  return GRAM_OK;
+}
+
+gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in, int32_t B, int on_host,
+                       gram_step_report* rep, cudaStream_t st) {
+  const gram_config& c = m->cfg;
+  gram_ctx* ctx = m->ctx;
+  if (c.n_layers <= 0 || c.task == GRAM_TASK_NONE) return gram_set_error(ctx, "gram_step needs both modules"), GRAM_ERR_ARG;
+  if (B <= 0 || B > c.B_max) return gram_set_error(ctx, "gram_step: B=%d outside 1..B_max=%d", B, c.B_max), GRAM_ERR_WORKSPACE;
+  if (!ids_in || !labels_in) return gram_set_error(ctx, "gram_step: null buffer"), GRAM_ERR_ARG;
+  const int64_t P = (int64_t)B * c.L;
+  const bool multi = c.K > 1;
+  cudaEvent_t* ev = m->ev;
+  GRAM_CUDA(ctx, cudaEventRecord(ev[0], st));
+  const int32_t* ids = ids_in;
+  const int32_t* labels = labels_in;
+  if (on_host) {
+    GRAM_CUDA(ctx, cudaMemcpyAsync(m->ids, ids_in, (size_t)P * 4, cudaMemcpyHostToDevice, st));
+    GRAM_CUDA(ctx, cudaMemcpyAsync(m->labels, labels_in, (size_t)P * 4, cudaMemcpyHostToDevice, st));
+    ids = m->ids;
+    labels = m->labels;
+  }
+  // stage 1
+  IndexWorkspace* iws = gram_index_ws(ctx);
+  GRAM_TRY(dedup_launch(ctx, iws, ids, P, c.n_items, m->unique, m->inverse, m->perm, m->seg_off, m->n_unique, st));
+  int32_t U = 0;
+  GRAM_TRY(read_i32(m, m->n_unique, &U, st));
+  if (U <= 0 || U > m->u_cap) return gram_set_error(ctx, "gram_step: dedup returned U=%d", U), GRAM_ERR_ID_RANGE;
+  GRAM_CUDA(ctx, cudaEventRecord(ev[1], st));
+  int32_t n_encoded = 0, n_touched = U, encoder_ran = 0;
+  if (!multi) {
+    // stage 2: one encoding per unique item (Eq. 4)
+    for (int32_t u0 = 0; u0 < U; u0 += m->mb) {
+      const int32_t n = (U - u0 < m->mb) ? U - u0 : m->mb;
+      GRAM_TRY(encoder_forward_chunk(m, nullptr, m->unique + u0, 0, n, (char*)m->H + (size_t)u0 * c.d * m->esz, st));
+    }
+    GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
+    // stage 3
+    GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, (int)m->esz, m->E, st));
+  } else {
+    GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
+    GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, (int)m->esz, m->E, st));
+  }
+  GRAM_CUDA(ctx, cudaEventRecord(ev[3], st));
+  // task module forward / backward (Eq. 5) and dL/dE
+  GRAM_TRY(task_forward_backward(m, m->E, labels, B, m->dE, m->loss, st));
+  GRAM_CUDA(ctx, cudaEventRecord(ev[4], st));
+  // stage 4 (Eq. 6)
+  if (!multi) {
+    GRAM_TRY(accumulate_launch(ctx, iws, m->dE, 0, m->perm, m->seg_off, P, U, nullptr, c.d, nullptr, 0, m->G, st));
+  } else {
+    GRAM_TRY(accumulate_launch(ctx, iws, m->dE, 0, m->perm, m->seg_off, P, U, nullptr, c.d, m->unique, 1, m->table, st));
+    GRAM_TRY(touched_mark_launch(ctx, m->unique, U, c.n_items, m->touched, st));
+  }
+  GRAM_CUDA(ctx, cudaEventRecord(ev[5], st));
+  // stage 5 (Eq. 7)
+  if (!multi) {
+    GRAM_CUDA(ctx, cudaMemsetAsync(m->ce.g, 0, m->ce.n * 4, st));
+    if (U <= m->mb) {
+      GRAM_TRY(encoder_backward_chunk(m, m->G, U, st));
+    } else {
+      // activations of one micro-batch at a time: run the forward again, then its backward
+      float* Gbase = m->G;
+      GRAM_TRY(encoder_pass(m, m->unique, U, false,
+                            [&](int32_t u0, int32_t, const float** G) { *G = Gbase + (size_t)u0 * c.d; return GRAM_OK; }, st));
+    }
+    n_encoded = U;
+    encoder_ran = 1;
+    GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st));
+    GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+  } else {
+    GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st));
+    ++m->step_in_window;
+    GRAM_TRY(touched_list_launch(ctx, m->touched, c.n_items, m->tlist, m->tcount, st));
+    GRAM_TRY(read_i32(m, m->tcount, &n_touched, st));
+    if (m->step_in_window >= c.K) {
+      GRAM_CUDA(ctx, cudaMemsetAsync(m->ce.g, 0, m->ce.n * 4, st));
+      GRAM_TRY(encoder_pass(m, m->tlist, n_touched, true,
+                            [&](int32_t u0, int32_t n, const float** G) {
+                              *G = m->G;
+                              return gather_launch(ctx, m->table, c.n_items, m->tlist + u0, n, c.d, 4, m->G, st);
+                            }, st));
+      GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+      GRAM_TRY(model_window_reset(m, st));
+      n_encoded = n_touched;
+      encoder_ran = 1;
+    }
+  }
+  GRAM_CUDA(ctx, cudaEventRecord(ev[6], st));
+  GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 1, m->loss, 4, cudaMemcpyDeviceToHost, st));
+  GRAM_CUDA(ctx, cudaStreamSynchronize(st));
+  if (rep) {
+    memset(rep, 0, sizeof(*rep));
+    memcpy(&rep->loss, m->h_pinned + 1, 4);
+    rep->n_positions = (int32_t)P;
+    rep->n_unique = U;
+    rep->boost_ratio = (float)P / (float)U;
+    rep->n_touched = n_touched;
+    rep->encoder_pass = encoder_ran;
+    rep->n_encoded = n_encoded;
+    float* ms[6] = {&rep->ms_dedup, &rep->ms_encode, &rep->ms_gather, &rep->ms_task, &rep->ms_accumulate, &rep->ms_backward};
+    for (int i = 0; i < 6; ++i) cudaEventElapsedTime(ms[i], ev[i], ev[i + 1]);
+    cudaEventElapsedTime(&rep->ms_total, ev[0], ev[6]);
+  }
+  return GRAM_OK;
+}

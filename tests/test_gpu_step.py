@@ -1,0 +1,194 @@
+"""Gradient parity of the whole step and of its stages with the oracle (end-to-end training), through the C ABI.
+
+Tolerances: max |g_gpu - g_oracle| / max |g_oracle| per parameter tensor, 1e-3 for fp32 contexts and 2e-2 for bf16.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gram_oracle as orc
+from paper_2204_04179_b200 import binding, synth
+from tests import gram_helpers as gh
+
+pytestmark = pytest.mark.gpu
+DEV = gh.DEV
+TOL = {"f32": 1e-3, "bf16": 2e-2}
+
+
+def small(**kw):
+    base = dict(name="s", n_items=40, l_t=8, vocab=50, d=32, n_heads=2, d_ff=64, n_layers=2, pooling="mean",
+                task="kt", task_layers=1, task_heads=2, task_d_ff=64, task_attn_only=True, B=4, L=12, zipf_s=1.1)
+    base.update(kw)
+    return synth.GramShape(**base)
+
+
+CASES = {
+    "tiny_cfg": synth.config("tiny"),
+    "cls_full_task": small(pooling="cls", task_attn_only=False, task_layers=2),
+    "odd_sizes": small(n_items=23, l_t=5, d=24, n_heads=3, d_ff=40, B=3, L=7, task_heads=2),
+    "nr": small(task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls"),
+    "tiny_bf16": synth.config("tiny").replace(dtype="bf16"),
+    "bf16_cls_full": small(dtype="bf16", pooling="cls", task_attn_only=False, d=64, d_ff=128, task_d_ff=128),
+    "bf16_nr": small(dtype="bf16", task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls", d=64, d_ff=128),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_single_step_matches_e2e(name):
+    shape = CASES[name]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=3)
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab)
+    tol = TOL[shape.dtype]
+    assert rep.n_unique == len(np.unique(ids)) and rep.encoder_pass == 1
+    assert rep.boost_ratio == pytest.approx(ids.size / rep.n_unique, rel=1e-6)
+    assert abs(rep.loss - want["loss"]) <= tol * abs(want["loss"])
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+    print(name, "worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= tol, (n1, e1)
+    assert e2 <= tol, (n2, e2)
+
+
+def test_host_entry_point_and_determinism():
+    shape = CASES["tiny_cfg"]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=5)
+    r1, a1, b1 = gh.gpu_single_step(shape, ce, tk, toks, ids, lab)
+    r2, a2, b2 = gh.gpu_single_step(shape, ce, tk, toks, ids, lab, host=True)
+    assert r1.loss == r2.loss
+    for k in a1:
+        assert np.array_equal(a1[k], a2[k]), k        # bit-identical across runs and entry points
+    for k in b1:
+        assert np.array_equal(b1[k], b2[k]), k
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_micro_batched_encoder_pass_gives_the_same_gradients(dtype):
+    shape = small(dtype=dtype, d=64, d_ff=128, task_d_ff=128, n_items=60, B=6, L=16)
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=7)
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    U = len(np.unique(ids))
+    assert U > 16
+    rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab, ce_micro_batch=7)     # several ragged passes
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+    assert e1 <= TOL[dtype] and e2 <= TOL[dtype], (e1, n1, e2, n2)
+
+
+def test_stages_one_by_one():
+    """gram_dedup -> gram_encode_unique -> gram_gather -> gram_task -> gram_accumulate -> gram_encoder_backward."""
+    shape = small(pooling="cls", task_attn_only=False)
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=9)
+    ref = orc.gram_single_step(shape, ce, tk, toks, ids, lab)
+    g = gh.make_ctx(shape, ce, tk, toks)
+    P, d = ids.size, shape.d
+    ids_d = torch.from_numpy(ids.ravel().copy()).to(DEV)
+    lab_d = torch.from_numpy(lab.ravel().copy()).to(DEV)
+    cap = min(P, shape.n_items)
+    unique = torch.zeros(cap, dtype=torch.int32, device=DEV); inverse = torch.zeros(P, dtype=torch.int32, device=DEV)
+    perm = torch.zeros(P, dtype=torch.int32, device=DEV); seg = torch.zeros(cap + 1, dtype=torch.int32, device=DEV)
+    nu = torch.zeros(1, dtype=torch.int32, device=DEV)
+    g.dedup(ids_d, shape.n_items, unique, inverse, perm, seg, nu)
+    U = int(nu.item())
+    assert np.array_equal(unique[:U].cpu().numpy(), ref["unique"]) and np.array_equal(inverse.cpu().numpy(), ref["inverse"])
+    H = torch.zeros(U, d, device=DEV)
+    g.encode_unique(None, unique, U, H, save_activations=True)
+    g.sync()
+    assert gh.rel_err(H.cpu().numpy(), ref["H"]) <= 1e-4
+    E = torch.zeros(P, d, device=DEV)
+    g.gather(H, inverse, E)
+    dE = torch.zeros(P, d, device=DEV); loss = torch.zeros(1, device=DEV)
+    g.task(E, lab_d, shape.B, dE, loss)
+    g.sync()
+    assert abs(float(loss.item()) - ref["loss"]) <= 1e-4 * abs(ref["loss"])
+    assert gh.rel_err(dE.cpu().numpy(), ref["dE"]) <= 1e-3
+    G = torch.zeros(U, d, device=DEV)
+    g.accumulate(dE, perm, seg, U, G)
+    g.sync()
+    assert gh.rel_err(G.cpu().numpy(), ref["G"]) <= 1e-3
+    g.zero_grads(binding.GRAM_MODULE_CE)
+    g.encoder_backward(G, unique, U)
+    gce, gtk = gh.gpu_grads(g, shape)
+    e1, n1 = gh.worst_rel_err(gce, ref["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, ref["grad_task"])
+    assert e1 <= 1e-3 and e2 <= 1e-3, (e1, n1, e2, n2)
+    # Fig. 1's count: the encoder backward ran over U rows, not P
+    assert U < P
+    g.close()
+
+
+def test_fig1_counts_through_the_step():
+    shape = small(n_items=10, B=3, L=4)
+    ce, tk, toks, _, lab = gh.make_inputs(shape, seed=1)
+    ids = np.array([[3, 7, 3, 9], [7, 7, 1, 3], [9, 4, 1, 3]], np.int32)      # 12 interactions, 5 items
+    rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab)
+    assert rep.n_positions == 12 and rep.n_unique == 5 and rep.n_encoded == 5
+    assert rep.boost_ratio == pytest.approx(2.4)
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    assert gh.worst_rel_err(gce, want["grad_ce"])[0] <= 1e-3
+
+
+def test_step_rejects_bad_input_without_faulting():
+    shape = small()
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=2)
+    g = gh.make_ctx(shape, ce, tk, toks)
+    bad = ids.copy(); bad[1, 2] = shape.n_items
+    with pytest.raises(binding.GramError) as e:
+        g.step(torch.from_numpy(bad).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)
+    assert e.value.status == 2
+    with pytest.raises(binding.GramError) as e:
+        g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B + 1)
+    assert e.value.status == 3
+    rep = g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)      # still usable
+    assert rep.n_unique == len(np.unique(ids))
+    g.close()
+
+
+@pytest.mark.parametrize("dtype,K", [("f32", 1), ("f32", 3), ("bf16", 2)])
+def test_multistep_window_matches_algorithm(dtype, K):
+    shape = small(dtype=dtype, d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=max(K, 2), pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=21)
+    lr = 0.05
+    batches = [synth.batch(shape, 21, step=k) for k in range(K)]
+    cfg_K = K if K > 1 else 2
+    g = gh.make_ctx(shape, ce, tk, toks, K=cfg_K, lr_task=lr, ce_micro_batch=16)
+    g.cache_fill()
+    _, _, cache0 = g.get_window(want_table=False, want_touched=False)
+    enc = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    assert gh.rel_err(cache0, enc) <= (1e-4 if dtype == "f32" else 2e-2)
+    # the oracle starts from the cache values the device really holds, so that bf16 rounding of the cache
+    # is an input, not an error
+    want = orc.multistep_window(shape, ce, tk, toks, batches, cache0.astype(np.float64), lr_task=lr,
+                                cache_bf16=(dtype == "bf16"))
+    reps = []
+    for k, (ids, lab) in enumerate(batches):
+        if K == 1 and k == 0:
+            pass
+        reps.append(g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B))
+        if k < cfg_K - 1 and k == K - 1 and K == 1:
+            break
+    tol = TOL[dtype]
+    for k in range(len(reps)):
+        assert abs(reps[k].loss - want["losses"][k]) <= tol * abs(want["losses"][k])
+    if K >= 2:
+        assert [r.encoder_pass for r in reps] == [0] * (K - 1) + [1]
+        assert reps[-1].n_touched == len(want["items"]) == reps[-1].n_encoded
+        gce, gtk = gh.gpu_grads(g, shape)
+        e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+        e2, n2 = gh.worst_rel_err(gtk, want["grad_task_last"])
+        assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+        tp = synth.unflatten(g.get_params(binding.GRAM_MODULE_TASK), synth.task_param_spec(shape))
+        for name in tp:
+            assert gh.rel_err(tp[name], want["task_params"][name]) <= tol, name
+        table, touched, cache = g.get_window()
+        assert np.all(table == 0) and np.all(touched == 0)                 # the window was cleared
+        assert gh.rel_err(cache, want["cache"]) <= tol
+    else:
+        # K = 1 of a K = 2 context: first step only; table and touched set equal the single-step sums
+        table, touched, _ = g.get_window(want_cache=False)
+        bits = np.unpackbits(touched.view(np.uint8), bitorder="little")[:shape.n_items].astype(bool)
+        ids, lab = batches[0]
+        assert np.array_equal(np.nonzero(bits)[0], np.unique(ids))
+        one = orc.multistep_window(shape, ce, tk, toks, batches[:1], cache0.astype(np.float64), lr_task=lr)
+        assert gh.rel_err(table, one["table"]) <= tol
+    g.close()
