@@ -60,8 +60,9 @@ enum { GRAM_MODULE_CE = 0, GRAM_MODULE_TASK = 1 };
  * with the n_cand candidates, softmax cross-entropy on candidate 0 averaged
  * over B.  A context with n_layers == 0 and task == GRAM_TASK_NONE serves only
  * the index and accumulation calls.
- * dtype = GRAM_BF16: matrix products take bf16 operands with fp32 accumulation,
- * activations are stored as bf16, parameters and their gradients stay fp32. */
+ * dtype = GRAM_BF16: matrix products and attention take bf16 operands with fp32
+ * accumulation; the residual stream, LayerNorm statistics, encodings,
+ * parameters and their gradients stay fp32.  GRAM_F32: everything fp32. */
 typedef struct gram_config {
   int32_t dtype;
   int32_t n_items, l_t, vocab;
@@ -132,10 +133,11 @@ gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n
 
 /* Stage 2, Eq. 4: d_H[u, :] = CE(tokens of item d_items[u]) for u < U, once per
  * unique item.  d_item_tokens int32 [n_items, l_t] (NULL = the context's copy).
- * d_H is [U, d] of the context's dtype.  save_activations != 0 keeps what
- * gram_encoder_backward needs (U must then fit one micro-batch). */
+ * d_H is fp32 [U, d] for either dtype (the residual stream stays fp32; bf16 is
+ * the element type of the matrix products' operands).  save_activations != 0
+ * keeps what gram_encoder_backward needs (U must then fit one micro-batch). */
 gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
-                               void* d_H, int save_activations, gram_stream stream);
+                               float* d_H, int save_activations, gram_stream stream);
 
 /* Stage 3: d_E[p, :] = d_src[d_index[p], :] for p < P.  Single-step: src = H,
  * index = inverse.  Multi-step: src = the encoding cache, index = ids.
@@ -164,10 +166,10 @@ gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int
                               int32_t* d_count, gram_stream stream);
 
 /* Task module forward and backward (Eq. 5 and the gradient of Eq. 8 with
- * respect to the encodings): d_E [B, L, d] of the context's dtype, d_labels
- * int32 [B, L] -> d_dE fp32 [B*L, d], d_loss fp32 [1]; task parameter
- * gradients are overwritten in the context. */
-gram_status gram_task(gram_ctx* ctx, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE,
+ * respect to the encodings): d_E fp32 [B, L, d], d_labels int32 [B, L] ->
+ * d_dE fp32 [B*L, d], d_loss fp32 [1]; task parameter gradients are
+ * overwritten in the context. */
+gram_status gram_task(gram_ctx* ctx, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE,
                       float* d_loss, gram_stream stream);
 
 /* Stage 5, Eq. 7: encoder parameter gradients += sum over u of J_u^T d_G[u, :],

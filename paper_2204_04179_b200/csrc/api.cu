@@ -187,11 +187,11 @@ gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens) {
   return model_set_item_tokens(ctx->model, h_tokens);
 }
 gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
-                               void* d_H, int save_activations, gram_stream stream) {
+                               float* d_H, int save_activations, gram_stream stream) {
   NEED_MODEL("gram_encode_unique");
   return model_encode(ctx->model, d_item_tokens, d_items, U, d_H, save_activations, S(stream));
 }
-gram_status gram_task(gram_ctx* ctx, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
+gram_status gram_task(gram_ctx* ctx, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
                       gram_stream stream) {
   NEED_MODEL("gram_task");
   return model_task(ctx->model, d_E, d_labels, B, d_dE, d_loss, S(stream));

@@ -13,9 +13,14 @@ namespace {
 // ============================================================================================
 struct EpiDev {
   const float* bias;
-  const void* residual;
+  const float* res;
+  const float* res_mean;
+  const float* res_rstd;
+  const float* res_gamma;
+  const float* res_beta;
   void* pre;
   const void* dgelu_pre;
+  void* copy_out;
   int gelu;
   int accumulate;
 };
@@ -27,18 +32,94 @@ template <typename CT> __device__ __forceinline__ void st_c(CT* p, float v);
 template <> __device__ __forceinline__ void st_c<float>(float* p, float v) { *p = v; }
 template <> __device__ __forceinline__ void st_c<bf16>(bf16* p, float v) { *p = __float2bfloat16(v); }
 
-template <typename CT>
+// one element; CT is C's type, OT the operands' type
+template <typename CT, typename OT>
 __device__ __forceinline__ void epilogue_store(const EpiDev& e, CT* C, int64_t ldc, int64_t m, int n, float acc) {
   float v = acc + (e.bias ? e.bias[n] : 0.f);
   const int64_t o = m * ldc + n;
   if (e.gelu) {
-    if (e.pre) st_c<CT>(reinterpret_cast<CT*>(e.pre) + o, v);
+    if (e.pre) st_c<OT>(reinterpret_cast<OT*>(e.pre) + o, v);
     v = gelu_f(v);
   }
-  if (e.dgelu_pre) v *= gelu_grad_f(ld_c<CT>(reinterpret_cast<const CT*>(e.dgelu_pre) + o));
-  if (e.residual) v += ld_c<CT>(reinterpret_cast<const CT*>(e.residual) + o);
+  if (e.dgelu_pre) v *= gelu_grad_f(ld_c<OT>(reinterpret_cast<const OT*>(e.dgelu_pre) + o));
+  if (e.res) {
+    float r = e.res[o];
+    if (e.res_mean) r = (r - e.res_mean[m]) * e.res_rstd[m] * e.res_gamma[n] + e.res_beta[n];
+    v += r;
+  }
   if (e.accumulate) v += ld_c<CT>(C + o);
   st_c<CT>(C + o, v);
+  if (e.copy_out) st_c<OT>(reinterpret_cast<OT*>(e.copy_out) + o, v);
+}
+
+// eight consecutive columns n..n+7 of row m (n and ldc multiples of 8): 16-byte accesses throughout
+__device__ __forceinline__ void ld8(const float* p, float (&x)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void ld8(const bf16* p, float (&x)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+    x[2 * i] = f.x;
+    x[2 * i + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void st8(float* p, const float (&x)[8]) {
+  *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(x[4], x[5], x[6], x[7]);
+}
+__device__ __forceinline__ void st8(bf16* p, const float (&x)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <typename CT>
+__device__ __forceinline__ void epilogue_store8(const EpiDev& e, CT* C, int64_t ldc, int64_t m, int n, float (&v)[8],
+                                                float mu, float rs) {
+  const int64_t o = m * ldc + n;
+  float t[8];
+  if (e.bias) {
+    ld8(e.bias + n, t);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] += t[i];
+  }
+  if (e.gelu) {
+    if (e.pre) st8(reinterpret_cast<bf16*>(e.pre) + o, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = gelu_f(v[i]);
+  }
+  if (e.dgelu_pre) {
+    ld8(reinterpret_cast<const bf16*>(e.dgelu_pre) + o, t);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] *= gelu_grad_f(t[i]);
+  }
+  if (e.res) {
+    ld8(e.res + o, t);
+    if (e.res_mean) {
+      float g[8], b[8];
+      ld8(e.res_gamma + n, g);
+      ld8(e.res_beta + n, b);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = (t[i] - mu) * rs * g[i] + b[i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] += t[i];
+  }
+  if (e.accumulate) {
+    ld8(reinterpret_cast<const float*>(C) + o, t);      // accumulation is offered for fp32 C only
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] += t[i];
+  }
+  st8(C + o, v);
+  if (e.copy_out) st8(reinterpret_cast<bf16*>(e.copy_out) + o, v);
 }
 
 constexpr int ST = 64, SK = 16;
@@ -84,7 +165,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const float* __restrict__
     for (int j = 0; j < 4; ++j) {
       int64_t m = m0 + ty + 16 * i;
       int n = n0 + tx + 16 * j;
-      if (m < M && n < N) epilogue_store<float>(e, C, ldc, m, n, acc[i][j]);
+      if (m < M && n < N) epilogue_store<float, float>(e, C, ldc, m, n, acc[i][j]);
     }
 }
 
@@ -326,45 +407,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       tc_fence_after();
       const int64_t m = (int64_t)tm * BM + q * 32 + lane;
       CT* Cs = C + (int64_t)split * a.split_stride;
+      float mu = 0.f, rs = 1.f;
+      if (a.epi.res_mean && m < a.M) {
+        mu = a.epi.res_mean[m];
+        rs = a.epi.res_rstd[m];
+      }
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t v[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
         const int n0 = tn * BN + c0;
-        if (m < a.M && n0 < a.N) {
-          const bool plain = !a.epi.gelu && !a.epi.dgelu_pre && !a.epi.residual && !a.epi.accumulate;
-          if (n0 + 32 <= a.N && plain) {
-            // fast path: bias only, 16-byte stores
-            if (sizeof(CT) == 4) {
-              float4* dst = reinterpret_cast<float4*>(Cs + m * a.ldc + n0);
+        if (m < a.M) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float4 o;
-                o.x = __uint_as_float(v[4 * j + 0]) + (a.epi.bias ? a.epi.bias[n0 + 4 * j + 0] : 0.f);
-                o.y = __uint_as_float(v[4 * j + 1]) + (a.epi.bias ? a.epi.bias[n0 + 4 * j + 1] : 0.f);
-                o.z = __uint_as_float(v[4 * j + 2]) + (a.epi.bias ? a.epi.bias[n0 + 4 * j + 2] : 0.f);
-                o.w = __uint_as_float(v[4 * j + 3]) + (a.epi.bias ? a.epi.bias[n0 + 4 * j + 3] : 0.f);
-                dst[j] = o;
-              }
-            } else {
-              uint4* dst = reinterpret_cast<uint4*>(Cs + m * a.ldc + n0);
+          for (int j = 0; j < 4; ++j) {
+            const int n = n0 + 8 * j;
+            if (n < a.N) {                       // N is a multiple of 8
+              float x[8];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint32_t w[4];
-#pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                  float x0 = __uint_as_float(v[8 * j + 2 * h]) + (a.epi.bias ? a.epi.bias[n0 + 8 * j + 2 * h] : 0.f);
-                  float x1 = __uint_as_float(v[8 * j + 2 * h + 1]) + (a.epi.bias ? a.epi.bias[n0 + 8 * j + 2 * h + 1] : 0.f);
-                  __nv_bfloat162 p = __floats2bfloat162_rn(x0, x1);
-                  w[h] = *reinterpret_cast<uint32_t*>(&p);
-                }
-                dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
-              }
+              for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(v[8 * j + i]);
+              epilogue_store8<CT>(a.epi, Cs, a.ldc, m, n, x, mu, rs);
             }
-          } else {
-#pragma unroll 4
-            for (int j = 0; j < 32; ++j)
-              if (n0 + j < a.N) epilogue_store<CT>(a.epi, Cs, a.ldc, m, n0 + j, __uint_as_float(v[j]));
           }
         }
       }
@@ -412,7 +474,7 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
     for (int s = 0; s < splits; ++s) acc += part[(int64_t)s * split_stride + i];
     const int64_t m = i / N;
     const int n = (int)(i - m * N);
-    epilogue_store<CT>(e, C, ldc, m, n, acc);
+    epilogue_store<CT, bf16>(e, C, ldc, m, n, acc);
   }
 }
 
@@ -487,7 +549,8 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   if (M < 0 || N < 0 || K < 0) return gram_set_error(ctx, "gemm: negative size"), GRAM_ERR_ARG;
   if (M == 0 || N == 0) return GRAM_OK;
   if (!A || !B || !C) return gram_set_error(ctx, "gemm: null operand"), GRAM_ERR_ARG;
-  EpiDev e{epi.bias, epi.residual, epi.pre, epi.dgelu_pre, epi.gelu, epi.accumulate};
+  EpiDev e{epi.bias, epi.res, epi.res_mean, epi.res_rstd, epi.res_gamma, epi.res_beta, epi.pre, epi.dgelu_pre, epi.copy_out,
+           epi.gelu, epi.accumulate};
   if (dtype == GRAM_F32) {
     if (!c_f32) return gram_set_error(ctx, "gemm: fp32 operands need an fp32 result"), GRAM_ERR_UNSUPPORTED;
     dim3 grid((unsigned)ceil_div(N, ST), (unsigned)ceil_div64(M, ST));
@@ -501,6 +564,8 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
       K == 0)
     return gram_set_error(ctx, "gemm: bf16 operands need 16-byte aligned rows (sizes multiples of 8)"), GRAM_ERR_UNSUPPORTED;
   if (e.accumulate && !c_f32) return gram_set_error(ctx, "gemm: accumulation needs an fp32 result"), GRAM_ERR_UNSUPPORTED;
+  if ((N % 8) || (e.bias && ((uintptr_t)e.bias % 16)) || (e.res_gamma && (((uintptr_t)e.res_gamma % 16) || ((uintptr_t)e.res_beta % 16))))
+    return gram_set_error(ctx, "gemm: N must be a multiple of 8 and the epilogue's vectors 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
   const int BNsel = (N % 256 == 0 || N > 1024) ? 256 : (N > 64 ? 128 : 64);
   CUtensorMap ma, mb;
   bool ok;
@@ -535,7 +600,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
     args.C = ws->splitk;
     args.ldc = N;
     args.split_stride = (int64_t)M * N;
-    args.epi = EpiDev{nullptr, nullptr, nullptr, nullptr, 0, 0};
+    args.epi = EpiDev{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0};
     if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else if (BNsel == 128) err = launch_tc_major<128, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else err = launch_tc_major<64, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);

@@ -6,14 +6,23 @@
 //   v = acc + bias[n]
 //   gelu:       pre(m, n) = v (if pre != null);  v = gelu(v)          (forward of the feed-forward layer)
 //   dgelu_pre:  v = v * gelu'(dgelu_pre(m, n))                        (backward through the GELU)
-//   residual:   v += residual(m, n)
+//   res:        v += r(m, n), r = res(m, n), or, when res_mean != null, LayerNorm applied on the fly:
+//               r = (res(m, n) - res_mean[m]) * res_rstd[m] * res_gamma[n] + res_beta[n]
+//               (the fp32 residual stream: a layer's input is the LayerNorm of the previous fp32 sum)
 //   accumulate: v += C(m, n)                                          (fp32 C only)
-// pre, dgelu_pre and residual have C's element type and leading dimension.
+//   copy_out:   copy_out(m, n) = v as well                            (operand-typed copy of the result)
+// res is fp32; pre, dgelu_pre and copy_out have the operands' element type (bf16 on the tensor
+// cores, float in the fp32 kernel).  All of them share C's leading dimension.
 struct GemmEpilogue {
   const float* bias = nullptr;
-  const void* residual = nullptr;
+  const float* res = nullptr;
+  const float* res_mean = nullptr;
+  const float* res_rstd = nullptr;
+  const float* res_gamma = nullptr;
+  const float* res_beta = nullptr;
   void* pre = nullptr;
   const void* dgelu_pre = nullptr;
+  void* copy_out = nullptr;
   int gelu = 0;
   int accumulate = 0;
 };

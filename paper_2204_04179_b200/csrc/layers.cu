@@ -30,11 +30,10 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 
 // ---------------------------------------------------------------------------- embedding
-template <typename T>
 __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const int32_t* __restrict__ items,
                                  int32_t first_item, int64_t n_tok, int32_t n_items_total, int l_t, int vocab, int d,
-                                 const float* __restrict__ tok_emb, const float* __restrict__ pos_emb, T* __restrict__ z0,
-                                 int32_t* __restrict__ tok_ids, int32_t* status) {
+                                 const float* __restrict__ tok_emb, const float* __restrict__ pos_emb,
+                                 float* __restrict__ z0, int32_t* __restrict__ tok_ids, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -57,7 +56,7 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const 
 
 // ---------------------------------------------------------------------------- LayerNorm
 template <typename T, int NP>   // NP pairs of columns per lane: d <= 64*NP
-__global__ void __launch_bounds__(256) ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ g,
+__global__ void __launch_bounds__(256) ln_fwd_kernel(const float* __restrict__ z, const float* __restrict__ g,
                                                      const float* __restrict__ b, T* __restrict__ y,
                                                      float* __restrict__ mean, float* __restrict__ rstd, int64_t rows,
                                                      int d) {
@@ -97,10 +96,11 @@ __global__ void __launch_bounds__(256) ln_fwd_kernel(const T* __restrict__ z, co
 }
 
 template <typename T, int NP>
-__global__ void __launch_bounds__(256) ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z,
+__global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ z,
                                                      const float* __restrict__ mean, const float* __restrict__ rstd,
-                                                     const float* __restrict__ g, T* __restrict__ dz,
-                                                     float* __restrict__ part, int64_t rows, int d) {
+                                                     const float* __restrict__ g, float* __restrict__ dz,
+                                                     T* __restrict__ dz_b, float* __restrict__ part, int64_t rows,
+                                                     int d) {
   extern __shared__ float sacc[];          // [2][d]: dgamma, dbeta of this block
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   const int64_t w = (int64_t)blockIdx.x * nwb + warp;
@@ -138,7 +138,11 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const T* __restrict__ dy, c
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
       const int c = 2 * (lane + 32 * i);
-      if (c < d) st2(dz + r * d + c, make_float2(rs * (gy[i].x - s1 - xh[i].x * s2), rs * (gy[i].y - s1 - xh[i].y * s2)));
+      if (c < d) {
+        const float2 o = make_float2(rs * (gy[i].x - s1 - xh[i].x * s2), rs * (gy[i].y - s1 - xh[i].y * s2));
+        st2(dz + r * d + c, o);
+        if (dz_b) st2(dz_b + r * d + c, o);
+      }
     }
   }
   for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sacc[i] = 0.f;
@@ -371,33 +375,36 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, in
   }
 }
 
-template <typename T>
-__global__ void periodic_rowsum_kernel(const T* __restrict__ X, int64_t n_groups, int period, int d, float* __restrict__ out) {
+__global__ void periodic_rowsum_kernel(const float* __restrict__ X, int64_t n_groups, int period, int d,
+                                       float* __restrict__ out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)period * d) return;
   const int s = (int)(i / d), c = (int)(i - (int64_t)s * d);
   float acc = 0.f;
-  for (int64_t u = 0; u < n_groups; ++u) acc += ldf(X + (u * period + s) * d + c);
+  for (int64_t u = 0; u < n_groups; ++u) acc += X[(u * period + s) * d + c];
   out[i] += acc;
 }
 
 // ---------------------------------------------------------------------------- pooling
-template <typename T>
-__global__ void pool_fwd_kernel(const T* __restrict__ x, T* __restrict__ H, int64_t n, int l_t, int d, int pooling) {
+__device__ __forceinline__ float stream_at(const StreamRef& x, int64_t row, int c, int d) {
+  float v = x.z[row * d + c];
+  if (x.mean) v = (v - x.mean[row]) * x.rstd[row] * x.gamma[c] + x.beta[c];
+  return v;
+}
+__global__ void pool_fwd_kernel(StreamRef x, float* __restrict__ H, int64_t n, int l_t, int d, int pooling) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * d) return;
   const int64_t u = i / d;
   const int c = (int)(i - u * d);
   if (pooling == GRAM_POOL_CLS) {
-    H[i] = x[u * l_t * d + c];
+    H[i] = stream_at(x, u * l_t, c, d);
   } else {
     float acc = 0.f;
-    for (int s = 0; s < l_t; ++s) acc += ldf(x + (u * l_t + s) * d + c);
-    stf(H + i, acc / l_t);
+    for (int s = 0; s < l_t; ++s) acc += stream_at(x, u * l_t + s, c, d);
+    H[i] = acc / l_t;
   }
 }
-template <typename T>
-__global__ void pool_bwd_kernel(const float* __restrict__ G, T* __restrict__ dx, int64_t n, int l_t, int d, int pooling) {
+__global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__ dx, int64_t n, int l_t, int d, int pooling) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * l_t * d) return;
   const int64_t t = i / d;
@@ -407,13 +414,14 @@ __global__ void pool_bwd_kernel(const float* __restrict__ G, T* __restrict__ dx,
   float v;
   if (pooling == GRAM_POOL_CLS) v = (s == 0) ? G[u * d + c] : 0.f;
   else v = G[u * d + c] / l_t;
-  stf(dx + i, v);
+  dx[i] = v;
 }
 
 // ---------------------------------------------------------------------------- KT task input / head
 template <typename T>
-__global__ void kt_input_fwd_kernel(const T* __restrict__ E, const float* __restrict__ pos, const float* __restrict__ resp,
-                                    const int32_t* __restrict__ labels, T* __restrict__ x, int64_t P, int L, int d) {
+__global__ void kt_input_fwd_kernel(const float* __restrict__ E, const float* __restrict__ pos,
+                                    const float* __restrict__ resp, const int32_t* __restrict__ labels,
+                                    float* __restrict__ x, T* __restrict__ x_b, int64_t P, int L, int d) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= P * d) return;
   const int64_t p = i / d;
@@ -421,11 +429,12 @@ __global__ void kt_input_fwd_kernel(const T* __restrict__ E, const float* __rest
   const int n = (int)(p % L);
   int prev = (n == 0) ? 2 : labels[p - 1];
   prev = prev < 0 ? 0 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);
-  stf(x + i, ldf(E + i) + pos[(int64_t)n * d + c] + resp[(int64_t)prev * d + c]);
+  const float v = E[i] + pos[(int64_t)n * d + c] + resp[(int64_t)prev * d + c];
+  x[i] = v;
+  stf(x_b + i, v);
 }
 // one thread per column: dE = dx; dpos[n, c] += sum_b; dresp[r, c] += sum over positions with prev == r
-template <typename T>
-__global__ void kt_input_bwd_kernel(const T* __restrict__ dx, const int32_t* __restrict__ labels, float* __restrict__ dE,
+__global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t* __restrict__ labels, float* __restrict__ dE,
                                     float* __restrict__ dpos, float* __restrict__ dresp, int B, int L, int d) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   const int n = blockIdx.y;
@@ -433,7 +442,7 @@ __global__ void kt_input_bwd_kernel(const T* __restrict__ dx, const int32_t* __r
   float ap = 0.f, r0 = 0.f, r1 = 0.f, r2 = 0.f;
   for (int b = 0; b < B; ++b) {
     const int64_t p = (int64_t)b * L + n;
-    const float v = ldf(dx + p * d + c);
+    const float v = dx[p * d + c];
     dE[p * d + c] = v;
     ap += v;
     int prev = (n == 0) ? 2 : labels[p - 1];
@@ -448,10 +457,10 @@ __global__ void kt_input_bwd_kernel(const T* __restrict__ dx, const int32_t* __r
 
 // warp per position; per-block partials: [d] for dw, then loss and db
 template <typename T>
-__global__ void __launch_bounds__(256) kt_head_kernel(const T* __restrict__ y, const float* __restrict__ w,
+__global__ void __launch_bounds__(256) kt_head_kernel(StreamRef y, const float* __restrict__ w,
                                                       const float* __restrict__ bias, const int32_t* __restrict__ labels,
-                                                      T* __restrict__ dy, float* __restrict__ part, int64_t P, int d,
-                                                      int64_t pstride) {
+                                                      float* __restrict__ dy, T* __restrict__ dy_b,
+                                                      float* __restrict__ part, int64_t P, int d, int64_t pstride) {
   extern __shared__ float sacc[];            // [d + 2]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   for (int i = threadIdx.x; i < d + 2; i += blockDim.x) sacc[i] = 0.f;
@@ -465,16 +474,19 @@ __global__ void __launch_bounds__(256) kt_head_kernel(const T* __restrict__ y, c
     float dzl = 0.f, lossr = 0.f;
     if (r < r1) {
       float acc = 0.f;
-      for (int c = lane; c < d; c += 32) acc += ldf(y + r * d + c) * w[c];
+      for (int c = lane; c < d; c += 32) acc += stream_at(y, r, c, d) * w[c];
       const float z = warp_sum(acc) + b0;
       const float lab = (float)labels[r];
       lossr = fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
       dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
-      for (int c = lane; c < d; c += 32) stf(dy + r * d + c, dzl * w[c]);
+      for (int c = lane; c < d; c += 32) {
+        dy[r * d + c] = dzl * w[c];
+        if (dy_b) stf(dy_b + r * d + c, dzl * w[c]);
+      }
     }
     for (int ww = 0; ww < nwb; ++ww) {       // rows of this round add in ascending order
       if (warp == ww && r < r1) {
-        for (int c = lane; c < d; c += 32) sacc[c] += dzl * ldf(y + r * d + c);
+        for (int c = lane; c < d; c += 32) sacc[c] += dzl * stream_at(y, r, c, d);
         if (lane == 0) { sacc[d] += lossr; sacc[d + 1] += dzl; }
       }
       __syncthreads();
@@ -497,7 +509,7 @@ __global__ void kt_head_reduce_kernel(const float* __restrict__ part, int nblock
 // ---------------------------------------------------------------------------- NR task (per user)
 // pre[b, n, :] = E[b, n, :] wa^T + ba is given.  One block per user.
 template <typename T>
-__global__ void __launch_bounds__(256) nr_user_kernel(const T* __restrict__ E, const T* __restrict__ pre,
+__global__ void __launch_bounds__(256) nr_user_kernel(const float* __restrict__ E, const T* __restrict__ pre,
                                                       const float* __restrict__ qa, float* __restrict__ dE,
                                                       T* __restrict__ dpre, float* __restrict__ part, int L, int n_cand,
                                                       int d, int d_a, float invB) {
@@ -510,7 +522,7 @@ __global__ void __launch_bounds__(256) nr_user_kernel(const T* __restrict__ E, c
   float* sc = du + d;            // [n_cand] scores, then ds
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
-  const T* Eb = E + (int64_t)b * L * d;
+  const float* Eb = E + (int64_t)b * L * d;
   const T* pb = pre + (int64_t)b * L * d_a;
   for (int n = warp; n < n_hist; n += nwb) {
     float acc = 0.f;
@@ -617,7 +629,7 @@ __global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, f
     w[i] -= lr * g[i];
 }
 template <typename T>
-__global__ void scatter_rows_kernel(const T* __restrict__ src, const int32_t* __restrict__ index, int64_t n, int d,
+__global__ void scatter_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ index, int64_t n, int d,
                                     int64_t n_dst_rows, T* __restrict__ dst, int32_t* status) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * d) return;
@@ -625,7 +637,7 @@ __global__ void scatter_rows_kernel(const T* __restrict__ src, const int32_t* __
   const int c = (int)(i - u * d);
   const int32_t r = index[u];
   if (r < 0 || r >= n_dst_rows) { gram_device_fail(status, GRAM_ERR_ID_RANGE); return; }
-  dst[(int64_t)r * d + c] = src[i];
+  stf(dst + (int64_t)r * d + c, src[i]);
 }
 
 inline int grid_for(int64_t n, int threads, int cap) {
@@ -654,37 +666,36 @@ template <typename F> gram_status set_smem(gram_ctx* ctx, F kern, size_t bytes) 
   else if ((d) <= 768) { constexpr int NP = 12; __VA_ARGS__; }                 \
   else { constexpr int NP = 16; __VA_ARGS__; }
 
-gram_status embed_forward(gram_ctx* ctx, int dtype, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
+gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, void* z0, int32_t* tok_ids, cudaStream_t st) {
+                          const float* pos_emb, float* z0, int32_t* tok_ids, cudaStream_t st) {
   const int64_t n_tok = (int64_t)n_chunk * l_t;
   if (n_tok == 0) return GRAM_OK;
   const int blocks = grid_for(n_tok * 32, 256, kNumSMs * 8);
-  DISPATCH_T(dtype, embed_fwd_kernel<T><<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t,
-                                                               vocab, d, tok_emb, pos_emb, (T*)z0, tok_ids,
-                                                               gram_status_word(ctx)));
+  embed_fwd_kernel<<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t, vocab, d, tok_emb,
+                                           pos_emb, z0, tok_ids, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status layernorm_forward(gram_ctx* ctx, int dtype, const void* z, const float* gamma, const float* beta, void* y,
+gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
                               float* mean, float* rstd, int64_t rows, int d, cudaStream_t st) {
   if (rows == 0) return GRAM_OK;
   if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
   const int blocks = grid_for(rows * 32, 256, kNumSMs * 8);
-  DISPATCH_T(dtype, DISPATCH_NP(d, ln_fwd_kernel<T, NP><<<blocks, 256, 0, st>>>((const T*)z, gamma, beta, (T*)y, mean, rstd, rows, d)));
+  DISPATCH_T(dtype, DISPATCH_NP(d, ln_fwd_kernel<T, NP><<<blocks, 256, 0, st>>>(z, gamma, beta, (T*)y, mean, rstd, rows, d)));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status layernorm_backward(gram_ctx* ctx, int dtype, const void* dy, const void* z, const float* mean,
-                               const float* rstd, const float* gamma, void* dz, float* dgamma, float* dbeta,
-                               float* scratch, int64_t rows, int d, cudaStream_t st) {
+gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const float* z, const float* mean,
+                               const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
+                               float* dbeta, float* scratch, int64_t rows, int d, cudaStream_t st) {
   if (rows == 0) return GRAM_OK;
   if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
   const int blocks = grid_for(rows * 32, 256, kRedBlocks);
   const size_t smem = (size_t)2 * d * sizeof(float);
-  DISPATCH_T(dtype, DISPATCH_NP(d, ln_bwd_kernel<T, NP><<<blocks, 256, smem, st>>>((const T*)dy, (const T*)z, mean, rstd, gamma, (T*)dz, scratch, rows, d)));
+  DISPATCH_T(dtype, DISPATCH_NP(d, ln_bwd_kernel<T, NP><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
   reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -737,66 +748,67 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
   return GRAM_OK;
 }
 
-gram_status periodic_rowsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t n_groups, int period, int d,
-                                       float* out, cudaStream_t st) {
+gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
+                                       cudaStream_t st) {
   if (n_groups == 0) return GRAM_OK;
   const int64_t n = (int64_t)period * d;
-  DISPATCH_T(dtype, periodic_rowsum_kernel<T><<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>((const T*)X, n_groups, period, d, out));
+  periodic_rowsum_kernel<<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>(X, n_groups, period, d, out);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status pool_forward(gram_ctx* ctx, int dtype, const void* x, void* H, int64_t n, int l_t, int d, int pooling,
+gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
                          cudaStream_t st) {
   if (n == 0) return GRAM_OK;
-  DISPATCH_T(dtype, pool_fwd_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>((const T*)x, (T*)H, n, l_t, d, pooling));
+  pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status pool_backward(gram_ctx* ctx, int dtype, const float* G, void* dx, int64_t n, int l_t, int d, int pooling,
+gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
                           cudaStream_t st) {
   if (n == 0) return GRAM_OK;
-  DISPATCH_T(dtype, pool_bwd_kernel<T><<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, (T*)dx, n, l_t, d, pooling));
+  pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status kt_input_forward(gram_ctx* ctx, int dtype, const void* E, const float* pos, const float* resp,
-                             const int32_t* labels, void* x, int B, int L, int d, cudaStream_t st) {
+gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const float* pos, const float* resp,
+                             const int32_t* labels, float* x, void* x_b, int B, int L, int d, cudaStream_t st) {
   const int64_t P = (int64_t)B * L;
   if (P == 0) return GRAM_OK;
-  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)ceil_div64(P * d, 256), 256, 0, st>>>((const T*)E, pos, resp, labels, (T*)x, P, L, d));
+  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)ceil_div64(P * d, 256), 256, 0, st>>>(E, pos, resp, labels, x, (T*)x_b, P, L, d));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status kt_head(gram_ctx* ctx, int dtype, const void* y, const float* w, const float* b, const int32_t* labels,
-                    void* dy, float* dw, float* db, float* loss, float* scratch, int64_t P, int d, cudaStream_t st) {
+gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w, const float* b, const int32_t* labels,
+                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int64_t P, int d,
+                    cudaStream_t st) {
   if (P == 0) return GRAM_OK;
   int blocks = (int)ceil_div64(P, 64);
   if (blocks > kRedBlocks) blocks = kRedBlocks;
   const int64_t pstride = d + 2;
   const size_t smem = (size_t)(d + 2) * sizeof(float);
-  DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>((const T*)y, w, b, labels, (T*)dy, scratch, P, d, pstride));
+  DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>(y, w, b, labels, dy, (T*)dy_b, scratch, P, d, pstride));
   kt_head_reduce_kernel<<<ceil_div(d + 2, 256), 256, 0, st>>>(scratch, blocks, pstride, d, 1.f / (float)P, dw, db, loss);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 // dE = dx, dpos += column sums over b, dresp += sums by previous response; scratch holds [L][3][d]
-gram_status kt_input_backward(gram_ctx* ctx, int dtype, const void* dx, const int32_t* labels, float* dE, float* dpos,
-                                 float* dresp, float* scratch, int B, int L, int d, cudaStream_t st) {
+gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* labels, float* dE, float* dpos,
+                              float* dresp, float* scratch, int B, int L, int d, cudaStream_t st) {
   if (B == 0) return GRAM_OK;
   if ((size_t)L * 3 * d * sizeof(float) > kRedScratchBytes) return gram_set_error(ctx, "kt task: L*d too large for the reduction scratch"), GRAM_ERR_UNSUPPORTED;
   dim3 grid((unsigned)ceil_div(d, 128), (unsigned)L);
-  DISPATCH_T(dtype, kt_input_bwd_kernel<T><<<grid, 128, 0, st>>>((const T*)dx, labels, dE, dpos, scratch, B, L, d));
+  kt_input_bwd_kernel<<<grid, 128, 0, st>>>(dx, labels, dE, dpos, scratch, B, L, d);
   reduce_partials_kernel<<<ceil_div(3 * d, 256), 256, 0, st>>>(scratch, L, (int64_t)3 * d, 3 * d, dresp, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status nr_user(gram_ctx* ctx, int dtype, const void* E, const void* pre, const float* qa, float* dE,
+gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, const float* qa, float* dE,
                            void* dpre, float* dqa, float* loss, float* scratch, int B, int L, int n_cand, int d, int d_a,
                            cudaStream_t st) {
   if (B == 0) return GRAM_OK;
@@ -804,7 +816,7 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const void* E, const void* pre, co
   const size_t smem = ((size_t)2 * L + 2 * d + n_cand) * sizeof(float);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, nr_user_kernel<T>, smem));
-    nr_user_kernel<T><<<B, 256, smem, st>>>((const T*)E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B);
+    nr_user_kernel<T><<<B, 256, smem, st>>>(E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B);
   });
   nr_reduce_kernel<<<ceil_div(d_a + 1, 256), 256, 0, st>>>(scratch, B, d_a, 1.f / (float)B, dqa, loss);
   GRAM_LAUNCH_CHECK(ctx);
@@ -830,10 +842,10 @@ gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
-gram_status scatter_rows(gram_ctx* ctx, int dtype, const void* src, const int32_t* index, int64_t n, int d,
+gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
-  DISPATCH_T(dtype, scatter_rows_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>((const T*)src, index, n, d, n_dst_rows, (T*)dst, gram_status_word(ctx)));
+  DISPATCH_T(dtype, scatter_rows_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(src, index, n, d, n_dst_rows, (T*)dst, gram_status_word(ctx)));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -8,18 +8,30 @@ constexpr int kRedBlocks = 592;            // upper bound on blocks that leave p
 // bytes of the reduction scratch: kRedBlocks partial rows of up to 2*4096 floats
 constexpr size_t kRedScratchBytes = (size_t)kRedBlocks * 2 * 4096 * sizeof(float);
 
-// z0[t, :] = tok_emb[token(t), :] + pos_emb[t % l_t, :], token(t) = item_tokens[items[t / l_t], t % l_t];
-// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.
-gram_status embed_forward(gram_ctx* ctx, int dtype, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
-                          int32_t n_items_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, void* z0, int32_t* tok_ids, cudaStream_t st);
+// A row-major [rows, d] view of the fp32 residual stream: either the values themselves (mean == null)
+// or LayerNorm of them, applied where they are read: (z - mean[row]) * rstd[row] * gamma[c] + beta[c].
+struct StreamRef {
+  const float* z = nullptr;
+  const float* mean = nullptr;
+  const float* rstd = nullptr;
+  const float* gamma = nullptr;
+  const float* beta = nullptr;
+};
 
-gram_status layernorm_forward(gram_ctx* ctx, int dtype, const void* z, const float* gamma, const float* beta, void* y,
+// z0[t, :] = tok_emb[token(t), :] + pos_emb[t % l_t, :] (fp32), token(t) = item_tokens[items[t / l_t], t % l_t];
+// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.
+gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
+                          int32_t n_items_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
+                          const float* pos_emb, float* z0, int32_t* tok_ids, cudaStream_t st);
+
+// y = LayerNorm(z): z is the fp32 stream, y the operand-typed copy the next matrix product reads
+gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
                               float* mean, float* rstd, int64_t rows, int d, cudaStream_t st);
-// dz = LayerNorm backward of dy at input z; dgamma += sum_rows dy * xhat; dbeta += sum_rows dy
-gram_status layernorm_backward(gram_ctx* ctx, int dtype, const void* dy, const void* z, const float* mean,
-                               const float* rstd, const float* gamma, void* dz, float* dgamma, float* dbeta,
-                               float* scratch, int64_t rows, int d, cudaStream_t st);
+// dz = LayerNorm backward of dy at input z (fp32, plus an operand-typed copy dz_b when not null);
+// dgamma += sum_rows dy * xhat; dbeta += sum_rows dy
+gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const float* z, const float* mean,
+                               const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
+                               float* dbeta, float* scratch, int64_t rows, int d, cudaStream_t st);
 
 // softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d]
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
@@ -27,42 +39,44 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq,
                                int S, int d, int n_heads, int causal, cudaStream_t st);
 
-// out[n] += sum_rows X[r, n]
+// out[n] += sum_rows X[r, n]   (X operand-typed)
 gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t rows, int N, float* out, float* scratch,
                               cudaStream_t st);
-// out[s, :] += sum_u X[u*period + s, :]  (s < period)
-gram_status periodic_rowsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t n_groups, int period, int d,
-                                       float* out, cudaStream_t st);
+// out[s, :] += sum_u X[u*period + s, :]  (s < period; X fp32)
+gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
+                                       cudaStream_t st);
 
-// H[u, :] = mean_s x[u*l_t + s, :] (mean) or x[u*l_t, :] (cls); H has type T
-gram_status pool_forward(gram_ctx* ctx, int dtype, const void* x, void* H, int64_t n, int l_t, int d, int pooling,
+// H[u, :] = mean_s x[u*l_t + s, :] (mean) or x[u*l_t, :] (cls), fp32
+gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
                          cudaStream_t st);
-// dx[u*l_t + s, :] from G[u, :] (fp32)
-gram_status pool_backward(gram_ctx* ctx, int dtype, const float* G, void* dx, int64_t n, int l_t, int d, int pooling,
+// dx[u*l_t + s, :] from G[u, :] (both fp32)
+gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
                           cudaStream_t st);
 
-// knowledge-tracing task input: x[b, n, :] = E[b, n, :] + pos[n, :] + resp[prev(b, n), :],
-// prev(b, 0) = 2, prev(b, n) = labels[b, n-1]
-gram_status kt_input_forward(gram_ctx* ctx, int dtype, const void* E, const float* pos, const float* resp,
-                             const int32_t* labels, void* x, int B, int L, int d, cudaStream_t st);
-// dE (fp32) = dx; dpos[n] += sum_b dx[b, n]; dresp[r] += sum over positions with prev == r
-gram_status kt_input_backward(gram_ctx* ctx, int dtype, const void* dx, const int32_t* labels, float* dE, float* dpos,
+// knowledge-tracing task input: x[b, n, :] = E[b, n, :] + pos[n, :] + resp[prev(b, n), :] (fp32, and an
+// operand-typed copy x_b), prev(b, 0) = 2, prev(b, n) = labels[b, n-1]
+gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const float* pos, const float* resp,
+                             const int32_t* labels, float* x, void* x_b, int B, int L, int d, cudaStream_t st);
+// dE = dx; dpos[n] += sum_b dx[b, n]; dresp[r] += sum over positions with prev == r
+gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* labels, float* dE, float* dpos,
                               float* dresp, float* scratch, int B, int L, int d, cudaStream_t st);
-// logit = y . w + b; loss = mean BCE; dy = (sigmoid(logit) - label) / (B*L) * w; dw, db accumulate
-gram_status kt_head(gram_ctx* ctx, int dtype, const void* y, const float* w, const float* b, const int32_t* labels,
-                    void* dy, float* dw, float* db, float* loss, float* scratch, int64_t P, int d, cudaStream_t st);
+// logit = y . w + b; loss = mean BCE; dy = (sigmoid(logit) - label) / (B*L) * w (fp32, and an operand-typed
+// copy dy_b when not null); dw, db accumulate
+gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w, const float* b, const int32_t* labels,
+                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int64_t P, int d,
+                    cudaStream_t st);
 
 // news-recommendation task, the part between the matrix products (one block per user):
-// given pre = E wa^T + ba [B*L, d_a], computes additive attention over the first L - n_cand encodings,
-// dot-product scores with the candidates and softmax cross-entropy on candidate 0 (averaged over B);
-// writes the direct part of dE (fp32 [B*L, d]), dpre (type T, zero rows for candidates), dqa +=, loss.
-gram_status nr_user(gram_ctx* ctx, int dtype, const void* E, const void* pre, const float* qa, float* dE, void* dpre,
+// given pre = E wa^T + ba [B*L, d_a] (operand-typed), computes additive attention over the first L - n_cand
+// encodings, dot-product scores with the candidates and softmax cross-entropy on candidate 0 (averaged over
+// B); writes the direct part of dE (fp32 [B*L, d]), dpre (operand-typed, zero rows for candidates), dqa +=, loss.
+gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, const float* qa, float* dE, void* dpre,
                     float* dqa, float* loss, float* scratch, int B, int L, int n_cand, int d, int d_a, cudaStream_t st);
 
 // element-wise helpers
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st);
 gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st);
 gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st);
-// dst[index[u], :] = src[u, :]
-gram_status scatter_rows(gram_ctx* ctx, int dtype, const void* src, const int32_t* index, int64_t n, int d,
+// dst[index[u], :] = src[u, :] (src fp32, dst operand-typed)
+gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st);

@@ -22,8 +22,11 @@ struct Module {
   bool wb_stale = true;
 };
 
+// saved per layer.  fp32: the residual sums z1, z2 (attention-only layers: outf) and LayerNorm statistics;
+// operand-typed (bf16 on the tensor cores): what the matrix products and attention read
 struct LayerActs {
-  void *qkv, *ctx, *z1, *h1, *u, *g, *z2, *out;
+  void *qkv, *ctx, *h1, *u, *g, *out;
+  float *z1, *z2, *outf;
   float *mean1, *rstd1, *mean2, *rstd2;
 };
 
@@ -33,7 +36,9 @@ struct Stack {
   int64_t cap = 0;                         // tokens the buffers hold
   std::vector<LayerOff> off;
   std::vector<LayerActs> acts;
-  void *dA = nullptr, *dB = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;   // backward scratch
+  // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
+  float *curf = nullptr, *othf = nullptr;
+  void *dzb = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;
 };
 
 struct Arena {
@@ -76,7 +81,8 @@ struct Model {
   // encoder
   size_t o_tok = 0, o_pos = 0, o_elng = 0, o_elnb = 0;
   Stack enc;
-  void *z0 = nullptr, *x0 = nullptr;
+  float* z0 = nullptr;               // token + position embedding, fp32
+  void* x0 = nullptr;                // its LayerNorm, operand-typed
   float *mean0 = nullptr, *rstd0 = nullptr;
   int32_t *tok_ids = nullptr, *tok_unique = nullptr, *tok_inverse = nullptr, *tok_perm = nullptr, *tok_seg = nullptr,
           *tok_nu = nullptr;
@@ -85,13 +91,15 @@ struct Model {
   // task
   size_t t_pos = 0, t_resp = 0, t_headw = 0, t_headb = 0, t_wa = 0, t_ba = 0, t_qa = 0;
   Stack tk;
-  void *tx = nullptr, *pre = nullptr, *dpre = nullptr;
+  float* tx = nullptr;               // task input stream, fp32
+  void *txb = nullptr, *pre = nullptr, *dpre = nullptr;
   // step buffers
   int32_t* item_tokens = nullptr;
   int32_t *ids = nullptr, *labels = nullptr, *unique = nullptr, *inverse = nullptr, *perm = nullptr, *seg_off = nullptr,
           *n_unique = nullptr;
   int32_t u_cap = 0;
-  void *H = nullptr, *E = nullptr;
+  float *H = nullptr, *E = nullptr;  // encodings per unique item / per position, fp32
+  void* Eb = nullptr;                // operand-typed copy of E (NR products; Multi-step gather from the cache)
   float *dE = nullptr, *G = nullptr, *loss = nullptr, *red = nullptr;
   // Multi-step window
   float* table = nullptr;
@@ -115,20 +123,23 @@ void stack_buffers(Arena& a, Stack& s, size_t esz) {
     x.qkv = a.take(T * 3 * d * esz);
     x.ctx = a.take(T * d * esz);
     x.out = a.take(T * d * esz);
-    if (!s.attn_only) {
-      x.z1 = a.take(T * d * esz);
+    if (s.attn_only) {
+      x.outf = (float*)a.take(T * d * 4);
+    } else {
+      x.z1 = (float*)a.take(T * d * 4);
       x.h1 = a.take(T * d * esz);
       x.u = a.take(T * f * esz);
       x.g = a.take(T * f * esz);
-      x.z2 = a.take(T * d * esz);
+      x.z2 = (float*)a.take(T * d * 4);
       x.mean1 = (float*)a.take(T * 4);
       x.rstd1 = (float*)a.take(T * 4);
       x.mean2 = (float*)a.take(T * 4);
       x.rstd2 = (float*)a.take(T * 4);
     }
   }
-  s.dA = a.take(T * d * esz);
-  s.dB = a.take(T * d * esz);
+  s.curf = (float*)a.take(T * d * 4);
+  s.othf = (float*)a.take(T * d * 4);
+  s.dzb = a.take(T * d * esz);
   s.dqkv = a.take(T * 3 * d * esz);
   s.dctx = a.take(T * d * esz);
   s.du = s.attn_only ? nullptr : a.take(T * f * esz);
@@ -140,7 +151,7 @@ void layout_buffers(Model* m, Arena& a) {
   const int64_t P = (int64_t)c.B_max * c.L;
   if (c.n_layers > 0) {
     const size_t T = (size_t)m->mb * c.l_t;
-    m->z0 = a.take(T * d * esz);
+    m->z0 = (float*)a.take(T * d * 4);
     m->x0 = a.take(T * d * esz);
     m->mean0 = (float*)a.take(T * 4);
     m->rstd0 = (float*)a.take(T * 4);
@@ -156,7 +167,8 @@ void layout_buffers(Model* m, Arena& a) {
   }
   if (c.task != GRAM_TASK_NONE) {
     if (c.task == GRAM_TASK_KT) {
-      m->tx = a.take((size_t)P * d * esz);
+      m->tx = (float*)a.take((size_t)P * d * 4);
+      m->txb = a.take((size_t)P * d * esz);
       stack_buffers(a, m->tk, esz);
     } else {
       m->pre = a.take((size_t)P * c.d_a * esz);
@@ -171,9 +183,10 @@ void layout_buffers(Model* m, Arena& a) {
   m->seg_off = (int32_t*)a.take(((size_t)m->u_cap + 1) * 4);
   m->n_unique = (int32_t*)a.take(4);
   const size_t hrows = (size_t)(m->u_cap > m->mb ? m->u_cap : m->mb);
-  m->H = a.take(hrows * d * esz);
+  m->H = (float*)a.take(hrows * d * 4);
   m->G = (float*)a.take(hrows * d * 4);
-  m->E = a.take((size_t)P * d * esz);
+  m->E = (float*)a.take((size_t)P * d * 4);
+  m->Eb = a.take((size_t)P * d * esz);
   m->dE = (float*)a.take((size_t)P * d * 4);
   m->loss = (float*)a.take(4);
   m->red = (float*)a.take(kRedScratchBytes);
@@ -212,15 +225,17 @@ inline const void* W(const Model* m, const Module& mod, size_t off) {
 }
 inline void* at(const Model* m, void* p, size_t elems) { return (char*)p + elems * m->esz; }
 
-// Y[T, N] = X[T, K] W[N, K]^T (+ epilogue), activations of type T
-gram_status mm_fwd(Model* m, const void* X, const void* Wt, void* Y, int64_t T, int N, int K, const GemmEpilogue& e,
-                   cudaStream_t st) {
-  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, X, 1, K, Wt, 1, K, Y, m->dtype == GRAM_F32, N, T, N, K, e, 0, st);
+// Y[T, N] = X[T, K] W[N, K]^T (+ epilogue); y_f32: Y is the fp32 stream, else operand-typed
+gram_status mm_fwd(Model* m, const void* X, const void* Wt, void* Y, bool y_f32, int64_t T, int N, int K,
+                   const GemmEpilogue& e, cudaStream_t st) {
+  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, X, 1, K, Wt, 1, K, Y, (y_f32 || m->dtype == GRAM_F32) ? 1 : 0, N, T,
+                     N, K, e, 0, st);
 }
 // dX[T, K] = dY[T, N] W[N, K] (+ epilogue)
-gram_status mm_dx(Model* m, const void* dY, const void* Wt, void* dX, int64_t T, int N, int K, const GemmEpilogue& e,
-                  cudaStream_t st) {
-  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 1, N, Wt, 0, K, dX, m->dtype == GRAM_F32, K, T, K, N, e, 0, st);
+gram_status mm_dx(Model* m, const void* dY, const void* Wt, void* dX, bool x_f32, int64_t T, int N, int K,
+                  const GemmEpilogue& e, cudaStream_t st) {
+  return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 1, N, Wt, 0, K, dX, (x_f32 || m->dtype == GRAM_F32) ? 1 : 0, K, T,
+                     K, N, e, 0, st);
 }
 // dW[N, K] += dY[T, N]^T X[T, K]   (fp32 result, the token dimension may be split)
 gram_status mm_dw(Model* m, const void* dY, const void* X, float* dW, int64_t T, int N, int K, cudaStream_t st) {
@@ -229,108 +244,131 @@ gram_status mm_dw(Model* m, const void* dY, const void* X, float* dW, int64_t T,
   return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 0, N, X, 0, K, dW, 1, K, N, K, T, e, 1, st);
 }
 
-gram_status stack_forward(Model* m, Module& mod, Stack& s, const void* x_in, int64_t n_seq, int S, cudaStream_t st,
-                          const void** out) {
+void set_res(GemmEpilogue& e, const StreamRef& x) {
+  e.res = x.z;
+  e.res_mean = x.mean;
+  e.res_rstd = x.rstd;
+  e.res_gamma = x.gamma;
+  e.res_beta = x.beta;
+}
+
+// x_in: the fp32 input stream; x_in_b: its operand-typed copy.  *out / *out_b: the same pair for the output.
+gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in, const void* x_in_b, int64_t n_seq, int S,
+                          cudaStream_t st, StreamRef* out, const void** out_b) {
   const int64_t T = n_seq * S;
   const int d = s.d, f = s.d_ff;
   gram_ctx* ctx = m->ctx;
-  const void* x = x_in;
+  StreamRef x = x_in;
+  const void* xb = x_in_b;
   for (int l = 0; l < s.n_layers; ++l) {
     const LayerOff& o = s.off[l];
     LayerActs& a = s.acts[l];
     GemmEpilogue e;
     e.bias = mod.w + o.bqkv;
-    GRAM_TRY(mm_fwd(m, x, W(m, mod, o.wqkv), a.qkv, T, 3 * d, d, e, st));
+    GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * d, d, e, st));
     GRAM_TRY(attention_forward(ctx, m->dtype, a.qkv, a.ctx, n_seq, S, d, s.heads, s.causal, st));
     e = GemmEpilogue();
     e.bias = mod.w + o.bo;
-    e.residual = x;
+    set_res(e, x);
     if (s.attn_only) {
-      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.out, T, d, d, e, st));
+      e.copy_out = a.out;
+      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.outf, true, T, d, d, e, st));       // out = x + ctx Wo^T + bo
+      x = StreamRef();
+      x.z = a.outf;
     } else {
-      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.z1, T, d, d, e, st));
+      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.z1, true, T, d, d, e, st));         // z1 = x + ctx Wo^T + bo
       GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z1, mod.w + o.ln1g, mod.w + o.ln1b, a.h1, a.mean1, a.rstd1, T, d, st));
       e = GemmEpilogue();
       e.bias = mod.w + o.b1;
       e.gelu = 1;
       e.pre = a.u;
-      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, T, f, d, e, st));
+      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, false, T, f, d, e, st));          // u = h1 W1^T + b1, g = gelu(u)
       e = GemmEpilogue();
       e.bias = mod.w + o.b2;
-      e.residual = a.h1;
-      GRAM_TRY(mm_fwd(m, a.g, W(m, mod, o.w2), a.z2, T, d, f, e, st));
+      StreamRef h1;
+      h1.z = a.z1; h1.mean = a.mean1; h1.rstd = a.rstd1; h1.gamma = mod.w + o.ln1g; h1.beta = mod.w + o.ln1b;
+      set_res(e, h1);
+      GRAM_TRY(mm_fwd(m, a.g, W(m, mod, o.w2), a.z2, true, T, d, f, e, st));           // z2 = LN1(z1) + g W2^T + b2
       GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z2, mod.w + o.ln2g, mod.w + o.ln2b, a.out, a.mean2, a.rstd2, T, d, st));
+      x = StreamRef();
+      x.z = a.z2; x.mean = a.mean2; x.rstd = a.rstd2; x.gamma = mod.w + o.ln2g; x.beta = mod.w + o.ln2b;
     }
-    x = a.out;
+    xb = a.out;
   }
   *out = x;
+  *out_b = xb;
   return GRAM_OK;
 }
 
-// the incoming gradient (with respect to the stack's output) is in s.dA; *d_in points at the
-// gradient with respect to x_in when this returns
-gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in, int64_t n_seq, int S, cudaStream_t st,
-                           void** d_in) {
+// On entry s.curf holds the gradient with respect to the stack's output (fp32; for a stack of
+// attention-only layers s.dzb holds its operand-typed copy as well).  On return *d_in points at the
+// fp32 gradient with respect to the input stream.
+gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, int64_t n_seq, int S, cudaStream_t st,
+                           float** d_in) {
   const int64_t T = n_seq * S;
   const int d = s.d, f = s.d_ff;
   gram_ctx* ctx = m->ctx;
   float* red = m->red;
-  void* cur = s.dA;
-  void* oth = s.dB;
+  float* cur = s.curf;
+  float* oth = s.othf;
   for (int l = s.n_layers - 1; l >= 0; --l) {
     const LayerOff& o = s.off[l];
     LayerActs& a = s.acts[l];
-    const void* x_l = (l == 0) ? x_in : s.acts[l - 1].out;
+    const void* xb_l = (l == 0) ? x_in_b : s.acts[l - 1].out;
     GemmEpilogue e;
     if (!s.attn_only) {
       // out = LN2(z2), z2 = h1 + W2 gelu(u) + b2, u = W1 h1 + b1, h1 = LN1(z1), z1 = x + Wo ctx + bo
-      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, mod.g + o.ln2g,
-                                  mod.g + o.ln2b, red, T, d, st));                       // oth = dz2
-      GRAM_TRY(colsum_accumulate(ctx, m->dtype, oth, T, d, mod.g + o.b2, red, st));
-      GRAM_TRY(mm_dw(m, oth, a.g, mod.g + o.w2, T, d, f, st));
+      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, s.dzb, mod.g + o.ln2g,
+                                  mod.g + o.ln2b, red, T, d, st));                       // oth, dzb = dz2
+      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.b2, red, st));
+      GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st));
       e = GemmEpilogue();
       e.dgelu_pre = a.u;
-      GRAM_TRY(mm_dx(m, oth, W(m, mod, o.w2), s.du, T, d, f, e, st));                    // du = (dz2 W2) * gelu'(u)
+      GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(u)
       GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
       GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st));
       e = GemmEpilogue();
-      e.residual = oth;
-      GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, T, f, d, e, st));                    // cur = dh1 = du W1 + dz2
-      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, mod.g + o.ln1g,
-                                  mod.g + o.ln1b, red, T, d, st));                       // oth = dz1
+      e.res = oth;
+      GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, true, T, f, d, e, st));              // cur = dh1 = du W1 + dz2
+      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, s.dzb, mod.g + o.ln1g,
+                                  mod.g + o.ln1b, red, T, d, st));                       // oth, dzb = dz1
     } else {
-      void* t = cur; cur = oth; oth = t;                                                 // oth = d(out)
+      float* t = cur; cur = oth; oth = t;                                                // oth = d(out), dzb its copy
     }
-    GRAM_TRY(colsum_accumulate(ctx, m->dtype, oth, T, d, mod.g + o.bo, red, st));
-    GRAM_TRY(mm_dw(m, oth, a.ctx, mod.g + o.wo, T, d, d, st));
+    GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
+    GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st));
     e = GemmEpilogue();
-    GRAM_TRY(mm_dx(m, oth, W(m, mod, o.wo), s.dctx, T, d, d, e, st));
+    GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.wo), s.dctx, false, T, d, d, e, st));
     GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, n_seq, S, d, s.heads, s.causal, st));
     GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
-    GRAM_TRY(mm_dw(m, s.dqkv, x_l, mod.g + o.wqkv, T, 3 * d, d, st));
+    GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st));
     e = GemmEpilogue();
-    e.residual = oth;
-    GRAM_TRY(mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, T, 3 * d, d, e, st));              // cur = dx = dqkv Wqkv + dz1
+    e.res = oth;
+    if (s.attn_only && l > 0) e.copy_out = s.dzb;                                        // the layer below reads it as an operand
+    GRAM_TRY(mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, true, T, 3 * d, d, e, st));        // cur = dx = dqkv Wqkv + dz1
   }
   *d_in = cur;
   return GRAM_OK;
 }
 
-// encoder forward over n items (d_items, or first_item.. when null): H_out [n, d] of type T
+// encoder forward over n items (d_items, or first_item.. when null): H_out [n, d] fp32
 gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t first_item,
-                                  int32_t n, void* H_out, cudaStream_t st) {
+                                  int32_t n, float* H_out, cudaStream_t st) {
   const gram_config& c = m->cfg;
   gram_ctx* ctx = m->ctx;
   if (n > m->mb) return gram_set_error(ctx, "encoder pass over %d items exceeds the micro-batch of %d", n, m->mb), GRAM_ERR_WORKSPACE;
   GRAM_TRY(refresh_bf16(m, m->ce, st));
   const int64_t T = (int64_t)n * c.l_t;
-  GRAM_TRY(embed_forward(ctx, m->dtype, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items,
-                         c.l_t, c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, st));
+  GRAM_TRY(embed_forward(ctx, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items, c.l_t,
+                         c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, st));
   GRAM_TRY(layernorm_forward(ctx, m->dtype, m->z0, m->ce.w + m->o_elng, m->ce.w + m->o_elnb, m->x0, m->mean0, m->rstd0, T,
                              c.d, st));
-  const void* out = nullptr;
-  GRAM_TRY(stack_forward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &out));
-  GRAM_TRY(pool_forward(ctx, m->dtype, out, H_out, n, c.l_t, c.d, c.pooling, st));
+  StreamRef x0;
+  x0.z = m->z0; x0.mean = m->mean0; x0.rstd = m->rstd0; x0.gamma = m->ce.w + m->o_elng; x0.beta = m->ce.w + m->o_elnb;
+  StreamRef out;
+  const void* out_b = nullptr;
+  GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
+  GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, st));
   m->saved_n = n;
   return GRAM_OK;
 }
@@ -341,22 +379,23 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   gram_ctx* ctx = m->ctx;
   if (n != m->saved_n) return gram_set_error(ctx, "encoder backward over %d items, but activations of %d are saved", n, m->saved_n), GRAM_ERR_ARG;
   const int64_t T = (int64_t)n * c.l_t;
-  GRAM_TRY(pool_backward(ctx, m->dtype, G, m->enc.dA, n, c.l_t, c.d, c.pooling, st));
-  void* dx0 = nullptr;
+  GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, st));
+  float* dx0 = nullptr;
   GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
-  void* dz0 = (dx0 == m->enc.dA) ? m->enc.dB : m->enc.dA;
-  GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, m->ce.g + m->o_elng,
-                              m->ce.g + m->o_elnb, m->red, T, c.d, st));
-  GRAM_TRY(periodic_rowsum_accumulate(ctx, m->dtype, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, st));
+  float* dz0 = (dx0 == m->enc.curf) ? m->enc.othf : m->enc.curf;
+  GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, nullptr,
+                              m->ce.g + m->o_elng, m->ce.g + m->o_elnb, m->red, T, c.d, st));
+  GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, st));
   // token-embedding gradient: sum dz0 over the occurrences of each token (same index kernels as stage 1 / 4)
   IndexWorkspace* iws = gram_index_ws(ctx);
   GRAM_TRY(dedup_launch(ctx, iws, m->tok_ids, T, c.vocab, m->tok_unique, m->tok_inverse, m->tok_perm, m->tok_seg, m->tok_nu, st));
-  GRAM_TRY(accumulate_launch(ctx, iws, dz0, m->dtype == GRAM_BF16, m->tok_perm, m->tok_seg, T, 0, m->tok_nu, c.d,
-                             m->tok_unique, 1, m->ce.g + m->o_tok, st));
+  GRAM_TRY(accumulate_launch(ctx, iws, dz0, 0, m->tok_perm, m->tok_seg, T, 0, m->tok_nu, c.d, m->tok_unique, 1,
+                             m->ce.g + m->o_tok, st));
   return GRAM_OK;
 }
 
-gram_status task_forward_backward(Model* m, const void* E, const int32_t* labels, int32_t B, float* dE, float* loss,
+// E: fp32 [B, L, d]
+gram_status task_forward_backward(Model* m, const float* E, const int32_t* labels, int32_t B, float* dE, float* loss,
                                   cudaStream_t st) {
   const gram_config& c = m->cfg;
   gram_ctx* ctx = m->ctx;
@@ -364,29 +403,37 @@ gram_status task_forward_backward(Model* m, const void* E, const int32_t* labels
   GRAM_TRY(refresh_bf16(m, m->task, st));
   GRAM_CUDA(ctx, cudaMemsetAsync(m->task.g, 0, m->task.n * 4, st));
   if (c.task == GRAM_TASK_KT) {
-    GRAM_TRY(kt_input_forward(ctx, m->dtype, E, m->task.w + m->t_pos, m->task.w + m->t_resp, labels, m->tx, B, c.L, c.d, st));
-    const void* y = nullptr;
-    GRAM_TRY(stack_forward(m, m->task, m->tk, m->tx, B, c.L, st, &y));
-    GRAM_TRY(kt_head(ctx, m->dtype, y, m->task.w + m->t_headw, m->task.w + m->t_headb, labels, m->tk.dA,
+    GRAM_TRY(kt_input_forward(ctx, m->dtype, E, m->task.w + m->t_pos, m->task.w + m->t_resp, labels, m->tx, m->txb, B, c.L,
+                              c.d, st));
+    StreamRef x;
+    x.z = m->tx;
+    StreamRef y;
+    const void* y_b = nullptr;
+    GRAM_TRY(stack_forward(m, m->task, m->tk, x, m->txb, B, c.L, st, &y, &y_b));
+    void* dy_b = (m->tk.attn_only && m->tk.n_layers > 0) ? m->tk.dzb : nullptr;
+    GRAM_TRY(kt_head(ctx, m->dtype, y, m->task.w + m->t_headw, m->task.w + m->t_headb, labels, m->tk.curf, dy_b,
                      m->task.g + m->t_headw, m->task.g + m->t_headb, loss, m->red, P, c.d, st));
-    void* dx = nullptr;
-    GRAM_TRY(stack_backward(m, m->task, m->tk, m->tx, B, c.L, st, &dx));
-    GRAM_TRY(kt_input_backward(ctx, m->dtype, dx, labels, dE, m->task.g + m->t_pos, m->task.g + m->t_resp, m->red, B, c.L,
-                               c.d, st));
+    float* dx = nullptr;
+    GRAM_TRY(stack_backward(m, m->task, m->tk, m->txb, B, c.L, st, &dx));
+    GRAM_TRY(kt_input_backward(ctx, dx, labels, dE, m->task.g + m->t_pos, m->task.g + m->t_resp, m->red, B, c.L, c.d, st));
     return GRAM_OK;
   }
   if (c.task == GRAM_TASK_NR) {
+    const void* Eb = E;                  // fp32 contexts: the stream is its own operand
+    if (m->dtype == GRAM_BF16) {
+      GRAM_TRY(convert_f32_to_bf16(ctx, E, (bf16*)m->Eb, (size_t)P * c.d, st));
+      Eb = m->Eb;
+    }
     GemmEpilogue e;
     e.bias = m->task.w + m->t_ba;
-    GRAM_TRY(mm_fwd(m, E, W(m, m->task, m->t_wa), m->pre, P, c.d_a, c.d, e, st));
+    GRAM_TRY(mm_fwd(m, Eb, W(m, m->task, m->t_wa), m->pre, false, P, c.d_a, c.d, e, st));
     GRAM_TRY(nr_user(ctx, m->dtype, E, m->pre, m->task.w + m->t_qa, dE, m->dpre, m->task.g + m->t_qa, loss, m->red, B, c.L,
                      c.n_cand, c.d, c.d_a, st));
     GRAM_TRY(colsum_accumulate(ctx, m->dtype, m->dpre, P, c.d_a, m->task.g + m->t_ba, m->red, st));
-    GRAM_TRY(mm_dw(m, m->dpre, E, m->task.g + m->t_wa, P, c.d_a, c.d, st));
+    GRAM_TRY(mm_dw(m, m->dpre, Eb, m->task.g + m->t_wa, P, c.d_a, c.d, st));
     e = GemmEpilogue();
     e.accumulate = 1;                    // dE already holds the direct part
-    GRAM_TRY(gemm_launch(ctx, gram_gemm_ws(ctx), m->dtype, m->dpre, 1, c.d_a, W(m, m->task, m->t_wa), 0, c.d, dE, 1, c.d, P,
-                         c.d, c.d_a, e, 0, st));
+    GRAM_TRY(mm_dx(m, m->dpre, W(m, m->task, m->t_wa), dE, true, P, c.d_a, c.d, e, st));
     return GRAM_OK;
   }
   return gram_set_error(ctx, "the context has no task module"), GRAM_ERR_ARG;
@@ -546,7 +593,7 @@ gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens) {
   return GRAM_OK;
 }
 
-gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, void* d_H, int save,
+gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, float* d_H, int save,
                          cudaStream_t st) {
   if (m->cfg.n_layers <= 0) return gram_set_error(m->ctx, "the context has no encoder"), GRAM_ERR_ARG;
   if (U < 0 || (U > 0 && (!d_items || !d_H))) return gram_set_error(m->ctx, "gram_encode_unique: bad argument"), GRAM_ERR_ARG;
@@ -554,13 +601,13 @@ gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* 
     return gram_set_error(m->ctx, "gram_encode_unique: %d items do not fit the micro-batch of %d when activations are kept", U, m->mb), GRAM_ERR_WORKSPACE;
   for (int32_t u0 = 0; u0 < U; u0 += m->mb) {
     const int32_t n = (U - u0 < m->mb) ? U - u0 : m->mb;
-    GRAM_TRY(encoder_forward_chunk(m, d_item_tokens, d_items + u0, 0, n, (char*)d_H + (size_t)u0 * m->cfg.d * m->esz, st));
+    GRAM_TRY(encoder_forward_chunk(m, d_item_tokens, d_items + u0, 0, n, d_H + (size_t)u0 * m->cfg.d, st));
   }
   if (!save || U == 0) m->saved_n = save ? 0 : -1;
   return GRAM_OK;
 }
 
-gram_status model_task(Model* m, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
+gram_status model_task(Model* m, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
                        cudaStream_t st) {
   if (B < 0 || B > m->cfg.B_max) return gram_set_error(m->ctx, "gram_task: B=%d exceeds B_max=%d", B, m->cfg.B_max), GRAM_ERR_WORKSPACE;
   if (B == 0) return GRAM_OK;
@@ -592,7 +639,9 @@ gram_status model_cache_fill(Model* m, cudaStream_t st) {
   const gram_config& c = m->cfg;
   for (int32_t u0 = 0; u0 < c.n_items; u0 += m->mb) {
     const int32_t n = (c.n_items - u0 < m->mb) ? c.n_items - u0 : m->mb;
-    GRAM_TRY(encoder_forward_chunk(m, nullptr, nullptr, u0, n, (char*)m->cache + (size_t)u0 * c.d * m->esz, st));
+    GRAM_TRY(encoder_forward_chunk(m, nullptr, nullptr, u0, n, m->H, st));
+    if (m->dtype == GRAM_BF16) GRAM_TRY(convert_f32_to_bf16(m->ctx, m->H, (bf16*)m->cache + (size_t)u0 * c.d, (size_t)n * c.d, st));
+    else GRAM_CUDA(m->ctx, cudaMemcpyAsync((float*)m->cache + (size_t)u0 * c.d, m->H, (size_t)n * c.d * 4, cudaMemcpyDeviceToDevice, st));
   }
   m->saved_n = -1;
   return GRAM_OK;
@@ -648,14 +697,19 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
     // stage 2: one encoding per unique item (Eq. 4)
     for (int32_t u0 = 0; u0 < U; u0 += m->mb) {
       const int32_t n = (U - u0 < m->mb) ? U - u0 : m->mb;
-      GRAM_TRY(encoder_forward_chunk(m, nullptr, m->unique + u0, 0, n, (char*)m->H + (size_t)u0 * c.d * m->esz, st));
+      GRAM_TRY(encoder_forward_chunk(m, nullptr, m->unique + u0, 0, n, m->H + (size_t)u0 * c.d, st));
     }
     GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
     // stage 3
-    GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, (int)m->esz, m->E, st));
+    GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, 4, m->E, st));
   } else {
     GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
-    GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, (int)m->esz, m->E, st));
+    if (m->dtype == GRAM_BF16) {       // rows of the bf16 cache, widened for the task module
+      GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 2, m->Eb, st));
+      GRAM_TRY(convert_to_f32(ctx, GRAM_BF16, m->Eb, m->E, (size_t)P * c.d, st));
+    } else {
+      GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 4, m->E, st));
+    }
   }
   GRAM_CUDA(ctx, cudaEventRecord(ev[3], st));
   // task module forward / backward (Eq. 5) and dL/dE

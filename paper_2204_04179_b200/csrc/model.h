@@ -14,9 +14,9 @@ gram_status model_set_params(Model* m, int module, const float* h, size_t n);
 gram_status model_get_params(Model* m, int module, float* h, size_t n, int grads);
 gram_status model_zero_grads(Model* m, int module, cudaStream_t st);
 gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens);
-gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, void* d_H,
+gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, float* d_H,
                          int save, cudaStream_t st);
-gram_status model_task(Model* m, const void* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
+gram_status model_task(Model* m, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,
                        cudaStream_t st);
 gram_status model_encoder_backward(Model* m, const float* d_G, const int32_t* d_items, int32_t U, cudaStream_t st);
 gram_status model_step(Model* m, const int32_t* ids, const int32_t* labels, int32_t B, int on_host,
