@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the GRAM training step (Single-step GRAM on the knowledge-tracing-shaped workload).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload kt|nr|tiny]
+
+A step is one pass of the whole path (dedup, encode unique items, gather, task module forward/backward,
+accumulate, encoder backward) over one batch of seeded synthetic histories.  Prints ONE JSON line.
+With --impl reference the CPU oracle (end-to-end training, one encoder call per interaction) is timed
+instead, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "interactions/sec per GRAM train step on 1 B200; accumulate/gather GB/s vs HBM peak"
+UNIT = "interactions/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops=p["bf16_tflops_sustained"], tflops_burst=p["bf16_tflops"], source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1400.0, tflops_burst=1590.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                                          "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample(shape, ce, tk, toks, ids, lab, n_pos):
+    """The oracle, as it stands, on the first n_pos positions of the first history: interactions/s."""
+    import torch
+    from oracle import gram_oracle as orc
+    sub = shape.replace(B=1, L=n_pos)
+    tk_sub = dict(tk)
+    tk_sub["pos"] = tk["pos"][:n_pos] if "pos" in tk else None
+    if tk_sub["pos"] is None:
+        del tk_sub["pos"]
+    t0 = time.time()
+    orc.e2e_step(sub, ce, tk_sub, toks, ids[:1, :n_pos], lab[:1, :n_pos])
+    dt = time.time() - t0
+    return n_pos / dt, dt, torch.get_num_threads()
+
+
+def bounded_sample_size(shape):
+    if shape.name == "tiny":
+        return shape.L
+    return min(shape.L, 48 if shape.task == "kt" else shape.L)
+
+
+def run_reference(args, shape):
+    from paper_2204_04179_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    ce = synth.encoder_params(shape, args.seed)
+    tk = synth.task_params(shape, args.seed)
+    toks = synth.item_tokens(args.seed, shape.n_items, shape.l_t, shape.vocab)
+    n_pos = min(bounded_sample_size(shape), 12 if shape.name != "tiny" else shape.L)
+    times, cores = [], 0
+    for k in range(args.warmup + args.steps):
+        ids, lab = synth.batch(shape, args.seed, step=k)
+        v, dt, cores = oracle_sample(shape, ce, tk, toks, ids, lab, n_pos)
+        if k >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n_pos * len(times) / total
+    sample = f"end-to-end oracle (float64, one encoder call per interaction) on the first {n_pos} positions of one history per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "B": 1, "L": n_pos, "n_items": shape.n_items, "note": "bounded sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def kernel_sweep_cell(binding, synth, torch, dev, peaks):
+    """dedup / gather / accumulate alone on one sweep cell larger than L2 (P=1e6, N=1e5, Zipf 1.1, d=768)."""
+    P, N, s, d = 1_000_000, 100_000, 1.1, 768
+    cfg = binding.GramConfig(); cfg.n_items = N; cfg.P_max = P; cfg.d_max = d; cfg.d = d
+    g = binding.Gram(cfg)
+    ids = torch.from_numpy(synth.zipf_ids(1, N, s, P)).to(dev)
+    cap = min(P, N)
+    unique = torch.empty(cap, dtype=torch.int32, device=dev); inverse = torch.empty(P, dtype=torch.int32, device=dev)
+    perm = torch.empty(P, dtype=torch.int32, device=dev); seg = torch.empty(cap + 1, dtype=torch.int32, device=dev)
+    nu = torch.zeros(1, dtype=torch.int32, device=dev)
+    g.dedup(ids, N, unique, inverse, perm, seg, nu); g.sync()
+    U = int(nu.item())
+    H = torch.randn(U, d, device=dev); E = torch.empty(P, d, device=dev)
+    dE = torch.randn(P, d, device=dev); G = torch.empty(U, d, device=dev)
+
+    def timeit(fn, n=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(n):
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize(); ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+    passes = (max(1, (N - 1).bit_length()) + 7) // 8
+    out = {}
+    for name, fn, nbytes in (
+            ("dedup", lambda: g.dedup(ids, N, unique, inverse, perm, seg, nu), (16 * passes + 20) * P + 8 * U),
+            ("gather_f32", lambda: g.gather(H, inverse, E), 4 * P * d + 4 * U * d + 4 * P),
+            ("accumulate", lambda: g.accumulate(dE, perm, seg, U, G), 4 * P * d + 4 * U * d + 4 * P + 4 * (U + 1))):
+        ms = timeit(fn)
+        out[name] = {"ms": ms, "GB/s": nbytes / ms / 1e6, "frac_of_" + peaks["source"] + "_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
+    out["cell"] = {"P": P, "n_items": N, "zipf_s": s, "d": d, "U": U}
+    g.close()
+    return out
+
+
+def run_gram(args, shape):
+    import torch
+    from paper_2204_04179_b200 import binding, synth
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    peaks = measured_peaks()
+
+    ce = synth.encoder_params(shape, args.seed)
+    tk = synth.task_params(shape, args.seed)
+    toks = synth.item_tokens(args.seed, shape.n_items, shape.l_t, shape.vocab)
+    over = {}
+    if args.micro_batch:
+        over["ce_micro_batch"] = args.micro_batch
+    cfg = binding.config_from_shape(shape, **over)
+    g = binding.Gram(cfg)
+    g.set_params(binding.GRAM_MODULE_CE, synth.flatten(ce))
+    g.set_params(binding.GRAM_MODULE_TASK, synth.flatten(tk))
+    g.set_item_tokens(toks)
+    P = shape.B * shape.L
+    n_total = args.warmup + args.steps
+    # every rank draws its own batches (weak scaling: per-GPU work is fixed, histories are independent)
+    batches = [synth.batch(shape, args.seed + 7919 * rank, step=k) for k in range(n_total)]
+    dev_batches = [(torch.from_numpy(i).to(dev), torch.from_numpy(l).to(dev)) for i, l in batches]
+    pinned = [(torch.from_numpy(i).pin_memory(), torch.from_numpy(l).pin_memory()) for i, l in batches]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident inputs ----
+    for k in range(args.warmup):
+        g.step(dev_batches[k][0], dev_batches[k][1], shape.B)
+    g.profile(True)
+    launches0 = g.launch_count()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    reports = []
+    for k in range(args.warmup, n_total):
+        reports.append(g.step(dev_batches[k][0], dev_batches[k][1], shape.B))
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    launches = g.launch_count() - launches0
+    kinds = g.profile_read()
+    g.profile(False)
+
+    # ---- end to end: host buffers through gram_step_host (copies inside the timed region) ----
+    for k in range(min(args.warmup, 1)):
+        g.step_host(pinned[k][0].numpy(), pinned[k][1].numpy(), shape.B)
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(args.warmup, n_total):
+        g.step_host(pinned[k][0].numpy(), pinned[k][1].numpy(), shape.B)
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+
+    if rank != 0:
+        g.close()
+        return
+    value = world * P * args.steps / (ms_total / 1e3)
+    e2e_value = world * P * args.steps / (ms_e2e / 1e3)
+    gm = kinds["gemm"]
+    achieved = gm["work"] / (gm["ms"] / 1e3) / 1e12 if gm["ms"] > 0 else 0.0
+    roofline = {"kernel": "gemm_tc_kernel (bf16 tcgen05, fp32 accumulate)" if shape.dtype == "bf16" else "gemm_f32_kernel",
+                "bound": "tensor" if shape.dtype == "bf16" else "alu",
+                "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
+                "peak_source": peaks["source"] + " bf16_tflops_sustained", "traffic": None,
+                "launches": gm["launches"], "avg_launch_ms": gm["ms"] / max(1, gm["launches"]),
+                "share_of_step": gm["ms"] / (ms_total if ms_total > 0 else 1)}
+    stage_ms = {k: statistics.mean(getattr(r, k) for r in reports)
+                for k in ("ms_dedup", "ms_encode", "ms_gather", "ms_task", "ms_accumulate", "ms_backward", "ms_total")}
+    per_kind = {}
+    for name, v in kinds.items():
+        if v["launches"] == 0:
+            continue
+        rate = v["work"] / (v["ms"] / 1e3) if v["ms"] > 0 else 0.0
+        is_flops = name in ("gemm", "attention")
+        per_kind[name] = {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps,
+                          ("TFLOP/s" if is_flops else "GB/s"): rate / (1e12 if is_flops else 1e9),
+                          "frac": rate / ((peaks["tflops"] * 1e12) if is_flops else (peaks["hbm_gbs"] * 1e9))}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": shape.dtype, "data": "synthetic",
+        "config": {"workload": shape.name, "B": shape.B, "L": shape.L, "n_items": shape.n_items, "l_t": shape.l_t,
+                   "encoder": f"{shape.n_layers}x{shape.d} ({shape.n_heads} heads, ffn {shape.d_ff}), {shape.pooling} pooling",
+                   "task": shape.task, "zipf_s": shape.zipf_s, "unique_items_per_step": statistics.mean(r.n_unique for r in reports),
+                   "boost_ratio_R": statistics.mean(r.boost_ratio for r in reports), "ce_micro_batch": int(cfg.ce_micro_batch),
+                   "l2": "working set (activations of >1e5 tokens) far larger than L2; no flush needed",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 GPU"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * P, "d2h_bytes_per_step": 12,
+                "ms_per_step": ms_e2e / args.steps},
+        "roofline": roofline, "stage_ms": stage_ms, "kernel_kinds": per_kind,
+    }
+    g.close()
+    if world == 1:
+        del dev_batches
+        torch.cuda.empty_cache()
+        try:
+            line["hbm_kernels"] = kernel_sweep_cell(binding, synth, torch, dev, peaks)
+        except Exception as ex:          # the sweep cell is extra information, never a reason to lose the line
+            line["hbm_kernels"] = {"error": repr(ex)}
+        n_pos = bounded_sample_size(shape)
+        v, dt, cores = oracle_sample(shape, ce, tk, toks, batches[0][0], batches[0][1], n_pos)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"end-to-end oracle (float64, one encoder call per interaction) on the first {n_pos} "
+                                          f"positions of one history of the same workload, {dt:.1f} s; linear in interactions"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="gram", choices=["gram", "reference"])
+    ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny"])
+    ap.add_argument("--micro-batch", type=int, default=0, help="items per encoder pass (0: the workload's default)")
+    ap.add_argument("--seed", type=int, default=0)
+    args = ap.parse_args()
+    from paper_2204_04179_b200 import synth
+    shape = synth.config(args.workload)
+    if args.workload in ("kt", "nr") and not args.micro_batch:
+        args.micro_batch = 5120 if args.workload == "kt" else 0
+    if args.impl == "reference":
+        run_reference(args, shape)
+    else:
+        run_gram(args, shape)
+
+
+if __name__ == "__main__":
+    main()

@@ -204,6 +204,22 @@ gram_status gram_window_reset(gram_ctx* ctx, gram_stream stream);
  * [ceil(n_items/32)], cache fp32 [n_items, d] (converted).  NULL skips one. */
 gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache);
 
+/* --- measurement -------------------------------------------------------------
+ * Kernel kinds for gram_profile_read. */
+enum { GRAM_K_GEMM = 0, GRAM_K_ATTENTION = 1, GRAM_K_LAYERNORM = 2, GRAM_K_COLSUM = 3, GRAM_K_EMBED_POOL = 4,
+       GRAM_K_DEDUP = 5, GRAM_K_GATHER = 6, GRAM_K_ACCUMULATE = 7, GRAM_K_TASK_HEAD = 8, GRAM_K_OTHER = 9,
+       GRAM_K_COUNT = 10 };
+/* enable != 0: from now on every kernel group the library launches is bracketed by
+ * CUDA events on its stream (a few microseconds of host time per group); 0 turns
+ * it off.  Either way the totals are cleared. */
+gram_status gram_profile(gram_ctx* ctx, int enable);
+/* Synchronises the device and returns, for one kind, the totals since the last
+ * gram_profile call: device milliseconds, algorithmic work (flops for
+ * GRAM_K_GEMM and GRAM_K_ATTENTION, bytes for the others) and kernel launches. */
+gram_status gram_profile_read(gram_ctx* ctx, int kind, double* ms, double* work, int64_t* launches);
+/* Kernels this context has launched since it was created (counted always). */
+gram_status gram_launch_count(const gram_ctx* ctx, int64_t* launches);
+
 /* --- a building block, exported so that it can be tested on its own --------
  * C[M, N] = A x B with bf16 operands and fp32 accumulation on the tensor cores.
  * a_kmajor != 0: A is [M, K] row-major, else [K, M] row-major; b_kmajor != 0:

@@ -28,7 +28,10 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_get_params", "gram_get_grads", "gram_zero_grads", "gram_set_item_tokens", "gram_dedup",
            "gram_encode_unique", "gram_gather", "gram_accumulate", "gram_accumulate_multistep", "gram_touched_list",
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
-           "gram_window_reset", "gram_get_window", "gram_gemm_bf16"]
+           "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
+           "gram_launch_count"]
+
+KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other"]
 
 
 class GramConfig(C.Structure):
@@ -220,6 +223,24 @@ class Gram:
         cache = np.empty((n, d), np.float32) if want_cache else None
         self._ck(lib().gram_get_window(self._h, _ptr(table), _ptr(touched), _ptr(cache)))
         return table, touched, cache
+
+    # measurement
+    def profile(self, enable: bool):
+        self._ck(lib().gram_profile(self._h, C.c_int(int(enable))))
+
+    def profile_read(self) -> dict:
+        """{kind: dict(ms, work, launches)} since the last profile() call."""
+        out = {}
+        for k, name in enumerate(KINDS):
+            ms, work, n = C.c_double(0), C.c_double(0), C.c_int64(0)
+            self._ck(lib().gram_profile_read(self._h, C.c_int(k), C.byref(ms), C.byref(work), C.byref(n)))
+            out[name] = dict(ms=ms.value, work=work.value, launches=n.value)
+        return out
+
+    def launch_count(self) -> int:
+        n = C.c_int64(0)
+        self._ck(lib().gram_launch_count(self._h, C.byref(n)))
+        return n.value
 
     def gemm_bf16(self, A, a_kmajor, Bm, b_kmajor, Cm, bias, accumulate, M, N, K, stream=None):
         import torch

@@ -7,8 +7,23 @@
 #include "gram_internal.h"
 #include "model.h"
 
+constexpr int kProfSlots = 16384;
+struct ProfRec {
+  int kind;
+  double work;
+  int launches;
+};
+
 struct gram_ctx {
   gram_config cfg;
+  // measurement
+  int64_t launch_count = 0;
+  bool prof_on = false;
+  cudaEvent_t* prof_ev = nullptr;       // [2 * kProfSlots], created on first enable
+  ProfRec* prof_rec = nullptr;
+  int prof_used = 0;
+  double prof_ms[GRAM_K_COUNT] = {}, prof_work[GRAM_K_COUNT] = {};
+  int64_t prof_launches[GRAM_K_COUNT] = {};
   char err[512];
   int32_t* d_status = nullptr;      // device status word (first device-side error)
   IndexWorkspace iws;
@@ -25,6 +40,32 @@ void gram_set_error(gram_ctx* ctx, const char* fmt, ...) {
 }
 
 int32_t* gram_status_word(gram_ctx* ctx) { return ctx->d_status; }
+
+void gram_prof_open(gram_ctx* ctx, int kind, double work, int launches, cudaStream_t st, int* slot) {
+  *slot = -1;
+  if (!ctx) return;
+  ctx->launch_count += launches;
+  if (!ctx->prof_on || ctx->prof_used >= kProfSlots) return;
+  const int k = ctx->prof_used++;
+  ctx->prof_rec[k] = ProfRec{kind, work, launches};
+  cudaEventRecord(ctx->prof_ev[2 * k], st);
+  *slot = k;
+}
+void gram_prof_close(gram_ctx* ctx, int slot, cudaStream_t st) { cudaEventRecord(ctx->prof_ev[2 * slot + 1], st); }
+
+// folds the recorded event pairs into the per-kind totals (the device must be idle)
+static void prof_fold(gram_ctx* ctx) {
+  for (int k = 0; k < ctx->prof_used; ++k) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->prof_ev[2 * k], ctx->prof_ev[2 * k + 1]) == cudaSuccess) {
+      const ProfRec& r = ctx->prof_rec[k];
+      ctx->prof_ms[r.kind] += ms;
+      ctx->prof_work[r.kind] += r.work;
+      ctx->prof_launches[r.kind] += r.launches;
+    }
+  }
+  ctx->prof_used = 0;
+}
 IndexWorkspace* gram_index_ws(gram_ctx* ctx) { return &ctx->iws; }
 GemmWorkspace* gram_gemm_ws(gram_ctx* ctx) { return &ctx->gws; }
 const gram_config* gram_cfg(const gram_ctx* ctx) { return &ctx->cfg; }
@@ -100,6 +141,11 @@ gram_status gram_destroy(gram_ctx* ctx) {
   if (!ctx) return GRAM_OK;
   cudaDeviceSynchronize();
   if (ctx->model) model_destroy(ctx->model);
+  if (ctx->prof_ev) {
+    for (int i = 0; i < 2 * kProfSlots; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+    delete[] ctx->prof_rec;
+  }
   index_ws_free(&ctx->iws);
   gemm_ws_free(&ctx->gws);
   cudaFree(ctx->d_status);
@@ -114,6 +160,41 @@ gram_status gram_sync(gram_ctx* ctx, gram_stream stream) {
 }
 
 const char* gram_last_error(const gram_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+gram_status gram_profile(gram_ctx* ctx, int enable) {
+  if (!ctx) return GRAM_ERR_ARG;
+  GRAM_CUDA(ctx, cudaDeviceSynchronize());
+  if (enable && !ctx->prof_ev) {
+    ctx->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfSlots];
+    ctx->prof_rec = new (std::nothrow) ProfRec[kProfSlots];
+    if (!ctx->prof_ev || !ctx->prof_rec) return gram_set_error(ctx, "out of host memory"), GRAM_ERR_CUDA;
+    for (int i = 0; i < 2 * kProfSlots; ++i) GRAM_CUDA(ctx, cudaEventCreate(&ctx->prof_ev[i]));
+  }
+  ctx->prof_on = enable != 0;
+  ctx->prof_used = 0;
+  for (int k = 0; k < GRAM_K_COUNT; ++k) {
+    ctx->prof_ms[k] = 0;
+    ctx->prof_work[k] = 0;
+    ctx->prof_launches[k] = 0;
+  }
+  return GRAM_OK;
+}
+
+gram_status gram_profile_read(gram_ctx* ctx, int kind, double* ms, double* work, int64_t* launches) {
+  if (!ctx || kind < 0 || kind >= GRAM_K_COUNT) return GRAM_ERR_ARG;
+  GRAM_CUDA(ctx, cudaDeviceSynchronize());
+  prof_fold(ctx);
+  if (ms) *ms = ctx->prof_ms[kind];
+  if (work) *work = ctx->prof_work[kind];
+  if (launches) *launches = ctx->prof_launches[kind];
+  return GRAM_OK;
+}
+
+gram_status gram_launch_count(const gram_ctx* ctx, int64_t* launches) {
+  if (!ctx || !launches) return GRAM_ERR_ARG;
+  *launches = ctx->launch_count;
+  return GRAM_OK;
+}
 
 gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n_items, int32_t* d_unique,
                        int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off, int32_t* d_n_unique,

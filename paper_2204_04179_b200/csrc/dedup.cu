@@ -308,8 +308,10 @@ gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids
   const int64_t nh = (int64_t)256 * nblocks;
   const int nh_tiles = (int)ceil_div64(nh, SCAN_THREADS * 4);
   int32_t* status = gram_status_word(ctx);
+  ProfScope prof(ctx, GRAM_K_DEDUP, (16.0 * passes + 20.0) * (double)P, 5 * passes + 4, st);
 
   const int32_t* kin = d_ids;
+
   const int32_t* vin = nullptr;
   int32_t* kbuf[2] = {ws->keys0, ws->keys1};
   int32_t* vbuf[2] = {ws->vals0, ws->vals1};

@@ -291,6 +291,7 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
     return gram_set_error(ctx, "gram_gather: null buffer"), GRAM_ERR_ARG;
   int32_t* status = gram_status_word(ctx);
   const int64_t row_bytes = (int64_t)d * elem_bytes;
+  ProfScope prof(ctx, GRAM_K_GATHER, (double)row_bytes * (double)(P + (n_src_rows < P ? n_src_rows : P)) + 4.0 * P, 1, st);
   const bool vec_ok = (row_bytes % 16 == 0) && ((uintptr_t)d_src % 16 == 0) && ((uintptr_t)d_E % 16 == 0);
   if (vec_ok) {
     const int nvec = (int)(row_bytes / 16);
@@ -341,6 +342,8 @@ gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_i
   if (nchunks > kAccMaxChunks) nchunks = kAccMaxChunks;
   const int64_t R = ceil_div64(P, nchunks);
   nchunks = ceil_div64(P, R);
+  ProfScope prof(ctx, GRAM_K_ACCUMULATE, (in_bf16 ? 2.0 : 4.0) * (double)P * d + 4.0 * (double)U * d + 4.0 * P + 4.0 * (U + 1),
+                 nchunks > 1 ? 2 : 1, st);
   if (d >= 256) {
     if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
     else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
@@ -355,6 +358,7 @@ gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_i
 gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items, uint32_t* d_bits,
                                 cudaStream_t st) {
   if (U <= 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_OTHER, 8.0 * U, 1, st);
   touched_mark_kernel<<<ceil_div(U, 256), 256, 0, st>>>(d_unique, U, n_items, d_bits, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -363,6 +367,7 @@ gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t 
 gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n_items, int32_t* d_list,
                                 int32_t* d_count, cudaStream_t st) {
   if (n_items <= 0 || !d_bits || !d_list || !d_count) return gram_set_error(ctx, "gram_touched_list: bad argument"), GRAM_ERR_ARG;
+  ProfScope prof(ctx, GRAM_K_OTHER, (double)n_items / 8.0, 1, st);
   touched_list_kernel<<<1, 1024, 0, st>>>(d_bits, n_items, d_list, d_count);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;

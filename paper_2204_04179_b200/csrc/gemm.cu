@@ -553,6 +553,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
            epi.gelu, epi.accumulate};
   if (dtype == GRAM_F32) {
     if (!c_f32) return gram_set_error(ctx, "gemm: fp32 operands need an fp32 result"), GRAM_ERR_UNSUPPORTED;
+    ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, 1, st);
     dim3 grid((unsigned)ceil_div(N, ST), (unsigned)ceil_div64(M, ST));
     gemm_f32_kernel<<<grid, 256, 0, st>>>((const float*)A, a_kmajor ? lda : 1, a_kmajor ? 1 : lda, (const float*)B,
                                           b_kmajor ? ldb : 1, b_kmajor ? 1 : ldb, (float*)C, ldc, M, N, K, e);
@@ -595,6 +596,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   splits = ceil_div(args.num_kb, args.kb_per_split);
   args.splits = splits;
   cudaError_t err;
+  ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, splits > 1 ? 2 : 1, st);
   const int grid = (int)((tiles * splits < kNumSMs) ? tiles * splits : kNumSMs);
   if (splits > 1) {
     args.C = ws->splitk;

@@ -76,6 +76,23 @@ gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t 
 gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n_items, int32_t* d_list,
                                 int32_t* d_count, cudaStream_t st);
 
+// ---------------------------------------------------------------------------
+// measurement: every launch wrapper opens a ProfScope.  It always counts the launches; when
+// profiling is on it also brackets them with CUDA events on the launching stream and files the
+// elapsed time and the algorithmic work (flops or bytes) under the kernel kind.
+// ---------------------------------------------------------------------------
+void gram_prof_open(gram_ctx* ctx, int kind, double work, int launches, cudaStream_t st, int* slot);
+void gram_prof_close(gram_ctx* ctx, int slot, cudaStream_t st);
+struct ProfScope {
+  gram_ctx* ctx;
+  cudaStream_t st;
+  int slot = -1;
+  ProfScope(gram_ctx* c, int kind, double work, int launches, cudaStream_t s) : ctx(c), st(s) {
+    gram_prof_open(c, kind, work, launches, s, &slot);
+  }
+  ~ProfScope() { if (slot >= 0) gram_prof_close(ctx, slot, st); }
+};
+
 // the device status word: kernels record the first error kind they meet
 __device__ __forceinline__ void gram_device_fail(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 int32_t* gram_status_word(gram_ctx* ctx);

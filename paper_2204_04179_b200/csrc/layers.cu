@@ -672,6 +672,7 @@ gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32
   const int64_t n_tok = (int64_t)n_chunk * l_t;
   if (n_tok == 0) return GRAM_OK;
   const int blocks = grid_for(n_tok * 32, 256, kNumSMs * 8);
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 8.0 * (double)n_tok * d, 1, st);
   embed_fwd_kernel<<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t, vocab, d, tok_emb,
                                            pos_emb, z0, tok_ids, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
@@ -683,6 +684,7 @@ gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const fl
   if (rows == 0) return GRAM_OK;
   if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
   const int blocks = grid_for(rows * 32, 256, kNumSMs * 8);
+  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (4.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
   DISPATCH_T(dtype, DISPATCH_NP(d, ln_fwd_kernel<T, NP><<<blocks, 256, 0, st>>>(z, gamma, beta, (T*)y, mean, rstd, rows, d)));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -695,6 +697,7 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
   if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
   const int blocks = grid_for(rows * 32, 256, kRedBlocks);
   const size_t smem = (size_t)2 * d * sizeof(float);
+  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st);
   DISPATCH_T(dtype, DISPATCH_NP(d, ln_bwd_kernel<T, NP><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
   reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
@@ -708,6 +711,7 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
+  ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
     attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale);
@@ -723,6 +727,7 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
+  ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
     attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);
@@ -742,6 +747,7 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
   const int64_t per = ceil_div64(rows, rb);
   rb = ceil_div64(rows, per);
   dim3 grid((unsigned)ceil_div(N, 64), (unsigned)rb);
+  ProfScope prof(ctx, GRAM_K_COLSUM, (double)rows * N * (dtype == GRAM_BF16 ? 2.0 : 4.0), 2, st);
   DISPATCH_T(dtype, colsum_kernel<T><<<grid, 256, 0, st>>>((const T*)X, rows, N, per, scratch));
   reduce_partials_kernel<<<ceil_div(N, 256), 256, 0, st>>>(scratch, (int)rb, (int64_t)N, N, out, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
@@ -752,6 +758,7 @@ gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_
                                        cudaStream_t st) {
   if (n_groups == 0) return GRAM_OK;
   const int64_t n = (int64_t)period * d;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n_groups * period * d, 1, st);
   periodic_rowsum_kernel<<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>(X, n_groups, period, d, out);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -760,6 +767,7 @@ gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
                          cudaStream_t st) {
   if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (pooling == GRAM_POOL_CLS ? 2 : l_t + 1), 1, st);
   pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -768,6 +776,7 @@ gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n,
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
                           cudaStream_t st) {
   if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (l_t + 1), 1, st);
   pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -777,6 +786,7 @@ gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const flo
                              const int32_t* labels, float* x, void* x_b, int B, int L, int d, cudaStream_t st) {
   const int64_t P = (int64_t)B * L;
   if (P == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)P * d * (8.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
   DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)ceil_div64(P * d, 256), 256, 0, st>>>(E, pos, resp, labels, x, (T*)x_b, P, L, d));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -790,6 +800,7 @@ gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w
   if (blocks > kRedBlocks) blocks = kRedBlocks;
   const int64_t pstride = d + 2;
   const size_t smem = (size_t)(d + 2) * sizeof(float);
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 12.0 * (double)P * d, 2, st);
   DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>(y, w, b, labels, dy, (T*)dy_b, scratch, P, d, pstride));
   kt_head_reduce_kernel<<<ceil_div(d + 2, 256), 256, 0, st>>>(scratch, blocks, pstride, d, 1.f / (float)P, dw, db, loss);
   GRAM_LAUNCH_CHECK(ctx);
@@ -802,6 +813,7 @@ gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* lab
   if (B == 0) return GRAM_OK;
   if ((size_t)L * 3 * d * sizeof(float) > kRedScratchBytes) return gram_set_error(ctx, "kt task: L*d too large for the reduction scratch"), GRAM_ERR_UNSUPPORTED;
   dim3 grid((unsigned)ceil_div(d, 128), (unsigned)L);
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 8.0 * (double)B * L * d, 2, st);
   kt_input_bwd_kernel<<<grid, 128, 0, st>>>(dx, labels, dE, dpos, scratch, B, L, d);
   reduce_partials_kernel<<<ceil_div(3 * d, 256), 256, 0, st>>>(scratch, L, (int64_t)3 * d, 3 * d, dresp, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
@@ -814,6 +826,7 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
   if (B == 0) return GRAM_OK;
   if (n_cand <= 0 || n_cand >= L) return gram_set_error(ctx, "nr task: need 0 < n_cand < L"), GRAM_ERR_ARG;
   const size_t smem = ((size_t)2 * L + 2 * d + n_cand) * sizeof(float);
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)B * L * (8.0 * d + 4.0 * d_a), 2, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, nr_user_kernel<T>, smem));
     nr_user_kernel<T><<<B, 256, smem, st>>>(E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B);
@@ -825,6 +838,7 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
 
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_OTHER, 6.0 * (double)n, 1, st);
   f32_to_bf16_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(in, out, n);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -832,12 +846,16 @@ gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_
 gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   if (dtype == GRAM_F32) GRAM_CUDA(ctx, cudaMemcpyAsync(out, in, n * sizeof(float), cudaMemcpyDeviceToDevice, st));
-  else bf16_to_f32_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>((const bf16*)in, out, n);
+  else {
+    ProfScope prof(ctx, GRAM_K_OTHER, 6.0 * (double)n, 1, st);
+    bf16_to_f32_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>((const bf16*)in, out, n);
+  }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st) {
   if (n == 0 || lr == 0.f) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_OTHER, 12.0 * (double)n, 1, st);
   sgd_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(w, g, lr, n);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -845,6 +863,7 @@ gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t
 gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_OTHER, (double)n * d * (4.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
   DISPATCH_T(dtype, scatter_rows_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(src, index, n, d, n_dst_rows, (T*)dst, gram_status_word(ctx)));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
