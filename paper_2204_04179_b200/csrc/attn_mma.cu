@@ -1,0 +1,324 @@
+// Attention over short sequences (S <= 128 tokens, head width 32 or 64) with bf16 tensor-core
+// products and fp32 softmax.  One block owns one (sequence, head): Q, K, V (and dO in the backward)
+// live in shared memory for the whole block, a warp owns 16 query rows (forward, first half of the
+// backward) or 16 key rows (second half of the backward), and score tiles never leave registers.
+// The sequences are far shorter than a 128-row tcgen05 tile, and attention is ~2% of the encoder's
+// flops, so this uses the warp-level m16n8k16 MMA; the kernel is bound by reading qkv once.
+#include "layers.h"
+
+namespace {
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2(float x, float y) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t ld32(const bf16* p) { return *reinterpret_cast<const uint32_t*>(p); }
+__device__ __forceinline__ float quad_max(float v) {
+  v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+__device__ __forceinline__ float quad_sum(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v + __shfl_xor_sync(0xffffffffu, v, 2);
+}
+
+// Fragment conventions of m16n8k16 (g = lane / 4, q = lane % 4):
+//   A (16 x 16, row-major source X[m][k]):  a0 = X[g][2q..], a1 = X[g+8][2q..], a2 = X[g][2q+8..], a3 = X[g+8][2q+8..]
+//   B (16 x 8, source stored as Y[n][k]):   b0 = Y[g][2q..], b1 = Y[g][2q+8..]
+//   C (16 x 8):                             c0,c1 = C[g][2q, 2q+1], c2,c3 = C[g+8][2q, 2q+1]
+// Every matrix therefore sits in shared memory with its contraction index contiguous; where a
+// product needs the other orientation a transposed copy is kept (row strides are padded by 8
+// elements, which makes the 32-bit fragment loads conflict-free).
+
+// scores of 16 query rows against all SP keys: p[nt][0..3] for key tile nt, normalised probabilities on return
+template <int SP, int DH>
+__device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf16* __restrict__ Ks, int r0, int S, int causal,
+                                           float scale, int g, int q, float (&p)[SP / 8][4]) {
+  constexpr int LD = DH + 8;
+#pragma unroll
+  for (int nt = 0; nt < SP / 8; ++nt) p[nt][0] = p[nt][1] = p[nt][2] = p[nt][3] = 0.f;
+#pragma unroll
+  for (int kt = 0; kt < DH / 16; ++kt) {
+    const uint32_t a0 = ld32(Qs + (r0 + g) * LD + kt * 16 + 2 * q), a1 = ld32(Qs + (r0 + g + 8) * LD + kt * 16 + 2 * q);
+    const uint32_t a2 = ld32(Qs + (r0 + g) * LD + kt * 16 + 8 + 2 * q), a3 = ld32(Qs + (r0 + g + 8) * LD + kt * 16 + 8 + 2 * q);
+#pragma unroll
+    for (int nt = 0; nt < SP / 8; ++nt) {
+      const uint32_t b0 = ld32(Ks + (nt * 8 + g) * LD + kt * 16 + 2 * q), b1 = ld32(Ks + (nt * 8 + g) * LD + kt * 16 + 8 + 2 * q);
+      mma16816(p[nt], a0, a1, a2, a3, b0, b1);
+    }
+  }
+  const int i0 = r0 + g, i1 = r0 + g + 8;
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < SP / 8; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = nt * 8 + 2 * q + (e & 1);
+      const int i = (e < 2) ? i0 : i1;
+      const bool ok = j < S && (!causal || j <= i);
+      p[nt][e] = ok ? p[nt][e] * scale : -INFINITY;
+    }
+    m0 = fmaxf(m0, fmaxf(p[nt][0], p[nt][1]));
+    m1 = fmaxf(m1, fmaxf(p[nt][2], p[nt][3]));
+  }
+  m0 = quad_max(m0);
+  m1 = quad_max(m1);
+  if (m0 == -INFINITY) m0 = 0.f;        // a padded query row of a causal tile past S: no key is visible
+  if (m1 == -INFINITY) m1 = 0.f;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < SP / 8; ++nt) {
+    p[nt][0] = __expf(p[nt][0] - m0); p[nt][1] = __expf(p[nt][1] - m0);
+    p[nt][2] = __expf(p[nt][2] - m1); p[nt][3] = __expf(p[nt][3] - m1);
+    l0 += p[nt][0] + p[nt][1];
+    l1 += p[nt][2] + p[nt][3];
+  }
+  l0 = quad_sum(l0);
+  l1 = quad_sum(l1);
+  const float r0i = l0 > 0.f ? 1.f / l0 : 0.f, r1i = l1 > 0.f ? 1.f / l1 : 0.f;
+#pragma unroll
+  for (int nt = 0; nt < SP / 8; ++nt) {
+    p[nt][0] *= r0i; p[nt][1] *= r0i;
+    p[nt][2] *= r1i; p[nt][3] *= r1i;
+  }
+}
+
+// rows [0, S) of one head's slice of a [tokens, ld] bf16 matrix -> shared memory, row-major (dst) and,
+// when dst_t != null, transposed (dst_t[c][s]); rows S..SP-1 are zero
+template <int SP, int DH>
+__device__ __forceinline__ void load_head(const bf16* __restrict__ src, int64_t ld, int S, bf16* __restrict__ dst,
+                                          bf16* __restrict__ dst_t) {
+  constexpr int LD = DH + 8, LT = SP + 8;
+  for (int i = threadIdx.x; i < SP * (DH / 8); i += blockDim.x) {
+    const int s = i / (DH / 8), c = (i - s * (DH / 8)) * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (s < S) v = *reinterpret_cast<const uint4*>(src + (int64_t)s * ld + c);
+    if (dst) *reinterpret_cast<uint4*>(dst + s * LD + c) = v;
+    if (dst_t) {
+      const bf16* e = reinterpret_cast<const bf16*>(&v);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dst_t[(c + k) * LT + s] = e[k];
+    }
+  }
+}
+
+template <int SP, int DH>
+__global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
+                                                           int n_heads, int causal, float scale) {
+  constexpr int LD = DH + 8, LT = SP + 8;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
+  bf16* Ks = Qs + SP * LD;
+  bf16* Vt = Ks + SP * LD;                       // [DH][SP + 8]
+  const int64_t seq = blockIdx.x / n_heads;
+  const int h = blockIdx.x % n_heads;
+  const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
+  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs, nullptr);
+  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks, nullptr);
+  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, nullptr, Vt);
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  for (int r0 = warp * 16; r0 < S; r0 += 64) {
+    float p[SP / 8][4];
+    score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
+    float o[DH / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+#pragma unroll
+    for (int kt = 0; kt < SP / 16; ++kt) {
+      const uint32_t a0 = pack2(p[2 * kt][0], p[2 * kt][1]), a1 = pack2(p[2 * kt][2], p[2 * kt][3]);
+      const uint32_t a2 = pack2(p[2 * kt + 1][0], p[2 * kt + 1][1]), a3 = pack2(p[2 * kt + 1][2], p[2 * kt + 1][3]);
+#pragma unroll
+      for (int nt = 0; nt < DH / 8; ++nt) {
+        const uint32_t b0 = ld32(Vt + (nt * 8 + g) * LT + kt * 16 + 2 * q), b1 = ld32(Vt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
+        mma16816(o[nt], a0, a1, a2, a3, b0, b1);
+      }
+    }
+    bf16* ob = out + seq * S * (int64_t)d + h * DH;
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) {
+      const int c = nt * 8 + 2 * q;
+      if (r0 + g < S) *reinterpret_cast<uint32_t*>(ob + (int64_t)(r0 + g) * d + c) = pack2(o[nt][0], o[nt][1]);
+      if (r0 + g + 8 < S) *reinterpret_cast<uint32_t*>(ob + (int64_t)(r0 + g + 8) * d + c) = pack2(o[nt][2], o[nt][3]);
+    }
+  }
+}
+
+template <int SP, int DH>
+__global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
+                                                           bf16* __restrict__ dqkv, int S, int d, int n_heads, int causal,
+                                                           float scale) {
+  constexpr int LD = DH + 8, LT = SP + 8;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // row-major [SP][DH+8]
+  bf16* Ks = Qs + SP * LD;
+  bf16* Vs = Ks + SP * LD;
+  bf16* dOs = Vs + SP * LD;
+  bf16* Qt = dOs + SP * LD;                       // transposed [DH][SP+8]
+  bf16* Kt = Qt + DH * LT;
+  bf16* dOt = Kt + DH * LT;
+  bf16* Pt = dOt + DH * LT;                       // [key j][query i], [SP][SP+8]
+  bf16* dSt = Pt + SP * LT;
+  const int64_t seq = blockIdx.x / n_heads;
+  const int h = blockIdx.x % n_heads;
+  const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
+  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs, Qt);
+  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks, Kt);
+  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs, nullptr);
+  load_head<SP, DH>(dctx + seq * S * (int64_t)d + h * DH, d, S, dOs, dOt);
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  bf16* dq = dqkv + seq * S * 3 * (int64_t)d + h * DH;
+  // ---- first half: 16 query rows per warp: P, dS (kept transposed in shared memory), dQ ----
+  for (int r0 = warp * 16; r0 < SP; r0 += 64) {
+    float p[SP / 8][4];
+    score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
+    float dp[SP / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
+#pragma unroll
+    for (int kt = 0; kt < DH / 16; ++kt) {        // dP = dO V^T
+      const uint32_t a0 = ld32(dOs + (r0 + g) * LD + kt * 16 + 2 * q), a1 = ld32(dOs + (r0 + g + 8) * LD + kt * 16 + 2 * q);
+      const uint32_t a2 = ld32(dOs + (r0 + g) * LD + kt * 16 + 8 + 2 * q), a3 = ld32(dOs + (r0 + g + 8) * LD + kt * 16 + 8 + 2 * q);
+#pragma unroll
+      for (int nt = 0; nt < SP / 8; ++nt) {
+        const uint32_t b0 = ld32(Vs + (nt * 8 + g) * LD + kt * 16 + 2 * q), b1 = ld32(Vs + (nt * 8 + g) * LD + kt * 16 + 8 + 2 * q);
+        mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
+      }
+    }
+    float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < SP / 8; ++nt) {
+      d0 += p[nt][0] * dp[nt][0] + p[nt][1] * dp[nt][1];
+      d1 += p[nt][2] * dp[nt][2] + p[nt][3] * dp[nt][3];
+    }
+    d0 = quad_sum(d0);
+    d1 = quad_sum(d1);
+#pragma unroll
+    for (int nt = 0; nt < SP / 8; ++nt) {         // dS = P (dP - delta) / sqrt(dh); stored as [j][i]
+      dp[nt][0] = p[nt][0] * (dp[nt][0] - d0) * scale; dp[nt][1] = p[nt][1] * (dp[nt][1] - d0) * scale;
+      dp[nt][2] = p[nt][2] * (dp[nt][2] - d1) * scale; dp[nt][3] = p[nt][3] * (dp[nt][3] - d1) * scale;
+      const int j = nt * 8 + 2 * q;
+      Pt[j * LT + r0 + g] = __float2bfloat16(p[nt][0]);       Pt[(j + 1) * LT + r0 + g] = __float2bfloat16(p[nt][1]);
+      Pt[j * LT + r0 + g + 8] = __float2bfloat16(p[nt][2]);   Pt[(j + 1) * LT + r0 + g + 8] = __float2bfloat16(p[nt][3]);
+      dSt[j * LT + r0 + g] = __float2bfloat16(dp[nt][0]);     dSt[(j + 1) * LT + r0 + g] = __float2bfloat16(dp[nt][1]);
+      dSt[j * LT + r0 + g + 8] = __float2bfloat16(dp[nt][2]); dSt[(j + 1) * LT + r0 + g + 8] = __float2bfloat16(dp[nt][3]);
+    }
+    float o[DH / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+#pragma unroll
+    for (int kt = 0; kt < SP / 16; ++kt) {        // dQ = dS K
+      const uint32_t a0 = pack2(dp[2 * kt][0], dp[2 * kt][1]), a1 = pack2(dp[2 * kt][2], dp[2 * kt][3]);
+      const uint32_t a2 = pack2(dp[2 * kt + 1][0], dp[2 * kt + 1][1]), a3 = pack2(dp[2 * kt + 1][2], dp[2 * kt + 1][3]);
+#pragma unroll
+      for (int nt = 0; nt < DH / 8; ++nt) {
+        const uint32_t b0 = ld32(Kt + (nt * 8 + g) * LT + kt * 16 + 2 * q), b1 = ld32(Kt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
+        mma16816(o[nt], a0, a1, a2, a3, b0, b1);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) {
+      const int c = nt * 8 + 2 * q;
+      if (r0 + g < S) *reinterpret_cast<uint32_t*>(dq + (int64_t)(r0 + g) * 3 * d + c) = pack2(o[nt][0], o[nt][1]);
+      if (r0 + g + 8 < S) *reinterpret_cast<uint32_t*>(dq + (int64_t)(r0 + g + 8) * 3 * d + c) = pack2(o[nt][2], o[nt][3]);
+    }
+  }
+  __syncthreads();
+  // ---- second half: 16 key rows per warp: dK = dS^T Q, dV = P^T dO ----
+  for (int j0 = warp * 16; j0 < S; j0 += 64) {
+    float dk[DH / 8][4], dv[DH / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) {
+      dk[nt][0] = dk[nt][1] = dk[nt][2] = dk[nt][3] = 0.f;
+      dv[nt][0] = dv[nt][1] = dv[nt][2] = dv[nt][3] = 0.f;
+    }
+#pragma unroll
+    for (int kt = 0; kt < SP / 16; ++kt) {
+      const uint32_t s0 = ld32(dSt + (j0 + g) * LT + kt * 16 + 2 * q), s1 = ld32(dSt + (j0 + g + 8) * LT + kt * 16 + 2 * q);
+      const uint32_t s2 = ld32(dSt + (j0 + g) * LT + kt * 16 + 8 + 2 * q), s3 = ld32(dSt + (j0 + g + 8) * LT + kt * 16 + 8 + 2 * q);
+      const uint32_t p0 = ld32(Pt + (j0 + g) * LT + kt * 16 + 2 * q), p1 = ld32(Pt + (j0 + g + 8) * LT + kt * 16 + 2 * q);
+      const uint32_t p2 = ld32(Pt + (j0 + g) * LT + kt * 16 + 8 + 2 * q), p3 = ld32(Pt + (j0 + g + 8) * LT + kt * 16 + 8 + 2 * q);
+#pragma unroll
+      for (int nt = 0; nt < DH / 8; ++nt) {
+        const uint32_t bq0 = ld32(Qt + (nt * 8 + g) * LT + kt * 16 + 2 * q), bq1 = ld32(Qt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
+        mma16816(dk[nt], s0, s1, s2, s3, bq0, bq1);
+        const uint32_t bo0 = ld32(dOt + (nt * 8 + g) * LT + kt * 16 + 2 * q), bo1 = ld32(dOt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
+        mma16816(dv[nt], p0, p1, p2, p3, bo0, bo1);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) {
+      const int c = nt * 8 + 2 * q;
+      if (j0 + g < S) {
+        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g) * 3 * d + d + c) = pack2(dk[nt][0], dk[nt][1]);
+        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g) * 3 * d + 2 * d + c) = pack2(dv[nt][0], dv[nt][1]);
+      }
+      if (j0 + g + 8 < S) {
+        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g + 8) * 3 * d + d + c) = pack2(dk[nt][2], dk[nt][3]);
+        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g + 8) * 3 * d + 2 * d + c) = pack2(dv[nt][2], dv[nt][3]);
+      }
+    }
+  }
+}
+
+template <int SP, int DH>
+gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
+                       cudaStream_t st) {
+  constexpr size_t smem = ((size_t)2 * SP * (DH + 8) + (size_t)DH * (SP + 8)) * 2;
+  auto kern = attn_fwd_mma_kernel<SP, DH>;
+  if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+template <int SP, int DH>
+gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, int64_t n_seq, int S, int d, int n_heads,
+                       int causal, cudaStream_t st) {
+  constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)3 * DH * (SP + 8) + (size_t)2 * SP * (SP + 8)) * 2;
+  static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
+  auto kern = attn_bwd_mma_kernel<SP, DH>;
+  if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+}  // namespace
+
+bool attention_mma_supported(int S, int d, int n_heads) {
+  const int dh = n_heads > 0 ? d / n_heads : 0;
+  return S >= 1 && S <= 128 && (dh == 32 || dh == 64) && dh * n_heads == d && d % 8 == 0;
+}
+
+#define ATTN_DISPATCH(FN, ...)                                                      \
+  do {                                                                              \
+    const int dh = d / n_heads;                                                     \
+    if (dh == 64) {                                                                 \
+      if (S <= 32) return FN<32, 64>(__VA_ARGS__);                                  \
+      if (S <= 64) return FN<64, 64>(__VA_ARGS__);                                  \
+      if (S <= 96) return FN<96, 64>(__VA_ARGS__);                                  \
+      return FN<128, 64>(__VA_ARGS__);                                              \
+    } else {                                                                        \
+      if (S <= 32) return FN<32, 32>(__VA_ARGS__);                                  \
+      if (S <= 64) return FN<64, 32>(__VA_ARGS__);                                  \
+      if (S <= 96) return FN<96, 32>(__VA_ARGS__);                                  \
+      return FN<128, 32>(__VA_ARGS__);                                              \
+    }                                                                               \
+  } while (0)
+
+gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
+                                  int causal, cudaStream_t st) {
+  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, st);
+}
+gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq, int S, int d,
+                                   int n_heads, int causal, cudaStream_t st) {
+  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, n_seq, S, d, n_heads, causal, st);
+}

@@ -712,6 +712,8 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
+  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
+    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
     attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale);
@@ -728,6 +730,8 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
+  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
+    return attention_backward_mma(ctx, qkv, dctx, dqkv, n_seq, S, d, n_heads, causal, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
     attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);

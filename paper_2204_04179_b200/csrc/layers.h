@@ -39,6 +39,13 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq,
                                int S, int d, int n_heads, int causal, cudaStream_t st);
 
+// the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
+bool attention_mma_supported(int S, int d, int n_heads);
+gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
+                                  int causal, cudaStream_t st);
+gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq, int S, int d,
+                                   int n_heads, int causal, cudaStream_t st);
+
 // out[n] += sum_rows X[r, n]   (X operand-typed)
 gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t rows, int N, float* out, float* scratch,
                               cudaStream_t st);

@@ -30,6 +30,11 @@ CASES = {
     "tiny_bf16": synth.config("tiny").replace(dtype="bf16"),
     "bf16_cls_full": small(dtype="bf16", pooling="cls", task_attn_only=False, d=64, d_ff=128, task_d_ff=128),
     "bf16_nr": small(dtype="bf16", task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls", d=64, d_ff=128),
+    # sequences that span several 16-row attention tiles with a ragged tail (70 tokens, 100 positions)
+    "long_seq": small(l_t=70, L=100, B=2, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30, task_attn_only=False),
+    "bf16_long_seq": small(dtype="bf16", l_t=70, L=100, B=2, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30,
+                           task_attn_only=False),
+    "bf16_seq128": small(dtype="bf16", l_t=128, L=128, B=1, d=64, n_heads=2, d_ff=64, task_d_ff=64, n_items=12, pooling="cls"),
 }
 
 
