@@ -227,6 +227,7 @@ def run_gram(args, shape):
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     launches = g.launch_count() - launches0
     kinds = g.profile_read()
+    sites = g.profile_dump()
     g.profile(False)
 
     # ---- end to end: host buffers through gram_step_host (copies inside the timed region) ----
@@ -279,6 +280,10 @@ def run_gram(args, shape):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * P, "d2h_bytes_per_step": 12,
                 "ms_per_step": ms_e2e / args.steps},
         "roofline": roofline, "stage_ms": stage_ms, "kernel_kinds": per_kind,
+        "call_sites": {t: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps,
+                           ("TFLOP/s" if v["kind"] in ("gemm", "attention") else "GB/s"):
+                               (v["work"] / (v["ms"] / 1e3) / (1e12 if v["kind"] in ("gemm", "attention") else 1e9)) if v["ms"] > 0 else 0.0}
+                       for t, v in sites.items()},
     }
     g.close()
     if world == 1:

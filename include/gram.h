@@ -217,6 +217,9 @@ gram_status gram_profile(gram_ctx* ctx, int enable);
  * gram_profile call: device milliseconds, algorithmic work (flops for
  * GRAM_K_GEMM and GRAM_K_ATTENTION, bytes for the others) and kernel launches. */
 gram_status gram_profile_read(gram_ctx* ctx, int kind, double* ms, double* work, int64_t* launches);
+/* The same totals per call site, as text: one line "tag kind ms work launches"
+ * per tag (the matrix products are tagged by their role, e.g. fwd_ffn1). */
+gram_status gram_profile_dump(gram_ctx* ctx, char* h_text, size_t n);
 /* Kernels this context has launched since it was created (counted always). */
 gram_status gram_launch_count(const gram_ctx* ctx, int64_t* launches);
 

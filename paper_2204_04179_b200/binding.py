@@ -29,7 +29,7 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_encode_unique", "gram_gather", "gram_accumulate", "gram_accumulate_multistep", "gram_touched_list",
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
-           "gram_launch_count"]
+           "gram_launch_count", "gram_profile_dump"]
 
 KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other"]
 
@@ -235,6 +235,16 @@ class Gram:
             ms, work, n = C.c_double(0), C.c_double(0), C.c_int64(0)
             self._ck(lib().gram_profile_read(self._h, C.c_int(k), C.byref(ms), C.byref(work), C.byref(n)))
             out[name] = dict(ms=ms.value, work=work.value, launches=n.value)
+        return out
+
+    def profile_dump(self) -> dict:
+        """{tag: dict(kind, ms, work, launches)} per call site since the last profile() call."""
+        buf = C.create_string_buffer(16384)
+        self._ck(lib().gram_profile_dump(self._h, buf, C.c_size_t(len(buf))))
+        out = {}
+        for line in buf.value.decode().splitlines():
+            tag, kind, ms, work, n = line.split()
+            out[tag] = dict(kind=KINDS[int(kind)], ms=float(ms), work=float(work), launches=int(n))
         return out
 
     def launch_count(self) -> int:

@@ -10,8 +10,16 @@
 constexpr int kProfSlots = 16384;
 struct ProfRec {
   int kind;
+  const char* tag;
   double work;
   int launches;
+};
+constexpr int kProfTags = 64;
+struct ProfTag {
+  const char* tag;
+  int kind;
+  double ms, work;
+  int64_t launches;
 };
 
 struct gram_ctx {
@@ -24,6 +32,8 @@ struct gram_ctx {
   int prof_used = 0;
   double prof_ms[GRAM_K_COUNT] = {}, prof_work[GRAM_K_COUNT] = {};
   int64_t prof_launches[GRAM_K_COUNT] = {};
+  ProfTag prof_tags[kProfTags] = {};
+  int prof_ntags = 0;
   char err[512];
   int32_t* d_status = nullptr;      // device status word (first device-side error)
   IndexWorkspace iws;
@@ -41,13 +51,13 @@ void gram_set_error(gram_ctx* ctx, const char* fmt, ...) {
 
 int32_t* gram_status_word(gram_ctx* ctx) { return ctx->d_status; }
 
-void gram_prof_open(gram_ctx* ctx, int kind, double work, int launches, cudaStream_t st, int* slot) {
+void gram_prof_open(gram_ctx* ctx, int kind, const char* tag, double work, int launches, cudaStream_t st, int* slot) {
   *slot = -1;
   if (!ctx) return;
   ctx->launch_count += launches;
   if (!ctx->prof_on || ctx->prof_used >= kProfSlots) return;
   const int k = ctx->prof_used++;
-  ctx->prof_rec[k] = ProfRec{kind, work, launches};
+  ctx->prof_rec[k] = ProfRec{kind, tag, work, launches};
   cudaEventRecord(ctx->prof_ev[2 * k], st);
   *slot = k;
 }
@@ -62,6 +72,16 @@ static void prof_fold(gram_ctx* ctx) {
       ctx->prof_ms[r.kind] += ms;
       ctx->prof_work[r.kind] += r.work;
       ctx->prof_launches[r.kind] += r.launches;
+      if (r.tag) {
+        int t = 0;
+        while (t < ctx->prof_ntags && ctx->prof_tags[t].tag != r.tag && strcmp(ctx->prof_tags[t].tag, r.tag) != 0) ++t;
+        if (t == ctx->prof_ntags && t < kProfTags) ctx->prof_tags[ctx->prof_ntags++] = ProfTag{r.tag, r.kind, 0, 0, 0};
+        if (t < kProfTags) {
+          ctx->prof_tags[t].ms += ms;
+          ctx->prof_tags[t].work += r.work;
+          ctx->prof_tags[t].launches += r.launches;
+        }
+      }
     }
   }
   ctx->prof_used = 0;
@@ -172,6 +192,7 @@ gram_status gram_profile(gram_ctx* ctx, int enable) {
   }
   ctx->prof_on = enable != 0;
   ctx->prof_used = 0;
+  ctx->prof_ntags = 0;
   for (int k = 0; k < GRAM_K_COUNT; ++k) {
     ctx->prof_ms[k] = 0;
     ctx->prof_work[k] = 0;
@@ -187,6 +208,19 @@ gram_status gram_profile_read(gram_ctx* ctx, int kind, double* ms, double* work,
   if (ms) *ms = ctx->prof_ms[kind];
   if (work) *work = ctx->prof_work[kind];
   if (launches) *launches = ctx->prof_launches[kind];
+  return GRAM_OK;
+}
+
+gram_status gram_profile_dump(gram_ctx* ctx, char* h_text, size_t n) {
+  if (!ctx || !h_text || n == 0) return GRAM_ERR_ARG;
+  GRAM_CUDA(ctx, cudaDeviceSynchronize());
+  prof_fold(ctx);
+  size_t o = 0;
+  h_text[0] = 0;
+  for (int t = 0; t < ctx->prof_ntags && o + 128 < n; ++t) {
+    const ProfTag& g = ctx->prof_tags[t];
+    o += (size_t)snprintf(h_text + o, n - o, "%s %d %.6f %.6e %lld\n", g.tag, g.kind, g.ms, g.work, (long long)g.launches);
+  }
   return GRAM_OK;
 }
 

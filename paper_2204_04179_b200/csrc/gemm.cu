@@ -1,5 +1,5 @@
 // Matrix products.  bf16: a persistent, warp-specialised tcgen05 kernel (one TMA producer warp, one
-// MMA-issuing warp, four epilogue warps; operands staged in 128-byte-swizzled shared memory by TMA,
+// MMA-issuing warp, eight epilogue warps; operands staged in 128-byte-swizzled shared memory by TMA,
 // fp32 accumulators double-buffered in tensor memory so that the epilogue of one tile overlaps the
 // main loop of the next).  fp32: a plain tiled CUDA-core kernel for the small fp32 configuration.
 #include <cuda.h>
@@ -38,10 +38,10 @@ __device__ __forceinline__ void epilogue_store(const EpiDev& e, CT* C, int64_t l
   float v = acc + (e.bias ? e.bias[n] : 0.f);
   const int64_t o = m * ldc + n;
   if (e.gelu) {
-    if (e.pre) st_c<OT>(reinterpret_cast<OT*>(e.pre) + o, v);
+    if (e.pre) st_c<OT>(reinterpret_cast<OT*>(e.pre) + o, gelu_grad_f(v));
     v = gelu_f(v);
   }
-  if (e.dgelu_pre) v *= gelu_grad_f(ld_c<OT>(reinterpret_cast<const OT*>(e.dgelu_pre) + o));
+  if (e.dgelu_pre) v *= ld_c<OT>(reinterpret_cast<const OT*>(e.dgelu_pre) + o);
   if (e.res) {
     float r = e.res[o];
     if (e.res_mean) r = (r - e.res_mean[m]) * e.res_rstd[m] * e.res_gamma[n] + e.res_beta[n];
@@ -52,74 +52,91 @@ __device__ __forceinline__ void epilogue_store(const EpiDev& e, CT* C, int64_t l
   if (e.copy_out) st_c<OT>(reinterpret_cast<OT*>(e.copy_out) + o, v);
 }
 
-// eight consecutive columns n..n+7 of row m (n and ldc multiples of 8): 16-byte accesses throughout
-__device__ __forceinline__ void ld8(const float* p, float (&x)[8]) {
-  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
-  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+// four consecutive columns n..n+3 of row m (n, ldc multiples of 4): the unit of the coalesced epilogue
+__device__ __forceinline__ void ld4(const float* p, float (&x)[4]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
 }
-__device__ __forceinline__ void ld8(const bf16* p, float (&x)[8]) {
-  const uint4 u = *reinterpret_cast<const uint4*>(p);
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
-    x[2 * i] = f.x;
-    x[2 * i + 1] = f.y;
-  }
+__device__ __forceinline__ void ld4(const bf16* p, float (&x)[4]) {
+  const uint2 u = *reinterpret_cast<const uint2*>(p);
+  const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+  const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+  x[0] = f0.x; x[1] = f0.y; x[2] = f1.x; x[3] = f1.y;
 }
-__device__ __forceinline__ void st8(float* p, const float (&x)[8]) {
+__device__ __forceinline__ void st4(float* p, const float (&x)[4]) {
   *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
-  *reinterpret_cast<float4*>(p + 4) = make_float4(x[4], x[5], x[6], x[7]);
 }
-__device__ __forceinline__ void st8(bf16* p, const float (&x)[8]) {
-  uint32_t w[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
-    w[i] = *reinterpret_cast<uint32_t*>(&h);
-  }
-  *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+__device__ __forceinline__ void st4(bf16* p, const float (&x)[4]) {
+  __nv_bfloat162 h0 = __floats2bfloat162_rn(x[0], x[1]), h1 = __floats2bfloat162_rn(x[2], x[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
 }
 
+// GELU and its derivative for the tensor-core epilogue.  erf comes from the rational approximation
+// 7.1.26 of Abramowitz & Stegun, erf(y) = 1 - (a1 t + ... + a5 t^5) exp(-y^2), t = 1 / (1 + p y), whose
+// absolute error is below 1.5e-7: far under the bf16 resolution of the values that are stored.  With
+// y = |x| / sqrt(2) the exponential exp(-x^2 / 2) is also the Gaussian density the derivative needs.
+__device__ __forceinline__ void gelu_parts(float x, float& cdf, float& pdf) {
+  const float ax = fabsf(x);
+  const float ex = __expf(-0.5f * x * x);
+  const float t = __fdividef(1.f, 1.f + 0.3275911f * 0.70710678f * ax);
+  const float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
+  const float erf_abs = 1.f - poly * ex;                  // erf(|x| / sqrt 2)
+  cdf = 0.5f * (1.f + copysignf(erf_abs, x));
+  pdf = 0.39894228f * ex;
+}
+
+// what one lane reads before it may store anything for its 4 columns of one row
+struct EpiLoads {
+  float res[4];
+  float pre[4];
+  float acc[4];
+};
 template <typename CT>
-__device__ __forceinline__ void epilogue_store8(const EpiDev& e, CT* C, int64_t ldc, int64_t m, int n, float (&v)[8],
-                                                float mu, float rs) {
+__device__ __forceinline__ void epilogue_load4(const EpiDev& e, const CT* C, int64_t ldc, int64_t m, int n, EpiLoads& L) {
   const int64_t o = m * ldc + n;
-  float t[8];
+  if (e.res) ld4(e.res + o, L.res);
+  if (e.dgelu_pre) ld4(reinterpret_cast<const bf16*>(e.dgelu_pre) + o, L.pre);
+  if (e.accumulate) ld4(reinterpret_cast<const float*>(C) + o, L.acc);      // accumulation is offered for fp32 C only
+}
+template <typename CT>
+__device__ __forceinline__ void epilogue_store4(const EpiDev& e, CT* C, int64_t ldc, int64_t m, int n, float (&v)[4],
+                                                const EpiLoads& L, const float (&bias)[4], const float (&gam)[4],
+                                                const float (&bet)[4], float mu, float rs) {
+  const int64_t o = m * ldc + n;
   if (e.bias) {
-    ld8(e.bias + n, t);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] += t[i];
+    for (int i = 0; i < 4; ++i) v[i] += bias[i];
   }
   if (e.gelu) {
-    if (e.pre) st8(reinterpret_cast<bf16*>(e.pre) + o, v);
+    float dg[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = gelu_f(v[i]);
+    for (int i = 0; i < 4; ++i) {
+      float c, p;
+      gelu_parts(v[i], c, p);
+      dg[i] = c + v[i] * p;        // gelu'(v), kept for the backward pass
+      v[i] = v[i] * c;             // gelu(v)
+    }
+    if (e.pre) st4(reinterpret_cast<bf16*>(e.pre) + o, dg);
   }
   if (e.dgelu_pre) {
-    ld8(reinterpret_cast<const bf16*>(e.dgelu_pre) + o, t);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] *= gelu_grad_f(t[i]);
+    for (int i = 0; i < 4; ++i) v[i] *= L.pre[i];
   }
   if (e.res) {
-    ld8(e.res + o, t);
     if (e.res_mean) {
-      float g[8], b[8];
-      ld8(e.res_gamma + n, g);
-      ld8(e.res_beta + n, b);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) t[i] = (t[i] - mu) * rs * g[i] + b[i];
+      for (int i = 0; i < 4; ++i) v[i] += (L.res[i] - mu) * rs * gam[i] + bet[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) v[i] += L.res[i];
     }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] += t[i];
   }
   if (e.accumulate) {
-    ld8(reinterpret_cast<const float*>(C) + o, t);      // accumulation is offered for fp32 C only
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] += t[i];
+    for (int i = 0; i < 4; ++i) v[i] += L.acc[i];
   }
-  st8(C + o, v);
-  if (e.copy_out) st8(reinterpret_cast<bf16*>(e.copy_out) + o, v);
+  st4(C + o, v);
+  if (e.copy_out) st4(reinterpret_cast<bf16*>(e.copy_out) + o, v);
 }
 
 constexpr int ST = 64, SK = 16;
@@ -173,7 +190,9 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const float* __restrict__
 // bf16 tcgen05 kernel
 // ============================================================================================
 constexpr int BM = 128, BK = 64;
-constexpr int TC_THREADS = 192;                  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int EPI_WARPS = 8;
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+constexpr int STAGE_LD = 33;                     // padded row of a warp's 32 x 32 transpose buffer
 constexpr uint64_t WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s: a wait that long has failed
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -274,7 +293,8 @@ template <int BN> struct TcCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int TMEM_COLS = 2 * BN;           // two accumulator buffers
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int EPI_BYTES = EPI_WARPS * 32 * STAGE_LD * 4;   // per-warp transpose buffers of the epilogue
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 template <int BN, bool A_K, bool B_K, typename CT>
@@ -286,8 +306,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
   uint8_t* gen_tiles = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + STAGES * Cfg::STAGE_BYTES);
-  const uint32_t bar0 = tiles + STAGES * Cfg::STAGE_BYTES;
+  float* epi_stage = reinterpret_cast<float*>(gen_tiles + STAGES * Cfg::STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES);
+  const uint32_t bar0 = tiles + STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES;
   // barrier slots: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem base, abort flag
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -304,7 +325,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 128);
+      mbar_init(tempty_bar(b), 32 * EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -395,7 +416,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     }
   } else {
     // ------------------------------ epilogue warps ----------------------------
-    const int q = warp & 3;                    // the TMEM lane quarter this warp may read
+    // A warp may read only its quarter of the TMEM lanes (rows q*32..q*32+31 of the tile); two warps
+    // share a quarter and split the columns.  Each 32 x 32 block is loaded one row per thread, turned
+    // through a padded shared-memory buffer, and then handled four rows per instruction with eight
+    // lanes per row, so that global loads and stores of a row are contiguous 128-byte pieces.
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int half = ew >> 2;
+    float* stage = epi_stage + ew * (32 * STAGE_LD);
     CT* C = reinterpret_cast<CT*>(a.C);
     int64_t it = 0;
     for (int64_t t = blockIdx.x; t < total && !failed; t += gridDim.x, ++it) {
@@ -405,33 +433,56 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       const int buf = (int)(it & 1);
       if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
       tc_fence_after();
-      const int64_t m = (int64_t)tm * BM + q * 32 + lane;
+      const int64_t row0 = (int64_t)tm * BM + q * 32;
       CT* Cs = C + (int64_t)split * a.split_stride;
-      float mu = 0.f, rs = 1.f;
-      if (a.epi.res_mean && m < a.M) {
-        mu = a.epi.res_mean[m];
-        rs = a.epi.res_rstd[m];
+      float mu_l = 0.f, rs_l = 1.f;               // LayerNorm statistics of row row0 + lane
+      if (a.epi.res_mean && row0 + lane < a.M) {
+        mu_l = a.epi.res_mean[row0 + lane];
+        rs_l = a.epi.res_rstd[row0 + lane];
       }
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         uint32_t v[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
-        const int n0 = tn * BN + c0;
-        if (m < a.M) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int n = n0 + 8 * j;
-            if (n < a.N) {                       // N is a multiple of 8
-              float x[8];
+        for (int j = 0; j < 32; ++j) stage[lane * STAGE_LD + j] = __uint_as_float(v[j]);
+        __syncwarp();
+        const int n = tn * BN + c0 + (lane & 7) * 4;
+        const bool col_ok = n < a.N;                // N is a multiple of 8
+        float bias4[4] = {0.f, 0.f, 0.f, 0.f}, gam4[4] = {0.f, 0.f, 0.f, 0.f}, bet4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (col_ok) {
+          if (a.epi.bias) ld4(a.epi.bias + n, bias4);
+          if (a.epi.res_mean) {
+            ld4(a.epi.res_gamma + n, gam4);
+            ld4(a.epi.res_beta + n, bet4);
+          }
+        }
+        // global loads of four rows are issued before the first store of those rows
 #pragma unroll
-              for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(v[8 * j + i]);
-              epilogue_store8<CT>(a.epi, Cs, a.ldc, m, n, x, mu, rs);
+        for (int hh = 0; hh < 2; ++hh) {
+          EpiLoads L[4];
+#pragma unroll
+          for (int r4 = 0; r4 < 4; ++r4) {
+            const int64_t m = row0 + (hh * 4 + r4) * 4 + (lane >> 3);
+            if (m < a.M && col_ok) epilogue_load4<CT>(a.epi, Cs, a.ldc, m, n, L[r4]);
+          }
+#pragma unroll
+          for (int r4 = 0; r4 < 4; ++r4) {
+            const int rl = (hh * 4 + r4) * 4 + (lane >> 3);
+            const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
+            const int64_t m = row0 + rl;
+            if (m < a.M && col_ok) {
+              float x[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) x[k] = stage[rl * STAGE_LD + (lane & 7) * 4 + k];
+              epilogue_store4<CT>(a.epi, Cs, a.ldc, m, n, x, L[r4], bias4, gam4, bet4, mu, rs);
             }
           }
         }
+        __syncwarp();
       }
       tc_fence_before();
-      mbar_arrive(tempty_bar(buf));           // 128 arrivals free the accumulator buffer
+      mbar_arrive(tempty_bar(buf));           // all epilogue threads free the accumulator buffer
     }
     if (failed && lane == 0) {
       *abort_flag = 1;
@@ -553,7 +604,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
            epi.gelu, epi.accumulate};
   if (dtype == GRAM_F32) {
     if (!c_f32) return gram_set_error(ctx, "gemm: fp32 operands need an fp32 result"), GRAM_ERR_UNSUPPORTED;
-    ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, 1, st);
+    ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, 1, st, epi.tag ? epi.tag : "gemm_f32");
     dim3 grid((unsigned)ceil_div(N, ST), (unsigned)ceil_div64(M, ST));
     gemm_f32_kernel<<<grid, 256, 0, st>>>((const float*)A, a_kmajor ? lda : 1, a_kmajor ? 1 : lda, (const float*)B,
                                           b_kmajor ? ldb : 1, b_kmajor ? 1 : ldb, (float*)C, ldc, M, N, K, e);
@@ -596,7 +647,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   splits = ceil_div(args.num_kb, args.kb_per_split);
   args.splits = splits;
   cudaError_t err;
-  ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, splits > 1 ? 2 : 1, st);
+  ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, splits > 1 ? 2 : 1, st, epi.tag ? epi.tag : "gemm");
   const int grid = (int)((tiles * splits < kNumSMs) ? tiles * splits : kNumSMs);
   if (splits > 1) {
     args.C = ws->splitk;

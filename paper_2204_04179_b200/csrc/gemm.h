@@ -4,8 +4,9 @@
 
 // What happens to an accumulator element acc(m, n) before it is stored to C(m, n):
 //   v = acc + bias[n]
-//   gelu:       pre(m, n) = v (if pre != null);  v = gelu(v)          (forward of the feed-forward layer)
-//   dgelu_pre:  v = v * gelu'(dgelu_pre(m, n))                        (backward through the GELU)
+//   gelu:       pre(m, n) = gelu'(v) (if pre != null);  v = gelu(v)   (forward of the feed-forward layer;
+//               the derivative shares erf and the exponential with the value, so it is saved here)
+//   dgelu_pre:  v = v * dgelu_pre(m, n)                               (backward through the GELU)
 //   res:        v += r(m, n), r = res(m, n), or, when res_mean != null, LayerNorm applied on the fly:
 //               r = (res(m, n) - res_mean[m]) * res_rstd[m] * res_gamma[n] + res_beta[n]
 //               (the fp32 residual stream: a layer's input is the LayerNorm of the previous fp32 sum)
@@ -25,6 +26,7 @@ struct GemmEpilogue {
   void* copy_out = nullptr;
   int gelu = 0;
   int accumulate = 0;
+  const char* tag = nullptr;   // names the call site in profiles (host side only)
 };
 
 struct GemmWorkspace {

@@ -81,14 +81,15 @@ gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n
 // profiling is on it also brackets them with CUDA events on the launching stream and files the
 // elapsed time and the algorithmic work (flops or bytes) under the kernel kind.
 // ---------------------------------------------------------------------------
-void gram_prof_open(gram_ctx* ctx, int kind, double work, int launches, cudaStream_t st, int* slot);
+void gram_prof_open(gram_ctx* ctx, int kind, const char* tag, double work, int launches, cudaStream_t st, int* slot);
 void gram_prof_close(gram_ctx* ctx, int slot, cudaStream_t st);
 struct ProfScope {
   gram_ctx* ctx;
   cudaStream_t st;
   int slot = -1;
-  ProfScope(gram_ctx* c, int kind, double work, int launches, cudaStream_t s) : ctx(c), st(s) {
-    gram_prof_open(c, kind, work, launches, s, &slot);
+  // tag: a string literal naming the call site (shown by gram_profile_dump)
+  ProfScope(gram_ctx* c, int kind, double work, int launches, cudaStream_t s, const char* tag = nullptr) : ctx(c), st(s) {
+    gram_prof_open(c, kind, tag, work, launches, s, &slot);
   }
   ~ProfScope() { if (slot >= 0) gram_prof_close(ctx, slot, st); }
 };

@@ -55,7 +55,15 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const 
 }
 
 // ---------------------------------------------------------------------------- LayerNorm
-template <typename T, int NP>   // NP pairs of columns per lane: d <= 64*NP
+__device__ __forceinline__ float4 ld4f(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st4t(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void st4t(bf16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+
+// a warp per row; lane l owns columns 4*(l + 32*i) .. +3 for i < NQ (d <= 128*NQ, d % 4 == 0)
+template <typename T, int NQ>
 __global__ void __launch_bounds__(256) ln_fwd_kernel(const float* __restrict__ z, const float* __restrict__ g,
                                                      const float* __restrict__ b, T* __restrict__ y,
                                                      float* __restrict__ mean, float* __restrict__ rstd, int64_t rows,
@@ -64,28 +72,32 @@ __global__ void __launch_bounds__(256) ln_fwd_kernel(const float* __restrict__ z
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t r = w; r < rows; r += nw) {
-    float2 v[NP];
+    float4 v[NQ];
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int c = 2 * (lane + 32 * i);
-      v[i] = (c < d) ? ld2(z + r * d + c) : make_float2(0.f, 0.f);
-      s += v[i].x + v[i].y;
+    for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
+      v[i] = (c < d) ? ld4f(z + r * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
     }
     const float mu = warp_sum(s) / d;
     float q = 0.f;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int c = 2 * (lane + 32 * i);
-      if (c < d) q += (v[i].x - mu) * (v[i].x - mu) + (v[i].y - mu) * (v[i].y - mu);
+    for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
+      if (c < d) {
+        const float a0 = v[i].x - mu, a1 = v[i].y - mu, a2 = v[i].z - mu, a3 = v[i].w - mu;
+        q += (a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3);
+      }
     }
     const float rs = rsqrtf(warp_sum(q) / d + kLnEps);
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int c = 2 * (lane + 32 * i);
+    for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
       if (c < d) {
-        float2 gg = ld2(g + c), bb = ld2(b + c);
-        st2(y + r * d + c, make_float2((v[i].x - mu) * rs * gg.x + bb.x, (v[i].y - mu) * rs * gg.y + bb.y));
+        const float4 gg = ld4f(g + c), bb = ld4f(b + c);
+        st4t(y + r * d + c, make_float4((v[i].x - mu) * rs * gg.x + bb.x, (v[i].y - mu) * rs * gg.y + bb.y,
+                                        (v[i].z - mu) * rs * gg.z + bb.z, (v[i].w - mu) * rs * gg.w + bb.w));
       }
     }
     if (lane == 0) {
@@ -95,7 +107,7 @@ __global__ void __launch_bounds__(256) ln_fwd_kernel(const float* __restrict__ z
   }
 }
 
-template <typename T, int NP>
+template <typename T, int NQ>
 __global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ z,
                                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                                      const float* __restrict__ g, float* __restrict__ dz,
@@ -105,43 +117,48 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ d
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   const int64_t w = (int64_t)blockIdx.x * nwb + warp;
   const int64_t nw = (int64_t)gridDim.x * nwb;
-  float2 ag[NP], ab[NP], gg[NP];
+  float4 ag[NQ], ab[NQ], gg[NQ];
 #pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    const int c = 2 * (lane + 32 * i);
-    ag[i] = make_float2(0.f, 0.f);
-    ab[i] = make_float2(0.f, 0.f);
-    gg[i] = (c < d) ? ld2(g + c) : make_float2(0.f, 0.f);
+  for (int i = 0; i < NQ; ++i) {
+    const int c = 4 * (lane + 32 * i);
+    ag[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    ab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    gg[i] = (c < d) ? ld4f(g + c) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int64_t r = w; r < rows; r += nw) {
     const float mu = mean[r], rs = rstd[r];
-    float2 xh[NP], gy[NP];
+    float4 xh[NQ], dd[NQ];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int c = 2 * (lane + 32 * i);
+    for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
       if (c < d) {
-        float2 zz = ld2(z + r * d + c), dd = ld2(dy + r * d + c);
-        xh[i] = make_float2((zz.x - mu) * rs, (zz.y - mu) * rs);
-        gy[i] = make_float2(dd.x * gg[i].x, dd.y * gg[i].y);
-        ag[i].x += dd.x * xh[i].x; ag[i].y += dd.y * xh[i].y;
-        ab[i].x += dd.x; ab[i].y += dd.y;
-        s1 += gy[i].x + gy[i].y;
-        s2 += gy[i].x * xh[i].x + gy[i].y * xh[i].y;
+        const float4 zz = ld4f(z + r * d + c);
+        dd[i] = ld4f(dy + r * d + c);
+        xh[i] = make_float4((zz.x - mu) * rs, (zz.y - mu) * rs, (zz.z - mu) * rs, (zz.w - mu) * rs);
       } else {
-        xh[i] = make_float2(0.f, 0.f);
-        gy[i] = make_float2(0.f, 0.f);
+        xh[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        dd[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
+    }
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) {
+      ag[i].x += dd[i].x * xh[i].x; ag[i].y += dd[i].y * xh[i].y; ag[i].z += dd[i].z * xh[i].z; ag[i].w += dd[i].w * xh[i].w;
+      ab[i].x += dd[i].x; ab[i].y += dd[i].y; ab[i].z += dd[i].z; ab[i].w += dd[i].w;
+      dd[i].x *= gg[i].x; dd[i].y *= gg[i].y; dd[i].z *= gg[i].z; dd[i].w *= gg[i].w;     // dy * gamma
+      s1 += (dd[i].x + dd[i].y) + (dd[i].z + dd[i].w);
+      s2 += (dd[i].x * xh[i].x + dd[i].y * xh[i].y) + (dd[i].z * xh[i].z + dd[i].w * xh[i].w);
     }
     s1 = warp_sum(s1) / d;
     s2 = warp_sum(s2) / d;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int c = 2 * (lane + 32 * i);
+    for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
       if (c < d) {
-        const float2 o = make_float2(rs * (gy[i].x - s1 - xh[i].x * s2), rs * (gy[i].y - s1 - xh[i].y * s2));
-        st2(dz + r * d + c, o);
-        if (dz_b) st2(dz_b + r * d + c, o);
+        const float4 o = make_float4(rs * (dd[i].x - s1 - xh[i].x * s2), rs * (dd[i].y - s1 - xh[i].y * s2),
+                                     rs * (dd[i].z - s1 - xh[i].z * s2), rs * (dd[i].w - s1 - xh[i].w * s2));
+        st4t(dz + r * d + c, o);
+        if (dz_b) st4t(dz_b + r * d + c, o);
       }
     }
   }
@@ -150,11 +167,11 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ d
   for (int ww = 0; ww < nwb; ++ww) {       // warps add in ascending order
     if (warp == ww) {
 #pragma unroll
-      for (int i = 0; i < NP; ++i) {
-        const int c = 2 * (lane + 32 * i);
+      for (int i = 0; i < NQ; ++i) {
+        const int c = 4 * (lane + 32 * i);
         if (c < d) {
-          sacc[c] += ag[i].x; sacc[c + 1] += ag[i].y;
-          sacc[d + c] += ab[i].x; sacc[d + c + 1] += ab[i].y;
+          sacc[c] += ag[i].x; sacc[c + 1] += ag[i].y; sacc[c + 2] += ag[i].z; sacc[c + 3] += ag[i].w;
+          sacc[d + c] += ab[i].x; sacc[d + c + 1] += ab[i].y; sacc[d + c + 2] += ab[i].z; sacc[d + c + 3] += ab[i].w;
         }
       }
     }
@@ -658,13 +675,12 @@ template <typename F> gram_status set_smem(gram_ctx* ctx, F kern, size_t bytes) 
 #define DISPATCH_T(dtype, ...)             \
   if ((dtype) == GRAM_F32) { typedef float T; __VA_ARGS__; } else { typedef bf16 T; __VA_ARGS__; }
 
-#define DISPATCH_NP(d, ...)                                                    \
-  if ((d) <= 64) { constexpr int NP = 1; __VA_ARGS__; }                        \
-  else if ((d) <= 128) { constexpr int NP = 2; __VA_ARGS__; }                  \
-  else if ((d) <= 256) { constexpr int NP = 4; __VA_ARGS__; }                  \
-  else if ((d) <= 512) { constexpr int NP = 8; __VA_ARGS__; }                  \
-  else if ((d) <= 768) { constexpr int NP = 12; __VA_ARGS__; }                 \
-  else { constexpr int NP = 16; __VA_ARGS__; }
+#define DISPATCH_NQ(d, ...)                                                    \
+  if ((d) <= 128) { constexpr int NQ = 1; __VA_ARGS__; }                       \
+  else if ((d) <= 256) { constexpr int NQ = 2; __VA_ARGS__; }                  \
+  else if ((d) <= 512) { constexpr int NQ = 4; __VA_ARGS__; }                  \
+  else if ((d) <= 768) { constexpr int NQ = 6; __VA_ARGS__; }                  \
+  else { constexpr int NQ = 8; __VA_ARGS__; }
 
 gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
@@ -682,10 +698,10 @@ gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32
 gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
                               float* mean, float* rstd, int64_t rows, int d, cudaStream_t st) {
   if (rows == 0) return GRAM_OK;
-  if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
+  if (d > 1024 || (d & 3)) return gram_set_error(ctx, "LayerNorm: d must be a multiple of 4 and at most 1024"), GRAM_ERR_UNSUPPORTED;
   const int blocks = grid_for(rows * 32, 256, kNumSMs * 8);
-  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (4.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
-  DISPATCH_T(dtype, DISPATCH_NP(d, ln_fwd_kernel<T, NP><<<blocks, 256, 0, st>>>(z, gamma, beta, (T*)y, mean, rstd, rows, d)));
+  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (4.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st, "ln_fwd");
+  DISPATCH_T(dtype, DISPATCH_NQ(d, ln_fwd_kernel<T, NQ><<<blocks, 256, 0, st>>>(z, gamma, beta, (T*)y, mean, rstd, rows, d)));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -694,11 +710,13 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
                                const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
                                float* dbeta, float* scratch, int64_t rows, int d, cudaStream_t st) {
   if (rows == 0) return GRAM_OK;
-  if (d > 1024 || (d & 1)) return gram_set_error(ctx, "LayerNorm: d must be even and at most 1024"), GRAM_ERR_UNSUPPORTED;
-  const int blocks = grid_for(rows * 32, 256, kRedBlocks);
+  if (d > 1024 || (d & 3)) return gram_set_error(ctx, "LayerNorm: d must be a multiple of 4 and at most 1024"), GRAM_ERR_UNSUPPORTED;
+  int cap = (int)(kRedScratchBytes / ((size_t)2 * d * sizeof(float)));
+  if (cap > kNumSMs * 8) cap = kNumSMs * 8;
+  const int blocks = grid_for(rows * 32, 256, cap);
   const size_t smem = (size_t)2 * d * sizeof(float);
-  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st);
-  DISPATCH_T(dtype, DISPATCH_NP(d, ln_bwd_kernel<T, NP><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
+  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st, "ln_bwd");
+  DISPATCH_T(dtype, DISPATCH_NQ(d, ln_bwd_kernel<T, NQ><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
   reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -711,7 +729,7 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
-  ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
+  ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_fwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
     return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, st);
   DISPATCH_T(dtype, {
@@ -729,7 +747,7 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
-  ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st);
+  ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
     return attention_backward_mma(ctx, qkv, dctx, dqkv, n_seq, S, d, n_heads, causal, st);
   DISPATCH_T(dtype, {
@@ -751,7 +769,7 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
   const int64_t per = ceil_div64(rows, rb);
   rb = ceil_div64(rows, per);
   dim3 grid((unsigned)ceil_div(N, 64), (unsigned)rb);
-  ProfScope prof(ctx, GRAM_K_COLSUM, (double)rows * N * (dtype == GRAM_BF16 ? 2.0 : 4.0), 2, st);
+  ProfScope prof(ctx, GRAM_K_COLSUM, (double)rows * N * (dtype == GRAM_BF16 ? 2.0 : 4.0), 2, st, "colsum");
   DISPATCH_T(dtype, colsum_kernel<T><<<grid, 256, 0, st>>>((const T*)X, rows, N, per, scratch));
   reduce_partials_kernel<<<ceil_div(N, 256), 256, 0, st>>>(scratch, (int)rb, (int64_t)N, N, out, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);

@@ -238,9 +238,11 @@ gram_status mm_dx(Model* m, const void* dY, const void* Wt, void* dX, bool x_f32
                      K, N, e, 0, st);
 }
 // dW[N, K] += dY[T, N]^T X[T, K]   (fp32 result, the token dimension may be split)
-gram_status mm_dw(Model* m, const void* dY, const void* X, float* dW, int64_t T, int N, int K, cudaStream_t st) {
+gram_status mm_dw(Model* m, const void* dY, const void* X, float* dW, int64_t T, int N, int K, cudaStream_t st,
+                  const char* tag = "dw") {
   GemmEpilogue e;
   e.accumulate = 1;
+  e.tag = tag;
   return gemm_launch(m->ctx, gram_gemm_ws(m->ctx), m->dtype, dY, 0, N, X, 0, K, dW, 1, K, N, K, T, e, 1, st);
 }
 
@@ -265,10 +267,12 @@ gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in
     LayerActs& a = s.acts[l];
     GemmEpilogue e;
     e.bias = mod.w + o.bqkv;
+    e.tag = "fwd_qkv";
     GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * d, d, e, st));
     GRAM_TRY(attention_forward(ctx, m->dtype, a.qkv, a.ctx, n_seq, S, d, s.heads, s.causal, st));
     e = GemmEpilogue();
     e.bias = mod.w + o.bo;
+    e.tag = "fwd_attn_out";
     set_res(e, x);
     if (s.attn_only) {
       e.copy_out = a.out;
@@ -282,9 +286,11 @@ gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in
       e.bias = mod.w + o.b1;
       e.gelu = 1;
       e.pre = a.u;
-      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, false, T, f, d, e, st));          // u = h1 W1^T + b1, g = gelu(u)
+      e.tag = "fwd_ffn1";
+      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, false, T, f, d, e, st));          // v = h1 W1^T + b1: g = gelu(v), u = gelu'(v)
       e = GemmEpilogue();
       e.bias = mod.w + o.b2;
+      e.tag = "fwd_ffn2";
       StreamRef h1;
       h1.z = a.z1; h1.mean = a.mean1; h1.rstd = a.rstd1; h1.gamma = mod.w + o.ln1g; h1.beta = mod.w + o.ln1b;
       set_res(e, h1);
@@ -321,14 +327,16 @@ gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, 
       GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, s.dzb, mod.g + o.ln2g,
                                   mod.g + o.ln2b, red, T, d, st));                       // oth, dzb = dz2
       GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.b2, red, st));
-      GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st));
+      GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st, "dw_ffn2"));
       e = GemmEpilogue();
       e.dgelu_pre = a.u;
-      GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(u)
+      e.tag = "dx_ffn2_dgelu";
+      GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(v), the saved u
       GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
-      GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st));
+      GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st, "dw_ffn1"));
       e = GemmEpilogue();
       e.res = oth;
+      e.tag = "dx_ffn1";
       GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, true, T, f, d, e, st));              // cur = dh1 = du W1 + dz2
       GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, s.dzb, mod.g + o.ln1g,
                                   mod.g + o.ln1b, red, T, d, st));                       // oth, dzb = dz1
@@ -336,14 +344,16 @@ gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, 
       float* t = cur; cur = oth; oth = t;                                                // oth = d(out), dzb its copy
     }
     GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
-    GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st));
+    GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st, "dw_attn_out"));
     e = GemmEpilogue();
+    e.tag = "dx_attn_out";
     GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.wo), s.dctx, false, T, d, d, e, st));
     GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, n_seq, S, d, s.heads, s.causal, st));
     GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
-    GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st));
+    GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
     e = GemmEpilogue();
     e.res = oth;
+    e.tag = "dx_qkv";
     if (s.attn_only && l > 0) e.copy_out = s.dzb;                                        // the layer below reads it as an operand
     GRAM_TRY(mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, true, T, 3 * d, d, e, st));        // cur = dx = dqkv Wqkv + dz1
   }
