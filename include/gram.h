@@ -223,6 +223,32 @@ gram_status gram_profile_dump(gram_ctx* ctx, char* h_text, size_t n);
 /* Kernels this context has launched since it was created (counted always). */
 gram_status gram_launch_count(const gram_ctx* ctx, int64_t* launches);
 
+/* --- the segmented sum without any allocation ----------------------------------
+ * (The paper has no counterpart to this call; it exists for the sake of callers.)
+ * Same result as gram_accumulate, d_G[u, :] = sum of d_dE[d_perm[j], :] over
+ * j in [d_seg_off[u], d_seg_off[u+1]), for code that is not allowed to allocate
+ * device memory: a plug-in running inside a host application that owns the
+ * allocator, a library called between the steps of a memory-planned job, a
+ * real-time loop.  It needs no context (creating one allocates): the partial
+ * sums that cross work-unit boundaries go to a fixed array inside the library
+ * image, about 4.9 MB, which every GPU that loads the library holds until the
+ * process exits.  The call uses no cudaMalloc/cudaFree and no allocating
+ * library routine; inputs and outputs are the caller's.
+ *   - Limits: d <= 1024 columns (a multiple of 4), P <= 2^31-1.  Larger sizes
+ *     return GRAM_ERR_WORKSPACE and a message in h_err.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call before any stream capture.
+ *   - All calls on a device share the one array: two calls that may run on the
+ *     GPU at the same time (different streams, different threads) race.  Order
+ *     them on one stream or with events.
+ *   - The order of additions differs from gram_accumulate's (fewer work units),
+ *     so results agree to rounding, not bit for bit; they are bit-identical
+ *     from call to call.  A position in d_perm outside [0, P) is read as row 0
+ *     and is not reported.
+ * h_err (may be NULL) receives a message of at most err_len bytes on failure. */
+gram_status gram_accumulate_static(const float* d_dE, const int32_t* d_perm, const int32_t* d_seg_off, int64_t P,
+                                   int32_t U, int32_t d, float* d_G, gram_stream stream, char* h_err, size_t err_len);
+
 /* --- a building block, exported so that it can be tested on its own --------
  * C[M, N] = A x B with bf16 operands and fp32 accumulation on the tensor cores.
  * a_kmajor != 0: A is [M, K] row-major, else [K, M] row-major; b_kmajor != 0:

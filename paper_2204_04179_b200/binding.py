@@ -29,7 +29,7 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_encode_unique", "gram_gather", "gram_accumulate", "gram_accumulate_multistep", "gram_touched_list",
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
-           "gram_launch_count", "gram_profile_dump"]
+           "gram_launch_count", "gram_profile_dump", "gram_accumulate_static"]
 
 KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other"]
 
@@ -258,3 +258,16 @@ class Gram:
                                       _ptr(Cm), C.c_int(int(Cm.dtype == torch.float32)), _ptr(bias),
                                       C.c_int(int(accumulate)), C.c_int64(M), C.c_int32(N), C.c_int64(K),
                                       _stream(stream)))
+
+
+def accumulate_static(dE, perm, seg_off, U, G, stream=None, P=None, d=None):
+    """gram_accumulate_static: the segmented sum with its scratch in a fixed array of the library, for
+    callers that may not allocate device memory.  Needs no context.  Raises GramError with the
+    library's message on failure."""
+    err = C.create_string_buffer(256)
+    P = dE.shape[0] if P is None else P
+    d = dE.shape[1] if d is None else d
+    st = lib().gram_accumulate_static(_ptr(dE), _ptr(perm), _ptr(seg_off), C.c_int64(P), C.c_int32(U), C.c_int32(d),
+                                      _ptr(G), _stream(stream), err, C.c_size_t(len(err)))
+    if st != 0:
+        raise GramError(st, err.value.decode())

@@ -372,3 +372,70 @@ gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// The segmented sum for callers that must not allocate.  Its chunk-boundary partial sums live in
+// a fixed array that is part of the library image, so the call touches no allocator at all.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kStaticChunks = 592;            // work units (4 per SM)
+constexpr int kStaticMaxD = 1024;             // widest row the fixed scratch can serve
+constexpr size_t kStaticPartialFloats = (size_t)kStaticChunks * 2 * kStaticMaxD;
+// [0, kStaticPartialFloats): partial sums; then 64 floats whose first word is the device status word
+static __device__ __align__(256) float g_static_scratch[kStaticPartialFloats + 64];
+
+constexpr int kMaxDevices = 64;
+float* g_static_ptr[kMaxDevices] = {};        // device address of the array, looked up once per device
+
+void static_fail(char* h_err, size_t n, const char* msg) {
+  if (h_err && n) snprintf(h_err, n, "%s", msg);
+}
+}  // namespace
+
+extern "C" gram_status gram_accumulate_static(const float* d_dE, const int32_t* d_perm, const int32_t* d_seg_off,
+                                               int64_t P, int32_t U, int32_t d, float* d_G, gram_stream stream,
+                                               char* h_err, size_t err_len) {
+  if (h_err && err_len) h_err[0] = 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (P < 0 || U < 0 || d <= 0 || U > P) return static_fail(h_err, err_len, "gram_accumulate_static: bad size"), GRAM_ERR_ARG;
+  if (d > kStaticMaxD) {
+    if (h_err && err_len) snprintf(h_err, err_len, "gram_accumulate_static: d=%d exceeds the fixed scratch's maximum of %d columns", d, kStaticMaxD);
+    return GRAM_ERR_WORKSPACE;
+  }
+  if (P > INT32_MAX) return static_fail(h_err, err_len, "gram_accumulate_static: P exceeds 2^31-1 positions"), GRAM_ERR_WORKSPACE;
+  if (P == 0 || U == 0) return GRAM_OK;
+  if (!d_dE || !d_perm || !d_seg_off || !d_G) return static_fail(h_err, err_len, "gram_accumulate_static: null buffer"), GRAM_ERR_ARG;
+  if (d % 4 != 0 || ((uintptr_t)d_dE % 16) || ((uintptr_t)d_G % 16))
+    return static_fail(h_err, err_len, "gram_accumulate_static: d must be a multiple of 4 and buffers 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return static_fail(h_err, err_len, "gram_accumulate_static: cannot identify the current device"), GRAM_ERR_CUDA;
+  if (!g_static_ptr[dev]) {
+    // in host code the array's name is only a handle: ask the runtime for its address on this device
+    float* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      if (h_err && err_len) snprintf(h_err, err_len, "gram_accumulate_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+      return GRAM_ERR_CUDA;
+    }
+    g_static_ptr[dev] = ptr;
+  }
+  float* partial = g_static_ptr[dev];
+  int32_t* status = reinterpret_cast<int32_t*>(partial + kStaticPartialFloats);
+  // the status word must start at zero; the partial sums need no clearing (each slot that is read in a
+  // call has been written earlier in the same call)
+  if (cudaMemsetAsync(status, 0, sizeof(int32_t), st) != cudaSuccess)
+    return static_fail(h_err, err_len, "gram_accumulate_static: clearing the status word failed"), GRAM_ERR_CUDA;
+  int64_t nchunks = ceil_div64(P, 16);
+  if (nchunks > kStaticChunks) nchunks = kStaticChunks;
+  const int64_t R = ceil_div64(P, nchunks);
+  nchunks = ceil_div64(P, R);
+  if (d >= 256) segsum_run<float, 2>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, status, nullptr, st);
+  else segsum_run<float, 1>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, status, nullptr, st);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    if (h_err && err_len) snprintf(h_err, err_len, "gram_accumulate_static: launch failed: %s", cudaGetErrorString(e));
+    return GRAM_ERR_CUDA;
+  }
+  return GRAM_OK;
+}
