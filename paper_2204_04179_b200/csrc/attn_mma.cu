@@ -1,6 +1,6 @@
 // Attention over short sequences (S <= 128 tokens, head width 32 or 64) with bf16 tensor-core
 // products and fp32 softmax.  One block owns one (sequence, head): Q, K, V (and dO in the backward)
-// live in shared memory for the whole block, a warp owns 16 query rows (forward, first half of the
+// live in shared memory (each once, row-major) for the whole block, a warp owns 16 query rows (forward, first half of the
 // backward) or 16 key rows (second half of the backward), and score tiles never leave registers.
 // The sequences are far shorter than a 128-row tcgen05 tile, and attention is ~2% of the encoder's
 // flops, so this uses the warp-level m16n8k16 MMA; the kernel is bound by reading qkv once.
@@ -33,9 +33,30 @@ __device__ __forceinline__ float quad_sum(float v) {
 //   A (16 x 16, row-major source X[m][k]):  a0 = X[g][2q..], a1 = X[g+8][2q..], a2 = X[g][2q+8..], a3 = X[g+8][2q+8..]
 //   B (16 x 8, source stored as Y[n][k]):   b0 = Y[g][2q..], b1 = Y[g][2q+8..]
 //   C (16 x 8):                             c0,c1 = C[g][2q, 2q+1], c2,c3 = C[g+8][2q, 2q+1]
-// Every matrix therefore sits in shared memory with its contraction index contiguous; where a
-// product needs the other orientation a transposed copy is kept (row strides are padded by 8
-// elements, which makes the 32-bit fragment loads conflict-free).
+// Where the contraction index is contiguous in shared memory (Q K^T, dO V^T) fragments are plain 32-bit
+// loads.  Where it is the row index (P V, dS K, dS^T Q, P^T dO) the 8 x 8 tiles are read with
+// ldmatrix.trans, so every matrix is kept once, row-major, with rows padded by 8 elements (conflict-free
+// for both access kinds).
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, const bf16* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(smem_addr(p)));
+}
+// B fragments of two adjacent n-tiles (n0, n0+8) for the k-tile k0, from a row-major S[k][n] with row stride ld:
+// (b0, b1) of tile n0 and (b2, b3) of tile n0 + 8
+__device__ __forceinline__ void load_b_trans(const bf16* S, int ld, int k0, int n0, int lane, uint32_t& b0, uint32_t& b1,
+                                             uint32_t& b2, uint32_t& b3) {
+  const int row = k0 + (lane & 7) + ((lane >> 3) & 1) * 8, col = n0 + (lane >> 4) * 8;
+  ldsm_x4_trans(b0, b1, b2, b3, S + row * ld + col);
+}
+// A fragment (m-tile m0, k-tile k0) of the transpose of a row-major S[k][m] with row stride ld
+__device__ __forceinline__ void load_a_trans(const bf16* S, int ld, int k0, int m0, int lane, uint32_t& a0, uint32_t& a1,
+                                             uint32_t& a2, uint32_t& a3) {
+  const int row = k0 + (lane & 7) + (lane >> 4) * 8, col = m0 + ((lane >> 3) & 1) * 8;
+  ldsm_x4_trans(a0, a1, a2, a3, S + row * ld + col);
+}
 
 // scores of 16 query rows against all SP keys: p[nt][0..3] for key tile nt, normalised probabilities on return
 template <int SP, int DH>
@@ -70,7 +91,7 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   }
   m0 = quad_max(m0);
   m1 = quad_max(m1);
-  if (m0 == -INFINITY) m0 = 0.f;        // a padded query row of a causal tile past S: no key is visible
+  if (m0 == -INFINITY) m0 = 0.f;        // no key is visible to this (padded) row
   if (m1 == -INFINITY) m1 = 0.f;
   float l0 = 0.f, l1 = 0.f;
 #pragma unroll
@@ -90,21 +111,33 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   }
 }
 
-// rows [0, S) of one head's slice of a [tokens, ld] bf16 matrix -> shared memory, row-major (dst) and,
-// when dst_t != null, transposed (dst_t[c][s]); rows S..SP-1 are zero
+// rows [0, S) of one head's slice of a [tokens, ld] bf16 matrix -> shared memory, row-major; rows S..SP-1 are zero
 template <int SP, int DH>
-__device__ __forceinline__ void load_head(const bf16* __restrict__ src, int64_t ld, int S, bf16* __restrict__ dst,
-                                          bf16* __restrict__ dst_t) {
-  constexpr int LD = DH + 8, LT = SP + 8;
+__device__ __forceinline__ void load_head(const bf16* __restrict__ src, int64_t ld, int S, bf16* __restrict__ dst) {
+  constexpr int LD = DH + 8;
   for (int i = threadIdx.x; i < SP * (DH / 8); i += blockDim.x) {
     const int s = i / (DH / 8), c = (i - s * (DH / 8)) * 8;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (s < S) v = *reinterpret_cast<const uint4*>(src + (int64_t)s * ld + c);
-    if (dst) *reinterpret_cast<uint4*>(dst + s * LD + c) = v;
-    if (dst_t) {
-      const bf16* e = reinterpret_cast<const bf16*>(&v);
+    *reinterpret_cast<uint4*>(dst + s * LD + c) = v;
+  }
+}
+
+// acc[nt] += A(16 x SP, from the C-layout registers x) * S[k][n] (row-major, SP x DH)
+template <int SP, int DH>
+__device__ __forceinline__ void mma_regs_times_rows(const float (&x)[SP / 8][4], const bf16* S, int lane,
+                                                    float (&acc)[DH / 8][4]) {
+  constexpr int LD = DH + 8;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) dst_t[(c + k) * LT + s] = e[k];
+  for (int kt = 0; kt < SP / 16; ++kt) {
+    const uint32_t a0 = pack2(x[2 * kt][0], x[2 * kt][1]), a1 = pack2(x[2 * kt][2], x[2 * kt][3]);
+    const uint32_t a2 = pack2(x[2 * kt + 1][0], x[2 * kt + 1][1]), a3 = pack2(x[2 * kt + 1][2], x[2 * kt + 1][3]);
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; nt += 2) {
+      uint32_t b0, b1, b2, b3;
+      load_b_trans(S, LD, kt * 16, nt * 8, lane, b0, b1, b2, b3);
+      mma16816(acc[nt], a0, a1, a2, a3, b0, b1);
+      mma16816(acc[nt + 1], a0, a1, a2, a3, b2, b3);
     }
   }
 }
@@ -112,17 +145,17 @@ __device__ __forceinline__ void load_head(const bf16* __restrict__ src, int64_t 
 template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
                                                            int n_heads, int causal, float scale) {
-  constexpr int LD = DH + 8, LT = SP + 8;
+  constexpr int LD = DH + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
   bf16* Ks = Qs + SP * LD;
-  bf16* Vt = Ks + SP * LD;                       // [DH][SP + 8]
+  bf16* Vs = Ks + SP * LD;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
   const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
-  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs, nullptr);
-  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks, nullptr);
-  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, nullptr, Vt);
+  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs);
+  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
+  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   for (int r0 = warp * 16; r0 < S; r0 += 64) {
@@ -131,16 +164,7 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
     float o[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-#pragma unroll
-    for (int kt = 0; kt < SP / 16; ++kt) {
-      const uint32_t a0 = pack2(p[2 * kt][0], p[2 * kt][1]), a1 = pack2(p[2 * kt][2], p[2 * kt][3]);
-      const uint32_t a2 = pack2(p[2 * kt + 1][0], p[2 * kt + 1][1]), a3 = pack2(p[2 * kt + 1][2], p[2 * kt + 1][3]);
-#pragma unroll
-      for (int nt = 0; nt < DH / 8; ++nt) {
-        const uint32_t b0 = ld32(Vt + (nt * 8 + g) * LT + kt * 16 + 2 * q), b1 = ld32(Vt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
-        mma16816(o[nt], a0, a1, a2, a3, b0, b1);
-      }
-    }
+    mma_regs_times_rows<SP, DH>(p, Vs, lane, o);              // O = P V
     bf16* ob = out + seq * S * (int64_t)d + h * DH;
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) {
@@ -155,28 +179,25 @@ template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
                                                            bf16* __restrict__ dqkv, int S, int d, int n_heads, int causal,
                                                            float scale) {
-  constexpr int LD = DH + 8, LT = SP + 8;
+  constexpr int LD = DH + 8, LP = SP + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // row-major [SP][DH+8]
+  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // [SP][DH+8]
   bf16* Ks = Qs + SP * LD;
   bf16* Vs = Ks + SP * LD;
   bf16* dOs = Vs + SP * LD;
-  bf16* Qt = dOs + SP * LD;                       // transposed [DH][SP+8]
-  bf16* Kt = Qt + DH * LT;
-  bf16* dOt = Kt + DH * LT;
-  bf16* Pt = dOt + DH * LT;                       // [key j][query i], [SP][SP+8]
-  bf16* dSt = Pt + SP * LT;
+  bf16* Ps = dOs + SP * LD;                       // [query i][key j], [SP][SP+8]
+  bf16* dSs = Ps + SP * LP;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
   const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
-  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs, Qt);
-  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks, Kt);
-  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs, nullptr);
-  load_head<SP, DH>(dctx + seq * S * (int64_t)d + h * DH, d, S, dOs, dOt);
+  load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs);
+  load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
+  load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
+  load_head<SP, DH>(dctx + seq * S * (int64_t)d + h * DH, d, S, dOs);
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   bf16* dq = dqkv + seq * S * 3 * (int64_t)d + h * DH;
-  // ---- first half: 16 query rows per warp: P, dS (kept transposed in shared memory), dQ ----
+  // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ ----
   for (int r0 = warp * 16; r0 < SP; r0 += 64) {
     float p[SP / 8][4];
     score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
@@ -202,28 +223,19 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
     d0 = quad_sum(d0);
     d1 = quad_sum(d1);
 #pragma unroll
-    for (int nt = 0; nt < SP / 8; ++nt) {         // dS = P (dP - delta) / sqrt(dh); stored as [j][i]
+    for (int nt = 0; nt < SP / 8; ++nt) {         // dS = P (dP - delta) / sqrt(dh)
       dp[nt][0] = p[nt][0] * (dp[nt][0] - d0) * scale; dp[nt][1] = p[nt][1] * (dp[nt][1] - d0) * scale;
       dp[nt][2] = p[nt][2] * (dp[nt][2] - d1) * scale; dp[nt][3] = p[nt][3] * (dp[nt][3] - d1) * scale;
       const int j = nt * 8 + 2 * q;
-      Pt[j * LT + r0 + g] = __float2bfloat16(p[nt][0]);       Pt[(j + 1) * LT + r0 + g] = __float2bfloat16(p[nt][1]);
-      Pt[j * LT + r0 + g + 8] = __float2bfloat16(p[nt][2]);   Pt[(j + 1) * LT + r0 + g + 8] = __float2bfloat16(p[nt][3]);
-      dSt[j * LT + r0 + g] = __float2bfloat16(dp[nt][0]);     dSt[(j + 1) * LT + r0 + g] = __float2bfloat16(dp[nt][1]);
-      dSt[j * LT + r0 + g + 8] = __float2bfloat16(dp[nt][2]); dSt[(j + 1) * LT + r0 + g + 8] = __float2bfloat16(dp[nt][3]);
+      *reinterpret_cast<uint32_t*>(Ps + (r0 + g) * LP + j) = pack2(p[nt][0], p[nt][1]);
+      *reinterpret_cast<uint32_t*>(Ps + (r0 + g + 8) * LP + j) = pack2(p[nt][2], p[nt][3]);
+      *reinterpret_cast<uint32_t*>(dSs + (r0 + g) * LP + j) = pack2(dp[nt][0], dp[nt][1]);
+      *reinterpret_cast<uint32_t*>(dSs + (r0 + g + 8) * LP + j) = pack2(dp[nt][2], dp[nt][3]);
     }
     float o[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-#pragma unroll
-    for (int kt = 0; kt < SP / 16; ++kt) {        // dQ = dS K
-      const uint32_t a0 = pack2(dp[2 * kt][0], dp[2 * kt][1]), a1 = pack2(dp[2 * kt][2], dp[2 * kt][3]);
-      const uint32_t a2 = pack2(dp[2 * kt + 1][0], dp[2 * kt + 1][1]), a3 = pack2(dp[2 * kt + 1][2], dp[2 * kt + 1][3]);
-#pragma unroll
-      for (int nt = 0; nt < DH / 8; ++nt) {
-        const uint32_t b0 = ld32(Kt + (nt * 8 + g) * LT + kt * 16 + 2 * q), b1 = ld32(Kt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
-        mma16816(o[nt], a0, a1, a2, a3, b0, b1);
-      }
-    }
+    mma_regs_times_rows<SP, DH>(dp, Ks, lane, o);             // dQ = dS K
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) {
       const int c = nt * 8 + 2 * q;
@@ -241,17 +253,19 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
       dv[nt][0] = dv[nt][1] = dv[nt][2] = dv[nt][3] = 0.f;
     }
 #pragma unroll
-    for (int kt = 0; kt < SP / 16; ++kt) {
-      const uint32_t s0 = ld32(dSt + (j0 + g) * LT + kt * 16 + 2 * q), s1 = ld32(dSt + (j0 + g + 8) * LT + kt * 16 + 2 * q);
-      const uint32_t s2 = ld32(dSt + (j0 + g) * LT + kt * 16 + 8 + 2 * q), s3 = ld32(dSt + (j0 + g + 8) * LT + kt * 16 + 8 + 2 * q);
-      const uint32_t p0 = ld32(Pt + (j0 + g) * LT + kt * 16 + 2 * q), p1 = ld32(Pt + (j0 + g + 8) * LT + kt * 16 + 2 * q);
-      const uint32_t p2 = ld32(Pt + (j0 + g) * LT + kt * 16 + 8 + 2 * q), p3 = ld32(Pt + (j0 + g + 8) * LT + kt * 16 + 8 + 2 * q);
+    for (int kt = 0; kt < SP / 16; ++kt) {        // contraction over query rows i = kt*16 ..
+      uint32_t s0, s1, s2, s3, p0, p1, p2, p3;
+      load_a_trans(dSs, LP, kt * 16, j0, lane, s0, s1, s2, s3);
+      load_a_trans(Ps, LP, kt * 16, j0, lane, p0, p1, p2, p3);
 #pragma unroll
-      for (int nt = 0; nt < DH / 8; ++nt) {
-        const uint32_t bq0 = ld32(Qt + (nt * 8 + g) * LT + kt * 16 + 2 * q), bq1 = ld32(Qt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
-        mma16816(dk[nt], s0, s1, s2, s3, bq0, bq1);
-        const uint32_t bo0 = ld32(dOt + (nt * 8 + g) * LT + kt * 16 + 2 * q), bo1 = ld32(dOt + (nt * 8 + g) * LT + kt * 16 + 8 + 2 * q);
-        mma16816(dv[nt], p0, p1, p2, p3, bo0, bo1);
+      for (int nt = 0; nt < DH / 8; nt += 2) {
+        uint32_t b0, b1, b2, b3;
+        load_b_trans(Qs, LD, kt * 16, nt * 8, lane, b0, b1, b2, b3);
+        mma16816(dk[nt], s0, s1, s2, s3, b0, b1);
+        mma16816(dk[nt + 1], s0, s1, s2, s3, b2, b3);
+        load_b_trans(dOs, LD, kt * 16, nt * 8, lane, b0, b1, b2, b3);
+        mma16816(dv[nt], p0, p1, p2, p3, b0, b1);
+        mma16816(dv[nt + 1], p0, p1, p2, p3, b2, b3);
       }
     }
 #pragma unroll
@@ -272,7 +286,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
 template <int SP, int DH>
 gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
                        cudaStream_t st) {
-  constexpr size_t smem = ((size_t)2 * SP * (DH + 8) + (size_t)DH * (SP + 8)) * 2;
+  constexpr size_t smem = (size_t)3 * SP * (DH + 8) * 2;
   auto kern = attn_fwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
@@ -282,7 +296,7 @@ gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq,
 template <int SP, int DH>
 gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, int64_t n_seq, int S, int d, int n_heads,
                        int causal, cudaStream_t st) {
-  constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)3 * DH * (SP + 8) + (size_t)2 * SP * (SP + 8)) * 2;
+  constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
   auto kern = attn_bwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
