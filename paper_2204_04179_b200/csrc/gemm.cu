@@ -297,7 +297,10 @@ template <int BN> struct TcCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int BN, bool A_K, bool B_K, typename CT>
+// DG: the epilogue is only "multiply by the saved GELU derivative, store bf16" (backward of the
+// feed-forward layer); the derivative's values for the whole tile are then fetched into registers
+// while the main loop of that tile is still running, which hides their HBM latency.
+template <int BN, bool A_K, bool B_K, typename CT, bool DG = false>
 __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                const __grid_constant__ CUtensorMap tmB, TcArgs a) {
   using Cfg = TcCfg<BN>;
@@ -431,10 +434,54 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       const int64_t r = t - (int64_t)split * a.n_tiles_m * a.n_tiles_n;
       const int tm = (int)(r / a.n_tiles_n), tn = (int)(r % a.n_tiles_n);
       const int buf = (int)(it & 1);
-      if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
-      tc_fence_after();
       const int64_t row0 = (int64_t)tm * BM + q * 32;
       CT* Cs = C + (int64_t)split * a.split_stride;
+      if constexpr (DG) {
+        uint2 pf[BN / 64][8];                       // packed bf16: 4 columns of one row per entry
+        const bf16* pre = reinterpret_cast<const bf16*>(a.epi.dgelu_pre);
+#pragma unroll
+        for (int blk = 0; blk < BN / 64; ++blk) {
+          const int n = tn * BN + half * (BN / 2) + blk * 32 + (lane & 7) * 4;
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr) {
+            const int64_t m = row0 + rr * 4 + (lane >> 3);
+            pf[blk][rr] = (m < a.M && n < a.N) ? *reinterpret_cast<const uint2*>(pre + m * a.ldc + n) : make_uint2(0u, 0u);
+          }
+        }
+        if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int blk = 0; blk < BN / 64; ++blk) {
+          const int c0 = half * (BN / 2) + blk * 32;
+          uint32_t v[32];
+          tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) stage[lane * STAGE_LD + j] = __uint_as_float(v[j]);
+          __syncwarp();
+          const int n = tn * BN + c0 + (lane & 7) * 4;
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr) {
+            const int rl = rr * 4 + (lane >> 3);
+            const int64_t m = row0 + rl;
+            if (m < a.M && n < a.N) {
+              const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].x));
+              const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].y));
+              float x[4];
+              x[0] = stage[rl * STAGE_LD + (lane & 7) * 4 + 0] * g0.x;
+              x[1] = stage[rl * STAGE_LD + (lane & 7) * 4 + 1] * g0.y;
+              x[2] = stage[rl * STAGE_LD + (lane & 7) * 4 + 2] * g1.x;
+              x[3] = stage[rl * STAGE_LD + (lane & 7) * 4 + 3] * g1.y;
+              st4(Cs + m * a.ldc + n, x);
+            }
+          }
+          __syncwarp();
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(buf));
+        continue;
+      }
+      if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
+      tc_fence_after();
       float mu_l = 0.f, rs_l = 1.f;               // LayerNorm statistics of row row0 + lane
       if (a.epi.res_mean && row0 + lane < a.M) {
         mu_l = a.epi.res_mean[row0 + lane];
@@ -560,9 +607,9 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool A_K, bool B_K, typename CT>
+template <int BN, bool A_K, bool B_K, typename CT, bool DG = false>
 cudaError_t launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st) {
-  auto kern = gemm_tc_kernel<BN, A_K, B_K, CT>;
+  auto kern = gemm_tc_kernel<BN, A_K, B_K, CT, DG>;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM_BYTES);
@@ -669,7 +716,13 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   args.ldc = ldc;
   args.split_stride = 0;
   args.epi = e;
-  if (c_f32) {
+  const bool dg_only = e.dgelu_pre && !e.bias && !e.res && !e.accumulate && !e.copy_out && !e.gelu && !c_f32 && a_kmajor &&
+                       !b_kmajor;
+  if (dg_only) {
+    if (BNsel == 256) err = launch_tc<256, true, false, bf16, true>(ma, mb, args, grid, st);
+    else if (BNsel == 128) err = launch_tc<128, true, false, bf16, true>(ma, mb, args, grid, st);
+    else err = launch_tc<64, true, false, bf16, true>(ma, mb, args, grid, st);
+  } else if (c_f32) {
     if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else if (BNsel == 128) err = launch_tc_major<128, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else err = launch_tc_major<64, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
