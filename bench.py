@@ -165,6 +165,7 @@ def kernel_sweep_cell(binding, synth, torch, dev, peaks):
 def run_gram(args, shape):
     import torch
     from paper_2204_04179_b200 import binding, synth
+    from paper_2204_04179_b200 import dist as gdist
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -184,6 +185,11 @@ def run_gram(args, shape):
     over = {}
     if args.micro_batch:
         over["ce_micro_batch"] = args.micro_batch
+    multistep = shape.K > 1
+    if multistep:                      # whole windows only: K-1 light steps and one step with the encoder pass
+        over["lr_task"] = 1e-3
+        args.warmup = max(shape.K, -(-args.warmup // shape.K) * shape.K)
+        args.steps = max(shape.K, -(-args.steps // shape.K) * shape.K)
     cfg = binding.config_from_shape(shape, **over)
     g = binding.Gram(cfg)
     g.set_params(binding.GRAM_MODULE_CE, synth.flatten(ce))
@@ -192,7 +198,7 @@ def run_gram(args, shape):
     P = shape.B * shape.L
     n_total = args.warmup + args.steps
     # every rank draws its own batches (weak scaling: per-GPU work is fixed, histories are independent)
-    batches = [synth.batch(shape, args.seed + 7919 * rank, step=k) for k in range(n_total)]
+    batches = [synth.batch(shape, gdist.rank_seed(args.seed, rank), step=k) for k in range(n_total)]
     dev_batches = [(torch.from_numpy(i).to(dev), torch.from_numpy(l).to(dev)) for i, l in batches]
     pinned = [(torch.from_numpy(i).pin_memory(), torch.from_numpy(l).pin_memory()) for i, l in batches]
 
@@ -202,13 +208,11 @@ def run_gram(args, shape):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return gdist.max_over_ranks(ms, dist, dev)
 
     # ---- device-resident inputs ----
+    if multistep:
+        g.cache_fill()                 # encodings of every item with the initial parameters (untimed set-up)
     for k in range(args.warmup):
         g.step(dev_batches[k][0], dev_batches[k][1], shape.B)
     g.profile(True)
@@ -298,6 +302,10 @@ def run_gram(args, shape):
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"end-to-end oracle (float64, one encoder call per interaction) on the first {n_pos} "
                                           f"positions of one history of the same workload, {dt:.1f} s; linear in interactions"}
+    if multistep:
+        line["multistep"] = {"K": shape.K, "windows_timed": args.steps // shape.K,
+                             "per_step": [{"k": i % shape.K, "ms": r.ms_total, "touched": r.n_touched,
+                                           "encoder_pass": r.encoder_pass, "n_encoded": r.n_encoded} for i, r in enumerate(reports)]}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -309,14 +317,14 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="gram", choices=["gram", "reference"])
-    ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny"])
+    ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny", "kt_multistep"])
     ap.add_argument("--micro-batch", type=int, default=0, help="items per encoder pass (0: the workload's default)")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     from paper_2204_04179_b200 import synth
     shape = synth.config(args.workload)
-    if args.workload in ("kt", "nr") and not args.micro_batch:
-        args.micro_batch = 5120 if args.workload == "kt" else 0
+    if args.workload in ("kt", "nr", "kt_multistep") and not args.micro_batch:
+        args.micro_batch = 0 if args.workload == "nr" else 5120
     if args.impl == "reference":
         run_reference(args, shape)
     else:
