@@ -3,6 +3,7 @@
 // fp32 accumulators double-buffered in tensor memory so that the epilogue of one tile overlaps the
 // main loop of the next).  fp32: a plain tiled CUDA-core kernel for the small fp32 configuration.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "gemm.h"
 
@@ -85,18 +86,17 @@ __device__ __forceinline__ void gelu_parts(float x, float& cdf, float& pdf) {
   pdf = 0.39894228f * ex;
 }
 
-// what one lane reads before it may store anything for its 4 columns of one row
+// what one lane reads before it may store anything for its 4 columns of one row: the residual, the
+// saved GELU derivative or the old value of C (the tensor-core path takes at most one of the three)
 struct EpiLoads {
-  float res[4];
-  float pre[4];
-  float acc[4];
+  float aux[4];
 };
 template <typename CT>
 __device__ __forceinline__ void epilogue_load4(const EpiDev& e, const CT* C, int64_t ldc, int64_t m, int n, EpiLoads& L) {
   const int64_t o = m * ldc + n;
-  if (e.res) ld4(e.res + o, L.res);
-  if (e.dgelu_pre) ld4(reinterpret_cast<const bf16*>(e.dgelu_pre) + o, L.pre);
-  if (e.accumulate) ld4(reinterpret_cast<const float*>(C) + o, L.acc);      // accumulation is offered for fp32 C only
+  if (e.res) ld4(e.res + o, L.aux);
+  else if (e.dgelu_pre) ld4(reinterpret_cast<const bf16*>(e.dgelu_pre) + o, L.aux);
+  else if (e.accumulate) ld4(reinterpret_cast<const float*>(C) + o, L.aux);      // accumulation is offered for fp32 C only
 }
 template <typename CT>
 __device__ __forceinline__ void epilogue_store4(const EpiDev& e, CT* C, int64_t ldc, int64_t m, int n, float (&v)[4],
@@ -118,22 +118,20 @@ __device__ __forceinline__ void epilogue_store4(const EpiDev& e, CT* C, int64_t 
     }
     if (e.pre) st4(reinterpret_cast<bf16*>(e.pre) + o, dg);
   }
-  if (e.dgelu_pre) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] *= L.pre[i];
-  }
   if (e.res) {
     if (e.res_mean) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) v[i] += (L.res[i] - mu) * rs * gam[i] + bet[i];
+      for (int i = 0; i < 4; ++i) v[i] += (L.aux[i] - mu) * rs * gam[i] + bet[i];
     } else {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) v[i] += L.res[i];
+      for (int i = 0; i < 4; ++i) v[i] += L.aux[i];
     }
-  }
-  if (e.accumulate) {
+  } else if (e.dgelu_pre) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] += L.acc[i];
+    for (int i = 0; i < 4; ++i) v[i] *= L.aux[i];
+  } else if (e.accumulate) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] += L.aux[i];
   }
   st4(C + o, v);
   if (e.copy_out) st4(reinterpret_cast<bf16*>(e.copy_out) + o, v);
@@ -192,7 +190,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const float* __restrict__
 constexpr int BM = 128, BK = 64;
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
-constexpr int STAGE_LD = 33;                     // padded row of a warp's 32 x 32 transpose buffer
+constexpr int STAGE_LD = 32;                     // a warp's 32 x 32 fp32 transpose buffer (swizzled, no padding)
 constexpr uint64_t WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s: a wait that long has failed
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -248,7 +246,9 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db
       "l"(da), "l"(db), "r"(idesc), "r"(accum)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 columns of this warp's 32 TMEM lanes: the load is issued without waiting, and the wait is a separate
+// step that names the registers, so that the compiler cannot move a use of them ahead of it
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -258,7 +258,27 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_ld32_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+// A warp's 32 x 32 fp32 transpose buffer: rows of eight 16-byte slots, slot j of row r stored at j ^ (r & 7).
+// Row-per-thread writes and eight-lanes-per-row reads are then both free of bank conflicts.
+__device__ __forceinline__ void stage_write_row(float* stage, int lane, const uint32_t (&v)[32]) {
+  float4* s4 = reinterpret_cast<float4*>(stage) + lane * 8;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    s4[j ^ (lane & 7)] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                     __uint_as_float(v[4 * j + 3]));
+}
+__device__ __forceinline__ float4 stage_read(const float* stage, int row, int slot) {
+  return reinterpret_cast<const float4*>(stage)[row * 8 + (slot ^ (row & 7))];
 }
 
 // Shared-memory matrix descriptor of a 128-byte-swizzled operand tile (bf16).
@@ -297,10 +317,222 @@ template <int BN> struct TcCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
+// The epilogue of one output tile for one epilogue warp: rows row0 .. row0+31 (TMEM lanes q*32..), columns
+// [half*BN/2, (half+1)*BN/2) of tile column tn.  A warp may read only its quarter of the TMEM lanes; two warps
+// share a quarter and split the columns.  Each 32 x 32 block is loaded one row per thread, turned through a
+// padded shared-memory buffer, and then handled four rows per instruction with eight lanes per row, so that
+// global loads and stores of a row are contiguous 128-byte pieces.  Returns false if the bounded wait for the
+// accumulator gave up.
 // DG: the epilogue is only "multiply by the saved GELU derivative, store bf16" (backward of the
 // feed-forward layer); the derivative's values for the whole tile are then fetched into registers
 // while the main loop of that tile is still running, which hides their HBM latency.
-template <int BN, bool A_K, bool B_K, typename CT, bool DG = false>
+// Epilogue variants fixed at compile time (the general one reads the EpiDev flags at run time):
+//   EPI_DG    multiply by the saved GELU derivative, bf16 out (values prefetched during the main loop)
+//   EPI_BIAS  (+ bias), bf16 or fp32 out
+//   EPI_GELU  + bias, GELU, saved derivative, both bf16
+//   EPI_RES   (+ bias) + fp32 residual (LayerNorm on the fly when res_mean is set), fp32 out (+ bf16 copy)
+enum { EPI_GENERAL = 0, EPI_DG = 1, EPI_BIAS = 2, EPI_GELU = 3, EPI_RES = 4 };
+
+template <int BN, typename CT, int MODE>
+__device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t row0, int tn, int half, int q, int lane,
+                                              float* stage, uint32_t tmem_base, int buf, uint32_t tfull_addr,
+                                              uint32_t parity, volatile int* abort_flag) {
+  if constexpr (MODE == EPI_DG) {
+    uint2 pf[BN / 64][8];                       // packed bf16: 4 columns of one row per entry
+    const int sub = lane >> 3, slot = lane & 7;
+    const int64_t rows_left = a.M - (row0 + sub);
+    const int64_t step = 4 * a.ldc;
+    const int ncol0 = tn * BN + half * (BN / 2) + slot * 4;
+    const int64_t o0 = (row0 + sub) * a.ldc + ncol0;
+    const bf16* pre = reinterpret_cast<const bf16*>(a.epi.dgelu_pre) + o0;
+#pragma unroll
+    for (int blk = 0; blk < BN / 64; ++blk) {
+      const bool col_ok = ncol0 + blk * 32 < a.N;
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr)
+        pf[blk][rr] = (col_ok && rr * 4 < rows_left) ? *reinterpret_cast<const uint2*>(pre + blk * 32 + rr * step) : make_uint2(0u, 0u);
+    }
+    if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+    tc_fence_after();
+#pragma unroll
+    for (int blk = 0; blk < BN / 64; ++blk) {
+      const int c0 = half * (BN / 2) + blk * 32;
+      uint32_t v[32];
+      tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
+      tc_ld32_wait(v);
+      stage_write_row(stage, lane, v);
+      __syncwarp();
+      if (ncol0 + blk * 32 < a.N) {
+        CT* cp = Cs + o0 + blk * 32;
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr) {
+          if (rr * 4 < rows_left) {
+            const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].x));
+            const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].y));
+            const float4 t = stage_read(stage, rr * 4 + sub, slot);
+            const float x[4] = {t.x * g0.x, t.y * g0.y, t.z * g1.x, t.w * g1.y};
+            st4(cp, x);
+          }
+          cp += step;
+        }
+      }
+      __syncwarp();
+    }
+    tc_fence_before();
+    return true;
+  } else if constexpr (MODE == EPI_BIAS || MODE == EPI_GELU || MODE == EPI_RES) {
+    if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+    tc_fence_after();
+    const int sub = lane >> 3, slot = lane & 7;
+    const int64_t rows_left = a.M - (row0 + sub);         // row rr*4 + sub exists iff rr*4 < rows_left
+    float mu_l = 0.f, rs_l = 1.f;
+    if constexpr (MODE == EPI_RES) {
+      if (a.epi.res_mean && row0 + lane < a.M) {
+        mu_l = a.epi.res_mean[row0 + lane];
+        rs_l = a.epi.res_rstd[row0 + lane];
+      }
+    }
+#pragma unroll 1
+    for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+      uint32_t v[32];
+      tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
+      tc_ld32_wait(v);
+      stage_write_row(stage, lane, v);
+      __syncwarp();
+      const int n = tn * BN + c0 + slot * 4;
+      if (n < a.N) {                                      // N is a multiple of 8
+        float b4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (a.epi.bias) ld4(a.epi.bias + n, b4);
+        const int64_t o0 = (row0 + sub) * a.ldc + n;      // element offset of this lane's first row
+        const int64_t step = 4 * a.ldc;
+        if constexpr (MODE == EPI_BIAS) {
+          CT* cp = Cs + o0;
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr) {
+            if (rr * 4 < rows_left) {
+              const float4 t = stage_read(stage, rr * 4 + sub, slot);
+              const float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
+              st4(cp, x);
+            }
+            cp += step;
+          }
+        } else if constexpr (MODE == EPI_GELU) {
+          CT* cp = Cs + o0;
+          bf16* pp = reinterpret_cast<bf16*>(a.epi.pre) + o0;
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr) {
+            if (rr * 4 < rows_left) {
+              const float4 t = stage_read(stage, rr * 4 + sub, slot);
+              float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
+              float dg[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float c, p;
+                gelu_parts(x[i], c, p);
+                dg[i] = c + x[i] * p;
+                x[i] *= c;
+              }
+              st4(cp, x);
+              st4(pp, dg);
+            }
+            cp += step;
+            pp += step;
+          }
+        } else {
+          float g4[4] = {0.f, 0.f, 0.f, 0.f}, be4[4] = {0.f, 0.f, 0.f, 0.f};
+          const bool ln = a.epi.res_mean != nullptr;
+          if (ln) {
+            ld4(a.epi.res_gamma + n, g4);
+            ld4(a.epi.res_beta + n, be4);
+          }
+          const float* rp = a.epi.res + o0;
+          float4 r4[8];
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr)                  // all residual loads first
+            r4[rr] = (rr * 4 < rows_left) ? *reinterpret_cast<const float4*>(rp + rr * step) : make_float4(0.f, 0.f, 0.f, 0.f);
+          CT* cp = Cs + o0;
+          bf16* qp = a.epi.copy_out ? reinterpret_cast<bf16*>(a.epi.copy_out) + o0 : nullptr;
+#pragma unroll
+          for (int rr = 0; rr < 8; ++rr) {
+            const int rl = rr * 4 + sub;
+            const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
+            if (rr * 4 < rows_left) {
+              const float4 t = stage_read(stage, rl, slot);
+              float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
+              if (ln) {
+                x[0] += (r4[rr].x - mu) * rs * g4[0] + be4[0];
+                x[1] += (r4[rr].y - mu) * rs * g4[1] + be4[1];
+                x[2] += (r4[rr].z - mu) * rs * g4[2] + be4[2];
+                x[3] += (r4[rr].w - mu) * rs * g4[3] + be4[3];
+              } else {
+                x[0] += r4[rr].x; x[1] += r4[rr].y; x[2] += r4[rr].z; x[3] += r4[rr].w;
+              }
+              st4(cp, x);
+              if (qp) st4(qp, x);
+            }
+            cp += step;
+            if (qp) qp += step;
+          }
+        }
+      }
+      __syncwarp();
+    }
+    tc_fence_before();
+    return true;
+  } else {
+    if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+    tc_fence_after();
+    float mu_l = 0.f, rs_l = 1.f;               // LayerNorm statistics of row row0 + lane
+    if (a.epi.res_mean && row0 + lane < a.M) {
+      mu_l = a.epi.res_mean[row0 + lane];
+      rs_l = a.epi.res_rstd[row0 + lane];
+    }
+#pragma unroll 1
+    for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+      uint32_t v[32];
+      tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
+      tc_ld32_wait(v);
+      stage_write_row(stage, lane, v);
+      __syncwarp();
+      const int n = tn * BN + c0 + (lane & 7) * 4;
+      const bool col_ok = n < a.N;                // N is a multiple of 8
+      float bias4[4] = {0.f, 0.f, 0.f, 0.f}, gam4[4] = {0.f, 0.f, 0.f, 0.f}, bet4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (col_ok) {
+        if (a.epi.bias) ld4(a.epi.bias + n, bias4);
+        if (a.epi.res_mean) {
+          ld4(a.epi.res_gamma + n, gam4);
+          ld4(a.epi.res_beta + n, bet4);
+        }
+      }
+      // global loads of four rows are issued before the first store of those rows
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        EpiLoads L[4];
+#pragma unroll
+        for (int r4 = 0; r4 < 4; ++r4) {
+          const int64_t m = row0 + (hh * 4 + r4) * 4 + (lane >> 3);
+          if (m < a.M && col_ok) epilogue_load4<CT>(a.epi, Cs, a.ldc, m, n, L[r4]);
+        }
+#pragma unroll
+        for (int r4 = 0; r4 < 4; ++r4) {
+          const int rl = (hh * 4 + r4) * 4 + (lane >> 3);
+          const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
+          const int64_t m = row0 + rl;
+          if (m < a.M && col_ok) {
+            const float4 t = stage_read(stage, rl, lane & 7);
+            float x[4] = {t.x, t.y, t.z, t.w};
+            epilogue_store4<CT>(a.epi, Cs, a.ldc, m, n, x, L[r4], bias4, gam4, bet4, mu, rs);
+          }
+        }
+      }
+      __syncwarp();
+    }
+    tc_fence_before();
+    return true;
+  }
+}
+
+template <int BN, bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
 __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                const __grid_constant__ CUtensorMap tmB, TcArgs a) {
   using Cfg = TcCfg<BN>;
@@ -419,10 +651,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     }
   } else {
     // ------------------------------ epilogue warps ----------------------------
-    // A warp may read only its quarter of the TMEM lanes (rows q*32..q*32+31 of the tile); two warps
-    // share a quarter and split the columns.  Each 32 x 32 block is loaded one row per thread, turned
-    // through a padded shared-memory buffer, and then handled four rows per instruction with eight
-    // lanes per row, so that global loads and stores of a row are contiguous 128-byte pieces.
     const int ew = warp - 2;
     const int q = warp & 3;
     const int half = ew >> 2;
@@ -436,99 +664,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       const int buf = (int)(it & 1);
       const int64_t row0 = (int64_t)tm * BM + q * 32;
       CT* Cs = C + (int64_t)split * a.split_stride;
-      if constexpr (DG) {
-        uint2 pf[BN / 64][8];                       // packed bf16: 4 columns of one row per entry
-        const bf16* pre = reinterpret_cast<const bf16*>(a.epi.dgelu_pre);
-#pragma unroll
-        for (int blk = 0; blk < BN / 64; ++blk) {
-          const int n = tn * BN + half * (BN / 2) + blk * 32 + (lane & 7) * 4;
-#pragma unroll
-          for (int rr = 0; rr < 8; ++rr) {
-            const int64_t m = row0 + rr * 4 + (lane >> 3);
-            pf[blk][rr] = (m < a.M && n < a.N) ? *reinterpret_cast<const uint2*>(pre + m * a.ldc + n) : make_uint2(0u, 0u);
-          }
-        }
-        if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int blk = 0; blk < BN / 64; ++blk) {
-          const int c0 = half * (BN / 2) + blk * 32;
-          uint32_t v[32];
-          tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) stage[lane * STAGE_LD + j] = __uint_as_float(v[j]);
-          __syncwarp();
-          const int n = tn * BN + c0 + (lane & 7) * 4;
-#pragma unroll
-          for (int rr = 0; rr < 8; ++rr) {
-            const int rl = rr * 4 + (lane >> 3);
-            const int64_t m = row0 + rl;
-            if (m < a.M && n < a.N) {
-              const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].x));
-              const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pf[blk][rr].y));
-              float x[4];
-              x[0] = stage[rl * STAGE_LD + (lane & 7) * 4 + 0] * g0.x;
-              x[1] = stage[rl * STAGE_LD + (lane & 7) * 4 + 1] * g0.y;
-              x[2] = stage[rl * STAGE_LD + (lane & 7) * 4 + 2] * g1.x;
-              x[3] = stage[rl * STAGE_LD + (lane & 7) * 4 + 3] * g1.y;
-              st4(Cs + m * a.ldc + n, x);
-            }
-          }
-          __syncwarp();
-        }
-        tc_fence_before();
-        mbar_arrive(tempty_bar(buf));
-        continue;
+      if (!epilogue_tile<BN, CT, MODE>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
+                                     (uint32_t)((it >> 1) & 1), abort_flag)) {
+        failed = true;
+        break;
       }
-      if (!mbar_wait(tfull_bar(buf), (uint32_t)((it >> 1) & 1), abort_flag)) { failed = true; break; }
-      tc_fence_after();
-      float mu_l = 0.f, rs_l = 1.f;               // LayerNorm statistics of row row0 + lane
-      if (a.epi.res_mean && row0 + lane < a.M) {
-        mu_l = a.epi.res_mean[row0 + lane];
-        rs_l = a.epi.res_rstd[row0 + lane];
-      }
-#pragma unroll 1
-      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) stage[lane * STAGE_LD + j] = __uint_as_float(v[j]);
-        __syncwarp();
-        const int n = tn * BN + c0 + (lane & 7) * 4;
-        const bool col_ok = n < a.N;                // N is a multiple of 8
-        float bias4[4] = {0.f, 0.f, 0.f, 0.f}, gam4[4] = {0.f, 0.f, 0.f, 0.f}, bet4[4] = {0.f, 0.f, 0.f, 0.f};
-        if (col_ok) {
-          if (a.epi.bias) ld4(a.epi.bias + n, bias4);
-          if (a.epi.res_mean) {
-            ld4(a.epi.res_gamma + n, gam4);
-            ld4(a.epi.res_beta + n, bet4);
-          }
-        }
-        // global loads of four rows are issued before the first store of those rows
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          EpiLoads L[4];
-#pragma unroll
-          for (int r4 = 0; r4 < 4; ++r4) {
-            const int64_t m = row0 + (hh * 4 + r4) * 4 + (lane >> 3);
-            if (m < a.M && col_ok) epilogue_load4<CT>(a.epi, Cs, a.ldc, m, n, L[r4]);
-          }
-#pragma unroll
-          for (int r4 = 0; r4 < 4; ++r4) {
-            const int rl = (hh * 4 + r4) * 4 + (lane >> 3);
-            const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
-            const int64_t m = row0 + rl;
-            if (m < a.M && col_ok) {
-              float x[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) x[k] = stage[rl * STAGE_LD + (lane & 7) * 4 + k];
-              epilogue_store4<CT>(a.epi, Cs, a.ldc, m, n, x, L[r4], bias4, gam4, bet4, mu, rs);
-            }
-          }
-        }
-        __syncwarp();
-      }
-      tc_fence_before();
       mbar_arrive(tempty_bar(buf));           // all epilogue threads free the accumulator buffer
     }
     if (failed && lane == 0) {
@@ -558,6 +698,241 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ============================================================================================
+// The same product on pairs of SMs (tcgen05 cta_group::2): a cluster of two CTAs owns a 256 x 256
+// output tile.  Each CTA stages its own 128 rows of A and its own 128 of the tile's 256 columns of B,
+// the leader CTA (cluster rank 0) issues one M256 N256 K16 MMA per step that reads both CTAs' shared
+// memory, and each CTA's tensor memory receives its 128 rows of the result.  Per CTA and k-block this
+// moves 32 KB through shared memory instead of 48 KB, which is what bounds the single-CTA kernel.
+// Protocol: each CTA's TMA loads signal the leader's "full" barrier (two arrivals with their byte
+// counts); the leader's commits arrive on the "empty" and "accumulator full" barriers of both CTAs
+// (one commit per CTA, no multicast); the epilogue warps of both CTAs arrive on the leader's
+// "accumulator empty" barrier.  Every wait is bounded as in the single-CTA kernel; the CTAs meet at a
+// cluster barrier before they exit so that neither releases shared or tensor memory the other may
+// still touch.
+// ============================================================================================
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_remote(uint32_t cluster_bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                                 uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t cluster_bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accum)
+      : "memory");
+}
+
+struct Tc2Cfg {
+  static constexpr int BN = 256;                       // columns of the pair's tile
+  static constexpr int A_BYTES = BM * BK * 2;          // this CTA's 128 rows of A
+  static constexpr int B_BYTES = (BN / 2) * BK * 2;    // this CTA's 128 columns of B
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = 6;
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int EPI_BYTES = EPI_WARPS * 32 * STAGE_LD * 4;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 + 256;
+};
+
+// n_tiles_m counts 256-row tiles here
+template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
+__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+  using Cfg = Tc2Cfg;
+  constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;       // the same offset in both CTAs of the pair
+  uint8_t* gen_tiles = smem_raw + (tiles - raw);
+  float* epi_stage = reinterpret_cast<float*>(gen_tiles + STAGES * Cfg::STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES);
+  const uint32_t bar0 = tiles + STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };                       // used in the leader
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };           // one per CTA
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };       // one per CTA
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };  // used in the leader
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 2);              // the two CTAs' producers, each with its byte count
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 2 * EPI_WARPS);   // one arrival per epilogue warp of either CTA
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                           // both CTAs' barriers exist before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int64_t total = (int64_t)a.n_tiles_m * a.n_tiles_n * a.splits;
+  const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  bool failed = false;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer (both CTAs) ------------------------------
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      for (int64_t t = cluster_id; t < total && !failed; t += n_clusters) {
+        const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
+        const int64_t r = t - (int64_t)split * a.n_tiles_m * a.n_tiles_n;
+        const int tm = (int)(r / a.n_tiles_n), tn = (int)(r % a.n_tiles_n);
+        const int kb0 = split * a.kb_per_split, kb1 = min(kb0 + a.kb_per_split, a.num_kb);
+        const int m0 = tm * 2 * BM + (int)rank * BM;            // this CTA's rows of A
+        const int n0 = tn * BN + (int)rank * (BN / 2);          // this CTA's columns of B
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+          mbar_arrive_expect_tx_remote(lead_full, Cfg::STAGE_BYTES);
+          const uint32_t sa = tiles + s * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
+          if (A_K) {
+            tma_load_2d_pair(sa, &tmA, kb * BK, m0, lead_full);
+          } else {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(sa + i * 8192, &tmA, m0 + i * 64, kb * BK, lead_full);
+          }
+          if (B_K) {
+            tma_load_2d_pair(sb, &tmB, kb * BK, n0, lead_full);
+          } else {
+#pragma unroll
+            for (int i = 0; i < BN / 128; ++i) tma_load_2d_pair(sb + i * 8192, &tmB, n0 + i * 64, kb * BK, lead_full);
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (failed) {
+        *abort_flag = 1;
+        gram_device_fail(a.status, GRAM_ERR_TIMEOUT);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader CTA only) ----------------------------
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_K ? 0u : 1u) << 15) |
+                                 ((B_K ? 0u : 1u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      int s = 0;
+      uint32_t ph = 0;
+      int64_t it = 0;
+      for (int64_t t = cluster_id; t < total && !failed; t += n_clusters, ++it) {
+        const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
+        const int kb0 = split * a.kb_per_split, kb1 = min(kb0 + a.kb_per_split, a.num_kb);
+        const int buf = (int)(it & 1);
+        if (!mbar_wait(tempty_bar(buf), (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + s * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = A_K ? make_desc(sa + k * 32, 16, 1024) : make_desc(sa + k * 2048, 8192, 1024);
+            const uint64_t db = B_K ? make_desc(sb + k * 32, 16, 1024) : make_desc(sb + k * 2048, 8192, 1024);
+            tc_mma_pair(tmem_d, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(map_to_cta(empty_bar(s), 0));      // the stage is free in both CTAs once these MMAs are done
+          tc_commit_pair(map_to_cta(empty_bar(s), 1));
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (failed) break;
+        tc_commit_pair(map_to_cta(tfull_bar(buf), 0));      // accumulator complete in both CTAs
+        tc_commit_pair(map_to_cta(tfull_bar(buf), 1));
+      }
+      if (failed) {
+        *abort_flag = 1;
+        gram_device_fail(a.status, GRAM_ERR_TIMEOUT);
+      }
+    }
+  } else {
+    // ------------------------------ epilogue warps (both CTAs) ------------------------------
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int half = ew >> 2;
+    float* stage = epi_stage + ew * (32 * STAGE_LD);
+    CT* C = reinterpret_cast<CT*>(a.C);
+    int64_t it = 0;
+    for (int64_t t = cluster_id; t < total && !failed; t += n_clusters, ++it) {
+      const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
+      const int64_t r = t - (int64_t)split * a.n_tiles_m * a.n_tiles_n;
+      const int tm = (int)(r / a.n_tiles_n), tn = (int)(r % a.n_tiles_n);
+      const int buf = (int)(it & 1);
+      const int64_t row0 = (int64_t)tm * 2 * BM + (int64_t)rank * BM + q * 32;
+      CT* Cs = C + (int64_t)split * a.split_stride;
+      if (!epilogue_tile<BN, CT, MODE>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
+                                     (uint32_t)((it >> 1) & 1), abort_flag)) {
+        failed = true;
+        break;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(buf), 0));
+    }
+    if (failed && lane == 0) {
+      *abort_flag = 1;
+      gram_device_fail(a.status, GRAM_ERR_TIMEOUT);
+    }
+  }
+
+  // ------------------------------ teardown --------------------------------------
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (warp == 1 && lane == 0) {           // let copies and MMAs already issued drain (bounded)
+      uint64_t t0 = clock64();
+      while (clock64() - t0 < WAIT_LIMIT_CYCLES / 64) {}
+    }
+    __syncthreads();
+  }
+  cluster_sync_all();                        // the peer no longer reads this CTA's memory or signals its barriers
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
                  : "memory");
   }
 }
@@ -607,9 +982,9 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool A_K, bool B_K, typename CT, bool DG = false>
+template <int BN, bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
 cudaError_t launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st) {
-  auto kern = gemm_tc_kernel<BN, A_K, B_K, CT, DG>;
+  auto kern = gemm_tc_kernel<BN, A_K, B_K, CT, MODE>;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM_BYTES);
@@ -627,6 +1002,38 @@ cudaError_t launch_tc_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUt
   if (a_k && !b_k) return launch_tc<BN, true, false, CT>(ma, mb, args, grid, st);
   if (!a_k && b_k) return launch_tc<BN, false, true, CT>(ma, mb, args, grid, st);
   return launch_tc<BN, false, false, CT>(ma, mb, args, grid, st);
+}
+
+template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
+cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st) {
+  auto kern = gemm_tc2_kernel<A_K, B_K, CT, MODE>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tc2Cfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = Tc2Cfg::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, args);
+}
+template <typename CT>
+cudaError_t launch_tc2_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid,
+                             cudaStream_t st) {
+  if (a_k && b_k) return launch_tc2<true, true, CT>(ma, mb, args, grid, st);
+  if (a_k && !b_k) return launch_tc2<true, false, CT>(ma, mb, args, grid, st);
+  if (!a_k && b_k) return launch_tc2<false, true, CT>(ma, mb, args, grid, st);
+  return launch_tc2<false, false, CT>(ma, mb, args, grid, st);
 }
 
 }  // namespace
@@ -663,14 +1070,19 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
       K == 0)
     return gram_set_error(ctx, "gemm: bf16 operands need 16-byte aligned rows (sizes multiples of 8)"), GRAM_ERR_UNSUPPORTED;
   if (e.accumulate && !c_f32) return gram_set_error(ctx, "gemm: accumulation needs an fp32 result"), GRAM_ERR_UNSUPPORTED;
+  if ((e.res != nullptr) + (e.dgelu_pre != nullptr) + (e.accumulate != 0) > 1)
+    return gram_set_error(ctx, "gemm: at most one of residual, GELU derivative and accumulation per product"), GRAM_ERR_UNSUPPORTED;
   if ((N % 8) || (e.bias && ((uintptr_t)e.bias % 16)) || (e.res_gamma && (((uintptr_t)e.res_gamma % 16) || ((uintptr_t)e.res_beta % 16))))
     return gram_set_error(ctx, "gemm: N must be a multiple of 8 and the epilogue's vectors 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
   const int BNsel = (N % 256 == 0 || N > 1024) ? 256 : (N > 64 ? 128 : 64);
+  // pairs of SMs (256 x 256 tiles) when the problem has full-height tiles; GRAM_GEMM_PAIR=0 keeps single CTAs
+  static const bool pair_enabled = []() { const char* v = getenv("GRAM_GEMM_PAIR"); return !(v && v[0] == '0'); }();
+  const bool pair = pair_enabled && BNsel == 256 && M >= 2 * BM;
   CUtensorMap ma, mb;
   bool ok;
   if (a_kmajor) ok = make_map(&ma, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM);
   else ok = make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, 64, BK);
-  if (b_kmajor) ok = ok && make_map(&mb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, BK, (uint32_t)BNsel);
+  if (b_kmajor) ok = ok && make_map(&mb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, BK, (uint32_t)(pair ? BNsel / 2 : BNsel));
   else ok = ok && make_map(&mb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 64, BK);
   if (!ok) return gram_set_error(ctx, "gemm: cuTensorMapEncodeTiled failed"), GRAM_ERR_CUDA;
 
@@ -678,13 +1090,14 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   args.M = M;
   args.N = N;
   args.num_kb = (int32_t)ceil_div64(K, BK);
-  args.n_tiles_m = (int32_t)ceil_div64(M, BM);
+  args.n_tiles_m = (int32_t)ceil_div64(M, pair ? 2 * BM : BM);
   args.n_tiles_n = ceil_div(N, BNsel);
   args.status = gram_status_word(ctx);
   const int64_t tiles = (int64_t)args.n_tiles_m * args.n_tiles_n;
+  const int units = pair ? kNumSMs / 2 : kNumSMs;        // CTAs, or CTA pairs, that run at once
   int splits = 1;
-  if (allow_splitk && tiles < kNumSMs && args.num_kb >= 16 && ws && ws->splitk) {
-    splits = (int)((2 * kNumSMs + tiles - 1) / tiles);
+  if (allow_splitk && tiles < units && args.num_kb >= 16 && ws && ws->splitk) {
+    splits = (int)((2 * units + tiles - 1) / tiles);
     if (splits > args.num_kb / 8) splits = args.num_kb / 8;
     const int64_t per = (int64_t)M * N * (int64_t)sizeof(float);
     if ((int64_t)splits * per > (int64_t)ws->splitk_bytes) splits = (int)(ws->splitk_bytes / per);
@@ -695,13 +1108,16 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   args.splits = splits;
   cudaError_t err;
   ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, splits > 1 ? 2 : 1, st, epi.tag ? epi.tag : "gemm");
-  const int grid = (int)((tiles * splits < kNumSMs) ? tiles * splits : kNumSMs);
+  const int grid = pair ? 2 * (int)((tiles * splits < units) ? tiles * splits : units)
+                        : (int)((tiles * splits < kNumSMs) ? tiles * splits : kNumSMs);
   if (splits > 1) {
     args.C = ws->splitk;
     args.ldc = N;
     args.split_stride = (int64_t)M * N;
     args.epi = EpiDev{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0};
-    if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
+    if (pair && !a_kmajor && !b_kmajor) err = launch_tc2<false, false, float, EPI_BIAS>(ma, mb, args, grid, st);
+    else if (pair) err = launch_tc2_major<float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
+    else if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else if (BNsel == 128) err = launch_tc_major<128, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else err = launch_tc_major<64, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     if (err != cudaSuccess) return gram_set_error(ctx, "gemm launch failed: %s", cudaGetErrorString(err)), GRAM_ERR_CUDA;
@@ -718,10 +1134,23 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   args.epi = e;
   const bool dg_only = e.dgelu_pre && !e.bias && !e.res && !e.accumulate && !e.copy_out && !e.gelu && !c_f32 && a_kmajor &&
                        !b_kmajor;
-  if (dg_only) {
-    if (BNsel == 256) err = launch_tc<256, true, false, bf16, true>(ma, mb, args, grid, st);
-    else if (BNsel == 128) err = launch_tc<128, true, false, bf16, true>(ma, mb, args, grid, st);
-    else err = launch_tc<64, true, false, bf16, true>(ma, mb, args, grid, st);
+  const bool others = e.gelu || e.dgelu_pre || e.res || e.accumulate || e.copy_out || e.pre;
+  const bool m_bias = !others;
+  const bool m_gelu = e.gelu && e.pre && !e.dgelu_pre && !e.res && !e.accumulate && !e.copy_out && !c_f32 && a_kmajor && b_kmajor;
+  const bool m_res = e.res && !e.gelu && !e.dgelu_pre && !e.accumulate && !e.pre && c_f32 && a_kmajor;
+  if (pair) {
+    if (dg_only) err = launch_tc2<true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
+    else if (m_gelu) err = launch_tc2<true, true, bf16, EPI_GELU>(ma, mb, args, grid, st);
+    else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);
+    else if (m_res && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES>(ma, mb, args, grid, st);
+    else if (m_bias && a_kmajor && b_kmajor && !c_f32) err = launch_tc2<true, true, bf16, EPI_BIAS>(ma, mb, args, grid, st);
+    else if (m_bias && a_kmajor && !b_kmajor && !c_f32) err = launch_tc2<true, false, bf16, EPI_BIAS>(ma, mb, args, grid, st);
+    else if (c_f32) err = launch_tc2_major<float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
+    else err = launch_tc2_major<bf16>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
+  } else if (dg_only) {
+    if (BNsel == 256) err = launch_tc<256, true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
+    else if (BNsel == 128) err = launch_tc<128, true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
+    else err = launch_tc<64, true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
   } else if (c_f32) {
     if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else if (BNsel == 128) err = launch_tc_major<128, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
