@@ -108,22 +108,24 @@ __global__ void __launch_bounds__(256) ln_fwd_kernel(const float* __restrict__ z
 }
 
 template <typename T, int NQ>
-__global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ z,
-                                                     const float* __restrict__ mean, const float* __restrict__ rstd,
-                                                     const float* __restrict__ g, float* __restrict__ dz,
-                                                     T* __restrict__ dz_b, float* __restrict__ part, int64_t rows,
-                                                     int d) {
-  extern __shared__ float sacc[];          // [2][d]: dgamma, dbeta of this block
+__global__ void __launch_bounds__(256, 2) ln_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ z,
+                                                        const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                        const float* __restrict__ g, float* __restrict__ dz,
+                                                        T* __restrict__ dz_b, float* __restrict__ part, int64_t rows,
+                                                        int d) {
+  extern __shared__ float sacc[];          // [2][d]: dgamma, dbeta of this block; then [d]: gamma
+  float* sgam = sacc + 2 * d;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   const int64_t w = (int64_t)blockIdx.x * nwb + warp;
   const int64_t nw = (int64_t)gridDim.x * nwb;
-  float4 ag[NQ], ab[NQ], gg[NQ];
+  for (int i = threadIdx.x; i < d; i += blockDim.x) sgam[i] = g[i];
+  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sacc[i] = 0.f;
+  __syncthreads();
+  float4 ag[NQ], ab[NQ];
 #pragma unroll
   for (int i = 0; i < NQ; ++i) {
-    const int c = 4 * (lane + 32 * i);
     ag[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     ab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    gg[i] = (c < d) ? ld4f(g + c) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int64_t r = w; r < rows; r += nw) {
     const float mu = mean[r], rs = rstd[r];
@@ -143,9 +145,11 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ d
     }
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
+      const int c = 4 * (lane + 32 * i);
+      const float4 gg = (c < d) ? *reinterpret_cast<const float4*>(sgam + c) : make_float4(0.f, 0.f, 0.f, 0.f);
       ag[i].x += dd[i].x * xh[i].x; ag[i].y += dd[i].y * xh[i].y; ag[i].z += dd[i].z * xh[i].z; ag[i].w += dd[i].w * xh[i].w;
       ab[i].x += dd[i].x; ab[i].y += dd[i].y; ab[i].z += dd[i].z; ab[i].w += dd[i].w;
-      dd[i].x *= gg[i].x; dd[i].y *= gg[i].y; dd[i].z *= gg[i].z; dd[i].w *= gg[i].w;     // dy * gamma
+      dd[i].x *= gg.x; dd[i].y *= gg.y; dd[i].z *= gg.z; dd[i].w *= gg.w;     // dy * gamma
       s1 += (dd[i].x + dd[i].y) + (dd[i].z + dd[i].w);
       s2 += (dd[i].x * xh[i].x + dd[i].y * xh[i].y) + (dd[i].z * xh[i].z + dd[i].w * xh[i].w);
     }
@@ -162,8 +166,6 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const float* __restrict__ d
       }
     }
   }
-  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sacc[i] = 0.f;
-  __syncthreads();
   for (int ww = 0; ww < nwb; ++ww) {       // warps add in ascending order
     if (warp == ww) {
 #pragma unroll
@@ -714,7 +716,7 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
   int cap = (int)(kRedScratchBytes / ((size_t)2 * d * sizeof(float)));
   if (cap > kNumSMs * 8) cap = kNumSMs * 8;
   const int blocks = grid_for(rows * 32, 256, cap);
-  const size_t smem = (size_t)2 * d * sizeof(float);
+  const size_t smem = (size_t)3 * d * sizeof(float);
   ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st, "ln_bwd");
   DISPATCH_T(dtype, DISPATCH_NQ(d, ln_bwd_kernel<T, NQ><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
   reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
