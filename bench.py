@@ -76,6 +76,23 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def gemm_traffic_per_row():
+    """DRAM bytes per token row of the forward qkv product from the committed ncu summary; None when gemm.cu has
+    changed since the counters were taken."""
+    import hashlib
+    prof = os.path.join(ROOT, "profiles", "gemm_tc2_fwd_qkv_shape.md")
+    src = os.path.join(ROOT, "paper_2204_04179_b200", "csrc", "gemm.cu")
+    if not (os.path.exists(prof) and os.path.exists(src)):
+        return None
+    kv = {}
+    for line in open(prof):
+        if ":" in line and line.split(":")[0] in ("gemm_cu_sha256", "dram_bytes_per_row"):
+            kv[line.split(":")[0]] = line.split(":", 1)[1].strip()
+    if kv.get("gemm_cu_sha256") != hashlib.sha256(open(src, "rb").read()).hexdigest():
+        return None
+    return float(kv["dram_bytes_per_row"])
+
+
 def oracle_sample(shape, ce, tk, toks, ids, lab, n_pos):
     """The oracle, as it stands, on the first n_pos positions of the first history: interactions/s."""
     import torch
@@ -257,8 +274,13 @@ def run_gram(args, shape):
                 "bound": "tensor" if shape.dtype == "bf16" else "alu",
                 "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
                 "peak_source": peaks["source"] + " bf16_tflops_sustained", "traffic": None,
+                "traffic_note": "DRAM bytes of one fwd_qkv launch (tokens x 2304 x 768), scaled by rows from the ncu capture "
+                                "in profiles/gemm_tc2_fwd_qkv_shape.md; null when gemm.cu changed since that capture",
                 "launches": gm["launches"], "avg_launch_ms": gm["ms"] / max(1, gm["launches"]),
                 "share_of_step": gm["ms"] / (ms_total if ms_total > 0 else 1)}
+    per_row = gemm_traffic_per_row()
+    if per_row is not None and shape.dtype == "bf16":
+        roofline["traffic"] = per_row * statistics.mean(r.n_unique for r in reports) * shape.l_t
     stage_ms = {k: statistics.mean(getattr(r, k) for r in reports)
                 for k in ("ms_dedup", "ms_encode", "ms_gather", "ms_task", "ms_accumulate", "ms_backward", "ms_total")}
     per_kind = {}

@@ -19,7 +19,6 @@ __device__ __forceinline__ uint32_t pack2(float x, float y) {
   __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
   return *reinterpret_cast<uint32_t*>(&h);
 }
-__device__ __forceinline__ uint32_t ld32(const bf16* p) { return *reinterpret_cast<const uint32_t*>(p); }
 __device__ __forceinline__ float quad_max(float v) {
   v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
   return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
@@ -44,6 +43,24 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t& r0, uint32_t& r1, uint32
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(smem_addr(p)));
 }
+__device__ __forceinline__ void ldsm_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, const bf16* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(smem_addr(p)));
+}
+// B fragments of two adjacent n-tiles (n0, n0+8) for the k-tile k0, from Y[n][k] (contraction index contiguous):
+// (b0, b1) of tile n0 and (b2, b3) of tile n0 + 8
+__device__ __forceinline__ void load_b_rows(const bf16* Y, int ld, int n0, int k0, int lane, uint32_t& b0, uint32_t& b1,
+                                            uint32_t& b2, uint32_t& b3) {
+  const int row = n0 + (lane & 7) + (lane >> 4) * 8, col = k0 + ((lane >> 3) & 1) * 8;
+  ldsm_x4(b0, b1, b2, b3, Y + row * ld + col);
+}
+// A fragment (rows m0.., k-tile k0) of a row-major X[m][k]
+__device__ __forceinline__ void load_a_rows(const bf16* X, int ld, int m0, int k0, int lane, uint32_t& a0, uint32_t& a1,
+                                            uint32_t& a2, uint32_t& a3) {
+  const int row = m0 + (lane & 7) + ((lane >> 3) & 1) * 8, col = k0 + (lane >> 4) * 8;
+  ldsm_x4(a0, a1, a2, a3, X + row * ld + col);
+}
 // B fragments of two adjacent n-tiles (n0, n0+8) for the k-tile k0, from a row-major S[k][n] with row stride ld:
 // (b0, b1) of tile n0 and (b2, b3) of tile n0 + 8
 __device__ __forceinline__ void load_b_trans(const bf16* S, int ld, int k0, int n0, int lane, uint32_t& b0, uint32_t& b1,
@@ -65,14 +82,17 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   constexpr int LD = DH + 8;
 #pragma unroll
   for (int nt = 0; nt < SP / 8; ++nt) p[nt][0] = p[nt][1] = p[nt][2] = p[nt][3] = 0.f;
+  const int lane = g * 4 + q;
 #pragma unroll
   for (int kt = 0; kt < DH / 16; ++kt) {
-    const uint32_t a0 = ld32(Qs + (r0 + g) * LD + kt * 16 + 2 * q), a1 = ld32(Qs + (r0 + g + 8) * LD + kt * 16 + 2 * q);
-    const uint32_t a2 = ld32(Qs + (r0 + g) * LD + kt * 16 + 8 + 2 * q), a3 = ld32(Qs + (r0 + g + 8) * LD + kt * 16 + 8 + 2 * q);
+    uint32_t a0, a1, a2, a3;
+    load_a_rows(Qs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
 #pragma unroll
-    for (int nt = 0; nt < SP / 8; ++nt) {
-      const uint32_t b0 = ld32(Ks + (nt * 8 + g) * LD + kt * 16 + 2 * q), b1 = ld32(Ks + (nt * 8 + g) * LD + kt * 16 + 8 + 2 * q);
+    for (int nt = 0; nt < SP / 8; nt += 2) {
+      uint32_t b0, b1, b2, b3;
+      load_b_rows(Ks, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
       mma16816(p[nt], a0, a1, a2, a3, b0, b1);
+      mma16816(p[nt + 1], a0, a1, a2, a3, b2, b3);
     }
   }
   const int i0 = r0 + g, i1 = r0 + g + 8;
@@ -206,12 +226,14 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
     for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
 #pragma unroll
     for (int kt = 0; kt < DH / 16; ++kt) {        // dP = dO V^T
-      const uint32_t a0 = ld32(dOs + (r0 + g) * LD + kt * 16 + 2 * q), a1 = ld32(dOs + (r0 + g + 8) * LD + kt * 16 + 2 * q);
-      const uint32_t a2 = ld32(dOs + (r0 + g) * LD + kt * 16 + 8 + 2 * q), a3 = ld32(dOs + (r0 + g + 8) * LD + kt * 16 + 8 + 2 * q);
+      uint32_t a0, a1, a2, a3;
+      load_a_rows(dOs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
 #pragma unroll
-      for (int nt = 0; nt < SP / 8; ++nt) {
-        const uint32_t b0 = ld32(Vs + (nt * 8 + g) * LD + kt * 16 + 2 * q), b1 = ld32(Vs + (nt * 8 + g) * LD + kt * 16 + 8 + 2 * q);
+      for (int nt = 0; nt < SP / 8; nt += 2) {
+        uint32_t b0, b1, b2, b3;
+        load_b_rows(Vs, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
         mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
+        mma16816(dp[nt + 1], a0, a1, a2, a3, b2, b3);
       }
     }
     float d0 = 0.f, d1 = 0.f;

@@ -182,18 +182,32 @@ __global__ void __launch_bounds__(256, 2) ln_bwd_kernel(const float* __restrict_
   for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) part[(int64_t)blockIdx.x * 2 * d + i] = sacc[i];
 }
 
-// out[c] += sum_b part[b*stride + c]   (two outputs when out2 != null: second half of each partial row)
-__global__ void reduce_partials_kernel(const float* __restrict__ part, int nblocks, int64_t stride, int n,
-                                       float* __restrict__ out, float* __restrict__ out2, float scale) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= n) return;
+// out[c] += scale * sum_b part[b*stride + c]   (two outputs when out2 != null: second half of each partial row).
+// A block owns 32 columns; its 8 warps take the partial rows b = w, w+8, ... and their sums are added in
+// ascending w, so the order of additions is fixed.
+__global__ void __launch_bounds__(256) reduce_partials_kernel(const float* __restrict__ part, int nblocks, int64_t stride,
+                                                              int n, float* __restrict__ out, float* __restrict__ out2,
+                                                              float scale) {
+  __shared__ float sa[8][32], sb[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
   float a = 0.f, b = 0.f;
-  for (int k = 0; k < nblocks; ++k) {
-    a += part[(int64_t)k * stride + c];
-    if (out2) b += part[(int64_t)k * stride + n + c];
+  if (c < n) {
+    for (int k = w; k < nblocks; k += 8) {
+      a += part[(int64_t)k * stride + c];
+      if (out2) b += part[(int64_t)k * stride + n + c];
+    }
   }
-  out[c] += a * scale;
-  if (out2) out2[c] += b * scale;
+  sa[w][lane] = a;
+  sb[w][lane] = b;
+  __syncthreads();
+  if (w == 0 && c < n) {
+    float ta = sa[0][lane], tb = sb[0][lane];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) { ta += sa[k][lane]; tb += sb[k][lane]; }
+    out[c] += ta * scale;
+    if (out2) out2[c] += tb * scale;
+  }
 }
 
 // ---------------------------------------------------------------------------- attention
@@ -719,7 +733,7 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
   const size_t smem = (size_t)3 * d * sizeof(float);
   ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st, "ln_bwd");
   DISPATCH_T(dtype, DISPATCH_NQ(d, ln_bwd_kernel<T, NQ><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
-  reduce_partials_kernel<<<ceil_div(d, 256), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
+  reduce_partials_kernel<<<ceil_div(d, 32), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -773,7 +787,7 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
   dim3 grid((unsigned)ceil_div(N, 64), (unsigned)rb);
   ProfScope prof(ctx, GRAM_K_COLSUM, (double)rows * N * (dtype == GRAM_BF16 ? 2.0 : 4.0), 2, st, "colsum");
   DISPATCH_T(dtype, colsum_kernel<T><<<grid, 256, 0, st>>>((const T*)X, rows, N, per, scratch));
-  reduce_partials_kernel<<<ceil_div(N, 256), 256, 0, st>>>(scratch, (int)rb, (int64_t)N, N, out, nullptr, 1.f);
+  reduce_partials_kernel<<<ceil_div(N, 32), 256, 0, st>>>(scratch, (int)rb, (int64_t)N, N, out, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -839,7 +853,7 @@ gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* lab
   dim3 grid((unsigned)ceil_div(d, 128), (unsigned)L);
   ProfScope prof(ctx, GRAM_K_TASK_HEAD, 8.0 * (double)B * L * d, 2, st);
   kt_input_bwd_kernel<<<grid, 128, 0, st>>>(dx, labels, dE, dpos, scratch, B, L, d);
-  reduce_partials_kernel<<<ceil_div(3 * d, 256), 256, 0, st>>>(scratch, L, (int64_t)3 * d, 3 * d, dresp, nullptr, 1.f);
+  reduce_partials_kernel<<<ceil_div(3 * d, 32), 256, 0, st>>>(scratch, L, (int64_t)3 * d, 3 * d, dresp, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
