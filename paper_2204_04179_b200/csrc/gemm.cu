@@ -1097,10 +1097,19 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   const int units = pair ? kNumSMs / 2 : kNumSMs;        // CTAs, or CTA pairs, that run at once
   int splits = 1;
   if (allow_splitk && tiles < units && args.num_kb >= 16 && ws && ws->splitk) {
-    splits = (int)((2 * units + tiles - 1) / tiles);
-    if (splits > args.num_kb / 8) splits = args.num_kb / 8;
+    // between 2 and 4 work units per CTA (pair); among those, the count that leaves the last wave fullest
     const int64_t per = (int64_t)M * N * (int64_t)sizeof(float);
-    if ((int64_t)splits * per > (int64_t)ws->splitk_bytes) splits = (int)(ws->splitk_bytes / per);
+    int lo = (int)((2 * units + tiles - 1) / tiles), hi = (int)((4 * units + tiles - 1) / tiles);
+    int cap = args.num_kb / 8;
+    if ((int64_t)cap * per > (int64_t)ws->splitk_bytes) cap = (int)(ws->splitk_bytes / per);
+    if (hi > cap) hi = cap;
+    if (lo > hi) lo = hi;
+    double best = -1.0;
+    for (int sp = lo; sp <= hi && sp >= 1; ++sp) {
+      const int64_t total = tiles * sp;
+      const double fill = (double)total / (double)(ceil_div64(total, units) * units);
+      if (fill > best + 1e-9) { best = fill; splits = sp; }
+    }
     if (splits < 1) splits = 1;
   }
   args.kb_per_split = ceil_div(args.num_kb, splits);
