@@ -318,7 +318,7 @@ template <int BN> struct TcCfg {
 };
 
 // The epilogue of one output tile for one epilogue warp: rows row0 .. row0+31 (TMEM lanes q*32..), columns
-// [half*BN/2, (half+1)*BN/2) of tile column tn.  A warp may read only its quarter of the TMEM lanes; two warps
+// [half*BN/PARTS, (half+1)*BN/PARTS) of tile column tn.  A warp may read only its quarter of the TMEM lanes; PARTS warps
 // share a quarter and split the columns.  Each 32 x 32 block is loaded one row per thread, turned through a
 // padded shared-memory buffer, and then handled four rows per instruction with eight lanes per row, so that
 // global loads and stores of a row are contiguous 128-byte pieces.  Returns false if the bounded wait for the
@@ -333,20 +333,20 @@ template <int BN> struct TcCfg {
 //   EPI_RES   (+ bias) + fp32 residual (LayerNorm on the fly when res_mean is set), fp32 out (+ bf16 copy)
 enum { EPI_GENERAL = 0, EPI_DG = 1, EPI_BIAS = 2, EPI_GELU = 3, EPI_RES = 4 };
 
-template <int BN, typename CT, int MODE>
+template <int BN, typename CT, int MODE, int PARTS = 2>
 __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t row0, int tn, int half, int q, int lane,
                                               float* stage, uint32_t tmem_base, int buf, uint32_t tfull_addr,
                                               uint32_t parity, volatile int* abort_flag) {
   if constexpr (MODE == EPI_DG) {
-    uint2 pf[BN / 64][8];                       // packed bf16: 4 columns of one row per entry
+    uint2 pf[BN / (32 * PARTS)][8];                       // packed bf16: 4 columns of one row per entry
     const int sub = lane >> 3, slot = lane & 7;
     const int64_t rows_left = a.M - (row0 + sub);
     const int64_t step = 4 * a.ldc;
-    const int ncol0 = tn * BN + half * (BN / 2) + slot * 4;
+    const int ncol0 = tn * BN + half * (BN / PARTS) + slot * 4;
     const int64_t o0 = (row0 + sub) * a.ldc + ncol0;
     const bf16* pre = reinterpret_cast<const bf16*>(a.epi.dgelu_pre) + o0;
 #pragma unroll
-    for (int blk = 0; blk < BN / 64; ++blk) {
+    for (int blk = 0; blk < BN / (32 * PARTS); ++blk) {
       const bool col_ok = ncol0 + blk * 32 < a.N;
 #pragma unroll
       for (int rr = 0; rr < 8; ++rr)
@@ -355,8 +355,8 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
     if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
     tc_fence_after();
 #pragma unroll
-    for (int blk = 0; blk < BN / 64; ++blk) {
-      const int c0 = half * (BN / 2) + blk * 32;
+    for (int blk = 0; blk < BN / (32 * PARTS); ++blk) {
+      const int c0 = half * (BN / PARTS) + blk * 32;
       uint32_t v[32];
       tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
       tc_ld32_wait(v);
@@ -393,7 +393,7 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
       }
     }
 #pragma unroll 1
-    for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+    for (int c0 = half * (BN / PARTS); c0 < (half + 1) * (BN / PARTS); c0 += 32) {
       uint32_t v[32];
       tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
       tc_ld32_wait(v);
@@ -488,7 +488,7 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
       rs_l = a.epi.res_rstd[row0 + lane];
     }
 #pragma unroll 1
-    for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+    for (int c0 = half * (BN / PARTS); c0 < (half + 1) * (BN / PARTS); c0 += 32) {
       uint32_t v[32];
       tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
       tc_ld32_wait(v);
@@ -752,22 +752,25 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t da, uint64
       : "memory");
 }
 
-struct Tc2Cfg {
+// EW epilogue warps per CTA: 8 (two per TMEM lane quarter) or, for the light epilogues whose register use allows
+// it, 16 (four per quarter, 64 columns each) with one pipeline stage fewer
+template <int EW> struct Tc2Cfg {
   static constexpr int BN = 256;                       // columns of the pair's tile
   static constexpr int A_BYTES = BM * BK * 2;          // this CTA's 128 rows of A
   static constexpr int B_BYTES = (BN / 2) * BK * 2;    // this CTA's 128 columns of B
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = 6;
+  static constexpr int STAGES = EW == 16 ? 5 : 6;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_BYTES = EPI_WARPS * 32 * STAGE_LD * 4;
+  static constexpr int THREADS = 64 + 32 * EW;
+  static constexpr int EPI_BYTES = EW * 32 * STAGE_LD * 4;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 + 256;
 };
 
 // n_tiles_m counts 256-row tiles here
-template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
-__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                                const __grid_constant__ CUtensorMap tmB, TcArgs a) {
-  using Cfg = Tc2Cfg;
+template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL, int EW = EPI_WARPS>
+__global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                  const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+  using Cfg = Tc2Cfg<EW>;
   constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -793,7 +796,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc2_kernel(const __grid_co
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 2 * EPI_WARPS);   // one arrival per epilogue warp of either CTA
+      mbar_init(tempty_bar(b), 2 * EW);          // one arrival per epilogue warp of either CTA
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -904,7 +907,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc2_kernel(const __grid_co
       const int buf = (int)(it & 1);
       const int64_t row0 = (int64_t)tm * 2 * BM + (int64_t)rank * BM + q * 32;
       CT* Cs = C + (int64_t)split * a.split_stride;
-      if (!epilogue_tile<BN, CT, MODE>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
+      if (!epilogue_tile<BN, CT, MODE, EW / 4>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
                                      (uint32_t)((it >> 1) & 1), abort_flag)) {
         failed = true;
         break;
@@ -1004,19 +1007,20 @@ cudaError_t launch_tc_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUt
   return launch_tc<BN, false, false, CT>(ma, mb, args, grid, st);
 }
 
-template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL>
+template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL, int EW = EPI_WARPS>
 cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st) {
-  auto kern = gemm_tc2_kernel<A_K, B_K, CT, MODE>;
+  using Tc2 = Tc2Cfg<EW>;
+  auto kern = gemm_tc2_kernel<A_K, B_K, CT, MODE, EW>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tc2Cfg::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tc2::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(TC_THREADS);
-  cfg.dynamicSmemBytes = Tc2Cfg::SMEM_BYTES;
+  cfg.blockDim = dim3(Tc2::THREADS);
+  cfg.dynamicSmemBytes = Tc2::SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1149,11 +1153,11 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   const bool m_res = e.res && !e.gelu && !e.dgelu_pre && !e.accumulate && !e.pre && c_f32 && a_kmajor;
   if (pair) {
     if (dg_only) err = launch_tc2<true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
-    else if (m_gelu) err = launch_tc2<true, true, bf16, EPI_GELU>(ma, mb, args, grid, st);
+    else if (m_gelu) err = launch_tc2<true, true, bf16, EPI_GELU, 16>(ma, mb, args, grid, st);
     else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);
     else if (m_res && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES>(ma, mb, args, grid, st);
-    else if (m_bias && a_kmajor && b_kmajor && !c_f32) err = launch_tc2<true, true, bf16, EPI_BIAS>(ma, mb, args, grid, st);
-    else if (m_bias && a_kmajor && !b_kmajor && !c_f32) err = launch_tc2<true, false, bf16, EPI_BIAS>(ma, mb, args, grid, st);
+    else if (m_bias && a_kmajor && b_kmajor && !c_f32) err = launch_tc2<true, true, bf16, EPI_BIAS, 16>(ma, mb, args, grid, st);
+    else if (m_bias && a_kmajor && !b_kmajor && !c_f32) err = launch_tc2<true, false, bf16, EPI_BIAS, 16>(ma, mb, args, grid, st);
     else if (c_f32) err = launch_tc2_major<float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else err = launch_tc2_major<bf16>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
   } else if (dg_only) {
