@@ -63,8 +63,8 @@ __global__ void gather_scalar_kernel(const T* __restrict__ src, int64_t n_src_ro
 //   - an item whose rows all lie inside the chunk is written to its output row directly;
 //   - the item that entered the chunk from the left leaves its part in partial[chunk][0];
 //   - the item that leaves the chunk to the right leaves its part in partial[chunk][1].
-// A second launch adds, for every item that spans chunks, partial[first][1] and then
-// partial[c][0] for the following chunks in ascending c.  The order of additions depends only
+// A second launch adds, for every item that spans chunks, partial[first][1] and the following
+// chunks' partial[c][0] in a fixed association (eight interleaved ascending runs, then their sum).  The order of additions depends only
 // on (P, U, seg_off), never on scheduling: repeated runs are bit-identical.
 // Algorithmic bytes: 4*P*d read + 4*U*d written + 4P (perm) + 4(U+1) (seg_off).
 // ---------------------------------------------------------------------------
@@ -183,44 +183,71 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
   }
 }
 
-// one warp per (chunk, slab): if an item starts in this chunk and runs past its end, add its parts
+// one block per (chunk, slab): if an item starts in this chunk and runs past its end, add its parts.  Warp w adds
+// the following chunks' parts number w, w+8, ... (ascending), warp 0 starts from this chunk's own part, and the
+// eight warp sums are added in ascending w: a fixed association, whatever the schedule.
 template <int VPL>
 __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __restrict__ seg_off, int64_t P, int32_t U,
                                                            int d, int64_t R, int nchunks, int nslabs,
                                                            const int32_t* __restrict__ rows, int add,
                                                            float* __restrict__ out, const float* __restrict__ partial,
                                                            const int32_t* __restrict__ d_U) {
+  __shared__ float4 red[8][VPL][32];
   if (d_U) U = *d_U;
   if (U <= 0) return;
-  const int lane = threadIdx.x & 31;
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (w >= (int64_t)nchunks * nslabs) return;
-  const int chunk = (int)(w / nslabs), slab = (int)(w - (int64_t)chunk * nslabs);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int chunk = blockIdx.x / nslabs, slab = blockIdx.x - chunk * nslabs;
   const int col0 = slab * (VPL * 128);
   const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
   if (c0 >= c1 || c1 >= P) return;
   const int32_t u = find_segment(seg_off, U, c1 - 1);
   const int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
-  if (seg_begin < c0 || seg_end <= c1) return;      // not the first chunk of a spanning item
+  if (seg_begin < c0 || seg_end <= c1) return;      // not the first chunk of a spanning item (same for the whole block)
   const int last = (int)((seg_end - 1) / R);
   float4 acc[VPL];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) {
-    int c = col0 + (v * 32 + lane) * 4;
-    acc[v] = (c < d) ? *reinterpret_cast<const float4*>(partial + ((int64_t)chunk * 2 + 1) * d + c)
-                     : make_float4(0.f, 0.f, 0.f, 0.f);
+    const int c = col0 + (v * 32 + lane) * 4;
+    acc[v] = (w == 0 && c < d) ? *reinterpret_cast<const float4*>(partial + ((int64_t)chunk * 2 + 1) * d + c)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  for (int c = chunk + 1; c <= last; ++c) {
+  for (int c = chunk + 1 + w; c <= last; c += 32) {   // four parts in flight per warp
+    float4 x[4][VPL];
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-      int cc = col0 + (v * 32 + lane) * 4;
-      if (cc < d) {
-        float4 x = *reinterpret_cast<const float4*>(partial + ((int64_t)c * 2 + 0) * d + cc);
-        acc[v].x += x.x; acc[v].y += x.y; acc[v].z += x.z; acc[v].w += x.w;
+    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int cc = col0 + (v * 32 + lane) * 4;
+        x[k][v] = (c + 8 * k <= last && cc < d) ? *reinterpret_cast<const float4*>(partial + ((int64_t)(c + 8 * k) * 2 + 0) * d + cc)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (c + 8 * k <= last) {
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+          acc[v].x += x[k][v].x; acc[v].y += x[k][v].y; acc[v].z += x[k][v].z; acc[v].w += x[k][v].w;
+        }
       }
     }
   }
-  store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) red[w][v][lane] = acc[v];
+  __syncthreads();
+  if (w == 0) {
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      float4 t = red[0][v][lane];
+#pragma unroll
+      for (int k = 1; k < 8; ++k) {
+        const float4 y = red[k][v][lane];
+        t.x += y.x; t.y += y.y; t.z += y.z; t.w += y.w;
+      }
+      acc[v] = t;
+    }
+    store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
+  }
 }
 
 __global__ void touched_mark_kernel(const int32_t* __restrict__ unique, int32_t U, int32_t n_items,
@@ -325,7 +352,7 @@ static void segsum_run(const void* d_in, const int32_t* d_perm, const int32_t* d
   segsum_chunks_kernel<InT, VPL, 8><<<blocks, 256, 0, st>>>((const InT*)d_in, d_perm, d_seg_off, P, U, d, R, nchunks, nslabs,
                                                             d_rows, add, d_out, partial, status, d_U);
   if (nchunks > 1)
-    segsum_fixup_kernel<VPL><<<blocks, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, d_U);
+    segsum_fixup_kernel<VPL><<<(unsigned)warps, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, d_U);
 }
 
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,

@@ -1152,7 +1152,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   const bool m_gelu = e.gelu && e.pre && !e.dgelu_pre && !e.res && !e.accumulate && !e.copy_out && !c_f32 && a_kmajor && b_kmajor;
   const bool m_res = e.res && !e.gelu && !e.dgelu_pre && !e.accumulate && !e.pre && c_f32 && a_kmajor;
   if (pair) {
-    if (dg_only) err = launch_tc2<true, false, bf16, EPI_DG>(ma, mb, args, grid, st);
+    if (dg_only) err = launch_tc2<true, false, bf16, EPI_DG, 16>(ma, mb, args, grid, st);
     else if (m_gelu) err = launch_tc2<true, true, bf16, EPI_GELU, 16>(ma, mb, args, grid, st);
     else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);
     else if (m_res && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES>(ma, mb, args, grid, st);

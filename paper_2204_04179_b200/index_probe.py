@@ -1,6 +1,7 @@
 """Times dedup, gather and accumulate alone on one sweep cell (seeded Zipf IDs, uniform gradients).
 
     python -m paper_2204_04179_b200.index_probe [--p 1000000] [--items 100000] [--s 1.1] [--d 768] [--iters 20]
+    python -m paper_2204_04179_b200.index_probe --sweep [--iters 10]
 
 Prints one JSON line with milliseconds and achieved GB/s (algorithmic bytes / time) per kernel.
 """
@@ -48,6 +49,23 @@ def run_cell(P, N, s, d, iters=20, dev="cuda:0", seed=1):
     return out
 
 
+def sweep(budget_gb: float = 12.0, iters: int = 10):
+    """The kernel sweep: P in 1e4..1e7, item pool 1e3..1e6, Zipf s in {0.8, 1.1, 1.5}, d in {256, 768, 1024}.
+    Cells whose gradient buffer (4*P*d bytes) exceeds the budget are listed as pruned, not run."""
+    import torch
+    for P in (10**4, 10**5, 10**6, 10**7):
+        for d in (256, 768, 1024):
+            if 4.0 * P * d > budget_gb * 1e9:
+                print(json.dumps({"P": P, "d": d, "pruned": f"4*P*d = {4.0 * P * d / 1e9:.1f} GB exceeds the {budget_gb:.0f} GB per-buffer budget"}), flush=True)
+                continue
+            for N in (10**3, 10**4, 10**5, 10**6):
+                for s in (0.8, 1.1, 1.5):
+                    r = run_cell(P, N, s, d, iters)
+                    r["l2_resident"] = r["working_set_MB"] < 126.0
+                    print(json.dumps(r), flush=True)
+                    torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--p", type=int, default=1_000_000)
@@ -55,8 +73,12 @@ def main():
     ap.add_argument("--s", type=float, default=1.1)
     ap.add_argument("--d", type=int, default=768)
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--sweep", action="store_true", help="run the whole grid (one JSON line per cell)")
     a = ap.parse_args()
-    print(json.dumps(run_cell(a.p, a.items, a.s, a.d, a.iters)))
+    if a.sweep:
+        sweep(iters=a.iters)
+    else:
+        print(json.dumps(run_cell(a.p, a.items, a.s, a.d, a.iters)))
 
 
 if __name__ == "__main__":
