@@ -83,12 +83,18 @@ template <> struct Row4<bf16> {
   }
 };
 
-__device__ __forceinline__ int32_t find_segment(const int32_t* __restrict__ seg_off, int32_t U, int64_t j) {
-  // largest u in [0, U) with seg_off[u] <= j
-  int32_t lo = 0, hi = U - 1;
-  while (lo < hi) {
-    int32_t mid = (lo + hi + 1) >> 1;
-    if (seg_off[mid] <= j) lo = mid; else hi = mid - 1;
+// largest u in [0, U) with seg_off[u] <= j, found by the whole warp: every lane probes one of 32 evenly spaced
+// entries per round, so U = 10^6 takes four dependent loads instead of twenty.  All 32 lanes must call it.
+__device__ __forceinline__ int32_t find_segment(const int32_t* __restrict__ seg_off, int32_t U, int64_t j, int lane) {
+  int32_t lo = 0, n = U;                       // the answer lies in [lo, lo + n) and seg_off[lo] <= j
+  while (n > 1) {
+    const int32_t step = (n + 31) >> 5;
+    const int32_t idx = lo + lane * step;
+    const bool ok = (lane * step < n) && (seg_off[idx] <= j);
+    const unsigned m = __ballot_sync(0xffffffffu, ok) | 1u;
+    const int k = 31 - __clz(m);
+    n = min(step, n - k * step);
+    lo += k * step;
   }
   return lo;
 }
@@ -128,7 +134,7 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
   const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
   if (c0 >= c1) return;
 
-  int32_t u = find_segment(seg_off, U, c0);
+  int32_t u = find_segment(seg_off, U, c0, lane);
   int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
   float4 acc[VPL];
 #pragma unroll
@@ -200,7 +206,7 @@ __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __rest
   const int col0 = slab * (VPL * 128);
   const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
   if (c0 >= c1 || c1 >= P) return;
-  const int32_t u = find_segment(seg_off, U, c1 - 1);
+  const int32_t u = find_segment(seg_off, U, c1 - 1, lane);
   const int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
   if (seg_begin < c0 || seg_end <= c1) return;      // not the first chunk of a spanning item (same for the whole block)
   const int last = (int)((seg_end - 1) / R);
