@@ -78,12 +78,71 @@ __device__ __forceinline__ void st4(bf16* p, const float (&x)[4]) {
 // y = |x| / sqrt(2) the exponential exp(-x^2 / 2) is also the Gaussian density the derivative needs.
 __device__ __forceinline__ void gelu_parts(float x, float& cdf, float& pdf) {
   const float ax = fabsf(x);
-  const float ex = __expf(-0.5f * x * x);
-  const float t = __fdividef(1.f, 1.f + 0.3275911f * 0.70710678f * ax);
+  float ex, t;                                            // flush-to-zero forms: one MUFU each, no range fix-up
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(ex) : "f"(x * x * -0.72134752f));            // exp(-x^2 / 2)
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678f, ax, 1.f)));
   const float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
   const float erf_abs = 1.f - poly * ex;                  // erf(|x| / sqrt 2)
   cdf = 0.5f * (1.f + copysignf(erf_abs, x));
   pdf = 0.39894228f * ex;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+// The same for two values at a time with the packed fp32 instructions of sm_100 (two lanes of one 64-bit
+// register): x holds the two pre-activations; on return g = gelu(x), dg = gelu'(x).  Half the instruction
+// slots of the scalar form, which is what bounds the epilogue of the first feed-forward product.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_const(float c) {
+  const uint64_t u = (uint64_t)__float_as_uint(c);
+  return u | (u << 32);
+}
+__device__ __forceinline__ void gelu_pair(uint64_t x, uint64_t& g, uint64_t& dg) {
+  float e0, e1, y0, y1;
+  f2_unpack(f2_mul(f2_mul(x, x), f2_const(-0.72134752f)), e0, e1);
+  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(e0));                          // exp(-x^2 / 2)
+  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(e1));
+  const uint64_t ex = f2_pack(e0, e1);
+  f2_unpack(f2_fma(x & 0x7FFFFFFF7FFFFFFFull, f2_const(0.3275911f * 0.70710678f), f2_const(1.f)), y0, y1);
+  asm("rcp.approx.ftz.f32 %0, %0;" : "+f"(y0));
+  asm("rcp.approx.ftz.f32 %0, %0;" : "+f"(y1));
+  const uint64_t t = f2_pack(y0, y1);
+  uint64_t p = f2_fma(t, f2_const(1.061405429f), f2_const(-1.453152027f));
+  p = f2_fma(p, t, f2_const(1.421413741f));
+  p = f2_fma(p, t, f2_const(-0.284496736f));
+  p = f2_fma(p, t, f2_const(0.254829592f));
+  p = f2_mul(p, t);
+  const uint64_t h = f2_fma(f2_mul(p, ex), f2_const(-0.5f), f2_const(0.5f));    // erf(|x| / sqrt 2) / 2
+  const uint64_t cdf = f2_add(h | (x & 0x8000000080000000ull), f2_const(0.5f));   // 1/2 + sign(x) * h
+  g = f2_mul(x, cdf);
+  dg = f2_fma(f2_mul(x, ex), f2_const(0.39894228f), cdf);
+}
+__device__ __forceinline__ uint32_t f2_to_bf16x2(uint64_t v) {
+  float lo, hi;
+  f2_unpack(v, lo, hi);
+  return pack_bf16x2(lo, hi);
 }
 
 // what one lane reads before it may store anything for its 4 columns of one row: the residual, the
@@ -232,6 +291,29 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
       "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
+}
+
+// bulk tensor store of a shared-memory box (the box is clipped at the tensor's edges) and its bookkeeping
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int32_t c0, int32_t c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(c0),
+               "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 unpack_bf16x2(uint32_t u) {
+  return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u));
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -752,25 +834,137 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t da, uint64
       : "memory");
 }
 
+// Epilogue of the pair kernel for bf16 results (EPI_BIAS, EPI_GELU, EPI_DG): one warp owns rows row0 .. row0+31
+// and NB blocks of 32 columns from global column col0 (tile column c_local).  A thread keeps its own row: 32
+// accumulators from tensor memory per block, the arithmetic, 64 bytes of bf16 written into a 32-row x 64-column
+// box in shared memory (128-byte rows whose 16-byte pieces are XOR-swizzled as the 128-byte swizzle of the
+// tensor map expects, which also keeps the writes free of bank conflicts).  Two blocks fill a box, and lane 0
+// hands it to a bulk tensor store, which writes whole 128-byte lines and clips the box at the matrix edges.
+// EPI_GELU fills a second box with the derivative; EPI_DG (NB = 2) first fetches the box of the saved derivative
+// with a bulk tensor load (issued before the wait for the accumulator), multiplies in place and stores the same
+// box.  The accumulator buffer is handed back as soon as the last block has been read.  sbuf: 4 KB (8 KB for
+// EPI_GELU), 1024-byte aligned, private to the warp.  Returns false if a bounded wait gave up.
+template <int MODE, int NB>
+__device__ __forceinline__ bool epilogue_tile_ts(const TcArgs& a, const CUtensorMap* tmC, const CUtensorMap* tmP, int32_t row0,
+                                                 int32_t col0, int c_local, int q, int lane, uint32_t sbuf,
+                                                 uint32_t tmem_base, int buf, uint32_t tfull_addr, uint32_t parity,
+                                                 volatile int* abort_flag, uint32_t tempty_remote, uint32_t ld_bar,
+                                                 uint32_t ld_parity) {
+  static_assert(MODE != EPI_DG || NB == 2, "the derivative's box is fetched once per tile");
+  const uint32_t swz = (uint32_t)(lane & 7);
+  const uint32_t srow = sbuf + (uint32_t)lane * 128u;
+  if constexpr (MODE == EPI_DG) {
+    if (lane == 0) {
+      bulk_wait_read_all();                                // the last tile's store has read the box
+      mbar_expect_tx(ld_bar, 4096);
+      tma_load_2d(sbuf, tmP, col0, row0, ld_bar);
+    }
+    __syncwarp();
+  }
+  if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+  tc_fence_after();
+  if constexpr (MODE == EPI_DG) {
+    if (!mbar_wait(ld_bar, ld_parity, abort_flag)) return false;
+  }
+  const bool rows_ok = row0 < a.M;                         // a box that starts below the matrix is not stored
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    uint32_t v[32];
+    tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c_local + b * 32), v);
+    tc_ld32_wait(v);
+    if (b == NB - 1) {                                     // every value of this tile is in registers now
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(tempty_remote);
+    }
+    const int nbx = col0 + (b >> 1) * 64;                  // first column of the box
+    const int n = col0 + b * 32;
+    if (nbx >= a.N || !rows_ok) continue;
+    const uint32_t p0 = (uint32_t)(b & 1) * 4u;            // this block's first 16-byte piece of the row
+    uint32_t oc[16];
+    if constexpr (MODE == EPI_DG) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint4 g4 = lds128(srow + (((p0 + (uint32_t)c) ^ swz) << 4));
+        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 gg = unpack_bf16x2(gw[i]);
+          oc[4 * c + i] = pack_bf16x2(__uint_as_float(v[8 * c + 2 * i]) * gg.x, __uint_as_float(v[8 * c + 2 * i + 1]) * gg.y);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        sts128(srow + (((p0 + (uint32_t)c) ^ swz) << 4), oc[4 * c], oc[4 * c + 1], oc[4 * c + 2], oc[4 * c + 3]);
+    } else {
+      uint32_t op[MODE == EPI_GELU ? 16 : 1];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (a.epi.bias && n + 4 * j < a.N) b4 = __ldg(reinterpret_cast<const float4*>(a.epi.bias + n + 4 * j));
+        if constexpr (MODE == EPI_GELU) {
+          uint64_t g0, g1, d0, d1;
+          gelu_pair(f2_add(f2_pack(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])), f2_pack(b4.x, b4.y)), g0, d0);
+          gelu_pair(f2_add(f2_pack(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])), f2_pack(b4.z, b4.w)), g1, d1);
+          oc[2 * j] = f2_to_bf16x2(g0);
+          oc[2 * j + 1] = f2_to_bf16x2(g1);
+          op[2 * j] = f2_to_bf16x2(d0);
+          op[2 * j + 1] = f2_to_bf16x2(d1);
+        } else {
+          oc[2 * j] = pack_bf16x2(__uint_as_float(v[4 * j]) + b4.x, __uint_as_float(v[4 * j + 1]) + b4.y);
+          oc[2 * j + 1] = pack_bf16x2(__uint_as_float(v[4 * j + 2]) + b4.z, __uint_as_float(v[4 * j + 3]) + b4.w);
+        }
+      }
+      if ((b & 1) == 0) {                                  // the last store from the box(es) has read them
+        if (lane == 0) bulk_wait_read_all();
+        __syncwarp();
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        sts128(srow + (((p0 + (uint32_t)c) ^ swz) << 4), oc[4 * c], oc[4 * c + 1], oc[4 * c + 2], oc[4 * c + 3]);
+      if constexpr (MODE == EPI_GELU) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          sts128(srow + 4096u + (((p0 + (uint32_t)c) ^ swz) << 4), op[4 * c], op[4 * c + 1], op[4 * c + 2], op[4 * c + 3]);
+      }
+    }
+    if (b & 1) {
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_2d(tmC, sbuf, nbx, row0);
+        if constexpr (MODE == EPI_GELU) tma_store_2d(tmP, sbuf + 4096, nbx, row0);
+        bulk_commit();
+      }
+    }
+  }
+  return true;
+}
+
 // EW epilogue warps per CTA: 8 (two per TMEM lane quarter) or, for the light epilogues whose register use allows
 // it, 16 (four per quarter, 64 columns each) with one pipeline stage fewer
-template <int EW> struct Tc2Cfg {
+template <int EW, int WARP_BYTES = 4096> struct Tc2Cfg {
   static constexpr int BN = 256;                       // columns of the pair's tile
   static constexpr int A_BYTES = BM * BK * 2;          // this CTA's 128 rows of A
   static constexpr int B_BYTES = (BN / 2) * BK * 2;    // this CTA's 128 columns of B
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = EW == 16 ? 5 : 6;
+  static constexpr int EPI_BYTES = EW * WARP_BYTES;    // the epilogue warps' private buffers
+  static constexpr int STAGES = (232448 - 1024 - 512 - EPI_BYTES) / STAGE_BYTES;   // 6 with 32 KB of buffers, 5 with 64 KB
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int THREADS = 64 + 32 * EW;
-  static constexpr int EPI_BYTES = EW * 32 * STAGE_LD * 4;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 + 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 + 512;
 };
 
-// n_tiles_m counts 256-row tiles here
+// n_tiles_m counts 256-row tiles here.  tmC / tmP: maps of the bf16 result and of the GELU-derivative matrix
+// (boxes of 32 rows x 64 columns, 128-byte swizzle) for the variants whose epilogue uses bulk tensor stores; unused otherwise.
 template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL, int EW = EPI_WARPS>
 __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                                  const __grid_constant__ CUtensorMap tmB, TcArgs a) {
-  using Cfg = Tc2Cfg<EW>;
+                                                                  const __grid_constant__ CUtensorMap tmB,
+                                                                  const __grid_constant__ CUtensorMap tmC,
+                                                                  const __grid_constant__ CUtensorMap tmP, TcArgs a) {
+  constexpr bool TS = sizeof(CT) == 2 && ((EW == 16 && MODE == EPI_DG) || MODE == EPI_BIAS || MODE == EPI_GELU);
+  constexpr int WARP_BYTES = (TS && MODE == EPI_GELU) ? 8192 : 4096;
+  using Cfg = Tc2Cfg<EW, WARP_BYTES>;
   constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -785,6 +979,7 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };  // used in the leader
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  auto ld_bar = [&](int w) { return bar0 + 8u * (2 * STAGES + 6 + w); };      // one per epilogue warp (EPI_DG loads)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -797,6 +992,9 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
       mbar_init(tempty_bar(b), 2 * EW);          // one arrival per epilogue warp of either CTA
+    }
+    if (TS) {
+      for (int w = 0; w < EW; ++w) mbar_init(ld_bar(w), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -822,6 +1020,7 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
+      const uint32_t lead_bar0 = map_to_cta(bar0, 0);          // the leader's barrier block, as seen from this CTA
       for (int64_t t = cluster_id; t < total && !failed; t += n_clusters) {
         const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
         const int64_t r = t - (int64_t)split * a.n_tiles_m * a.n_tiles_n;
@@ -831,7 +1030,7 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
         const int n0 = tn * BN + (int)rank * (BN / 2);          // this CTA's columns of B
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { failed = true; break; }
-          const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+          const uint32_t lead_full = lead_bar0 + 8u * s;           // the leader's full_bar(s)
           mbar_arrive_expect_tx_remote(lead_full, Cfg::STAGE_BYTES);
           const uint32_t sa = tiles + s * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
           if (A_K) {
@@ -862,6 +1061,13 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
       int s = 0;
       uint32_t ph = 0;
       int64_t it = 0;
+      // This thread shares its scheduler with four busy epilogue warps, so the loop is kept to a few instructions
+      // per k-block: the descriptors of stage 0 are built once (a later stage or k-step only adds to the 14-bit
+      // address field, which cannot overflow inside shared memory), and so are the barrier addresses of both CTAs.
+      const uint64_t da0 = A_K ? make_desc(tiles, 16, 1024) : make_desc(tiles, 8192, 1024);
+      const uint64_t db0 = B_K ? make_desc(tiles + Cfg::A_BYTES, 16, 1024) : make_desc(tiles + Cfg::A_BYTES, 8192, 1024);
+      constexpr uint32_t ka = (A_K ? 32 : 2048) >> 4, kbs = (B_K ? 32 : 2048) >> 4;
+      const uint32_t rbar0 = map_to_cta(bar0, 0), rbar1 = map_to_cta(bar0, 1);
       for (int64_t t = cluster_id; t < total && !failed; t += n_clusters, ++it) {
         const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
         const int kb0 = split * a.kb_per_split, kb1 = min(kb0 + a.kb_per_split, a.num_kb);
@@ -869,23 +1075,26 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
         if (!mbar_wait(tempty_bar(buf), (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+        uint32_t acc = 0u;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
-          const uint32_t sa = tiles + s * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
+          const uint32_t soff = (uint32_t)(s * (Cfg::STAGE_BYTES >> 4));
+          const uint64_t da = da0 + soff, db = db0 + soff;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t da = A_K ? make_desc(sa + k * 32, 16, 1024) : make_desc(sa + k * 2048, 8192, 1024);
-            const uint64_t db = B_K ? make_desc(sb + k * 32, 16, 1024) : make_desc(sb + k * 2048, 8192, 1024);
-            tc_mma_pair(tmem_d, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            tc_mma_pair(tmem_d, da + (uint64_t)(k * ka), db + (uint64_t)(k * kbs), idesc, acc);
+            acc = 1u;
           }
-          tc_commit_pair(map_to_cta(empty_bar(s), 0));      // the stage is free in both CTAs once these MMAs are done
-          tc_commit_pair(map_to_cta(empty_bar(s), 1));
+          const uint32_t eb = 8u * (uint32_t)(STAGES + s);  // empty_bar(s): the stage is free in both CTAs once these MMAs are done
+          tc_commit_pair(rbar0 + eb);
+          tc_commit_pair(rbar1 + eb);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (failed) break;
-        tc_commit_pair(map_to_cta(tfull_bar(buf), 0));      // accumulator complete in both CTAs
-        tc_commit_pair(map_to_cta(tfull_bar(buf), 1));
+        const uint32_t fb = 8u * (uint32_t)(2 * STAGES + buf);   // tfull_bar(buf): accumulator complete in both CTAs
+        tc_commit_pair(rbar0 + fb);
+        tc_commit_pair(rbar1 + fb);
       }
       if (failed) {
         *abort_flag = 1;
@@ -906,15 +1115,27 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
       const int tm = (int)(r / a.n_tiles_n), tn = (int)(r % a.n_tiles_n);
       const int buf = (int)(it & 1);
       const int64_t row0 = (int64_t)tm * 2 * BM + (int64_t)rank * BM + q * 32;
-      CT* Cs = C + (int64_t)split * a.split_stride;
-      if (!epilogue_tile<BN, CT, MODE, EW / 4>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
-                                     (uint32_t)((it >> 1) & 1), abort_flag)) {
-        failed = true;
-        break;
+      if constexpr (TS) {
+        constexpr int NB = 32 / EW;               // blocks of 32 columns per warp
+        if (!epilogue_tile_ts<MODE, NB>(a, &tmC, &tmP, (int32_t)row0, tn * BN + half * (NB * 32), half * (NB * 32), q, lane,
+                                    tiles + STAGES * Cfg::STAGE_BYTES + (uint32_t)(ew * WARP_BYTES), tmem_base, buf, tfull_bar(buf),
+                                    (uint32_t)((it >> 1) & 1), abort_flag, map_to_cta(tempty_bar(buf), 0), ld_bar(ew),
+                                    (uint32_t)(it & 1))) {
+          failed = true;
+          break;
+        }
+      } else {
+        CT* Cs = C + (int64_t)split * a.split_stride;
+        if (!epilogue_tile<BN, CT, MODE, EW / 4>(a, Cs, row0, tn, half, q, lane, stage, tmem_base, buf, tfull_bar(buf),
+                                                 (uint32_t)((it >> 1) & 1), abort_flag)) {
+          failed = true;
+          break;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(buf), 0));
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(buf), 0));
     }
+    if (TS && lane == 0) bulk_wait_all();       // this warp's stores are complete before the CTA may exit
     if (failed && lane == 0) {
       *abort_flag = 1;
       gram_device_fail(a.status, GRAM_ERR_TIMEOUT);
@@ -973,7 +1194,7 @@ EncodeTiledFn get_encode_fn() {
 
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `ld` elements apart
 bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_inner,
-              uint32_t box_outer) {
+              uint32_t box_outer, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {inner, outer};
@@ -981,7 +1202,7 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t es[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1008,8 +1229,9 @@ cudaError_t launch_tc_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUt
 }
 
 template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL, int EW = EPI_WARPS>
-cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st) {
-  using Tc2 = Tc2Cfg<EW>;
+cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st,
+                       const CUtensorMap* mc = nullptr, const CUtensorMap* mp = nullptr) {
+  using Tc2 = Tc2Cfg<EW, (sizeof(CT) == 2 && MODE == EPI_GELU) ? 8192 : 4096>;
   auto kern = gemm_tc2_kernel<A_K, B_K, CT, MODE, EW>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -1029,7 +1251,7 @@ cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArg
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, ma, mb, args);
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, mc ? *mc : ma, mp ? *mp : (mc ? *mc : ma), args);
 }
 template <typename CT>
 cudaError_t launch_tc2_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid,
@@ -1152,12 +1374,20 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   const bool m_gelu = e.gelu && e.pre && !e.dgelu_pre && !e.res && !e.accumulate && !e.copy_out && !c_f32 && a_kmajor && b_kmajor;
   const bool m_res = e.res && !e.gelu && !e.dgelu_pre && !e.accumulate && !e.pre && c_f32 && a_kmajor;
   if (pair) {
-    if (dg_only) err = launch_tc2<true, false, bf16, EPI_DG, 16>(ma, mb, args, grid, st);
-    else if (m_gelu) err = launch_tc2<true, true, bf16, EPI_GELU, 16>(ma, mb, args, grid, st);
+    // bf16 results leave through bulk tensor stores: maps of C and of the GELU-derivative matrix (boxes of 32 rows x 64 columns)
+    const void* aux = e.gelu ? e.pre : e.dgelu_pre;
+    const bool ts = !c_f32 && M < (int64_t)1 << 31 && (!aux || (uintptr_t)aux % 16 == 0);
+    CUtensorMap mc, mp;
+    bool ts_ok = ts && make_map(&mc, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, 32);
+    if (ts_ok && aux) ts_ok = make_map(&mp, aux, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, 32);
+    const CUtensorMap* pc = &mc;
+    const CUtensorMap* pp = aux ? &mp : &mc;
+    if (dg_only && ts_ok) err = launch_tc2<true, false, bf16, EPI_DG, 16>(ma, mb, args, grid, st, pc, pp);
+    else if (m_gelu && ts_ok) err = launch_tc2<true, true, bf16, EPI_GELU, 8>(ma, mb, args, grid, st, pc, pp);
     else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);
     else if (m_res && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES>(ma, mb, args, grid, st);
-    else if (m_bias && a_kmajor && b_kmajor && !c_f32) err = launch_tc2<true, true, bf16, EPI_BIAS, 16>(ma, mb, args, grid, st);
-    else if (m_bias && a_kmajor && !b_kmajor && !c_f32) err = launch_tc2<true, false, bf16, EPI_BIAS, 16>(ma, mb, args, grid, st);
+    else if (m_bias && a_kmajor && b_kmajor && ts_ok) err = launch_tc2<true, true, bf16, EPI_BIAS, 8>(ma, mb, args, grid, st, pc, pp);
+    else if (m_bias && a_kmajor && !b_kmajor && ts_ok) err = launch_tc2<true, false, bf16, EPI_BIAS, 8>(ma, mb, args, grid, st, pc, pp);
     else if (c_f32) err = launch_tc2_major<float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else err = launch_tc2_major<bf16>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
   } else if (dg_only) {
