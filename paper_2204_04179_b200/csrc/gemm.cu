@@ -22,6 +22,7 @@ struct EpiDev {
   void* pre;
   const void* dgelu_pre;
   void* copy_out;
+  float* colsum_part;
   int gelu;
   int accumulate;
 };
@@ -936,6 +937,25 @@ __device__ __forceinline__ bool epilogue_tile_ts(const TcArgs& a, const CUtensor
         if constexpr (MODE == EPI_GELU) tma_store_2d(tmP, sbuf + 4096, nbx, row0);
         bulk_commit();
       }
+      if constexpr (MODE == EPI_DG) {
+        if (a.epi.colsum_part) {
+          // column sums of the box as stored (rows and columns outside the matrix hold zeros): lane c adds
+          // columns 2c, 2c+1 over the 32 rows in ascending order and writes row (row0 / 32) of the partial sums
+          float s0 = 0.f, s1 = 0.f;
+          const uint32_t piece = (uint32_t)(lane >> 2), word = (uint32_t)(lane & 3) * 4u;
+#pragma unroll 8
+          for (uint32_t r = 0; r < 32; ++r) {
+            uint32_t w;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(sbuf + r * 128u + ((piece ^ (r & 7u)) << 4) + word) : "memory");
+            const float2 f = unpack_bf16x2(w);
+            s0 += f.x;
+            s1 += f.y;
+          }
+          const int cc = nbx + 2 * lane;
+          if (cc < a.N) *reinterpret_cast<float2*>(a.epi.colsum_part + (int64_t)(row0 >> 5) * a.N + cc) = make_float2(s0, s1);
+          __syncwarp();                                    // every lane has read the box before it is refilled
+        }
+      }
     }
   }
   return true;
@@ -1264,6 +1284,15 @@ cudaError_t launch_tc2_major(bool a_k, bool b_k, const CUtensorMap& ma, const CU
 
 }  // namespace
 
+static bool pair_enabled_env() {
+  static const bool on = []() { const char* v = getenv("GRAM_GEMM_PAIR"); return !(v && v[0] == '0'); }();
+  return on;
+}
+bool gemm_fused_colsum(int dtype, int64_t M, int N) {
+  const bool bn256 = (N % 256 == 0 || N > 1024);
+  return dtype == GRAM_BF16 && pair_enabled_env() && bn256 && M >= 2 * BM && M < ((int64_t)1 << 31) && get_encode_fn() != nullptr;
+}
+
 gram_status gemm_ws_alloc(gram_ctx* ctx, GemmWorkspace* ws, size_t splitk_bytes) {
   ws->splitk_bytes = splitk_bytes;
   if (splitk_bytes) GRAM_CUDA(ctx, cudaMalloc(&ws->splitk, splitk_bytes));
@@ -1281,7 +1310,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   if (M == 0 || N == 0) return GRAM_OK;
   if (!A || !B || !C) return gram_set_error(ctx, "gemm: null operand"), GRAM_ERR_ARG;
   EpiDev e{epi.bias, epi.res, epi.res_mean, epi.res_rstd, epi.res_gamma, epi.res_beta, epi.pre, epi.dgelu_pre, epi.copy_out,
-           epi.gelu, epi.accumulate};
+           epi.colsum_part, epi.gelu, epi.accumulate};
   if (dtype == GRAM_F32) {
     if (!c_f32) return gram_set_error(ctx, "gemm: fp32 operands need an fp32 result"), GRAM_ERR_UNSUPPORTED;
     ProfScope prof(ctx, GRAM_K_GEMM, 2.0 * (double)M * N * (double)K, 1, st, epi.tag ? epi.tag : "gemm_f32");
@@ -1302,8 +1331,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
     return gram_set_error(ctx, "gemm: N must be a multiple of 8 and the epilogue's vectors 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
   const int BNsel = (N % 256 == 0 || N > 1024) ? 256 : (N > 64 ? 128 : 64);
   // pairs of SMs (256 x 256 tiles) when the problem has full-height tiles; GRAM_GEMM_PAIR=0 keeps single CTAs
-  static const bool pair_enabled = []() { const char* v = getenv("GRAM_GEMM_PAIR"); return !(v && v[0] == '0'); }();
-  const bool pair = pair_enabled && BNsel == 256 && M >= 2 * BM;
+  const bool pair = pair_enabled_env() && BNsel == 256 && M >= 2 * BM;
   CUtensorMap ma, mb;
   bool ok;
   if (a_kmajor) ok = make_map(&ma, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM);
@@ -1349,7 +1377,7 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
     args.C = ws->splitk;
     args.ldc = N;
     args.split_stride = (int64_t)M * N;
-    args.epi = EpiDev{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0};
+    args.epi = EpiDev{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0};
     if (pair && !a_kmajor && !b_kmajor) err = launch_tc2<false, false, float, EPI_BIAS>(ma, mb, args, grid, st);
     else if (pair) err = launch_tc2_major<float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
     else if (BNsel == 256) err = launch_tc_major<256, float>(a_kmajor, b_kmajor, ma, mb, args, grid, st);
@@ -1367,6 +1395,8 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
   args.ldc = ldc;
   args.split_stride = 0;
   args.epi = e;
+  if (e.colsum_part && !(pair && e.dgelu_pre && !c_f32))
+    return gram_set_error(ctx, "gemm: column-sum partials need the paired GELU-derivative variant"), GRAM_ERR_UNSUPPORTED;
   const bool dg_only = e.dgelu_pre && !e.bias && !e.res && !e.accumulate && !e.copy_out && !e.gelu && !c_f32 && a_kmajor &&
                        !b_kmajor;
   const bool others = e.gelu || e.dgelu_pre || e.res || e.accumulate || e.copy_out || e.pre;
@@ -1382,6 +1412,8 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
     if (ts_ok && aux) ts_ok = make_map(&mp, aux, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, 32);
     const CUtensorMap* pc = &mc;
     const CUtensorMap* pp = aux ? &mp : &mc;
+    if (e.colsum_part && !(dg_only && ts_ok))
+      return gram_set_error(ctx, "gemm: column-sum partials need the GELU-derivative variant with bulk stores"), GRAM_ERR_UNSUPPORTED;
     if (dg_only && ts_ok) err = launch_tc2<true, false, bf16, EPI_DG, 16>(ma, mb, args, grid, st, pc, pp);
     else if (m_gelu && ts_ok) err = launch_tc2<true, true, bf16, EPI_GELU, 8>(ma, mb, args, grid, st, pc, pp);
     else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);

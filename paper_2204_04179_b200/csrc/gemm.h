@@ -12,6 +12,9 @@
 //               (the fp32 residual stream: a layer's input is the LayerNorm of the previous fp32 sum)
 //   accumulate: v += C(m, n)                                          (fp32 C only)
 //   copy_out:   copy_out(m, n) = v as well                            (operand-typed copy of the result)
+//   colsum_part: with dgelu_pre on the tensor cores only (see gemm_fused_colsum): row i of this fp32
+//               [ceil(M / 32), N] matrix receives the column sums of rows 32 i .. 32 i + 31 of the stored
+//               (rounded) result, i.e. the partial sums of the bias gradient of the layer below
 // res is fp32; pre, dgelu_pre and copy_out have the operands' element type (bf16 on the tensor
 // cores, float in the fp32 kernel).  All of them share C's leading dimension.
 struct GemmEpilogue {
@@ -24,6 +27,7 @@ struct GemmEpilogue {
   void* pre = nullptr;
   const void* dgelu_pre = nullptr;
   void* copy_out = nullptr;
+  float* colsum_part = nullptr;
   int gelu = 0;
   int accumulate = 0;
   const char* tag = nullptr;   // names the call site in profiles (host side only)
@@ -44,6 +48,9 @@ struct GemmWorkspace {
 gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void* A, int a_kmajor, int64_t lda,
                         const void* B, int b_kmajor, int64_t ldb, void* C, int c_f32, int64_t ldc, int64_t M, int N,
                         int64_t K, const GemmEpilogue& epi, int allow_splitk, cudaStream_t st);
+
+// true when gemm_launch(dtype, ..., M, N, ...) with dgelu_pre set runs the variant that can fill colsum_part
+bool gemm_fused_colsum(int dtype, int64_t M, int N);
 
 gram_status gemm_ws_alloc(gram_ctx* ctx, GemmWorkspace* ws, size_t splitk_bytes);
 void gemm_ws_free(GemmWorkspace* ws);

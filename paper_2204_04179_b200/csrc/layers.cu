@@ -112,20 +112,24 @@ __global__ void __launch_bounds__(256, 2) ln_bwd_kernel(const float* __restrict_
                                                         const float* __restrict__ mean, const float* __restrict__ rstd,
                                                         const float* __restrict__ g, float* __restrict__ dz,
                                                         T* __restrict__ dz_b, float* __restrict__ part, int64_t rows,
-                                                        int d) {
-  extern __shared__ float sacc[];          // [2][d]: dgamma, dbeta of this block; then [d]: gamma
-  float* sgam = sacc + 2 * d;
+                                                        int d, int want_col) {
+  // [3][d]: dgamma, dbeta and the column sums of dz of this block; then [d]: gamma; then, when the column sums
+  // are wanted, one float4 per (warp, i, lane): each thread's running column sums (registers are all taken)
+  extern __shared__ float sacc[];
+  float* sgam = sacc + 3 * d;
+  float4* scol = reinterpret_cast<float4*>(sgam + d) + (threadIdx.x >> 5) * (NQ * 32) + (threadIdx.x & 31);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   const int64_t w = (int64_t)blockIdx.x * nwb + warp;
   const int64_t nw = (int64_t)gridDim.x * nwb;
   for (int i = threadIdx.x; i < d; i += blockDim.x) sgam[i] = g[i];
-  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sacc[i] = 0.f;
+  for (int i = threadIdx.x; i < 3 * d; i += blockDim.x) sacc[i] = 0.f;
   __syncthreads();
   float4 ag[NQ], ab[NQ];
 #pragma unroll
   for (int i = 0; i < NQ; ++i) {
     ag[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     ab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (want_col) scol[i * 32] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int64_t r = w; r < rows; r += nw) {
     const float mu = mean[r], rs = rstd[r];
@@ -163,6 +167,11 @@ __global__ void __launch_bounds__(256, 2) ln_bwd_kernel(const float* __restrict_
                                      rs * (dd[i].z - s1 - xh[i].z * s2), rs * (dd[i].w - s1 - xh[i].w * s2));
         st4t(dz + r * d + c, o);
         if (dz_b) st4t(dz_b + r * d + c, o);
+        if (want_col) {
+          float4 t = scol[i * 32];
+          t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+          scol[i * 32] = t;
+        }
       }
     }
   }
@@ -174,12 +183,16 @@ __global__ void __launch_bounds__(256, 2) ln_bwd_kernel(const float* __restrict_
         if (c < d) {
           sacc[c] += ag[i].x; sacc[c + 1] += ag[i].y; sacc[c + 2] += ag[i].z; sacc[c + 3] += ag[i].w;
           sacc[d + c] += ab[i].x; sacc[d + c + 1] += ab[i].y; sacc[d + c + 2] += ab[i].z; sacc[d + c + 3] += ab[i].w;
+          if (want_col) {
+            const float4 t = scol[i * 32];
+            sacc[2 * d + c] += t.x; sacc[2 * d + c + 1] += t.y; sacc[2 * d + c + 2] += t.z; sacc[2 * d + c + 3] += t.w;
+          }
         }
       }
     }
     __syncthreads();
   }
-  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) part[(int64_t)blockIdx.x * 2 * d + i] = sacc[i];
+  for (int i = threadIdx.x; i < 3 * d; i += blockDim.x) part[(int64_t)blockIdx.x * 3 * d + i] = sacc[i];
 }
 
 // out[c] += scale * sum_b part[b*stride + c]   (two outputs when out2 != null: second half of each partial row).
@@ -724,16 +737,18 @@ gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const fl
 
 gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const float* z, const float* mean,
                                const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
-                               float* dbeta, float* scratch, int64_t rows, int d, cudaStream_t st) {
+                               float* dbeta, float* dcol, float* scratch, int64_t rows, int d, cudaStream_t st) {
   if (rows == 0) return GRAM_OK;
   if (d > 1024 || (d & 3)) return gram_set_error(ctx, "LayerNorm: d must be a multiple of 4 and at most 1024"), GRAM_ERR_UNSUPPORTED;
-  int cap = (int)(kRedScratchBytes / ((size_t)2 * d * sizeof(float)));
+  int cap = (int)(kRedScratchBytes / ((size_t)3 * d * sizeof(float)));
   if (cap > kNumSMs * 8) cap = kNumSMs * 8;
   const int blocks = grid_for(rows * 32, 256, cap);
-  const size_t smem = (size_t)3 * d * sizeof(float);
-  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 2, st, "ln_bwd");
-  DISPATCH_T(dtype, DISPATCH_NQ(d, ln_bwd_kernel<T, NQ><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d)));
-  reduce_partials_kernel<<<ceil_div(d, 32), 256, 0, st>>>(scratch, blocks, (int64_t)2 * d, d, dgamma, dbeta, 1.f);
+  const int nq = d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : d <= 768 ? 6 : 8;   // float4 per lane: the kernel's NQ
+  const size_t smem = (size_t)4 * d * sizeof(float) + (dcol ? (size_t)8 * nq * 32 * sizeof(float4) : 0);
+  ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), dcol ? 3 : 2, st, "ln_bwd");
+  DISPATCH_T(dtype, DISPATCH_NQ(d, ln_bwd_kernel<T, NQ><<<blocks, 256, smem, st>>>(dy, z, mean, rstd, gamma, dz, (T*)dz_b, scratch, rows, d, dcol ? 1 : 0)));
+  reduce_partials_kernel<<<ceil_div(d, 32), 256, 0, st>>>(scratch, blocks, (int64_t)3 * d, d, dgamma, dbeta, 1.f);
+  if (dcol) reduce_partials_kernel<<<ceil_div(d, 32), 256, 0, st>>>(scratch + 2 * d, blocks, (int64_t)3 * d, d, dcol, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -770,6 +785,41 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
     attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);
   });
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+// fold[g][c] = sum of part[r][c] over the rows r = g, g + G, g + 2G, ... (G = gridDim.y), warps taking every
+// eighth of them and adding their sums in ascending order
+__global__ void __launch_bounds__(256) fold_partials_kernel(const float* __restrict__ part, int64_t nrows, int n,
+                                                            float* __restrict__ fold) {
+  __shared__ float sa[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
+  const int64_t G = gridDim.y;
+  float a = 0.f;
+  if (c < n) {
+    for (int64_t r = blockIdx.y + (int64_t)w * G; r < nrows; r += 8 * G) a += part[r * n + c];
+  }
+  sa[w][lane] = a;
+  __syncthreads();
+  if (w == 0 && c < n) {
+    float t = sa[0][lane];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) t += sa[k][lane];
+    fold[(int64_t)blockIdx.y * n + c] = t;
+  }
+}
+
+gram_status colsum_from_partials(gram_ctx* ctx, const float* part, int64_t nrows, int N, float* out, float* scratch,
+                                 cudaStream_t st) {
+  if (nrows == 0 || N == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_COLSUM, (double)nrows * N * 4.0, 2, st, "colsum_partials");
+  int G = 32;                                             // rows of the folded matrix (fixed: the order of additions depends on it)
+  if ((size_t)G * N * sizeof(float) > kRedScratchBytes) G = (int)(kRedScratchBytes / ((size_t)N * sizeof(float)));
+  if (G < 1) return gram_set_error(ctx, "column sums: N too large for the reduction scratch"), GRAM_ERR_UNSUPPORTED;
+  fold_partials_kernel<<<dim3((unsigned)ceil_div(N, 32), (unsigned)G), 256, 0, st>>>(part, nrows, N, scratch);
+  reduce_partials_kernel<<<ceil_div(N, 32), 256, 0, st>>>(scratch, G, (int64_t)N, N, out, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

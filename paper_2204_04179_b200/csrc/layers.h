@@ -28,10 +28,11 @@ gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32
 gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
                               float* mean, float* rstd, int64_t rows, int d, cudaStream_t st);
 // dz = LayerNorm backward of dy at input z (fp32, plus an operand-typed copy dz_b when not null);
-// dgamma += sum_rows dy * xhat; dbeta += sum_rows dy
+// dgamma += sum_rows dy * xhat; dbeta += sum_rows dy; dcol += sum_rows dz when dcol is not null (the bias
+// gradient of the product whose output gradient dz is)
 gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const float* z, const float* mean,
                                const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
-                               float* dbeta, float* scratch, int64_t rows, int d, cudaStream_t st);
+                               float* dbeta, float* dcol, float* scratch, int64_t rows, int d, cudaStream_t st);
 
 // softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d]
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
@@ -47,6 +48,9 @@ gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* d
                                    int n_heads, int causal, cudaStream_t st);
 
 // out[n] += sum_rows X[r, n]   (X operand-typed)
+// out[c] += sum over the nrows rows of part[., c] (fp32 [nrows, N]; partial column sums left by a fused producer)
+gram_status colsum_from_partials(gram_ctx* ctx, const float* part, int64_t nrows, int N, float* out, float* scratch,
+                                 cudaStream_t st);
 gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t rows, int N, float* out, float* scratch,
                               cudaStream_t st);
 // out[s, :] += sum_u X[u*period + s, :]  (s < period; X fp32)

@@ -39,6 +39,7 @@ struct Stack {
   // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
   float *curf = nullptr, *othf = nullptr;
   void *dzb = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;
+  float* cpart = nullptr;                  // [ceil(cap / 32)][max(d_ff, 3 d)] column-sum partials written by fused producers
 };
 
 struct Arena {
@@ -143,6 +144,7 @@ void stack_buffers(Arena& a, Stack& s, size_t esz) {
   s.dqkv = a.take(T * 3 * d * esz);
   s.dctx = a.take(T * d * esz);
   s.du = s.attn_only ? nullptr : a.take(T * f * esz);
+  s.cpart = (float*)a.take(((T + 31) / 32) * (f > 3 * d ? f : 3 * d) * 4);
 }
 
 void layout_buffers(Model* m, Arena& a) {
@@ -325,25 +327,27 @@ gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, 
     if (!s.attn_only) {
       // out = LN2(z2), z2 = h1 + W2 gelu(u) + b2, u = W1 h1 + b1, h1 = LN1(z1), z1 = x + Wo ctx + bo
       GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, s.dzb, mod.g + o.ln2g,
-                                  mod.g + o.ln2b, red, T, d, st));                       // oth, dzb = dz2
-      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.b2, red, st));
+                                  mod.g + o.ln2b, mod.g + o.b2, red, T, d, st));         // oth, dzb = dz2; db2 += its column sums
       GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st, "dw_ffn2"));
       e = GemmEpilogue();
       e.dgelu_pre = a.u;
       e.tag = "dx_ffn2_dgelu";
+      const bool fused_b1 = gemm_fused_colsum(m->dtype, T, f);                           // the product's epilogue also adds up its columns
+      if (fused_b1) e.colsum_part = s.cpart;
       GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(v), the saved u
-      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
+      if (fused_b1) GRAM_TRY(colsum_from_partials(ctx, s.cpart, (T + 31) / 32, f, mod.g + o.b1, red, st));
+      else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
       GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st, "dw_ffn1"));
       e = GemmEpilogue();
       e.res = oth;
       e.tag = "dx_ffn1";
       GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, true, T, f, d, e, st));              // cur = dh1 = du W1 + dz2
       GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, s.dzb, mod.g + o.ln1g,
-                                  mod.g + o.ln1b, red, T, d, st));                       // oth, dzb = dz1
+                                  mod.g + o.ln1b, mod.g + o.bo, red, T, d, st));         // oth, dzb = dz1; dbo += its column sums
     } else {
       float* t = cur; cur = oth; oth = t;                                                // oth = d(out), dzb its copy
+      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
     }
-    GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
     GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st, "dw_attn_out"));
     e = GemmEpilogue();
     e.tag = "dx_attn_out";
@@ -394,7 +398,7 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
   float* dz0 = (dx0 == m->enc.curf) ? m->enc.othf : m->enc.curf;
   GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, nullptr,
-                              m->ce.g + m->o_elng, m->ce.g + m->o_elnb, m->red, T, c.d, st));
+                              m->ce.g + m->o_elng, m->ce.g + m->o_elnb, nullptr, m->red, T, c.d, st));
   GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, st));
   // token-embedding gradient: sum dz0 over the occurrences of each token (same index kernels as stage 1 / 4)
   IndexWorkspace* iws = gram_index_ws(ctx);
