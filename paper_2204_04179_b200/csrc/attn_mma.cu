@@ -131,15 +131,46 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   }
 }
 
-// rows [0, S) of one head's slice of a [tokens, ld] bf16 matrix -> shared memory, row-major; rows S..SP-1 are zero
+// rows [0, S) of one head's slice of a [tokens, ld] bf16 matrix -> shared memory, row-major; rows S..SP-1 are zero.
+// The copies are asynchronous (16 bytes each, no registers in between): loads_done() before the tile is read.
 template <int SP, int DH>
 __device__ __forceinline__ void load_head(const bf16* __restrict__ src, int64_t ld, int S, bf16* __restrict__ dst) {
   constexpr int LD = DH + 8;
   for (int i = threadIdx.x; i < SP * (DH / 8); i += blockDim.x) {
     const int s = i / (DH / 8), c = (i - s * (DH / 8)) * 8;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (s < S) v = *reinterpret_cast<const uint4*>(src + (int64_t)s * ld + c);
-    *reinterpret_cast<uint4*>(dst + s * LD + c) = v;
+    if (s < S) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst + s * LD + c)), "l"(src + (int64_t)s * ld + c)
+                   : "memory");
+    } else {
+      *reinterpret_cast<uint4*>(dst + s * LD + c) = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+__device__ __forceinline__ void loads_done() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+}
+// rows [row_begin, row_end) (below S) of a shared-memory tile -> one head's slice of a [tokens, ld] matrix, 16 bytes
+// per thread, whole 128-byte (64-byte for DH = 32) row pieces per eight (four) threads
+template <int DH>
+__device__ __forceinline__ void store_rows(const bf16* __restrict__ src, int row_begin, int row_end, int S, bf16* __restrict__ dst,
+                                           int64_t ld, int tid, int nthreads) {
+  constexpr int LD = DH + 8;
+  if (row_end > S) row_end = S;
+  for (int i = tid; i < (row_end - row_begin) * (DH / 8); i += nthreads) {
+    const int s = row_begin + i / (DH / 8), c = (i % (DH / 8)) * 8;
+    *reinterpret_cast<uint4*>(dst + (int64_t)s * ld + c) = *reinterpret_cast<const uint4*>(src + s * LD + c);
+  }
+}
+// the C-layout registers of a 16 x DH tile (rows r0 + g and r0 + g + 8) -> bf16 in a shared-memory tile
+template <int DH>
+__device__ __forceinline__ void stage_tile(const float (&o)[DH / 8][4], bf16* __restrict__ dst, int r0, int g, int q) {
+  constexpr int LD = DH + 8;
+#pragma unroll
+  for (int nt = 0; nt < DH / 8; ++nt) {
+    const int c = nt * 8 + 2 * q;
+    *reinterpret_cast<uint32_t*>(dst + (r0 + g) * LD + c) = pack2(o[nt][0], o[nt][1]);
+    *reinterpret_cast<uint32_t*>(dst + (r0 + g + 8) * LD + c) = pack2(o[nt][2], o[nt][3]);
   }
 }
 
@@ -176,8 +207,9 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs);
   load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
   load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
-  __syncthreads();
+  loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  bf16* ob = out + seq * S * (int64_t)d + h * DH;
   for (int r0 = warp * 16; r0 < S; r0 += 64) {
     float p[SP / 8][4];
     score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
@@ -185,20 +217,18 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     mma_regs_times_rows<SP, DH>(p, Vs, lane, o);              // O = P V
-    bf16* ob = out + seq * S * (int64_t)d + h * DH;
-#pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) {
-      const int c = nt * 8 + 2 * q;
-      if (r0 + g < S) *reinterpret_cast<uint32_t*>(ob + (int64_t)(r0 + g) * d + c) = pack2(o[nt][0], o[nt][1]);
-      if (r0 + g + 8 < S) *reinterpret_cast<uint32_t*>(ob + (int64_t)(r0 + g + 8) * d + c) = pack2(o[nt][2], o[nt][3]);
-    }
+    // the 16 rows of Q are this warp's alone and no longer needed: O goes through them so that it leaves in whole rows
+    __syncwarp();
+    stage_tile<DH>(o, Qs, r0, g, q);
+    __syncwarp();
+    store_rows<DH>(Qs, r0, r0 + 16, S, ob, d, lane, 32);
   }
 }
 
 template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
-                                                           bf16* __restrict__ dqkv, int S, int d, int n_heads, int causal,
-                                                           float scale) {
+                                                           bf16* __restrict__ dqkv, float* __restrict__ colpart, int S, int d,
+                                                           int n_heads, int causal, float scale) {
   constexpr int LD = DH + 8, LP = SP + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // [SP][DH+8]
@@ -214,59 +244,65 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
   load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
   load_head<SP, DH>(dctx + seq * S * (int64_t)d + h * DH, d, S, dOs);
-  __syncthreads();
+  loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   bf16* dq = dqkv + seq * S * 3 * (int64_t)d + h * DH;
-  // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ ----
-  for (int r0 = warp * 16; r0 < SP; r0 += 64) {
-    float p[SP / 8][4];
-    score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
-    float dp[SP / 8][4];
+  // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ (kept in registers as bf16 pairs) ----
+  constexpr int NIT = (SP + 63) / 64;
+  uint32_t dqp[NIT][DH / 8][2];
 #pragma unroll
-    for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
+  for (int it = 0; it < NIT; ++it) {
+    const int r0 = warp * 16 + it * 64;
+    if (r0 < SP) {
+      float p[SP / 8][4];
+      score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
+      float dp[SP / 8][4];
 #pragma unroll
-    for (int kt = 0; kt < DH / 16; ++kt) {        // dP = dO V^T
-      uint32_t a0, a1, a2, a3;
-      load_a_rows(dOs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
+      for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
 #pragma unroll
-      for (int nt = 0; nt < SP / 8; nt += 2) {
-        uint32_t b0, b1, b2, b3;
-        load_b_rows(Vs, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
-        mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
-        mma16816(dp[nt + 1], a0, a1, a2, a3, b2, b3);
+      for (int kt = 0; kt < DH / 16; ++kt) {        // dP = dO V^T
+        uint32_t a0, a1, a2, a3;
+        load_a_rows(dOs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
+#pragma unroll
+        for (int nt = 0; nt < SP / 8; nt += 2) {
+          uint32_t b0, b1, b2, b3;
+          load_b_rows(Vs, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
+          mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
+          mma16816(dp[nt + 1], a0, a1, a2, a3, b2, b3);
+        }
       }
-    }
-    float d0 = 0.f, d1 = 0.f;
+      float d0 = 0.f, d1 = 0.f;
 #pragma unroll
-    for (int nt = 0; nt < SP / 8; ++nt) {
-      d0 += p[nt][0] * dp[nt][0] + p[nt][1] * dp[nt][1];
-      d1 += p[nt][2] * dp[nt][2] + p[nt][3] * dp[nt][3];
-    }
-    d0 = quad_sum(d0);
-    d1 = quad_sum(d1);
+      for (int nt = 0; nt < SP / 8; ++nt) {
+        d0 += p[nt][0] * dp[nt][0] + p[nt][1] * dp[nt][1];
+        d1 += p[nt][2] * dp[nt][2] + p[nt][3] * dp[nt][3];
+      }
+      d0 = quad_sum(d0);
+      d1 = quad_sum(d1);
 #pragma unroll
-    for (int nt = 0; nt < SP / 8; ++nt) {         // dS = P (dP - delta) / sqrt(dh)
-      dp[nt][0] = p[nt][0] * (dp[nt][0] - d0) * scale; dp[nt][1] = p[nt][1] * (dp[nt][1] - d0) * scale;
-      dp[nt][2] = p[nt][2] * (dp[nt][2] - d1) * scale; dp[nt][3] = p[nt][3] * (dp[nt][3] - d1) * scale;
-      const int j = nt * 8 + 2 * q;
-      *reinterpret_cast<uint32_t*>(Ps + (r0 + g) * LP + j) = pack2(p[nt][0], p[nt][1]);
-      *reinterpret_cast<uint32_t*>(Ps + (r0 + g + 8) * LP + j) = pack2(p[nt][2], p[nt][3]);
-      *reinterpret_cast<uint32_t*>(dSs + (r0 + g) * LP + j) = pack2(dp[nt][0], dp[nt][1]);
-      *reinterpret_cast<uint32_t*>(dSs + (r0 + g + 8) * LP + j) = pack2(dp[nt][2], dp[nt][3]);
-    }
-    float o[DH / 8][4];
+      for (int nt = 0; nt < SP / 8; ++nt) {         // dS = P (dP - delta) / sqrt(dh)
+        dp[nt][0] = p[nt][0] * (dp[nt][0] - d0) * scale; dp[nt][1] = p[nt][1] * (dp[nt][1] - d0) * scale;
+        dp[nt][2] = p[nt][2] * (dp[nt][2] - d1) * scale; dp[nt][3] = p[nt][3] * (dp[nt][3] - d1) * scale;
+        const int j = nt * 8 + 2 * q;
+        *reinterpret_cast<uint32_t*>(Ps + (r0 + g) * LP + j) = pack2(p[nt][0], p[nt][1]);
+        *reinterpret_cast<uint32_t*>(Ps + (r0 + g + 8) * LP + j) = pack2(p[nt][2], p[nt][3]);
+        *reinterpret_cast<uint32_t*>(dSs + (r0 + g) * LP + j) = pack2(dp[nt][0], dp[nt][1]);
+        *reinterpret_cast<uint32_t*>(dSs + (r0 + g + 8) * LP + j) = pack2(dp[nt][2], dp[nt][3]);
+      }
+      float o[DH / 8][4];
 #pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-    mma_regs_times_rows<SP, DH>(dp, Ks, lane, o);             // dQ = dS K
+      for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+      mma_regs_times_rows<SP, DH>(dp, Ks, lane, o);             // dQ = dS K
 #pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) {
-      const int c = nt * 8 + 2 * q;
-      if (r0 + g < S) *reinterpret_cast<uint32_t*>(dq + (int64_t)(r0 + g) * 3 * d + c) = pack2(o[nt][0], o[nt][1]);
-      if (r0 + g + 8 < S) *reinterpret_cast<uint32_t*>(dq + (int64_t)(r0 + g + 8) * 3 * d + c) = pack2(o[nt][2], o[nt][3]);
+      for (int nt = 0; nt < DH / 8; ++nt) {
+        dqp[it][nt][0] = pack2(o[nt][0], o[nt][1]);
+        dqp[it][nt][1] = pack2(o[nt][2], o[nt][3]);
+      }
     }
   }
   __syncthreads();
-  // ---- second half: 16 key rows per warp: dK = dS^T Q, dV = P^T dO ----
+  // ---- second half: 16 key rows per warp: dK = dS^T Q, dV = P^T dO; K and V are no longer read, so the results
+  // ---- replace this warp's rows of them
   for (int j0 = warp * 16; j0 < S; j0 += 64) {
     float dk[DH / 8][4], dv[DH / 8][4];
 #pragma unroll
@@ -290,17 +326,35 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
         mma16816(dv[nt + 1], p0, p1, p2, p3, b2, b3);
       }
     }
+    stage_tile<DH>(dk, Ks, j0, g, q);
+    stage_tile<DH>(dv, Vs, j0, g, q);
+  }
+  __syncthreads();                                 // Q is no longer read either: dQ replaces it
 #pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) {
-      const int c = nt * 8 + 2 * q;
-      if (j0 + g < S) {
-        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g) * 3 * d + d + c) = pack2(dk[nt][0], dk[nt][1]);
-        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g) * 3 * d + 2 * d + c) = pack2(dv[nt][0], dv[nt][1]);
+  for (int it = 0; it < NIT; ++it) {
+    const int r0 = warp * 16 + it * 64;
+    if (r0 < SP) {
+#pragma unroll
+      for (int nt = 0; nt < DH / 8; ++nt) {
+        const int c = nt * 8 + 2 * q;
+        *reinterpret_cast<uint32_t*>(Qs + (r0 + g) * LD + c) = dqp[it][nt][0];
+        *reinterpret_cast<uint32_t*>(Qs + (r0 + g + 8) * LD + c) = dqp[it][nt][1];
       }
-      if (j0 + g + 8 < S) {
-        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g + 8) * 3 * d + d + c) = pack2(dk[nt][2], dk[nt][3]);
-        *reinterpret_cast<uint32_t*>(dq + (int64_t)(j0 + g + 8) * 3 * d + 2 * d + c) = pack2(dv[nt][2], dv[nt][3]);
-      }
+    }
+  }
+  __syncthreads();
+  store_rows<DH>(Qs, 0, S, S, dq, 3 * (int64_t)d, threadIdx.x, blockDim.x);
+  store_rows<DH>(Ks, 0, S, S, dq + d, 3 * (int64_t)d, threadIdx.x, blockDim.x);
+  store_rows<DH>(Vs, 0, S, S, dq + 2 * d, 3 * (int64_t)d, threadIdx.x, blockDim.x);
+  if (colpart) {
+    // column sums of the three gradient tiles as stored (bf16), rows in ascending order: row `seq` of the partial
+    // sums of the bias gradient of the Q, K, V projection
+    for (int c = threadIdx.x; c < 3 * DH; c += blockDim.x) {
+      const int which = c / DH, col = c - which * DH;
+      const bf16* M = Qs + which * (SP * LD) + col;
+      float a = 0.f;
+      for (int r = 0; r < S; ++r) a += __bfloat162float(M[r * LD]);
+      colpart[seq * 3 * (int64_t)d + which * d + h * DH + col] = a;
     }
   }
 }
@@ -316,13 +370,13 @@ gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq,
   return GRAM_OK;
 }
 template <int SP, int DH>
-gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, int64_t n_seq, int S, int d, int n_heads,
-                       int causal, cudaStream_t st) {
+gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, float* colpart, int64_t n_seq, int S, int d,
+                       int n_heads, int causal, cudaStream_t st) {
   constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
   auto kern = attn_bwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -354,7 +408,7 @@ gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int
                                   int causal, cudaStream_t st) {
   ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, st);
 }
-gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq, int S, int d,
-                                   int n_heads, int causal, cudaStream_t st) {
-  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, n_seq, S, d, n_heads, causal, st);
+gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq,
+                                   int S, int d, int n_heads, int causal, cudaStream_t st) {
+  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, st);
 }

@@ -771,8 +771,8 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   return GRAM_OK;
 }
 
-gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq,
-                               int S, int d, int n_heads, int causal, cudaStream_t st) {
+gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
+                               int64_t n_seq, int S, int d, int n_heads, int causal, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
@@ -780,7 +780,8 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_backward_mma(ctx, qkv, dctx, dqkv, n_seq, S, d, n_heads, causal, st);
+    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, st);
+  if (colpart) return gram_set_error(ctx, "attention: fused column sums need the tensor-core kernel"), GRAM_ERR_UNSUPPORTED;
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
     attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);

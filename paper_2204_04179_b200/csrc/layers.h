@@ -37,14 +37,16 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 // softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d]
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
                               int n_heads, int causal, cudaStream_t st);
-gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq,
-                               int S, int d, int n_heads, int causal, cudaStream_t st);
+// colpart (may be null; only where attention_mma_supported and dtype is bf16): fp32 [n_seq, 3d], row s receives the
+// column sums of sequence s's rows of dqkv, the partial sums of the bias gradient of the Q, K, V projection
+gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
+                               int64_t n_seq, int S, int d, int n_heads, int causal, cudaStream_t st);
 
 // the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
 bool attention_mma_supported(int S, int d, int n_heads);
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
                                   int causal, cudaStream_t st);
-gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, int64_t n_seq, int S, int d,
+gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq, int S, int d,
                                    int n_heads, int causal, cudaStream_t st);
 
 // out[n] += sum_rows X[r, n]   (X operand-typed)

@@ -39,7 +39,8 @@ struct Stack {
   // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
   float *curf = nullptr, *othf = nullptr;
   void *dzb = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;
-  float* cpart = nullptr;                  // [ceil(cap / 32)][max(d_ff, 3 d)] column-sum partials written by fused producers
+  float* cpart = nullptr;                  // column-sum partials written by fused producers
+  size_t cpart_elems = 0;
 };
 
 struct Arena {
@@ -144,7 +145,8 @@ void stack_buffers(Arena& a, Stack& s, size_t esz) {
   s.dqkv = a.take(T * 3 * d * esz);
   s.dctx = a.take(T * d * esz);
   s.du = s.attn_only ? nullptr : a.take(T * f * esz);
-  s.cpart = (float*)a.take(((T + 31) / 32) * (f > 3 * d ? f : 3 * d) * 4);
+  s.cpart_elems = ((T + 31) / 32) * (f > 3 * d ? f : 3 * d);     // [ceil(T / 32)][d_ff] or [sequences][3 d]
+  s.cpart = (float*)a.take(s.cpart_elems * 4);
 }
 
 void layout_buffers(Model* m, Arena& a) {
@@ -352,8 +354,12 @@ gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, 
     e = GemmEpilogue();
     e.tag = "dx_attn_out";
     GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.wo), s.dctx, false, T, d, d, e, st));
-    GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, n_seq, S, d, s.heads, s.causal, st));
-    GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
+    const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
+                            (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
+    GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
+                                s.causal, st));
+    if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, red, st));
+    else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
     GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
     e = GemmEpilogue();
     e.res = oth;
