@@ -278,7 +278,7 @@ gram_status index_ws_alloc(gram_ctx* ctx, IndexWorkspace* ws, int64_t P_max, int
                  (size_t)ceil_div64(P_max > 0 ? P_max : 1, SCAN_THREADS * 4) + 8;
   GRAM_CUDA(ctx, cudaMalloc(&ws->block_sums, nsums * sizeof(int32_t)));
   GRAM_CUDA(ctx, cudaMalloc(&ws->rank_table, (size_t)(n_items_max > 0 ? n_items_max : 1) * sizeof(int32_t)));
-  GRAM_CUDA(ctx, cudaMalloc(&ws->partial, (size_t)kAccMaxChunks * 2 * (d_max > 0 ? d_max : 1) * sizeof(float)));
+  GRAM_CUDA(ctx, cudaMalloc(&ws->partial, ((size_t)kAccMaxChunks * 2 * (d_max > 0 ? d_max : 1) + 2 * kAccMaxChunks) * sizeof(float)));
   return GRAM_OK;
 }
 

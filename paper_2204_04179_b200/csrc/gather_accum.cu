@@ -123,7 +123,8 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
                                                             int d, int64_t R, int nchunks, int nslabs,
                                                             const int32_t* __restrict__ rows, int add,
                                                             float* __restrict__ out, float* __restrict__ partial,
-                                                            int32_t* status, const int32_t* __restrict__ d_U) {
+                                                            int2* __restrict__ span, int32_t* status,
+                                                            const int32_t* __restrict__ d_U) {
   if (d_U) U = *d_U;            // the number of items may live on the device
   if (U <= 0) return;
   const int lane = threadIdx.x & 31;
@@ -181,12 +182,15 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
     }
   }
   // the item still open at the end of the chunk
+  int2 sp = make_int2(-1, 0);
   if (seg_end <= c1) {             // it ends exactly at the chunk end
     if (seg_begin >= c0) store_row<VPL>(out, rows ? rows[u] : u, d, col0, lane, acc, add != 0);
     else store_row<VPL>(partial, (int64_t)chunk * 2 + 0, d, col0, lane, acc, false);
   } else {                         // it continues to the right
     store_row<VPL>(partial, (int64_t)chunk * 2 + (seg_begin >= c0 ? 1 : 0), d, col0, lane, acc, false);
+    if (seg_begin >= c0) sp = make_int2(u, (int)((seg_end - 1) / R));      // it starts here: the fix-up adds its parts
   }
+  if (slab == 0 && lane == 0) span[chunk] = sp;   // (item, last chunk it reaches), or -1: nothing to fix up from here
 }
 
 // one block per (chunk, slab): if an item starts in this chunk and runs past its end, add its parts.  Warp w adds
@@ -197,7 +201,7 @@ __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __rest
                                                            int d, int64_t R, int nchunks, int nslabs,
                                                            const int32_t* __restrict__ rows, int add,
                                                            float* __restrict__ out, const float* __restrict__ partial,
-                                                           const int32_t* __restrict__ d_U) {
+                                                           const int2* __restrict__ span, const int32_t* __restrict__ d_U) {
   __shared__ float4 red[8][VPL][32];
   if (d_U) U = *d_U;
   if (U <= 0) return;
@@ -206,10 +210,10 @@ __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __rest
   const int col0 = slab * (VPL * 128);
   const int64_t c0 = (int64_t)chunk * R, c1 = min(c0 + R, P);
   if (c0 >= c1 || c1 >= P) return;
-  const int32_t u = find_segment(seg_off, U, c1 - 1, lane);
-  const int64_t seg_begin = seg_off[u], seg_end = seg_off[u + 1];
-  if (seg_begin < c0 || seg_end <= c1) return;      // not the first chunk of a spanning item (same for the whole block)
-  const int last = (int)((seg_end - 1) / R);
+  const int2 sp = span[chunk];                       // left by the first launch
+  if (sp.x < 0) return;                              // no item starts here and runs on (same for the whole block)
+  const int32_t u = sp.x;
+  const int last = min(sp.y, nchunks - 1);
   float4 acc[VPL];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) {
@@ -350,15 +354,15 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
 
 template <typename InT, int VPL>
 static void segsum_run(const void* d_in, const int32_t* d_perm, const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d,
-                       int64_t R, int nchunks, const int32_t* d_rows, int add, float* d_out, float* partial,
+                       int64_t R, int nchunks, const int32_t* d_rows, int add, float* d_out, float* partial, int2* span,
                        int32_t* status, const int32_t* d_U, cudaStream_t st) {
   const int nslabs = ceil_div(d, VPL * 128);
   const int64_t warps = (int64_t)nchunks * nslabs;
   const int blocks = (int)ceil_div64(warps, 8);
   segsum_chunks_kernel<InT, VPL, 8><<<blocks, 256, 0, st>>>((const InT*)d_in, d_perm, d_seg_off, P, U, d, R, nchunks, nslabs,
-                                                            d_rows, add, d_out, partial, status, d_U);
+                                                            d_rows, add, d_out, partial, span, status, d_U);
   if (nchunks > 1)
-    segsum_fixup_kernel<VPL><<<(unsigned)warps, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, d_U);
+    segsum_fixup_kernel<VPL><<<(unsigned)warps, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, span, d_U);
 }
 
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
@@ -375,14 +379,15 @@ gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_i
   if (nchunks > kAccMaxChunks) nchunks = kAccMaxChunks;
   const int64_t R = ceil_div64(P, nchunks);
   nchunks = ceil_div64(P, R);
+  int2* span = reinterpret_cast<int2*>(ws->partial + (size_t)kAccMaxChunks * 2 * (ws->d_max > 0 ? ws->d_max : 1));   // after the partial sums
   ProfScope prof(ctx, GRAM_K_ACCUMULATE, (in_bf16 ? 2.0 : 4.0) * (double)P * d + 4.0 * (double)U * d + 4.0 * P + 4.0 * (U + 1),
                  nchunks > 1 ? 2 : 1, st);
   if (d >= 256) {
-    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
-    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
+    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
+    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
   } else {
-    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
-    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, gram_status_word(ctx), d_U, st);
+    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
+    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
   }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -414,8 +419,9 @@ namespace {
 constexpr int kStaticChunks = 592;            // work units (4 per SM)
 constexpr int kStaticMaxD = 1024;             // widest row the fixed scratch can serve
 constexpr size_t kStaticPartialFloats = (size_t)kStaticChunks * 2 * kStaticMaxD;
-// [0, kStaticPartialFloats): partial sums; then 64 floats whose first word is the device status word
-static __device__ __align__(256) float g_static_scratch[kStaticPartialFloats + 64];
+// [0, kStaticPartialFloats): partial sums; then 64 floats whose first word is the device status word; then one
+// (item, last chunk) pair per work unit
+static __device__ __align__(256) float g_static_scratch[kStaticPartialFloats + 64 + 2 * kStaticChunks];
 
 constexpr int kMaxDevices = 64;
 float* g_static_ptr[kMaxDevices] = {};        // device address of the array, looked up once per device
@@ -455,16 +461,17 @@ extern "C" gram_status gram_accumulate_static(const float* d_dE, const int32_t* 
   }
   float* partial = g_static_ptr[dev];
   int32_t* status = reinterpret_cast<int32_t*>(partial + kStaticPartialFloats);
-  // the status word must start at zero; the partial sums need no clearing (each slot that is read in a
-  // call has been written earlier in the same call)
+  int2* span = reinterpret_cast<int2*>(partial + kStaticPartialFloats + 64);
+  // the status word must start at zero; the partial sums and the (item, last chunk) pairs need no clearing
+  // (each slot that is read in a call has been written earlier in the same call)
   if (cudaMemsetAsync(status, 0, sizeof(int32_t), st) != cudaSuccess)
     return static_fail(h_err, err_len, "gram_accumulate_static: clearing the status word failed"), GRAM_ERR_CUDA;
   int64_t nchunks = ceil_div64(P, 16);
   if (nchunks > kStaticChunks) nchunks = kStaticChunks;
   const int64_t R = ceil_div64(P, nchunks);
   nchunks = ceil_div64(P, R);
-  if (d >= 256) segsum_run<float, 2>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, status, nullptr, st);
-  else segsum_run<float, 1>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, status, nullptr, st);
+  if (d >= 256) segsum_run<float, 2>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, span, status, nullptr, st);
+  else segsum_run<float, 1>(d_dE, d_perm, d_seg_off, P, U, d, R, (int)nchunks, nullptr, 0, d_G, partial, span, status, nullptr, st);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     if (h_err && err_len) snprintf(h_err, err_len, "gram_accumulate_static: launch failed: %s", cudaGetErrorString(e));

@@ -50,7 +50,7 @@ struct IndexWorkspace {
   int32_t* hist = nullptr;        // [256 * n_sort_blocks] digit-major block histograms
   int32_t* block_sums = nullptr;  // scan scratch
   int32_t* rank_table = nullptr;  // [n_items_max] item ID -> index in unique
-  float* partial = nullptr;       // [kAccMaxChunks * 2 * d_max] chunk-boundary partial sums
+  float* partial = nullptr;       // [kAccMaxChunks * 2 * d_max] chunk-boundary partial sums, then kAccMaxChunks (item, last chunk) pairs
   int32_t n_sort_blocks = 0;
 };
 
