@@ -24,6 +24,10 @@ What it states, and from where in the paper:
 * `unique_inverse_bruteforce`, `unique_inverse`, `segment_sum`,
   `table_accumulate`: the index work and the per-item sums on their own.
 * `boost_ratio`: the speed-boost ratio R (Section 4.4).
+* `noam_rate`, `adam_update`, `train_steps_adam`: the optimiser of Section A
+  (implementation details): Adam with the Noam learning-rate scheme, written
+  from the two published definitions; `train_steps_adam` applies it to the
+  end-to-end gradients of successive batches.
 
 Arithmetic is float64 throughout unless a caller passes another dtype: the
 paper never fixes a precision.  Derivatives of the end-to-end definition come
@@ -34,8 +38,10 @@ Pins (tests/test_oracle_*.py): brute force on tiny inputs, the worked count
 of Fig. 1, finite differences on a 1-layer encoder, closed forms of softmax /
 LayerNorm / GELU / BCE, the Proposition (e2e == single-step), the pseudo-loss
 identity (Eqs. 1-3), K = 1 reducing to single-step, and conservation of
-column sums.  The Multi-step *trajectory* beyond those is pinned only by the
-readings below: parity unpinned by the paper for that part.
+column sums; for the optimiser, torch.optim.Adam at a constant rate, the closed
+form of the first step, and the closed-form values of the Noam curve.  The
+Multi-step *trajectory* beyond those is pinned only by the readings below:
+parity unpinned by the paper for that part.
 """
 from __future__ import annotations
 
@@ -382,3 +388,50 @@ def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache,
     cache[items] = round_to_bf16(newc) if cache_bf16 else newc
     return dict(losses=losses, grad_ce=_grads(th_ce), grad_task_last=grad_task_last, task_params=cur_task,
                 table=table, touched=touched, cache=cache, items=items.astype(np.int32))
+
+
+# ---------------------------------------------------------------------------
+# Optimiser (Section A, implementation details: "Adam with Noam scheduler", learning rate 1e-4)
+# ---------------------------------------------------------------------------
+def noam_rate(t: int, peak: float, warmup: int) -> float:
+    """Learning rate at update t = 1, 2, ... under the Noam scheme (Vaswani et al. 2017, Eq. 3):
+    rate proportional to min(t^-0.5, t * warmup^-1.5).  The paper gives one learning rate (1e-4) and no warm-up
+    length; the reading taken here scales the curve so that its maximum, reached at t = warmup, is `peak`:
+    rate = peak * min(t / warmup, sqrt(warmup / t)).  warmup <= 0 means a constant rate."""
+    if warmup <= 0:
+        return float(peak)
+    t = float(t)
+    return float(peak) * min(t / warmup, math.sqrt(warmup / t))
+
+
+def adam_update(w: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, t: int, rate: float,
+                beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8) -> None:
+    """One Adam update in place (Kingma & Ba 2015, Algorithm 1), float64 arithmetic on whatever arrays are
+    passed: first and second moment estimates, their bias corrections at update t (t >= 1), and the step."""
+    g = g.astype(np.float64)
+    m[...] = beta1 * m + (1.0 - beta1) * g
+    v[...] = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** t)
+    v_hat = v / (1.0 - beta2 ** t)
+    w[...] = w - rate * m_hat / (np.sqrt(v_hat) + eps)
+
+
+def train_steps_adam(shape, ce_params, task_params, item_tokens, batches, peak_ce: float, peak_task: float,
+                     warmup: int, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8):
+    """Successive end-to-end training steps (Section 3.3) with the Adam + Noam update applied to both modules
+    after every batch (Single-step GRAM has the same gradients, hence the same trajectory).  batches: list of
+    (ids, labels).  Returns (ce_params, task_params, losses) with float64 parameter copies."""
+    ce = OrderedDict((k, np.array(a, dtype=np.float64)) for k, a in ce_params.items())
+    tk = OrderedDict((k, np.array(a, dtype=np.float64)) for k, a in task_params.items())
+    state = {id(d): (OrderedDict((k, np.zeros_like(a)) for k, a in d.items()),
+                     OrderedDict((k, np.zeros_like(a)) for k, a in d.items())) for d in (ce, tk)}
+    losses = []
+    for t, (ids, labels) in enumerate(batches, start=1):
+        r = e2e_step(shape, ce, tk, item_tokens, ids, labels)
+        losses.append(r["loss"])
+        for params, grads, peak in ((ce, r["grad_ce"], peak_ce), (tk, r["grad_task"], peak_task)):
+            m, v = state[id(params)]
+            rate = noam_rate(t, peak, warmup)
+            for k in params:
+                adam_update(params[k], grads[k], m[k], v[k], t, rate, beta1, beta2, eps)
+    return ce, tk, losses
