@@ -175,6 +175,20 @@ def kernel_sweep_cell(binding, synth, torch, dev, peaks):
         ms = timeit(fn)
         out[name] = {"ms": ms, "GB/s": nbytes / ms / 1e6, "frac_of_" + peaks["source"] + "_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
     out["cell"] = {"P": P, "n_items": N, "zipf_s": s, "d": d, "U": U}
+    del H, E, dE, G
+    # the optimiser's update on a parameter vector the size of the BERT-base-shaped encoder (with its bf16 copy)
+    n = 108_891_648
+    w = torch.randn(n, device=dev) * 0.02; gr = torch.randn(n, device=dev) * 1e-3
+    m = torch.zeros(n, device=dev); v = torch.zeros(n, device=dev); wb = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    step = [0]
+
+    def adam():
+        step[0] += 1
+        g.adam_update(w, gr, m, v, step[0], 1e-4, w_bf16=wb)
+    ms = timeit(adam)
+    nbytes = 30 * n
+    out["adam_update"] = {"ms": ms, "GB/s": nbytes / ms / 1e6, "frac_of_" + peaks["source"] + "_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"],
+                          "params": n}
     g.close()
     return out
 

@@ -48,6 +48,7 @@ enum { GRAM_F32 = 0, GRAM_BF16 = 1 };                 /* element types */
 enum { GRAM_POOL_MEAN = 0, GRAM_POOL_CLS = 1 };       /* item pooling */
 enum { GRAM_TASK_NONE = 0, GRAM_TASK_KT = 1, GRAM_TASK_NR = 2 };
 enum { GRAM_MODULE_CE = 0, GRAM_MODULE_TASK = 1 };
+enum { GRAM_OPT_SGD = 0, GRAM_OPT_ADAM = 1 };
 
 /* Shapes of the two modules and of the batches a context serves.
  * CE (Section 3.2; Appendix D: attention layers of width 768): token + position
@@ -75,6 +76,10 @@ typedef struct gram_config {
   int32_t ce_micro_batch;      /* items per encoder pass, bounds activation memory (Section 6.3); 0 = all at once */
   float lr_task;               /* SGD step applied to the task parameters after every gram_step (0 = none) */
   float lr_ce;                 /* SGD step applied to the encoder parameters after an encoder pass (0 = none) */
+  int32_t optimizer;           /* GRAM_OPT_SGD: plain steps of lr_task / lr_ce.  GRAM_OPT_ADAM: Adam with the Noam
+                                  learning-rate scheme (Section A); lr_task / lr_ce are then the peak rates */
+  int32_t noam_warmup;         /* updates until the peak rate; <= 0: constant rate */
+  float adam_beta1, adam_beta2, adam_eps;   /* <= 0: 0.9, 0.999, 1e-8 */
 } gram_config;
 
 typedef struct gram_step_report {
@@ -113,6 +118,12 @@ gram_status gram_get_params(gram_ctx* ctx, int module, float* h_params, size_t n
 /* Gradients of the last gram_step / gram_encoder_backward / gram_task, same layout (synchronises). */
 gram_status gram_get_grads(gram_ctx* ctx, int module, float* h_grads, size_t n);
 gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream);
+/* The configured update of one module from its current gradients (what gram_step applies by itself): an SGD step,
+ * or one Adam update at the module's next update count with the Noam rate of that count.  For callers that drive
+ * the stages one by one. */
+gram_status gram_optimizer_step(gram_ctx* ctx, int module, gram_stream stream);
+/* Clears the Adam moment estimates and update counts of both modules (a context starts cleared). */
+gram_status gram_optimizer_reset(gram_ctx* ctx, gram_stream stream);
 /* Token IDs c_i of every item (Table 1), int32 [n_items, l_t], copied to the device. */
 gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens);
 
@@ -208,7 +219,7 @@ gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, 
  * Kernel kinds for gram_profile_read. */
 enum { GRAM_K_GEMM = 0, GRAM_K_ATTENTION = 1, GRAM_K_LAYERNORM = 2, GRAM_K_COLSUM = 3, GRAM_K_EMBED_POOL = 4,
        GRAM_K_DEDUP = 5, GRAM_K_GATHER = 6, GRAM_K_ACCUMULATE = 7, GRAM_K_TASK_HEAD = 8, GRAM_K_OTHER = 9,
-       GRAM_K_COUNT = 10 };
+       GRAM_K_OPTIMIZER = 10, GRAM_K_COUNT = 11 };
 /* enable != 0: from now on every kernel group the library launches is bracketed by
  * CUDA events on its stream (a few microseconds of host time per group); 0 turns
  * it off.  Either way the totals are cleared. */
@@ -258,6 +269,20 @@ gram_status gram_accumulate_static(const float* d_dE, const int32_t* d_perm, con
 gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
                            int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
                            gram_stream stream);
+
+/* --- the optimiser's two pieces, exported so that they can be tested on their own (Section A: "Adam with Noam
+ * scheduler") -------------------------------------------------------------
+ * gram_noam_rate (host only): *h_rate = peak * min(t / warmup, sqrt(warmup / t)) for update t >= 1, the Noam curve
+ * scaled so that its maximum, at t = warmup, is `peak`; warmup <= 0 gives the constant `peak`.
+ * gram_adam_update: one Adam update of n fp32 parameters in place at update count t >= 1:
+ *   m = beta1 m + (1 - beta1) g;  v = beta2 v + (1 - beta2) g^2;
+ *   w -= rate * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+ * d_w, d_g, d_m, d_v: device fp32 [n], 16-byte aligned; d_w_bf16 (may be NULL): device bf16 [n] that receives the
+ * rounded new parameters (the copy the tensor cores read).  The two bias corrections are formed on the host in
+ * double precision. */
+gram_status gram_noam_rate(int64_t t, float peak, int32_t warmup, float* h_rate);
+gram_status gram_adam_update(gram_ctx* ctx, float* d_w, const float* d_g, float* d_m, float* d_v, size_t n, int64_t t,
+                             float rate, float beta1, float beta2, float eps, void* d_w_bf16, gram_stream stream);
 
 #ifdef __cplusplus
 }

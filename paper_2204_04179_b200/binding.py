@@ -20,6 +20,7 @@ GRAM_F32, GRAM_BF16 = 0, 1
 GRAM_POOL_MEAN, GRAM_POOL_CLS = 0, 1
 GRAM_TASK_NONE, GRAM_TASK_KT, GRAM_TASK_NR = 0, 1, 2
 GRAM_MODULE_CE, GRAM_MODULE_TASK = 0, 1
+GRAM_OPT_SGD, GRAM_OPT_ADAM = 0, 1
 STATUS = {0: "GRAM_OK", 1: "GRAM_ERR_ARG", 2: "GRAM_ERR_ID_RANGE", 3: "GRAM_ERR_WORKSPACE", 4: "GRAM_ERR_UNSUPPORTED",
           5: "GRAM_ERR_CUDA", 6: "GRAM_ERR_TIMEOUT"}
 
@@ -29,9 +30,11 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_encode_unique", "gram_gather", "gram_accumulate", "gram_accumulate_multistep", "gram_touched_list",
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
-           "gram_launch_count", "gram_profile_dump", "gram_accumulate_static"]
+           "gram_launch_count", "gram_profile_dump", "gram_accumulate_static", "gram_optimizer_step",
+           "gram_optimizer_reset", "gram_noam_rate", "gram_adam_update"]
 
-KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other"]
+KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other",
+         "optimizer"]
 
 
 class GramConfig(C.Structure):
@@ -39,7 +42,8 @@ class GramConfig(C.Structure):
                                           "pooling", "task", "task_layers", "task_heads", "task_d_ff",
                                           "task_attn_only", "d_a", "n_cand", "B_max", "L")] + \
                [("P_max", C.c_int64), ("d_max", C.c_int32), ("K", C.c_int32), ("ce_micro_batch", C.c_int32),
-                ("lr_task", C.c_float), ("lr_ce", C.c_float)]
+                ("lr_task", C.c_float), ("lr_ce", C.c_float), ("optimizer", C.c_int32), ("noam_warmup", C.c_int32),
+                ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float)]
 
 
 class GramStepReport(C.Structure):
@@ -74,6 +78,15 @@ def lib():
         L.gram_last_error.restype = C.c_char_p
         _lib = L
     return _lib
+
+
+def noam_rate(t: int, peak: float, warmup: int) -> float:
+    """The library's host-side learning-rate curve (no GPU needed)."""
+    out = C.c_float(0)
+    st = lib().gram_noam_rate(C.c_int64(int(t)), C.c_float(peak), C.c_int32(int(warmup)), C.byref(out))
+    if st != 0:
+        raise GramError(st, "gram_noam_rate")
+    return out.value
 
 
 def config_from_shape(shape, **over) -> GramConfig:
@@ -160,6 +173,17 @@ class Gram:
 
     def zero_grads(self, module: int, stream=None):
         self._ck(lib().gram_zero_grads(self._h, module, _stream(stream)))
+
+    def optimizer_step(self, module: int, stream=None):
+        self._ck(lib().gram_optimizer_step(self._h, module, _stream(stream)))
+
+    def optimizer_reset(self, stream=None):
+        self._ck(lib().gram_optimizer_reset(self._h, _stream(stream)))
+
+    def adam_update(self, w, g, m, v, t, rate, beta1=0.9, beta2=0.999, eps=1e-8, w_bf16=None, stream=None):
+        self._ck(lib().gram_adam_update(self._h, _ptr(w), _ptr(g), _ptr(m), _ptr(v), C.c_size_t(w.numel()), C.c_int64(int(t)),
+                                        C.c_float(rate), C.c_float(beta1), C.c_float(beta2), C.c_float(eps), _ptr(w_bf16),
+                                        _stream(stream)))
 
     def set_item_tokens(self, tokens: np.ndarray):
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)

@@ -6,6 +6,7 @@
 #include "gemm.h"
 #include "gram_internal.h"
 #include "model.h"
+#include "layers.h"
 
 constexpr int kProfSlots = 16384;
 struct ProfRec {
@@ -296,6 +297,27 @@ gram_status gram_get_grads(gram_ctx* ctx, int module, float* h, size_t n) {
 gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream) {
   NEED_MODEL("gram_zero_grads");
   return model_zero_grads(ctx->model, module, S(stream));
+}
+gram_status gram_optimizer_step(gram_ctx* ctx, int module, gram_stream stream) {
+  NEED_MODEL("gram_optimizer_step");
+  return model_optimizer_step(ctx->model, module, S(stream));
+}
+gram_status gram_optimizer_reset(gram_ctx* ctx, gram_stream stream) {
+  NEED_MODEL("gram_optimizer_reset");
+  return model_optimizer_reset(ctx->model, S(stream));
+}
+gram_status gram_noam_rate(int64_t t, float peak, int32_t warmup, float* h_rate) {
+  if (!h_rate || t < 1) return GRAM_ERR_ARG;
+  *h_rate = (float)noam_rate(t, (double)peak, warmup);
+  return GRAM_OK;
+}
+gram_status gram_adam_update(gram_ctx* ctx, float* d_w, const float* d_g, float* d_m, float* d_v, size_t n, int64_t t,
+                             float rate, float beta1, float beta2, float eps, void* d_w_bf16, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  if (n && (!d_w || !d_g || !d_m || !d_v)) return gram_set_error(ctx, "gram_adam_update: null buffer"), GRAM_ERR_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f))
+    return gram_set_error(ctx, "gram_adam_update: beta1 and beta2 must lie in [0, 1)"), GRAM_ERR_ARG;
+  return adam_update(ctx, d_w, d_g, d_m, d_v, d_w_bf16, n, t, rate, beta1, beta2, eps, S(stream));
 }
 gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens) {
   NEED_MODEL("gram_set_item_tokens");

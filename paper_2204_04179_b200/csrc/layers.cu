@@ -942,9 +942,65 @@ gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out,
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
+// Adam (Kingma & Ba, Algorithm 1) on four values per thread; c1, c2: the bias corrections 1 / (1 - beta^t)
+template <bool WB>
+__global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m,
+                                                   float* __restrict__ v, bf16* __restrict__ wb, size_t n, float rate,
+                                                   float beta1, float beta2, float eps, float c1, float c2) {
+  const size_t n4 = n >> 2;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 ww = reinterpret_cast<float4*>(w)[i];
+    const float4 gg = __ldcs(reinterpret_cast<const float4*>(g) + i);
+    float4 mm = reinterpret_cast<float4*>(m)[i], vv = reinterpret_cast<float4*>(v)[i];
+    float* pw = &ww.x; const float* pg = &gg.x; float* pm = &mm.x; float* pv = &vv.x;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      pm[k] = beta1 * pm[k] + (1.f - beta1) * pg[k];
+      pv[k] = beta2 * pv[k] + (1.f - beta2) * pg[k] * pg[k];
+      pw[k] -= rate * (pm[k] * c1) / (sqrtf(pv[k] * c2) + eps);
+    }
+    reinterpret_cast<float4*>(w)[i] = ww;
+    reinterpret_cast<float4*>(m)[i] = mm;
+    reinterpret_cast<float4*>(v)[i] = vv;
+    if (WB) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(ww.x, ww.y), hi = __floats2bfloat162_rn(ww.z, ww.w);
+      uint2 o;
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(wb)[i] = o;
+    }
+  }
+  // the last n % 4 values
+  for (size_t i = (n4 << 2) + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float gi = g[i];
+    const float mi = beta1 * m[i] + (1.f - beta1) * gi;
+    const float vi = beta2 * v[i] + (1.f - beta2) * gi * gi;
+    const float wi = w[i] - rate * (mi * c1) / (sqrtf(vi * c2) + eps);
+    m[i] = mi; v[i] = vi; w[i] = wi;
+    if (WB) wb[i] = __float2bfloat16(wi);
+  }
+}
+
+gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float* v, void* wb, size_t n, int64_t t, float rate,
+                        float beta1, float beta2, float eps, cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if (t < 1) return gram_set_error(ctx, "Adam: the update count starts at 1"), GRAM_ERR_ARG;
+  if (((uintptr_t)w | (uintptr_t)g | (uintptr_t)m | (uintptr_t)v) % 16 || (wb && (uintptr_t)wb % 8))
+    return gram_set_error(ctx, "Adam: buffers must be 16-byte aligned"), GRAM_ERR_UNSUPPORTED;
+  const float c1 = (float)(1.0 / (1.0 - pow((double)beta1, (double)t)));
+  const float c2 = (float)(1.0 / (1.0 - pow((double)beta2, (double)t)));
+  ProfScope prof(ctx, GRAM_K_OPTIMIZER, (double)n * (28.0 + (wb ? 2.0 : 0.0)), 1, st, "adam");
+  const int grid = grid_for((int64_t)((n + 3) / 4), 256, kNumSMs * 8);
+  if (wb) adam_kernel<true><<<grid, 256, 0, st>>>(w, g, m, v, (bf16*)wb, n, rate, beta1, beta2, eps, c1, c2);
+  else adam_kernel<false><<<grid, 256, 0, st>>>(w, g, m, v, nullptr, n, rate, beta1, beta2, eps, c1, c2);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
 gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st) {
   if (n == 0 || lr == 0.f) return GRAM_OK;
-  ProfScope prof(ctx, GRAM_K_OTHER, 12.0 * (double)n, 1, st);
+  ProfScope prof(ctx, GRAM_K_OPTIMIZER, 12.0 * (double)n, 1, st, "sgd");
   sgd_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(w, g, lr, n);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;

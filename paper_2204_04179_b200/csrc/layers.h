@@ -90,6 +90,9 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st);
 gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st);
 gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st);
+// one Adam update at count t >= 1 (Kingma & Ba, Algorithm 1); wb (may be null): bf16 copy of the new parameters
+gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float* v, void* wb, size_t n, int64_t t, float rate,
+                        float beta1, float beta2, float eps, cudaStream_t st);
 // dst[index[u], :] = src[u, :] (src fp32, dst operand-typed)
 gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st);

@@ -20,6 +20,8 @@ struct Module {
   float* g = nullptr;      // fp32 gradients
   bf16* wb = nullptr;      // bf16 copy of the parameters (bf16 contexts), refreshed when stale
   bool wb_stale = true;
+  float *am = nullptr, *av = nullptr;   // Adam moment estimates (contexts created with GRAM_OPT_ADAM)
+  int64_t updates = 0;     // updates applied so far (the count Adam's bias corrections and the Noam rate take)
 };
 
 // saved per layer.  fp32: the residual sums z1, z2 (attention-only layers: outf) and LayerNorm statistics;
@@ -115,6 +117,15 @@ struct Model {
   int32_t* h_pinned = nullptr;       // [4] pinned host words for small read-backs
 };
 
+// the Noam curve scaled to peak at update `warmup` (Section A; Vaswani et al. 2017, Eq. 3)
+double noam_rate(int64_t t, double peak, int warmup) {
+  if (warmup <= 0) return peak;
+  const double x = (double)t, w = (double)warmup;
+  const double up = x / w, down = sqrt(w / x);
+  return peak * (up < down ? up : down);
+}
+
+
 namespace {
 
 void stack_buffers(Arena& a, Stack& s, size_t esz) {
@@ -203,13 +214,19 @@ void layout_buffers(Model* m, Arena& a) {
   }
 }
 
-gram_status module_alloc(gram_ctx* ctx, Module* mod, size_t n, bool want_bf16) {
+gram_status module_alloc(gram_ctx* ctx, Module* mod, size_t n, bool want_bf16, bool want_adam) {
   mod->n = n;
   if (n == 0) return GRAM_OK;
   GRAM_CUDA(ctx, cudaMalloc(&mod->w, n * 4));
   GRAM_CUDA(ctx, cudaMalloc(&mod->g, n * 4));
   GRAM_CUDA(ctx, cudaMemset(mod->w, 0, n * 4));
   GRAM_CUDA(ctx, cudaMemset(mod->g, 0, n * 4));
+  if (want_adam) {
+    GRAM_CUDA(ctx, cudaMalloc(&mod->am, n * 4));
+    GRAM_CUDA(ctx, cudaMalloc(&mod->av, n * 4));
+    GRAM_CUDA(ctx, cudaMemset(mod->am, 0, n * 4));
+    GRAM_CUDA(ctx, cudaMemset(mod->av, 0, n * 4));
+  }
   if (want_bf16) GRAM_CUDA(ctx, cudaMalloc(&mod->wb, n * 2));
   mod->wb_stale = true;
   return GRAM_OK;
@@ -466,8 +483,20 @@ gram_status read_i32(Model* m, const int32_t* d_ptr, int32_t* out, cudaStream_t 
   return GRAM_OK;
 }
 
+// the configured update of one module from its gradients: lr is the SGD step or Adam's peak rate
 gram_status apply_sgd(Model* m, Module& mod, float lr, cudaStream_t st) {
   if (lr == 0.f || mod.n == 0) return GRAM_OK;
+  const gram_config& c = m->cfg;
+  ++mod.updates;
+  if (c.optimizer == GRAM_OPT_ADAM) {
+    const float b1 = c.adam_beta1 > 0.f ? c.adam_beta1 : 0.9f, b2 = c.adam_beta2 > 0.f ? c.adam_beta2 : 0.999f;
+    const float eps = c.adam_eps > 0.f ? c.adam_eps : 1e-8f;
+    const float rate = (float)noam_rate(mod.updates, lr, c.noam_warmup);
+    GRAM_TRY(adam_update(m->ctx, mod.w, mod.g, mod.am, mod.av, m->dtype == GRAM_BF16 ? mod.wb : nullptr, mod.n, mod.updates, rate,
+                         b1, b2, eps, st));
+    mod.wb_stale = false;                       // the kernel wrote the bf16 copy as well
+    return GRAM_OK;
+  }
   GRAM_TRY(sgd_update(m->ctx, mod.w, mod.g, lr, mod.n, st));
   mod.wb_stale = true;
   return GRAM_OK;
@@ -490,6 +519,24 @@ gram_status encoder_pass(Model* m, const int32_t* d_items, int32_t n_total, bool
 
 }  // namespace
 
+gram_status model_optimizer_step(Model* m, int module, cudaStream_t st) {
+  Module* mod = module == GRAM_MODULE_CE ? &m->ce : module == GRAM_MODULE_TASK ? &m->task : nullptr;
+  if (!mod) return gram_set_error(m->ctx, "unknown module %d", module), GRAM_ERR_ARG;
+  return apply_sgd(m, *mod, module == GRAM_MODULE_CE ? m->cfg.lr_ce : m->cfg.lr_task, st);
+}
+
+gram_status model_optimizer_reset(Model* m, cudaStream_t st) {
+  for (Module* mod : {&m->ce, &m->task}) {
+    mod->updates = 0;
+    if (mod->am && mod->n) {
+      GRAM_CUDA(m->ctx, cudaMemsetAsync(mod->am, 0, mod->n * 4, st));
+      GRAM_CUDA(m->ctx, cudaMemsetAsync(mod->av, 0, mod->n * 4, st));
+    }
+  }
+  return GRAM_OK;
+}
+
+
 // ===========================================================================================
 gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   *out = nullptr;
@@ -506,6 +553,8 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   if (c.dtype == GRAM_BF16 && (c.d % 8 || c.d_ff % 8 || c.task_d_ff % 8 || c.d_a % 8))
     return gram_set_error(ctx, "bf16 contexts need widths that are multiples of 8"), GRAM_ERR_UNSUPPORTED;
   if (c.B_max <= 0 || c.L <= 0) return gram_set_error(ctx, "B_max and L must be positive"), GRAM_ERR_ARG;
+  if (c.optimizer != GRAM_OPT_SGD && c.optimizer != GRAM_OPT_ADAM) return gram_set_error(ctx, "unknown optimizer %d", c.optimizer), GRAM_ERR_ARG;
+  if (c.adam_beta1 >= 1.f || c.adam_beta2 >= 1.f) return gram_set_error(ctx, "Adam: beta1 and beta2 must be below 1"), GRAM_ERR_ARG;
   // ---- parameter layouts (the order include/gram.h documents) ----
   size_t at = 0;
   if (c.n_layers > 0) {
@@ -520,7 +569,7 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
     m->enc.off.resize(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) at = layer_layout(&m->enc.off[l], at, c.d, c.d_ff, 0);
   }
-  GRAM_TRY(module_alloc(ctx, &m->ce, at, c.dtype == GRAM_BF16));
+  GRAM_TRY(module_alloc(ctx, &m->ce, at, c.dtype == GRAM_BF16, c.optimizer == GRAM_OPT_ADAM));
   at = 0;
   if (c.task == GRAM_TASK_KT) {
     if (c.task_layers > 0 && (c.task_heads <= 0 || c.d % c.task_heads)) return gram_set_error(ctx, "bad task shape"), GRAM_ERR_ARG;
@@ -538,7 +587,7 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
     m->t_ba = at; at += c.d_a;
     m->t_qa = at; at += c.d_a;
   }
-  GRAM_TRY(module_alloc(ctx, &m->task, at, c.dtype == GRAM_BF16));
+  GRAM_TRY(module_alloc(ctx, &m->task, at, c.dtype == GRAM_BF16, c.optimizer == GRAM_OPT_ADAM));
   // ---- sizes ----
   const int64_t P = (int64_t)c.B_max * c.L;
   m->u_cap = (int32_t)(P < c.n_items ? P : c.n_items);
@@ -562,8 +611,8 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
 
 void model_destroy(Model* m) {
   if (!m) return;
-  cudaFree(m->ce.w); cudaFree(m->ce.g); cudaFree(m->ce.wb);
-  cudaFree(m->task.w); cudaFree(m->task.g); cudaFree(m->task.wb);
+  cudaFree(m->ce.w); cudaFree(m->ce.g); cudaFree(m->ce.wb); cudaFree(m->ce.am); cudaFree(m->ce.av);
+  cudaFree(m->task.w); cudaFree(m->task.g); cudaFree(m->task.wb); cudaFree(m->task.am); cudaFree(m->task.av);
   cudaFree(m->arena);
   for (int i = 0; i < 8; ++i) if (m->ev[i]) cudaEventDestroy(m->ev[i]);
   if (m->h_pinned) cudaFreeHost(m->h_pinned);

@@ -13,6 +13,9 @@ gram_status model_param_count(const Model* m, int module, size_t* n);
 gram_status model_set_params(Model* m, int module, const float* h, size_t n);
 gram_status model_get_params(Model* m, int module, float* h, size_t n, int grads);
 gram_status model_zero_grads(Model* m, int module, cudaStream_t st);
+gram_status model_optimizer_step(Model* m, int module, cudaStream_t st);
+gram_status model_optimizer_reset(Model* m, cudaStream_t st);
+double noam_rate(int64_t t, double peak, int warmup);
 gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens);
 gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, float* d_H,
                          int save, cudaStream_t st);

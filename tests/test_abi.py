@@ -47,3 +47,12 @@ def test_config_struct_matches_header_field_order():
             typ, rest = decl.split(None, 1)
             fields += [(f.strip(), typ) for f in rest.split(",")]
     assert [(n, ctype[t]) for n, t in fields] == list(binding.GramStepReport._fields_)
+
+
+def test_noam_rate_host_function_matches_the_oracle():
+    """Host logic, no GPU: the library's learning-rate curve against the oracle's (fp32 result of a double formula)."""
+    from oracle import gram_oracle as O
+    for warm in (0, 1, 7, 4000):
+        for t in (1, 2, 6, 7, 8, 100, 3999, 4000, 4001, 10**6):
+            got = binding.noam_rate(t, 1e-4, warm)
+            assert abs(got - O.noam_rate(t, 1e-4, warm)) <= 1e-7 * 1e-4 + 6e-8 * got
