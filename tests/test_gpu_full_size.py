@@ -1,0 +1,156 @@
+"""Parity at the full size of the knowledge-tracing workload (B = 256 histories x L = 100 positions, 10,000 items,
+BERT-base-shaped encoder, bf16), in the launch configuration the benchmark times (all unique items in one encoder
+pass), stage by stage through the C ABI.
+
+The per-occurrence oracle cannot run 25,600 encoder calls, so each stage is compared on outputs the oracle can compute
+one by one, from inputs the oracle builds itself, and on properties that hold at any size:
+
+* dedup: every index output against the oracle, bit-exact;
+* encode: sampled rows of H against the oracle's encoder forward;
+* gather: E[p] == H[inverse[p]] bit-exact for every position;
+* task module: the gradient rows dL/dE of one whole history against the oracle (histories are independent in the
+  knowledge-tracing module, and the loss is a mean over all B*L predictions);
+* accumulate: sampled rows of G against a float64 sum over that item's occurrences, and conservation of column sums;
+* encoder backward: the VJP is linear in its cotangent, so a cotangent that is zero except for a few sampled items
+  yields exactly those items' gradient, which the oracle computes as the gradient of the pseudo-loss (Eq. 9) with
+  pseudo-targets h - g; the kernels still run over all unique items' activations.  With token-0 pooling the last
+  LayerNorm's bias gradient is the plain column sum of G.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gram_oracle as orc
+from paper_2204_04179_b200 import binding, synth
+from tests import gram_helpers as gh
+
+pytestmark = pytest.mark.gpu
+DEV = gh.DEV
+TOL = 2e-2
+
+
+def _row_err(got, want):
+    got = np.asarray(got, np.float64); want = np.asarray(want, np.float64)
+    return float(np.abs(got - want).max() / np.abs(want).max())
+
+
+def test_kt_workload_stage_by_stage():
+    shape = synth.config("kt")
+    seed = 0
+    ce = synth.encoder_params(shape, seed)
+    tk = synth.task_params(shape, seed)
+    toks = synth.item_tokens(seed, shape.n_items, shape.l_t, shape.vocab)
+    ids, lab = synth.batch(shape, seed, step=0)
+    P, d, B, L = ids.size, shape.d, shape.B, shape.L
+    assert (B, L, shape.n_items, d, shape.n_layers) == (256, 100, 10_000, 768, 12)
+    g = gh.make_ctx(shape, ce, tk, toks, ce_micro_batch=5120)
+    rng = np.random.default_rng(5)
+
+    # ---- stage 1 ----
+    ids_d = torch.from_numpy(ids.ravel().copy()).to(DEV)
+    lab_d = torch.from_numpy(lab.ravel().copy()).to(DEV)
+    cap = min(P, shape.n_items)
+    unique = torch.zeros(cap, dtype=torch.int32, device=DEV); inverse = torch.zeros(P, dtype=torch.int32, device=DEV)
+    perm = torch.zeros(P, dtype=torch.int32, device=DEV); seg = torch.zeros(cap + 1, dtype=torch.int32, device=DEV)
+    nu = torch.zeros(1, dtype=torch.int32, device=DEV)
+    g.dedup(ids_d, shape.n_items, unique, inverse, perm, seg, nu)
+    g.sync()
+    U = int(nu.item())
+    w_unique, w_inverse, w_perm, w_seg = orc.unique_inverse(ids)
+    assert U == len(w_unique) and 4000 < U <= 5120
+    assert np.array_equal(unique[:U].cpu().numpy(), w_unique) and np.array_equal(inverse.cpu().numpy(), w_inverse)
+    assert np.array_equal(perm.cpu().numpy(), w_perm) and np.array_equal(seg[:U + 1].cpu().numpy(), w_seg)
+
+    # ---- stage 2: sampled encodings ----
+    H = torch.zeros(U, d, device=DEV)
+    g.encode_unique(None, unique, U, H, save_activations=True)
+    g.sync()
+    counts = np.diff(w_seg)
+    sample_u = sorted({0, U - 1, int(np.argmax(counts))} | {int(x) for x in rng.integers(0, U, 3)})
+    want_H = orc.encode_all(shape, ce, toks, [w_unique[u] for u in sample_u])
+    H_np = H.cpu().numpy()
+    for k, u in enumerate(sample_u):
+        assert _row_err(H_np[u], want_H[k]) <= TOL, (u, _row_err(H_np[u], want_H[k]))
+
+    # ---- stage 3: every position, exact ----
+    E = torch.zeros(P, d, device=DEV)
+    g.gather(H, inverse, E)
+    g.sync()
+    assert torch.equal(E, H[inverse.long()])
+
+    # ---- task module: one whole history against the oracle ----
+    dE = torch.zeros(P, d, device=DEV); loss = torch.zeros(1, device=DEV)
+    g.task(E, lab_d, B, dE, loss)
+    g.sync()
+    b = int(rng.integers(0, B))
+    hist_items, hist_inv = np.unique(ids[b], return_inverse=True)
+    E_b = orc.encode_all(shape, ce, toks, hist_items)[hist_inv]                      # the oracle's own encodings
+    th_cf = orc.as_torch(tk)
+    E_t = torch.tensor(E_b[None], dtype=torch.float64, requires_grad=True)
+    loss_b = orc.task_loss(th_cf, E_t, lab[b:b + 1], shape.replace(B=1))             # mean over this history's L
+    loss_b.backward()
+    want_dE_b = E_t.grad[0].numpy() / B                                              # mean over all B*L predictions
+    got_dE_b = dE.view(B, L, d)[b].cpu().numpy()
+    assert _row_err(got_dE_b, want_dE_b) <= TOL, _row_err(got_dE_b, want_dE_b)
+    assert np.isfinite(float(loss.item())) and 0.3 < float(loss.item()) < 1.5       # near log 2 at this initialisation
+
+    # ---- stage 4 ----
+    G = torch.zeros(U, d, device=DEV)
+    g.accumulate(dE, perm, seg, U, G)
+    g.sync()
+    dE64 = dE.double()
+    col = dE64.sum(0)
+    assert float((G.double().sum(0) - col).abs().max()) <= 1e-5 * float(dE64.abs().sum(0).max())
+    for u in sample_u:
+        rows = torch.from_numpy(w_perm[w_seg[u]:w_seg[u + 1]].astype(np.int64)).to(DEV)
+        want = dE64[rows].sum(0)
+        bound = float(dE64[rows].abs().sum(0).max()) * len(rows) * 2.0 ** -24 + 1e-12
+        assert float((G[u].double() - want).abs().max()) <= bound, u
+
+    # ---- stage 5: the VJP of a few sampled items, computed over the full set of saved activations ----
+    picks = sorted({int(x) for x in rng.integers(0, U, 3)})
+    items = [int(w_unique[u]) for u in picks]
+    g_rows = rng.standard_normal((len(picks), d))
+    G_sparse = torch.zeros(U, d, device=DEV)
+    G_sparse[torch.tensor(picks, device=DEV)] = torch.from_numpy(g_rows).float().to(DEV)
+    g.zero_grads(binding.GRAM_MODULE_CE)
+    g.encoder_backward(G_sparse, unique, U)
+    gce, _ = gh.gpu_grads(g, shape)
+    h = orc.encode_all(shape, ce, toks, items)
+    _, want_g = orc.pseudo_loss_grad(shape, ce, toks, items, h - g_rows)             # Eq. 9 with h~ = h - g
+    worst, name = gh.worst_rel_err(gce, want_g)
+    print("full-size encoder backward, 3 sampled items: worst tensor", name, worst)
+    assert worst <= TOL, (name, worst)
+
+    # the full cotangent: the last LayerNorm's bias gradient is the column sum of G (token-0 pooling)
+    g.zero_grads(binding.GRAM_MODULE_CE)
+    g.encoder_backward(G, unique, U)
+    gce, _ = gh.gpu_grads(g, shape)
+    last = f"l{shape.n_layers - 1}.ln2_b"
+    want_b = G.double().sum(0).cpu().numpy()
+    assert _row_err(gce[last], want_b) <= 1e-4
+    for k, v in gce.items():
+        assert np.all(np.isfinite(v)), k
+    g.close()
+
+
+def test_kt_workload_step_equals_stages_and_micro_batches():
+    """gram_step at full size: the same report counts as the oracle's index work, and gradients that do not depend
+    on how the unique items are cut into encoder passes (a property that holds at any size)."""
+    shape = synth.config("kt")
+    seed = 0
+    ce = synth.encoder_params(shape, seed)
+    tk = synth.task_params(shape, seed)
+    toks = synth.item_tokens(seed, shape.n_items, shape.l_t, shape.vocab)
+    ids, lab = synth.batch(shape, seed, step=1)
+    U = len(np.unique(ids))
+    grads = []
+    for mb in (5120, 1536):
+        rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab, ce_micro_batch=mb)
+        assert rep.n_unique == U and rep.n_encoded == U and rep.n_positions == ids.size
+        grads.append((rep.loss, gce, gtk))
+    assert abs(grads[0][0] - grads[1][0]) <= 1e-5 * abs(grads[0][0])
+    for k in grads[0][1]:
+        assert gh.rel_err(grads[1][1][k], grads[0][1][k]) <= 2e-3, k
+    for k in grads[0][2]:
+        assert np.array_equal(grads[1][2][k], grads[0][2][k]), k        # the task module does not see the cut
