@@ -47,11 +47,9 @@ struct IndexWorkspace {
   int32_t n_items_max = 0;
   int32_t d_max = 0;
   int32_t *keys0 = nullptr, *keys1 = nullptr, *vals0 = nullptr, *vals1 = nullptr;  // [P_max] radix ping-pong
-  int32_t* hist = nullptr;        // [256 * n_sort_blocks] digit-major block histograms
-  int32_t* block_sums = nullptr;  // scan scratch
+  uint32_t* sort_ctl = nullptr;   // tile tickets, digit totals and per-tile status words of the sort (cleared per call)
   int32_t* rank_table = nullptr;  // [n_items_max] item ID -> index in unique
   float* partial = nullptr;       // [kAccMaxChunks * 2 * d_max] chunk-boundary partial sums, then kAccMaxChunks (item, last chunk) pairs
-  int32_t n_sort_blocks = 0;
 };
 
 gram_status index_ws_alloc(gram_ctx* ctx, IndexWorkspace* ws, int64_t P_max, int32_t n_items_max, int32_t d_max);
