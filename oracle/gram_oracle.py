@@ -21,6 +21,9 @@ What it states, and from where in the paper:
   states that this is not equivalent to end-to-end training, so there is no
   plain definition to reduce to; the readings taken where the algorithm is
   silent are listed in the function's docstring.
+* `multistep_window_pseudo_target`: the same window under the trainable-embedding
+  reading of Section 4.3 (the task module keeps using the modified embedding
+  h~, the encoder regresses towards it with the pseudo-loss of Eq. 9).
 * `unique_inverse_bruteforce`, `unique_inverse`, `segment_sum`,
   `table_accumulate`: the index work and the per-item sums on their own.
 * `boost_ratio`: the speed-boost ratio R (Section 4.4).
@@ -38,7 +41,9 @@ Pins (tests/test_oracle_*.py): brute force on tiny inputs, the worked count
 of Fig. 1, finite differences on a 1-layer encoder, closed forms of softmax /
 LayerNorm / GELU / BCE, the Proposition (e2e == single-step), the pseudo-loss
 identity (Eqs. 1-3), K = 1 reducing to single-step, and conservation of
-column sums; for the optimiser, torch.optim.Adam at a constant rate, the closed
+column sums; for the trainable-embedding window, torch.optim.SGD(lr=1) on an
+embedding parameter, finite differences of the pseudo-loss with a stale cache,
+and K = 1 with a fresh cache reducing to end-to-end training; for the optimiser, torch.optim.Adam at a constant rate, the closed
 form of the first step, and the closed-form values of the Noam curve.  The
 Multi-step *trajectory* beyond those is pinned only by the readings below:
 parity unpinned by the paper for that part.
@@ -388,6 +393,59 @@ def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache,
     cache[items] = round_to_bf16(newc) if cache_bf16 else newc
     return dict(losses=losses, grad_ce=_grads(th_ce), grad_task_last=grad_task_last, task_params=cur_task,
                 table=table, touched=touched, cache=cache, items=items.astype(np.int32))
+
+
+def multistep_window_pseudo_target(shape, ce_params, task_params, item_tokens, batches, cache, lr_task: float,
+                                   dtype=torch.float64):
+    """One window of K = len(batches) steps of Algorithm 1 under the *trainable-embedding* reading of
+    Section 4.3: the content representation of an item is a trainable embedding h~_i that the task module
+    keeps using after it has been modified ("based on updated content representations, we repeat the
+    process"), and the encoder regresses towards it (Eq. 9).
+
+    * h~ starts as `cache` [n_items, d] (encoder outputs computed before the window).
+    * Step 1 (Eq. 4) inside the window: the task module reads E[p] = h~[ids[p]], i.e. the cached encoding
+      minus every gradient the item has received so far in this window.
+    * Step 2 (Eq. 5): plain SGD with rate lr_task on the task parameters after every step.
+    * Step 3 (Eq. 6): h~[i] <- h~[i] - dL/dE[p] for every occurrence p of item i, in position order
+      (SGD with learning rate 1 on the embedding, as the paper prescribes).
+    * Step 4 after the K-th step, over all items modified in the window: the gradient of the pseudo-loss
+      1/2 sum_i (h~_i - CE(c_i; theta))^2 at the current encoder parameters, i.e. the encoder's VJP with
+      cotangent CE(c_i; theta) - h~_i.  When `cache` is stale (computed with older encoder parameters) that
+      cotangent carries the staleness CE(c_i; theta) - cache[i] besides the accumulated gradients.  The
+      forward values CE(c_i; theta) replace cache[i].
+
+    Returns dict(losses [K], grad_ce, grad_task_last, task_params, h_tilde (before the encoder pass), items,
+    cache (updated))."""
+    n_items, d = cache.shape
+    cache = np.array(cache, dtype=np.float64)
+    h_tilde = cache.copy()
+    modified = np.zeros(n_items, dtype=bool)
+    cur_task = OrderedDict((k, np.array(v, dtype=np.float64)) for k, v in task_params.items())
+    losses = []
+    grad_task_last = None
+    for ids, labels in batches:
+        ids = np.asarray(ids)
+        B, L = ids.shape
+        th_cf = as_torch(cur_task, dtype)
+        E = torch.tensor(h_tilde[ids.ravel()], dtype=dtype).reshape(B, L, d).requires_grad_(True)
+        loss = task_loss(th_cf, E, labels, shape)
+        loss.backward()
+        losses.append(float(loss.detach()))
+        grad_task_last = _grads(th_cf)
+        for k in cur_task:
+            cur_task[k] = cur_task[k] - lr_task * grad_task_last[k]
+        dE = E.grad.reshape(B * L, d).numpy()
+        for p, i in enumerate(ids.ravel()):
+            h_tilde[int(i), :] -= dE[p, :]
+            modified[int(i)] = True
+    items = np.nonzero(modified)[0]
+    th_ce = as_torch(ce_params, dtype)
+    H = torch.stack([ce_forward(th_ce, item_tokens[int(i)], shape) for i in items])
+    pseudo = 0.5 * ((torch.tensor(h_tilde[items], dtype=dtype) - H) ** 2).sum()
+    pseudo.backward()
+    cache[items] = H.detach().numpy()
+    return dict(losses=losses, grad_ce=_grads(th_ce), grad_task_last=grad_task_last, task_params=cur_task,
+                h_tilde=h_tilde, items=items.astype(np.int32), cache=cache, pseudo_loss=float(pseudo.detach()))
 
 
 # ---------------------------------------------------------------------------

@@ -251,3 +251,81 @@ def test_multistep_later_steps_see_updated_task_parameters():
     b = orc.multistep_window(shape, ce, tk, toks, batches, cache, lr_task=0.0)
     assert a["losses"][0] == pytest.approx(b["losses"][0], rel=1e-13)
     assert abs(a["losses"][1] - b["losses"][1]) > 1e-6
+
+
+# ---- Multi-step under the trainable-embedding reading (Section 4.3, Eqs. 6 and 9) ------------------------------------
+
+def test_pseudo_target_window_k1_fresh_cache_is_e2e():
+    # one step, cache computed with the current encoder: h~ - CE = -sum dL/dE, so Eq. 9's gradient is end-to-end's
+    shape = small_shape(pooling="cls")
+    ce, tk, toks, ids, lab = make(shape, seed=4)
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    got = orc.multistep_window_pseudo_target(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.1)
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    assert abs(got["losses"][0] - want["loss"]) < 1e-12
+    for k in want["grad_ce"]:
+        np.testing.assert_allclose(got["grad_ce"][k], want["grad_ce"][k], rtol=1e-9, atol=1e-12)
+    assert np.array_equal(got["items"], np.unique(ids))
+
+
+def test_pseudo_target_embedding_follows_library_sgd_with_rate_one():
+    # "treating it as trainable embedding": a torch Parameter updated by torch.optim.SGD(lr=1) over the same batches
+    # must end at the oracle's h~ (duplicates of an item inside a batch add up through autograd's index backward)
+    shape = small_shape(n_items=6, B=2, L=6)
+    ce, tk, toks, _, _ = make(shape, seed=6)
+    batches = [synth.batch(shape, 6, step=k) for k in range(3)]
+    assert any(len(np.unique(i)) < i.size for i, _ in batches)                    # duplicates inside a batch
+    assert len(np.intersect1d(batches[0][0], batches[1][0])) > 0                  # and an item seen in two steps
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    lr = 0.2
+    got = orc.multistep_window_pseudo_target(shape, ce, tk, toks, batches, cache, lr_task=lr)
+    emb = torch.nn.Parameter(torch.tensor(cache, dtype=T64))
+    th = orc.as_torch(tk)
+    opt_e = torch.optim.SGD([emb], lr=1.0)
+    opt_t = torch.optim.SGD(list(th.values()), lr=lr)
+    losses = []
+    for ids, lab in batches:
+        opt_e.zero_grad(); opt_t.zero_grad()
+        E = emb[torch.as_tensor(ids.astype(np.int64))]
+        loss = orc.task_loss(th, E, lab, shape)
+        loss.backward()
+        opt_e.step(); opt_t.step()
+        losses.append(float(loss.detach()))
+    np.testing.assert_allclose(got["losses"], losses, rtol=1e-12)
+    np.testing.assert_allclose(got["h_tilde"], emb.detach().numpy(), rtol=1e-12, atol=1e-14)
+    for k in th:
+        np.testing.assert_allclose(got["task_params"][k], th[k].detach().numpy(), rtol=1e-12, atol=1e-14)
+    # the later step really saw the modified embedding: with the unmodified cache its loss differs
+    plain = orc.multistep_window(shape, ce, tk, toks, batches, cache, lr_task=lr)
+    assert abs(plain["losses"][0] - got["losses"][0]) < 1e-14 and abs(plain["losses"][1] - got["losses"][1]) > 1e-9
+
+
+def test_pseudo_target_gradient_with_a_stale_cache_matches_finite_differences():
+    # a cache computed with other encoder parameters: the cotangent CE(c; theta) - h~ then carries the staleness term.
+    # Central differences of the pseudo-loss of Eq. 9 (h~ held constant) pin its sign and scale.
+    shape = small_shape(n_items=5, B=1, L=4, d=8, d_ff=16, vocab=12)
+    ce, tk, toks, ids, lab = make(shape, seed=8)
+    ce = OrderedDict((k, np.asarray(v, np.float64)) for k, v in ce.items())        # so that +-eps is exact enough
+    ce_old = OrderedDict((k, v + 0.05 * np.random.default_rng(1).standard_normal(v.shape)) for k, v in ce.items())
+    cache = orc.encode_all(shape, ce_old, toks, range(shape.n_items))
+    got = orc.multistep_window_pseudo_target(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0)
+    items, h_t = got["items"], got["h_tilde"][got["items"]]
+
+    def pseudo(params):
+        H = orc.encode_all(shape, params, toks, items)
+        return 0.5 * float(((h_t - H) ** 2).sum())
+    assert abs(pseudo(ce) - got["pseudo_loss"]) < 1e-12
+    rng = np.random.default_rng(2)
+    for name in ("l0.wqkv", "l0.w2", "tok_emb", "l0.ln2_b"):
+        flat_idx = rng.integers(0, ce[name].size, 3)
+        for fi in flat_idx:
+            idx = np.unravel_index(fi, ce[name].shape)
+            eps = 1e-6
+            up = OrderedDict((k, v.copy()) for k, v in ce.items()); up[name][idx] += eps
+            dn = OrderedDict((k, v.copy()) for k, v in ce.items()); dn[name][idx] -= eps
+            fd = (pseudo(up) - pseudo(dn)) / (2 * eps)
+            assert abs(fd - got["grad_ce"][name][idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, got["grad_ce"][name][idx])
+    # dropping the staleness term (the table-only cotangent of the other reading) gives a different gradient here
+    plain = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0)
+    assert max(np.abs(plain["grad_ce"][k] - got["grad_ce"][k]).max() for k in ce) > 1e-4
+    np.testing.assert_allclose(got["cache"][items], orc.encode_all(shape, ce, toks, items), rtol=1e-13)
