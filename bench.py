@@ -222,6 +222,8 @@ def run_gram(args, shape):
     multistep = shape.K > 1
     if multistep:                      # whole windows only: K-1 light steps and one step with the encoder pass
         over["lr_task"] = 1e-3
+        if args.multistep_variant == "pseudo_target":
+            over["multistep_variant"] = binding.GRAM_MULTI_PSEUDO_TARGET
         args.warmup = max(shape.K, -(-args.warmup // shape.K) * shape.K)
         args.steps = max(shape.K, -(-args.steps // shape.K) * shape.K)
     cfg = binding.config_from_shape(shape, **over)
@@ -342,7 +344,7 @@ def run_gram(args, shape):
                                 "sample": f"end-to-end oracle (float64, one encoder call per interaction) on the first {n_pos} "
                                           f"positions of one history of the same workload, {dt:.1f} s; linear in interactions"}
     if multistep:
-        line["multistep"] = {"K": shape.K, "windows_timed": args.steps // shape.K,
+        line["multistep"] = {"K": shape.K, "windows_timed": args.steps // shape.K, "variant": args.multistep_variant,
                              "per_step": [{"k": i % shape.K, "ms": r.ms_total, "touched": r.n_touched,
                                            "encoder_pass": r.encoder_pass, "n_encoded": r.n_encoded} for i, r in enumerate(reports)]}
     print(json.dumps(line))
@@ -358,6 +360,8 @@ def main():
     ap.add_argument("--impl", default="gram", choices=["gram", "reference"])
     ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny", "kt_multistep"])
     ap.add_argument("--micro-batch", type=int, default=0, help="items per encoder pass (0: the workload's default)")
+    ap.add_argument("--multistep-variant", default="table", choices=["table", "pseudo_target"],
+                    help="kt_multistep: separate gradient table with unchanged cached encodings, or pseudo-targets (Section 4.3)")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     from paper_2204_04179_b200 import synth

@@ -49,6 +49,18 @@ enum { GRAM_POOL_MEAN = 0, GRAM_POOL_CLS = 1 };       /* item pooling */
 enum { GRAM_TASK_NONE = 0, GRAM_TASK_KT = 1, GRAM_TASK_NR = 2 };
 enum { GRAM_MODULE_CE = 0, GRAM_MODULE_TASK = 1 };
 enum { GRAM_OPT_SGD = 0, GRAM_OPT_ADAM = 1 };
+/* Multi-step GRAM (Section 4.2, Algorithm 1 with N > 1), how a window treats the content representations:
+ * GRAM_MULTI_TABLE: the task module reads the unchanged cached encodings during the whole window, the
+ *   gradients of Eq. 6 go to a separate per-item table, and the encoder's cotangent is table[i].
+ * GRAM_MULTI_PSEUDO_TARGET: the trainable-embedding reading of Section 4.3 ("treating it as trainable
+ *   embedding", "based on updated content representations, we repeat the process"): the task module reads
+ *   the pseudo-target h~_i = cache[i] - table[i], i.e. the cached encoding minus every gradient the item
+ *   has received so far in the window (Eq. 6, SGD with learning rate 1), and the encoder regresses
+ *   towards it with the pseudo-loss of Eq. 9: its cotangent is CE(c_i; theta) - h~_i, which carries the
+ *   staleness CE(c_i; theta) - cache[i] of the cache besides the accumulated gradients.  The cache is
+ *   kept in fp32 in this variant whatever the context's dtype: pseudo-targets differ from the
+ *   encodings by gradient-sized amounts that bf16 would round away. */
+enum { GRAM_MULTI_TABLE = 0, GRAM_MULTI_PSEUDO_TARGET = 1 };
 
 /* Shapes of the two modules and of the batches a context serves.
  * CE (Section 3.2; Appendix D: attention layers of width 768): token + position
@@ -80,6 +92,7 @@ typedef struct gram_config {
                                   learning-rate scheme (Section A); lr_task / lr_ce are then the peak rates */
   int32_t noam_warmup;         /* updates until the peak rate; <= 0: constant rate */
   float adam_beta1, adam_beta2, adam_eps;   /* <= 0: 0.9, 0.999, 1e-8 */
+  int32_t multistep_variant;   /* K > 1: GRAM_MULTI_TABLE or GRAM_MULTI_PSEUDO_TARGET */
 } gram_config;
 
 typedef struct gram_step_report {

@@ -21,6 +21,7 @@ GRAM_POOL_MEAN, GRAM_POOL_CLS = 0, 1
 GRAM_TASK_NONE, GRAM_TASK_KT, GRAM_TASK_NR = 0, 1, 2
 GRAM_MODULE_CE, GRAM_MODULE_TASK = 0, 1
 GRAM_OPT_SGD, GRAM_OPT_ADAM = 0, 1
+GRAM_MULTI_TABLE, GRAM_MULTI_PSEUDO_TARGET = 0, 1
 STATUS = {0: "GRAM_OK", 1: "GRAM_ERR_ARG", 2: "GRAM_ERR_ID_RANGE", 3: "GRAM_ERR_WORKSPACE", 4: "GRAM_ERR_UNSUPPORTED",
           5: "GRAM_ERR_CUDA", 6: "GRAM_ERR_TIMEOUT"}
 
@@ -43,7 +44,8 @@ class GramConfig(C.Structure):
                                           "task_attn_only", "d_a", "n_cand", "B_max", "L")] + \
                [("P_max", C.c_int64), ("d_max", C.c_int32), ("K", C.c_int32), ("ce_micro_batch", C.c_int32),
                 ("lr_task", C.c_float), ("lr_ce", C.c_float), ("optimizer", C.c_int32), ("noam_warmup", C.c_int32),
-                ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float)]
+                ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float),
+                ("multistep_variant", C.c_int32)]
 
 
 class GramStepReport(C.Structure):

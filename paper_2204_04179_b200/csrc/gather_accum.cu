@@ -56,6 +56,44 @@ __global__ void gather_scalar_kernel(const T* __restrict__ src, int64_t n_src_ro
   }
 }
 
+// out[r, :] = a[index[r], :] - b[index[r], :], or x[r, :] - that; a warp per row, 4 floats per lane and step
+__global__ void __launch_bounds__(256) gather_diff_kernel(const float* __restrict__ a, const float* __restrict__ b,
+                                                          int64_t n_src_rows, const int32_t* __restrict__ index, int64_t n,
+                                                          int d, const float* __restrict__ x, float* __restrict__ out,
+                                                          int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const bool vec = (d & 3) == 0;
+  for (int64_t r = warp; r < n; r += nwarps) {
+    int32_t i = index[r];
+    if (i < 0 || i >= n_src_rows) {
+      gram_device_fail(status, GRAM_ERR_ID_RANGE);
+      i = 0;
+    }
+    const float* pa = a + (int64_t)i * d;
+    const float* pb = b + (int64_t)i * d;
+    const float* px = x ? x + r * d : nullptr;
+    float* po = out + r * d;
+    if (vec) {
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 va = *reinterpret_cast<const float4*>(pa + c), vb = *reinterpret_cast<const float4*>(pb + c);
+        float4 v = make_float4(va.x - vb.x, va.y - vb.y, va.z - vb.z, va.w - vb.w);
+        if (px) {
+          const float4 vx = *reinterpret_cast<const float4*>(px + c);
+          v = make_float4(vx.x - v.x, vx.y - v.y, vx.z - v.z, vx.w - v.w);
+        }
+        *reinterpret_cast<float4*>(po + c) = v;
+      }
+    } else {
+      for (int c = lane; c < d; c += 32) {
+        const float v = pa[c] - pb[c];
+        po[c] = px ? px[c] - v : v;
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------
 // segmented sum.  The sorted order j in [0, P) is cut into nchunks equal chunks of R rows; the
 // columns into slabs of VPL*128 floats.  One warp owns one (chunk, slab): it walks its rows in
@@ -348,6 +386,19 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
     else
       gather_scalar_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)d_src, n_src_rows, d_index, P, d, (bf16*)d_E, status);
   }
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status gather_diff_launch(gram_ctx* ctx, const float* d_a, const float* d_b, int64_t n_src_rows, const int32_t* d_index,
+                               int64_t n, int32_t d, const float* d_x, float* d_out, cudaStream_t st) {
+  if (n < 0 || d <= 0 || n_src_rows <= 0 || (n > 0 && (!d_a || !d_b || !d_index || !d_out)))
+    return gram_set_error(ctx, "gather of pseudo-targets: bad argument"), GRAM_ERR_ARG;
+  if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_GATHER, (double)n * d * 4.0 * (d_x ? 4.0 : 3.0) + 4.0 * (double)n, 1, st);
+  int blocks = (int)ceil_div64(n, 8);
+  if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+  gather_diff_kernel<<<blocks, 256, 0, st>>>(d_a, d_b, n_src_rows, d_index, n, d, d_x, d_out, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

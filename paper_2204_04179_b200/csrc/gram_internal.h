@@ -62,6 +62,12 @@ gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids
 gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
                           int32_t d, int elem_bytes, void* d_E, cudaStream_t st);
 
+// out[r, :] = a[index[r], :] - b[index[r], :] (d_x == NULL), or d_x[r, :] - (a[index[r], :] - b[index[r], :]); fp32 rows.
+// Multi-step with pseudo-targets: the first form is h~ = cache - table gathered into the positions (Eq. 6), the
+// second the cotangent CE(c) - h~ of the pseudo-loss (Eq. 9).
+gram_status gather_diff_launch(gram_ctx* ctx, const float* d_a, const float* d_b, int64_t n_src_rows, const int32_t* d_index,
+                               int64_t n, int32_t d, const float* d_x, float* d_out, cudaStream_t st);
+
 // in_bf16: rows of d_in are bf16 instead of fp32.  d_U (may be NULL): the number of segments is read
 // from the device instead of U.  d_rows (may be NULL): output row of segment u is d_rows[u] instead
 // of u.  add != 0: out[row] += sum instead of out[row] = sum.

@@ -109,6 +109,8 @@ struct Model {
   float* table = nullptr;
   uint32_t* touched = nullptr;
   void* cache = nullptr;
+  int cache_dtype = GRAM_F32;        // element type of the cache: the context's, or fp32 with pseudo-targets
+  bool pseudo = false;               // Multi-step with pseudo-targets (GRAM_MULTI_PSEUDO_TARGET)
   int32_t *tlist = nullptr, *tcount = nullptr;
   int step_in_window = 0;
   char* arena = nullptr;
@@ -208,7 +210,7 @@ void layout_buffers(Model* m, Arena& a) {
   if (c.K > 1) {
     m->table = (float*)a.take((size_t)c.n_items * d * 4);
     m->touched = (uint32_t*)a.take((size_t)((c.n_items + 31) / 32) * 4);
-    m->cache = a.take((size_t)c.n_items * d * esz);
+    m->cache = a.take((size_t)c.n_items * d * (m->cache_dtype == GRAM_BF16 ? 2 : 4));
     m->tlist = (int32_t*)a.take((size_t)c.n_items * 4);
     m->tcount = (int32_t*)a.take(4);
   }
@@ -509,9 +511,9 @@ gram_status encoder_pass(Model* m, const int32_t* d_items, int32_t n_total, bool
   for (int32_t u0 = 0; u0 < n_total; u0 += m->mb) {
     const int32_t n = (n_total - u0 < m->mb) ? n_total - u0 : m->mb;
     GRAM_TRY(encoder_forward_chunk(m, nullptr, d_items + u0, 0, n, m->H, st));
-    if (update_cache) GRAM_TRY(scatter_rows(m->ctx, m->dtype, m->H, d_items + u0, n, m->cfg.d, m->cfg.n_items, m->cache, st));
     const float* G = nullptr;
-    GRAM_TRY(G_of(u0, n, &G));
+    GRAM_TRY(G_of(u0, n, &G));                 // may read the cache rows of these items: before they are replaced
+    if (update_cache) GRAM_TRY(scatter_rows(m->ctx, m->cache_dtype, m->H, d_items + u0, n, m->cfg.d, m->cfg.n_items, m->cache, st));
     GRAM_TRY(encoder_backward_chunk(m, G, n, st));
   }
   return GRAM_OK;
@@ -555,6 +557,10 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   if (c.B_max <= 0 || c.L <= 0) return gram_set_error(ctx, "B_max and L must be positive"), GRAM_ERR_ARG;
   if (c.optimizer != GRAM_OPT_SGD && c.optimizer != GRAM_OPT_ADAM) return gram_set_error(ctx, "unknown optimizer %d", c.optimizer), GRAM_ERR_ARG;
   if (c.adam_beta1 >= 1.f || c.adam_beta2 >= 1.f) return gram_set_error(ctx, "Adam: beta1 and beta2 must be below 1"), GRAM_ERR_ARG;
+  if (c.multistep_variant != GRAM_MULTI_TABLE && c.multistep_variant != GRAM_MULTI_PSEUDO_TARGET)
+    return gram_set_error(ctx, "unknown multistep_variant %d", c.multistep_variant), GRAM_ERR_ARG;
+  m->pseudo = c.K > 1 && c.multistep_variant == GRAM_MULTI_PSEUDO_TARGET;
+  m->cache_dtype = m->pseudo ? GRAM_F32 : c.dtype;
   // ---- parameter layouts (the order include/gram.h documents) ----
   size_t at = 0;
   if (c.n_layers > 0) {
@@ -709,7 +715,7 @@ gram_status model_cache_fill(Model* m, cudaStream_t st) {
   for (int32_t u0 = 0; u0 < c.n_items; u0 += m->mb) {
     const int32_t n = (c.n_items - u0 < m->mb) ? c.n_items - u0 : m->mb;
     GRAM_TRY(encoder_forward_chunk(m, nullptr, nullptr, u0, n, m->H, st));
-    if (m->dtype == GRAM_BF16) GRAM_TRY(convert_f32_to_bf16(m->ctx, m->H, (bf16*)m->cache + (size_t)u0 * c.d, (size_t)n * c.d, st));
+    if (m->cache_dtype == GRAM_BF16) GRAM_TRY(convert_f32_to_bf16(m->ctx, m->H, (bf16*)m->cache + (size_t)u0 * c.d, (size_t)n * c.d, st));
     else GRAM_CUDA(m->ctx, cudaMemcpyAsync((float*)m->cache + (size_t)u0 * c.d, m->H, (size_t)n * c.d * 4, cudaMemcpyDeviceToDevice, st));
   }
   m->saved_n = -1;
@@ -727,7 +733,7 @@ gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, floa
     const size_t rows_per = (size_t)((int64_t)c.B_max * c.L);
     for (size_t r0 = 0; r0 < (size_t)c.n_items; r0 += rows_per) {
       const size_t nr = ((size_t)c.n_items - r0 < rows_per) ? (size_t)c.n_items - r0 : rows_per;
-      GRAM_TRY(convert_to_f32(m->ctx, m->dtype, (char*)m->cache + r0 * c.d * m->esz, m->dE, nr * c.d, 0));
+      GRAM_TRY(convert_to_f32(m->ctx, m->cache_dtype, (char*)m->cache + r0 * c.d * (m->cache_dtype == GRAM_BF16 ? 2 : 4), m->dE, nr * c.d, 0));
       GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
       GRAM_CUDA(m->ctx, cudaMemcpy(h_cache + r0 * c.d, m->dE, nr * c.d * 4, cudaMemcpyDeviceToHost));
     }
@@ -773,7 +779,9 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
     GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, 4, m->E, st));
   } else {
     GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
-    if (m->dtype == GRAM_BF16) {       // rows of the bf16 cache, widened for the task module
+    if (m->pseudo) {                   // the pseudo-targets h~ = cache - table of the items at every position (Eq. 6)
+      GRAM_TRY(gather_diff_launch(ctx, (const float*)m->cache, m->table, c.n_items, ids, P, c.d, nullptr, m->E, st));
+    } else if (m->cache_dtype == GRAM_BF16) {       // rows of the bf16 cache, widened for the task module
       GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 2, m->Eb, st));
       GRAM_TRY(convert_to_f32(ctx, GRAM_BF16, m->Eb, m->E, (size_t)P * c.d, st));
     } else {
@@ -817,6 +825,9 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
       GRAM_TRY(encoder_pass(m, m->tlist, n_touched, true,
                             [&](int32_t u0, int32_t n, const float** G) {
                               *G = m->G;
+                              if (m->pseudo)       // Eq. 9: CE(c_i) - h~_i, with the forward values of this pass in H
+                                return gather_diff_launch(ctx, (const float*)m->cache, m->table, c.n_items, m->tlist + u0, n, c.d,
+                                                          m->H, m->G, st);
                               return gather_launch(ctx, m->table, c.n_items, m->tlist + u0, n, c.d, 4, m->G, st);
                             }, st));
       GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));

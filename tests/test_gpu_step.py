@@ -197,3 +197,66 @@ def test_multistep_window_matches_algorithm(dtype, K):
         one = orc.multistep_window(shape, ce, tk, toks, batches[:1], cache0.astype(np.float64), lr_task=lr)
         assert gh.rel_err(table, one["table"]) <= tol
     g.close()
+
+
+def test_multistep_pseudo_target_two_windows_f32():
+    """GRAM_MULTI_PSEUDO_TARGET against Algorithm 1 under the trainable-embedding reading (Section 4.3): two windows of
+    K = 3 steps with an encoder update in between, so that the second window's cache is stale and the cotangent of
+    Eq. 9 carries CE(c; theta) - cache besides the accumulated gradients."""
+    K = 3
+    shape = small(dtype="f32", d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=23)
+    lr_t, lr_c = 0.05, 0.02
+    batches = [synth.batch(shape, 23, step=k) for k in range(2 * K)]
+    g = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=lr_t, lr_ce=lr_c, ce_micro_batch=16,
+                    multistep_variant=binding.GRAM_MULTI_PSEUDO_TARGET)
+    g.cache_fill()
+    _, _, cache0 = g.get_window(want_table=False, want_touched=False)
+    assert gh.rel_err(cache0, orc.encode_all(shape, ce, toks, range(shape.n_items))) <= 1e-4
+    cur_ce = {k: np.asarray(v, np.float64) for k, v in ce.items()}
+    cur_tk = {k: np.asarray(v, np.float64) for k, v in tk.items()}
+    cache = cache0.astype(np.float64)
+    plain_losses = orc.multistep_window(shape, ce, tk, toks, batches[:K], cache, lr_task=lr_t)["losses"]
+    for w in range(2):
+        want = orc.multistep_window_pseudo_target(shape, cur_ce, cur_tk, toks, batches[w * K:(w + 1) * K], cache, lr_task=lr_t)
+        reps = [g.step(torch.from_numpy(i).to(DEV), torch.from_numpy(l).to(DEV), shape.B) for i, l in batches[w * K:(w + 1) * K]]
+        assert [r.encoder_pass for r in reps] == [0] * (K - 1) + [1]
+        assert reps[-1].n_touched == len(want["items"]) == reps[-1].n_encoded
+        for k in range(K):
+            assert abs(reps[k].loss - want["losses"][k]) <= 1e-4 * abs(want["losses"][k]), (w, k)
+        if w == 0:      # the later steps really read the modified embeddings, not the cached ones
+            assert abs(reps[1].loss - plain_losses[1]) > 10 * abs(reps[1].loss - want["losses"][1])
+        gce, gtk = gh.gpu_grads(g, shape)
+        e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+        e2, n2 = gh.worst_rel_err(gtk, want["grad_task_last"])
+        print("window", w, "worst CE", e1, n1, "worst task", e2, n2)
+        assert e1 <= 1e-3 and e2 <= 1e-3, (w, e1, n1, e2, n2)
+        _, _, cache_gpu = g.get_window(want_table=False, want_touched=False)
+        assert gh.rel_err(cache_gpu, want["cache"]) <= 1e-4
+        cur_ce = {k: cur_ce[k] - lr_c * want["grad_ce"][k] for k in cur_ce}
+        cur_tk = want["task_params"]
+        cache = want["cache"]
+    g.close()
+
+
+def test_multistep_pseudo_target_first_window_bf16():
+    # a bf16 context keeps the cache in fp32 for this variant; in the first window after a cache fill the staleness
+    # term is zero on both sides, so the comparison is the usual one for bf16 encoders
+    K = 2
+    shape = small(dtype="bf16", d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=25)
+    batches = [synth.batch(shape, 25, step=k) for k in range(K)]
+    g = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=0.05, ce_micro_batch=16,
+                    multistep_variant=binding.GRAM_MULTI_PSEUDO_TARGET)
+    g.cache_fill()
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    want = orc.multistep_window_pseudo_target(shape, ce, tk, toks, batches, cache, lr_task=0.05)
+    reps = [g.step(torch.from_numpy(i).to(DEV), torch.from_numpy(l).to(DEV), shape.B) for i, l in batches]
+    for k in range(K):
+        assert abs(reps[k].loss - want["losses"][k]) <= 2e-2 * abs(want["losses"][k])
+    gce, gtk = gh.gpu_grads(g, shape)
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task_last"])
+    print("bf16 pseudo-target worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= 2e-2 and e2 <= 2e-2, (e1, n1, e2, n2)
+    g.close()
