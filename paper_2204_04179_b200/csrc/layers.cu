@@ -686,6 +686,16 @@ __global__ void scatter_rows_kernel(const float* __restrict__ src, const int32_t
   stf(dst + (int64_t)r * d + c, src[i]);
 }
 
+// rows of `words` 32-bit words copied between two layouts whose rows are in_stride / out_stride words apart
+__global__ void strided_rows_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out, int64_t n, int64_t in_stride,
+                                    int64_t out_stride, int words) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * words) return;
+  const int64_t r = i / words;
+  const int c = (int)(i - r * words);
+  out[r * out_stride + c] = in[r * in_stride + c];
+}
+
 inline int grid_for(int64_t n, int threads, int cap) {
   int64_t b = (n + threads - 1) / threads;
   if (b > cap) b = cap;
@@ -1010,6 +1020,29 @@ gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32
   if (n == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_OTHER, (double)n * d * (4.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
   DISPATCH_T(dtype, scatter_rows_kernel<T><<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(src, index, n, d, n_dst_rows, (T*)dst, gram_status_word(ctx)));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
+                              cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if ((d * elem_bytes) % 4) return gram_set_error(ctx, "row copy: rows must be whole 32-bit words"), GRAM_ERR_ARG;
+  const int words = d * elem_bytes / 4;
+  ProfScope prof(ctx, GRAM_K_OTHER, 2.0 * (double)n * d * elem_bytes, 1, st);
+  strided_rows_kernel<<<(unsigned)ceil_div64(n * words, 256), 256, 0, st>>>((const uint32_t*)in, (uint32_t*)out, n, stride * words,
+                                                                          words, words);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
+                             cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if ((d * elem_bytes) % 4) return gram_set_error(ctx, "row copy: rows must be whole 32-bit words"), GRAM_ERR_ARG;
+  const int words = d * elem_bytes / 4;
+  ProfScope prof(ctx, GRAM_K_OTHER, 2.0 * (double)n * d * elem_bytes, 1, st);
+  strided_rows_kernel<<<(unsigned)ceil_div64(n * words, 256), 256, 0, st>>>((const uint32_t*)in, (uint32_t*)out, n, words,
+                                                                          stride * words, words);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -96,3 +96,9 @@ gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float
 // dst[index[u], :] = src[u, :] (src fp32, dst operand-typed)
 gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st);
+// out[r, :] = in[r * stride, :] for r < n: every stride-th row of a [n*stride, d] matrix of elem_bytes-byte elements
+gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
+                              cudaStream_t st);
+// out[r * stride, :] = in[r, :] for r < n; the other rows of out are left as they are
+gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
+                             cudaStream_t st);

@@ -85,6 +85,12 @@ struct Model {
   // encoder
   size_t o_tok = 0, o_pos = 0, o_elng = 0, o_elnb = 0;
   Stack enc;
+  // With token-0 pooling only row 0 of every item's last-layer output is ever read, so the row-wise part of the
+  // last layer (output projection, feed-forward, both LayerNorms) runs on those rows alone: `tail` holds their
+  // activations and scratch (one row per item), tail_* the layer's input stream at those rows.
+  bool cls_tail = false;
+  Stack tail;
+  float *tail_z = nullptr, *tail_mean = nullptr, *tail_rstd = nullptr;
   float* z0 = nullptr;               // token + position embedding, fp32
   void* x0 = nullptr;                // its LayerNorm, operand-typed
   float *mean0 = nullptr, *rstd0 = nullptr;
@@ -180,6 +186,12 @@ void layout_buffers(Model* m, Arena& a) {
     m->tok_seg = (int32_t*)a.take((tu + 1) * 4);
     m->tok_nu = (int32_t*)a.take(4);
     stack_buffers(a, m->enc, esz);
+    if (m->cls_tail) {
+      stack_buffers(a, m->tail, esz);
+      m->tail_z = (float*)a.take((size_t)m->mb * d * 4);
+      m->tail_mean = (float*)a.take((size_t)m->mb * 4);
+      m->tail_rstd = (float*)a.take((size_t)m->mb * 4);
+    }
     m->item_tokens = (int32_t*)a.take((size_t)c.n_items * c.l_t * 4);
   }
   if (c.task != GRAM_TASK_NONE) {
@@ -277,114 +289,163 @@ void set_res(GemmEpilogue& e, const StreamRef& x) {
   e.res_beta = x.beta;
 }
 
-// x_in: the fp32 input stream; x_in_b: its operand-typed copy.  *out / *out_b: the same pair for the output.
-gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in, const void* x_in_b, int64_t n_seq, int S,
-                          cudaStream_t st, StreamRef* out, const void** out_b) {
+// ---- one transformer layer in two parts, forward --------------------------------------------
+// the attention part over whole sequences: qkv = x Wqkv^T + bqkv, ctx = softmax(Q K^T / sqrt(dh)) V
+gram_status layer_attention_forward(Model* m, Module& mod, Stack& s, int l, const void* xb, int64_t n_seq, int S, cudaStream_t st) {
   const int64_t T = n_seq * S;
-  const int d = s.d, f = s.d_ff;
+  const LayerOff& o = s.off[l];
+  LayerActs& a = s.acts[l];
+  GemmEpilogue e;
+  e.bias = mod.w + o.bqkv;
+  e.tag = "fwd_qkv";
+  GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * s.d, s.d, e, st));
+  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, st);
+}
+
+// the row-wise rest of the layer over T rows: output projection + residual, LayerNorm, feed-forward + residual,
+// LayerNorm.  x: the layer's input stream at those rows; ctx_in: the attention output at those rows; a: where the
+// activations of these rows are kept.  The rows need not be whole sequences.
+gram_status layer_rest_forward(Model* m, Module& mod, const LayerOff& o, LayerActs& a, int d, int f, int attn_only,
+                               const StreamRef& x, const void* ctx_in, int64_t T, cudaStream_t st, StreamRef* x_out,
+                               const void** xb_out) {
   gram_ctx* ctx = m->ctx;
+  GemmEpilogue e;
+  e.bias = mod.w + o.bo;
+  e.tag = "fwd_attn_out";
+  set_res(e, x);
+  if (attn_only) {
+    e.copy_out = a.out;
+    GRAM_TRY(mm_fwd(m, ctx_in, W(m, mod, o.wo), a.outf, true, T, d, d, e, st));       // out = x + ctx Wo^T + bo
+    *x_out = StreamRef();
+    x_out->z = a.outf;
+  } else {
+    GRAM_TRY(mm_fwd(m, ctx_in, W(m, mod, o.wo), a.z1, true, T, d, d, e, st));         // z1 = x + ctx Wo^T + bo
+    GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z1, mod.w + o.ln1g, mod.w + o.ln1b, a.h1, a.mean1, a.rstd1, T, d, st));
+    e = GemmEpilogue();
+    e.bias = mod.w + o.b1;
+    e.gelu = 1;
+    e.pre = a.u;
+    e.tag = "fwd_ffn1";
+    GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, false, T, f, d, e, st));          // v = h1 W1^T + b1: g = gelu(v), u = gelu'(v)
+    e = GemmEpilogue();
+    e.bias = mod.w + o.b2;
+    e.tag = "fwd_ffn2";
+    StreamRef h1;
+    h1.z = a.z1; h1.mean = a.mean1; h1.rstd = a.rstd1; h1.gamma = mod.w + o.ln1g; h1.beta = mod.w + o.ln1b;
+    set_res(e, h1);
+    GRAM_TRY(mm_fwd(m, a.g, W(m, mod, o.w2), a.z2, true, T, d, f, e, st));           // z2 = LN1(z1) + g W2^T + b2
+    GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z2, mod.w + o.ln2g, mod.w + o.ln2b, a.out, a.mean2, a.rstd2, T, d, st));
+    *x_out = StreamRef();
+    x_out->z = a.z2; x_out->mean = a.mean2; x_out->rstd = a.rstd2; x_out->gamma = mod.w + o.ln2g; x_out->beta = mod.w + o.ln2b;
+  }
+  *xb_out = a.out;
+  return GRAM_OK;
+}
+
+// x_in: the fp32 input stream; x_in_b: its operand-typed copy.  *out / *out_b: the same pair for the output of
+// layer n_full - 1.  Layers [0, n_full) run completely; when n_full < n_layers, layer n_full runs its attention
+// part only (its ctx is left in s.acts[n_full].ctx) and *out / *out_b describe that layer's input.
+gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in, const void* x_in_b, int64_t n_seq, int S,
+                          cudaStream_t st, StreamRef* out, const void** out_b, int n_full = -1) {
+  const int64_t T = n_seq * S;
+  if (n_full < 0) n_full = s.n_layers;
   StreamRef x = x_in;
   const void* xb = x_in_b;
-  for (int l = 0; l < s.n_layers; ++l) {
-    const LayerOff& o = s.off[l];
-    LayerActs& a = s.acts[l];
-    GemmEpilogue e;
-    e.bias = mod.w + o.bqkv;
-    e.tag = "fwd_qkv";
-    GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * d, d, e, st));
-    GRAM_TRY(attention_forward(ctx, m->dtype, a.qkv, a.ctx, n_seq, S, d, s.heads, s.causal, st));
-    e = GemmEpilogue();
-    e.bias = mod.w + o.bo;
-    e.tag = "fwd_attn_out";
-    set_res(e, x);
-    if (s.attn_only) {
-      e.copy_out = a.out;
-      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.outf, true, T, d, d, e, st));       // out = x + ctx Wo^T + bo
-      x = StreamRef();
-      x.z = a.outf;
-    } else {
-      GRAM_TRY(mm_fwd(m, a.ctx, W(m, mod, o.wo), a.z1, true, T, d, d, e, st));         // z1 = x + ctx Wo^T + bo
-      GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z1, mod.w + o.ln1g, mod.w + o.ln1b, a.h1, a.mean1, a.rstd1, T, d, st));
-      e = GemmEpilogue();
-      e.bias = mod.w + o.b1;
-      e.gelu = 1;
-      e.pre = a.u;
-      e.tag = "fwd_ffn1";
-      GRAM_TRY(mm_fwd(m, a.h1, W(m, mod, o.w1), a.g, false, T, f, d, e, st));          // v = h1 W1^T + b1: g = gelu(v), u = gelu'(v)
-      e = GemmEpilogue();
-      e.bias = mod.w + o.b2;
-      e.tag = "fwd_ffn2";
-      StreamRef h1;
-      h1.z = a.z1; h1.mean = a.mean1; h1.rstd = a.rstd1; h1.gamma = mod.w + o.ln1g; h1.beta = mod.w + o.ln1b;
-      set_res(e, h1);
-      GRAM_TRY(mm_fwd(m, a.g, W(m, mod, o.w2), a.z2, true, T, d, f, e, st));           // z2 = LN1(z1) + g W2^T + b2
-      GRAM_TRY(layernorm_forward(ctx, m->dtype, a.z2, mod.w + o.ln2g, mod.w + o.ln2b, a.out, a.mean2, a.rstd2, T, d, st));
-      x = StreamRef();
-      x.z = a.z2; x.mean = a.mean2; x.rstd = a.rstd2; x.gamma = mod.w + o.ln2g; x.beta = mod.w + o.ln2b;
-    }
-    xb = a.out;
+  for (int l = 0; l < n_full; ++l) {
+    GRAM_TRY(layer_attention_forward(m, mod, s, l, xb, n_seq, S, st));
+    GRAM_TRY(layer_rest_forward(m, mod, s.off[l], s.acts[l], s.d, s.d_ff, s.attn_only, x, s.acts[l].ctx, T, st, &x, &xb));
   }
+  if (n_full < s.n_layers) GRAM_TRY(layer_attention_forward(m, mod, s, n_full, xb, n_seq, S, st));
   *out = x;
   *out_b = xb;
   return GRAM_OK;
 }
 
-// On entry s.curf holds the gradient with respect to the stack's output (fp32; for a stack of
-// attention-only layers s.dzb holds its operand-typed copy as well).  On return *d_in points at the
-// fp32 gradient with respect to the input stream.
-gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, int64_t n_seq, int S, cudaStream_t st,
-                           float** d_in) {
-  const int64_t T = n_seq * S;
+// ---- the same two parts, backward -----------------------------------------------------------
+// Rows part.  On entry *cur holds the gradient with respect to the layer's output at T rows (for an attention-only
+// layer s.dzb holds its operand-typed copy as well); s supplies the scratch (dzb, du, dctx, cpart), a the saved
+// activations of those rows.  On return s.dctx holds the gradient with respect to the attention output, *oth the
+// gradient that reaches the layer's input through the residual connection (fp32), and *cur is free.
+gram_status layer_rest_backward(Model* m, Module& mod, const LayerOff& o, Stack& s, LayerActs& a, int64_t T, float** cur_io,
+                                float** oth_io, cudaStream_t st) {
   const int d = s.d, f = s.d_ff;
   gram_ctx* ctx = m->ctx;
   float* red = m->red;
+  float* cur = *cur_io;
+  float* oth = *oth_io;
+  GemmEpilogue e;
+  if (!s.attn_only) {
+    // out = LN2(z2), z2 = h1 + W2 gelu(u) + b2, u = W1 h1 + b1, h1 = LN1(z1), z1 = x + Wo ctx + bo
+    GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, s.dzb, mod.g + o.ln2g,
+                                mod.g + o.ln2b, mod.g + o.b2, red, T, d, st));         // oth, dzb = dz2; db2 += its column sums
+    GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st, "dw_ffn2"));
+    e = GemmEpilogue();
+    e.dgelu_pre = a.u;
+    e.tag = "dx_ffn2_dgelu";
+    const bool fused_b1 = gemm_fused_colsum(m->dtype, T, f);                           // the product's epilogue also adds up its columns
+    if (fused_b1) e.colsum_part = s.cpart;
+    GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(v), the saved u
+    if (fused_b1) GRAM_TRY(colsum_from_partials(ctx, s.cpart, (T + 31) / 32, f, mod.g + o.b1, red, st));
+    else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
+    GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st, "dw_ffn1"));
+    e = GemmEpilogue();
+    e.res = oth;
+    e.tag = "dx_ffn1";
+    GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, true, T, f, d, e, st));              // cur = dh1 = du W1 + dz2
+    GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, s.dzb, mod.g + o.ln1g,
+                                mod.g + o.ln1b, mod.g + o.bo, red, T, d, st));         // oth, dzb = dz1; dbo += its column sums
+  } else {
+    float* t = cur; cur = oth; oth = t;                                                // oth = d(out), dzb its copy
+    GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
+  }
+  GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st, "dw_attn_out"));
+  e = GemmEpilogue();
+  e.tag = "dx_attn_out";
+  GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.wo), s.dctx, false, T, d, d, e, st));
+  *cur_io = cur;
+  *oth_io = oth;
+  return GRAM_OK;
+}
+
+// Attention part over whole sequences.  s.dctx: gradient with respect to the attention output; oth: the residual
+// part of the gradient with respect to the layer's input.  Writes cur = dqkv Wqkv + oth, the gradient with respect
+// to the layer's input; copy_b: the layer below reads it as an operand as well (attention-only stacks).
+gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, const void* xb_l, int64_t n_seq, int S, float* cur,
+                                     const float* oth, bool copy_b, cudaStream_t st) {
+  const int64_t T = n_seq * S;
+  const int d = s.d;
+  gram_ctx* ctx = m->ctx;
+  const LayerOff& o = s.off[l];
+  LayerActs& a = s.acts[l];
+  const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
+                          (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
+  GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
+                              s.causal, st));
+  if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, m->red, st));
+  else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, m->red, st));
+  GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
+  GemmEpilogue e;
+  e.res = oth;
+  e.tag = "dx_qkv";
+  if (copy_b) e.copy_out = s.dzb;
+  return mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, true, T, 3 * d, d, e, st);          // cur = dx = dqkv Wqkv + dz1
+}
+
+// On entry s.curf holds the gradient with respect to the stack's output (fp32; for a stack of
+// attention-only layers s.dzb holds its operand-typed copy as well).  With top_attention_only the rows part of
+// the top layer has been done by the caller: s.dctx and s.othf hold what layer_rest_backward leaves, and the
+// top layer runs its attention part only.  On return *d_in points at the fp32 gradient with respect to the input
+// stream.
+gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, int64_t n_seq, int S, cudaStream_t st,
+                           float** d_in, bool top_attention_only = false) {
+  const int64_t T = n_seq * S;
   float* cur = s.curf;
   float* oth = s.othf;
   for (int l = s.n_layers - 1; l >= 0; --l) {
-    const LayerOff& o = s.off[l];
-    LayerActs& a = s.acts[l];
     const void* xb_l = (l == 0) ? x_in_b : s.acts[l - 1].out;
-    GemmEpilogue e;
-    if (!s.attn_only) {
-      // out = LN2(z2), z2 = h1 + W2 gelu(u) + b2, u = W1 h1 + b1, h1 = LN1(z1), z1 = x + Wo ctx + bo
-      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z2, a.mean2, a.rstd2, mod.w + o.ln2g, oth, s.dzb, mod.g + o.ln2g,
-                                  mod.g + o.ln2b, mod.g + o.b2, red, T, d, st));         // oth, dzb = dz2; db2 += its column sums
-      GRAM_TRY(mm_dw(m, s.dzb, a.g, mod.g + o.w2, T, d, f, st, "dw_ffn2"));
-      e = GemmEpilogue();
-      e.dgelu_pre = a.u;
-      e.tag = "dx_ffn2_dgelu";
-      const bool fused_b1 = gemm_fused_colsum(m->dtype, T, f);                           // the product's epilogue also adds up its columns
-      if (fused_b1) e.colsum_part = s.cpart;
-      GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.w2), s.du, false, T, d, f, e, st));           // du = (dz2 W2) * gelu'(v), the saved u
-      if (fused_b1) GRAM_TRY(colsum_from_partials(ctx, s.cpart, (T + 31) / 32, f, mod.g + o.b1, red, st));
-      else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.du, T, f, mod.g + o.b1, red, st));
-      GRAM_TRY(mm_dw(m, s.du, a.h1, mod.g + o.w1, T, f, d, st, "dw_ffn1"));
-      e = GemmEpilogue();
-      e.res = oth;
-      e.tag = "dx_ffn1";
-      GRAM_TRY(mm_dx(m, s.du, W(m, mod, o.w1), cur, true, T, f, d, e, st));              // cur = dh1 = du W1 + dz2
-      GRAM_TRY(layernorm_backward(ctx, m->dtype, cur, a.z1, a.mean1, a.rstd1, mod.w + o.ln1g, oth, s.dzb, mod.g + o.ln1g,
-                                  mod.g + o.ln1b, mod.g + o.bo, red, T, d, st));         // oth, dzb = dz1; dbo += its column sums
-    } else {
-      float* t = cur; cur = oth; oth = t;                                                // oth = d(out), dzb its copy
-      GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dzb, T, d, mod.g + o.bo, red, st));
-    }
-    GRAM_TRY(mm_dw(m, s.dzb, a.ctx, mod.g + o.wo, T, d, d, st, "dw_attn_out"));
-    e = GemmEpilogue();
-    e.tag = "dx_attn_out";
-    GRAM_TRY(mm_dx(m, s.dzb, W(m, mod, o.wo), s.dctx, false, T, d, d, e, st));
-    const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
-                            (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
-    GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
-                                s.causal, st));
-    if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, red, st));
-    else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, red, st));
-    GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
-    e = GemmEpilogue();
-    e.res = oth;
-    e.tag = "dx_qkv";
-    if (s.attn_only && l > 0) e.copy_out = s.dzb;                                        // the layer below reads it as an operand
-    GRAM_TRY(mm_dx(m, s.dqkv, W(m, mod, o.wqkv), cur, true, T, 3 * d, d, e, st));        // cur = dx = dqkv Wqkv + dz1
+    if (!(top_attention_only && l == s.n_layers - 1))
+      GRAM_TRY(layer_rest_backward(m, mod, s.off[l], s, s.acts[l], T, &cur, &oth, st));
+    GRAM_TRY(layer_attention_backward(m, mod, s, l, xb_l, n_seq, S, cur, oth, s.attn_only && l > 0, st));
   }
   *d_in = cur;
   return GRAM_OK;
@@ -406,8 +467,26 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   x0.z = m->z0; x0.mean = m->mean0; x0.rstd = m->rstd0; x0.gamma = m->ce.w + m->o_elng; x0.beta = m->ce.w + m->o_elnb;
   StreamRef out;
   const void* out_b = nullptr;
-  GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
-  GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, st));
+  if (!m->cls_tail) {
+    GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, st));
+  } else {
+    // all layers but the last, and the last layer's attention over whole sequences
+    const int last = c.n_layers - 1;
+    StreamRef x;
+    const void* xb = nullptr;
+    GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &x, &xb, last));
+    // row 0 of every item: the attention output and the last layer's input stream (values and LayerNorm statistics)
+    LayerActs& ta = m->tail.acts[0];
+    GRAM_TRY(take_strided_rows(ctx, m->enc.acts[last].ctx, n, c.l_t, c.d, (int)m->esz, ta.ctx, st));
+    GRAM_TRY(take_strided_rows(ctx, x.z, n, c.l_t, c.d, 4, m->tail_z, st));
+    GRAM_TRY(take_strided_rows(ctx, x.mean, n, c.l_t, 1, 4, m->tail_mean, st));
+    GRAM_TRY(take_strided_rows(ctx, x.rstd, n, c.l_t, 1, 4, m->tail_rstd, st));
+    StreamRef xr = x;
+    xr.z = m->tail_z; xr.mean = m->tail_mean; xr.rstd = m->tail_rstd;
+    GRAM_TRY(layer_rest_forward(m, m->ce, m->tail.off[0], ta, c.d, c.d_ff, 0, xr, ta.ctx, n, st, &out, &out_b));
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, 1, c.d, c.pooling, st));       // one row per item: the pooled row itself
+  }
   m->saved_n = n;
   return GRAM_OK;
 }
@@ -418,9 +497,24 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   gram_ctx* ctx = m->ctx;
   if (n != m->saved_n) return gram_set_error(ctx, "encoder backward over %d items, but activations of %d are saved", n, m->saved_n), GRAM_ERR_ARG;
   const int64_t T = (int64_t)n * c.l_t;
-  GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, st));
   float* dx0 = nullptr;
-  GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
+  if (!m->cls_tail) {
+    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, st));
+    GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
+  } else {
+    // the row-wise part of the last layer on one row per item
+    Stack& tl = m->tail;
+    GRAM_TRY(pool_backward(ctx, G, tl.curf, n, 1, c.d, c.pooling, st));
+    float* cur = tl.curf;
+    float* oth = tl.othf;
+    GRAM_TRY(layer_rest_backward(m, m->ce, tl.off[0], tl, tl.acts[0], n, &cur, &oth, st));
+    // back into whole sequences: every other row of the two gradients is zero
+    GRAM_CUDA(ctx, cudaMemsetAsync(m->enc.dctx, 0, (size_t)T * c.d * m->esz, st));
+    GRAM_CUDA(ctx, cudaMemsetAsync(m->enc.othf, 0, (size_t)T * c.d * 4, st));
+    GRAM_TRY(put_strided_rows(ctx, tl.dctx, n, c.l_t, c.d, (int)m->esz, m->enc.dctx, st));
+    GRAM_TRY(put_strided_rows(ctx, oth, n, c.l_t, c.d, 4, m->enc.othf, st));
+    GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0, true));
+  }
   float* dz0 = (dx0 == m->enc.curf) ? m->enc.othf : m->enc.curf;
   GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, nullptr,
                               m->ce.g + m->o_elng, m->ce.g + m->o_elnb, nullptr, m->red, T, c.d, st));
@@ -602,6 +696,13 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   m->mb = (int32_t)mb;
   m->enc.cap = (int64_t)m->mb * c.l_t;
   m->tk.cap = P;
+  m->cls_tail = c.n_layers > 0 && c.pooling == GRAM_POOL_CLS && c.l_t > 1;
+  if (m->cls_tail) {
+    m->tail.d = c.d; m->tail.heads = c.n_heads; m->tail.d_ff = c.d_ff; m->tail.n_layers = 1;
+    m->tail.attn_only = 0; m->tail.causal = 0;
+    m->tail.cap = m->mb;
+    m->tail.off.assign(1, m->enc.off.back());
+  }
   Arena dry;
   layout_buffers(m, dry);
   m->arena_bytes = dry.off + 256;
