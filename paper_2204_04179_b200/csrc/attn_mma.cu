@@ -19,6 +19,11 @@ __device__ __forceinline__ uint32_t pack2(float x, float y) {
   __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
   return *reinterpret_cast<uint32_t*>(&h);
 }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float quad_max(float v) {
   v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
   return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
@@ -75,8 +80,10 @@ __device__ __forceinline__ void load_a_trans(const bf16* S, int ld, int k0, int 
   ldsm_x4_trans(a0, a1, a2, a3, S + row * ld + col);
 }
 
-// scores of 16 query rows against all SP keys: p[nt][0..3] for key tile nt, normalised probabilities on return
-template <int SP, int DH>
+// scores of 16 query rows against all SP keys: p[nt][0..3] for key tile nt, normalised probabilities on return.
+// MASK = false: every key is visible to every row (S == SP, no causal mask), the per-element tests are left out.
+// The 1/sqrt(dh) scale is folded into the exponent: exp(scale (s - max s)) = exp2(c s - c max s), c = scale log2(e).
+template <int SP, int DH, bool MASK>
 __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf16* __restrict__ Ks, int r0, int S, int causal,
                                            float scale, int g, int q, float (&p)[SP / 8][4]) {
   constexpr int LD = DH + 8;
@@ -99,12 +106,14 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
   for (int nt = 0; nt < SP / 8; ++nt) {
+    if (MASK) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int j = nt * 8 + 2 * q + (e & 1);
-      const int i = (e < 2) ? i0 : i1;
-      const bool ok = j < S && (!causal || j <= i);
-      p[nt][e] = ok ? p[nt][e] * scale : -INFINITY;
+      for (int e = 0; e < 4; ++e) {
+        const int j = nt * 8 + 2 * q + (e & 1);
+        const int i = (e < 2) ? i0 : i1;
+        const bool ok = j < S && (!causal || j <= i);
+        if (!ok) p[nt][e] = -INFINITY;
+      }
     }
     m0 = fmaxf(m0, fmaxf(p[nt][0], p[nt][1]));
     m1 = fmaxf(m1, fmaxf(p[nt][2], p[nt][3]));
@@ -113,11 +122,13 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
   m1 = quad_max(m1);
   if (m0 == -INFINITY) m0 = 0.f;        // no key is visible to this (padded) row
   if (m1 == -INFINITY) m1 = 0.f;
+  const float c = scale * 1.4426950408889634f;
+  const float mc0 = m0 * c, mc1 = m1 * c;
   float l0 = 0.f, l1 = 0.f;
 #pragma unroll
   for (int nt = 0; nt < SP / 8; ++nt) {
-    p[nt][0] = __expf(p[nt][0] - m0); p[nt][1] = __expf(p[nt][1] - m0);
-    p[nt][2] = __expf(p[nt][2] - m1); p[nt][3] = __expf(p[nt][3] - m1);
+    p[nt][0] = fast_exp2(fmaf(p[nt][0], c, -mc0)); p[nt][1] = fast_exp2(fmaf(p[nt][1], c, -mc0));
+    p[nt][2] = fast_exp2(fmaf(p[nt][2], c, -mc1)); p[nt][3] = fast_exp2(fmaf(p[nt][3], c, -mc1));
     l0 += p[nt][0] + p[nt][1];
     l1 += p[nt][2] + p[nt][3];
   }
@@ -212,7 +223,8 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   bf16* ob = out + seq * S * (int64_t)d + h * DH;
   for (int r0 = warp * 16; r0 < S; r0 += 64) {
     float p[SP / 8][4];
-    score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
+    if (S == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, S, causal, scale, g, q, p);
+    else score_rows<SP, DH, true>(Qs, Ks, r0, S, causal, scale, g, q, p);
     float o[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
@@ -255,7 +267,8 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
     const int r0 = warp * 16 + it * 64;
     if (r0 < SP) {
       float p[SP / 8][4];
-      score_rows<SP, DH>(Qs, Ks, r0, S, causal, scale, g, q, p);
+      if (S == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, S, causal, scale, g, q, p);
+      else score_rows<SP, DH, true>(Qs, Ks, r0, S, causal, scale, g, q, p);
       float dp[SP / 8][4];
 #pragma unroll
       for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
