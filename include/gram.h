@@ -139,6 +139,13 @@ gram_status gram_optimizer_step(gram_ctx* ctx, int module, gram_stream stream);
 gram_status gram_optimizer_reset(gram_ctx* ctx, gram_stream stream);
 /* Token IDs c_i of every item (Table 1), int32 [n_items, l_t], copied to the device. */
 gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens);
+/* Texts of different lengths (Table 3 lists 5 to 271 tokens per item; Appendix D pads or truncates to a maximum):
+ * h_lengths int32 [n_items], item i's text is its first h_lengths[i] tokens (1 .. l_t), the remaining slots of its
+ * row of h_tokens are padding whose values are never used.  The encoder then attends over the text tokens only and
+ * mean pooling averages over them; an item encodes exactly as it would in a model whose l_t is its own length.
+ * Padding slots are still computed (storage stays [n_items, l_t]); their outputs are never read and their gradients
+ * are zero.  NULL restores texts of exactly l_t tokens (the state after gram_create). */
+gram_status gram_set_item_lengths(gram_ctx* ctx, const int32_t* h_lengths);
 
 /* --- the five stages (Algorithm 1; Fig. 1) -------------------------------- */
 

@@ -193,9 +193,11 @@ def transformer_layer(x, th, pre, n_heads, causal, attn_only=False):
 
 
 def ce_forward(th: Dict[str, torch.Tensor], tokens, shape) -> torch.Tensor:
-    """h = CE(c; theta_CE) for ONE item: tokens [l_t] -> encoding [d]."""
+    """h = CE(c; theta_CE) for ONE item: tokens [n] -> encoding [d], n <= l_t.  A text shorter than l_t is simply a
+    shorter sequence (positions 0..n-1): no padding exists on this side, so attention and pooling range over the
+    text alone (Section 3.2: c_i is the item's own token sequence; Table 3: lengths vary from item to item)."""
     tok = torch.as_tensor(np.asarray(tokens), dtype=torch.long)
-    x = th["tok_emb"][tok] + th["pos_emb"]
+    x = th["tok_emb"][tok] + th["pos_emb"][:tok.shape[0]]
     x = layer_norm(x, th["emb_ln_g"], th["emb_ln_b"])
     for l in range(shape.n_layers):
         x = transformer_layer(x, th, f"l{l}.", shape.n_heads, causal=False)

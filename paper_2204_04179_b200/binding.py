@@ -27,7 +27,8 @@ STATUS = {0: "GRAM_OK", 1: "GRAM_ERR_ARG", 2: "GRAM_ERR_ID_RANGE", 3: "GRAM_ERR_
 
 # every symbol include/gram.h declares
 SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_param_count", "gram_set_params",
-           "gram_get_params", "gram_get_grads", "gram_zero_grads", "gram_set_item_tokens", "gram_dedup",
+           "gram_get_params", "gram_get_grads", "gram_zero_grads", "gram_set_item_tokens", "gram_set_item_lengths",
+           "gram_dedup",
            "gram_encode_unique", "gram_gather", "gram_accumulate", "gram_accumulate_multistep", "gram_touched_list",
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
@@ -190,6 +191,14 @@ class Gram:
     def set_item_tokens(self, tokens: np.ndarray):
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)
         self._ck(lib().gram_set_item_tokens(self._h, _ptr(tokens)))
+
+    def set_item_lengths(self, lengths: Optional[np.ndarray]):
+        if lengths is None:
+            self._ck(lib().gram_set_item_lengths(self._h, C.c_void_p(0)))
+            return
+        lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+        assert lengths.size == self.cfg.n_items
+        self._ck(lib().gram_set_item_lengths(self._h, _ptr(lengths)))
 
     # stages
     def dedup(self, ids, n_items, unique, inverse, perm, seg_off, n_unique, stream=None):

@@ -323,6 +323,10 @@ gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens) {
   NEED_MODEL("gram_set_item_tokens");
   return model_set_item_tokens(ctx->model, h_tokens);
 }
+gram_status gram_set_item_lengths(gram_ctx* ctx, const int32_t* h_lengths) {
+  NEED_MODEL("gram_set_item_lengths");
+  return model_set_item_lengths(ctx->model, h_lengths);
+}
 gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
                                float* d_H, int save_activations, gram_stream stream) {
   NEED_MODEL("gram_encode_unique");

@@ -206,7 +206,8 @@ __device__ __forceinline__ void mma_regs_times_rows(const float (&x)[SP / 8][4],
 
 template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
-                                                           int n_heads, int causal, float scale) {
+                                                           int n_heads, int causal, float scale,
+                                                           const int32_t* __restrict__ seq_len) {
   constexpr int LD = DH + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
@@ -221,10 +222,11 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   bf16* ob = out + seq * S * (int64_t)d + h * DH;
+  const int Sv = seq_len ? seq_len[seq] : S;      // keys that are text; the rows after them are padding
   for (int r0 = warp * 16; r0 < S; r0 += 64) {
     float p[SP / 8][4];
-    if (S == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, S, causal, scale, g, q, p);
-    else score_rows<SP, DH, true>(Qs, Ks, r0, S, causal, scale, g, q, p);
+    if (Sv == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+    else score_rows<SP, DH, true>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
     float o[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
@@ -240,7 +242,8 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
 template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
                                                            bf16* __restrict__ dqkv, float* __restrict__ colpart, int S, int d,
-                                                           int n_heads, int causal, float scale) {
+                                                           int n_heads, int causal, float scale,
+                                                           const int32_t* __restrict__ seq_len) {
   constexpr int LD = DH + 8, LP = SP + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // [SP][DH+8]
@@ -259,6 +262,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   bf16* dq = dqkv + seq * S * 3 * (int64_t)d + h * DH;
+  const int Sv = seq_len ? seq_len[seq] : S;
   // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ (kept in registers as bf16 pairs) ----
   constexpr int NIT = (SP + 63) / 64;
   uint32_t dqp[NIT][DH / 8][2];
@@ -267,8 +271,8 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
     const int r0 = warp * 16 + it * 64;
     if (r0 < SP) {
       float p[SP / 8][4];
-      if (S == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, S, causal, scale, g, q, p);
-      else score_rows<SP, DH, true>(Qs, Ks, r0, S, causal, scale, g, q, p);
+      if (Sv == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+      else score_rows<SP, DH, true>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
       float dp[SP / 8][4];
 #pragma unroll
       for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
@@ -374,22 +378,22 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
 
 template <int SP, int DH>
 gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
-                       cudaStream_t st) {
+                       const int32_t* seq_len, cudaStream_t st) {
   constexpr size_t smem = (size_t)3 * SP * (DH + 8) * 2;
   auto kern = attn_fwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 template <int SP, int DH>
 gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                       int n_heads, int causal, cudaStream_t st) {
+                       int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
   constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
   auto kern = attn_bwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH));
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -418,10 +422,10 @@ bool attention_mma_supported(int S, int d, int n_heads) {
   } while (0)
 
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, cudaStream_t st) {
-  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, st);
+                                  int causal, const int32_t* seq_len, cudaStream_t st) {
+  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, seq_len, st);
 }
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq,
-                                   int S, int d, int n_heads, int causal, cudaStream_t st) {
-  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, st);
+                                   int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
+  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, st);
 }

@@ -33,7 +33,8 @@ __device__ __forceinline__ float warp_max(float v) {
 __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const int32_t* __restrict__ items,
                                  int32_t first_item, int64_t n_tok, int32_t n_items_total, int l_t, int vocab, int d,
                                  const float* __restrict__ tok_emb, const float* __restrict__ pos_emb,
-                                 float* __restrict__ z0, int32_t* __restrict__ tok_ids, int32_t* status) {
+                                 float* __restrict__ z0, int32_t* __restrict__ tok_ids,
+                                 const int32_t* __restrict__ item_len, int32_t* __restrict__ seq_len, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -45,6 +46,10 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const 
     int32_t tok = item_tokens[(int64_t)item * l_t + s];
     if (tok < 0 || tok >= vocab) { gram_device_fail(status, GRAM_ERR_ID_RANGE); tok = 0; }
     if (lane == 0) tok_ids[t] = tok;
+    if (seq_len && s == 0 && lane == 0) {        // tokens of this item that are text, the rest is padding
+      int32_t n = item_len[item];
+      seq_len[u] = n < 1 ? 1 : (n > l_t ? l_t : n);
+    }
     const float* te = tok_emb + (int64_t)tok * d;
     const float* pe = pos_emb + (int64_t)s * d;
     for (int c = 2 * lane; c < d; c += 64) {
@@ -228,7 +233,8 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float* __res
 // stride; a warp owns one query row at a time, with keys spread over lanes (S <= 128).
 template <typename T>
 __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out, int S, int d,
-                                                       int n_heads, int causal, float scale) {
+                                                       int n_heads, int causal, float scale,
+                                                       const int32_t* __restrict__ seq_len) {
   extern __shared__ float sm[];
   const int dh = d / n_heads, ld = dh + 1;
   float* Q = sm;
@@ -236,6 +242,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
   float* V = K + S * ld;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
+  const int Sv = seq_len ? seq_len[seq] : S;          // keys that are text; rows past them are padding
   const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
   for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
     const int s = i / dh, c = i - s * dh;
@@ -253,7 +260,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
     for (int jj = 0; jj < 4; ++jj) {
       const int j = lane + 32 * jj;
       float sc = -INFINITY;
-      if (j < S && (!causal || j <= i)) {
+      if (j < Sv && (!causal || j <= i)) {
         float acc = 0.f;
         for (int c = 0; c < dh; ++c) acc += Q[i * ld + c] * K[j * ld + c];
         sc = acc * scale;
@@ -270,7 +277,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
     }
     l = warp_sum(l);
     const float inv = 1.f / l;
-    const int jmax = causal ? i + 1 : S;
+    const int jmax = min(causal ? i + 1 : S, Sv);
     float o0 = 0.f, o1 = 0.f;      // columns lane and lane + 32 (dh <= 64)
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
@@ -291,7 +298,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
 template <typename T>
 __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dctx,
                                                        T* __restrict__ dqkv, int S, int d, int n_heads, int causal,
-                                                       float scale) {
+                                                       float scale, const int32_t* __restrict__ seq_len) {
   extern __shared__ float sm[];
   const int dh = d / n_heads, ld = dh + 1, lp = S + 1;
   float* Q = sm;
@@ -304,6 +311,7 @@ __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv
   const int h = blockIdx.x % n_heads;
   const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
   const T* dbase = dctx + seq * S * (int64_t)d + h * dh;
+  const int Sv = seq_len ? seq_len[seq] : S;
   for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
     const int s = i / dh, c = i - s * dh;
     const T* p = base + (int64_t)s * 3 * d + c;
@@ -323,7 +331,7 @@ __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv
     for (int jj = 0; jj < 4; ++jj) {
       const int j = lane + 32 * jj;
       float sc = -INFINITY, g = 0.f;
-      if (j < S && (!causal || j <= i)) {
+      if (j < Sv && (!causal || j <= i)) {
         float acc = 0.f;
         for (int c = 0; c < dh; ++c) {
           acc += Q[i * ld + c] * K[j * ld + c];
@@ -361,7 +369,7 @@ __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv
         dS[i * lp + j] = ds[jj];
       }
     }
-    const int jmax = causal ? i + 1 : S;
+    const int jmax = min(causal ? i + 1 : S, Sv);
     float o0 = 0.f, o1 = 0.f;
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
@@ -437,7 +445,8 @@ __device__ __forceinline__ float stream_at(const StreamRef& x, int64_t row, int 
   if (x.mean) v = (v - x.mean[row]) * x.rstd[row] * x.gamma[c] + x.beta[c];
   return v;
 }
-__global__ void pool_fwd_kernel(StreamRef x, float* __restrict__ H, int64_t n, int l_t, int d, int pooling) {
+__global__ void pool_fwd_kernel(StreamRef x, float* __restrict__ H, int64_t n, int l_t, int d, int pooling,
+                                const int32_t* __restrict__ seq_len) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * d) return;
   const int64_t u = i / d;
@@ -445,12 +454,14 @@ __global__ void pool_fwd_kernel(StreamRef x, float* __restrict__ H, int64_t n, i
   if (pooling == GRAM_POOL_CLS) {
     H[i] = stream_at(x, u * l_t, c, d);
   } else {
+    const int len = seq_len ? seq_len[u] : l_t;      // mean over the tokens that are text
     float acc = 0.f;
-    for (int s = 0; s < l_t; ++s) acc += stream_at(x, u * l_t + s, c, d);
-    H[i] = acc / l_t;
+    for (int s = 0; s < len; ++s) acc += stream_at(x, u * l_t + s, c, d);
+    H[i] = acc / len;
   }
 }
-__global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__ dx, int64_t n, int l_t, int d, int pooling) {
+__global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__ dx, int64_t n, int l_t, int d, int pooling,
+                                const int32_t* __restrict__ seq_len) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * l_t * d) return;
   const int64_t t = i / d;
@@ -459,7 +470,10 @@ __global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__
   const int s = (int)(t - u * l_t);
   float v;
   if (pooling == GRAM_POOL_CLS) v = (s == 0) ? G[u * d + c] : 0.f;
-  else v = G[u * d + c] / l_t;
+  else {
+    const int len = seq_len ? seq_len[u] : l_t;
+    v = s < len ? G[u * d + c] / len : 0.f;
+  }
   dx[i] = v;
 }
 
@@ -723,13 +737,14 @@ template <typename F> gram_status set_smem(gram_ctx* ctx, F kern, size_t bytes) 
 
 gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, float* z0, int32_t* tok_ids, cudaStream_t st) {
+                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* item_len, int32_t* seq_len,
+                          cudaStream_t st) {
   const int64_t n_tok = (int64_t)n_chunk * l_t;
   if (n_tok == 0) return GRAM_OK;
   const int blocks = grid_for(n_tok * 32, 256, kNumSMs * 8);
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 8.0 * (double)n_tok * d, 1, st);
   embed_fwd_kernel<<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t, vocab, d, tok_emb,
-                                           pos_emb, z0, tok_ids, gram_status_word(ctx));
+                                           pos_emb, z0, tok_ids, item_len, item_len ? seq_len : nullptr, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -764,7 +779,7 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 }
 
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, cudaStream_t st) {
+                              int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
@@ -772,17 +787,17 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_fwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, st);
+    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
-    attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale);
+    attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale, seq_len);
   });
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, cudaStream_t st) {
+                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
@@ -790,11 +805,11 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, st);
+    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, st);
   if (colpart) return gram_set_error(ctx, "attention: fused column sums need the tensor-core kernel"), GRAM_ERR_UNSUPPORTED;
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
-    attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale);
+    attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale, seq_len);
   });
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -864,19 +879,19 @@ gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_
 }
 
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
-                         cudaStream_t st) {
+                         const int32_t* seq_len, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (pooling == GRAM_POOL_CLS ? 2 : l_t + 1), 1, st);
-  pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling);
+  pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling, seq_len);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
-                          cudaStream_t st) {
+                          const int32_t* seq_len, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (l_t + 1), 1, st);
-  pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling);
+  pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling, seq_len);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

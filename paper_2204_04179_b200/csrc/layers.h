@@ -19,10 +19,12 @@ struct StreamRef {
 };
 
 // z0[t, :] = tok_emb[token(t), :] + pos_emb[t % l_t, :] (fp32), token(t) = item_tokens[items[t / l_t], t % l_t];
-// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.
+// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.  item_len (may be null): tokens of each
+// item that are text (the rest of its l_t slots is padding); seq_len[u] then receives the length of chunk item u.
 gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_items_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, float* z0, int32_t* tok_ids, cudaStream_t st);
+                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* item_len, int32_t* seq_len,
+                          cudaStream_t st);
 
 // y = LayerNorm(z): z is the fp32 stream, y the operand-typed copy the next matrix product reads
 gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
@@ -34,20 +36,22 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
                                const float* rstd, const float* gamma, float* dz, void* dz_b, float* dgamma,
                                float* dbeta, float* dcol, float* scratch, int64_t rows, int d, cudaStream_t st);
 
-// softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d]
+// softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d].
+// seq_len (may be null): only the first seq_len[s] rows of sequence s are keys; the rows after them are padding,
+// whose outputs are finite and never read, and whose gradients are zero.
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, cudaStream_t st);
+                              int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
 // colpart (may be null; only where attention_mma_supported and dtype is bf16): fp32 [n_seq, 3d], row s receives the
 // column sums of sequence s's rows of dqkv, the partial sums of the bias gradient of the Q, K, V projection
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, cudaStream_t st);
+                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
 
 // the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
 bool attention_mma_supported(int S, int d, int n_heads);
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, cudaStream_t st);
+                                  int causal, const int32_t* seq_len, cudaStream_t st);
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                                   int n_heads, int causal, cudaStream_t st);
+                                   int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
 
 // out[n] += sum_rows X[r, n]   (X operand-typed)
 // out[c] += sum over the nrows rows of part[., c] (fp32 [nrows, N]; partial column sums left by a fused producer)
@@ -59,12 +63,12 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
 gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
                                        cudaStream_t st);
 
-// H[u, :] = mean_s x[u*l_t + s, :] (mean) or x[u*l_t, :] (cls), fp32
+// H[u, :] = mean_s x[u*l_t + s, :] (mean; over the first seq_len[u] tokens when seq_len is given) or x[u*l_t, :] (cls), fp32
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
-                         cudaStream_t st);
+                         const int32_t* seq_len, cudaStream_t st);
 // dx[u*l_t + s, :] from G[u, :] (both fp32)
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
-                          cudaStream_t st);
+                          const int32_t* seq_len, cudaStream_t st);
 
 // knowledge-tracing task input: x[b, n, :] = E[b, n, :] + pos[n, :] + resp[prev(b, n), :] (fp32, and an
 // operand-typed copy x_b), prev(b, 0) = 2, prev(b, n) = labels[b, n-1]

@@ -36,6 +36,7 @@ struct LayerActs {
 struct Stack {
   int d = 0, heads = 0, d_ff = 0, n_layers = 0, attn_only = 0, causal = 0;
   int64_t cap = 0;                         // tokens the buffers hold
+  const int32_t* seq_len = nullptr;        // per sequence: rows that are text (null: all S); set per pass
   std::vector<LayerOff> off;
   std::vector<LayerActs> acts;
   // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
@@ -96,6 +97,9 @@ struct Model {
   float *mean0 = nullptr, *rstd0 = nullptr;
   int32_t *tok_ids = nullptr, *tok_unique = nullptr, *tok_inverse = nullptr, *tok_perm = nullptr, *tok_seg = nullptr,
           *tok_nu = nullptr;
+  int32_t* item_len = nullptr;       // [n_items] tokens of each item that are text (variable-length texts), else null
+  int32_t* item_len_buf = nullptr;   // its storage
+  int32_t* seq_len = nullptr;        // [mb] the same for the items of the current encoder pass
   int32_t mb = 0;                    // items per encoder pass
   int32_t saved_n = -1;              // items whose activations the last encoder pass saved (-1: none)
   // task
@@ -185,6 +189,8 @@ void layout_buffers(Model* m, Arena& a) {
     m->tok_perm = (int32_t*)a.take(T * 4);
     m->tok_seg = (int32_t*)a.take((tu + 1) * 4);
     m->tok_nu = (int32_t*)a.take(4);
+    m->item_len_buf = (int32_t*)a.take((size_t)c.n_items * 4);
+    m->seq_len = (int32_t*)a.take((size_t)m->mb * 4);
     stack_buffers(a, m->enc, esz);
     if (m->cls_tail) {
       stack_buffers(a, m->tail, esz);
@@ -299,7 +305,7 @@ gram_status layer_attention_forward(Model* m, Module& mod, Stack& s, int l, cons
   e.bias = mod.w + o.bqkv;
   e.tag = "fwd_qkv";
   GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * s.d, s.d, e, st));
-  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, st);
+  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, st);
 }
 
 // the row-wise rest of the layer over T rows: output projection + residual, LayerNorm, feed-forward + residual,
@@ -420,7 +426,7 @@ gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, con
   const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
                           (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
   GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
-                              s.causal, st));
+                              s.causal, s.seq_len, st));
   if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, m->red, st));
   else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, m->red, st));
   GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
@@ -460,7 +466,9 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   GRAM_TRY(refresh_bf16(m, m->ce, st));
   const int64_t T = (int64_t)n * c.l_t;
   GRAM_TRY(embed_forward(ctx, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items, c.l_t,
-                         c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, st));
+                         c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, m->item_len, m->seq_len, st));
+  const int32_t* seq_len = m->item_len ? m->seq_len : nullptr;
+  m->enc.seq_len = seq_len;
   GRAM_TRY(layernorm_forward(ctx, m->dtype, m->z0, m->ce.w + m->o_elng, m->ce.w + m->o_elnb, m->x0, m->mean0, m->rstd0, T,
                              c.d, st));
   StreamRef x0;
@@ -469,7 +477,7 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   const void* out_b = nullptr;
   if (!m->cls_tail) {
     GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
-    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, st));
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, seq_len, st));
   } else {
     // all layers but the last, and the last layer's attention over whole sequences
     const int last = c.n_layers - 1;
@@ -485,7 +493,7 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
     StreamRef xr = x;
     xr.z = m->tail_z; xr.mean = m->tail_mean; xr.rstd = m->tail_rstd;
     GRAM_TRY(layer_rest_forward(m, m->ce, m->tail.off[0], ta, c.d, c.d_ff, 0, xr, ta.ctx, n, st, &out, &out_b));
-    GRAM_TRY(pool_forward(ctx, out, H_out, n, 1, c.d, c.pooling, st));       // one row per item: the pooled row itself
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, 1, c.d, c.pooling, nullptr, st));       // one row per item: the pooled row itself
   }
   m->saved_n = n;
   return GRAM_OK;
@@ -499,12 +507,12 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   const int64_t T = (int64_t)n * c.l_t;
   float* dx0 = nullptr;
   if (!m->cls_tail) {
-    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, st));
+    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, m->enc.seq_len, st));
     GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
   } else {
     // the row-wise part of the last layer on one row per item
     Stack& tl = m->tail;
-    GRAM_TRY(pool_backward(ctx, G, tl.curf, n, 1, c.d, c.pooling, st));
+    GRAM_TRY(pool_backward(ctx, G, tl.curf, n, 1, c.d, c.pooling, nullptr, st));
     float* cur = tl.curf;
     float* oth = tl.othf;
     GRAM_TRY(layer_rest_backward(m, m->ce, tl.off[0], tl, tl.acts[0], n, &cur, &oth, st));
@@ -766,6 +774,22 @@ gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens) {
   if (!h_tokens || !m->item_tokens) return gram_set_error(m->ctx, "gram_set_item_tokens: no encoder or null tokens"), GRAM_ERR_ARG;
   GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
   GRAM_CUDA(m->ctx, cudaMemcpy(m->item_tokens, h_tokens, (size_t)m->cfg.n_items * m->cfg.l_t * 4, cudaMemcpyHostToDevice));
+  return GRAM_OK;
+}
+
+gram_status model_set_item_lengths(Model* m, const int32_t* h_len) {
+  if (!m->item_len_buf) return gram_set_error(m->ctx, "gram_set_item_lengths: the context has no encoder"), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  m->saved_n = -1;
+  if (!h_len) {                         // back to texts of exactly l_t tokens
+    m->item_len = nullptr;
+    return GRAM_OK;
+  }
+  for (int32_t i = 0; i < m->cfg.n_items; ++i)
+    if (h_len[i] < 1 || h_len[i] > m->cfg.l_t)
+      return gram_set_error(m->ctx, "gram_set_item_lengths: item %d has length %d outside 1..%d", i, h_len[i], m->cfg.l_t), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaMemcpy(m->item_len_buf, h_len, (size_t)m->cfg.n_items * 4, cudaMemcpyHostToDevice));
+  m->item_len = m->item_len_buf;
   return GRAM_OK;
 }
 

@@ -17,6 +17,7 @@ gram_status model_optimizer_step(Model* m, int module, cudaStream_t st);
 gram_status model_optimizer_reset(Model* m, cudaStream_t st);
 double noam_rate(int64_t t, double peak, int warmup);
 gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens);
+gram_status model_set_item_lengths(Model* m, const int32_t* h_len);
 gram_status model_encode(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U, float* d_H,
                          int save, cudaStream_t st);
 gram_status model_task(Model* m, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE, float* d_loss,

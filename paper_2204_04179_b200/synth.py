@@ -108,6 +108,21 @@ def item_tokens(seed: int, n_items: int, l_t: int, vocab: int) -> np.ndarray:
     return _rng(seed, _S_TOKENS).integers(0, vocab, size=(n_items, l_t), dtype=np.int32)
 
 
+def item_lengths(seed: int, n_items: int, l_t: int, shortest: int = 1) -> np.ndarray:
+    """Text lengths for variable-length items, uniform over shortest..l_t: int32 [n_items] (the paper's texts run
+    from 5 to 271 tokens, Table 3); at least one item gets the full l_t and one the shortest length."""
+    n = _rng(seed, _S_TOKENS + 7).integers(shortest, l_t + 1, size=n_items, dtype=np.int32)
+    n[0] = l_t
+    if n_items > 1:
+        n[1] = shortest
+    return n
+
+
+def ragged(tokens: np.ndarray, lengths: np.ndarray):
+    """The texts without their padding: a list of int32 arrays, item i holding its first lengths[i] tokens."""
+    return [np.asarray(tokens[i, :int(lengths[i])]) for i in range(tokens.shape[0])]
+
+
 def labels(seed: int, B: int, L: int, p: float, step: int = 0) -> np.ndarray:
     """Bernoulli(p) responses, int32 [B, L]."""
     return (_rng(seed, _S_LABELS + 1000 * step).random((B, L)) < p).astype(np.int32)

@@ -260,3 +260,55 @@ def test_multistep_pseudo_target_first_window_bf16():
     print("bf16 pseudo-target worst CE", e1, n1, "worst task", e2, n2)
     assert e1 <= 2e-2 and e2 <= 2e-2, (e1, n1, e2, n2)
     g.close()
+
+
+VARLEN = {
+    "f32_mean": small(l_t=9, pooling="mean"),
+    "f32_cls_full_task": small(l_t=9, pooling="cls", task_attn_only=False, task_layers=2),
+    "f32_nr": small(task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls", l_t=7),
+    # tensor-core attention: texts of 1..40 tokens in a 64-row tile, and 1..70 in a 96-row tile
+    "bf16_mean_40": small(dtype="bf16", l_t=40, d=64, n_heads=2, d_ff=128, task_d_ff=128, n_items=30, pooling="mean"),
+    "bf16_cls_70": small(dtype="bf16", l_t=70, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30, pooling="cls", B=2),
+}
+
+
+@pytest.mark.parametrize("name", list(VARLEN))
+def test_texts_of_different_lengths(name):
+    """gram_set_item_lengths: padded storage on the device, plain shorter sequences in the oracle."""
+    shape = VARLEN[name]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=31)
+    lengths = synth.item_lengths(31, shape.n_items, shape.l_t)
+    assert lengths.min() == 1 and lengths.max() == shape.l_t
+    want = orc.e2e_step(shape, ce, tk, synth.ragged(toks, lengths), ids, lab)
+    junk = toks.copy()
+    for i, n in enumerate(lengths):                       # whatever sits in the padding slots must not matter
+        junk[i, n:] = (junk[i, n:] * 7 + 3) % shape.vocab
+    tol = TOL[shape.dtype]
+    results = []
+    for tokens in (toks, junk):
+        g = gh.make_ctx(shape, ce, tk, tokens)
+        g.set_item_lengths(lengths)
+        rep = g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)
+        gce, gtk = gh.gpu_grads(g, shape)
+        g.close()
+        assert abs(rep.loss - want["loss"]) <= tol * abs(want["loss"])
+        e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+        e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+        print(name, "worst CE", e1, n1, "worst task", e2, n2)
+        assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+        results.append((rep.loss, gce))
+    assert results[0][0] == results[1][0]
+    for k in results[0][1]:
+        if k != "tok_emb":                                # the padding tokens' embedding rows receive exact zeros either way
+            assert np.array_equal(results[0][1][k], results[1][1][k]), k
+    # back to fixed-length texts
+    g = gh.make_ctx(shape, ce, tk, toks)
+    g.set_item_lengths(lengths)
+    g.set_item_lengths(None)
+    rep = g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)
+    full = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    assert abs(rep.loss - full["loss"]) <= tol * abs(full["loss"])
+    with pytest.raises(binding.GramError):
+        bad = lengths.copy(); bad[3] = shape.l_t + 1
+        g.set_item_lengths(bad)
+    g.close()

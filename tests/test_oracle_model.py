@@ -329,3 +329,47 @@ def test_pseudo_target_gradient_with_a_stale_cache_matches_finite_differences():
     plain = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0)
     assert max(np.abs(plain["grad_ce"][k] - got["grad_ce"][k]).max() for k in ce) > 1e-4
     np.testing.assert_allclose(got["cache"][items], orc.encode_all(shape, ce, toks, items), rtol=1e-13)
+
+
+# ---- texts of different lengths (Table 3: 5 to 271 tokens per item) ---------------------------------------------------
+
+def test_short_text_equals_library_layer_with_padding_mask():
+    # the oracle encodes a short text as a short sequence; a padded sequence run through torch's own encoder layer
+    # with a key-padding mask must give the same rows for the text tokens
+    d, heads, dff, n, l_t = 16, 4, 24, 5, 9
+    p = synth._draw_params(synth._layer_spec("x.", d, dff, False), np.random.default_rng(5), 0.4, False)
+    th = orc.as_torch(p, T64, requires_grad=False)
+    lib = torch.nn.TransformerEncoderLayer(d, heads, dff, dropout=0.0, activation="gelu", layer_norm_eps=orc.LN_EPS,
+                                           batch_first=True, norm_first=False, dtype=T64)
+    with torch.no_grad():
+        lib.self_attn.in_proj_weight.copy_(th["x.wqkv"]); lib.self_attn.in_proj_bias.copy_(th["x.bqkv"])
+        lib.self_attn.out_proj.weight.copy_(th["x.wo"]); lib.self_attn.out_proj.bias.copy_(th["x.bo"])
+        lib.linear1.weight.copy_(th["x.w1"]); lib.linear1.bias.copy_(th["x.b1"])
+        lib.linear2.weight.copy_(th["x.w2"]); lib.linear2.bias.copy_(th["x.b2"])
+        lib.norm1.weight.copy_(th["x.ln1_g"]); lib.norm1.bias.copy_(th["x.ln1_b"])
+        lib.norm2.weight.copy_(th["x.ln2_g"]); lib.norm2.bias.copy_(th["x.ln2_b"])
+    lib.train()
+    x = torch.randn(l_t, d, dtype=T64, generator=torch.Generator().manual_seed(4))      # rows n.. play the padding
+    pad = torch.zeros(1, l_t, dtype=torch.bool); pad[0, n:] = True
+    with torch.no_grad():
+        want = lib(x[None], src_key_padding_mask=pad)[0, :n]
+        got = orc.transformer_layer(x[:n], th, "x.", heads, causal=False)
+    np.testing.assert_allclose(got.numpy(), want.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_short_text_encoding_ignores_what_follows_it():
+    shape = small_shape(l_t=6, pooling="mean")
+    ce, tk, toks, ids, lab = make(shape, seed=9)
+    th = orc.as_torch(ce, T64, requires_grad=False)
+    with torch.no_grad():
+        a = orc.ce_forward(th, toks[0][:4], shape)
+        other = toks[0].copy(); other[4:] = (other[4:] + 1) % shape.vocab
+        b = orc.ce_forward(th, other[:4], shape)
+        full = orc.ce_forward(th, toks[0], shape)
+    assert torch.equal(a, b) and not torch.allclose(a, full)
+    # mean pooling is over the text tokens: a one-token text pools to that token's own output row
+    one = orc.ce_forward(th, toks[0][:1], shape)
+    x = orc.layer_norm(th["tok_emb"][int(toks[0][0])] + th["pos_emb"][0], th["emb_ln_g"], th["emb_ln_b"])[None]
+    for l in range(shape.n_layers):
+        x = orc.transformer_layer(x, th, f"l{l}.", shape.n_heads, causal=False)
+    np.testing.assert_allclose(one.numpy(), x[0].numpy(), rtol=1e-13)
