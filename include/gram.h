@@ -235,6 +235,22 @@ gram_status gram_window_reset(gram_ctx* ctx, gram_stream stream);
  * [ceil(n_items/32)], cache fp32 [n_items, d] (converted).  NULL skips one. */
 gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache);
 
+/* --- checkpoint / resume (the paper keeps the checkpoint of the best validation epoch, Section A) ------------------
+ * Everything a context holds besides what the caller gave it: parameters (gram_get_params / gram_set_params), the
+ * optimiser's state, and for K > 1 the open window.  Exported by one context and imported into another context of the
+ * same configuration, training continues bit for bit.  All calls synchronise. */
+/* Multi-step: gram_get_window plus the number of steps already taken in the open window (0 .. K-1). */
+gram_status gram_state_export(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache, int32_t* steps_in_window);
+/* Multi-step: the reverse.  Arrays as in gram_get_window (NULL leaves that part as it is); the cache is rounded to the
+ * context's cache type (bf16 contexts with GRAM_MULTI_TABLE), so values that came from gram_state_export are restored
+ * exactly. */
+gram_status gram_state_import(gram_ctx* ctx, const float* h_table, const uint32_t* h_touched, const float* h_cache,
+                              int32_t steps_in_window);
+/* Optimiser state of one module: update count, and for GRAM_OPT_ADAM the two moment estimates in the parameters'
+ * layout (h_m, h_v fp32 [gram_param_count]; ignored and may be NULL for GRAM_OPT_SGD). */
+gram_status gram_optimizer_export(gram_ctx* ctx, int module, float* h_m, float* h_v, int64_t* updates);
+gram_status gram_optimizer_import(gram_ctx* ctx, int module, const float* h_m, const float* h_v, int64_t updates);
+
 /* --- measurement -------------------------------------------------------------
  * Kernel kinds for gram_profile_read. */
 enum { GRAM_K_GEMM = 0, GRAM_K_ATTENTION = 1, GRAM_K_LAYERNORM = 2, GRAM_K_COLSUM = 3, GRAM_K_EMBED_POOL = 4,

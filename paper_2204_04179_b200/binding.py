@@ -33,7 +33,8 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_task", "gram_encoder_backward", "gram_step", "gram_step_host", "gram_cache_fill",
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
            "gram_launch_count", "gram_profile_dump", "gram_accumulate_static", "gram_optimizer_step",
-           "gram_optimizer_reset", "gram_noam_rate", "gram_adam_update"]
+           "gram_optimizer_reset", "gram_noam_rate", "gram_adam_update", "gram_state_export", "gram_state_import",
+           "gram_optimizer_export", "gram_optimizer_import"]
 
 KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other",
          "optimizer"]
@@ -258,6 +259,36 @@ class Gram:
         cache = np.empty((n, d), np.float32) if want_cache else None
         self._ck(lib().gram_get_window(self._h, _ptr(table), _ptr(touched), _ptr(cache)))
         return table, touched, cache
+
+    # checkpoint / resume
+    def state_export(self):
+        """(table, touched, cache, steps_in_window) of the open Multi-step window."""
+        n, d = self.cfg.n_items, self.cfg.d
+        table = np.empty((n, d), np.float32); touched = np.empty((n + 31) // 32, np.uint32); cache = np.empty((n, d), np.float32)
+        steps = C.c_int32(0)
+        self._ck(lib().gram_state_export(self._h, _ptr(table), _ptr(touched), _ptr(cache), C.byref(steps)))
+        return table, touched, cache, steps.value
+
+    def state_import(self, table, touched, cache, steps_in_window: int):
+        table = None if table is None else np.ascontiguousarray(table, np.float32)
+        touched = None if touched is None else np.ascontiguousarray(touched, np.uint32)
+        cache = None if cache is None else np.ascontiguousarray(cache, np.float32)
+        self._ck(lib().gram_state_import(self._h, _ptr(table), _ptr(touched), _ptr(cache), C.c_int32(int(steps_in_window))))
+
+    def optimizer_export(self, module: int):
+        """(m, v, updates) of one module; m and v are None for plain SGD."""
+        n = self.param_count(module)
+        adam = self.cfg.optimizer == GRAM_OPT_ADAM
+        m = np.empty(n, np.float32) if adam else None
+        v = np.empty(n, np.float32) if adam else None
+        upd = C.c_int64(0)
+        self._ck(lib().gram_optimizer_export(self._h, module, _ptr(m), _ptr(v), C.byref(upd)))
+        return m, v, upd.value
+
+    def optimizer_import(self, module: int, m, v, updates: int):
+        m = None if m is None else np.ascontiguousarray(m, np.float32)
+        v = None if v is None else np.ascontiguousarray(v, np.float32)
+        self._ck(lib().gram_optimizer_import(self._h, module, _ptr(m), _ptr(v), C.c_int64(int(updates))))
 
     # measurement
     def profile(self, enable: bool):

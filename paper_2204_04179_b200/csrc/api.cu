@@ -366,6 +366,23 @@ gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, 
   NEED_MODEL("gram_get_window");
   return model_get_window(ctx->model, h_table, h_touched, h_cache);
 }
+gram_status gram_state_export(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache, int32_t* steps_in_window) {
+  NEED_MODEL("gram_state_export");
+  return model_state_export(ctx->model, h_table, h_touched, h_cache, steps_in_window);
+}
+gram_status gram_state_import(gram_ctx* ctx, const float* h_table, const uint32_t* h_touched, const float* h_cache,
+                              int32_t steps_in_window) {
+  NEED_MODEL("gram_state_import");
+  return model_state_import(ctx->model, h_table, h_touched, h_cache, steps_in_window);
+}
+gram_status gram_optimizer_export(gram_ctx* ctx, int module, float* h_m, float* h_v, int64_t* updates) {
+  NEED_MODEL("gram_optimizer_export");
+  return model_optimizer_export(ctx->model, module, h_m, h_v, updates);
+}
+gram_status gram_optimizer_import(gram_ctx* ctx, int module, const float* h_m, const float* h_v, int64_t updates) {
+  NEED_MODEL("gram_optimizer_import");
+  return model_optimizer_import(ctx->model, module, h_m, h_v, updates);
+}
 gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
                            int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
                            gram_stream stream) {

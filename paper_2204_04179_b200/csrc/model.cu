@@ -866,6 +866,62 @@ gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, floa
   return GRAM_OK;
 }
 
+gram_status model_state_export(Model* m, float* h_table, uint32_t* h_touched, float* h_cache, int32_t* steps) {
+  GRAM_TRY(model_get_window(m, h_table, h_touched, h_cache));
+  if (steps) *steps = m->step_in_window;
+  return GRAM_OK;
+}
+
+gram_status model_state_import(Model* m, const float* h_table, const uint32_t* h_touched, const float* h_cache, int32_t steps) {
+  if (!m->table) return gram_set_error(m->ctx, "the context was created with K <= 1"), GRAM_ERR_ARG;
+  const gram_config& c = m->cfg;
+  if (steps < 0 || steps >= c.K) return gram_set_error(m->ctx, "gram_state_import: %d steps in a window of %d", steps, c.K), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  if (h_table) GRAM_CUDA(m->ctx, cudaMemcpy(m->table, h_table, (size_t)c.n_items * c.d * 4, cudaMemcpyHostToDevice));
+  if (h_touched) GRAM_CUDA(m->ctx, cudaMemcpy(m->touched, h_touched, (size_t)((c.n_items + 31) / 32) * 4, cudaMemcpyHostToDevice));
+  if (h_cache) {
+    if (m->cache_dtype == GRAM_F32) {
+      GRAM_CUDA(m->ctx, cudaMemcpy(m->cache, h_cache, (size_t)c.n_items * c.d * 4, cudaMemcpyHostToDevice));
+    } else {      // through the fp32 gradient buffer, a batch's worth of rows at a time
+      const size_t rows_per = (size_t)((int64_t)c.B_max * c.L);
+      for (size_t r0 = 0; r0 < (size_t)c.n_items; r0 += rows_per) {
+        const size_t nr = ((size_t)c.n_items - r0 < rows_per) ? (size_t)c.n_items - r0 : rows_per;
+        GRAM_CUDA(m->ctx, cudaMemcpy(m->dE, h_cache + r0 * c.d, nr * c.d * 4, cudaMemcpyHostToDevice));
+        GRAM_TRY(convert_f32_to_bf16(m->ctx, m->dE, (bf16*)m->cache + r0 * c.d, nr * c.d, 0));
+        GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+      }
+    }
+  }
+  m->step_in_window = steps;
+  return GRAM_OK;
+}
+
+gram_status model_optimizer_export(Model* m, int module, float* h_m, float* h_v, int64_t* updates) {
+  Module* mod = module == GRAM_MODULE_CE ? &m->ce : module == GRAM_MODULE_TASK ? &m->task : nullptr;
+  if (!mod) return gram_set_error(m->ctx, "unknown module %d", module), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  if (updates) *updates = mod->updates;
+  if (mod->am && mod->n) {
+    if (!h_m || !h_v) return gram_set_error(m->ctx, "gram_optimizer_export: Adam state needs both moment buffers"), GRAM_ERR_ARG;
+    GRAM_CUDA(m->ctx, cudaMemcpy(h_m, mod->am, mod->n * 4, cudaMemcpyDeviceToHost));
+    GRAM_CUDA(m->ctx, cudaMemcpy(h_v, mod->av, mod->n * 4, cudaMemcpyDeviceToHost));
+  }
+  return GRAM_OK;
+}
+
+gram_status model_optimizer_import(Model* m, int module, const float* h_m, const float* h_v, int64_t updates) {
+  Module* mod = module == GRAM_MODULE_CE ? &m->ce : module == GRAM_MODULE_TASK ? &m->task : nullptr;
+  if (!mod || updates < 0) return gram_set_error(m->ctx, "gram_optimizer_import: bad module or update count"), GRAM_ERR_ARG;
+  GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  if (mod->am && mod->n) {
+    if (!h_m || !h_v) return gram_set_error(m->ctx, "gram_optimizer_import: Adam state needs both moment buffers"), GRAM_ERR_ARG;
+    GRAM_CUDA(m->ctx, cudaMemcpy(mod->am, h_m, mod->n * 4, cudaMemcpyHostToDevice));
+    GRAM_CUDA(m->ctx, cudaMemcpy(mod->av, h_v, mod->n * 4, cudaMemcpyHostToDevice));
+  }
+  mod->updates = updates;
+  return GRAM_OK;
+}
+
 gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in, int32_t B, int on_host,
                        gram_step_report* rep, cudaStream_t st) {
   const gram_config& c = m->cfg;

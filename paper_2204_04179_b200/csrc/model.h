@@ -28,6 +28,10 @@ gram_status model_step(Model* m, const int32_t* ids, const int32_t* labels, int3
 gram_status model_cache_fill(Model* m, cudaStream_t st);
 gram_status model_window_reset(Model* m, cudaStream_t st);
 gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, float* h_cache);
+gram_status model_state_export(Model* m, float* h_table, uint32_t* h_touched, float* h_cache, int32_t* steps);
+gram_status model_state_import(Model* m, const float* h_table, const uint32_t* h_touched, const float* h_cache, int32_t steps);
+gram_status model_optimizer_export(Model* m, int module, float* h_m, float* h_v, int64_t* updates);
+gram_status model_optimizer_import(Model* m, int module, const float* h_m, const float* h_v, int64_t updates);
 float* model_table(Model* m);
 uint32_t* model_touched(Model* m);
 

@@ -312,3 +312,44 @@ def test_texts_of_different_lengths(name):
         bad = lengths.copy(); bad[3] = shape.l_t + 1
         g.set_item_lengths(bad)
     g.close()
+
+
+@pytest.mark.parametrize("dtype,variant", [("f32", binding.GRAM_MULTI_TABLE), ("bf16", binding.GRAM_MULTI_TABLE),
+                                           ("f32", binding.GRAM_MULTI_PSEUDO_TARGET)])
+def test_checkpoint_and_resume_continue_bit_for_bit(dtype, variant):
+    """Parameters, optimiser state and the open Multi-step window exported after two steps of a window of three and
+    imported into a fresh context: the third step (with its encoder pass and both Adam updates) gives identical
+    results in both contexts."""
+    K = 3
+    shape = small(dtype=dtype, d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=41)
+    batches = [synth.batch(shape, 41, step=k) for k in range(K + 1)]
+    over = dict(K=K, lr_task=1e-2, lr_ce=1e-2, ce_micro_batch=16, multistep_variant=variant, optimizer=binding.GRAM_OPT_ADAM,
+                noam_warmup=4)
+    a = gh.make_ctx(shape, ce, tk, toks, **over)
+    a.cache_fill()
+    to_dev = lambda x: torch.from_numpy(x).to(DEV)
+    for k in range(4):                     # one whole window (so that the optimiser state is not trivial), then one step
+        a.step(to_dev(batches[k % (K + 1)][0]), to_dev(batches[k % (K + 1)][1]), shape.B)
+    table, touched, cache, steps = a.state_export()
+    assert steps == 1 and touched.any() and np.abs(table).max() > 0
+    b = gh.make_ctx(shape, ce, tk, toks, **over)
+    for mod in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK):
+        b.set_params(mod, a.get_params(mod))
+        m_, v_, upd = a.optimizer_export(mod)
+        assert upd == (1 if mod == binding.GRAM_MODULE_CE else 4) and np.abs(m_).max() > 0
+        b.optimizer_import(mod, m_, v_, upd)
+    b.state_import(table, touched, cache, steps)
+    for k in (1, 2):
+        ra = a.step(to_dev(batches[k][0]), to_dev(batches[k][1]), shape.B)
+        rb = b.step(to_dev(batches[k][0]), to_dev(batches[k][1]), shape.B)
+        assert ra.loss == rb.loss and ra.n_touched == rb.n_touched and ra.encoder_pass == rb.encoder_pass
+    assert rb.encoder_pass == 1
+    for mod in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK):
+        assert np.array_equal(a.get_params(mod), b.get_params(mod))
+        assert np.array_equal(a.get_grads(mod), b.get_grads(mod))
+    ta, ua, ca, sa = a.state_export(); tb, ub, cb, sb = b.state_export()
+    assert sa == sb == 0 and np.array_equal(ca, cb) and np.array_equal(ta, tb) and np.array_equal(ua, ub)
+    with pytest.raises(binding.GramError):
+        b.state_import(None, None, None, K)
+    a.close(); b.close()
