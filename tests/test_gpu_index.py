@@ -185,3 +185,54 @@ def test_multistep_table_and_touched():
     chk = np.zeros((N, d)); np.add.at(chk, ids, dE_np.astype(np.float64))
     np.testing.assert_allclose(t2, chk, rtol=1e-12, atol=1e-12)
     g.close()
+
+
+@pytest.mark.parametrize("s", [0.8, 1.5])
+def test_largest_sweep_cell(s):
+    """The largest cell of the kernel sweep that the benchmark's probe runs (P = 10^7 positions, 10^6 items, d = 256):
+    every dedup output against the oracle, bit-exact; the segmented sum on sampled items against a float64 sum of that
+    item's rows, plus conservation of column sums; the gather on every position.  s = 1.5 puts more than a third of
+    all positions on one item, s = 0.8 leaves almost every item of the pool in the batch."""
+    P, N, d = 10_000_000, 1_000_000, 256
+    ids = synth.zipf_ids(13, N, s, P)
+    g = index_ctx(P, N, d_max=d)
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, N)
+    want = orc.unique_inverse(ids)
+    assert U == len(want[0])
+    for got, w, name in zip((unique, inverse, perm, seg_off), want, ("unique", "inverse", "perm", "seg_off")):
+        assert np.array_equal(got, w), name
+    counts = np.diff(seg_off)
+    if s == 1.5:
+        assert counts.max() > P // 3
+    else:
+        assert U > 900_000
+    gen = torch.Generator(device=DEV); gen.manual_seed(17)
+    dE = torch.rand(P, d, device=DEV, generator=gen) * 2 - 1                 # uniform(-1, 1), the sweep's gradients
+    perm_d, so_d = torch.from_numpy(perm).to(DEV), torch.from_numpy(seg_off).to(DEV)
+    G = torch.full((U, d), float("nan"), device=DEV)
+    g.accumulate(dE, perm_d, so_d, U, G)
+    g.sync()
+    col = dE.sum(0, dtype=torch.float64)
+    assert float((G.sum(0, dtype=torch.float64) - col).abs().max()) <= 1e-6 * float(dE.abs().sum(0, dtype=torch.float64).max())
+    rng = np.random.default_rng(3)
+    sample = {0, U - 1, int(np.argmax(counts)), int(np.argmin(counts))} | {int(u) for u in rng.integers(0, U, 60)}
+    for u in sorted(sample):
+        rows = perm[seg_off[u]:seg_off[u + 1]].astype(np.int64)
+        x = dE[torch.from_numpy(rows).to(DEV)].cpu().numpy().astype(np.float64)
+        ref = np.zeros(d)
+        for r in range(min(len(rows), 2000)):                               # the oracle's loop: rows in ascending order
+            ref += x[r]
+        if len(rows) > 2000:
+            ref += x[2000:].sum(0)
+        bound = len(rows) * 2.0 ** -24 * np.abs(x).sum(0).max() + 1e-12
+        assert np.abs(G[u].cpu().numpy().astype(np.float64) - ref).max() <= bound, (u, len(rows))
+    del dE
+    H = torch.rand(U, d, device=DEV, generator=gen)
+    inv_d = torch.from_numpy(inverse).to(DEV)
+    E = torch.empty(P, d, device=DEV)
+    g.gather(H, inv_d, E)
+    g.sync()
+    for p0 in range(0, P, 2_000_000):                                        # every position, in slices to bound memory
+        sl = slice(p0, min(P, p0 + 2_000_000))
+        assert torch.equal(E[sl], H[inv_d[sl].long()])
+    g.close()
