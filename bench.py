@@ -122,6 +122,8 @@ def run_reference(args, shape):
     ce = synth.encoder_params(shape, args.seed)
     tk = synth.task_params(shape, args.seed)
     toks = synth.item_tokens(args.seed, shape.n_items, shape.l_t, shape.vocab)
+    if args.var_len:
+        toks = synth.ragged(toks, synth.item_lengths(args.seed, shape.n_items, shape.l_t, shortest=min(4, shape.l_t)))
     n_pos = min(bounded_sample_size(shape), 12 if shape.name != "tiny" else shape.L)
     times, cores = [], 0
     for k in range(args.warmup + args.steps):
@@ -231,6 +233,10 @@ def run_gram(args, shape):
     g.set_params(binding.GRAM_MODULE_CE, synth.flatten(ce))
     g.set_params(binding.GRAM_MODULE_TASK, synth.flatten(tk))
     g.set_item_tokens(toks)
+    lengths = None
+    if args.var_len:                   # texts of 4 .. l_t tokens, uniform: the encoder then works on packed rows
+        lengths = synth.item_lengths(args.seed, shape.n_items, shape.l_t, shortest=min(4, shape.l_t))
+        g.set_item_lengths(lengths)
     P = shape.B * shape.L
     n_total = args.warmup + args.steps
     # every rank draws its own batches (weak scaling: per-GPU work is fixed, histories are independent)
@@ -320,6 +326,7 @@ def run_gram(args, shape):
                    "task": shape.task, "zipf_s": shape.zipf_s, "unique_items_per_step": statistics.mean(r.n_unique for r in reports),
                    "boost_ratio_R": statistics.mean(r.boost_ratio for r in reports), "ce_micro_batch": int(cfg.ce_micro_batch),
                    "l2": "working set (activations of >1e5 tokens) far larger than L2; no flush needed",
+                   "text_lengths": ("uniform 4..l_t, mean %.1f tokens" % float(lengths.mean())) if lengths is not None else "all l_t",
                    "parallelism": f"replicas x{world}" if world > 1 else "1 GPU"},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * P, "d2h_bytes_per_step": 12,
@@ -339,7 +346,8 @@ def run_gram(args, shape):
         except Exception as ex:          # the sweep cell is extra information, never a reason to lose the line
             line["hbm_kernels"] = {"error": repr(ex)}
         n_pos = bounded_sample_size(shape)
-        v, dt, cores = oracle_sample(shape, ce, tk, toks, batches[0][0], batches[0][1], n_pos)
+        toks_o = synth.ragged(toks, lengths) if lengths is not None else toks
+        v, dt, cores = oracle_sample(shape, ce, tk, toks_o, batches[0][0], batches[0][1], n_pos)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"end-to-end oracle (float64, one encoder call per interaction) on the first {n_pos} "
                                           f"positions of one history of the same workload, {dt:.1f} s; linear in interactions"}
@@ -362,6 +370,7 @@ def main():
     ap.add_argument("--micro-batch", type=int, default=0, help="items per encoder pass (0: the workload's default)")
     ap.add_argument("--multistep-variant", default="table", choices=["table", "pseudo_target"],
                     help="kt_multistep: separate gradient table with unchanged cached encodings, or pseudo-targets (Section 4.3)")
+    ap.add_argument("--var-len", action="store_true", help="item texts of different lengths (uniform 4..l_t) instead of all l_t")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     from paper_2204_04179_b200 import synth

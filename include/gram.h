@@ -143,8 +143,9 @@ gram_status gram_set_item_tokens(gram_ctx* ctx, const int32_t* h_tokens);
  * h_lengths int32 [n_items], item i's text is its first h_lengths[i] tokens (1 .. l_t), the remaining slots of its
  * row of h_tokens are padding whose values are never used.  The encoder then attends over the text tokens only and
  * mean pooling averages over them; an item encodes exactly as it would in a model whose l_t is its own length.
- * Padding slots are still computed (storage stays [n_items, l_t]); their outputs are never read and their gradients
- * are zero.  NULL restores texts of exactly l_t tokens (the state after gram_create). */
+ * On the device the token rows of an encoder pass are then packed (item after item, no rows for padding), so a pass
+ * costs the sum of its items' lengths, not n * l_t; the pass reads that sum back from the device once (it
+ * synchronises the stream).  NULL restores texts of exactly l_t tokens (the state after gram_create). */
 gram_status gram_set_item_lengths(gram_ctx* ctx, const int32_t* h_lengths);
 
 /* --- the five stages (Algorithm 1; Fig. 1) -------------------------------- */

@@ -207,7 +207,8 @@ __device__ __forceinline__ void mma_regs_times_rows(const float (&x)[SP / 8][4],
 template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
                                                            int n_heads, int causal, float scale,
-                                                           const int32_t* __restrict__ seq_len) {
+                                                           const int32_t* __restrict__ seq_len,
+                                                           const int32_t* __restrict__ seq_off) {
   constexpr int LD = DH + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
@@ -215,13 +216,18 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   bf16* Vs = Ks + SP * LD;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
-  const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
+  int64_t row0 = seq * S;
+  if (seq_off) {                                  // packed rows: this sequence is rows seq_off .. + seq_len, no padding
+    row0 = seq_off[seq];
+    S = seq_len[seq];
+  }
+  const bf16* base = qkv + row0 * 3 * (int64_t)d + h * DH;
   load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs);
   load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
   load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
   loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
-  bf16* ob = out + seq * S * (int64_t)d + h * DH;
+  bf16* ob = out + row0 * (int64_t)d + h * DH;
   const int Sv = seq_len ? seq_len[seq] : S;      // keys that are text; the rows after them are padding
   for (int r0 = warp * 16; r0 < S; r0 += 64) {
     float p[SP / 8][4];
@@ -243,7 +249,8 @@ template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
                                                            bf16* __restrict__ dqkv, float* __restrict__ colpart, int S, int d,
                                                            int n_heads, int causal, float scale,
-                                                           const int32_t* __restrict__ seq_len) {
+                                                           const int32_t* __restrict__ seq_len,
+                                                           const int32_t* __restrict__ seq_off) {
   constexpr int LD = DH + 8, LP = SP + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // [SP][DH+8]
@@ -254,14 +261,19 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   bf16* dSs = Ps + SP * LP;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
-  const bf16* base = qkv + seq * S * 3 * (int64_t)d + h * DH;
+  int64_t row0 = seq * S;
+  if (seq_off) {
+    row0 = seq_off[seq];
+    S = seq_len[seq];
+  }
+  const bf16* base = qkv + row0 * 3 * (int64_t)d + h * DH;
   load_head<SP, DH>(base, 3 * (int64_t)d, S, Qs);
   load_head<SP, DH>(base + d, 3 * (int64_t)d, S, Ks);
   load_head<SP, DH>(base + 2 * d, 3 * (int64_t)d, S, Vs);
-  load_head<SP, DH>(dctx + seq * S * (int64_t)d + h * DH, d, S, dOs);
+  load_head<SP, DH>(dctx + row0 * (int64_t)d + h * DH, d, S, dOs);
   loads_done();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
-  bf16* dq = dqkv + seq * S * 3 * (int64_t)d + h * DH;
+  bf16* dq = dqkv + row0 * 3 * (int64_t)d + h * DH;
   const int Sv = seq_len ? seq_len[seq] : S;
   // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ (kept in registers as bf16 pairs) ----
   constexpr int NIT = (SP + 63) / 64;
@@ -378,22 +390,22 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
 
 template <int SP, int DH>
 gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
-                       const int32_t* seq_len, cudaStream_t st) {
+                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   constexpr size_t smem = (size_t)3 * SP * (DH + 8) * 2;
   auto kern = attn_fwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len);
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 template <int SP, int DH>
 gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                       int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
+                       int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
   auto kern = attn_bwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len);
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -422,10 +434,11 @@ bool attention_mma_supported(int S, int d, int n_heads) {
   } while (0)
 
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, const int32_t* seq_len, cudaStream_t st) {
-  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, seq_len, st);
+                                  int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
+  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
 }
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq,
-                                   int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
-  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, st);
+                                   int S, int d, int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+                                   cudaStream_t st) {
+  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
 }

@@ -34,7 +34,7 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const 
                                  int32_t first_item, int64_t n_tok, int32_t n_items_total, int l_t, int vocab, int d,
                                  const float* __restrict__ tok_emb, const float* __restrict__ pos_emb,
                                  float* __restrict__ z0, int32_t* __restrict__ tok_ids,
-                                 const int32_t* __restrict__ item_len, int32_t* __restrict__ seq_len, int32_t* status) {
+                                 const int32_t* __restrict__ seq_len, const int32_t* __restrict__ seq_off, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -45,16 +45,17 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ item_tokens, const 
     if (item < 0 || item >= n_items_total) { gram_device_fail(status, GRAM_ERR_ID_RANGE); item = 0; }
     int32_t tok = item_tokens[(int64_t)item * l_t + s];
     if (tok < 0 || tok >= vocab) { gram_device_fail(status, GRAM_ERR_ID_RANGE); tok = 0; }
-    if (lane == 0) tok_ids[t] = tok;
-    if (seq_len && s == 0 && lane == 0) {        // tokens of this item that are text, the rest is padding
-      int32_t n = item_len[item];
-      seq_len[u] = n < 1 ? 1 : (n > l_t ? l_t : n);
+    int64_t row = t;
+    if (seq_off) {                               // packed rows: item u owns rows seq_off[u] .. + seq_len[u], no padding
+      if (s >= seq_len[u]) continue;
+      row = (int64_t)seq_off[u] + s;
     }
+    if (lane == 0) tok_ids[row] = tok;
     const float* te = tok_emb + (int64_t)tok * d;
     const float* pe = pos_emb + (int64_t)s * d;
     for (int c = 2 * lane; c < d; c += 64) {
       float2 a = ld2(te + c), b = ld2(pe + c);
-      st2(z0 + t * d + c, make_float2(a.x + b.x, a.y + b.y));
+      st2(z0 + row * d + c, make_float2(a.x + b.x, a.y + b.y));
     }
   }
 }
@@ -234,16 +235,22 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float* __res
 template <typename T>
 __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out, int S, int d,
                                                        int n_heads, int causal, float scale,
-                                                       const int32_t* __restrict__ seq_len) {
+                                                       const int32_t* __restrict__ seq_len,
+                                                       const int32_t* __restrict__ seq_off) {
   extern __shared__ float sm[];
   const int dh = d / n_heads, ld = dh + 1;
+  int64_t row0 = (int64_t)(blockIdx.x / n_heads) * S;
+  if (seq_off) {                                  // packed rows: this sequence is rows seq_off .. + seq_len
+    row0 = seq_off[blockIdx.x / n_heads];
+    S = seq_len[blockIdx.x / n_heads];
+  }
   float* Q = sm;
   float* K = Q + S * ld;
   float* V = K + S * ld;
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
   const int Sv = seq_len ? seq_len[seq] : S;          // keys that are text; rows past them are padding
-  const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
+  const T* base = qkv + row0 * 3 * (int64_t)d + h * dh;
   for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
     const int s = i / dh, c = i - s * dh;
     const T* p = base + (int64_t)s * 3 * d + c;
@@ -289,7 +296,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
         if (lane + 32 < dh) o1 += pj * V[j * ld + lane + 32];
       }
     }
-    T* o = out + (seq * S + i) * (int64_t)d + h * dh;
+    T* o = out + (row0 + i) * (int64_t)d + h * dh;
     if (lane < dh) stf(o + lane, o0 * inv);
     if (lane + 32 < dh) stf(o + lane + 32, o1 * inv);
   }
@@ -298,8 +305,14 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(const T* __restrict__ qkv
 template <typename T>
 __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dctx,
                                                        T* __restrict__ dqkv, int S, int d, int n_heads, int causal,
-                                                       float scale, const int32_t* __restrict__ seq_len) {
+                                                       float scale, const int32_t* __restrict__ seq_len,
+                                                       const int32_t* __restrict__ seq_off) {
   extern __shared__ float sm[];
+  int64_t row0 = (int64_t)(blockIdx.x / n_heads) * S;
+  if (seq_off) {
+    row0 = seq_off[blockIdx.x / n_heads];
+    S = seq_len[blockIdx.x / n_heads];
+  }
   const int dh = d / n_heads, ld = dh + 1, lp = S + 1;
   float* Q = sm;
   float* K = Q + S * ld;
@@ -309,8 +322,8 @@ __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv
   float* dS = Pm + S * lp;       // [S][S+1] gradient of the scaled scores
   const int64_t seq = blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
-  const T* base = qkv + seq * S * 3 * (int64_t)d + h * dh;
-  const T* dbase = dctx + seq * S * (int64_t)d + h * dh;
+  const T* base = qkv + row0 * 3 * (int64_t)d + h * dh;
+  const T* dbase = dctx + row0 * (int64_t)d + h * dh;
   const int Sv = seq_len ? seq_len[seq] : S;
   for (int i = threadIdx.x; i < S * dh; i += blockDim.x) {
     const int s = i / dh, c = i - s * dh;
@@ -322,7 +335,7 @@ __global__ void __launch_bounds__(128) attn_bwd_kernel(const T* __restrict__ qkv
   }
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
-  T* dbq = dqkv + seq * S * 3 * (int64_t)d + h * dh;
+  T* dbq = dqkv + row0 * 3 * (int64_t)d + h * dh;
   // phase 1: one query row per warp: probabilities, dS, and dQ
   for (int i = warp; i < S; i += nwb) {
     float p[4], dp[4];
@@ -430,12 +443,18 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, in
 }
 
 __global__ void periodic_rowsum_kernel(const float* __restrict__ X, int64_t n_groups, int period, int d,
-                                       float* __restrict__ out) {
+                                       float* __restrict__ out, const int32_t* __restrict__ seq_len,
+                                       const int32_t* __restrict__ seq_off) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)period * d) return;
   const int s = (int)(i / d), c = (int)(i - (int64_t)s * d);
   float acc = 0.f;
-  for (int64_t u = 0; u < n_groups; ++u) acc += X[(u * period + s) * d + c];
+  if (seq_off) {                                   // packed rows: group u has seq_len[u] rows starting at seq_off[u]
+    for (int64_t u = 0; u < n_groups; ++u)
+      if (s < seq_len[u]) acc += X[((int64_t)seq_off[u] + s) * d + c];
+  } else {
+    for (int64_t u = 0; u < n_groups; ++u) acc += X[(u * period + s) * d + c];
+  }
   out[i] += acc;
 }
 
@@ -446,22 +465,23 @@ __device__ __forceinline__ float stream_at(const StreamRef& x, int64_t row, int 
   return v;
 }
 __global__ void pool_fwd_kernel(StreamRef x, float* __restrict__ H, int64_t n, int l_t, int d, int pooling,
-                                const int32_t* __restrict__ seq_len) {
+                                const int32_t* __restrict__ seq_len, const int32_t* __restrict__ seq_off) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * d) return;
   const int64_t u = i / d;
   const int c = (int)(i - u * d);
+  const int64_t row0 = seq_off ? (int64_t)seq_off[u] : u * l_t;
   if (pooling == GRAM_POOL_CLS) {
-    H[i] = stream_at(x, u * l_t, c, d);
+    H[i] = stream_at(x, row0, c, d);
   } else {
     const int len = seq_len ? seq_len[u] : l_t;      // mean over the tokens that are text
     float acc = 0.f;
-    for (int s = 0; s < len; ++s) acc += stream_at(x, u * l_t + s, c, d);
+    for (int s = 0; s < len; ++s) acc += stream_at(x, row0 + s, c, d);
     H[i] = acc / len;
   }
 }
 __global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__ dx, int64_t n, int l_t, int d, int pooling,
-                                const int32_t* __restrict__ seq_len) {
+                                const int32_t* __restrict__ seq_len, const int32_t* __restrict__ seq_off) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * l_t * d) return;
   const int64_t t = i / d;
@@ -473,6 +493,10 @@ __global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__
   else {
     const int len = seq_len ? seq_len[u] : l_t;
     v = s < len ? G[u * d + c] / len : 0.f;
+  }
+  if (seq_off) {                                   // packed rows: the padding slots have no row
+    if (s < seq_len[u]) dx[((int64_t)seq_off[u] + s) * d + c] = v;
+    return;
   }
   dx[i] = v;
 }
@@ -701,13 +725,64 @@ __global__ void scatter_rows_kernel(const float* __restrict__ src, const int32_t
 }
 
 // rows of `words` 32-bit words copied between two layouts whose rows are in_stride / out_stride words apart
+// in_rows / out_rows (may be null): row r of that side is row in_rows[r] / out_rows[r] instead of r
 __global__ void strided_rows_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out, int64_t n, int64_t in_stride,
-                                    int64_t out_stride, int words) {
+                                    int64_t out_stride, int words, const int32_t* __restrict__ in_rows,
+                                    const int32_t* __restrict__ out_rows) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * words) return;
   const int64_t r = i / words;
   const int c = (int)(i - r * words);
-  out[r * out_stride + c] = in[r * in_stride + c];
+  const int64_t ri = in_rows ? in_rows[r] : r, ro = out_rows ? out_rows[r] : r;
+  out[ro * out_stride + c] = in[ri * in_stride + c];
+}
+
+// lengths and first rows of the sequences of one encoder pass: seq_len[u] = item_len[item(u)] (clamped to 1..l_t),
+// seq_off = its exclusive prefix sum, seq_off[n] = total rows.  One block; item(u) = items[u] or first_item + u.
+__global__ void __launch_bounds__(1024) seq_layout_kernel(const int32_t* __restrict__ item_len, const int32_t* __restrict__ items,
+                                                          int32_t first_item, int32_t n, int32_t n_items_total, int l_t,
+                                                          int32_t* __restrict__ seq_len, int32_t* __restrict__ seq_off,
+                                                          int32_t* status) {
+  __shared__ int32_t sw[33];
+  __shared__ int32_t carry_s;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (int32_t base = 0; base < n; base += 1024) {
+    const int32_t u = base + threadIdx.x;
+    int32_t len = 0;
+    if (u < n) {
+      int32_t item = items ? items[u] : first_item + u;
+      if (item < 0 || item >= n_items_total) { gram_device_fail(status, GRAM_ERR_ID_RANGE); item = 0; }
+      len = item_len[item];
+      len = len < 1 ? 1 : (len > l_t ? l_t : len);
+      seq_len[u] = len;
+    }
+    // inclusive scan over the block
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t incl = len;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) sw[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int32_t w = sw[lane], wi = w;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += t;
+      }
+      sw[lane] = wi - w;
+      if (lane == 31) sw[32] = wi;
+    }
+    __syncthreads();
+    const int32_t carry = carry_s;
+    if (u < n) seq_off[u] = carry + sw[warp] + incl - len;
+    __syncthreads();
+    if (threadIdx.x == 0) carry_s = carry + sw[32];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) seq_off[n] = carry_s;
 }
 
 inline int grid_for(int64_t n, int threads, int cap) {
@@ -737,14 +812,14 @@ template <typename F> gram_status set_smem(gram_ctx* ctx, F kern, size_t bytes) 
 
 gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* item_len, int32_t* seq_len,
+                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* seq_len, const int32_t* seq_off,
                           cudaStream_t st) {
   const int64_t n_tok = (int64_t)n_chunk * l_t;
   if (n_tok == 0) return GRAM_OK;
   const int blocks = grid_for(n_tok * 32, 256, kNumSMs * 8);
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 8.0 * (double)n_tok * d, 1, st);
   embed_fwd_kernel<<<blocks, 256, 0, st>>>(item_tokens, items, first_item, n_tok, n_items_total, l_t, vocab, d, tok_emb,
-                                           pos_emb, z0, tok_ids, item_len, item_len ? seq_len : nullptr, gram_status_word(ctx));
+                                           pos_emb, z0, tok_ids, seq_len, seq_off, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -779,7 +854,7 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 }
 
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
+                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
@@ -787,17 +862,18 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_fwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, st);
+    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
-    attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale, seq_len);
+    attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale, seq_len, seq_off);
   });
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st) {
+                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
+                               const int32_t* seq_off, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
@@ -805,11 +881,11 @@ gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const 
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, st);
+    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
   if (colpart) return gram_set_error(ctx, "attention: fused column sums need the tensor-core kernel"), GRAM_ERR_UNSUPPORTED;
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
-    attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale, seq_len);
+    attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale, seq_len, seq_off);
   });
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
@@ -869,29 +945,29 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
 }
 
 gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
-                                       cudaStream_t st) {
+                                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   if (n_groups == 0) return GRAM_OK;
   const int64_t n = (int64_t)period * d;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n_groups * period * d, 1, st);
-  periodic_rowsum_kernel<<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>(X, n_groups, period, d, out);
+  periodic_rowsum_kernel<<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>(X, n_groups, period, d, out, seq_len, seq_off);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
-                         const int32_t* seq_len, cudaStream_t st) {
+                         const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (pooling == GRAM_POOL_CLS ? 2 : l_t + 1), 1, st);
-  pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling, seq_len);
+  pool_fwd_kernel<<<(unsigned)ceil_div64(n * d, 256), 256, 0, st>>>(x, H, n, l_t, d, pooling, seq_len, seq_off);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
-                          const int32_t* seq_len, cudaStream_t st) {
+                          const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * d * (l_t + 1), 1, st);
-  pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling, seq_len);
+  pool_bwd_kernel<<<(unsigned)ceil_div64(n * l_t * d, 256), 256, 0, st>>>(G, dx, n, l_t, d, pooling, seq_len, seq_off);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -1039,25 +1115,35 @@ gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32
   return GRAM_OK;
 }
 
-gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
-                              cudaStream_t st) {
+gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, const int32_t* rows, int d,
+                              int elem_bytes, void* out, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   if ((d * elem_bytes) % 4) return gram_set_error(ctx, "row copy: rows must be whole 32-bit words"), GRAM_ERR_ARG;
   const int words = d * elem_bytes / 4;
   ProfScope prof(ctx, GRAM_K_OTHER, 2.0 * (double)n * d * elem_bytes, 1, st);
-  strided_rows_kernel<<<(unsigned)ceil_div64(n * words, 256), 256, 0, st>>>((const uint32_t*)in, (uint32_t*)out, n, stride * words,
-                                                                          words, words);
+  strided_rows_kernel<<<(unsigned)ceil_div64(n * words, 256), 256, 0, st>>>((const uint32_t*)in, (uint32_t*)out, n,
+                                                                          rows ? words : stride * words, words, words, rows,
+                                                                          nullptr);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
-gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
-                             cudaStream_t st) {
+gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, const int32_t* rows, int d,
+                             int elem_bytes, void* out, cudaStream_t st) {
   if (n == 0) return GRAM_OK;
   if ((d * elem_bytes) % 4) return gram_set_error(ctx, "row copy: rows must be whole 32-bit words"), GRAM_ERR_ARG;
   const int words = d * elem_bytes / 4;
   ProfScope prof(ctx, GRAM_K_OTHER, 2.0 * (double)n * d * elem_bytes, 1, st);
   strided_rows_kernel<<<(unsigned)ceil_div64(n * words, 256), 256, 0, st>>>((const uint32_t*)in, (uint32_t*)out, n, words,
-                                                                          stride * words, words);
+                                                                          rows ? words : stride * words, words, nullptr, rows);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status sequence_layout(gram_ctx* ctx, const int32_t* item_len, const int32_t* items, int32_t first_item, int32_t n,
+                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, cudaStream_t st) {
+  if (n <= 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 12.0 * (double)n, 1, st);
+  seq_layout_kernel<<<1, 1024, 0, st>>>(item_len, items, first_item, n, n_items_total, l_t, seq_len, seq_off, gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -19,12 +19,17 @@ struct StreamRef {
 };
 
 // z0[t, :] = tok_emb[token(t), :] + pos_emb[t % l_t, :] (fp32), token(t) = item_tokens[items[t / l_t], t % l_t];
-// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.  item_len (may be null): tokens of each
-// item that are text (the rest of its l_t slots is padding); seq_len[u] then receives the length of chunk item u.
+// tok_ids[t] = token(t).  items == null means items[u] = first_item + u.  seq_len / seq_off (both or neither): packed
+// rows for texts of different lengths: item u's tokens 0 .. seq_len[u]-1 go to rows seq_off[u] .. and its padding
+// slots get no row at all.
 gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32_t* items, int32_t first_item,
                           int32_t n_items_chunk, int32_t n_items_total, int l_t, int vocab, int d, const float* tok_emb,
-                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* item_len, int32_t* seq_len,
+                          const float* pos_emb, float* z0, int32_t* tok_ids, const int32_t* seq_len, const int32_t* seq_off,
                           cudaStream_t st);
+// seq_len[u] = item_len[item(u)] for the n items of an encoder pass and seq_off = its exclusive prefix sum
+// (seq_off[n] = rows in total)
+gram_status sequence_layout(gram_ctx* ctx, const int32_t* item_len, const int32_t* items, int32_t first_item, int32_t n,
+                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, cudaStream_t st);
 
 // y = LayerNorm(z): z is the fp32 stream, y the operand-typed copy the next matrix product reads
 gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
@@ -38,20 +43,22 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 
 // softmax(Q K^T / sqrt(dh)) V per (sequence, head); qkv is [n_seq*S, 3d] (Q | K | V), ctx [n_seq*S, d].
 // seq_len (may be null): only the first seq_len[s] rows of sequence s are keys; the rows after them are padding,
-// whose outputs are finite and never read, and whose gradients are zero.
+// whose outputs are finite and never read, and whose gradients are zero.  seq_off (may be null, needs seq_len): packed
+// rows, sequence s is rows seq_off[s] .. seq_off[s] + seq_len[s] (at most S of them) and there is no padding.
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
+                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 // colpart (may be null; only where attention_mma_supported and dtype is bf16): fp32 [n_seq, 3d], row s receives the
 // column sums of sequence s's rows of dqkv, the partial sums of the bias gradient of the Q, K, V projection
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
+                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
+                               const int32_t* seq_off, cudaStream_t st);
 
 // the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
 bool attention_mma_supported(int S, int d, int n_heads);
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, const int32_t* seq_len, cudaStream_t st);
+                                  int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                                   int n_heads, int causal, const int32_t* seq_len, cudaStream_t st);
+                                   int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 
 // out[n] += sum_rows X[r, n]   (X operand-typed)
 // out[c] += sum over the nrows rows of part[., c] (fp32 [nrows, N]; partial column sums left by a fused producer)
@@ -60,15 +67,16 @@ gram_status colsum_from_partials(gram_ctx* ctx, const float* part, int64_t nrows
 gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t rows, int N, float* out, float* scratch,
                               cudaStream_t st);
 // out[s, :] += sum_u X[u*period + s, :]  (s < period; X fp32)
+// packed rows (seq_len, seq_off not null): out[s, :] += sum over the groups u with s < seq_len[u] of X[seq_off[u] + s, :]
 gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
-                                       cudaStream_t st);
+                                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 
 // H[u, :] = mean_s x[u*l_t + s, :] (mean; over the first seq_len[u] tokens when seq_len is given) or x[u*l_t, :] (cls), fp32
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,
-                         const int32_t* seq_len, cudaStream_t st);
-// dx[u*l_t + s, :] from G[u, :] (both fp32)
+                         const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
+// dx[u*l_t + s, :] from G[u, :] (both fp32); with seq_off the rows of item u are seq_off[u] + s
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
-                          const int32_t* seq_len, cudaStream_t st);
+                          const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 
 // knowledge-tracing task input: x[b, n, :] = E[b, n, :] + pos[n, :] + resp[prev(b, n), :] (fp32, and an
 // operand-typed copy x_b), prev(b, 0) = 2, prev(b, n) = labels[b, n-1]
@@ -100,9 +108,9 @@ gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float
 // dst[index[u], :] = src[u, :] (src fp32, dst operand-typed)
 gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st);
-// out[r, :] = in[r * stride, :] for r < n: every stride-th row of a [n*stride, d] matrix of elem_bytes-byte elements
-gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
-                              cudaStream_t st);
-// out[r * stride, :] = in[r, :] for r < n; the other rows of out are left as they are
-gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, int d, int elem_bytes, void* out,
-                             cudaStream_t st);
+// out[r, :] = in[row(r), :] for r < n, row(r) = rows[r] when rows is given, else r * stride; elem_bytes-byte elements
+gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, const int32_t* rows, int d,
+                              int elem_bytes, void* out, cudaStream_t st);
+// out[row(r), :] = in[r, :] for r < n; the other rows of out are left as they are
+gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, const int32_t* rows, int d,
+                             int elem_bytes, void* out, cudaStream_t st);

@@ -37,6 +37,8 @@ struct Stack {
   int d = 0, heads = 0, d_ff = 0, n_layers = 0, attn_only = 0, causal = 0;
   int64_t cap = 0;                         // tokens the buffers hold
   const int32_t* seq_len = nullptr;        // per sequence: rows that are text (null: all S); set per pass
+  const int32_t* seq_off = nullptr;        // packed rows: first row of each sequence (null: sequence s starts at row s*S)
+  int64_t packed_rows = 0;                 // packed rows: rows in total (0: n_seq * S)
   std::vector<LayerOff> off;
   std::vector<LayerActs> acts;
   // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
@@ -100,6 +102,8 @@ struct Model {
   int32_t* item_len = nullptr;       // [n_items] tokens of each item that are text (variable-length texts), else null
   int32_t* item_len_buf = nullptr;   // its storage
   int32_t* seq_len = nullptr;        // [mb] the same for the items of the current encoder pass
+  int32_t* seq_off = nullptr;        // [mb + 1] first packed row of each of them; [n] = rows of the pass
+  int64_t saved_rows = 0;            // token rows of the last encoder pass (packed when the texts differ in length)
   int32_t mb = 0;                    // items per encoder pass
   int32_t saved_n = -1;              // items whose activations the last encoder pass saved (-1: none)
   // task
@@ -191,6 +195,7 @@ void layout_buffers(Model* m, Arena& a) {
     m->tok_nu = (int32_t*)a.take(4);
     m->item_len_buf = (int32_t*)a.take((size_t)c.n_items * 4);
     m->seq_len = (int32_t*)a.take((size_t)m->mb * 4);
+    m->seq_off = (int32_t*)a.take(((size_t)m->mb + 1) * 4);
     stack_buffers(a, m->enc, esz);
     if (m->cls_tail) {
       stack_buffers(a, m->tail, esz);
@@ -298,14 +303,14 @@ void set_res(GemmEpilogue& e, const StreamRef& x) {
 // ---- one transformer layer in two parts, forward --------------------------------------------
 // the attention part over whole sequences: qkv = x Wqkv^T + bqkv, ctx = softmax(Q K^T / sqrt(dh)) V
 gram_status layer_attention_forward(Model* m, Module& mod, Stack& s, int l, const void* xb, int64_t n_seq, int S, cudaStream_t st) {
-  const int64_t T = n_seq * S;
+  const int64_t T = s.packed_rows ? s.packed_rows : n_seq * S;
   const LayerOff& o = s.off[l];
   LayerActs& a = s.acts[l];
   GemmEpilogue e;
   e.bias = mod.w + o.bqkv;
   e.tag = "fwd_qkv";
   GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * s.d, s.d, e, st));
-  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, st);
+  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, s.seq_off, st);
 }
 
 // the row-wise rest of the layer over T rows: output projection + residual, LayerNorm, feed-forward + residual,
@@ -353,7 +358,7 @@ gram_status layer_rest_forward(Model* m, Module& mod, const LayerOff& o, LayerAc
 // part only (its ctx is left in s.acts[n_full].ctx) and *out / *out_b describe that layer's input.
 gram_status stack_forward(Model* m, Module& mod, Stack& s, const StreamRef& x_in, const void* x_in_b, int64_t n_seq, int S,
                           cudaStream_t st, StreamRef* out, const void** out_b, int n_full = -1) {
-  const int64_t T = n_seq * S;
+  const int64_t T = s.packed_rows ? s.packed_rows : n_seq * S;
   if (n_full < 0) n_full = s.n_layers;
   StreamRef x = x_in;
   const void* xb = x_in_b;
@@ -418,7 +423,7 @@ gram_status layer_rest_backward(Model* m, Module& mod, const LayerOff& o, Stack&
 // to the layer's input; copy_b: the layer below reads it as an operand as well (attention-only stacks).
 gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, const void* xb_l, int64_t n_seq, int S, float* cur,
                                      const float* oth, bool copy_b, cudaStream_t st) {
-  const int64_t T = n_seq * S;
+  const int64_t T = s.packed_rows ? s.packed_rows : n_seq * S;
   const int d = s.d;
   gram_ctx* ctx = m->ctx;
   const LayerOff& o = s.off[l];
@@ -426,7 +431,7 @@ gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, con
   const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
                           (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
   GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
-                              s.causal, s.seq_len, st));
+                              s.causal, s.seq_len, s.seq_off, st));
   if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, m->red, st));
   else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, m->red, st));
   GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
@@ -444,7 +449,7 @@ gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, con
 // stream.
 gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, int64_t n_seq, int S, cudaStream_t st,
                            float** d_in, bool top_attention_only = false) {
-  const int64_t T = n_seq * S;
+  const int64_t T = s.packed_rows ? s.packed_rows : n_seq * S;
   float* cur = s.curf;
   float* oth = s.othf;
   for (int l = s.n_layers - 1; l >= 0; --l) {
@@ -457,6 +462,8 @@ gram_status stack_backward(Model* m, Module& mod, Stack& s, const void* x_in_b, 
   return GRAM_OK;
 }
 
+gram_status read_i32(Model* m, const int32_t* d_ptr, int32_t* out, cudaStream_t st);
+
 // encoder forward over n items (d_items, or first_item.. when null): H_out [n, d] fp32
 gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const int32_t* d_items, int32_t first_item,
                                   int32_t n, float* H_out, cudaStream_t st) {
@@ -464,11 +471,25 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   gram_ctx* ctx = m->ctx;
   if (n > m->mb) return gram_set_error(ctx, "encoder pass over %d items exceeds the micro-batch of %d", n, m->mb), GRAM_ERR_WORKSPACE;
   GRAM_TRY(refresh_bf16(m, m->ce, st));
-  const int64_t T = (int64_t)n * c.l_t;
-  GRAM_TRY(embed_forward(ctx, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items, c.l_t,
-                         c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, m->item_len, m->seq_len, st));
-  const int32_t* seq_len = m->item_len ? m->seq_len : nullptr;
+  // texts of different lengths: rows are packed, item u owns rows seq_off[u] .. + seq_len[u] and padding has no rows
+  const int32_t* seq_len = nullptr;
+  const int32_t* seq_off = nullptr;
+  int64_t T = (int64_t)n * c.l_t;
+  if (m->item_len) {
+    GRAM_TRY(sequence_layout(ctx, m->item_len, d_items, first_item, n, c.n_items, c.l_t, m->seq_len, m->seq_off, st));
+    int32_t rows = 0;
+    GRAM_TRY(read_i32(m, m->seq_off + n, &rows, st));
+    if (rows < n || rows > T) return gram_set_error(ctx, "encoder pass: %d token rows for %d items", rows, n), GRAM_ERR_ID_RANGE;
+    T = rows;
+    seq_len = m->seq_len;
+    seq_off = m->seq_off;
+  }
   m->enc.seq_len = seq_len;
+  m->enc.seq_off = seq_off;
+  m->enc.packed_rows = seq_off ? T : 0;
+  m->saved_rows = T;
+  GRAM_TRY(embed_forward(ctx, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items, c.l_t,
+                         c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, seq_len, seq_off, st));
   GRAM_TRY(layernorm_forward(ctx, m->dtype, m->z0, m->ce.w + m->o_elng, m->ce.w + m->o_elnb, m->x0, m->mean0, m->rstd0, T,
                              c.d, st));
   StreamRef x0;
@@ -477,7 +498,7 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   const void* out_b = nullptr;
   if (!m->cls_tail) {
     GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
-    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, seq_len, st));
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
   } else {
     // all layers but the last, and the last layer's attention over whole sequences
     const int last = c.n_layers - 1;
@@ -486,14 +507,14 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
     GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &x, &xb, last));
     // row 0 of every item: the attention output and the last layer's input stream (values and LayerNorm statistics)
     LayerActs& ta = m->tail.acts[0];
-    GRAM_TRY(take_strided_rows(ctx, m->enc.acts[last].ctx, n, c.l_t, c.d, (int)m->esz, ta.ctx, st));
-    GRAM_TRY(take_strided_rows(ctx, x.z, n, c.l_t, c.d, 4, m->tail_z, st));
-    GRAM_TRY(take_strided_rows(ctx, x.mean, n, c.l_t, 1, 4, m->tail_mean, st));
-    GRAM_TRY(take_strided_rows(ctx, x.rstd, n, c.l_t, 1, 4, m->tail_rstd, st));
+    GRAM_TRY(take_strided_rows(ctx, m->enc.acts[last].ctx, n, c.l_t, seq_off, c.d, (int)m->esz, ta.ctx, st));
+    GRAM_TRY(take_strided_rows(ctx, x.z, n, c.l_t, seq_off, c.d, 4, m->tail_z, st));
+    GRAM_TRY(take_strided_rows(ctx, x.mean, n, c.l_t, seq_off, 1, 4, m->tail_mean, st));
+    GRAM_TRY(take_strided_rows(ctx, x.rstd, n, c.l_t, seq_off, 1, 4, m->tail_rstd, st));
     StreamRef xr = x;
     xr.z = m->tail_z; xr.mean = m->tail_mean; xr.rstd = m->tail_rstd;
     GRAM_TRY(layer_rest_forward(m, m->ce, m->tail.off[0], ta, c.d, c.d_ff, 0, xr, ta.ctx, n, st, &out, &out_b));
-    GRAM_TRY(pool_forward(ctx, out, H_out, n, 1, c.d, c.pooling, nullptr, st));       // one row per item: the pooled row itself
+    GRAM_TRY(pool_forward(ctx, out, H_out, n, 1, c.d, c.pooling, nullptr, nullptr, st));       // one row per item: the pooled row itself
   }
   m->saved_n = n;
   return GRAM_OK;
@@ -504,29 +525,31 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   const gram_config& c = m->cfg;
   gram_ctx* ctx = m->ctx;
   if (n != m->saved_n) return gram_set_error(ctx, "encoder backward over %d items, but activations of %d are saved", n, m->saved_n), GRAM_ERR_ARG;
-  const int64_t T = (int64_t)n * c.l_t;
+  const int64_t T = m->saved_rows;
+  const int32_t* seq_len = m->enc.seq_len;
+  const int32_t* seq_off = m->enc.seq_off;
   float* dx0 = nullptr;
   if (!m->cls_tail) {
-    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, m->enc.seq_len, st));
+    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
     GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
   } else {
     // the row-wise part of the last layer on one row per item
     Stack& tl = m->tail;
-    GRAM_TRY(pool_backward(ctx, G, tl.curf, n, 1, c.d, c.pooling, nullptr, st));
+    GRAM_TRY(pool_backward(ctx, G, tl.curf, n, 1, c.d, c.pooling, nullptr, nullptr, st));
     float* cur = tl.curf;
     float* oth = tl.othf;
     GRAM_TRY(layer_rest_backward(m, m->ce, tl.off[0], tl, tl.acts[0], n, &cur, &oth, st));
     // back into whole sequences: every other row of the two gradients is zero
     GRAM_CUDA(ctx, cudaMemsetAsync(m->enc.dctx, 0, (size_t)T * c.d * m->esz, st));
     GRAM_CUDA(ctx, cudaMemsetAsync(m->enc.othf, 0, (size_t)T * c.d * 4, st));
-    GRAM_TRY(put_strided_rows(ctx, tl.dctx, n, c.l_t, c.d, (int)m->esz, m->enc.dctx, st));
-    GRAM_TRY(put_strided_rows(ctx, oth, n, c.l_t, c.d, 4, m->enc.othf, st));
+    GRAM_TRY(put_strided_rows(ctx, tl.dctx, n, c.l_t, seq_off, c.d, (int)m->esz, m->enc.dctx, st));
+    GRAM_TRY(put_strided_rows(ctx, oth, n, c.l_t, seq_off, c.d, 4, m->enc.othf, st));
     GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0, true));
   }
   float* dz0 = (dx0 == m->enc.curf) ? m->enc.othf : m->enc.curf;
   GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, nullptr,
                               m->ce.g + m->o_elng, m->ce.g + m->o_elnb, nullptr, m->red, T, c.d, st));
-  GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, st));
+  GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, seq_len, seq_off, st));
   // token-embedding gradient: sum dz0 over the occurrences of each token (same index kernels as stage 1 / 4)
   IndexWorkspace* iws = gram_index_ws(ctx);
   GRAM_TRY(dedup_launch(ctx, iws, m->tok_ids, T, c.vocab, m->tok_unique, m->tok_inverse, m->tok_perm, m->tok_seg, m->tok_nu, st));
