@@ -215,7 +215,8 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
         next item e_n, and predicts r_n (Section 3.1): input
         x_n = E[b, n] + pos[n] + resp[r_{n-1}] (resp row 2 marks "no previous
         response" at n = 0), causal attention, logit_n = head_w . y_n + head_b,
-        binary cross-entropy, averaged over all B*L predictions.
+        binary cross-entropy, averaged over all B*L predictions (over the real
+        ones when histories end in padding, label -1).
     nr: additive attention over the first L - n_cand encodings gives the user
         vector, dot products with the n_cand candidate encodings give scores,
         loss = -log softmax(scores)[0] (the first candidate is the click),
@@ -224,18 +225,27 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
     B, L, d = E.shape
     lab = torch.as_tensor(np.asarray(labels), dtype=torch.long)
     if shape.task == "kt":
+        # A history shorter than L ends in padding, marked by label -1 (Appendix D: sequences are cut or padded to a
+        # maximum length).  Padding is simply absent here: history b is the sequence of its first n_b positions,
+        # and the mean runs over the sum of the n_b real predictions.
         total = E.new_zeros(())
+        n_pred = 0
         for b in range(B):
-            prev = torch.cat([torch.full((1,), 2, dtype=torch.long), lab[b, :-1]])
-            x = E[b] + th["pos"] + th["resp"][prev]
+            neg = (lab[b] < 0).nonzero()
+            n = int(neg[0]) if len(neg) else L
+            if n == 0:
+                continue
+            prev = torch.cat([torch.full((1,), 2, dtype=torch.long), lab[b, :n - 1]])
+            x = E[b, :n] + th["pos"][:n] + th["resp"][prev]
             for l in range(shape.task_layers):
                 x = transformer_layer(x, th, f"t{l}.", shape.task_heads, causal=True,
                                       attn_only=shape.task_attn_only)
             z = x @ th["head_w"] + th["head_b"]
-            y = lab[b].to(E.dtype)
+            y = lab[b, :n].to(E.dtype)
             # BCE with logits: softplus(z) - y*z, written with a stable softplus
             total = total + (torch.clamp(z, min=0) + torch.log1p(torch.exp(-z.abs())) - y * z).sum()
-        return total / (B * L)
+            n_pred += n
+        return total / max(n_pred, 1)
     if shape.task == "nr":
         n_hist = L - shape.n_cand
         total = E.new_zeros(())

@@ -373,3 +373,33 @@ def test_short_text_encoding_ignores_what_follows_it():
     for l in range(shape.n_layers):
         x = orc.transformer_layer(x, th, f"l{l}.", shape.n_heads, causal=False)
     np.testing.assert_allclose(one.numpy(), x[0].numpy(), rtol=1e-13)
+
+
+# ---- histories of different lengths (padding at the end, label -1) -----------------------------------------------------
+
+def test_padded_history_is_the_shorter_history():
+    # two histories, the second with n < L real positions: the loss is the prediction-weighted mean of the two
+    # histories evaluated on their own (the second one as a batch whose L is n), and nothing at a padded position
+    # (its encoding, its gradient) takes part
+    shape = small_shape(B=2, L=6, task_attn_only=False, task_layers=2)
+    ce, tk, toks, ids, lab = make(shape, seed=12)
+    n = 4
+    lab = lab.copy(); lab[1, n:] = -1
+    E = torch.randn(2, 6, shape.d, dtype=T64, generator=torch.Generator().manual_seed(1))
+    th = orc.as_torch(tk, T64)
+    Eg = E.clone().requires_grad_(True)
+    loss = orc.task_loss(th, Eg, lab, shape)
+    loss.backward()
+    with torch.no_grad():
+        one = orc.task_loss(th, E[:1], lab[:1], shape.replace(B=1))
+        th_short = dict(th); th_short["pos"] = th["pos"][:n]
+        two = orc.task_loss(th_short, E[1:, :n], lab[1:, :n], shape.replace(B=1, L=n))
+    assert abs(float(loss) - (6 * float(one) + n * float(two)) / (6 + n)) < 1e-13
+    assert torch.count_nonzero(Eg.grad[1, n:]) == 0 and torch.count_nonzero(Eg.grad[1, :n]) > 0
+    E2 = E.clone(); E2[1, n:] += 3.0
+    with torch.no_grad():
+        assert float(orc.task_loss(th, E2, lab, shape)) == float(loss.detach())
+    # the mean is over real predictions, not over B*L
+    lab_all = lab.copy(); lab_all[1, n:] = 0
+    with torch.no_grad():
+        assert abs(float(orc.task_loss(th, E, lab_all, shape)) - float(loss.detach())) > 1e-6
