@@ -200,7 +200,11 @@ gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int
 /* Task module forward and backward (Eq. 5 and the gradient of Eq. 8 with
  * respect to the encodings): d_E fp32 [B, L, d], d_labels int32 [B, L] ->
  * d_dE fp32 [B*L, d], d_loss fp32 [1]; task parameter gradients are
- * overwritten in the context. */
+ * overwritten in the context.  Labels are 0 or 1.  For GRAM_TASK_KT a history
+ * shorter than L ends in padding (Appendix D: sequences are cut or padded to a
+ * maximum length): its padded positions carry label -1 and any valid item ID,
+ * are not predicted, receive a zero row of d_dE, and the loss is the mean over
+ * the real predictions of the batch.  The same holds for gram_step. */
 gram_status gram_task(gram_ctx* ctx, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE,
                       float* d_loss, gram_stream stream);
 

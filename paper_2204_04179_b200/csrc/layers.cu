@@ -512,7 +512,7 @@ __global__ void kt_input_fwd_kernel(const float* __restrict__ E, const float* __
   const int c = (int)(i - p * d);
   const int n = (int)(p % L);
   int prev = (n == 0) ? 2 : labels[p - 1];
-  prev = prev < 0 ? 0 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);
+  prev = prev < 0 ? 2 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);      // after a padded position (label -1): only at padded rows
   const float v = E[i] + pos[(int64_t)n * d + c] + resp[(int64_t)prev * d + c];
   x[i] = v;
   stf(x_b + i, v);
@@ -544,12 +544,13 @@ template <typename T>
 __global__ void __launch_bounds__(256) kt_head_kernel(StreamRef y, const float* __restrict__ w,
                                                       const float* __restrict__ bias, const int32_t* __restrict__ labels,
                                                       float* __restrict__ dy, T* __restrict__ dy_b,
-                                                      float* __restrict__ part, int64_t P, int d, int64_t pstride) {
+                                                      float* __restrict__ part, int64_t P, int d, int64_t pstride,
+                                                      const int32_t* __restrict__ n_real) {
   extern __shared__ float sacc[];            // [d + 2]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
   for (int i = threadIdx.x; i < d + 2; i += blockDim.x) sacc[i] = 0.f;
   __syncthreads();
-  const float b0 = bias[0], invP = 1.f / (float)P;
+  const float b0 = bias[0], invP = 1.f / (float)max(*n_real, 1);   // the mean runs over the real predictions
   // rows are dealt to blocks in contiguous ranges so that each block adds its rows in order
   const int64_t per = (P + gridDim.x - 1) / gridDim.x;
   const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(r0 + per, P);
@@ -560,9 +561,12 @@ __global__ void __launch_bounds__(256) kt_head_kernel(StreamRef y, const float* 
       float acc = 0.f;
       for (int c = lane; c < d; c += 32) acc += stream_at(y, r, c, d) * w[c];
       const float z = warp_sum(acc) + b0;
-      const float lab = (float)labels[r];
-      lossr = fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
-      dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
+      const int32_t li = labels[r];
+      const float lab = (float)li;
+      if (li >= 0) {                          // label -1: padding at the end of a history, not predicted
+        lossr = fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
+        dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
+      }
       for (int c = lane; c < d; c += 32) {
         dy[r * d + c] = dzl * w[c];
         if (dy_b) stf(dy_b + r * d + c, dzl * w[c]);
@@ -579,15 +583,25 @@ __global__ void __launch_bounds__(256) kt_head_kernel(StreamRef y, const float* 
   for (int i = threadIdx.x; i < d + 2; i += blockDim.x) part[(int64_t)blockIdx.x * pstride + i] = sacc[i];
 }
 
-__global__ void kt_head_reduce_kernel(const float* __restrict__ part, int nblocks, int64_t pstride, int d, float invP,
-                                      float* __restrict__ dw, float* __restrict__ db, float* __restrict__ loss) {
+__global__ void kt_head_reduce_kernel(const float* __restrict__ part, int nblocks, int64_t pstride, int d,
+                                      const int32_t* __restrict__ n_real, float* __restrict__ dw, float* __restrict__ db,
+                                      float* __restrict__ loss) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= d + 2) return;
+  const float invP = 1.f / (float)max(*n_real, 1);
   float a = 0.f;
   for (int k = 0; k < nblocks; ++k) a += part[(int64_t)k * pstride + c];
   if (c < d) dw[c] += a;
   else if (c == d) loss[0] = a * invP;
   else db[0] += a;
+}
+
+// positions with a label >= 0 (integer adds: the count does not depend on their order); *n_real must start at zero
+__global__ void count_real_kernel(const int32_t* __restrict__ labels, int64_t P, int32_t* __restrict__ n_real) {
+  int32_t c = 0;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < P; p += (int64_t)gridDim.x * blockDim.x) c += labels[p] >= 0;
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(n_real, c);
 }
 
 // ---------------------------------------------------------------------------- NR task (per user)
@@ -983,16 +997,18 @@ gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const flo
 }
 
 gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w, const float* b, const int32_t* labels,
-                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int64_t P, int d,
-                    cudaStream_t st) {
+                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int32_t* n_real, int64_t P,
+                    int d, cudaStream_t st) {
   if (P == 0) return GRAM_OK;
   int blocks = (int)ceil_div64(P, 64);
   if (blocks > kRedBlocks) blocks = kRedBlocks;
   const int64_t pstride = d + 2;
   const size_t smem = (size_t)(d + 2) * sizeof(float);
-  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 12.0 * (double)P * d, 2, st);
-  DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>(y, w, b, labels, dy, (T*)dy_b, scratch, P, d, pstride));
-  kt_head_reduce_kernel<<<ceil_div(d + 2, 256), 256, 0, st>>>(scratch, blocks, pstride, d, 1.f / (float)P, dw, db, loss);
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 12.0 * (double)P * d, 3, st);
+  GRAM_CUDA(ctx, cudaMemsetAsync(n_real, 0, sizeof(int32_t), st));
+  count_real_kernel<<<grid_for(P, 256, kNumSMs), 256, 0, st>>>(labels, P, n_real);
+  DISPATCH_T(dtype, kt_head_kernel<T><<<blocks, 256, smem, st>>>(y, w, b, labels, dy, (T*)dy_b, scratch, P, d, pstride, n_real));
+  kt_head_reduce_kernel<<<ceil_div(d + 2, 256), 256, 0, st>>>(scratch, blocks, pstride, d, n_real, dw, db, loss);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -85,11 +85,12 @@ gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const flo
 // dE = dx; dpos[n] += sum_b dx[b, n]; dresp[r] += sum over positions with prev == r
 gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* labels, float* dE, float* dpos,
                               float* dresp, float* scratch, int B, int L, int d, cudaStream_t st);
-// logit = y . w + b; loss = mean BCE; dy = (sigmoid(logit) - label) / (B*L) * w (fp32, and an operand-typed
-// copy dy_b when not null); dw, db accumulate
+// logit = y . w + b; loss = mean BCE over the positions with a label >= 0 (label -1: padding at the end of a history,
+// not predicted); dy = (sigmoid(logit) - label) / (their number) * w, zero at padded positions (fp32, and an
+// operand-typed copy dy_b when not null); dw, db accumulate; n_real: one device word of scratch for that number
 gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w, const float* b, const int32_t* labels,
-                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int64_t P, int d,
-                    cudaStream_t st);
+                    float* dy, void* dy_b, float* dw, float* db, float* loss, float* scratch, int32_t* n_real, int64_t P,
+                    int d, cudaStream_t st);
 
 // news-recommendation task, the part between the matrix products (one block per user):
 // given pre = E wa^T + ba [B*L, d_a] (operand-typed), computes additive attention over the first L - n_cand

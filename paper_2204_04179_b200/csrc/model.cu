@@ -119,6 +119,7 @@ struct Model {
   float *H = nullptr, *E = nullptr;  // encodings per unique item / per position, fp32
   void* Eb = nullptr;                // operand-typed copy of E (NR products; Multi-step gather from the cache)
   float *dE = nullptr, *G = nullptr, *loss = nullptr, *red = nullptr;
+  int32_t* n_real = nullptr;         // predictions of the batch that are not padding
   // Multi-step window
   float* table = nullptr;
   uint32_t* touched = nullptr;
@@ -229,6 +230,7 @@ void layout_buffers(Model* m, Arena& a) {
   m->Eb = a.take((size_t)P * d * esz);
   m->dE = (float*)a.take((size_t)P * d * 4);
   m->loss = (float*)a.take(4);
+  m->n_real = (int32_t*)a.take(4);
   m->red = (float*)a.take(kRedScratchBytes);
   if (c.K > 1) {
     m->table = (float*)a.take((size_t)c.n_items * d * 4);
@@ -576,7 +578,7 @@ gram_status task_forward_backward(Model* m, const float* E, const int32_t* label
     GRAM_TRY(stack_forward(m, m->task, m->tk, x, m->txb, B, c.L, st, &y, &y_b));
     void* dy_b = (m->tk.attn_only && m->tk.n_layers > 0) ? m->tk.dzb : nullptr;
     GRAM_TRY(kt_head(ctx, m->dtype, y, m->task.w + m->t_headw, m->task.w + m->t_headb, labels, m->tk.curf, dy_b,
-                     m->task.g + m->t_headw, m->task.g + m->t_headb, loss, m->red, P, c.d, st));
+                     m->task.g + m->t_headw, m->task.g + m->t_headb, loss, m->red, m->n_real, P, c.d, st));
     float* dx = nullptr;
     GRAM_TRY(stack_backward(m, m->task, m->tk, m->txb, B, c.L, st, &dx));
     GRAM_TRY(kt_input_backward(ctx, dx, labels, dE, m->task.g + m->t_pos, m->task.g + m->t_resp, m->red, B, c.L, c.d, st));

@@ -353,3 +353,34 @@ def test_checkpoint_and_resume_continue_bit_for_bit(dtype, variant):
     with pytest.raises(binding.GramError):
         b.state_import(None, None, None, K)
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("name", ["tiny_cfg", "cls_full_task", "bf16_cls_full"])
+def test_histories_that_end_in_padding(name):
+    """Label -1 marks padding at the end of a history: no prediction there, zero gradient rows, loss averaged over the
+    real predictions; the oracle evaluates the shorter histories themselves."""
+    shape = CASES[name]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=33)
+    lab = lab.copy()
+    rng = np.random.default_rng(0)
+    lens = rng.integers(1, shape.L + 1, shape.B)
+    lens[0] = shape.L
+    for b, n in enumerate(lens):
+        lab[b, n:] = -1
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab)
+    tol = TOL[shape.dtype]
+    assert abs(rep.loss - want["loss"]) <= tol * abs(want["loss"])
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+    print(name, "worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+    # the gradient rows of padded positions are exactly zero
+    g = gh.make_ctx(shape, ce, tk, toks)
+    P, d = ids.size, shape.d
+    E = torch.randn(P, d, device=DEV); dE = torch.full((P, d), float("nan"), device=DEV); loss = torch.zeros(1, device=DEV)
+    g.task(E, torch.from_numpy(lab.ravel().copy()).to(DEV), shape.B, dE, loss)
+    g.sync()
+    pad = torch.from_numpy((lab.ravel() < 0)).to(DEV)
+    assert pad.any() and torch.count_nonzero(dE[pad]) == 0 and torch.isfinite(dE).all()
+    g.close()

@@ -394,7 +394,7 @@ def test_padded_history_is_the_shorter_history():
         one = orc.task_loss(th, E[:1], lab[:1], shape.replace(B=1))
         th_short = dict(th); th_short["pos"] = th["pos"][:n]
         two = orc.task_loss(th_short, E[1:, :n], lab[1:, :n], shape.replace(B=1, L=n))
-    assert abs(float(loss) - (6 * float(one) + n * float(two)) / (6 + n)) < 1e-13
+    assert abs(float(loss.detach()) - (6 * float(one) + n * float(two)) / (6 + n)) < 1e-13
     assert torch.count_nonzero(Eg.grad[1, n:]) == 0 and torch.count_nonzero(Eg.grad[1, :n]) > 0
     E2 = E.clone(); E2[1, n:] += 3.0
     with torch.no_grad():
