@@ -384,3 +384,27 @@ def test_histories_that_end_in_padding(name):
     pad = torch.from_numpy((lab.ravel() < 0)).to(DEV)
     assert pad.any() and torch.count_nonzero(dE[pad]) == 0 and torch.isfinite(dE).all()
     g.close()
+
+
+def test_multistep_window_with_texts_of_different_lengths():
+    # the cache fill (items by range) and the encoder pass over the touched items (items by list) both run on packed rows
+    K = 2
+    shape = small(dtype="f32", d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls", l_t=9)
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=27)
+    lengths = synth.item_lengths(27, shape.n_items, shape.l_t)
+    ragged = synth.ragged(toks, lengths)
+    batches = [synth.batch(shape, 27, step=k) for k in range(K)]
+    g = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=0.05, ce_micro_batch=16)
+    g.set_item_lengths(lengths)
+    g.cache_fill()
+    _, _, cache0 = g.get_window(want_table=False, want_touched=False)
+    assert gh.rel_err(cache0, orc.encode_all(shape, ce, ragged, range(shape.n_items))) <= 1e-4
+    want = orc.multistep_window(shape, ce, tk, ragged, batches, cache0.astype(np.float64), lr_task=0.05)
+    reps = [g.step(torch.from_numpy(i).to(DEV), torch.from_numpy(l).to(DEV), shape.B) for i, l in batches]
+    assert reps[-1].encoder_pass == 1 and reps[-1].n_encoded == len(want["items"])
+    gce, gtk = gh.gpu_grads(g, shape)
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    assert e1 <= 1e-3, (e1, n1)
+    _, _, cache = g.get_window(want_table=False, want_touched=False)
+    assert gh.rel_err(cache, want["cache"]) <= 1e-4
+    g.close()
