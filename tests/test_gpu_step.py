@@ -269,7 +269,10 @@ VARLEN = {
     # tensor-core attention: texts of 1..40 tokens in a 64-row tile, and 1..70 in a 96-row tile
     "bf16_mean_40": small(dtype="bf16", l_t=40, d=64, n_heads=2, d_ff=128, task_d_ff=128, n_items=30, pooling="mean"),
     "bf16_cls_70": small(dtype="bf16", l_t=70, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30, pooling="cls", B=2),
+    # several ragged encoder passes of 7 items, each with its own packed layout
+    "f32_cls_micro_batches": small(l_t=9, pooling="cls", n_items=60, B=6, L=16),
 }
+VARLEN_OVER = {"f32_cls_micro_batches": dict(ce_micro_batch=7)}
 
 
 @pytest.mark.parametrize("name", list(VARLEN))
@@ -285,8 +288,9 @@ def test_texts_of_different_lengths(name):
         junk[i, n:] = (junk[i, n:] * 7 + 3) % shape.vocab
     tol = TOL[shape.dtype]
     results = []
+    over = VARLEN_OVER.get(name, {})
     for tokens in (toks, junk):
-        g = gh.make_ctx(shape, ce, tk, tokens)
+        g = gh.make_ctx(shape, ce, tk, tokens, **over)
         g.set_item_lengths(lengths)
         rep = g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)
         gce, gtk = gh.gpu_grads(g, shape)
