@@ -208,13 +208,14 @@ template <int SP, int DH>
 __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
                                                            int n_heads, int causal, float scale,
                                                            const int32_t* __restrict__ seq_len,
-                                                           const int32_t* __restrict__ seq_off) {
+                                                           const int32_t* __restrict__ seq_off,
+                                                           const int32_t* __restrict__ seq_list) {
   constexpr int LD = DH + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
   bf16* Ks = Qs + SP * LD;
   bf16* Vs = Ks + SP * LD;
-  const int64_t seq = blockIdx.x / n_heads;
+  const int64_t seq = seq_list ? seq_list[blockIdx.x / n_heads] : blockIdx.x / n_heads;   // this launch's share of the sequences
   const int h = blockIdx.x % n_heads;
   int64_t row0 = seq * S;
   if (seq_off) {                                  // packed rows: this sequence is rows seq_off .. + seq_len, no padding
@@ -250,7 +251,8 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
                                                            bf16* __restrict__ dqkv, float* __restrict__ colpart, int S, int d,
                                                            int n_heads, int causal, float scale,
                                                            const int32_t* __restrict__ seq_len,
-                                                           const int32_t* __restrict__ seq_off) {
+                                                           const int32_t* __restrict__ seq_off,
+                                                           const int32_t* __restrict__ seq_list) {
   constexpr int LD = DH + 8, LP = SP + 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);   // [SP][DH+8]
@@ -259,7 +261,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   bf16* dOs = Vs + SP * LD;
   bf16* Ps = dOs + SP * LD;                       // [query i][key j], [SP][SP+8]
   bf16* dSs = Ps + SP * LP;
-  const int64_t seq = blockIdx.x / n_heads;
+  const int64_t seq = seq_list ? seq_list[blockIdx.x / n_heads] : blockIdx.x / n_heads;
   const int h = blockIdx.x % n_heads;
   int64_t row0 = seq * S;
   if (seq_off) {
@@ -390,22 +392,23 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
 
 template <int SP, int DH>
 gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
-                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
+                       const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list, cudaStream_t st) {
   constexpr size_t smem = (size_t)3 * SP * (DH + 8) * 2;
   auto kern = attn_fwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off);
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 template <int SP, int DH>
 gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                       int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
+                       int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,
+                       cudaStream_t st) {
   constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
   auto kern = attn_bwd_mma_kernel<SP, DH>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off);
+  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -434,11 +437,12 @@ bool attention_mma_supported(int S, int d, int n_heads) {
   } while (0)
 
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
-  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
+                                  int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,
+                                  cudaStream_t st) {
+  ATTN_DISPATCH(launch_fwd, ctx, (const bf16*)qkv, (bf16*)out, n_seq, S, d, n_heads, causal, seq_len, seq_off, seq_list, st);
 }
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq,
                                    int S, int d, int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
-                                   cudaStream_t st) {
-  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
+                                   const int32_t* seq_list, cudaStream_t st) {
+  ATTN_DISPATCH(launch_bwd, ctx, (const bf16*)qkv, (const bf16*)dctx, (bf16*)dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, seq_list, st);
 }

@@ -756,6 +756,7 @@ __global__ void strided_rows_kernel(const uint32_t* __restrict__ in, uint32_t* _
 __global__ void __launch_bounds__(1024) seq_layout_kernel(const int32_t* __restrict__ item_len, const int32_t* __restrict__ items,
                                                           int32_t first_item, int32_t n, int32_t n_items_total, int l_t,
                                                           int32_t* __restrict__ seq_len, int32_t* __restrict__ seq_off,
+                                                          int32_t* __restrict__ group_list, int32_t* __restrict__ info,
                                                           int32_t* status) {
   __shared__ int32_t sw[33];
   __shared__ int32_t carry_s;
@@ -796,7 +797,47 @@ __global__ void __launch_bounds__(1024) seq_layout_kernel(const int32_t* __restr
     if (threadIdx.x == 0) carry_s = carry + sw[32];
     __syncthreads();
   }
-  if (threadIdx.x == 0) seq_off[n] = carry_s;
+  if (threadIdx.x == 0) {
+    seq_off[n] = carry_s;
+    info[4] = carry_s;
+  }
+  __syncthreads();
+  // the sequence numbers grouped by length (1..32, 33..64, 65..96, 97.. rows), ascending inside a group
+  int32_t placed = 0;
+  for (int gi = 0; gi < 4; ++gi) {
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < n; base += 1024) {
+      const int32_t u = base + threadIdx.x;
+      int32_t in = 0;
+      if (u < n) {
+        const int32_t b = (seq_len[u] - 1) >> 5;
+        in = (b > 3 ? 3 : b) == gi;
+      }
+      const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+      const uint32_t vote = __ballot_sync(0xffffffffu, in);
+      if (lane == 0) sw[warp] = __popc(vote);
+      __syncthreads();
+      if (warp == 0) {
+        int32_t w = sw[lane], wi = w;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+          if (lane >= o) wi += t;
+        }
+        sw[lane] = wi - w;
+        if (lane == 31) sw[32] = wi;
+      }
+      __syncthreads();
+      const int32_t carry = carry_s;
+      if (in) group_list[placed + carry + sw[warp] + __popc(vote & ((1u << lane) - 1u))] = u;
+      __syncthreads();
+      if (threadIdx.x == 0) carry_s = carry + sw[32];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) info[gi] = carry_s;
+    placed += carry_s;
+    __syncthreads();
+  }
 }
 
 inline int grid_for(int64_t n, int threads, int cap) {
@@ -868,15 +909,25 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 }
 
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
+                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+                              const SeqGroups* groups, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_fwd");
-  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
+  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads)) {
+    if (!groups || !seq_off) return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
+    int32_t first = 0;
+    for (int gi = 0; gi < 4; ++gi) {                 // one launch per length group, with the smallest tile that fits
+      if (groups->count[gi] > 0)
+        GRAM_TRY(attention_forward_mma(ctx, qkv, out, groups->count[gi], S < 32 * (gi + 1) ? S : 32 * (gi + 1), d, n_heads,
+                                       causal, seq_len, seq_off, groups->list + first, st));
+      first += groups->count[gi];
+    }
+    return GRAM_OK;
+  }
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_fwd_kernel<T>, smem));
     attn_fwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (T*)out, S, d, n_heads, causal, scale, seq_len, seq_off);
@@ -887,15 +938,25 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
 
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
                                int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
-                               const int32_t* seq_off, cudaStream_t st) {
+                               const int32_t* seq_off, const SeqGroups* groups, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
   if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
   const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
-  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads))
-    return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, st);
+  if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads)) {
+    if (!groups || !seq_off)
+      return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
+    int32_t first = 0;
+    for (int gi = 0; gi < 4; ++gi) {
+      if (groups->count[gi] > 0)
+        GRAM_TRY(attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, groups->count[gi], S < 32 * (gi + 1) ? S : 32 * (gi + 1), d,
+                                        n_heads, causal, seq_len, seq_off, groups->list + first, st));
+      first += groups->count[gi];
+    }
+    return GRAM_OK;
+  }
   if (colpart) return gram_set_error(ctx, "attention: fused column sums need the tensor-core kernel"), GRAM_ERR_UNSUPPORTED;
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
@@ -1156,10 +1217,12 @@ gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t s
 }
 
 gram_status sequence_layout(gram_ctx* ctx, const int32_t* item_len, const int32_t* items, int32_t first_item, int32_t n,
-                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, cudaStream_t st) {
+                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, int32_t* group_list,
+                            int32_t* info, cudaStream_t st) {
   if (n <= 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 12.0 * (double)n, 1, st);
-  seq_layout_kernel<<<1, 1024, 0, st>>>(item_len, items, first_item, n, n_items_total, l_t, seq_len, seq_off, gram_status_word(ctx));
+  seq_layout_kernel<<<1, 1024, 0, st>>>(item_len, items, first_item, n, n_items_total, l_t, seq_len, seq_off, group_list, info,
+                                        gram_status_word(ctx));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -8,6 +8,14 @@ constexpr int kRedBlocks = 592;            // upper bound on blocks that leave p
 // bytes of the reduction scratch: kRedBlocks partial rows of up to 2*4096 floats
 constexpr size_t kRedScratchBytes = (size_t)kRedBlocks * 2 * 4096 * sizeof(float);
 
+// Packed sequences grouped by length for the tensor-core attention kernels, whose tile height is a template
+// argument: list (device) holds the sequence numbers with 1..32 rows first, then 33..64, 65..96, 97..128;
+// count (host) says how many there are of each.  A launch per group uses the smallest tile that fits.
+struct SeqGroups {
+  const int32_t* list = nullptr;
+  int32_t count[4] = {0, 0, 0, 0};
+};
+
 // A row-major [rows, d] view of the fp32 residual stream: either the values themselves (mean == null)
 // or LayerNorm of them, applied where they are read: (z - mean[row]) * rstd[row] * gamma[c] + beta[c].
 struct StreamRef {
@@ -28,8 +36,11 @@ gram_status embed_forward(gram_ctx* ctx, const int32_t* item_tokens, const int32
                           cudaStream_t st);
 // seq_len[u] = item_len[item(u)] for the n items of an encoder pass and seq_off = its exclusive prefix sum
 // (seq_off[n] = rows in total)
+// Also: group_list [n] = the sequence numbers grouped by length (SeqGroups), info[0..3] = the size of each group,
+// info[4] = rows in total (device words the caller reads back).
 gram_status sequence_layout(gram_ctx* ctx, const int32_t* item_len, const int32_t* items, int32_t first_item, int32_t n,
-                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, cudaStream_t st);
+                            int32_t n_items_total, int l_t, int32_t* seq_len, int32_t* seq_off, int32_t* group_list,
+                            int32_t* info, cudaStream_t st);
 
 // y = LayerNorm(z): z is the fp32 stream, y the operand-typed copy the next matrix product reads
 gram_status layernorm_forward(gram_ctx* ctx, int dtype, const float* z, const float* gamma, const float* beta, void* y,
@@ -45,20 +56,24 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 // seq_len (may be null): only the first seq_len[s] rows of sequence s are keys; the rows after them are padding,
 // whose outputs are finite and never read, and whose gradients are zero.  seq_off (may be null, needs seq_len): packed
 // rows, sequence s is rows seq_off[s] .. seq_off[s] + seq_len[s] (at most S of them) and there is no padding.
+// groups (may be null, packed rows only): the sequences grouped by length, see SeqGroups.
 gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
+                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+                              const SeqGroups* groups, cudaStream_t st);
 // colpart (may be null; only where attention_mma_supported and dtype is bf16): fp32 [n_seq, 3d], row s receives the
 // column sums of sequence s's rows of dqkv, the partial sums of the bias gradient of the Q, K, V projection
 gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
                                int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
-                               const int32_t* seq_off, cudaStream_t st);
+                               const int32_t* seq_off, const SeqGroups* groups, cudaStream_t st);
 
 // the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
 bool attention_mma_supported(int S, int d, int n_heads);
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
-                                  int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
+                                  int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,
+                                  cudaStream_t st);
 gram_status attention_backward_mma(gram_ctx* ctx, const void* qkv, const void* dctx, void* dqkv, float* colpart, int64_t n_seq, int S, int d,
-                                   int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
+                                   int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+                                   const int32_t* seq_list, cudaStream_t st);
 
 // out[n] += sum_rows X[r, n]   (X operand-typed)
 // out[c] += sum over the nrows rows of part[., c] (fp32 [nrows, N]; partial column sums left by a fused producer)

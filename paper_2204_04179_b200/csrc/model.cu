@@ -39,6 +39,8 @@ struct Stack {
   const int32_t* seq_len = nullptr;        // per sequence: rows that are text (null: all S); set per pass
   const int32_t* seq_off = nullptr;        // packed rows: first row of each sequence (null: sequence s starts at row s*S)
   int64_t packed_rows = 0;                 // packed rows: rows in total (0: n_seq * S)
+  SeqGroups groups;                        // packed rows: the sequences grouped by length
+  bool grouped = false;
   std::vector<LayerOff> off;
   std::vector<LayerActs> acts;
   // backward scratch: the gradient stream (fp32, two buffers) and operand-typed branch gradients
@@ -103,6 +105,8 @@ struct Model {
   int32_t* item_len_buf = nullptr;   // its storage
   int32_t* seq_len = nullptr;        // [mb] the same for the items of the current encoder pass
   int32_t* seq_off = nullptr;        // [mb + 1] first packed row of each of them; [n] = rows of the pass
+  int32_t* seq_groups = nullptr;     // [mb] their numbers grouped by length (for the attention kernels' tile sizes)
+  int32_t* seq_info = nullptr;       // [8] group sizes and the row total, read back by the host
   int64_t saved_rows = 0;            // token rows of the last encoder pass (packed when the texts differ in length)
   int32_t mb = 0;                    // items per encoder pass
   int32_t saved_n = -1;              // items whose activations the last encoder pass saved (-1: none)
@@ -131,7 +135,7 @@ struct Model {
   char* arena = nullptr;
   size_t arena_bytes = 0;
   cudaEvent_t ev[8] = {};
-  int32_t* h_pinned = nullptr;       // [4] pinned host words for small read-backs
+  int32_t* h_pinned = nullptr;       // [16] pinned host words for small read-backs
 };
 
 // the Noam curve scaled to peak at update `warmup` (Section A; Vaswani et al. 2017, Eq. 3)
@@ -197,6 +201,8 @@ void layout_buffers(Model* m, Arena& a) {
     m->item_len_buf = (int32_t*)a.take((size_t)c.n_items * 4);
     m->seq_len = (int32_t*)a.take((size_t)m->mb * 4);
     m->seq_off = (int32_t*)a.take(((size_t)m->mb + 1) * 4);
+    m->seq_groups = (int32_t*)a.take((size_t)m->mb * 4);
+    m->seq_info = (int32_t*)a.take(8 * 4);
     stack_buffers(a, m->enc, esz);
     if (m->cls_tail) {
       stack_buffers(a, m->tail, esz);
@@ -312,7 +318,7 @@ gram_status layer_attention_forward(Model* m, Module& mod, Stack& s, int l, cons
   e.bias = mod.w + o.bqkv;
   e.tag = "fwd_qkv";
   GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * s.d, s.d, e, st));
-  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, s.seq_off, st);
+  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, s.seq_off, s.grouped ? &s.groups : nullptr, st);
 }
 
 // the row-wise rest of the layer over T rows: output projection + residual, LayerNorm, feed-forward + residual,
@@ -433,7 +439,7 @@ gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, con
   const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
                           (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
   GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
-                              s.causal, s.seq_len, s.seq_off, st));
+                              s.causal, s.seq_len, s.seq_off, s.grouped ? &s.groups : nullptr, st));
   if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, m->red, st));
   else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, m->red, st));
   GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
@@ -478,10 +484,19 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   const int32_t* seq_off = nullptr;
   int64_t T = (int64_t)n * c.l_t;
   if (m->item_len) {
-    GRAM_TRY(sequence_layout(ctx, m->item_len, d_items, first_item, n, c.n_items, c.l_t, m->seq_len, m->seq_off, st));
-    int32_t rows = 0;
-    GRAM_TRY(read_i32(m, m->seq_off + n, &rows, st));
-    if (rows < n || rows > T) return gram_set_error(ctx, "encoder pass: %d token rows for %d items", rows, n), GRAM_ERR_ID_RANGE;
+    GRAM_TRY(sequence_layout(ctx, m->item_len, d_items, first_item, n, c.n_items, c.l_t, m->seq_len, m->seq_off,
+                             m->seq_groups, m->seq_info, st));
+    GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 4, m->seq_info, 5 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    GRAM_CUDA(ctx, cudaStreamSynchronize(st));
+    const int32_t rows = m->h_pinned[8];
+    int32_t in_groups = 0;
+    for (int gi = 0; gi < 4; ++gi) {
+      m->enc.groups.count[gi] = m->h_pinned[4 + gi];
+      in_groups += m->h_pinned[4 + gi];
+    }
+    if (rows < n || rows > T || in_groups != n)
+      return gram_set_error(ctx, "encoder pass: %d token rows, %d grouped sequences for %d items", rows, in_groups, n), GRAM_ERR_ID_RANGE;
+    m->enc.groups.list = m->seq_groups;
     T = rows;
     seq_len = m->seq_len;
     seq_off = m->seq_off;
@@ -489,6 +504,7 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   m->enc.seq_len = seq_len;
   m->enc.seq_off = seq_off;
   m->enc.packed_rows = seq_off ? T : 0;
+  m->enc.grouped = seq_off != nullptr;
   m->saved_rows = T;
   GRAM_TRY(embed_forward(ctx, d_item_tokens ? d_item_tokens : m->item_tokens, d_items, first_item, n, c.n_items, c.l_t,
                          c.vocab, c.d, m->ce.w + m->o_tok, m->ce.w + m->o_pos, m->z0, m->tok_ids, seq_len, seq_off, st));
@@ -745,7 +761,7 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   real.base = m->arena;
   layout_buffers(m, real);
   for (int i = 0; i < 8; ++i) GRAM_CUDA(ctx, cudaEventCreate(&m->ev[i]));
-  GRAM_CUDA(ctx, cudaMallocHost(&m->h_pinned, 16));
+  GRAM_CUDA(ctx, cudaMallocHost(&m->h_pinned, 16 * sizeof(int32_t)));
   return GRAM_OK;
 }
 
