@@ -304,7 +304,7 @@ def run_gram(args, shape):
                 "launches": gm["launches"], "avg_launch_ms": gm["ms"] / max(1, gm["launches"]),
                 "share_of_step": gm["ms"] / (ms_total if ms_total > 0 else 1)}
     per_row = gemm_traffic_per_row()
-    if per_row is not None and shape.dtype == "bf16":
+    if per_row is not None and shape.dtype == "bf16" and lengths is None:      # rows per launch are known only for fixed-length texts
         roofline["traffic"] = per_row * statistics.mean(r.n_unique for r in reports) * shape.l_t
     stage_ms = {k: statistics.mean(getattr(r, k) for r in reports)
                 for k in ("ms_dedup", "ms_encode", "ms_gather", "ms_task", "ms_accumulate", "ms_backward", "ms_total")}

@@ -895,7 +895,7 @@ gram_status model_get_window(Model* m, float* h_table, uint32_t* h_touched, floa
   if (h_table) GRAM_CUDA(m->ctx, cudaMemcpy(h_table, m->table, (size_t)c.n_items * c.d * 4, cudaMemcpyDeviceToHost));
   if (h_touched) GRAM_CUDA(m->ctx, cudaMemcpy(h_touched, m->touched, (size_t)((c.n_items + 31) / 32) * 4, cudaMemcpyDeviceToHost));
   if (h_cache) {
-    // convert through the gradient buffer G is too small in general: stage through dE-sized chunks
+    // converted to fp32 on the device through the per-position gradient buffer, a batch's worth of rows at a time
     const size_t rows_per = (size_t)((int64_t)c.B_max * c.L);
     for (size_t r0 = 0; r0 < (size_t)c.n_items; r0 += rows_per) {
       const size_t nr = ((size_t)c.n_items - r0 < rows_per) ? (size_t)c.n_items - r0 : rows_per;
