@@ -83,7 +83,8 @@ __device__ __forceinline__ void load_a_trans(const bf16* S, int ld, int k0, int 
 // scores of 16 query rows against all SP keys: p[nt][0..3] for key tile nt, normalised probabilities on return.
 // MASK = false: every key is visible to every row (S == SP, no causal mask), the per-element tests are left out.
 // The 1/sqrt(dh) scale is folded into the exponent: exp(scale (s - max s)) = exp2(c s - c max s), c = scale log2(e).
-template <int SP, int DH, bool MASK>
+// SKIP (causal launches): key tiles that no row of this query tile can see are not multiplied at all.
+template <int SP, int DH, bool MASK, bool SKIP = false>
 __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf16* __restrict__ Ks, int r0, int S, int causal,
                                            float scale, int g, int q, float (&p)[SP / 8][4]) {
   constexpr int LD = DH + 8;
@@ -96,10 +97,12 @@ __device__ __forceinline__ void score_rows(const bf16* __restrict__ Qs, const bf
     load_a_rows(Qs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
 #pragma unroll
     for (int nt = 0; nt < SP / 8; nt += 2) {
-      uint32_t b0, b1, b2, b3;
-      load_b_rows(Ks, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
-      mma16816(p[nt], a0, a1, a2, a3, b0, b1);
-      mma16816(p[nt + 1], a0, a1, a2, a3, b2, b3);
+      if (!SKIP || nt * 8 <= r0 + 15) {        // later keys are masked for every row of the tile: their scores stay 0, then -inf
+        uint32_t b0, b1, b2, b3;
+        load_b_rows(Ks, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
+        mma16816(p[nt], a0, a1, a2, a3, b0, b1);
+        mma16816(p[nt + 1], a0, a1, a2, a3, b2, b3);
+      }
     }
   }
   const int i0 = r0 + g, i1 = r0 + g + 8;
@@ -186,12 +189,14 @@ __device__ __forceinline__ void stage_tile(const float (&o)[DH / 8][4], bf16* __
 }
 
 // acc[nt] += A(16 x SP, from the C-layout registers x) * S[k][n] (row-major, SP x DH)
-template <int SP, int DH>
+// LIMIT: the columns of x from n_rows on are zero (keys a causal tile cannot see), their 16-row tiles are skipped.
+template <int SP, int DH, bool LIMIT = false>
 __device__ __forceinline__ void mma_regs_times_rows(const float (&x)[SP / 8][4], const bf16* S, int lane,
-                                                    float (&acc)[DH / 8][4]) {
+                                                    float (&acc)[DH / 8][4], int n_rows = 0) {
   constexpr int LD = DH + 8;
 #pragma unroll
   for (int kt = 0; kt < SP / 16; ++kt) {
+    if (LIMIT && kt * 16 >= n_rows) continue;
     const uint32_t a0 = pack2(x[2 * kt][0], x[2 * kt][1]), a1 = pack2(x[2 * kt][2], x[2 * kt][3]);
     const uint32_t a2 = pack2(x[2 * kt + 1][0], x[2 * kt + 1][1]), a3 = pack2(x[2 * kt + 1][2], x[2 * kt + 1][3]);
 #pragma unroll
@@ -204,8 +209,9 @@ __device__ __forceinline__ void mma_regs_times_rows(const float (&x)[SP / 8][4],
   }
 }
 
-template <int SP, int DH>
-__global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
+// NW warps per block; CAUSAL launches skip the tiles above the diagonal.
+template <int SP, int DH, int NW, bool CAUSAL>
+__global__ void __launch_bounds__(NW * 32) attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int S, int d,
                                                            int n_heads, int causal, float scale,
                                                            const int32_t* __restrict__ seq_len,
                                                            const int32_t* __restrict__ seq_off,
@@ -230,14 +236,14 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   bf16* ob = out + row0 * (int64_t)d + h * DH;
   const int Sv = seq_len ? seq_len[seq] : S;      // keys that are text; the rows after them are padding
-  for (int r0 = warp * 16; r0 < S; r0 += 64) {
+  for (int r0 = warp * 16; r0 < S; r0 += NW * 16) {
     float p[SP / 8][4];
-    if (Sv == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
-    else score_rows<SP, DH, true>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+    if (!CAUSAL && Sv == SP) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+    else score_rows<SP, DH, true, CAUSAL>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
     float o[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-    mma_regs_times_rows<SP, DH>(p, Vs, lane, o);              // O = P V
+    mma_regs_times_rows<SP, DH, CAUSAL>(p, Vs, lane, o, r0 + 16);              // O = P V
     // the 16 rows of Q are this warp's alone and no longer needed: O goes through them so that it leaves in whole rows
     __syncwarp();
     stage_tile<DH>(o, Qs, r0, g, q);
@@ -246,8 +252,8 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const bf16* __restric
   }
 }
 
-template <int SP, int DH>
-__global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
+template <int SP, int DH, int NW, bool CAUSAL>
+__global__ void __launch_bounds__(NW * 32) attn_bwd_mma_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dctx,
                                                            bf16* __restrict__ dqkv, float* __restrict__ colpart, int S, int d,
                                                            int n_heads, int causal, float scale,
                                                            const int32_t* __restrict__ seq_len,
@@ -278,15 +284,15 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   bf16* dq = dqkv + row0 * 3 * (int64_t)d + h * DH;
   const int Sv = seq_len ? seq_len[seq] : S;
   // ---- first half: 16 query rows per warp: P, dS (kept in shared memory), dQ (kept in registers as bf16 pairs) ----
-  constexpr int NIT = (SP + 63) / 64;
+  constexpr int NIT = (SP + 16 * NW - 1) / (16 * NW);
   uint32_t dqp[NIT][DH / 8][2];
 #pragma unroll
   for (int it = 0; it < NIT; ++it) {
-    const int r0 = warp * 16 + it * 64;
+    const int r0 = warp * 16 + it * (16 * NW);
     if (r0 < SP) {
       float p[SP / 8][4];
-      if (Sv == SP && !causal) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
-      else score_rows<SP, DH, true>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+      if (!CAUSAL && Sv == SP) score_rows<SP, DH, false>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
+      else score_rows<SP, DH, true, CAUSAL>(Qs, Ks, r0, Sv, causal, scale, g, q, p);
       float dp[SP / 8][4];
 #pragma unroll
       for (int nt = 0; nt < SP / 8; ++nt) dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
@@ -296,10 +302,12 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
         load_a_rows(dOs, LD, r0, kt * 16, lane, a0, a1, a2, a3);
 #pragma unroll
         for (int nt = 0; nt < SP / 8; nt += 2) {
-          uint32_t b0, b1, b2, b3;
-          load_b_rows(Vs, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
-          mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
-          mma16816(dp[nt + 1], a0, a1, a2, a3, b2, b3);
+          if (!CAUSAL || nt * 8 <= r0 + 15) {   // the probabilities of keys out of sight are zero: dP there is not needed
+            uint32_t b0, b1, b2, b3;
+            load_b_rows(Vs, LD, nt * 8, kt * 16, lane, b0, b1, b2, b3);
+            mma16816(dp[nt], a0, a1, a2, a3, b0, b1);
+            mma16816(dp[nt + 1], a0, a1, a2, a3, b2, b3);
+          }
         }
       }
       float d0 = 0.f, d1 = 0.f;
@@ -323,7 +331,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
       float o[DH / 8][4];
 #pragma unroll
       for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-      mma_regs_times_rows<SP, DH>(dp, Ks, lane, o);             // dQ = dS K
+      mma_regs_times_rows<SP, DH, CAUSAL>(dp, Ks, lane, o, r0 + 16);             // dQ = dS K
 #pragma unroll
       for (int nt = 0; nt < DH / 8; ++nt) {
         dqp[it][nt][0] = pack2(o[nt][0], o[nt][1]);
@@ -334,7 +342,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   __syncthreads();
   // ---- second half: 16 key rows per warp: dK = dS^T Q, dV = P^T dO; K and V are no longer read, so the results
   // ---- replace this warp's rows of them
-  for (int j0 = warp * 16; j0 < S; j0 += 64) {
+  for (int j0 = warp * 16; j0 < S; j0 += NW * 16) {
     float dk[DH / 8][4], dv[DH / 8][4];
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) {
@@ -343,6 +351,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
     }
 #pragma unroll
     for (int kt = 0; kt < SP / 16; ++kt) {        // contraction over query rows i = kt*16 ..
+      if (CAUSAL && kt * 16 + 15 < j0) continue;  // queries before these keys cannot see them: P and dS are zero there
       uint32_t s0, s1, s2, s3, p0, p1, p2, p3;
       load_a_trans(dSs, LP, kt * 16, j0, lane, s0, s1, s2, s3);
       load_a_trans(Ps, LP, kt * 16, j0, lane, p0, p1, p2, p3);
@@ -363,7 +372,7 @@ __global__ void __launch_bounds__(128) attn_bwd_mma_kernel(const bf16* __restric
   __syncthreads();                                 // Q is no longer read either: dQ replaces it
 #pragma unroll
   for (int it = 0; it < NIT; ++it) {
-    const int r0 = warp * 16 + it * 64;
+    const int r0 = warp * 16 + it * (16 * NW);
     if (r0 < SP) {
 #pragma unroll
       for (int nt = 0; nt < DH / 8; ++nt) {
@@ -394,9 +403,10 @@ template <int SP, int DH>
 gram_status launch_fwd(gram_ctx* ctx, const bf16* qkv, bf16* out, int64_t n_seq, int S, int d, int n_heads, int causal,
                        const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list, cudaStream_t st) {
   constexpr size_t smem = (size_t)3 * SP * (DH + 8) * 2;
-  auto kern = attn_fwd_mma_kernel<SP, DH>;
+  constexpr int NW = SP >= 96 ? 8 : 4;                // one 16-row query tile per warp up to 128 rows
+  auto kern = causal ? attn_fwd_mma_kernel<SP, DH, NW, true> : attn_fwd_mma_kernel<SP, DH, NW, false>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
+  kern<<<(unsigned)(n_seq * n_heads), NW * 32, smem, st>>>(qkv, out, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -406,9 +416,10 @@ gram_status launch_bwd(gram_ctx* ctx, const bf16* qkv, const bf16* dctx, bf16* d
                        cudaStream_t st) {
   constexpr size_t smem = ((size_t)4 * SP * (DH + 8) + (size_t)2 * SP * (SP + 8)) * 2;
   static_assert(smem <= 227 * 1024, "attention backward tile exceeds shared memory");
-  auto kern = attn_bwd_mma_kernel<SP, DH>;
+  constexpr int NW = SP >= 96 ? 8 : 4;
+  auto kern = causal ? attn_bwd_mma_kernel<SP, DH, NW, true> : attn_bwd_mma_kernel<SP, DH, NW, false>;
   if (smem > 48 * 1024) GRAM_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<(unsigned)(n_seq * n_heads), 128, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
+  kern<<<(unsigned)(n_seq * n_heads), NW * 32, smem, st>>>(qkv, dctx, dqkv, colpart, S, d, n_heads, causal, 1.f / sqrtf((float)DH), seq_len, seq_off, seq_list);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
