@@ -442,20 +442,24 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, in
   }
 }
 
-__global__ void periodic_rowsum_kernel(const float* __restrict__ X, int64_t n_groups, int period, int d,
-                                       float* __restrict__ out, const int32_t* __restrict__ seq_len,
-                                       const int32_t* __restrict__ seq_off) {
+// blockIdx.y owns the groups [y * per, (y + 1) * per) and leaves their sum in part[y][period * d]; with one chunk
+// (part == null) the sum is added to out directly
+__global__ void periodic_rowsum_kernel(const float* __restrict__ X, int64_t n_groups, int64_t per, int period, int d,
+                                       float* __restrict__ out, float* __restrict__ part,
+                                       const int32_t* __restrict__ seq_len, const int32_t* __restrict__ seq_off) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)period * d) return;
   const int s = (int)(i / d), c = (int)(i - (int64_t)s * d);
+  const int64_t u0 = (int64_t)blockIdx.y * per, u1 = min(u0 + per, n_groups);
   float acc = 0.f;
   if (seq_off) {                                   // packed rows: group u has seq_len[u] rows starting at seq_off[u]
-    for (int64_t u = 0; u < n_groups; ++u)
+    for (int64_t u = u0; u < u1; ++u)
       if (s < seq_len[u]) acc += X[((int64_t)seq_off[u] + s) * d + c];
   } else {
-    for (int64_t u = 0; u < n_groups; ++u) acc += X[(u * period + s) * d + c];
+    for (int64_t u = u0; u < u1; ++u) acc += X[(u * period + s) * d + c];
   }
-  out[i] += acc;
+  if (part) part[(int64_t)blockIdx.y * period * d + i] = acc;
+  else out[i] += acc;
 }
 
 // ---------------------------------------------------------------------------- pooling
@@ -1020,11 +1024,20 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
 }
 
 gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
-                                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
+                                       float* scratch, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st) {
   if (n_groups == 0) return GRAM_OK;
   const int64_t n = (int64_t)period * d;
-  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n_groups * period * d, 1, st);
-  periodic_rowsum_kernel<<<(unsigned)ceil_div64(n, 128), 128, 0, st>>>(X, n_groups, period, d, out, seq_len, seq_off);
+  // the groups are cut into chunks that are summed side by side; the chunk sums are then added in ascending order
+  int64_t chunks = n_groups / 64;
+  const int64_t fit = (int64_t)(kRedScratchBytes / sizeof(float)) / n;
+  if (chunks > 64) chunks = 64;
+  if (chunks > fit) chunks = fit;
+  if (chunks < 2 || !scratch || n > INT32_MAX) chunks = 1;
+  const int64_t per = ceil_div64(n_groups, chunks);
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n_groups * period * d, chunks > 1 ? 2 : 1, st);
+  dim3 grid((unsigned)ceil_div64(n, 128), (unsigned)chunks);
+  periodic_rowsum_kernel<<<grid, 128, 0, st>>>(X, n_groups, per, period, d, out, chunks > 1 ? scratch : nullptr, seq_len, seq_off);
+  if (chunks > 1) reduce_partials_kernel<<<ceil_div((int)n, 32), 256, 0, st>>>(scratch, (int)chunks, n, (int)n, out, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

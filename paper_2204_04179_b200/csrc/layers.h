@@ -83,8 +83,9 @@ gram_status colsum_accumulate(gram_ctx* ctx, int dtype, const void* X, int64_t r
                               cudaStream_t st);
 // out[s, :] += sum_u X[u*period + s, :]  (s < period; X fp32)
 // packed rows (seq_len, seq_off not null): out[s, :] += sum over the groups u with s < seq_len[u] of X[seq_off[u] + s, :]
+// scratch (may be null): kRedScratchBytes of reduction scratch, lets the groups be summed in parallel chunks
 gram_status periodic_rowsum_accumulate(gram_ctx* ctx, const float* X, int64_t n_groups, int period, int d, float* out,
-                                       const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
+                                       float* scratch, const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 
 // H[u, :] = mean_s x[u*l_t + s, :] (mean; over the first seq_len[u] tokens when seq_len is given) or x[u*l_t, :] (cls), fp32
 gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n, int l_t, int d, int pooling,

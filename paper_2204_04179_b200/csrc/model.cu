@@ -567,7 +567,7 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   float* dz0 = (dx0 == m->enc.curf) ? m->enc.othf : m->enc.curf;
   GRAM_TRY(layernorm_backward(ctx, m->dtype, dx0, m->z0, m->mean0, m->rstd0, m->ce.w + m->o_elng, dz0, nullptr,
                               m->ce.g + m->o_elng, m->ce.g + m->o_elnb, nullptr, m->red, T, c.d, st));
-  GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, seq_len, seq_off, st));
+  GRAM_TRY(periodic_rowsum_accumulate(ctx, dz0, n, c.l_t, c.d, m->ce.g + m->o_pos, m->red, seq_len, seq_off, st));
   // token-embedding gradient: sum dz0 over the occurrences of each token (same index kernels as stage 1 / 4)
   IndexWorkspace* iws = gram_index_ws(ctx);
   GRAM_TRY(dedup_launch(ctx, iws, m->tok_ids, T, c.vocab, m->tok_unique, m->tok_inverse, m->tok_perm, m->tok_seg, m->tok_nu, st));
