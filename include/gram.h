@@ -171,6 +171,14 @@ gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n
 gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, const int32_t* d_items, int32_t U,
                                float* d_H, int save_activations, gram_stream stream);
 
+/* Failure detection: every wait of one thread block on another (the tile look-back of gram_dedup, the pipeline
+ * barriers of the matrix products) has a poll limit, after which the kernel records GRAM_ERR_TIMEOUT in the context,
+ * writes nothing more and returns, so that a stuck wait costs about a second instead of the device.  This call shows
+ * it: it launches the dedup's run-length kernel with a predecessor tile that never runs.  It returns GRAM_OK once the
+ * launch is queued; the next gram_sync takes about a second and returns GRAM_ERR_TIMEOUT; the context stays usable.
+ * (No counterpart in the paper.) */
+gram_status gram_selftest_bounded_wait(gram_ctx* ctx, gram_stream stream);
+
 /* Stage 3: d_E[p, :] = d_src[d_index[p], :] for p < P.  Single-step: src = H,
  * index = inverse.  Multi-step: src = the encoding cache, index = ids.
  * Rows are d elements of `dtype`; n_src_rows bounds the index (ID_RANGE else). */

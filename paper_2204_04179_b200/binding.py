@@ -34,7 +34,7 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
            "gram_launch_count", "gram_profile_dump", "gram_accumulate_static", "gram_optimizer_step",
            "gram_optimizer_reset", "gram_noam_rate", "gram_adam_update", "gram_state_export", "gram_state_import",
-           "gram_optimizer_export", "gram_optimizer_import"]
+           "gram_optimizer_export", "gram_optimizer_import", "gram_selftest_bounded_wait"]
 
 KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other",
          "optimizer"]
@@ -200,6 +200,10 @@ class Gram:
         lengths = np.ascontiguousarray(lengths, dtype=np.int32)
         assert lengths.size == self.cfg.n_items
         self._ck(lib().gram_set_item_lengths(self._h, _ptr(lengths)))
+
+    def selftest_bounded_wait(self, stream=None):
+        """Queues a wait that nothing satisfies; the next sync() raises GramError with status GRAM_ERR_TIMEOUT."""
+        self._ck(lib().gram_selftest_bounded_wait(self._h, _stream(stream)))
 
     # stages
     def dedup(self, ids, n_items, unique, inverse, perm, seg_off, n_unique, stream=None):

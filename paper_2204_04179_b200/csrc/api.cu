@@ -238,6 +238,10 @@ gram_status gram_dedup(gram_ctx* ctx, const int32_t* d_ids, int64_t P, int32_t n
   return dedup_launch(ctx, &ctx->iws, d_ids, P, n_items, d_unique, d_inverse, d_perm, d_seg_off, d_n_unique, S(stream));
 }
 
+gram_status gram_selftest_bounded_wait(gram_ctx* ctx, gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  return dedup_wait_selftest(ctx, &ctx->iws, S(stream));
+}
 gram_status gram_gather(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
                         int32_t d, int dtype, void* d_E, gram_stream stream) {
   if (!ctx) return GRAM_ERR_ARG;

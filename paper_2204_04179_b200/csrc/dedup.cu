@@ -475,6 +475,22 @@ void index_ws_free(IndexWorkspace* ws) {
   *ws = IndexWorkspace();
 }
 
+// A wait that nothing satisfies, to show that it ends: the run-length kernel is launched as tile 1 of a
+// one-key input whose tile 0 never runs, so its look-back finds no status word, gives up after kSpinLimit
+// polls (about a second), records GRAM_ERR_TIMEOUT and writes nothing.
+gram_status dedup_wait_selftest(gram_ctx* ctx, IndexWorkspace* ws, cudaStream_t st) {
+  if (ws->P_max < 2) return gram_set_error(ctx, "the bounded-wait self-test needs a context with P_max >= 2"), GRAM_ERR_WORKSPACE;
+  uint32_t* ctl = ws->sort_ctl;
+  GRAM_CUDA(ctx, cudaMemsetAsync(ctl, 0, (size_t)(CTL_WORDS + 2) * sizeof(uint32_t), st));
+  static const int32_t one = 1;
+  GRAM_CUDA(ctx, cudaMemcpyAsync(reinterpret_cast<int32_t*>(ctl) + CTL_RLE_TICKET, &one, sizeof(one), cudaMemcpyHostToDevice, st));
+  GRAM_CUDA(ctx, cudaMemsetAsync(ws->keys0, 0, sizeof(int32_t), st));
+  rle_kernel<<<1, RLE_THREADS, 0, st>>>(ws->keys0, 1, 2, 1, 1, ctl + CTL_WORDS, reinterpret_cast<int32_t*>(ctl) + CTL_RLE_TICKET,
+                                        ws->keys1, ws->vals0, ws->rank_table, ws->vals1, gram_status_word(ctx));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
 gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids, int64_t P, int32_t n_items,
                          int32_t* d_unique, int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off,
                          int32_t* d_n_unique, cudaStream_t st) {

@@ -59,6 +59,8 @@ gram_status dedup_launch(gram_ctx* ctx, IndexWorkspace* ws, const int32_t* d_ids
                          int32_t* d_unique, int32_t* d_inverse, int32_t* d_perm, int32_t* d_seg_off,
                          int32_t* d_n_unique, cudaStream_t st);
 
+gram_status dedup_wait_selftest(gram_ctx* ctx, IndexWorkspace* ws, cudaStream_t st);
+
 gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
                           int32_t d, int elem_bytes, void* d_E, cudaStream_t st);
 

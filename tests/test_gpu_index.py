@@ -236,3 +236,21 @@ def test_largest_sweep_cell(s):
         sl = slice(p0, min(P, p0 + 2_000_000))
         assert torch.equal(E[sl], H[inv_d[sl].long()])
     g.close()
+
+
+def test_a_wait_that_nothing_satisfies_ends_with_a_status():
+    """The look-back of the dedup's run-length kernel, started as a tile whose predecessor never runs, gives up after its
+    poll limit: the host reads GRAM_ERR_TIMEOUT, nothing faults, and the context keeps working."""
+    import time
+    g = index_ctx(4096, 100)
+    g.selftest_bounded_wait()
+    t0 = time.time()
+    with pytest.raises(binding.GramError) as e:
+        g.sync()
+    assert e.value.status == 6
+    assert time.time() - t0 < 30
+    ids = synth.zipf_ids(2, 100, 1.1, 4096)
+    U, unique, inverse, perm, seg_off = run_dedup(g, ids, 100)
+    want = orc.unique_inverse(ids)
+    assert U == len(want[0]) and np.array_equal(inverse, want[1]) and np.array_equal(perm, want[2])
+    g.close()
