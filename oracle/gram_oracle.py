@@ -355,7 +355,8 @@ def encode_all(shape, ce_params, item_tokens, items, dtype=torch.float64) -> np.
 
 
 def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache, lr_task: float,
-                     cache_bf16: bool = False, dtype=torch.float64):
+                     cache_bf16: bool = False, dtype=torch.float64, lr_ce: Optional[float] = None,
+                     refresh_after_update: bool = False):
     """One window of K = len(batches) steps of Algorithm 1, then the encoder
     pass.  Readings where the algorithm is silent or ambiguous:
 
@@ -373,9 +374,15 @@ def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache,
       window, with cotangent table[i]; its forward uses the current encoder
       parameters, and that forward value replaces cache[i].
 
+    * lr_ce (optional): the encoder then takes a plain SGD step of that rate
+      with the window's gradient (returned as ce_params).  With
+      refresh_after_update the touched items are encoded once more with the
+      updated parameters and those values go to the cache, which is Eq. 4 read
+      literally (h is produced with the parameters of the current step).
+
     Returns dict(losses [K], grad_ce (sum over touched items in ascending item
     order), grad_task_last, task_params (after K SGD steps), table, touched,
-    cache (updated))."""
+    cache (updated), ce_params (after the step, when lr_ce is given))."""
     n_items, d = cache.shape
     cache = np.array(cache, dtype=np.float64)
     if cache_bf16:
@@ -402,9 +409,15 @@ def multistep_window(shape, ce_params, task_params, item_tokens, batches, cache,
     H = torch.stack([ce_forward(th_ce, item_tokens[int(i)], shape) for i in items])
     H.backward(torch.tensor(table[items], dtype=dtype))
     newc = H.detach().numpy()
+    grad_ce = _grads(th_ce)
+    new_ce = None
+    if lr_ce is not None:
+        new_ce = OrderedDict((k, np.asarray(v, dtype=np.float64) - lr_ce * grad_ce[k]) for k, v in ce_params.items())
+        if refresh_after_update:
+            newc = encode_all(shape, new_ce, item_tokens, items, dtype)
     cache[items] = round_to_bf16(newc) if cache_bf16 else newc
-    return dict(losses=losses, grad_ce=_grads(th_ce), grad_task_last=grad_task_last, task_params=cur_task,
-                table=table, touched=touched, cache=cache, items=items.astype(np.int32))
+    return dict(losses=losses, grad_ce=grad_ce, grad_task_last=grad_task_last, task_params=cur_task,
+                table=table, touched=touched, cache=cache, items=items.astype(np.int32), ce_params=new_ce)
 
 
 def multistep_window_pseudo_target(shape, ce_params, task_params, item_tokens, batches, cache, lr_task: float,

@@ -403,3 +403,25 @@ def test_padded_history_is_the_shorter_history():
     lab_all = lab.copy(); lab_all[1, n:] = 0
     with torch.no_grad():
         assert abs(float(orc.task_loss(th, E, lab_all, shape)) - float(loss.detach())) > 1e-6
+
+
+def test_refreshed_cache_makes_one_step_windows_end_to_end_training():
+    # windows of one step, SGD on the encoder, cache refreshed after the update: when the next batch only uses items the
+    # previous one touched, its loss and gradient are those of end-to-end training at the updated parameters (Eq. 4
+    # with the parameters of the current step); without the refresh the cache is one update stale and they differ
+    shape = small_shape(pooling="cls")
+    ce, tk, toks, ids, lab = make(shape, seed=14)
+    cache = orc.encode_all(shape, ce, toks, range(shape.n_items))
+    lr_c = 0.05
+    w1 = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0, lr_ce=lr_c, refresh_after_update=True)
+    lab2 = 1 - lab
+    w2 = orc.multistep_window(shape, w1["ce_params"], tk, toks, [(ids, lab2)], w1["cache"], lr_task=0.0)
+    e2e = orc.e2e_step(shape, w1["ce_params"], tk, toks, ids, lab2)
+    assert abs(w2["losses"][0] - e2e["loss"]) < 1e-12
+    for k in e2e["grad_ce"]:
+        np.testing.assert_allclose(w2["grad_ce"][k], e2e["grad_ce"][k], rtol=1e-9, atol=1e-12)
+    for k in ce:      # and the step itself was plain SGD with the window's gradient
+        np.testing.assert_allclose(w1["ce_params"][k], np.asarray(ce[k], np.float64) - lr_c * w1["grad_ce"][k], rtol=0, atol=0)
+    stale = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0, lr_ce=lr_c)
+    s2 = orc.multistep_window(shape, stale["ce_params"], tk, toks, [(ids, lab2)], stale["cache"], lr_task=0.0)
+    assert abs(s2["losses"][0] - e2e["loss"]) > 1e-7
