@@ -93,6 +93,10 @@ typedef struct gram_config {
   int32_t noam_warmup;         /* updates until the peak rate; <= 0: constant rate */
   float adam_beta1, adam_beta2, adam_eps;   /* <= 0: 0.9, 0.999, 1e-8 */
   int32_t multistep_variant;   /* K > 1: GRAM_MULTI_TABLE or GRAM_MULTI_PSEUDO_TARGET */
+  int32_t refresh_after_update; /* K > 1: after the encoder update at the end of a window, encode the touched items once
+                                   more with the new parameters and store those encodings in the cache (Algorithm 1,
+                                   Eq. 4 produces h with the parameters of the current step); 0: the cache keeps the
+                                   forward values of the encoder pass, one update old */
 } gram_config;
 
 typedef struct gram_step_report {

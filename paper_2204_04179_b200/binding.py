@@ -47,7 +47,7 @@ class GramConfig(C.Structure):
                [("P_max", C.c_int64), ("d_max", C.c_int32), ("K", C.c_int32), ("ce_micro_batch", C.c_int32),
                 ("lr_task", C.c_float), ("lr_ce", C.c_float), ("optimizer", C.c_int32), ("noam_warmup", C.c_int32),
                 ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float),
-                ("multistep_variant", C.c_int32)]
+                ("multistep_variant", C.c_int32), ("refresh_after_update", C.c_int32)]
 
 
 class GramStepReport(C.Structure):

@@ -1053,6 +1053,14 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
                               return gather_launch(ctx, m->table, c.n_items, m->tlist + u0, n, c.d, 4, m->G, st);
                             }, st));
       GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+      if (c.refresh_after_update) {      // Eq. 4 with the updated parameters: the next window reads fresh encodings
+        for (int32_t u0 = 0; u0 < n_touched; u0 += m->mb) {
+          const int32_t n = (n_touched - u0 < m->mb) ? n_touched - u0 : m->mb;
+          GRAM_TRY(encoder_forward_chunk(m, nullptr, m->tlist + u0, 0, n, m->H, st));
+          GRAM_TRY(scatter_rows(ctx, m->cache_dtype, m->H, m->tlist + u0, n, c.d, c.n_items, m->cache, st));
+        }
+        m->saved_n = -1;
+      }
       GRAM_TRY(model_window_reset(m, st));
       n_encoded = n_touched;
       encoder_ran = 1;

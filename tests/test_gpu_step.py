@@ -406,3 +406,33 @@ def test_multistep_window_with_texts_of_different_lengths():
     _, _, cache = g.get_window(want_table=False, want_touched=False)
     assert gh.rel_err(cache, want["cache"]) <= 1e-4
     g.close()
+
+
+def test_multistep_cache_refresh_after_the_encoder_update():
+    """refresh_after_update: after a window's encoder step the touched items are encoded again with the new parameters,
+    so the next window reads fresh encodings (two windows against the oracle; without the flag the cache differs)."""
+    K = 2
+    shape = small(dtype="f32", d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=43)
+    lr_t, lr_c = 0.05, 0.05
+    batches = [synth.batch(shape, 43, step=k) for k in range(2 * K)]
+    g = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=lr_t, lr_ce=lr_c, ce_micro_batch=16, refresh_after_update=1)
+    g.cache_fill()
+    _, _, cache0 = g.get_window(want_table=False, want_touched=False)
+    cur_ce, cur_tk, cache = ce, tk, cache0.astype(np.float64)
+    for w in range(2):
+        want = orc.multistep_window(shape, cur_ce, cur_tk, toks, batches[w * K:(w + 1) * K], cache, lr_task=lr_t, lr_ce=lr_c,
+                                    refresh_after_update=True)
+        reps = [g.step(torch.from_numpy(i).to(DEV), torch.from_numpy(l).to(DEV), shape.B) for i, l in batches[w * K:(w + 1) * K]]
+        for k in range(K):
+            assert abs(reps[k].loss - want["losses"][k]) <= 1e-4 * abs(want["losses"][k]), (w, k)
+        gce, _ = gh.gpu_grads(g, shape)
+        e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+        assert e1 <= 1e-3, (w, e1, n1)
+        _, _, cache_gpu = g.get_window(want_table=False, want_touched=False)
+        assert gh.rel_err(cache_gpu, want["cache"]) <= 1e-4
+        if w == 0:
+            stale = orc.multistep_window(shape, cur_ce, cur_tk, toks, batches[:K], cache, lr_task=lr_t, lr_ce=lr_c)
+            assert gh.rel_err(cache_gpu, stale["cache"]) > 1e-3
+        cur_ce, cur_tk, cache = want["ce_params"], want["task_params"], want["cache"]
+    g.close()
