@@ -205,6 +205,12 @@ def ce_forward(th: Dict[str, torch.Tensor], tokens, shape) -> torch.Tensor:
         return x.mean(dim=0)
     if shape.pooling == "cls":
         return x[0]
+    if shape.pooling == "additive":
+        # additive attention over the item's tokens (Appendix D: the news encoder pools its token outputs with
+        # additive attention): a_s = q . tanh(W x_s + b), alpha = softmax(a), h = sum_s alpha_s x_s
+        a = torch.tanh(x @ th["pool_wa"].T + th["pool_ba"]) @ th["pool_qa"]
+        alpha = softmax_rows(a[None, :])[0]
+        return alpha @ x
     raise KeyError(shape.pooling)
 
 

@@ -42,7 +42,7 @@ class GramShape:
     n_heads: int = 2
     d_ff: int = 256
     n_layers: int = 2
-    pooling: str = "mean"         # "mean" or "cls"
+    pooling: str = "mean"         # "mean", "cls" (token 0) or "additive" (additive attention of width d_a over the tokens)
     # task module
     task: str = "kt"              # "kt" (causal attention over a history) or "nr" (additive attention)
     task_layers: int = 1
@@ -163,6 +163,8 @@ def encoder_param_spec(s: GramShape):
             ("emb_ln_g", (s.d,)), ("emb_ln_b", (s.d,))]
     for l in range(s.n_layers):
         spec += _layer_spec(f"l{l}.", s.d, s.d_ff, False)
+    if s.pooling == "additive":          # additive-attention pooling over an item's tokens (width d_a)
+        spec += [("pool_wa", (s.d_a, s.d)), ("pool_ba", (s.d_a,)), ("pool_qa", (s.d_a,))]
     return spec
 
 

@@ -425,3 +425,46 @@ def test_refreshed_cache_makes_one_step_windows_end_to_end_training():
     stale = orc.multistep_window(shape, ce, tk, toks, [(ids, lab)], cache, lr_task=0.0, lr_ce=lr_c)
     s2 = orc.multistep_window(shape, stale["ce_params"], tk, toks, [(ids, lab2)], stale["cache"], lr_task=0.0)
     assert abs(s2["losses"][0] - e2e["loss"]) > 1e-7
+
+
+# ---- additive-attention pooling of an item's tokens ---------------------------------------------------------------------
+
+def test_additive_pooling_special_cases_and_finite_differences():
+    shape = small_shape(pooling="additive", d_a=6, l_t=5)
+    ce, tk, toks, ids, lab = make(shape, seed=16)
+    ce = OrderedDict((k, np.asarray(v, np.float64)) for k, v in ce.items())
+    th = orc.as_torch(ce, T64, requires_grad=False)
+    # q = 0: every score is equal, the pooled vector is the plain mean of the token outputs
+    z = OrderedDict(ce); z["pool_qa"] = np.zeros_like(ce["pool_qa"])
+    mean_shape = shape.replace(pooling="mean")
+    a = orc.encode_all(shape, z, toks, [0, 3])
+    b = orc.encode_all(mean_shape, {k: v for k, v in ce.items() if not k.startswith("pool_")}, toks, [0, 3])
+    np.testing.assert_allclose(a, b, rtol=1e-13)
+    # one dominant score: a huge q along tanh's saturated sign pattern of one token picks that token's output (convex
+    # combination in general: inside the hull of the token outputs)
+    with torch.no_grad():
+        h = orc.ce_forward(th, toks[1], shape)
+        x = th["tok_emb"][torch.as_tensor(toks[1], dtype=torch.long)] + th["pos_emb"]
+        x = orc.layer_norm(x, th["emb_ln_g"], th["emb_ln_b"])
+        for l in range(shape.n_layers):
+            x = orc.transformer_layer(x, th, f"l{l}.", shape.n_heads, causal=False)
+        al = torch.linalg.lstsq(x.T, h[:, None]).solution[:, 0]            # h = sum alpha_s x_s has a solution ...
+        assert torch.allclose(x.T @ al, h, atol=1e-10)
+        sc = torch.tanh(x @ th["pool_wa"].T + th["pool_ba"]) @ th["pool_qa"]
+        want = torch.softmax(sc, 0)                                           # ... and it is the library softmax of the scores
+        assert torch.allclose(want @ x, h, atol=1e-13) and abs(float(want.sum()) - 1) < 1e-14
+    # gradients of the end-to-end step through the pooling parameters against central differences
+    res = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    def loss_at(params):
+        thp = orc.as_torch(params, T64, requires_grad=False)
+        with torch.no_grad():
+            E = torch.stack([torch.stack([orc.ce_forward(thp, toks[int(i)], shape) for i in row]) for row in ids])
+            return float(orc.task_loss(orc.as_torch(tk, T64, requires_grad=False), E, lab, shape))
+    rng = np.random.default_rng(0)
+    for name in ("pool_wa", "pool_ba", "pool_qa", "l0.w1"):
+        for fi in rng.integers(0, ce[name].size, 2):
+            idx = np.unravel_index(fi, ce[name].shape)
+            up = OrderedDict((k, v.copy()) for k, v in ce.items()); up[name][idx] += 1e-6
+            dn = OrderedDict((k, v.copy()) for k, v in ce.items()); dn[name][idx] -= 1e-6
+            fd = (loss_at(up) - loss_at(dn)) / 2e-6
+            assert abs(fd - res["grad_ce"][name][idx]) <= 1e-7 + 1e-5 * abs(fd), (name, idx, fd, res["grad_ce"][name][idx])
