@@ -45,7 +45,9 @@ typedef enum gram_status {
 } gram_status;
 
 enum { GRAM_F32 = 0, GRAM_BF16 = 1 };                 /* element types */
-enum { GRAM_POOL_MEAN = 0, GRAM_POOL_CLS = 1 };       /* item pooling */
+/* item pooling: mean over the tokens, token 0, or additive attention over the tokens (Appendix D; width d_a):
+ * a_s = q . tanh(W x_s + b), alpha = softmax(a), h = sum_s alpha_s x_s */
+enum { GRAM_POOL_MEAN = 0, GRAM_POOL_CLS = 1, GRAM_POOL_ADDITIVE = 2 };
 enum { GRAM_TASK_NONE = 0, GRAM_TASK_KT = 1, GRAM_TASK_NR = 2 };
 enum { GRAM_MODULE_CE = 0, GRAM_MODULE_TASK = 1 };
 enum { GRAM_OPT_SGD = 0, GRAM_OPT_ADAM = 1 };
@@ -125,7 +127,7 @@ const char* gram_last_error(const gram_ctx* ctx);
 /* Number of fp32 parameters of a module.  The flat layout is, for CE:
  * tok_emb[vocab,d] pos_emb[l_t,d] emb_ln_g[d] emb_ln_b[d], then per layer
  * wqkv[3d,d] bqkv[3d] wo[d,d] bo[d] ln1_g ln1_b w1[d_ff,d] b1[d_ff] w2[d,d_ff]
- * b2[d] ln2_g ln2_b; for KT: pos[L,d] resp[3,d], the layers (attention-only
+ * b2[d] ln2_g ln2_b, then for GRAM_POOL_ADDITIVE pool_wa[d_a,d] pool_ba[d_a] pool_qa[d_a]; for KT: pos[L,d] resp[3,d], the layers (attention-only
  * layers hold wqkv bqkv wo bo), head_w[d] head_b[1]; for NR: wa[d_a,d] ba[d_a]
  * qa[d_a].  Rows 0..d-1 of wqkv produce Q, the next d K, the last d V; head h
  * owns columns h*d/n_heads .. of each. */

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgram.so")
 
 GRAM_F32, GRAM_BF16 = 0, 1
-GRAM_POOL_MEAN, GRAM_POOL_CLS = 0, 1
+GRAM_POOL_MEAN, GRAM_POOL_CLS, GRAM_POOL_ADDITIVE = 0, 1, 2
 GRAM_TASK_NONE, GRAM_TASK_KT, GRAM_TASK_NR = 0, 1, 2
 GRAM_MODULE_CE, GRAM_MODULE_TASK = 0, 1
 GRAM_OPT_SGD, GRAM_OPT_ADAM = 0, 1
@@ -100,7 +100,7 @@ def config_from_shape(shape, **over) -> GramConfig:
     for k in ("n_items", "l_t", "vocab", "d", "n_heads", "d_ff", "n_layers", "task_layers", "task_heads", "task_d_ff",
               "d_a", "n_cand", "L", "K"):
         setattr(cfg, k, int(getattr(shape, k)))
-    cfg.pooling = GRAM_POOL_MEAN if shape.pooling == "mean" else GRAM_POOL_CLS
+    cfg.pooling = {"mean": GRAM_POOL_MEAN, "cls": GRAM_POOL_CLS, "additive": GRAM_POOL_ADDITIVE}[shape.pooling]
     cfg.task = {"kt": GRAM_TASK_KT, "nr": GRAM_TASK_NR}[shape.task]
     cfg.task_attn_only = int(shape.task_attn_only)
     cfg.B_max = int(shape.B)

@@ -505,6 +505,91 @@ __global__ void pool_bwd_kernel(const float* __restrict__ G, float* __restrict__
   dx[i] = v;
 }
 
+// additive-attention pooling, one block per item: scores a_s = q . tanh(pre[s, :]) over the item's rows, alpha = softmax,
+// H[u, :] = sum_s alpha_s x[s, :]; alpha is kept for the backward pass
+template <typename T>
+__global__ void __launch_bounds__(128) pool_additive_fwd_kernel(StreamRef x, const T* __restrict__ pre, const float* __restrict__ q,
+                                                                float* __restrict__ H, float* __restrict__ alpha, int l_t, int d,
+                                                                int pa, const int32_t* __restrict__ seq_len,
+                                                                const int32_t* __restrict__ seq_off) {
+  __shared__ float sa[128];
+  const int64_t u = blockIdx.x;
+  const int64_t row0 = seq_off ? (int64_t)seq_off[u] : u * l_t;
+  const int S = seq_len ? seq_len[u] : l_t;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int s = warp; s < S; s += 4) {
+    float acc = 0.f;
+    for (int j = lane; j < pa; j += 32) acc += q[j] * tanhf(ldf(pre + (row0 + s) * pa + j));
+    acc = warp_sum(acc);
+    if (lane == 0) sa[s] = acc;
+  }
+  __syncthreads();
+  if (warp == 0) {                      // softmax over the S <= 128 scores
+    float m = -INFINITY;
+    for (int s = lane; s < S; s += 32) m = fmaxf(m, sa[s]);
+    m = warp_max(m);
+    float l = 0.f;
+    for (int s = lane; s < S; s += 32) { const float e = __expf(sa[s] - m); sa[s] = e; l += e; }
+    l = warp_sum(l);
+    const float inv = 1.f / l;
+    for (int s = lane; s < S; s += 32) { sa[s] *= inv; alpha[row0 + s] = sa[s]; }
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.f;
+    for (int s = 0; s < S; ++s) acc += sa[s] * stream_at(x, row0 + s, c, d);
+    H[u * d + c] = acc;
+  }
+}
+
+// backward of the above for the cotangent G[u, :]: dx[s, :] = alpha_s G (the part that does not go through the scores),
+// dpre[s, j] = da_s q_j (1 - tanh^2 pre[s, j]) with da = alpha (dalpha - sum alpha dalpha), dalpha_s = G . x[s, :];
+// qpart[u, j] = sum_s da_s tanh(pre[s, j]) (summed over items by the caller, in order)
+template <typename T>
+__global__ void __launch_bounds__(128) pool_additive_bwd_kernel(StreamRef x, const T* __restrict__ pre, const float* __restrict__ q,
+                                                                const float* __restrict__ alpha, const float* __restrict__ G,
+                                                                float* __restrict__ dx, T* __restrict__ dpre,
+                                                                float* __restrict__ qpart, int l_t, int d, int pa,
+                                                                const int32_t* __restrict__ seq_len,
+                                                                const int32_t* __restrict__ seq_off) {
+  __shared__ float sda[128], sal[128];
+  __shared__ float sdelta;
+  const int64_t u = blockIdx.x;
+  const int64_t row0 = seq_off ? (int64_t)seq_off[u] : u * l_t;
+  const int S = seq_len ? seq_len[u] : l_t;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int s = warp; s < S; s += 4) {
+    float acc = 0.f;
+    for (int c = lane; c < d; c += 32) acc += G[u * d + c] * stream_at(x, row0 + s, c, d);
+    acc = warp_sum(acc);
+    if (lane == 0) { sda[s] = acc; sal[s] = alpha[row0 + s]; }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float dl = 0.f;
+    for (int s = lane; s < S; s += 32) dl += sal[s] * sda[s];
+    dl = warp_sum(dl);
+    if (lane == 0) sdelta = dl;
+  }
+  __syncthreads();
+  for (int s = threadIdx.x; s < S; s += blockDim.x) sda[s] = sal[s] * (sda[s] - sdelta);
+  __syncthreads();
+  for (int j = threadIdx.x; j < pa; j += blockDim.x) {
+    const float qj = q[j];
+    float acc = 0.f;
+    for (int s = 0; s < S; ++s) {
+      const float t = tanhf(ldf(pre + (row0 + s) * pa + j));
+      stf(dpre + (row0 + s) * pa + j, sda[s] * qj * (1.f - t * t));
+      acc += sda[s] * t;
+    }
+    qpart[u * pa + j] = acc;
+  }
+  for (int64_t i = threadIdx.x; i < (int64_t)S * d; i += blockDim.x) {
+    const int s = (int)(i / d), c = (int)(i - (int64_t)s * d);
+    dx[(row0 + s) * d + c] = sal[s] * G[u * d + c];
+  }
+}
+
 // ---------------------------------------------------------------------------- KT task input / head
 template <typename T>
 __global__ void kt_input_fwd_kernel(const float* __restrict__ E, const float* __restrict__ pos,
@@ -1236,6 +1321,31 @@ gram_status sequence_layout(gram_ctx* ctx, const int32_t* item_len, const int32_
   ProfScope prof(ctx, GRAM_K_EMBED_POOL, 12.0 * (double)n, 1, st);
   seq_layout_kernel<<<1, 1024, 0, st>>>(item_len, items, first_item, n, n_items_total, l_t, seq_len, seq_off, group_list, info,
                                         gram_status_word(ctx));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status pool_additive_forward(gram_ctx* ctx, int dtype, const StreamRef& x, const void* pre, const float* q, float* H,
+                                  float* alpha, int64_t n, int l_t, int d, int pa, const int32_t* seq_len, const int32_t* seq_off,
+                                  cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if (l_t > 128) return gram_set_error(ctx, "additive pooling: at most 128 tokens per item"), GRAM_ERR_UNSUPPORTED;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * l_t * (d + pa), 1, st);
+  DISPATCH_T(dtype, pool_additive_fwd_kernel<T><<<(unsigned)n, 128, 0, st>>>(x, (const T*)pre, q, H, alpha, l_t, d, pa, seq_len, seq_off));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status pool_additive_backward(gram_ctx* ctx, int dtype, const StreamRef& x, const void* pre, const float* q,
+                                   const float* alpha, const float* G, float* dx, void* dpre, float* dq, float* scratch,
+                                   int64_t n, int l_t, int d, int pa, const int32_t* seq_len, const int32_t* seq_off,
+                                   cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  if ((size_t)n * pa * sizeof(float) > kRedScratchBytes)
+    return gram_set_error(ctx, "additive pooling: %lld items x %d exceed the reduction scratch", (long long)n, pa), GRAM_ERR_WORKSPACE;
+  ProfScope prof(ctx, GRAM_K_EMBED_POOL, 4.0 * (double)n * l_t * (2 * d + 2 * pa), 2, st);
+  DISPATCH_T(dtype, pool_additive_bwd_kernel<T><<<(unsigned)n, 128, 0, st>>>(x, (const T*)pre, q, alpha, G, dx, (T*)dpre, scratch, l_t, d,
+                                                                            pa, seq_len, seq_off));
+  reduce_partials_kernel<<<ceil_div(pa, 32), 256, 0, st>>>(scratch, (int)n, pa, pa, dq, nullptr, 1.f);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

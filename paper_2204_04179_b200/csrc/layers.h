@@ -131,3 +131,14 @@ gram_status take_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t 
 // out[row(r), :] = in[r, :] for r < n; the other rows of out are left as they are
 gram_status put_strided_rows(gram_ctx* ctx, const void* in, int64_t n, int64_t stride, const int32_t* rows, int d,
                              int elem_bytes, void* out, cudaStream_t st);
+// Additive-attention pooling over an item's tokens: given pre = x Wa^T + ba [rows, pa] (operand-typed),
+// a_s = q . tanh(pre[s]), alpha = softmax over the item's tokens (saved, fp32 [rows]), H[u] = sum_s alpha_s x[s].
+gram_status pool_additive_forward(gram_ctx* ctx, int dtype, const StreamRef& x, const void* pre, const float* q, float* H,
+                                  float* alpha, int64_t n, int l_t, int d, int pa, const int32_t* seq_len, const int32_t* seq_off,
+                                  cudaStream_t st);
+// Its backward for the cotangent G [n, d]: dx (fp32 [rows, d], overwritten) receives the part alpha_s G, dpre (operand-typed
+// [rows, pa]) the gradient with respect to pre, dq += the gradient of q; scratch: kRedScratchBytes.
+gram_status pool_additive_backward(gram_ctx* ctx, int dtype, const StreamRef& x, const void* pre, const float* q,
+                                   const float* alpha, const float* G, float* dx, void* dpre, float* dq, float* scratch,
+                                   int64_t n, int l_t, int d, int pa, const int32_t* seq_len, const int32_t* seq_off,
+                                   cudaStream_t st);

@@ -89,6 +89,12 @@ struct Model {
   Module ce, task;
   // encoder
   size_t o_tok = 0, o_pos = 0, o_elng = 0, o_elnb = 0;
+  // additive-attention pooling (GRAM_POOL_ADDITIVE): parameters, saved scores and the encoder output they pool
+  size_t o_pwa = 0, o_pba = 0, o_pqa = 0;
+  void *pool_pre = nullptr, *pool_dpre = nullptr;
+  float* pool_alpha = nullptr;
+  StreamRef pool_x;
+  const void* pool_xb = nullptr;
   Stack enc;
   // With token-0 pooling only row 0 of every item's last-layer output is ever read, so the row-wise part of the
   // last layer (output projection, feed-forward, both LayerNorms) runs on those rows alone: `tail` holds their
@@ -204,6 +210,11 @@ void layout_buffers(Model* m, Arena& a) {
     m->seq_groups = (int32_t*)a.take((size_t)m->mb * 4);
     m->seq_info = (int32_t*)a.take(8 * 4);
     stack_buffers(a, m->enc, esz);
+    if (c.pooling == GRAM_POOL_ADDITIVE) {
+      m->pool_pre = a.take(T * c.d_a * esz);
+      m->pool_dpre = a.take(T * c.d_a * esz);
+      m->pool_alpha = (float*)a.take(T * 4);
+    }
     if (m->cls_tail) {
       stack_buffers(a, m->tail, esz);
       m->tail_z = (float*)a.take((size_t)m->mb * d * 4);
@@ -516,7 +527,17 @@ gram_status encoder_forward_chunk(Model* m, const int32_t* d_item_tokens, const 
   const void* out_b = nullptr;
   if (!m->cls_tail) {
     GRAM_TRY(stack_forward(m, m->ce, m->enc, x0, m->x0, n, c.l_t, st, &out, &out_b));
-    GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
+    if (c.pooling == GRAM_POOL_ADDITIVE) {
+      GemmEpilogue e;
+      e.bias = m->ce.w + m->o_pba;
+      GRAM_TRY(mm_fwd(m, out_b, W(m, m->ce, m->o_pwa), m->pool_pre, false, T, c.d_a, c.d, e, st));     // pre = x Wa^T + ba
+      GRAM_TRY(pool_additive_forward(ctx, m->dtype, out, m->pool_pre, m->ce.w + m->o_pqa, H_out, m->pool_alpha, n, c.l_t, c.d,
+                                     c.d_a, seq_len, seq_off, st));
+      m->pool_x = out;
+      m->pool_xb = out_b;
+    } else {
+      GRAM_TRY(pool_forward(ctx, out, H_out, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
+    }
   } else {
     // all layers but the last, and the last layer's attention over whole sequences
     const int last = c.n_layers - 1;
@@ -548,7 +569,17 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   const int32_t* seq_off = m->enc.seq_off;
   float* dx0 = nullptr;
   if (!m->cls_tail) {
-    GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
+    if (c.pooling == GRAM_POOL_ADDITIVE) {
+      GRAM_TRY(pool_additive_backward(ctx, m->dtype, m->pool_x, m->pool_pre, m->ce.w + m->o_pqa, m->pool_alpha, G, m->enc.curf,
+                                      m->pool_dpre, m->ce.g + m->o_pqa, m->red, n, c.l_t, c.d, c.d_a, seq_len, seq_off, st));
+      GRAM_TRY(colsum_accumulate(ctx, m->dtype, m->pool_dpre, T, c.d_a, m->ce.g + m->o_pba, m->red, st));
+      GRAM_TRY(mm_dw(m, m->pool_dpre, m->pool_xb, m->ce.g + m->o_pwa, T, c.d_a, c.d, st));
+      GemmEpilogue e;
+      e.accumulate = 1;                  // the stream gradient already holds alpha_s G
+      GRAM_TRY(mm_dx(m, m->pool_dpre, W(m, m->ce, m->o_pwa), m->enc.curf, true, T, c.d_a, c.d, e, st));
+    } else {
+      GRAM_TRY(pool_backward(ctx, G, m->enc.curf, n, c.l_t, c.d, c.pooling, seq_len, seq_off, st));
+    }
     GRAM_TRY(stack_backward(m, m->ce, m->enc, m->x0, n, c.l_t, st, &dx0));
   } else {
     // the row-wise part of the last layer on one row per item
@@ -717,6 +748,14 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
     m->enc.attn_only = 0; m->enc.causal = 0;
     m->enc.off.resize(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) at = layer_layout(&m->enc.off[l], at, c.d, c.d_ff, 0);
+    if (c.pooling == GRAM_POOL_ADDITIVE) {
+      if (c.d_a <= 0) return gram_set_error(ctx, "additive pooling needs d_a > 0"), GRAM_ERR_ARG;
+      m->o_pwa = at; at += (size_t)c.d_a * c.d;
+      m->o_pba = at; at += c.d_a;
+      m->o_pqa = at; at += c.d_a;
+    } else if (c.pooling != GRAM_POOL_MEAN && c.pooling != GRAM_POOL_CLS) {
+      return gram_set_error(ctx, "unknown pooling %d", c.pooling), GRAM_ERR_ARG;
+    }
   }
   GRAM_TRY(module_alloc(ctx, &m->ce, at, c.dtype == GRAM_BF16, c.optimizer == GRAM_OPT_ADAM));
   at = 0;

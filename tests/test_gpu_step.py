@@ -436,3 +436,34 @@ def test_multistep_cache_refresh_after_the_encoder_update():
             assert gh.rel_err(cache_gpu, stale["cache"]) > 1e-3
         cur_ce, cur_tk, cache = want["ce_params"], want["task_params"], want["cache"]
     g.close()
+
+
+ADDITIVE = {
+    "f32_kt": small(pooling="additive", d_a=16),
+    "f32_nr_odd": small(task="nr", task_layers=0, n_cand=3, L=9, d_a=12, pooling="additive", l_t=7, d=24, n_heads=3, d_ff=40),
+    "bf16_kt": small(dtype="bf16", pooling="additive", d_a=16, d=64, d_ff=128, task_d_ff=128, l_t=24, n_items=30),
+}
+
+
+@pytest.mark.parametrize("name", list(ADDITIVE))
+@pytest.mark.parametrize("var_len", [False, True])
+def test_additive_attention_pooling(name, var_len):
+    """GRAM_POOL_ADDITIVE against the oracle, with texts of one length and of different lengths (packed rows)."""
+    shape = ADDITIVE[name]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=37)
+    assert "pool_wa" in ce and ce["pool_wa"].shape == (shape.d_a, shape.d)
+    lengths = synth.item_lengths(37, shape.n_items, shape.l_t) if var_len else None
+    want = orc.e2e_step(shape, ce, tk, synth.ragged(toks, lengths) if var_len else toks, ids, lab)
+    g = gh.make_ctx(shape, ce, tk, toks, ce_micro_batch=11)
+    if var_len:
+        g.set_item_lengths(lengths)
+    rep = g.step(torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV), shape.B)
+    gce, gtk = gh.gpu_grads(g, shape)
+    g.close()
+    tol = TOL[shape.dtype]
+    assert abs(rep.loss - want["loss"]) <= tol * abs(want["loss"])
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+    print(name, var_len, "worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+    assert np.abs(gce["pool_qa"]).max() > 0 and np.abs(gce["pool_wa"]).max() > 0
