@@ -218,7 +218,11 @@ gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int
  * shorter than L ends in padding (Appendix D: sequences are cut or padded to a
  * maximum length): its padded positions carry label -1 and any valid item ID,
  * are not predicted, receive a zero row of d_dE, and the loss is the mean over
- * the real predictions of the batch.  The same holds for gram_step. */
+ * the real predictions of the batch.  For GRAM_TASK_NR a user with fewer
+ * clicks than history slots marks the empty slots (any of the first
+ * L - n_cand positions) with label -1; they take no part in the user vector
+ * and receive a zero row of d_dE; at least one slot per user must hold a click.
+ * The same holds for gram_step. */
 gram_status gram_task(gram_ctx* ctx, const float* d_E, const int32_t* d_labels, int32_t B, float* d_dE,
                       float* d_loss, gram_stream stream);
 

@@ -226,7 +226,8 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
     nr: additive attention over the first L - n_cand encodings gives the user
         vector, dot products with the n_cand candidate encodings give scores,
         loss = -log softmax(scores)[0] (the first candidate is the click),
-        averaged over the B users.
+        averaged over the B users.  History slots with label -1 hold no click
+        (a user with fewer clicks than slots) and take no part.
     """
     B, L, d = E.shape
     lab = torch.as_tensor(np.asarray(labels), dtype=torch.long)
@@ -257,6 +258,8 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
         total = E.new_zeros(())
         for b in range(B):
             hist, cand = E[b, :n_hist], E[b, n_hist:]
+            # a click history shorter than its slots: the slots with label -1 hold no click and are simply left out
+            hist = hist[(lab[b, :n_hist] >= 0).nonzero()[:, 0]]
             a = torch.tanh(hist @ th["wa"].T + th["ba"]) @ th["qa"]
             alpha = softmax_rows(a[None, :])[0]
             u = alpha @ hist

@@ -699,7 +699,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) nr_user_kernel(const float* __restrict__ E, const T* __restrict__ pre,
                                                       const float* __restrict__ qa, float* __restrict__ dE,
                                                       T* __restrict__ dpre, float* __restrict__ part, int L, int n_cand,
-                                                      int d, int d_a, float invB) {
+                                                      int d, int d_a, float invB, const int32_t* __restrict__ labels) {
   extern __shared__ float sm[];
   const int n_hist = L - n_cand;
   float* a = sm;                 // [L] scores / alpha
@@ -715,6 +715,7 @@ __global__ void __launch_bounds__(256) nr_user_kernel(const float* __restrict__ 
     float acc = 0.f;
     for (int k = lane; k < d_a; k += 32) acc += qa[k] * tanhf(ldf(pb + (int64_t)n * d_a + k));
     acc = warp_sum(acc);
+    if (labels && labels[(int64_t)b * L + n] < 0) acc = -INFINITY;       // a slot without a click takes no part
     if (lane == 0) a[n] = acc;
   }
   __syncthreads();
@@ -722,10 +723,12 @@ __global__ void __launch_bounds__(256) nr_user_kernel(const float* __restrict__ 
     float m = -INFINITY;
     for (int n = lane; n < n_hist; n += 32) m = fmaxf(m, a[n]);
     m = warp_max(m);
+    if (m == -INFINITY) m = 0.f;                                           // no click at all: every weight is zero
     float l = 0.f;
     for (int n = lane; n < n_hist; n += 32) l += __expf(a[n] - m);
     l = warp_sum(l);
-    for (int n = lane; n < n_hist; n += 32) a[n] = __expf(a[n] - m) / l;
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    for (int n = lane; n < n_hist; n += 32) a[n] = __expf(a[n] - m) * inv;
   }
   __syncthreads();
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
@@ -1186,15 +1189,15 @@ gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* lab
 }
 
 gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, const float* qa, float* dE,
-                           void* dpre, float* dqa, float* loss, float* scratch, int B, int L, int n_cand, int d, int d_a,
-                           cudaStream_t st) {
+                           void* dpre, float* dqa, float* loss, float* scratch, const int32_t* labels, int B, int L, int n_cand,
+                           int d, int d_a, cudaStream_t st) {
   if (B == 0) return GRAM_OK;
   if (n_cand <= 0 || n_cand >= L) return gram_set_error(ctx, "nr task: need 0 < n_cand < L"), GRAM_ERR_ARG;
   const size_t smem = ((size_t)2 * L + 2 * d + n_cand) * sizeof(float);
   ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)B * L * (8.0 * d + 4.0 * d_a), 2, st);
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, nr_user_kernel<T>, smem));
-    nr_user_kernel<T><<<B, 256, smem, st>>>(E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B);
+    nr_user_kernel<T><<<B, 256, smem, st>>>(E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B, labels);
   });
   nr_reduce_kernel<<<ceil_div(d_a + 1, 256), 256, 0, st>>>(scratch, B, d_a, 1.f / (float)B, dqa, loss);
   GRAM_LAUNCH_CHECK(ctx);

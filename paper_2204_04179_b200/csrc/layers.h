@@ -111,9 +111,11 @@ gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w
 // news-recommendation task, the part between the matrix products (one block per user):
 // given pre = E wa^T + ba [B*L, d_a] (operand-typed), computes additive attention over the first L - n_cand
 // encodings, dot-product scores with the candidates and softmax cross-entropy on candidate 0 (averaged over
-// B); writes the direct part of dE (fp32 [B*L, d]), dpre (operand-typed, zero rows for candidates), dqa +=, loss.
+// B; history slots whose label is negative hold no click and take no part, labels may be null); writes the direct
+// part of dE (fp32 [B*L, d]), dpre (operand-typed, zero rows for candidates), dqa +=, loss.
 gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, const float* qa, float* dE, void* dpre,
-                    float* dqa, float* loss, float* scratch, int B, int L, int n_cand, int d, int d_a, cudaStream_t st);
+                    float* dqa, float* loss, float* scratch, const int32_t* labels, int B, int L, int n_cand, int d, int d_a,
+                    cudaStream_t st);
 
 // element-wise helpers
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st);

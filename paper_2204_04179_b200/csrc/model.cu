@@ -640,7 +640,7 @@ gram_status task_forward_backward(Model* m, const float* E, const int32_t* label
     GemmEpilogue e;
     e.bias = m->task.w + m->t_ba;
     GRAM_TRY(mm_fwd(m, Eb, W(m, m->task, m->t_wa), m->pre, false, P, c.d_a, c.d, e, st));
-    GRAM_TRY(nr_user(ctx, m->dtype, E, m->pre, m->task.w + m->t_qa, dE, m->dpre, m->task.g + m->t_qa, loss, m->red, B, c.L,
+    GRAM_TRY(nr_user(ctx, m->dtype, E, m->pre, m->task.w + m->t_qa, dE, m->dpre, m->task.g + m->t_qa, loss, m->red, labels, B, c.L,
                      c.n_cand, c.d, c.d_a, st));
     GRAM_TRY(colsum_accumulate(ctx, m->dtype, m->dpre, P, c.d_a, m->task.g + m->t_ba, m->red, st));
     GRAM_TRY(mm_dw(m, m->dpre, Eb, m->task.g + m->t_wa, P, c.d_a, c.d, st));

@@ -467,3 +467,27 @@ def test_additive_attention_pooling(name, var_len):
     print(name, var_len, "worst CE", e1, n1, "worst task", e2, n2)
     assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
     assert np.abs(gce["pool_qa"]).max() > 0 and np.abs(gce["pool_wa"]).max() > 0
+
+
+@pytest.mark.parametrize("name", ["nr", "bf16_nr"])
+def test_click_histories_with_empty_slots(name):
+    """NR: history slots with label -1 hold no click: they take no part in the user vector and get zero gradient rows."""
+    shape = CASES[name]
+    ce, tk, toks, ids, lab = gh.make_inputs(shape, seed=39)
+    lab = np.zeros_like(lab)
+    n_hist = shape.L - shape.n_cand
+    rng = np.random.default_rng(1)
+    for b in range(shape.B):
+        empty = rng.choice(n_hist, size=rng.integers(0, n_hist), replace=False)     # at least one click stays
+        lab[b, empty] = -1
+    assert (lab < 0).any()
+    want = orc.e2e_step(shape, ce, tk, toks, ids, lab)
+    rep, gce, gtk = gh.gpu_single_step(shape, ce, tk, toks, ids, lab)
+    tol = TOL[shape.dtype]
+    assert abs(rep.loss - want["loss"]) <= tol * abs(want["loss"])
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task"])
+    print(name, "worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+    full = orc.e2e_step(shape, ce, tk, toks, ids, np.zeros_like(lab))
+    assert abs(full["loss"] - want["loss"]) > 1e-6                                  # the mask matters

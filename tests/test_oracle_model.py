@@ -468,3 +468,24 @@ def test_additive_pooling_special_cases_and_finite_differences():
             dn = OrderedDict((k, v.copy()) for k, v in ce.items()); dn[name][idx] -= 1e-6
             fd = (loss_at(up) - loss_at(dn)) / 2e-6
             assert abs(fd - res["grad_ce"][name][idx]) <= 1e-7 + 1e-5 * abs(fd), (name, idx, fd, res["grad_ce"][name][idx])
+
+
+def test_empty_click_slots_are_left_out():
+    # NR: history slots with label -1 take no part: the loss equals that of the same users with those rows removed
+    shape = small_shape(task="nr", task_layers=0, n_cand=2, L=7, d_a=6, B=2, pooling="cls")
+    tk = synth.task_params(shape, 3, sigma=0.3, plain=False)
+    th = orc.as_torch(tk, T64)
+    E = torch.randn(2, 7, shape.d, dtype=T64, generator=torch.Generator().manual_seed(5))
+    lab = np.zeros((2, 7), np.int32)
+    lab[0, [1, 3]] = -1
+    lab[1, 4] = -1
+    Eg = E.clone().requires_grad_(True)
+    loss = orc.task_loss(th, Eg, lab, shape)
+    loss.backward()
+    with torch.no_grad():
+        keep0 = [0, 2, 4, 5, 6]; keep1 = [0, 1, 2, 3, 5, 6]
+        l0 = orc.task_loss(th, E[0:1, keep0], np.zeros((1, 5), np.int32), shape.replace(B=1, L=5))
+        l1 = orc.task_loss(th, E[1:2, keep1], np.zeros((1, 6), np.int32), shape.replace(B=1, L=6))
+    assert abs(float(loss.detach()) - (float(l0) + float(l1)) / 2) < 1e-13
+    assert torch.count_nonzero(Eg.grad[0, [1, 3]]) == 0 and torch.count_nonzero(Eg.grad[1, 4]) == 0
+    assert torch.count_nonzero(Eg.grad[0, 0]) > 0
