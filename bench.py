@@ -144,6 +144,51 @@ def run_reference(args, shape):
     }))
 
 
+def stack_flops(tokens, n_layers, d, d_ff, seq, attn_only=False):
+    """Forward flops of n_layers transformer layers over `tokens` rows in sequences of `seq` rows: the four projections,
+    the feed-forward products (2 flops per multiply-add) and the two attention products."""
+    per_layer = 2.0 * 4 * d * d + (0.0 if attn_only else 2.0 * 2 * d * d_ff) + 4.0 * seq * d
+    return tokens * n_layers * per_layer
+
+
+def stage_fractions(shape, stage_ms, U, peaks):
+    """Algorithmic work of each stage of a Single-step step (fixed-length texts) over its device time, against the
+    roofline that bounds it: HBM bytes for dedup, gather and accumulate, bf16 tensor flops for the three model stages.
+    With token-0 pooling the row-wise part of the last encoder layer is needed for one row per item only; the flops
+    counted are those the method needs, not the ones a plain implementation would spend."""
+    P, d, N = shape.B * shape.L, shape.d, shape.n_items
+    passes = (max(1, (N - 1).bit_length()) + 7) // 8
+    T = U * shape.l_t
+    enc = stack_flops(T, shape.n_layers, d, shape.d_ff, shape.l_t)
+    if shape.pooling == "cls" and shape.n_layers > 0:          # output projection + feed-forward of the last layer: U rows, not T
+        enc -= (T - U) * (2.0 * d * d + 2.0 * 2 * d * shape.d_ff)
+    if shape.task == "kt":
+        task = 3.0 * stack_flops(P, shape.task_layers, d, shape.task_d_ff, shape.L / 2.0, shape.task_attn_only)   # causal: half the scores
+    else:
+        task = 3.0 * 2.0 * P * d * shape.d_a
+    work = {"ms_dedup": ((16 * passes + 20) * P + 8 * U, "hbm"),
+            "ms_encode": (enc, "tensor"),
+            "ms_gather": (4.0 * P * d + 4.0 * U * d + 4 * P, "hbm"),
+            "ms_task": (task, "tensor"),
+            "ms_accumulate": (4.0 * P * d + 4.0 * U * d + 4 * P + 4 * (U + 1), "hbm"),
+            "ms_backward": (2.0 * enc, "tensor")}
+    out = {}
+    for k, (w, bound) in work.items():
+        ms = stage_ms[k]
+        if ms <= 0:
+            continue
+        rate = w / (ms / 1e3)
+        if bound == "hbm":
+            out[k[3:]] = {"bound": "hbm", "GB/s": rate / 1e9, "frac": rate / (peaks["hbm_gbs"] * 1e9)}
+        elif shape.dtype == "bf16":
+            out[k[3:]] = {"bound": "tensor", "TFLOP/s": rate / 1e12, "frac": rate / (peaks["tflops"] * 1e12)}
+        else:       # fp32 contexts run on the plain ALUs: 148 SMs x 128 fused multiply-adds per clock x 1.965 GHz
+            out[k[3:]] = {"bound": "alu", "TFLOP/s": rate / 1e12, "frac": rate / (148 * 128 * 2 * 1.965e9)}
+    out["note"] = ("algorithmic bytes or flops of the stage / its device time; dedup, gather and accumulate move tens of MB here "
+                   "(L2-resident, launch-latency scale): their HBM fractions are taken on the larger cell under hbm_kernels")
+    return out
+
+
 def kernel_sweep_cell(binding, synth, torch, dev, peaks):
     """dedup / gather / accumulate alone on one sweep cell larger than L2 (P=1e6, N=1e5, Zipf 1.1, d=768)."""
     P, N, s, d = 1_000_000, 100_000, 1.1, 768
@@ -308,6 +353,8 @@ def run_gram(args, shape):
         roofline["traffic"] = per_row * statistics.mean(r.n_unique for r in reports) * shape.l_t
     stage_ms = {k: statistics.mean(getattr(r, k) for r in reports)
                 for k in ("ms_dedup", "ms_encode", "ms_gather", "ms_task", "ms_accumulate", "ms_backward", "ms_total")}
+    stage_roofline = stage_fractions(shape, stage_ms, statistics.mean(r.n_unique for r in reports), peaks) \
+        if (not multistep and lengths is None) else None
     per_kind = {}
     for name, v in kinds.items():
         if v["launches"] == 0:
@@ -331,7 +378,7 @@ def run_gram(args, shape):
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * P, "d2h_bytes_per_step": 12,
                 "ms_per_step": ms_e2e / args.steps},
-        "roofline": roofline, "stage_ms": stage_ms, "kernel_kinds": per_kind,
+        "roofline": roofline, "stage_ms": stage_ms, "stage_roofline": stage_roofline, "kernel_kinds": per_kind,
         "call_sites": {t: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps,
                            ("TFLOP/s" if v["kind"] in ("gemm", "attention") else "GB/s"):
                                (v["work"] / (v["ms"] / 1e3) / (1e12 if v["kind"] in ("gemm", "attention") else 1e9)) if v["ms"] > 0 else 0.0}
