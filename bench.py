@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the GRAM training step (Single-step GRAM on the knowledge-tracing-shaped workload).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload kt|nr|tiny|kt_multistep|kt_6l]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload kt|nr|tiny|kt_multistep|kt_6l|nr_additive]
 
 A step is one pass of the whole path (dedup, encode unique items, gather, task module forward/backward,
 accumulate, encoder backward) over one batch of seeded synthetic histories.  Prints ONE JSON line.
@@ -413,7 +413,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="gram", choices=["gram", "reference"])
-    ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny", "kt_multistep", "kt_6l"])
+    ap.add_argument("--workload", default="kt", choices=["kt", "nr", "tiny", "kt_multistep", "kt_6l", "nr_additive"])
     ap.add_argument("--micro-batch", type=int, default=0, help="items per encoder pass (0: the workload's default)")
     ap.add_argument("--multistep-variant", default="table", choices=["table", "pseudo_target"],
                     help="kt_multistep: separate gradient table with unchanged cached encodings, or pseudo-targets (Section 4.3)")
@@ -422,8 +422,8 @@ def main():
     args = ap.parse_args()
     from paper_2204_04179_b200 import synth
     shape = synth.config(args.workload)
-    if args.workload in ("kt", "nr", "kt_multistep", "kt_6l") and not args.micro_batch:
-        args.micro_batch = 0 if args.workload == "nr" else 5120
+    if args.workload in ("kt", "nr", "kt_multistep", "kt_6l", "nr_additive") and not args.micro_batch:
+        args.micro_batch = 0 if args.workload in ("nr", "nr_additive") else 5120
     if args.impl == "reference":
         run_reference(args, shape)
     else:

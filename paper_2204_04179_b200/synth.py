@@ -83,6 +83,8 @@ def config(name: str) -> GramShape:
                          task="nr", task_layers=0, d_a=256, n_cand=5, B=64, L=55)
     if name == "kt_multistep":    # Multi-step GRAM on the knowledge-tracing shape
         return config("kt").replace(name="kt_multistep", K=8)
+    if name == "nr_additive":     # news recommendation with the paper's item pooling (additive attention over the title tokens)
+        return config("nr").replace(name="nr_additive", pooling="additive")
     if name == "kt_6l":           # the same with the paper's own encoder depth (Appendix D: a 6-layer, 768-wide model)
         return config("kt").replace(name="kt_6l", n_layers=6)
     raise KeyError(name)
