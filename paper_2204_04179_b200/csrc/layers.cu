@@ -595,16 +595,18 @@ template <typename T>
 __global__ void kt_input_fwd_kernel(const float* __restrict__ E, const float* __restrict__ pos,
                                     const float* __restrict__ resp, const int32_t* __restrict__ labels,
                                     float* __restrict__ x, T* __restrict__ x_b, int64_t P, int L, int d) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= P * d) return;
-  const int64_t p = i / d;
-  const int c = (int)(i - p * d);
+  const int64_t p = blockIdx.x;                  // one block per position
   const int n = (int)(p % L);
   int prev = (n == 0) ? 2 : labels[p - 1];
   prev = prev < 0 ? 2 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);      // after a padded position (label -1): only at padded rows
-  const float v = E[i] + pos[(int64_t)n * d + c] + resp[(int64_t)prev * d + c];
-  x[i] = v;
-  stf(x_b + i, v);
+  const float* e = E + p * d;
+  const float* pe = pos + (int64_t)n * d;
+  const float* re = resp + (int64_t)prev * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = e[c] + pe[c] + re[c];
+    x[p * d + c] = v;
+    stf(x_b + p * d + c, v);
+  }
 }
 // one thread per column: dE = dx; dpos[n, c] += sum_b; dresp[r, c] += sum over positions with prev == r
 __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t* __restrict__ labels, float* __restrict__ dE,
@@ -613,6 +615,7 @@ __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t*
   const int n = blockIdx.y;
   if (c >= d) return;
   float ap = 0.f, r0 = 0.f, r1 = 0.f, r2 = 0.f;
+#pragma unroll 4
   for (int b = 0; b < B; ++b) {
     const int64_t p = (int64_t)b * L + n;
     const float v = dx[p * d + c];
@@ -628,48 +631,71 @@ __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t*
   dresp[((int64_t)n * 3 + 2) * d + c] = r2;
 }
 
-// warp per position; per-block partials: [d] for dw, then loss and db
+// warp per position; per-block partials: [d] for dw, then loss and db.  A warp keeps the sums of its own rows in
+// registers (d <= 1024); the warps' sums are added in warp order at the end, so the order of additions is fixed.
 template <typename T>
 __global__ void __launch_bounds__(256) kt_head_kernel(StreamRef y, const float* __restrict__ w,
                                                       const float* __restrict__ bias, const int32_t* __restrict__ labels,
                                                       float* __restrict__ dy, T* __restrict__ dy_b,
                                                       float* __restrict__ part, int64_t P, int d, int64_t pstride,
                                                       const int32_t* __restrict__ n_real) {
-  extern __shared__ float sacc[];            // [d + 2]
+  extern __shared__ float sacc[];            // [warps][d + 2]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwb = blockDim.x >> 5;
-  for (int i = threadIdx.x; i < d + 2; i += blockDim.x) sacc[i] = 0.f;
-  __syncthreads();
   const float b0 = bias[0], invP = 1.f / (float)max(*n_real, 1);   // the mean runs over the real predictions
-  // rows are dealt to blocks in contiguous ranges so that each block adds its rows in order
+  // rows are dealt to blocks in contiguous ranges, and inside a block to warps round-robin
   const int64_t per = (P + gridDim.x - 1) / gridDim.x;
   const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(r0 + per, P);
-  for (int64_t rb = r0; rb < r1; rb += nwb) {
-    const int64_t r = rb + warp;
-    float dzl = 0.f, lossr = 0.f;
-    if (r < r1) {
-      float acc = 0.f;
-      for (int c = lane; c < d; c += 32) acc += stream_at(y, r, c, d) * w[c];
-      const float z = warp_sum(acc) + b0;
-      const int32_t li = labels[r];
-      const float lab = (float)li;
-      if (li >= 0) {                          // label -1: padding at the end of a history, not predicted
-        lossr = fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
-        dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
+  float acc_w[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) acc_w[i] = 0.f;
+  float acc_loss = 0.f, acc_db = 0.f;
+  for (int64_t r = r0 + warp; r < r1; r += nwb) {
+    float yv[32];
+    float acc = 0.f;
+    const bool ln = y.mean != nullptr;             // the stream's LayerNorm, its row statistics read once
+    const float mu = ln ? y.mean[r] : 0.f, rs = ln ? y.rstd[r] : 1.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int c = lane + 32 * i;
+      yv[i] = 0.f;
+      if (c < d) {
+        const float v = y.z[r * d + c];
+        yv[i] = ln ? (v - mu) * rs * y.gamma[c] + y.beta[c] : v;
+        acc += yv[i] * w[c];
       }
-      for (int c = lane; c < d; c += 32) {
+    }
+    const float z = warp_sum(acc) + b0;
+    const int32_t li = labels[r];
+    const float lab = (float)li;
+    float dzl = 0.f;
+    if (li >= 0) {                          // label -1: padding at the end of a history, not predicted
+      acc_loss += fmaxf(z, 0.f) + log1pf(__expf(-fabsf(z))) - lab * z;
+      dzl = (1.f / (1.f + __expf(-z)) - lab) * invP;
+    }
+    acc_db += dzl;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int c = lane + 32 * i;
+      if (c < d) {
         dy[r * d + c] = dzl * w[c];
         if (dy_b) stf(dy_b + r * d + c, dzl * w[c]);
+        acc_w[i] += dzl * yv[i];
       }
-    }
-    for (int ww = 0; ww < nwb; ++ww) {       // rows of this round add in ascending order
-      if (warp == ww && r < r1) {
-        for (int c = lane; c < d; c += 32) sacc[c] += dzl * stream_at(y, r, c, d);
-        if (lane == 0) { sacc[d] += lossr; sacc[d + 1] += dzl; }
-      }
-      __syncthreads();
     }
   }
-  for (int i = threadIdx.x; i < d + 2; i += blockDim.x) part[(int64_t)blockIdx.x * pstride + i] = sacc[i];
+  float* mine = sacc + (size_t)warp * (d + 2);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int c = lane + 32 * i;
+    if (c < d) mine[c] = acc_w[i];
+  }
+  if (lane == 0) { mine[d] = acc_loss; mine[d + 1] = acc_db; }
+  __syncthreads();
+  for (int i = threadIdx.x; i < d + 2; i += blockDim.x) {
+    float a = 0.f;
+    for (int ww = 0; ww < nwb; ++ww) a += sacc[(size_t)ww * (d + 2) + i];
+    part[(int64_t)blockIdx.x * pstride + i] = a;
+  }
 }
 
 __global__ void kt_head_reduce_kernel(const float* __restrict__ part, int nblocks, int64_t pstride, int d,
@@ -1153,7 +1179,7 @@ gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const flo
   const int64_t P = (int64_t)B * L;
   if (P == 0) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)P * d * (8.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
-  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)ceil_div64(P * d, 256), 256, 0, st>>>(E, pos, resp, labels, x, (T*)x_b, P, L, d));
+  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)P, d >= 256 ? 256 : 64, 0, st>>>(E, pos, resp, labels, x, (T*)x_b, P, L, d));
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -1165,7 +1191,8 @@ gram_status kt_head(gram_ctx* ctx, int dtype, const StreamRef& y, const float* w
   int blocks = (int)ceil_div64(P, 64);
   if (blocks > kRedBlocks) blocks = kRedBlocks;
   const int64_t pstride = d + 2;
-  const size_t smem = (size_t)(d + 2) * sizeof(float);
+  if (d > 1024) return gram_set_error(ctx, "kt head: d must be at most 1024"), GRAM_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)8 * (d + 2) * sizeof(float);
   ProfScope prof(ctx, GRAM_K_TASK_HEAD, 12.0 * (double)P * d, 3, st);
   GRAM_CUDA(ctx, cudaMemsetAsync(n_real, 0, sizeof(int32_t), st));
   count_real_kernel<<<grid_for(P, 256, kNumSMs), 256, 0, st>>>(labels, P, n_real);
