@@ -615,14 +615,25 @@ __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t*
   const int n = blockIdx.y;
   if (c >= d) return;
   float ap = 0.f, r0 = 0.f, r1 = 0.f, r2 = 0.f;
-#pragma unroll 4
-  for (int b = 0; b < B; ++b) {
-    const int64_t p = (int64_t)b * L + n;
-    const float v = dx[p * d + c];
-    dE[p * d + c] = v;
-    ap += v;
-    int prev = (n == 0) ? 2 : labels[p - 1];
-    if (prev == 0) r0 += v; else if (prev == 1) r1 += v; else r2 += v;
+  constexpr int UB = 8;                          // histories per round: their loads are issued together
+  for (int b0 = 0; b0 < B; b0 += UB) {
+    float v[UB];
+    int prev[UB];
+#pragma unroll
+    for (int k = 0; k < UB; ++k) {
+      const int64_t p = (int64_t)(b0 + k) * L + n;
+      const bool ok = b0 + k < B;
+      v[k] = ok ? dx[p * d + c] : 0.f;
+      prev[k] = (ok && n > 0) ? labels[p - 1] : 2;
+    }
+#pragma unroll
+    for (int k = 0; k < UB; ++k) {              // sums in ascending history order
+      if (b0 + k < B) {
+        dE[((int64_t)(b0 + k) * L + n) * d + c] = v[k];
+        ap += v[k];
+        if (prev[k] == 0) r0 += v[k]; else if (prev[k] == 1) r1 += v[k]; else r2 += v[k];
+      }
+    }
   }
   dpos[(int64_t)n * d + c] += ap;
   // per-position partial of dresp, reduced over n by the caller: part[n][3][d]
