@@ -27,8 +27,8 @@ What it states, and from where in the paper:
 * `unique_inverse_bruteforce`, `unique_inverse`, `segment_sum`,
   `table_accumulate`: the index work and the per-item sums on their own.
 * `boost_ratio`: the speed-boost ratio R (Section 4.4).
-* `noam_rate`, `adam_update`, `train_steps_adam`: the optimiser of Section A
-  (implementation details): Adam with the Noam learning-rate scheme, written
+* `noam_rate`, `adam_update`, `train_steps_adam`: the optimiser of Appendix D
+  (experiment details): Adam with the Noam learning-rate scheme, written
   from the two published definitions; `train_steps_adam` applies it to the
   end-to-end gradients of successive batches.
 
@@ -39,7 +39,11 @@ combination with central finite differences and closed forms.
 
 Pins (tests/test_oracle_*.py): brute force on tiny inputs, the worked count
 of Fig. 1, finite differences on a 1-layer encoder, closed forms of softmax /
-LayerNorm / GELU / BCE, the Proposition (e2e == single-step), the pseudo-loss
+LayerNorm / GELU, the task module's pieces one by one (`kt_logits`: no label
+leak and the one-position closed form; `bce_with_logits_sum` and
+`softmax_ce_first`: the library losses at random logits; `nr_user_vector`:
+mean at q = 0, a one-click history, the library softmax; each with planted
+mistakes that must fail), the Proposition (e2e == single-step), the pseudo-loss
 identity (Eqs. 1-3), K = 1 reducing to single-step, and conservation of
 column sums; for the trainable-embedding window, torch.optim.SGD(lr=1) on an
 embedding parameter, finite differences of the pseudo-loss with a stale cache,
@@ -214,18 +218,57 @@ def ce_forward(th: Dict[str, torch.Tensor], tokens, shape) -> torch.Tensor:
     raise KeyError(shape.pooling)
 
 
+def kt_logits(th: Dict[str, torch.Tensor], E_hist: torch.Tensor, labels_hist, shape) -> torch.Tensor:
+    """Logits of ONE knowledge-tracing history: E_hist [n, d] (encodings of its n items), labels_hist [n]
+    (responses r_0..r_{n-1}) -> z [n].  Prediction n sees interactions (e_m, r_m) for m < n and the item e_n
+    (Section 3.1), never r_n itself: x_n = E_hist[n] + pos[n] + resp[r_{n-1}], with resp row 2 standing for
+    "no previous response" at n = 0; causal layers; z_n = head_w . y_n + head_b."""
+    n = E_hist.shape[0]
+    lab = torch.as_tensor(np.asarray(labels_hist), dtype=torch.long)
+    prev = torch.cat([torch.full((1,), 2, dtype=torch.long), lab[:n - 1]])
+    x = E_hist + th["pos"][:n] + th["resp"][prev]
+    for l in range(shape.task_layers):
+        x = transformer_layer(x, th, f"t{l}.", shape.task_heads, causal=True, attn_only=shape.task_attn_only)
+    return x @ th["head_w"] + th["head_b"]
+
+
+def bce_with_logits_sum(z: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """Sum over predictions of -[y log sigma(z) + (1 - y) log(1 - sigma(z))] = softplus(z) - y z, the binary
+    cross-entropy of Eq. 8 for correctness labels y in {0, 1}, written with a stable softplus."""
+    return (torch.clamp(z, min=0) + torch.log1p(torch.exp(-z.abs())) - y * z).sum()
+
+
+def nr_user_vector(th: Dict[str, torch.Tensor], clicked: torch.Tensor) -> torch.Tensor:
+    """User vector from the encodings of the clicked items [m, d]: additive attention (Appendix D),
+    a_n = qa . tanh(wa h_n + ba), alpha = softmax(a), u = sum_n alpha_n h_n."""
+    a = torch.tanh(clicked @ th["wa"].T + th["ba"]) @ th["qa"]
+    alpha = softmax_rows(a[None, :])[0]
+    return alpha @ clicked
+
+
+def nr_scores(th: Dict[str, torch.Tensor], clicked: torch.Tensor, cand: torch.Tensor, shape) -> torch.Tensor:
+    """Scores of ONE user's candidates: s_j = u . c_j, u the user vector of the clicked items (which first pass
+    through `task_layers` non-causal self-attention layers over the clicked items when the shape has any:
+    Appendix D, a single MHSA layer in the news task)."""
+    x = clicked
+    for l in range(shape.task_layers):
+        x = transformer_layer(x, th, f"t{l}.", shape.task_heads, causal=False, attn_only=shape.task_attn_only)
+    return cand @ nr_user_vector(th, x)
+
+
+def softmax_ce_first(s: torch.Tensor) -> torch.Tensor:
+    """-log softmax(s)[0]: the clicked candidate is listed first, the sampled negatives follow."""
+    m = s.max()
+    return -(s[0] - m - torch.log(torch.exp(s - m).sum()))
+
+
 def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> torch.Tensor:
     """The CF objective (Eq. 8) over a mini-batch: E [B, L, d] -> scalar.
 
-    kt: the model sees interactions (e_1, r_1) .. (e_{n-1}, r_{n-1}) and the
-        next item e_n, and predicts r_n (Section 3.1): input
-        x_n = E[b, n] + pos[n] + resp[r_{n-1}] (resp row 2 marks "no previous
-        response" at n = 0), causal attention, logit_n = head_w . y_n + head_b,
-        binary cross-entropy, averaged over all B*L predictions (over the real
-        ones when histories end in padding, label -1).
-    nr: additive attention over the first L - n_cand encodings gives the user
-        vector, dot products with the n_cand candidate encodings give scores,
-        loss = -log softmax(scores)[0] (the first candidate is the click),
+    kt: `kt_logits` per history, binary cross-entropy, averaged over all B*L
+        predictions (over the real ones when histories end in padding, label -1).
+    nr: `nr_scores` per user over the first L - n_cand encodings (the click
+        history) and the n_cand candidate encodings, loss = -log softmax(scores)[0],
         averaged over the B users.  History slots with label -1 hold no click
         (a user with fewer clicks than slots) and take no part.
     """
@@ -242,15 +285,8 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
             n = int(neg[0]) if len(neg) else L
             if n == 0:
                 continue
-            prev = torch.cat([torch.full((1,), 2, dtype=torch.long), lab[b, :n - 1]])
-            x = E[b, :n] + th["pos"][:n] + th["resp"][prev]
-            for l in range(shape.task_layers):
-                x = transformer_layer(x, th, f"t{l}.", shape.task_heads, causal=True,
-                                      attn_only=shape.task_attn_only)
-            z = x @ th["head_w"] + th["head_b"]
-            y = lab[b, :n].to(E.dtype)
-            # BCE with logits: softplus(z) - y*z, written with a stable softplus
-            total = total + (torch.clamp(z, min=0) + torch.log1p(torch.exp(-z.abs())) - y * z).sum()
+            z = kt_logits(th, E[b, :n], lab[b, :n], shape)
+            total = total + bce_with_logits_sum(z, lab[b, :n].to(E.dtype))
             n_pred += n
         return total / max(n_pred, 1)
     if shape.task == "nr":
@@ -260,11 +296,7 @@ def task_loss(th: Dict[str, torch.Tensor], E: torch.Tensor, labels, shape) -> to
             hist, cand = E[b, :n_hist], E[b, n_hist:]
             # a click history shorter than its slots: the slots with label -1 hold no click and are simply left out
             hist = hist[(lab[b, :n_hist] >= 0).nonzero()[:, 0]]
-            a = torch.tanh(hist @ th["wa"].T + th["ba"]) @ th["qa"]
-            alpha = softmax_rows(a[None, :])[0]
-            u = alpha @ hist
-            s = cand @ u
-            total = total - (s[0] - s.max() - torch.log(torch.exp(s - s.max()).sum()))
+            total = total + softmax_ce_first(nr_scores(th, hist, cand, shape))
         return total / B
     raise KeyError(shape.task)
 
@@ -433,8 +465,8 @@ def multistep_window_pseudo_target(shape, ce_params, task_params, item_tokens, b
                                    dtype=torch.float64):
     """One window of K = len(batches) steps of Algorithm 1 under the *trainable-embedding* reading of
     Section 4.3: the content representation of an item is a trainable embedding h~_i that the task module
-    keeps using after it has been modified ("based on updated content representations, we repeat the
-    process"), and the encoder regresses towards it (Eq. 9).
+    keeps using after it has been modified (later steps of the window run on the updated representations),
+    and the encoder regresses towards it (Eq. 9).
 
     * h~ starts as `cache` [n_items, d] (encoder outputs computed before the window).
     * Step 1 (Eq. 4) inside the window: the task module reads E[p] = h~[ids[p]], i.e. the cached encoding
@@ -483,7 +515,7 @@ def multistep_window_pseudo_target(shape, ce_params, task_params, item_tokens, b
 
 
 # ---------------------------------------------------------------------------
-# Optimiser (Section A, implementation details: "Adam with Noam scheduler", learning rate 1e-4)
+# Optimiser (Appendix D, experiment details: Adam under the Noam learning-rate scheme, rate 1e-4)
 # ---------------------------------------------------------------------------
 def noam_rate(t: int, peak: float, warmup: int) -> float:
     """Learning rate at update t = 1, 2, ... under the Noam scheme (Vaswani et al. 2017, Eq. 3):

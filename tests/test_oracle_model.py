@@ -95,23 +95,169 @@ def test_losses_at_zero_parameters():
     assert float(orc.task_loss(orc.as_torch(z, T64, False), E, lab, nr)) == pytest.approx(math.log(5), rel=1e-14)
 
 
-def test_kt_task_does_not_see_the_label_it_predicts():
-    # prediction n may depend on responses 0..n-1 only (Section 3.1)
-    shape = small_shape(task_attn_only=False)
-    ce, tk, toks, ids, lab = make(shape)
-    th = orc.as_torch(tk, T64, False)
-    E = torch.randn(1, shape.L, shape.d, dtype=T64, generator=torch.Generator().manual_seed(0))
+# ---- the task module's pieces: each pinned on the oracle's own function, each with a planted mistake -----------------
 
-    def logits(labels):
-        prev = torch.cat([torch.full((1,), 2, dtype=torch.long), torch.as_tensor(labels[0, :-1], dtype=torch.long)])
-        x = E[0] + th["pos"] + th["resp"][prev]
+def _must_fail(check, *args):
+    with pytest.raises(AssertionError):
+        check(*args)
+
+
+def _check_no_label_leak(logits_fn):
+    # prediction n may depend on responses 0..n-1 only (Section 3.1): two label rows that differ at position 3
+    # give identical logits 0..3 and a different logit 4
+    shape = small_shape(task_attn_only=False)
+    _, tk, _, _, _ = make(shape)
+    th = orc.as_torch(tk, T64, False)
+    E = torch.randn(shape.L, shape.d, dtype=T64, generator=torch.Generator().manual_seed(0))
+    a = np.array([1, 0, 1, 1, 0]); b = a.copy(); b[3] = 0
+    with torch.no_grad():
+        la, lb = logits_fn(th, E, a, shape), logits_fn(th, E, b, shape)
+    assert la.shape == (shape.L,)
+    np.testing.assert_allclose(la[:4].numpy(), lb[:4].numpy(), rtol=0, atol=0)      # logits 0..3 unchanged
+    assert abs(float(la[4] - lb[4])) > 1e-9                                         # logit 4 sees response 3
+    # position 0 uses the "no previous response" row 2 of resp: it moves with that row and with nothing else of resp
+    th2 = dict(th); th2["resp"] = th["resp"].clone(); th2["resp"][2] += 0.5
+    th3 = dict(th); th3["resp"] = th["resp"].clone(); th3["resp"][:2] += 0.5
+    with torch.no_grad():
+        assert abs(float(logits_fn(th2, E, a, shape)[0] - la[0])) > 1e-9
+        assert float(logits_fn(th3, E, a, shape)[0]) == float(la[0])
+
+
+def test_kt_logits_do_not_see_the_label_they_predict():
+    _check_no_label_leak(orc.kt_logits)
+
+    def leaky(th, E, labels, shape):          # planted mistake: position n reads its own response r_n
+        lab = torch.as_tensor(np.asarray(labels), dtype=torch.long)
+        x = E + th["pos"][:E.shape[0]] + th["resp"][lab]
         for l in range(shape.task_layers):
             x = orc.transformer_layer(x, th, f"t{l}.", shape.task_heads, True, shape.task_attn_only)
         return x @ th["head_w"] + th["head_b"]
-    a = np.array([[1, 0, 1, 1, 0]]); b = a.copy(); b[0, 3] = 0
-    la, lb = logits(a), logits(b)
-    np.testing.assert_allclose(la[:4].numpy(), lb[:4].numpy(), rtol=0, atol=0)      # logits 0..3 unchanged
-    assert abs(float(la[4] - lb[4])) > 1e-9                                         # logit 4 sees response 3
+
+    def shifted_two(th, E, labels, shape):    # planted mistake: response n-2 instead of n-1
+        lab = torch.as_tensor(np.asarray(labels), dtype=torch.long)
+        prev = torch.cat([torch.full((2,), 2, dtype=torch.long), lab[:E.shape[0] - 2]])
+        x = E + th["pos"][:E.shape[0]] + th["resp"][prev]
+        for l in range(shape.task_layers):
+            x = orc.transformer_layer(x, th, f"t{l}.", shape.task_heads, True, shape.task_attn_only)
+        return x @ th["head_w"] + th["head_b"]
+    _must_fail(_check_no_label_leak, leaky)
+    _must_fail(_check_no_label_leak, shifted_two)
+
+
+def test_kt_logits_with_one_position_is_the_plain_head():
+    # a one-position history: causal attention over one key returns V itself, so with identity V / output
+    # projections the logit is head_w . 2 x_0 + head_b with x_0 = e_0 + pos_0 + resp_2 (closed form)
+    shape = small_shape(L=1)
+    d = shape.d
+    th = orc.as_torch(synth.task_params(shape, 1, sigma=0.3, plain=False), T64, False)
+    th["t0.wqkv"][2 * d:] = torch.eye(d, dtype=T64); th["t0.bqkv"].zero_()
+    th["t0.wo"] = torch.eye(d, dtype=T64); th["t0.bo"].zero_()
+    e0 = torch.randn(1, d, dtype=T64, generator=torch.Generator().manual_seed(3))
+    x0 = e0[0] + th["pos"][0] + th["resp"][2]
+    z = orc.kt_logits(th, e0, np.array([1]), shape)
+    assert float(z[0]) == pytest.approx(float(2 * x0 @ th["head_w"] + th["head_b"][0]), rel=1e-13)
+
+
+def _check_bce(sum_fn):
+    g = torch.Generator().manual_seed(5)
+    z = torch.randn(40, dtype=T64, generator=g) * 4
+    y = (torch.rand(40, generator=g) < 0.6).to(T64)
+    want = torch.nn.functional.binary_cross_entropy_with_logits(z, y, reduction="sum")
+    assert float(sum_fn(z, y)) == pytest.approx(float(want), rel=1e-13)
+    # far tails stay finite and keep their asymptote |z| on the wrong side, 0 on the right side
+    zt = torch.tensor([800.0, -800.0], dtype=T64)
+    assert float(sum_fn(zt, torch.tensor([0.0, 1.0], dtype=T64))) == pytest.approx(1600.0, rel=1e-14)
+    assert float(sum_fn(zt, torch.tensor([1.0, 0.0], dtype=T64))) == pytest.approx(0.0, abs=1e-300)
+
+
+def test_binary_cross_entropy_matches_the_library_at_random_logits():
+    _check_bce(orc.bce_with_logits_sum)
+    _must_fail(_check_bce, lambda z, y: (torch.nn.functional.softplus(z) + y * z).sum())          # sign of y z
+    _must_fail(_check_bce, lambda z, y: (torch.nn.functional.softplus(z) - (1 - y) * z).sum())    # inverted labels
+    _must_fail(_check_bce, lambda z, y: (torch.nn.functional.softplus(-z) - y * z).sum())         # softplus of -z
+
+
+def _check_first_candidate_ce(ce_fn):
+    g = torch.Generator().manual_seed(6)
+    for n in (2, 5):
+        s = torch.randn(n, dtype=T64, generator=g) * 3
+        want = torch.nn.functional.cross_entropy(s[None], torch.zeros(1, dtype=torch.long))
+        assert float(ce_fn(s)) == pytest.approx(float(want), rel=1e-13)
+    assert float(ce_fn(torch.tensor([900.0, 0.0, -900.0], dtype=T64))) == pytest.approx(0.0, abs=1e-300)
+    assert float(ce_fn(torch.tensor([0.0, 900.0], dtype=T64))) == pytest.approx(900.0, rel=1e-14)
+
+
+def test_candidate_cross_entropy_takes_the_first_candidate_as_the_click():
+    _check_first_candidate_ce(orc.softmax_ce_first)
+    _must_fail(_check_first_candidate_ce, lambda s: -torch.log_softmax(s, 0)[-1])     # positive = last candidate
+    _must_fail(_check_first_candidate_ce, lambda s: torch.log_softmax(s, 0)[0])       # sign
+    _must_fail(_check_first_candidate_ce, lambda s: -torch.log_softmax(-s, 0)[0])     # sign of the scores
+
+
+def _check_user_vector(user_fn):
+    shape = small_shape(task="nr", n_cand=3, L=8, d_a=6, task_layers=0)
+    th = orc.as_torch(synth.task_params(shape, 2, sigma=0.5, plain=False), T64, False)
+    h = torch.randn(5, shape.d, dtype=T64, generator=torch.Generator().manual_seed(7))
+    # q = 0: every score equal, the user vector is the plain mean of the clicked rows
+    th0 = dict(th); th0["qa"] = torch.zeros_like(th["qa"])
+    np.testing.assert_allclose(user_fn(th0, h).numpy(), h.mean(0).numpy(), rtol=1e-13)
+    # a one-click history: the user vector is that row, whatever the parameters
+    np.testing.assert_allclose(user_fn(th, h[2:3]).numpy(), h[2].numpy(), rtol=1e-14)
+    # general case: the weights are the library softmax of q . tanh(W h + b), a convex combination
+    w = torch.softmax(torch.tanh(torch.nn.functional.linear(h, th["wa"], th["ba"])) @ th["qa"], 0)
+    np.testing.assert_allclose(user_fn(th, h).numpy(), (w[:, None] * h).sum(0).numpy(), rtol=1e-13)
+    # one saturated score picks its row: scale q so that row 4's score dominates
+    t = torch.tanh(torch.nn.functional.linear(h, th["wa"], th["ba"]))
+    thq = dict(th); thq["qa"] = 500.0 * (t[4] - t[:4].mean(0))
+    sc = t @ thq["qa"]
+    assert float(sc[4] - sc[:4].max()) > 50
+    np.testing.assert_allclose(user_fn(thq, h).numpy(), h[4].numpy(), rtol=1e-12)
+
+
+def test_user_vector_closed_forms():
+    _check_user_vector(orc.nr_user_vector)
+
+    def no_tanh(th, h):                       # planted mistake: scores without the tanh
+        return torch.softmax(torch.nn.functional.linear(h, th["wa"], th["ba"]) @ th["qa"], 0) @ h
+
+    def weights_on_projection(th, h):         # planted mistake: sums the projected rows instead of the encodings
+        t = torch.tanh(torch.nn.functional.linear(h, th["wa"], th["ba"]))
+        return torch.nn.functional.pad(torch.softmax(t @ th["qa"], 0) @ t, (0, h.shape[1] - t.shape[1]))
+
+    def unnormalised(th, h):                  # planted mistake: exp weights without the softmax's division
+        return torch.exp(torch.tanh(torch.nn.functional.linear(h, th["wa"], th["ba"])) @ th["qa"]) @ h
+    _must_fail(_check_user_vector, no_tanh)
+    _must_fail(_check_user_vector, weights_on_projection)
+    _must_fail(_check_user_vector, unnormalised)
+
+
+def test_scores_are_dot_products_with_the_user_vector_and_task_loss_is_the_mean_of_its_pieces():
+    nr = small_shape(task="nr", n_cand=3, L=8, d_a=6, task_layers=0, B=3)
+    th = orc.as_torch(synth.task_params(nr, 2, sigma=0.5, plain=False), T64, False)
+    E = torch.randn(nr.B, nr.L, nr.d, dtype=T64, generator=torch.Generator().manual_seed(8))
+    lab = np.zeros((nr.B, nr.L), np.int32)
+    with torch.no_grad():
+        s = orc.nr_scores(th, E[0, :5], E[0, 5:], nr)
+        u = orc.nr_user_vector(th, E[0, :5])
+        np.testing.assert_allclose(s.numpy(), [float(E[0, 5 + j] @ u) for j in range(3)], rtol=1e-13)
+        # the batch loss is the library cross-entropy (target 0, mean over users) of the per-user scores
+        S = torch.stack([orc.nr_scores(th, E[b, :5], E[b, 5:], nr) for b in range(nr.B)])
+        want = torch.nn.functional.cross_entropy(S, torch.zeros(nr.B, dtype=torch.long))
+        assert float(orc.task_loss(th, E, lab, nr)) == pytest.approx(float(want), rel=1e-13)
+        # candidates are the LAST n_cand positions of a user's row: permuting the history rows leaves the loss alone,
+        # swapping a history row with a candidate does not
+        Ep = E.clone(); Ep[:, :5] = E[:, [4, 2, 0, 1, 3]]
+        assert float(orc.task_loss(th, Ep, lab, nr)) == pytest.approx(float(want), rel=1e-13)
+        Es = E.clone(); Es[:, 0], Es[:, 5] = E[:, 5], E[:, 0]
+        assert abs(float(orc.task_loss(th, Es, lab, nr)) - float(want)) > 1e-6
+    kt = small_shape(task_attn_only=False, B=3)
+    thk = orc.as_torch(synth.task_params(kt, 2, sigma=0.3, plain=False), T64, False)
+    Ek = torch.randn(kt.B, kt.L, kt.d, dtype=T64, generator=torch.Generator().manual_seed(9))
+    labk = synth.labels(3, kt.B, kt.L, 0.6)
+    with torch.no_grad():
+        Z = torch.stack([orc.kt_logits(thk, Ek[b], labk[b], kt) for b in range(kt.B)])
+        want = torch.nn.functional.binary_cross_entropy_with_logits(Z, torch.as_tensor(labk, dtype=T64), reduction="mean")
+        assert float(orc.task_loss(thk, Ek, labk, kt)) == pytest.approx(float(want), rel=1e-13)
 
 
 # ---- derivatives: central finite differences on a 1-layer encoder ----------
@@ -269,7 +415,7 @@ def test_pseudo_target_window_k1_fresh_cache_is_e2e():
 
 
 def test_pseudo_target_embedding_follows_library_sgd_with_rate_one():
-    # "treating it as trainable embedding": a torch Parameter updated by torch.optim.SGD(lr=1) over the same batches
+    # the encoding treated as a trainable embedding (Section 4.3): a torch Parameter updated by torch.optim.SGD(lr=1) over the same batches
     # must end at the oracle's h~ (duplicates of an item inside a batch add up through autograd's index backward)
     shape = small_shape(n_items=6, B=2, L=6)
     ce, tk, toks, _, _ = make(shape, seed=6)
