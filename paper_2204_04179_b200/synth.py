@@ -85,6 +85,8 @@ def config(name: str) -> GramShape:
         return config("kt").replace(name="kt_multistep", K=8)
     if name == "nr_additive":     # news recommendation with the paper's item pooling (additive attention over the title tokens)
         return config("nr").replace(name="nr_additive", pooling="additive")
+    if name == "nr_mhsa":         # news recommendation with one self-attention layer over the clicked items (Appendix D)
+        return config("nr").replace(name="nr_mhsa", task_layers=1, task_heads=12, task_attn_only=True)
     if name == "kt_6l":           # the same with the paper's own encoder depth (Appendix D: a 6-layer, 768-wide model)
         return config("kt").replace(name="kt_6l", n_layers=6)
     raise KeyError(name)
@@ -178,7 +180,10 @@ def task_param_spec(s: GramShape):
         spec += [("head_w", (s.d,)), ("head_b", (1,))]
         return spec
     if s.task == "nr":
-        return [("wa", (s.d_a, s.d)), ("ba", (s.d_a,)), ("qa", (s.d_a,))]
+        spec = []
+        for l in range(s.task_layers):       # self-attention layers over the clicked items, ahead of the additive attention
+            spec += _layer_spec(f"t{l}.", s.d, s.task_d_ff, s.task_attn_only)
+        return spec + [("wa", (s.d_a, s.d)), ("ba", (s.d_a,)), ("qa", (s.d_a,))]
     raise KeyError(s.task)
 
 

@@ -269,12 +269,14 @@ def _loss_only(shape, ce, tk, toks, ids, lab):
         return float(orc.task_loss(th_cf, E, lab, shape))
 
 
-@pytest.mark.parametrize("variant", ["kt_attn_mean", "kt_full_cls", "nr_cls"])
+@pytest.mark.parametrize("variant", ["kt_attn_mean", "kt_full_cls", "nr_cls", "nr_mhsa"])
 def test_e2e_gradients_match_finite_differences(variant):
     if variant == "kt_attn_mean":
         shape = small_shape()
     elif variant == "kt_full_cls":
         shape = small_shape(pooling="cls", task_attn_only=False)
+    elif variant == "nr_mhsa":
+        shape = small_shape(pooling="cls", task="nr", n_cand=3, L=7, d_a=5, task_layers=1, task_attn_only=True)
     else:
         shape = small_shape(pooling="cls", task="nr", n_cand=3, L=6, d_a=5, task_layers=0)
     ce, tk, toks, ids, lab = make(shape, seed=4)
@@ -614,6 +616,36 @@ def test_additive_pooling_special_cases_and_finite_differences():
             dn = OrderedDict((k, v.copy()) for k, v in ce.items()); dn[name][idx] -= 1e-6
             fd = (loss_at(up) - loss_at(dn)) / 2e-6
             assert abs(fd - res["grad_ce"][name][idx]) <= 1e-7 + 1e-5 * abs(fd), (name, idx, fd, res["grad_ce"][name][idx])
+
+
+def test_user_self_attention_layer_is_the_library_attention_with_empty_slots_masked():
+    # NR with one self-attention layer over the clicked items (Appendix D): the scores equal those computed from
+    # torch.nn.MultiheadAttention run over ALL history slots with the empty ones masked as keys, its rows for
+    # the clicked slots (plus the residual) fed to the user vector
+    shape = small_shape(task="nr", task_layers=1, task_heads=4, task_attn_only=True, n_cand=3, L=9, d_a=6, B=1)
+    d = shape.d
+    tk = synth.task_params(shape, 5, sigma=0.4, plain=False)
+    assert list(tk)[:4] == ["t0.wqkv", "t0.bqkv", "t0.wo", "t0.bo"] and list(tk)[-3:] == ["wa", "ba", "qa"]
+    th = orc.as_torch(tk, T64, False)
+    E = torch.randn(9, d, dtype=T64, generator=torch.Generator().manual_seed(11))
+    clicked = [0, 2, 3, 5]                                   # slots 1 and 4 are empty
+    mha = torch.nn.MultiheadAttention(d, 4, dropout=0.0, batch_first=True, dtype=T64)
+    with torch.no_grad():
+        mha.in_proj_weight.copy_(th["t0.wqkv"]); mha.in_proj_bias.copy_(th["t0.bqkv"])
+        mha.out_proj.weight.copy_(th["t0.wo"]); mha.out_proj.bias.copy_(th["t0.bo"])
+        pad = torch.ones(1, 6, dtype=torch.bool); pad[0, clicked] = False
+        y = E[None, :6] + mha(E[None, :6], E[None, :6], E[None, :6], key_padding_mask=pad, need_weights=False)[0]
+        want = E[6:] @ orc.nr_user_vector(th, y[0, clicked])
+        got = orc.nr_scores(th, E[clicked], E[6:], shape)
+    np.testing.assert_allclose(got.numpy(), want.numpy(), rtol=1e-11)
+    # and task_loss routes the same way: label -1 marks the empty slots
+    lab = np.zeros((1, 9), np.int32); lab[0, [1, 4]] = -1
+    with torch.no_grad():
+        loss = orc.task_loss(th, E[None], lab, shape)
+    assert float(loss) == pytest.approx(float(torch.nn.functional.cross_entropy(want[None], torch.zeros(1, dtype=torch.long))), rel=1e-11)
+    # the layer matters: without it the scores differ
+    with torch.no_grad():
+        assert float((orc.nr_scores(th, E[clicked], E[6:], shape.replace(task_layers=0)) - got).abs().max()) > 1e-3
 
 
 def test_empty_click_slots_are_left_out():
