@@ -54,8 +54,8 @@ enum { GRAM_OPT_SGD = 0, GRAM_OPT_ADAM = 1 };
 /* Multi-step GRAM (Section 4.2, Algorithm 1 with N > 1), how a window treats the content representations:
  * GRAM_MULTI_TABLE: the task module reads the unchanged cached encodings during the whole window, the
  *   gradients of Eq. 6 go to a separate per-item table, and the encoder's cotangent is table[i].
- * GRAM_MULTI_PSEUDO_TARGET: the trainable-embedding reading of Section 4.3 ("treating it as trainable
- *   embedding", "based on updated content representations, we repeat the process"): the task module reads
+ * GRAM_MULTI_PSEUDO_TARGET: the other reading of Section 4.3 and Algorithm 1, step 3 (Eqs. 6 and 9), in which an
+ *   item's representation is itself a trainable embedding that later steps keep using: the task module reads
  *   the pseudo-target h~_i = cache[i] - table[i], i.e. the cached encoding minus every gradient the item
  *   has received so far in the window (Eq. 6, SGD with learning rate 1), and the encoder regresses
  *   towards it with the pseudo-loss of Eq. 9: its cotangent is CE(c_i; theta) - h~_i, which carries the
@@ -91,7 +91,7 @@ typedef struct gram_config {
   float lr_task;               /* SGD step applied to the task parameters after every gram_step (0 = none) */
   float lr_ce;                 /* SGD step applied to the encoder parameters after an encoder pass (0 = none) */
   int32_t optimizer;           /* GRAM_OPT_SGD: plain steps of lr_task / lr_ce.  GRAM_OPT_ADAM: Adam with the Noam
-                                  learning-rate scheme (Section A); lr_task / lr_ce are then the peak rates */
+                                  learning-rate scheme (Appendix D); lr_task / lr_ce are then the peak rates */
   int32_t noam_warmup;         /* updates until the peak rate; <= 0: constant rate */
   float adam_beta1, adam_beta2, adam_eps;   /* <= 0: 0.9, 0.999, 1e-8 */
   int32_t multistep_variant;   /* K > 1: GRAM_MULTI_TABLE or GRAM_MULTI_PSEUDO_TARGET */
@@ -99,6 +99,10 @@ typedef struct gram_config {
                                    more with the new parameters and store those encodings in the cache (Algorithm 1,
                                    Eq. 4 produces h with the parameters of the current step); 0: the cache keeps the
                                    forward values of the encoder pass, one update old */
+  int32_t defer_update;        /* != 0: gram_step computes gradients and applies no update; the caller calls
+                                  gram_optimizer_step itself, e.g. after averaging the gradients over data-parallel
+                                  replicas (Section 5.1 trains with distributed data parallelism).  Not with
+                                  refresh_after_update, which encodes with the updated parameters inside the step */
 } gram_config;
 
 typedef struct gram_step_report {
@@ -137,6 +141,11 @@ gram_status gram_get_params(gram_ctx* ctx, int module, float* h_params, size_t n
 /* Gradients of the last gram_step / gram_encoder_backward / gram_task, same layout (synchronises). */
 gram_status gram_get_grads(gram_ctx* ctx, int module, float* h_grads, size_t n);
 gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream);
+/* Device address and length of a module's fp32 gradient buffer (same layout as the parameters).  The buffer
+ * belongs to the context and lives as long as it; a data-parallel trainer all-reduces it in place between
+ * gram_step (with defer_update) and gram_optimizer_step (Section 5.1).  Work queued on the stream that ran the
+ * step must have finished, or be ordered, before another stream touches the buffer. */
+gram_status gram_grads_device(gram_ctx* ctx, int module, float** d_grads, size_t* n);
 /* The configured update of one module from its current gradients (what gram_step applies by itself): an SGD step,
  * or one Adam update at the module's next update count with the Noam rate of that count.  For callers that drive
  * the stages one by one. */
@@ -185,7 +194,8 @@ gram_status gram_encode_unique(gram_ctx* ctx, const int32_t* d_item_tokens, cons
  * (No counterpart in the paper.) */
 gram_status gram_selftest_bounded_wait(gram_ctx* ctx, gram_stream stream);
 
-/* Stage 3: d_E[p, :] = d_src[d_index[p], :] for p < P.  Single-step: src = H,
+/* Stage 3 (Section 4.3: the encoder's output h_i is handed to the task module, which completes the forward pass
+ * with it; Fig. 1 draws the copies): d_E[p, :] = d_src[d_index[p], :] for p < P.  Single-step: src = H,
  * index = inverse.  Multi-step: src = the encoding cache, index = ids.
  * Rows are d elements of `dtype`; n_src_rows bounds the index (ID_RANGE else). */
 gram_status gram_gather(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, const int32_t* d_index, int64_t P,
@@ -258,7 +268,7 @@ gram_status gram_window_reset(gram_ctx* ctx, gram_stream stream);
  * [ceil(n_items/32)], cache fp32 [n_items, d] (converted).  NULL skips one. */
 gram_status gram_get_window(gram_ctx* ctx, float* h_table, uint32_t* h_touched, float* h_cache);
 
-/* --- checkpoint / resume (the paper keeps the checkpoint of the best validation epoch, Section A) ------------------
+/* --- checkpoint / resume (the paper keeps the checkpoint of the best validation epoch, Appendix D) ------------------
  * Everything a context holds besides what the caller gave it: parameters (gram_get_params / gram_set_params), the
  * optimiser's state, and for K > 1 the open window.  Exported by one context and imported into another context of the
  * same configuration, training continues bit for bit.  All calls synchronise. */
@@ -329,8 +339,35 @@ gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const v
                            int c_f32, const float* d_bias, int accumulate, int64_t M, int32_t N, int64_t K,
                            gram_stream stream);
 
-/* --- the optimiser's two pieces, exported so that they can be tested on their own (Section A: "Adam with Noam
- * scheduler") -------------------------------------------------------------
+/* The same product followed by one of the fused epilogues the encoder's layers use (Appendix D: attention layers of
+ * width 768; each epilogue replaces a separate pass over the [M, N] result):
+ *   v = acc + d_bias[n]
+ *   gelu != 0:        d_gelu_grad_out(m, n) = gelu'(v) (bf16, may be NULL);  v = gelu(v)     (erf form)
+ *   d_gelu_grad_in:   v *= d_gelu_grad_in(m, n) (bf16)
+ *   d_res:            v += d_res(m, n) (fp32), or, when d_res_mean is given, LayerNorm applied where it is read:
+ *                     v += (d_res(m, n) - d_res_mean[m]) * d_res_rstd[m] * d_res_gamma[n] + d_res_beta[n]
+ *   accumulate != 0:  v += C(m, n)                                                   (fp32 C only)
+ *   d_copy_bf16:      bf16 copy of the stored result
+ * At most one of d_res, d_gelu_grad_in and accumulate per call.  All [M, N] matrices share C's leading
+ * dimension N.  e == NULL is a plain product. */
+typedef struct gram_gemm_epilogue {
+  const float* d_bias;
+  const float* d_res;
+  const float* d_res_mean;
+  const float* d_res_rstd;
+  const float* d_res_gamma;
+  const float* d_res_beta;
+  void* d_gelu_grad_out;
+  const void* d_gelu_grad_in;
+  void* d_copy_bf16;
+  int32_t gelu, accumulate;
+} gram_gemm_epilogue;
+gram_status gram_gemm_bf16_epilogue(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
+                                    int c_f32, const gram_gemm_epilogue* e, int64_t M, int32_t N, int64_t K,
+                                    gram_stream stream);
+
+/* --- the optimiser's two pieces, exported so that they can be tested on their own (Appendix D: Adam under the
+ * Noam learning-rate scheme) ----------------------------------------------
  * gram_noam_rate (host only): *h_rate = peak * min(t / warmup, sqrt(warmup / t)) for update t >= 1, the Noam curve
  * scaled so that its maximum, at t = warmup, is `peak`; warmup <= 0 gives the constant `peak`.
  * gram_adam_update: one Adam update of n fp32 parameters in place at update count t >= 1:

@@ -34,7 +34,8 @@ SYMBOLS = ["gram_create", "gram_destroy", "gram_sync", "gram_last_error", "gram_
            "gram_window_reset", "gram_get_window", "gram_gemm_bf16", "gram_profile", "gram_profile_read",
            "gram_launch_count", "gram_profile_dump", "gram_accumulate_static", "gram_optimizer_step",
            "gram_optimizer_reset", "gram_noam_rate", "gram_adam_update", "gram_state_export", "gram_state_import",
-           "gram_optimizer_export", "gram_optimizer_import", "gram_selftest_bounded_wait"]
+           "gram_optimizer_export", "gram_optimizer_import", "gram_selftest_bounded_wait", "gram_grads_device",
+           "gram_gemm_bf16_epilogue"]
 
 KINDS = ["gemm", "attention", "layernorm", "colsum", "embed_pool", "dedup", "gather", "accumulate", "task_head", "other",
          "optimizer"]
@@ -47,7 +48,13 @@ class GramConfig(C.Structure):
                [("P_max", C.c_int64), ("d_max", C.c_int32), ("K", C.c_int32), ("ce_micro_batch", C.c_int32),
                 ("lr_task", C.c_float), ("lr_ce", C.c_float), ("optimizer", C.c_int32), ("noam_warmup", C.c_int32),
                 ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float),
-                ("multistep_variant", C.c_int32), ("refresh_after_update", C.c_int32)]
+                ("multistep_variant", C.c_int32), ("refresh_after_update", C.c_int32), ("defer_update", C.c_int32)]
+
+
+class GramGemmEpilogue(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("d_bias", "d_res", "d_res_mean", "d_res_rstd", "d_res_gamma", "d_res_beta",
+                                          "d_gelu_grad_out", "d_gelu_grad_in", "d_copy_bf16")] + \
+               [("gelu", C.c_int32), ("accumulate", C.c_int32)]
 
 
 class GramStepReport(C.Structure):
@@ -174,6 +181,12 @@ class Gram:
         out = np.empty(self.param_count(module), np.float32)
         self._ck(lib().gram_get_grads(self._h, module, _ptr(out), C.c_size_t(out.size)))
         return out
+
+    def grads_device(self, module: int):
+        """(device address, element count) of a module's fp32 gradient buffer."""
+        p, n = C.c_void_p(0), C.c_size_t(0)
+        self._ck(lib().gram_grads_device(self._h, module, C.byref(p), C.byref(n)))
+        return p.value or 0, n.value
 
     def zero_grads(self, module: int, stream=None):
         self._ck(lib().gram_zero_grads(self._h, module, _stream(stream)))
@@ -328,6 +341,21 @@ class Gram:
                                       _ptr(Cm), C.c_int(int(Cm.dtype == torch.float32)), _ptr(bias),
                                       C.c_int(int(accumulate)), C.c_int64(M), C.c_int32(N), C.c_int64(K),
                                       _stream(stream)))
+
+
+    def gemm_bf16_epilogue(self, A, a_kmajor, Bm, b_kmajor, Cm, M, N, K, bias=None, res=None, res_ln=None, gelu=False,
+                           gelu_grad_out=None, gelu_grad_in=None, copy_bf16=None, accumulate=False, stream=None):
+        """res_ln: (mean, rstd, gamma, beta) applied to `res` where it is read."""
+        import torch
+        e = GramGemmEpilogue()
+        e.d_bias = _ptr(bias); e.d_res = _ptr(res)
+        if res_ln is not None:
+            e.d_res_mean, e.d_res_rstd, e.d_res_gamma, e.d_res_beta = (_ptr(t) for t in res_ln)
+        e.d_gelu_grad_out = _ptr(gelu_grad_out); e.d_gelu_grad_in = _ptr(gelu_grad_in); e.d_copy_bf16 = _ptr(copy_bf16)
+        e.gelu = int(gelu); e.accumulate = int(accumulate)
+        self._ck(lib().gram_gemm_bf16_epilogue(self._h, _ptr(A), C.c_int(int(a_kmajor)), _ptr(Bm), C.c_int(int(b_kmajor)),
+                                               _ptr(Cm), C.c_int(int(Cm.dtype == torch.float32)), C.byref(e), C.c_int64(M),
+                                               C.c_int32(N), C.c_int64(K), _stream(stream)))
 
 
 def accumulate_static(dE, perm, seg_off, U, G, stream=None, P=None, d=None):

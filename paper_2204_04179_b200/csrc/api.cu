@@ -268,7 +268,7 @@ gram_status gram_accumulate_multistep(gram_ctx* ctx, const float* d_dE, const in
     if (!d_touched_bits) d_touched_bits = model_touched(ctx->model);
   }
   GRAM_TRY(accumulate_launch(ctx, &ctx->iws, d_dE, 0, d_perm, d_seg_off, P, U, nullptr, d, d_unique, 1, d_table, S(stream)));
-  return touched_mark_launch(ctx, d_unique, U, n_items, d_touched_bits, S(stream));
+  return touched_mark_launch(ctx, d_unique, U, nullptr, n_items, d_touched_bits, nullptr, 0, S(stream));
 }
 
 gram_status gram_touched_list(gram_ctx* ctx, const uint32_t* d_touched_bits, int32_t n_items, int32_t* d_list,
@@ -301,6 +301,11 @@ gram_status gram_get_grads(gram_ctx* ctx, int module, float* h, size_t n) {
 gram_status gram_zero_grads(gram_ctx* ctx, int module, gram_stream stream) {
   NEED_MODEL("gram_zero_grads");
   return model_zero_grads(ctx->model, module, S(stream));
+}
+gram_status gram_grads_device(gram_ctx* ctx, int module, float** d_grads, size_t* n) {
+  NEED_MODEL("gram_grads_device");
+  if (!d_grads || !n) return gram_set_error(ctx, "gram_grads_device: null output"), GRAM_ERR_ARG;
+  return model_grads_device(ctx->model, module, d_grads, n);
 }
 gram_status gram_optimizer_step(gram_ctx* ctx, int module, gram_stream stream) {
   NEED_MODEL("gram_optimizer_step");
@@ -398,6 +403,29 @@ gram_status gram_gemm_bf16(gram_ctx* ctx, const void* d_A, int a_kmajor, const v
   e.accumulate = accumulate;
   return gemm_launch(ctx, &ctx->gws, GRAM_BF16, d_A, a_kmajor, a_kmajor ? K : M, d_B, b_kmajor, b_kmajor ? K : N, d_C,
                      c_f32, N, M, N, K, e, 1, S(stream));
+}
+
+gram_status gram_gemm_bf16_epilogue(gram_ctx* ctx, const void* d_A, int a_kmajor, const void* d_B, int b_kmajor, void* d_C,
+                                    int c_f32, const gram_gemm_epilogue* ep, int64_t M, int32_t N, int64_t K,
+                                    gram_stream stream) {
+  if (!ctx) return GRAM_ERR_ARG;
+  if (M < 0 || N < 0 || K <= 0 || (M % 8) || (N % 8) || (K % 8))
+    return gram_set_error(ctx, "gram_gemm_bf16_epilogue: M, N, K must be positive multiples of 8"), GRAM_ERR_ARG;
+  GemmEpilogue e;
+  if (ep) {
+    if (ep->d_res_mean && !(ep->d_res && ep->d_res_rstd && ep->d_res_gamma && ep->d_res_beta))
+      return gram_set_error(ctx, "gram_gemm_bf16_epilogue: LayerNorm on the residual needs all of res, mean, rstd, gamma, beta"), GRAM_ERR_ARG;
+    e.bias = ep->d_bias;
+    e.res = ep->d_res; e.res_mean = ep->d_res_mean; e.res_rstd = ep->d_res_rstd; e.res_gamma = ep->d_res_gamma; e.res_beta = ep->d_res_beta;
+    e.pre = ep->d_gelu_grad_out;
+    e.dgelu_pre = ep->d_gelu_grad_in;
+    e.copy_out = ep->d_copy_bf16;
+    e.gelu = ep->gelu;
+    e.accumulate = ep->accumulate;
+    e.tag = "gemm_epilogue";
+  }
+  return gemm_launch(ctx, &ctx->gws, GRAM_BF16, d_A, a_kmajor, a_kmajor ? K : M, d_B, b_kmajor, b_kmajor ? K : N, d_C,
+                     c_f32, N, M, N, K, e, 0, S(stream));
 }
 
 }  // extern "C"

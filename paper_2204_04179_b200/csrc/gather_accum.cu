@@ -56,6 +56,47 @@ __global__ void gather_scalar_kernel(const T* __restrict__ src, int64_t n_src_ro
   }
 }
 
+// dst[p, :] (fp32) = src[index[p], :] (bf16): the Multi-step gather from a bf16 encoding cache, widened on the way so
+// that the task module's fp32 input is written once.  A warp per row, 8 elements (16 bytes in, 32 out) per lane and step.
+template <int ROWS>
+__global__ void __launch_bounds__(256) gather_widen_kernel(const uint4* __restrict__ src, int64_t n_src_rows,
+                                                           const int32_t* __restrict__ index, int64_t P, int nvec,
+                                                           float4* __restrict__ dst, int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t p0 = warp * ROWS; p0 < P; p0 += nwarps * ROWS) {
+    int64_t row[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      int64_t p = p0 + r;
+      int32_t i = (p < P) ? index[p] : 0;
+      if (i < 0 || i >= n_src_rows) {
+        gram_device_fail(status, GRAM_ERR_ID_RANGE);
+        i = 0;
+      }
+      row[r] = i;
+    }
+    for (int c = lane; c < nvec; c += 32) {
+      uint4 v[ROWS];
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) v[r] = __ldg(src + row[r] * nvec + c);
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) {
+        if (p0 + r < P) {
+          const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v[r].x));
+          const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v[r].y));
+          const float2 e = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v[r].z));
+          const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v[r].w));
+          float4* q = dst + ((p0 + r) * nvec + c) * 2;
+          __stcs(q, make_float4(a.x, a.y, b.x, b.y));
+          __stcs(q + 1, make_float4(e.x, e.y, f.x, f.y));
+        }
+      }
+    }
+  }
+}
+
 // out[r, :] = a[index[r], :] - b[index[r], :], or x[r, :] - that; a warp per row, 4 floats per lane and step
 __global__ void __launch_bounds__(256) gather_diff_kernel(const float* __restrict__ a, const float* __restrict__ b,
                                                           int64_t n_src_rows, const int32_t* __restrict__ index, int64_t n,
@@ -162,9 +203,11 @@ __global__ void __launch_bounds__(256) segsum_chunks_kernel(const InT* __restric
                                                             const int32_t* __restrict__ rows, int add,
                                                             float* __restrict__ out, float* __restrict__ partial,
                                                             int2* __restrict__ span, int32_t* status,
-                                                            const int32_t* __restrict__ d_U) {
+                                                            const int32_t* __restrict__ d_U,
+                                                            const int32_t* __restrict__ gate) {
   if (d_U) U = *d_U;            // the number of items may live on the device
   if (U <= 0) return;
+  if (gate && *gate) return;    // an earlier kernel of the step reported an error: leave the accumulated rows alone
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (w >= (int64_t)nchunks * nslabs) return;
@@ -239,10 +282,12 @@ __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __rest
                                                            int d, int64_t R, int nchunks, int nslabs,
                                                            const int32_t* __restrict__ rows, int add,
                                                            float* __restrict__ out, const float* __restrict__ partial,
-                                                           const int2* __restrict__ span, const int32_t* __restrict__ d_U) {
+                                                           const int2* __restrict__ span, const int32_t* __restrict__ d_U,
+                                                           const int32_t* __restrict__ gate) {
   __shared__ float4 red[8][VPL][32];
   if (d_U) U = *d_U;
   if (U <= 0) return;
+  if (gate && *gate) return;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int chunk = blockIdx.x / nslabs, slab = blockIdx.x - chunk * nslabs;
   const int col0 = slab * (VPL * 128);
@@ -298,16 +343,23 @@ __global__ void __launch_bounds__(256) segsum_fixup_kernel(const int32_t* __rest
   }
 }
 
-__global__ void touched_mark_kernel(const int32_t* __restrict__ unique, int32_t U, int32_t n_items,
-                                    uint32_t* __restrict__ bits, int32_t* status) {
-  int32_t u = blockIdx.x * blockDim.x + threadIdx.x;
-  if (u >= U) return;
-  int32_t i = unique[u];
-  if (i < 0 || i >= n_items) {
-    gram_device_fail(status, GRAM_ERR_ID_RANGE);
-    return;
+// d_U (may be null): the number of items lives on the device.  count (may be null): one word that counts the set
+// bits (integer adds: the total does not depend on their order).  gated: nothing is marked once the status word is set.
+__global__ void touched_mark_kernel(const int32_t* __restrict__ unique, int32_t U, const int32_t* __restrict__ d_U,
+                                    int32_t n_items, uint32_t* __restrict__ bits, int32_t* __restrict__ count,
+                                    int32_t* status, int gated) {
+  if (d_U) U = *d_U;
+  if (gated && *status) return;
+  for (int32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
+    const int32_t i = unique[u];
+    if (i < 0 || i >= n_items) {
+      gram_device_fail(status, GRAM_ERR_ID_RANGE);
+      continue;
+    }
+    const uint32_t bit = 1u << (i & 31);
+    const uint32_t old = atomicOr(&bits[i >> 5], bit);
+    if (count && !(old & bit)) atomicAdd(count, 1);
   }
-  atomicOr(&bits[i >> 5], 1u << (i & 31));
 }
 
 // ascending list of set bits, one block
@@ -390,6 +442,22 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
   return GRAM_OK;
 }
 
+gram_status gather_widen_launch(gram_ctx* ctx, const void* d_src_bf16, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                                int32_t d, float* d_E, cudaStream_t st) {
+  if (P < 0 || d <= 0 || n_src_rows <= 0 || (d % 8) || ((uintptr_t)d_src_bf16 % 16) || ((uintptr_t)d_E % 16))
+    return gram_set_error(ctx, "widening gather: bad argument (rows of a multiple of 8 elements, 16-byte aligned)"), GRAM_ERR_ARG;
+  if (P == 0) return GRAM_OK;
+  if (!d_src_bf16 || !d_index || !d_E) return gram_set_error(ctx, "widening gather: null buffer"), GRAM_ERR_ARG;
+  ProfScope prof(ctx, GRAM_K_GATHER, 4.0 * (double)d * (double)P + 2.0 * (double)d * (double)(n_src_rows < P ? n_src_rows : P) + 4.0 * P, 1, st);
+  constexpr int ROWS = 4;
+  int blocks = (int)ceil_div64(ceil_div64(P, ROWS), 8);
+  if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+  gather_widen_kernel<ROWS><<<blocks, 256, 0, st>>>((const uint4*)d_src_bf16, n_src_rows, d_index, P, d / 8, (float4*)d_E,
+                                                    gram_status_word(ctx));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
 gram_status gather_diff_launch(gram_ctx* ctx, const float* d_a, const float* d_b, int64_t n_src_rows, const int32_t* d_index,
                                int64_t n, int32_t d, const float* d_x, float* d_out, cudaStream_t st) {
   if (n < 0 || d <= 0 || n_src_rows <= 0 || (n > 0 && (!d_a || !d_b || !d_index || !d_out)))
@@ -406,19 +474,19 @@ gram_status gather_diff_launch(gram_ctx* ctx, const float* d_a, const float* d_b
 template <typename InT, int VPL>
 static void segsum_run(const void* d_in, const int32_t* d_perm, const int32_t* d_seg_off, int64_t P, int32_t U, int32_t d,
                        int64_t R, int nchunks, const int32_t* d_rows, int add, float* d_out, float* partial, int2* span,
-                       int32_t* status, const int32_t* d_U, cudaStream_t st) {
+                       int32_t* status, const int32_t* d_U, cudaStream_t st, const int32_t* gate = nullptr) {
   const int nslabs = ceil_div(d, VPL * 128);
   const int64_t warps = (int64_t)nchunks * nslabs;
   const int blocks = (int)ceil_div64(warps, 8);
   segsum_chunks_kernel<InT, VPL, 8><<<blocks, 256, 0, st>>>((const InT*)d_in, d_perm, d_seg_off, P, U, d, R, nchunks, nslabs,
-                                                            d_rows, add, d_out, partial, span, status, d_U);
+                                                            d_rows, add, d_out, partial, span, status, d_U, gate);
   if (nchunks > 1)
-    segsum_fixup_kernel<VPL><<<(unsigned)warps, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, span, d_U);
+    segsum_fixup_kernel<VPL><<<(unsigned)warps, 256, 0, st>>>(d_seg_off, P, U, d, R, nchunks, nslabs, d_rows, add, d_out, partial, span, d_U, gate);
 }
 
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
                               const int32_t* d_seg_off, int64_t P, int32_t U, const int32_t* d_U, int32_t d,
-                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st) {
+                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st, int gated) {
   if (P < 0 || U < 0 || d <= 0 || U > P) return gram_set_error(ctx, "gram_accumulate: bad argument"), GRAM_ERR_ARG;
   if (P == 0 || (U == 0 && !d_U)) return GRAM_OK;
   if (!d_in || !d_perm || !d_seg_off || !d_out) return gram_set_error(ctx, "gram_accumulate: null buffer"), GRAM_ERR_ARG;
@@ -433,22 +501,27 @@ gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_i
   int2* span = reinterpret_cast<int2*>(ws->partial + (size_t)kAccMaxChunks * 2 * (ws->d_max > 0 ? ws->d_max : 1));   // after the partial sums
   ProfScope prof(ctx, GRAM_K_ACCUMULATE, (in_bf16 ? 2.0 : 4.0) * (double)P * d + 4.0 * (double)U * d + 4.0 * P + 4.0 * (U + 1),
                  nchunks > 1 ? 2 : 1, st);
+  int32_t* sw = gram_status_word(ctx);
+  const int32_t* gate = gated ? sw : nullptr;
   if (d >= 256) {
-    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
-    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
+    if (in_bf16) segsum_run<bf16, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, sw, d_U, st, gate);
+    else segsum_run<float, 2>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, sw, d_U, st, gate);
   } else {
-    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
-    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, gram_status_word(ctx), d_U, st);
+    if (in_bf16) segsum_run<bf16, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, sw, d_U, st, gate);
+    else segsum_run<float, 1>(d_in, d_perm, d_seg_off, P, U, d, R, (int)nchunks, d_rows, add, d_out, ws->partial, span, sw, d_U, st, gate);
   }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items, uint32_t* d_bits,
-                                cudaStream_t st) {
-  if (U <= 0) return GRAM_OK;
+gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, const int32_t* d_U, int32_t n_items,
+                                uint32_t* d_bits, int32_t* d_count, int gated, cudaStream_t st) {
+  if (U <= 0 && !d_U) return GRAM_OK;
+  if (d_U) U = n_items;                              // upper bound for the launch shape
   ProfScope prof(ctx, GRAM_K_OTHER, 8.0 * U, 1, st);
-  touched_mark_kernel<<<ceil_div(U, 256), 256, 0, st>>>(d_unique, U, n_items, d_bits, gram_status_word(ctx));
+  int blocks = ceil_div(U, 256);
+  if (blocks > kNumSMs * 4) blocks = kNumSMs * 4;
+  touched_mark_kernel<<<blocks, 256, 0, st>>>(d_unique, U, d_U, n_items, d_bits, d_count, gram_status_word(ctx), gated);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -70,15 +70,22 @@ gram_status gather_launch(gram_ctx* ctx, const void* d_src, int64_t n_src_rows, 
 gram_status gather_diff_launch(gram_ctx* ctx, const float* d_a, const float* d_b, int64_t n_src_rows, const int32_t* d_index,
                                int64_t n, int32_t d, const float* d_x, float* d_out, cudaStream_t st);
 
+// d_E[p, :] (fp32) = d_src_bf16[d_index[p], :] (bf16 rows of d elements, d a multiple of 8): gather and widen in one pass
+gram_status gather_widen_launch(gram_ctx* ctx, const void* d_src_bf16, int64_t n_src_rows, const int32_t* d_index, int64_t P,
+                                int32_t d, float* d_E, cudaStream_t st);
+
 // in_bf16: rows of d_in are bf16 instead of fp32.  d_U (may be NULL): the number of segments is read
 // from the device instead of U.  d_rows (may be NULL): output row of segment u is d_rows[u] instead
-// of u.  add != 0: out[row] += sum instead of out[row] = sum.
+// of u.  add != 0: out[row] += sum instead of out[row] = sum.  gated != 0: the kernels leave d_out alone
+// when the context's status word already holds an error (a step that must not change state after a bad input).
 gram_status accumulate_launch(gram_ctx* ctx, IndexWorkspace* ws, const void* d_in, int in_bf16, const int32_t* d_perm,
                               const int32_t* d_seg_off, int64_t P, int32_t U, const int32_t* d_U, int32_t d,
-                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st);
+                              const int32_t* d_rows, int add, float* d_out, cudaStream_t st, int gated = 0);
 
-gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, int32_t n_items,
-                                uint32_t* d_bits, cudaStream_t st);
+// sets bit d_unique[u] for u < U (U read from d_U when that is not NULL); d_count (may be NULL) counts the bits that
+// were not set before; gated as above
+gram_status touched_mark_launch(gram_ctx* ctx, const int32_t* d_unique, int32_t U, const int32_t* d_U, int32_t n_items,
+                                uint32_t* d_bits, int32_t* d_count, int gated, cudaStream_t st);
 gram_status touched_list_launch(gram_ctx* ctx, const uint32_t* d_bits, int32_t n_items, int32_t* d_list,
                                 int32_t* d_count, cudaStream_t st);
 

@@ -591,24 +591,35 @@ __global__ void __launch_bounds__(128) pool_additive_bwd_kernel(StreamRef x, con
 }
 
 // ---------------------------------------------------------------------------- KT task input / head
-template <typename T>
-__global__ void kt_input_fwd_kernel(const float* __restrict__ E, const float* __restrict__ pos,
-                                    const float* __restrict__ resp, const int32_t* __restrict__ labels,
-                                    float* __restrict__ x, T* __restrict__ x_b, int64_t P, int L, int d) {
+// ET: element type of the encodings.  index (may be null): the encoding of position p is row index[p] of E (the gather
+// of stage 3 done where its result is consumed: E is then the matrix of encodings per item, n_rows of them).
+template <typename T, typename ET>
+__global__ void kt_input_fwd_kernel(const ET* __restrict__ E, const int32_t* __restrict__ index, int64_t n_rows,
+                                    const float* __restrict__ pos, const float* __restrict__ resp,
+                                    const int32_t* __restrict__ labels, float* __restrict__ x, T* __restrict__ x_b, int64_t P,
+                                    int L, int d, int32_t* status) {
   const int64_t p = blockIdx.x;                  // one block per position
   const int n = (int)(p % L);
   int prev = (n == 0) ? 2 : labels[p - 1];
   prev = prev < 0 ? 2 : (prev > 1 ? (n == 0 ? 2 : 1) : prev);      // after a padded position (label -1): only at padded rows
-  const float* e = E + p * d;
+  int64_t row = p;
+  if (index) {
+    row = index[p];
+    if (row < 0 || row >= n_rows) {
+      if (threadIdx.x == 0) gram_device_fail(status, GRAM_ERR_ID_RANGE);
+      row = 0;
+    }
+  }
+  const ET* e = E + row * d;
   const float* pe = pos + (int64_t)n * d;
   const float* re = resp + (int64_t)prev * d;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float v = e[c] + pe[c] + re[c];
+    const float v = ldf(e + c) + pe[c] + re[c];
     x[p * d + c] = v;
     stf(x_b + p * d + c, v);
   }
 }
-// one thread per column: dE = dx; dpos[n, c] += sum_b; dresp[r, c] += sum over positions with prev == r
+// one thread per column: dE = dx (when dE is not null); dpos[n, c] += sum_b; dresp[r, c] += sum over positions with prev == r
 __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t* __restrict__ labels, float* __restrict__ dE,
                                     float* __restrict__ dpos, float* __restrict__ dresp, int B, int L, int d) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -629,7 +640,7 @@ __global__ void kt_input_bwd_kernel(const float* __restrict__ dx, const int32_t*
 #pragma unroll
     for (int k = 0; k < UB; ++k) {              // sums in ascending history order
       if (b0 + k < B) {
-        dE[((int64_t)(b0 + k) * L + n) * d + c] = v[k];
+        if (dE) dE[((int64_t)(b0 + k) * L + n) * d + c] = v[k];
         ap += v[k];
         if (prev[k] == 0) r0 += v[k]; else if (prev[k] == 1) r1 += v[k]; else r2 += v[k];
       }
@@ -851,7 +862,9 @@ __global__ void bf16_to_f32_kernel(const bf16* __restrict__ in, float* __restric
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     out[i] = __bfloat162float(in[i]);
 }
-__global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float lr, size_t n) {
+// gate (may be null): a device word; nothing is updated when it is not zero (an error met earlier in the step)
+__global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float lr, size_t n, const int32_t* __restrict__ gate) {
+  if (gate && *gate) return;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     w[i] -= lr * g[i];
 }
@@ -1185,12 +1198,19 @@ gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, i
   return GRAM_OK;
 }
 
-gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const float* pos, const float* resp,
-                             const int32_t* labels, float* x, void* x_b, int B, int L, int d, cudaStream_t st) {
+gram_status kt_input_forward(gram_ctx* ctx, int dtype, const void* E, int e_bf16, const int32_t* index, int64_t n_rows,
+                             const float* pos, const float* resp, const int32_t* labels, float* x, void* x_b, int B, int L,
+                             int d, cudaStream_t st) {
   const int64_t P = (int64_t)B * L;
   if (P == 0) return GRAM_OK;
-  ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)P * d * (8.0 + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
-  DISPATCH_T(dtype, kt_input_fwd_kernel<T><<<(unsigned)P, d >= 256 ? 256 : 64, 0, st>>>(E, pos, resp, labels, x, (T*)x_b, P, L, d));
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)P * d * ((e_bf16 ? 6.0 : 8.0) + (dtype == GRAM_BF16 ? 2.0 : 4.0)), 1, st);
+  const int threads = d >= 256 ? 256 : 64;
+  int32_t* sw = gram_status_word(ctx);
+  if (e_bf16) {
+    DISPATCH_T(dtype, kt_input_fwd_kernel<T, bf16><<<(unsigned)P, threads, 0, st>>>((const bf16*)E, index, n_rows, pos, resp, labels, x, (T*)x_b, P, L, d, sw));
+  } else {
+    DISPATCH_T(dtype, kt_input_fwd_kernel<T, float><<<(unsigned)P, threads, 0, st>>>((const float*)E, index, n_rows, pos, resp, labels, x, (T*)x_b, P, L, d, sw));
+  }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -1263,7 +1283,9 @@ gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out,
 template <bool WB>
 __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m,
                                                    float* __restrict__ v, bf16* __restrict__ wb, size_t n, float rate,
-                                                   float beta1, float beta2, float eps, float c1, float c2) {
+                                                   float beta1, float beta2, float eps, float c1, float c2,
+                                                   const int32_t* __restrict__ gate) {
+  if (gate && *gate) return;                    // an error met earlier in the step: no update
   const size_t n4 = n >> 2;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
@@ -1300,7 +1322,7 @@ __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ w, const 
 }
 
 gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float* v, void* wb, size_t n, int64_t t, float rate,
-                        float beta1, float beta2, float eps, cudaStream_t st) {
+                        float beta1, float beta2, float eps, cudaStream_t st, const int32_t* gate) {
   if (n == 0) return GRAM_OK;
   if (t < 1) return gram_set_error(ctx, "Adam: the update count starts at 1"), GRAM_ERR_ARG;
   if (((uintptr_t)w | (uintptr_t)g | (uintptr_t)m | (uintptr_t)v) % 16 || (wb && (uintptr_t)wb % 8))
@@ -1309,16 +1331,16 @@ gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float
   const float c2 = (float)(1.0 / (1.0 - pow((double)beta2, (double)t)));
   ProfScope prof(ctx, GRAM_K_OPTIMIZER, (double)n * (28.0 + (wb ? 2.0 : 0.0)), 1, st, "adam");
   const int grid = grid_for((int64_t)((n + 3) / 4), 256, kNumSMs * 8);
-  if (wb) adam_kernel<true><<<grid, 256, 0, st>>>(w, g, m, v, (bf16*)wb, n, rate, beta1, beta2, eps, c1, c2);
-  else adam_kernel<false><<<grid, 256, 0, st>>>(w, g, m, v, nullptr, n, rate, beta1, beta2, eps, c1, c2);
+  if (wb) adam_kernel<true><<<grid, 256, 0, st>>>(w, g, m, v, (bf16*)wb, n, rate, beta1, beta2, eps, c1, c2, gate);
+  else adam_kernel<false><<<grid, 256, 0, st>>>(w, g, m, v, nullptr, n, rate, beta1, beta2, eps, c1, c2, gate);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
 
-gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st) {
+gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st, const int32_t* gate) {
   if (n == 0 || lr == 0.f) return GRAM_OK;
   ProfScope prof(ctx, GRAM_K_OPTIMIZER, 12.0 * (double)n, 1, st, "sgd");
-  sgd_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(w, g, lr, n);
+  sgd_kernel<<<grid_for((int64_t)n, 256, kNumSMs * 16), 256, 0, st>>>(w, g, lr, n, gate);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -94,11 +94,15 @@ gram_status pool_forward(gram_ctx* ctx, const StreamRef& x, float* H, int64_t n,
 gram_status pool_backward(gram_ctx* ctx, const float* G, float* dx, int64_t n, int l_t, int d, int pooling,
                           const int32_t* seq_len, const int32_t* seq_off, cudaStream_t st);
 
-// knowledge-tracing task input: x[b, n, :] = E[b, n, :] + pos[n, :] + resp[prev(b, n), :] (fp32, and an
-// operand-typed copy x_b), prev(b, 0) = 2, prev(b, n) = labels[b, n-1]
-gram_status kt_input_forward(gram_ctx* ctx, int dtype, const float* E, const float* pos, const float* resp,
-                             const int32_t* labels, float* x, void* x_b, int B, int L, int d, cudaStream_t st);
-// dE = dx; dpos[n] += sum_b dx[b, n]; dresp[r] += sum over positions with prev == r
+// knowledge-tracing task input: x[b, n, :] = e(b, n) + pos[n, :] + resp[prev(b, n), :] (fp32, and an
+// operand-typed copy x_b), prev(b, 0) = 2, prev(b, n) = labels[b, n-1].  e(b, n) = E[b*L + n, :] when index is null,
+// else E[index[b*L + n], :] with E holding n_rows rows (the gather of stage 3 fused into this load); e_bf16: E's rows
+// are bf16 (the Multi-step encoding cache) instead of fp32.
+gram_status kt_input_forward(gram_ctx* ctx, int dtype, const void* E, int e_bf16, const int32_t* index, int64_t n_rows,
+                             const float* pos, const float* resp, const int32_t* labels, float* x, void* x_b, int B, int L,
+                             int d, cudaStream_t st);
+// dE = dx (skipped when dE is null: the caller then reads dx itself as the gradient with respect to the encodings);
+// dpos[n] += sum_b dx[b, n]; dresp[r] += sum over positions with prev == r
 gram_status kt_input_backward(gram_ctx* ctx, const float* dx, const int32_t* labels, float* dE, float* dpos,
                               float* dresp, float* scratch, int B, int L, int d, cudaStream_t st);
 // logit = y . w + b; loss = mean BCE over the positions with a label >= 0 (label -1: padding at the end of a history,
@@ -120,10 +124,11 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
 // element-wise helpers
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st);
 gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st);
-gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st);
+// gate (may be null): a device word; the update is skipped when it is not zero
+gram_status sgd_update(gram_ctx* ctx, float* w, const float* g, float lr, size_t n, cudaStream_t st, const int32_t* gate = nullptr);
 // one Adam update at count t >= 1 (Kingma & Ba, Algorithm 1); wb (may be null): bf16 copy of the new parameters
 gram_status adam_update(gram_ctx* ctx, float* w, const float* g, float* m, float* v, void* wb, size_t n, int64_t t, float rate,
-                        float beta1, float beta2, float eps, cudaStream_t st);
+                        float beta1, float beta2, float eps, cudaStream_t st, const int32_t* gate = nullptr);
 // dst[index[u], :] = src[u, :] (src fp32, dst operand-typed)
 gram_status scatter_rows(gram_ctx* ctx, int dtype, const float* src, const int32_t* index, int64_t n, int d,
                          int64_t n_dst_rows, void* dst, cudaStream_t st);

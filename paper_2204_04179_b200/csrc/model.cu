@@ -144,7 +144,7 @@ struct Model {
   int32_t* h_pinned = nullptr;       // [16] pinned host words for small read-backs
 };
 
-// the Noam curve scaled to peak at update `warmup` (Section A; Vaswani et al. 2017, Eq. 3)
+// the Noam curve scaled to peak at update `warmup` (Appendix D; Vaswani et al. 2017, Eq. 3)
 double noam_rate(int64_t t, double peak, int warmup) {
   if (warmup <= 0) return peak;
   const double x = (double)t, w = (double)warmup;
@@ -607,17 +607,30 @@ gram_status encoder_backward_chunk(Model* m, const float* G, int32_t n, cudaStre
   return GRAM_OK;
 }
 
-// E: fp32 [B, L, d]
-gram_status task_forward_backward(Model* m, const float* E, const int32_t* labels, int32_t B, float* dE, float* loss,
-                                  cudaStream_t st) {
+// Where the task module finds the encoding of position p: row p of `rows` (index == null, rows is fp32 [B*L, d]), or
+// row index[p] of `rows` (n_rows rows of fp32, or of bf16 when rows_bf16: the Multi-step cache), i.e. stage 3 left to
+// the task module's first load.
+struct EncodingSource {
+  const void* rows = nullptr;
+  int rows_bf16 = 0;
+  const int32_t* index = nullptr;
+  int64_t n_rows = 0;
+};
+
+// Task module forward and backward.  dE (may be null for the KT task): receives dL/dE, fp32 [B*L, d].  *dE_at is set to
+// where dL/dE can be read after the call: dE when given, else the task module's own input-gradient buffer (the KT input
+// is a sum, so its gradient is the gradient of the encodings, row for row).
+gram_status task_forward_backward(Model* m, const EncodingSource& src, const int32_t* labels, int32_t B, float* dE, float* loss,
+                                  const float** dE_at, cudaStream_t st) {
   const gram_config& c = m->cfg;
   gram_ctx* ctx = m->ctx;
   const int64_t P = (int64_t)B * c.L;
   GRAM_TRY(refresh_bf16(m, m->task, st));
   GRAM_CUDA(ctx, cudaMemsetAsync(m->task.g, 0, m->task.n * 4, st));
+  if (dE_at) *dE_at = dE;
   if (c.task == GRAM_TASK_KT) {
-    GRAM_TRY(kt_input_forward(ctx, m->dtype, E, m->task.w + m->t_pos, m->task.w + m->t_resp, labels, m->tx, m->txb, B, c.L,
-                              c.d, st));
+    GRAM_TRY(kt_input_forward(ctx, m->dtype, src.rows, src.rows_bf16, src.index, src.n_rows, m->task.w + m->t_pos,
+                              m->task.w + m->t_resp, labels, m->tx, m->txb, B, c.L, c.d, st));
     StreamRef x;
     x.z = m->tx;
     StreamRef y;
@@ -629,9 +642,12 @@ gram_status task_forward_backward(Model* m, const float* E, const int32_t* label
     float* dx = nullptr;
     GRAM_TRY(stack_backward(m, m->task, m->tk, m->txb, B, c.L, st, &dx));
     GRAM_TRY(kt_input_backward(ctx, dx, labels, dE, m->task.g + m->t_pos, m->task.g + m->t_resp, m->red, B, c.L, c.d, st));
+    if (!dE && dE_at) *dE_at = dx;
     return GRAM_OK;
   }
   if (c.task == GRAM_TASK_NR) {
+    if (src.index || src.rows_bf16 || !dE) return gram_set_error(ctx, "the news task reads materialised fp32 encodings"), GRAM_ERR_ARG;
+    const float* E = (const float*)src.rows;
     const void* Eb = E;                  // fp32 contexts: the stream is its own operand
     if (m->dtype == GRAM_BF16) {
       GRAM_TRY(convert_f32_to_bf16(ctx, E, (bf16*)m->Eb, (size_t)P * c.d, st));
@@ -660,8 +676,11 @@ gram_status read_i32(Model* m, const int32_t* d_ptr, int32_t* out, cudaStream_t 
 }
 
 // the configured update of one module from its gradients: lr is the SGD step or Adam's peak rate
-gram_status apply_sgd(Model* m, Module& mod, float lr, cudaStream_t st) {
+// gated: the kernel leaves the parameters alone when the context's status word holds an error (the caller then takes
+// the update count back)
+gram_status apply_sgd(Model* m, Module& mod, float lr, cudaStream_t st, bool gated = false) {
   if (lr == 0.f || mod.n == 0) return GRAM_OK;
+  const int32_t* gate = gated ? gram_status_word(m->ctx) : nullptr;
   const gram_config& c = m->cfg;
   ++mod.updates;
   if (c.optimizer == GRAM_OPT_ADAM) {
@@ -669,11 +688,11 @@ gram_status apply_sgd(Model* m, Module& mod, float lr, cudaStream_t st) {
     const float eps = c.adam_eps > 0.f ? c.adam_eps : 1e-8f;
     const float rate = (float)noam_rate(mod.updates, lr, c.noam_warmup);
     GRAM_TRY(adam_update(m->ctx, mod.w, mod.g, mod.am, mod.av, m->dtype == GRAM_BF16 ? mod.wb : nullptr, mod.n, mod.updates, rate,
-                         b1, b2, eps, st));
+                         b1, b2, eps, st, gate));
     mod.wb_stale = false;                       // the kernel wrote the bf16 copy as well
     return GRAM_OK;
   }
-  GRAM_TRY(sgd_update(m->ctx, mod.w, mod.g, lr, mod.n, st));
+  GRAM_TRY(sgd_update(m->ctx, mod.w, mod.g, lr, mod.n, st, gate));
   mod.wb_stale = true;
   return GRAM_OK;
 }
@@ -733,6 +752,8 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   if (c.adam_beta1 >= 1.f || c.adam_beta2 >= 1.f) return gram_set_error(ctx, "Adam: beta1 and beta2 must be below 1"), GRAM_ERR_ARG;
   if (c.multistep_variant != GRAM_MULTI_TABLE && c.multistep_variant != GRAM_MULTI_PSEUDO_TARGET)
     return gram_set_error(ctx, "unknown multistep_variant %d", c.multistep_variant), GRAM_ERR_ARG;
+  if (c.defer_update && c.refresh_after_update)
+    return gram_set_error(ctx, "defer_update cannot be combined with refresh_after_update"), GRAM_ERR_UNSUPPORTED;
   m->pseudo = c.K > 1 && c.multistep_variant == GRAM_MULTI_PSEUDO_TARGET;
   m->cache_dtype = m->pseudo ? GRAM_F32 : c.dtype;
   // ---- parameter layouts (the order include/gram.h documents) ----
@@ -850,6 +871,14 @@ gram_status model_zero_grads(Model* m, int module, cudaStream_t st) {
   return GRAM_OK;
 }
 
+gram_status model_grads_device(Model* m, int module, float** d_grads, size_t* n) {
+  Module* mod = pick(m, module);
+  if (!mod) return gram_set_error(m->ctx, "unknown module %d", module), GRAM_ERR_ARG;
+  *d_grads = mod->g;
+  *n = mod->n;
+  return GRAM_OK;
+}
+
 gram_status model_set_item_tokens(Model* m, const int32_t* h_tokens) {
   if (!h_tokens || !m->item_tokens) return gram_set_error(m->ctx, "gram_set_item_tokens: no encoder or null tokens"), GRAM_ERR_ARG;
   GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
@@ -892,7 +921,9 @@ gram_status model_task(Model* m, const float* d_E, const int32_t* d_labels, int3
   if (B < 0 || B > m->cfg.B_max) return gram_set_error(m->ctx, "gram_task: B=%d exceeds B_max=%d", B, m->cfg.B_max), GRAM_ERR_WORKSPACE;
   if (B == 0) return GRAM_OK;
   if (!d_E || !d_labels || !d_dE || !d_loss) return gram_set_error(m->ctx, "gram_task: null buffer"), GRAM_ERR_ARG;
-  return task_forward_backward(m, d_E, d_labels, B, d_dE, d_loss, st);
+  EncodingSource src;
+  src.rows = d_E;
+  return task_forward_backward(m, src, d_labels, B, d_dE, d_loss, nullptr, st);
 }
 
 gram_status model_encoder_backward(Model* m, const float* d_G, const int32_t* d_items, int32_t U, cudaStream_t st) {
@@ -910,6 +941,7 @@ gram_status model_window_reset(Model* m, cudaStream_t st) {
   if (!m->table) return gram_set_error(m->ctx, "the context was created with K <= 1"), GRAM_ERR_ARG;
   GRAM_CUDA(m->ctx, cudaMemsetAsync(m->table, 0, (size_t)m->cfg.n_items * m->cfg.d * 4, st));
   GRAM_CUDA(m->ctx, cudaMemsetAsync(m->touched, 0, (size_t)((m->cfg.n_items + 31) / 32) * 4, st));
+  GRAM_CUDA(m->ctx, cudaMemsetAsync(m->tcount, 0, sizeof(int32_t), st));
   m->step_in_window = 0;
   return GRAM_OK;
 }
@@ -958,7 +990,11 @@ gram_status model_state_import(Model* m, const float* h_table, const uint32_t* h
   if (steps < 0 || steps >= c.K) return gram_set_error(m->ctx, "gram_state_import: %d steps in a window of %d", steps, c.K), GRAM_ERR_ARG;
   GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
   if (h_table) GRAM_CUDA(m->ctx, cudaMemcpy(m->table, h_table, (size_t)c.n_items * c.d * 4, cudaMemcpyHostToDevice));
-  if (h_touched) GRAM_CUDA(m->ctx, cudaMemcpy(m->touched, h_touched, (size_t)((c.n_items + 31) / 32) * 4, cudaMemcpyHostToDevice));
+  if (h_touched) {
+    GRAM_CUDA(m->ctx, cudaMemcpy(m->touched, h_touched, (size_t)((c.n_items + 31) / 32) * 4, cudaMemcpyHostToDevice));
+    GRAM_TRY(touched_list_launch(m->ctx, m->touched, c.n_items, m->tlist, m->tcount, 0));     // recount the set bits
+    GRAM_CUDA(m->ctx, cudaDeviceSynchronize());
+  }
   if (h_cache) {
     if (m->cache_dtype == GRAM_F32) {
       GRAM_CUDA(m->ctx, cudaMemcpy(m->cache, h_cache, (size_t)c.n_items * c.d * 4, cudaMemcpyHostToDevice));
@@ -1002,6 +1038,29 @@ gram_status model_optimizer_import(Model* m, int module, const float* h_m, const
   return GRAM_OK;
 }
 
+// reads a few device words with one wait: out[k] = *d_ptr[k]
+static gram_status read_words(Model* m, const int32_t* const* d_ptr, int n, int32_t* out, cudaStream_t st) {
+  for (int k = 0; k < n; ++k)
+    GRAM_CUDA(m->ctx, cudaMemcpyAsync(m->h_pinned + k, d_ptr[k], 4, cudaMemcpyDeviceToHost, st));
+  GRAM_CUDA(m->ctx, cudaStreamSynchronize(st));
+  for (int k = 0; k < n; ++k) out[k] = m->h_pinned[k];
+  return GRAM_OK;
+}
+
+// an error word read back from the device: clears it and names it
+static gram_status device_error(Model* m, int32_t code, cudaStream_t st) {
+  GRAM_CUDA(m->ctx, cudaMemsetAsync(gram_status_word(m->ctx), 0, sizeof(int32_t), st));
+  GRAM_CUDA(m->ctx, cudaStreamSynchronize(st));
+  gram_set_error(m->ctx, code == GRAM_ERR_ID_RANGE ? "gram_step: an ID outside its range was met on the device; the step changed no state"
+                                                   : (code == GRAM_ERR_TIMEOUT ? "gram_step: a bounded device-side wait ran out" : "gram_step: device-side error"));
+  return (gram_status)code;
+}
+
+// Host synchronisation points: Single-step waits once after the dedup (it needs U to size the encoder pass, and reads the
+// status word in the same wait, so a batch with an ID out of range is rejected before anything else runs) and once at the
+// end.  A Multi-step step without encoder pass waits once, at the end: U stays on the device, and every kernel that
+// changes state that outlives the step (table, touched bits, task parameters) is gated on the status word, so a rejected
+// batch still changes nothing.  The K-th step of a window waits once more to read the number of touched items.
 gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in, int32_t B, int on_host,
                        gram_step_report* rep, cudaStream_t st) {
   const gram_config& c = m->cfg;
@@ -1011,7 +1070,9 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
   if (!ids_in || !labels_in) return gram_set_error(ctx, "gram_step: null buffer"), GRAM_ERR_ARG;
   const int64_t P = (int64_t)B * c.L;
   const bool multi = c.K > 1;
+  const bool kt = c.task == GRAM_TASK_KT;
   cudaEvent_t* ev = m->ev;
+  int32_t* status = gram_status_word(ctx);
   GRAM_CUDA(ctx, cudaEventRecord(ev[0], st));
   const int32_t* ids = ids_in;
   const int32_t* labels = labels_in;
@@ -1024,45 +1085,38 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
   // stage 1
   IndexWorkspace* iws = gram_index_ws(ctx);
   GRAM_TRY(dedup_launch(ctx, iws, ids, P, c.n_items, m->unique, m->inverse, m->perm, m->seg_off, m->n_unique, st));
-  int32_t U = 0;
-  GRAM_TRY(read_i32(m, m->n_unique, &U, st));
-  if (U <= 0 || U > m->u_cap) return gram_set_error(ctx, "gram_step: dedup returned U=%d", U), GRAM_ERR_ID_RANGE;
-  GRAM_CUDA(ctx, cudaEventRecord(ev[1], st));
-  int32_t n_encoded = 0, n_touched = U, encoder_ran = 0;
+  int32_t U = 0, n_encoded = 0, n_touched = 0, encoder_ran = 0;
+  const float* dE_at = nullptr;
   if (!multi) {
+    const int32_t* words[2] = {m->n_unique, status};
+    int32_t got[2] = {0, 0};
+    GRAM_TRY(read_words(m, words, 2, got, st));
+    if (got[1] != 0) return device_error(m, got[1], st);
+    U = got[0];
+    if (U <= 0 || U > m->u_cap) return gram_set_error(ctx, "gram_step: dedup returned U=%d", U), GRAM_ERR_ID_RANGE;
+    GRAM_CUDA(ctx, cudaEventRecord(ev[1], st));
     // stage 2: one encoding per unique item (Eq. 4)
     for (int32_t u0 = 0; u0 < U; u0 += m->mb) {
       const int32_t n = (U - u0 < m->mb) ? U - u0 : m->mb;
       GRAM_TRY(encoder_forward_chunk(m, nullptr, m->unique + u0, 0, n, m->H + (size_t)u0 * c.d, st));
     }
     GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
-    // stage 3
-    GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, 4, m->E, st));
-  } else {
-    GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
-    if (m->pseudo) {                   // the pseudo-targets h~ = cache - table of the items at every position (Eq. 6)
-      GRAM_TRY(gather_diff_launch(ctx, (const float*)m->cache, m->table, c.n_items, ids, P, c.d, nullptr, m->E, st));
-    } else if (m->cache_dtype == GRAM_BF16) {       // rows of the bf16 cache, widened for the task module
-      GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 2, m->Eb, st));
-      GRAM_TRY(convert_to_f32(ctx, GRAM_BF16, m->Eb, m->E, (size_t)P * c.d, st));
+    // stage 3: the KT task module gathers H[inverse[p]] in its first load; the NR module reads a materialised E
+    EncodingSource src;
+    if (kt) {
+      src.rows = m->H; src.index = m->inverse; src.n_rows = U;
     } else {
-      GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 4, m->E, st));
+      GRAM_TRY(gather_launch(ctx, m->H, U, m->inverse, P, c.d, 4, m->E, st));
+      src.rows = m->E;
     }
-  }
-  GRAM_CUDA(ctx, cudaEventRecord(ev[3], st));
-  // task module forward / backward (Eq. 5) and dL/dE
-  GRAM_TRY(task_forward_backward(m, m->E, labels, B, m->dE, m->loss, st));
-  GRAM_CUDA(ctx, cudaEventRecord(ev[4], st));
-  // stage 4 (Eq. 6)
-  if (!multi) {
-    GRAM_TRY(accumulate_launch(ctx, iws, m->dE, 0, m->perm, m->seg_off, P, U, nullptr, c.d, nullptr, 0, m->G, st));
-  } else {
-    GRAM_TRY(accumulate_launch(ctx, iws, m->dE, 0, m->perm, m->seg_off, P, U, nullptr, c.d, m->unique, 1, m->table, st));
-    GRAM_TRY(touched_mark_launch(ctx, m->unique, U, c.n_items, m->touched, st));
-  }
-  GRAM_CUDA(ctx, cudaEventRecord(ev[5], st));
-  // stage 5 (Eq. 7)
-  if (!multi) {
+    GRAM_CUDA(ctx, cudaEventRecord(ev[3], st));
+    // task module forward / backward (Eq. 5) and dL/dE
+    GRAM_TRY(task_forward_backward(m, src, labels, B, kt ? nullptr : m->dE, m->loss, &dE_at, st));
+    GRAM_CUDA(ctx, cudaEventRecord(ev[4], st));
+    // stage 4 (Eq. 6)
+    GRAM_TRY(accumulate_launch(ctx, iws, dE_at, 0, m->perm, m->seg_off, P, U, nullptr, c.d, nullptr, 0, m->G, st));
+    GRAM_CUDA(ctx, cudaEventRecord(ev[5], st));
+    // stage 5 (Eq. 7)
     GRAM_CUDA(ctx, cudaMemsetAsync(m->ce.g, 0, m->ce.n * 4, st));
     if (U <= m->mb) {
       GRAM_TRY(encoder_backward_chunk(m, m->G, U, st));
@@ -1073,15 +1127,51 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
                             [&](int32_t u0, int32_t, const float** G) { *G = Gbase + (size_t)u0 * c.d; return GRAM_OK; }, st));
     }
     n_encoded = U;
+    n_touched = U;
     encoder_ran = 1;
-    GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st));
-    GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+    if (!c.defer_update) {
+      GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st));
+      GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+    }
   } else {
-    GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st));
-    ++m->step_in_window;
-    GRAM_TRY(touched_list_launch(ctx, m->touched, c.n_items, m->tlist, m->tcount, st));
-    GRAM_TRY(read_i32(m, m->tcount, &n_touched, st));
-    if (m->step_in_window >= c.K) {
+    GRAM_CUDA(ctx, cudaEventRecord(ev[1], st));
+    GRAM_CUDA(ctx, cudaEventRecord(ev[2], st));
+    // stage 3 from the cache (Section 4.2): fused into the KT module's first load, materialised otherwise
+    EncodingSource src;
+    if (m->pseudo) {                   // the pseudo-targets h~ = cache - table of the items at every position (Eq. 6)
+      GRAM_TRY(gather_diff_launch(ctx, (const float*)m->cache, m->table, c.n_items, ids, P, c.d, nullptr, m->E, st));
+      src.rows = m->E;
+    } else if (kt) {
+      src.rows = m->cache; src.rows_bf16 = m->cache_dtype == GRAM_BF16; src.index = ids; src.n_rows = c.n_items;
+    } else if (m->cache_dtype == GRAM_BF16) {       // rows of the bf16 cache, widened on the way
+      GRAM_TRY(gather_widen_launch(ctx, m->cache, c.n_items, ids, P, c.d, m->E, st));
+      src.rows = m->E;
+    } else {
+      GRAM_TRY(gather_launch(ctx, m->cache, c.n_items, ids, P, c.d, 4, m->E, st));
+      src.rows = m->E;
+    }
+    GRAM_CUDA(ctx, cudaEventRecord(ev[3], st));
+    GRAM_TRY(task_forward_backward(m, src, labels, B, kt ? nullptr : m->dE, m->loss, &dE_at, st));
+    GRAM_CUDA(ctx, cudaEventRecord(ev[4], st));
+    // stage 4 (Eq. 6) into the table; U is read on the device
+    GRAM_TRY(accumulate_launch(ctx, iws, dE_at, 0, m->perm, m->seg_off, P, 0, m->n_unique, c.d, m->unique, 1, m->table, st, 1));
+    GRAM_TRY(touched_mark_launch(ctx, m->unique, 0, m->n_unique, c.n_items, m->touched, m->tcount, 1, st));
+    GRAM_CUDA(ctx, cudaEventRecord(ev[5], st));
+    const int64_t task_updates = m->task.updates;
+    if (!c.defer_update) GRAM_TRY(apply_sgd(m, m->task, c.lr_task, st, true));
+    if (m->step_in_window + 1 >= c.K) {
+      // last step of the window: the list of touched items and its length are needed on the host now
+      GRAM_TRY(touched_list_launch(ctx, m->touched, c.n_items, m->tlist, m->tcount, st));
+      const int32_t* words[3] = {m->tcount, m->n_unique, status};
+      int32_t got[3] = {0, 0, 0};
+      GRAM_TRY(read_words(m, words, 3, got, st));
+      if (got[2] != 0) {
+        m->task.updates = task_updates;
+        m->task.wb_stale = true;
+        return device_error(m, got[2], st);
+      }
+      n_touched = got[0];
+      U = got[1];
       GRAM_CUDA(ctx, cudaMemsetAsync(m->ce.g, 0, m->ce.n * 4, st));
       GRAM_TRY(encoder_pass(m, m->tlist, n_touched, true,
                             [&](int32_t u0, int32_t n, const float** G) {
@@ -1091,7 +1181,7 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
                                                           m->H, m->G, st);
                               return gather_launch(ctx, m->table, c.n_items, m->tlist + u0, n, c.d, 4, m->G, st);
                             }, st));
-      GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
+      if (!c.defer_update) GRAM_TRY(apply_sgd(m, m->ce, c.lr_ce, st));
       if (c.refresh_after_update) {      // Eq. 4 with the updated parameters: the next window reads fresh encodings
         for (int32_t u0 = 0; u0 < n_touched; u0 += m->mb) {
           const int32_t n = (n_touched - u0 < m->mb) ? n_touched - u0 : m->mb;
@@ -1103,17 +1193,36 @@ gram_status model_step(Model* m, const int32_t* ids_in, const int32_t* labels_in
       GRAM_TRY(model_window_reset(m, st));
       n_encoded = n_touched;
       encoder_ran = 1;
+      GRAM_CUDA(ctx, cudaEventRecord(ev[6], st));
+      GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 12, m->loss, 4, cudaMemcpyDeviceToHost, st));
+      GRAM_CUDA(ctx, cudaStreamSynchronize(st));
+    } else {
+      GRAM_CUDA(ctx, cudaEventRecord(ev[6], st));
+      GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 12, m->loss, 4, cudaMemcpyDeviceToHost, st));
+      const int32_t* words[3] = {m->tcount, m->n_unique, status};
+      int32_t got[3] = {0, 0, 0};
+      GRAM_TRY(read_words(m, words, 3, got, st));           // the step's only wait
+      if (got[2] != 0) {
+        m->task.updates = task_updates;
+        m->task.wb_stale = true;
+        return device_error(m, got[2], st);
+      }
+      n_touched = got[0];
+      U = got[1];
+      ++m->step_in_window;
     }
   }
-  GRAM_CUDA(ctx, cudaEventRecord(ev[6], st));
-  GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 1, m->loss, 4, cudaMemcpyDeviceToHost, st));
-  GRAM_CUDA(ctx, cudaStreamSynchronize(st));
+  if (!multi) {
+    GRAM_CUDA(ctx, cudaEventRecord(ev[6], st));
+    GRAM_CUDA(ctx, cudaMemcpyAsync(m->h_pinned + 12, m->loss, 4, cudaMemcpyDeviceToHost, st));
+    GRAM_CUDA(ctx, cudaStreamSynchronize(st));
+  }
   if (rep) {
     memset(rep, 0, sizeof(*rep));
-    memcpy(&rep->loss, m->h_pinned + 1, 4);
+    memcpy(&rep->loss, m->h_pinned + 12, 4);
     rep->n_positions = (int32_t)P;
     rep->n_unique = U;
-    rep->boost_ratio = (float)P / (float)U;
+    rep->boost_ratio = U > 0 ? (float)P / (float)U : 0.f;
     rep->n_touched = n_touched;
     rep->encoder_pass = encoder_ran;
     rep->n_encoded = n_encoded;

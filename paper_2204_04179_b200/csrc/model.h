@@ -13,6 +13,7 @@ gram_status model_param_count(const Model* m, int module, size_t* n);
 gram_status model_set_params(Model* m, int module, const float* h, size_t n);
 gram_status model_get_params(Model* m, int module, float* h, size_t n, int grads);
 gram_status model_zero_grads(Model* m, int module, cudaStream_t st);
+gram_status model_grads_device(Model* m, int module, float** d_grads, size_t* n);
 gram_status model_optimizer_step(Model* m, int module, cudaStream_t st);
 gram_status model_optimizer_reset(Model* m, cudaStream_t st);
 double noam_rate(int64_t t, double peak, int warmup);

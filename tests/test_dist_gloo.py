@@ -29,6 +29,23 @@ out = dict(rank=rank, rows=int(my_ids.shape[0]), U=U, ids=my_ids.tolist(),
            ms_max=gdist.max_over_ranks(ms, dist), total=gdist.sum_over_ranks(my_ids.size, dist),
            thr=gdist.job_throughput(my_ids.size, ms, dist),
            seed=gdist.rank_seed(3, rank))
+# data-parallel gradients: every rank differentiates the loss of ITS histories (a mean over its own predictions);
+# after the weighted all-reduce both hold the gradient of the whole batch
+import torch
+shape2 = synth.GramShape(name="s", n_items=9, l_t=4, vocab=20, d=16, n_heads=2, d_ff=32, n_layers=1, pooling="cls", task="kt",
+                         task_layers=1, task_heads=2, task_d_ff=32, task_attn_only=False, B=5, L=6, zipf_s=1.1)
+ce = synth.encoder_params(shape2, 3, sigma=0.3, plain=False); tk = synth.task_params(shape2, 3, sigma=0.3, plain=False)
+toks = synth.item_tokens(3, shape2.n_items, shape2.l_t, shape2.vocab)
+ids2, lab2 = synth.batch(shape2, 3)
+lab2 = lab2.copy(); lab2[4, 3:] = -1                  # the last history ends in padding: 3 predictions instead of 6
+s_ids, s_lab = gdist.shard_batch(ids2, lab2, rank, 2) # 3 histories on rank 0 (18 predictions), 2 on rank 1 (9 predictions)
+r = orc.e2e_step(shape2.replace(B=s_ids.shape[0]), ce, tk, toks, s_ids, s_lab)
+grads = [torch.tensor(v) for v in list(r["grad_ce"].values()) + list(r["grad_task"].values())]
+n_pred = gdist.n_predictions(shape2, s_lab)
+total = gdist.allreduce_weighted_mean(grads, n_pred, dist)
+names = list(r["grad_ce"]) + list(r["grad_task"])
+out["n_pred"] = n_pred; out["total_pred"] = total
+out["grads"] = {n: t.numpy().tolist() for n, t in zip(names, grads) if n in ("l0.w1", "head_w", "pos", "tok_emb")}
 print("RESULT " + json.dumps(out), flush=True)
 dist.barrier()
 dist.destroy_process_group()
@@ -73,3 +90,22 @@ def test_two_ranks_over_gloo():
         assert abs(res[r]["thr"] - 30.0 / 0.015) < 1e-9
     assert res[0]["seed"] != res[1]["seed"]
     assert res[0]["U"] == len(np.unique(ids[:3])) and res[1]["U"] == len(np.unique(ids[3:]))
+    # the averaged gradients equal end-to-end training on the whole batch (Eq. 8's mean runs over all predictions)
+    from oracle import gram_oracle as orc
+    shape2 = synth.GramShape(name="s", n_items=9, l_t=4, vocab=20, d=16, n_heads=2, d_ff=32, n_layers=1, pooling="cls", task="kt",
+                             task_layers=1, task_heads=2, task_d_ff=32, task_attn_only=False, B=5, L=6, zipf_s=1.1)
+    ce = synth.encoder_params(shape2, 3, sigma=0.3, plain=False); tk = synth.task_params(shape2, 3, sigma=0.3, plain=False)
+    toks = synth.item_tokens(3, shape2.n_items, shape2.l_t, shape2.vocab)
+    ids2, lab2 = synth.batch(shape2, 3)
+    lab2 = lab2.copy(); lab2[4, 3:] = -1
+    whole = orc.e2e_step(shape2, ce, tk, toks, ids2, lab2)
+    assert (res[0]["n_pred"], res[1]["n_pred"]) == (18, 9) and res[0]["total_pred"] == 27.0
+    for r in (0, 1):
+        for name, got in res[r]["grads"].items():
+            want = whole["grad_ce"][name] if name in whole["grad_ce"] else whole["grad_task"][name]
+            assert np.abs(np.array(got) - want).max() <= 1e-12 * max(1.0, np.abs(want).max()), (r, name)
+    # an unweighted mean of the two ranks' gradients would be wrong here: the shards hold 18 and 9 predictions
+    plain = orc.e2e_step(shape2.replace(B=3), ce, tk, toks, ids2[:3], lab2[:3])
+    other = orc.e2e_step(shape2.replace(B=2), ce, tk, toks, ids2[3:], lab2[3:])
+    naive = 0.5 * (plain["grad_task"]["head_w"] + other["grad_task"]["head_w"])
+    assert np.abs(naive - whole["grad_task"]["head_w"]).max() > 1e-6

@@ -149,6 +149,71 @@ def test_step_rejects_bad_input_without_faulting():
     g.close()
 
 
+@pytest.mark.parametrize("K,opt", [(1, binding.GRAM_OPT_SGD), (3, binding.GRAM_OPT_SGD), (3, binding.GRAM_OPT_ADAM)])
+def test_a_rejected_step_changes_no_state(K, opt):
+    # a batch with an item ID out of range is refused with GRAM_ERR_ID_RANGE, and nothing that outlives the step has
+    # moved: parameters of both modules, the optimiser's state and counts, the Multi-step table, touched bits, cache and
+    # the position inside the window are bit-identical to what they were, also with learning rates above zero, in the
+    # middle of a window and on its last step
+    shape = small(d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=5)
+    g = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=0.05, lr_ce=0.02, optimizer=opt, ce_micro_batch=16)
+    if K > 1:
+        g.cache_fill()
+
+    def snapshot(c=None):
+        c = g if c is None else c
+        st = [c.get_params(binding.GRAM_MODULE_CE), c.get_params(binding.GRAM_MODULE_TASK)]
+        for mod in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK):
+            m, v, upd = c.optimizer_export(mod)
+            st += [np.array([upd])] + ([m, v] if m is not None else [])
+        if K > 1:
+            table, touched, cache, steps = c.state_export()
+            st += [table, touched, cache, np.array([steps])]
+        return st
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a, np.int32)).to(DEV)
+    n_good = 0
+    for step in range(2 * K + 1):
+        ids, lab = synth.batch(shape, 5, step=step)
+        if K > 1 and step in (1, K - 1 + K):          # mid-window, and on what would be the window's last step
+            before = snapshot()
+            bad = ids.copy(); bad[2, 3] = shape.n_items + 7
+            for host in (False, True):
+                with pytest.raises(binding.GramError) as e:
+                    if host:
+                        g.step_host(np.ascontiguousarray(bad, np.int32), np.ascontiguousarray(lab, np.int32), shape.B)
+                    else:
+                        g.step(dev(bad), dev(lab), shape.B)
+                assert e.value.status == 2
+                for a, b in zip(before, snapshot()):
+                    assert np.array_equal(a, b)
+        if K == 1 and step == 1:
+            before = snapshot()
+            bad = ids.copy(); bad[0, 0] = -1
+            with pytest.raises(binding.GramError) as e:
+                g.step(dev(bad), dev(lab), shape.B)
+            assert e.value.status == 2
+            for a, b in zip(before, snapshot()):
+                assert np.array_equal(a, b)
+        rep = g.step(dev(ids), dev(lab), shape.B)                # the context stays usable and keeps its place
+        n_good += 1
+        assert rep.n_unique == len(np.unique(ids))
+        if K > 1:
+            assert rep.encoder_pass == int(n_good % K == 0)
+    # the rejected steps left no trace: a second context that never saw them ends in the same state
+    g2 = gh.make_ctx(shape, ce, tk, toks, K=K, lr_task=0.05, lr_ce=0.02, optimizer=opt, ce_micro_batch=16)
+    if K > 1:
+        g2.cache_fill()
+    for step in range(2 * K + 1):
+        ids, lab = synth.batch(shape, 5, step=step)
+        g2.step(dev(ids), dev(lab), shape.B)
+    for x, y in zip(snapshot(g), snapshot(g2)):
+        assert np.array_equal(x, y)
+    g.close(); g2.close()
+
+
 @pytest.mark.parametrize("dtype,K", [("f32", 1), ("f32", 3), ("bf16", 2)])
 def test_multistep_window_matches_algorithm(dtype, K):
     shape = small(dtype=dtype, d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=max(K, 2), pooling="cls")

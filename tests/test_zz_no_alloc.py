@@ -75,3 +75,53 @@ def test_static_scratch_rejects_rows_beyond_its_maximum():
     binding.accumulate_static(dE, perm, seg, 8, G)
     torch.cuda.synchronize()
     assert torch.equal(G, dE)
+
+
+def test_static_scratch_narrow_rows_spanning_many_work_units():
+    # rows of 64 columns (one 128-column slab per warp) with a heavy-tailed draw: the hottest items span many of the
+    # 592 work units, so the second launch really adds partial sums on this path as well
+    P, N, s, d = 200_000, 3_000, 1.5, 64
+    cfg = binding.GramConfig(); cfg.n_items = N; cfg.P_max = P; cfg.d_max = d; cfg.d = d
+    g = binding.Gram(cfg)
+    ids = synth.zipf_ids(77, N, s, P)
+    dE_np = synth.position_gradients(77, P, d)
+    U, perm, seg = _dedup(g, ids, N)
+    seg_np, perm_np = seg[:U + 1].cpu().numpy(), perm.cpu().numpy()
+    counts = np.diff(seg_np)
+    assert counts.max() > 16 * (P // 592)                     # one item alone covers more than sixteen work units
+    dE = torch.from_numpy(dE_np).to(DEV)
+    got = torch.full((U, d), float("nan"), device=DEV)
+    binding.accumulate_static(dE, perm, seg, U, got)
+    torch.cuda.synchronize()
+    exact = np.zeros((U, d)); inv = np.empty(P, np.int64)
+    inv[perm_np] = np.repeat(np.arange(U), counts)
+    np.add.at(exact, inv, dE_np.astype(np.float64))
+    c = counts.astype(np.float64)[:, None]
+    assert np.all(np.abs(got.cpu().numpy() - exact) <= c * 2.0 ** -24 * c + 1e-6)
+    # a position outside the batch in d_perm is documented to be read as row 0, without an error
+    bad = perm.clone(); j = int(seg_np[3])                    # first occurrence of item 3
+    bad[j] = P
+    again = torch.full((U, d), float("nan"), device=DEV)
+    binding.accumulate_static(dE, bad, seg, U, again)
+    torch.cuda.synchronize()
+    moved = exact.copy()
+    moved[3] += dE_np[0].astype(np.float64) - dE_np[perm_np[j]].astype(np.float64)
+    assert np.all(np.abs(again.cpu().numpy() - moved) <= c * 2.0 ** -24 * c + 1e-6)
+    g.close()
+
+
+def test_static_scratch_refuses_what_it_cannot_serve():
+    perm = torch.arange(8, dtype=torch.int32, device=DEV); seg = torch.arange(9, dtype=torch.int32, device=DEV)
+    with pytest.raises(binding.GramError) as e:               # rows must be whole 16-byte pieces
+        binding.accumulate_static(torch.zeros(8, 6, device=DEV), perm, seg, 8, torch.zeros(8, 6, device=DEV))
+    assert e.value.status == 4
+    base = torch.zeros(8 * 16 + 1, device=DEV)
+    with pytest.raises(binding.GramError) as e:               # an output that does not start on a 16-byte boundary
+        binding.accumulate_static(torch.zeros(8, 16, device=DEV), perm, seg, 8, base[1:].view(8, 16))
+    assert e.value.status == 4
+    with pytest.raises(binding.GramError) as e:               # more positions than 32-bit offsets reach (sizes only, no memory touched)
+        binding.accumulate_static(torch.zeros(8, 16, device=DEV), perm, seg, 8, torch.zeros(8, 16, device=DEV), P=2 ** 31, d=16)
+    assert e.value.status == 3
+    with pytest.raises(binding.GramError) as e:
+        binding.accumulate_static(torch.zeros(8, 16, device=DEV), perm, seg, 9, torch.zeros(8, 16, device=DEV), P=8, d=16)
+    assert e.value.status == 1                                # more items than positions
