@@ -182,7 +182,7 @@ def stage_fractions(shape, stage_ms, U, peaks):
     out = {}
     for k, (w, bound) in work.items():
         ms = stage_ms[k]
-        if ms <= 0:
+        if ms <= 0 or (k == "ms_gather" and shape.task == "kt"):     # the KT module gathers in its first load: no stage of its own
             continue
         rate = w / (ms / 1e3)
         if bound == "hbm":

@@ -1050,15 +1050,28 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
   return GRAM_OK;
 }
 
-gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, float* lse, int64_t rows, int64_t n_seq, int S,
+                              int d, int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
                               const SeqGroups* groups, cudaStream_t st) {
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
-  if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
-  const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
+  if (dh * n_heads != d) return gram_set_error(ctx, "attention: d is not a multiple of the head count"), GRAM_ERR_ARG;
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 4.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_fwd");
+  if (dtype == GRAM_BF16 && attention_tc_supported(S, d, n_heads)) {
+    if (!groups || !seq_off) return attention_forward_tc(ctx, qkv, out, lse, rows, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
+    int32_t first = 0;
+    for (int gi = 0; gi < 4; ++gi) {                 // one launch per length group, with the smallest slot that fits
+      const int bound = gi < 3 ? (S < 32 * (gi + 1) ? S : 32 * (gi + 1)) : S;
+      if (groups->count[gi] > 0)
+        GRAM_TRY(attention_forward_tc(ctx, qkv, out, lse, rows, groups->count[gi], bound, d, n_heads, causal, seq_len, seq_off,
+                                      groups->list + first, st));
+      first += groups->count[gi];
+    }
+    return GRAM_OK;
+  }
+  if (S > 128 || dh > 64) return gram_set_error(ctx, "attention: this element type and head width need S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)3 * S * (dh + 1) * sizeof(float);
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads)) {
     if (!groups || !seq_off) return attention_forward_mma(ctx, qkv, out, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
     int32_t first = 0;
@@ -1078,28 +1091,54 @@ gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* o
   return GRAM_OK;
 }
 
-gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
+gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, const void* octx, const float* lse,
+                               float* delta, void* dqkv, float* colpart, int64_t colpart_cap_rows, int64_t* colpart_rows_used,
+                               int64_t rows, int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
                                const int32_t* seq_off, const SeqGroups* groups, cudaStream_t st) {
+  if (colpart_rows_used) *colpart_rows_used = 0;
   if (n_seq == 0) return GRAM_OK;
   const int dh = d / n_heads;
-  if (S > 128 || dh > 64 || dh * n_heads != d) return gram_set_error(ctx, "attention: needs S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
-  const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
+  if (dh * n_heads != d) return gram_set_error(ctx, "attention: d is not a multiple of the head count"), GRAM_ERR_ARG;
   const float scale = 1.f / sqrtf((float)dh);
   ProfScope prof(ctx, GRAM_K_ATTENTION, 10.0 * (double)n_seq * n_heads * S * S * dh, 1, st, "attn_bwd");
+  const bool grouped = groups && seq_off;
+  if (dtype == GRAM_BF16 && attention_tc_supported(S, d, n_heads)) {
+    auto bound = [&](int gi) { return gi < 3 ? (S < 32 * (gi + 1) ? S : 32 * (gi + 1)) : S; };
+    int64_t need = 0;
+    if (!grouped) need = attention_tc_colpart_rows(n_seq, S);
+    else for (int gi = 0; gi < 4; ++gi) need += groups->count[gi] > 0 ? attention_tc_colpart_rows(groups->count[gi], bound(gi)) : 0;
+    float* cp = (colpart && need <= colpart_cap_rows) ? colpart : nullptr;      // partial column sums only when they fit
+    if (cp && colpart_rows_used) *colpart_rows_used = need;
+    if (!grouped)
+      return attention_backward_tc(ctx, qkv, dctx, octx, lse, delta, dqkv, cp, 0, rows, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
+    int32_t first = 0;
+    int64_t row0 = 0;
+    for (int gi = 0; gi < 4; ++gi) {
+      if (groups->count[gi] > 0) {
+        GRAM_TRY(attention_backward_tc(ctx, qkv, dctx, octx, lse, delta, dqkv, cp, row0, rows, groups->count[gi], bound(gi), d, n_heads,
+                                       causal, seq_len, seq_off, groups->list + first, st));
+        row0 += attention_tc_colpart_rows(groups->count[gi], bound(gi));
+      }
+      first += groups->count[gi];
+    }
+    return GRAM_OK;
+  }
+  if (S > 128 || dh > 64) return gram_set_error(ctx, "attention: this element type and head width need S <= 128 and head width <= 64"), GRAM_ERR_UNSUPPORTED;
+  const size_t smem = ((size_t)4 * S * (dh + 1) + (size_t)2 * S * (S + 1)) * sizeof(float);
   if (dtype == GRAM_BF16 && attention_mma_supported(S, d, n_heads)) {
-    if (!groups || !seq_off)
-      return attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
+    float* cp = (colpart && n_seq <= colpart_cap_rows) ? colpart : nullptr;    // one row of partial sums per sequence
+    if (cp && colpart_rows_used) *colpart_rows_used = n_seq;
+    if (!grouped)
+      return attention_backward_mma(ctx, qkv, dctx, dqkv, cp, n_seq, S, d, n_heads, causal, seq_len, seq_off, nullptr, st);
     int32_t first = 0;
     for (int gi = 0; gi < 4; ++gi) {
       if (groups->count[gi] > 0)
-        GRAM_TRY(attention_backward_mma(ctx, qkv, dctx, dqkv, colpart, groups->count[gi], S < 32 * (gi + 1) ? S : 32 * (gi + 1), d,
+        GRAM_TRY(attention_backward_mma(ctx, qkv, dctx, dqkv, cp, groups->count[gi], S < 32 * (gi + 1) ? S : 32 * (gi + 1), d,
                                         n_heads, causal, seq_len, seq_off, groups->list + first, st));
       first += groups->count[gi];
     }
     return GRAM_OK;
   }
-  if (colpart) return gram_set_error(ctx, "attention: fused column sums need the tensor-core kernel"), GRAM_ERR_UNSUPPORTED;
   DISPATCH_T(dtype, {
     GRAM_TRY(set_smem(ctx, attn_bwd_kernel<T>, smem));
     attn_bwd_kernel<T><<<(unsigned)(n_seq * n_heads), 128, smem, st>>>((const T*)qkv, (const T*)dctx, (T*)dqkv, S, d, n_heads, causal, scale, seq_len, seq_off);

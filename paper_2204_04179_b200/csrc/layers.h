@@ -57,16 +57,33 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
 // whose outputs are finite and never read, and whose gradients are zero.  seq_off (may be null, needs seq_len): packed
 // rows, sequence s is rows seq_off[s] .. seq_off[s] + seq_len[s] (at most S of them) and there is no padding.
 // groups (may be null, packed rows only): the sequences grouped by length, see SeqGroups.
-gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, int64_t n_seq, int S, int d,
-                              int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
+// rows: token rows in use (n_seq * S, or the packed total).  lse (may be null): fp32 [n_heads, rows], receives per row and
+// head the base-2 logarithm of the softmax denominator plus the scaled row maximum (what the tensor-core backward reads
+// instead of recomputing the row statistics); written by the tcgen05 kernel only.
+gram_status attention_forward(gram_ctx* ctx, int dtype, const void* qkv, void* out, float* lse, int64_t rows, int64_t n_seq, int S,
+                              int d, int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off,
                               const SeqGroups* groups, cudaStream_t st);
-// colpart (may be null; only where attention_mma_supported and dtype is bf16): fp32 [n_seq, 3d], row s receives the
-// column sums of sequence s's rows of dqkv, the partial sums of the bias gradient of the Q, K, V projection
-gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, void* dqkv, float* colpart,
-                               int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
+// octx: the forward pass's output; lse: its row statistics; delta: scratch fp32 [n_heads, rows] (the last three are read by
+// the tcgen05 kernels only; octx and delta only for sequences of more than 128 rows).
+// colpart (may be null): fp32 partial column sums of dqkv, the partial sums of the bias gradient of the Q, K, V projection:
+// the tensor-core kernels fill one row of 3d sums per tile (tcgen05) or per sequence (warp-level kernel) when those rows
+// number at most colpart_cap_rows, and report the count in *colpart_rows_used (0: nothing was written, sum dqkv instead).
+gram_status attention_backward(gram_ctx* ctx, int dtype, const void* qkv, const void* dctx, const void* octx, const float* lse,
+                               float* delta, void* dqkv, float* colpart, int64_t colpart_cap_rows, int64_t* colpart_rows_used,
+                               int64_t rows, int64_t n_seq, int S, int d, int n_heads, int causal, const int32_t* seq_len,
                                const int32_t* seq_off, const SeqGroups* groups, cudaStream_t st);
 
-// the tensor-core kernels behind the two calls above (bf16, S <= 128, head width 32 or 64)
+// the tcgen05 kernels behind the two calls above (bf16, head width 64, sequences of any length)
+bool attention_tc_supported(int S, int d, int n_heads);
+gram_status attention_forward_tc(gram_ctx* ctx, const void* qkv, void* out, float* lse, int64_t rows, int64_t n_seq, int S, int d,
+                                 int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,
+                                 cudaStream_t st);
+int64_t attention_tc_colpart_rows(int64_t n_seq, int S);
+gram_status attention_backward_tc(gram_ctx* ctx, const void* qkv, const void* dctx, const void* octx, const float* lse, float* delta,
+                                  void* dqkv, float* colpart, int64_t colpart_row0, int64_t rows, int64_t n_seq, int S, int d,
+                                  int n_heads, int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,
+                                  cudaStream_t st);
+// the warp-level tensor-core kernels (bf16, S <= 128, head width 32 or 64)
 bool attention_mma_supported(int S, int d, int n_heads);
 gram_status attention_forward_mma(gram_ctx* ctx, const void* qkv, void* out, int64_t n_seq, int S, int d, int n_heads,
                                   int causal, const int32_t* seq_len, const int32_t* seq_off, const int32_t* seq_list,

@@ -30,6 +30,7 @@ struct LayerActs {
   void *qkv, *ctx, *h1, *u, *g, *out;
   float *z1, *z2, *outf;
   float *mean1, *rstd1, *mean2, *rstd2;
+  float* lse;                              // [heads, rows] softmax row statistics of the attention (tensor-core kernels)
 };
 
 // a run of post-LayerNorm transformer layers over sequences of S tokens
@@ -48,6 +49,7 @@ struct Stack {
   void *dzb = nullptr, *dqkv = nullptr, *du = nullptr, *dctx = nullptr;
   float* cpart = nullptr;                  // column-sum partials written by fused producers
   size_t cpart_elems = 0;
+  float* delta = nullptr;                  // [heads, rows] scratch of the attention backward over long sequences
 };
 
 struct Arena {
@@ -163,6 +165,7 @@ void stack_buffers(Arena& a, Stack& s, size_t esz) {
     x.qkv = a.take(T * 3 * d * esz);
     x.ctx = a.take(T * d * esz);
     x.out = a.take(T * d * esz);
+    x.lse = (float*)a.take(T * (size_t)(s.heads > 0 ? s.heads : 1) * 4);
     if (s.attn_only) {
       x.outf = (float*)a.take(T * d * 4);
     } else {
@@ -185,6 +188,7 @@ void stack_buffers(Arena& a, Stack& s, size_t esz) {
   s.du = s.attn_only ? nullptr : a.take(T * f * esz);
   s.cpart_elems = ((T + 31) / 32) * (f > 3 * d ? f : 3 * d);     // [ceil(T / 32)][d_ff] or [sequences][3 d]
   s.cpart = (float*)a.take(s.cpart_elems * 4);
+  s.delta = (float*)a.take(T * (size_t)(s.heads > 0 ? s.heads : 1) * 4);
 }
 
 void layout_buffers(Model* m, Arena& a) {
@@ -329,7 +333,8 @@ gram_status layer_attention_forward(Model* m, Module& mod, Stack& s, int l, cons
   e.bias = mod.w + o.bqkv;
   e.tag = "fwd_qkv";
   GRAM_TRY(mm_fwd(m, xb, W(m, mod, o.wqkv), a.qkv, false, T, 3 * s.d, s.d, e, st));
-  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, n_seq, S, s.d, s.heads, s.causal, s.seq_len, s.seq_off, s.grouped ? &s.groups : nullptr, st);
+  return attention_forward(m->ctx, m->dtype, a.qkv, a.ctx, a.lse, T, n_seq, S, s.d, s.heads, s.causal, s.seq_len, s.seq_off,
+                           s.grouped ? &s.groups : nullptr, st);
 }
 
 // the row-wise rest of the layer over T rows: output projection + residual, LayerNorm, feed-forward + residual,
@@ -447,11 +452,12 @@ gram_status layer_attention_backward(Model* m, Module& mod, Stack& s, int l, con
   gram_ctx* ctx = m->ctx;
   const LayerOff& o = s.off[l];
   LayerActs& a = s.acts[l];
-  const bool fused_bqkv = m->dtype == GRAM_BF16 && attention_mma_supported(S, d, s.heads) &&
-                          (size_t)n_seq * 3 * d <= s.cpart_elems;                      // the kernel also adds up dqkv's columns
-  GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, s.dqkv, fused_bqkv ? s.cpart : nullptr, n_seq, S, d, s.heads,
-                              s.causal, s.seq_len, s.seq_off, s.grouped ? &s.groups : nullptr, st));
-  if (fused_bqkv) GRAM_TRY(colsum_from_partials(ctx, s.cpart, n_seq, 3 * d, mod.g + o.bqkv, m->red, st));
+  // the tensor-core kernels also add up dqkv's columns, as partial sums that fit the scratch or not at all
+  int64_t part_rows = 0;
+  GRAM_TRY(attention_backward(ctx, m->dtype, a.qkv, s.dctx, a.ctx, a.lse, s.delta, s.dqkv, s.cpart,
+                              (int64_t)(s.cpart_elems / ((size_t)3 * d)), &part_rows, T, n_seq, S, d, s.heads, s.causal, s.seq_len,
+                              s.seq_off, s.grouped ? &s.groups : nullptr, st));
+  if (part_rows > 0) GRAM_TRY(colsum_from_partials(ctx, s.cpart, part_rows, 3 * d, mod.g + o.bqkv, m->red, st));
   else GRAM_TRY(colsum_accumulate(ctx, m->dtype, s.dqkv, T, 3 * d, mod.g + o.bqkv, m->red, st));
   GRAM_TRY(mm_dw(m, s.dqkv, xb_l, mod.g + o.wqkv, T, 3 * d, d, st, "dw_qkv"));
   GemmEpilogue e;

@@ -35,6 +35,28 @@ CASES = {
     "bf16_long_seq": small(dtype="bf16", l_t=70, L=100, B=2, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30,
                            task_attn_only=False),
     "bf16_seq128": small(dtype="bf16", l_t=128, L=128, B=1, d=64, n_heads=2, d_ff=64, task_d_ff=64, n_items=12, pooling="cls"),
+    # heads of width 64: the tcgen05 attention kernels.  Sequences packed into 128-row tiles in slots of 16 (whole tiles in
+    # one copy) and 32 rows with an empty slot at the end (3 histories), slots wider than the sequences (24 in 32, 20 in 32),
+    # two sequences per tile, and one sequence per tile with a ragged tail (100 of 128 rows, causal)
+    "bf16_dh64_s16": small(dtype="bf16", d=128, n_heads=2, task_heads=2, d_ff=128, task_d_ff=128, l_t=16, L=32, B=3, n_items=40,
+                           pooling="cls", task_attn_only=False),
+    "bf16_dh64_s24": small(dtype="bf16", d=128, n_heads=2, task_heads=2, d_ff=128, task_d_ff=128, l_t=24, L=20, B=5, n_items=40,
+                           pooling="mean"),
+    "bf16_dh64_s64": small(dtype="bf16", d=128, n_heads=2, task_heads=2, d_ff=128, task_d_ff=128, l_t=64, L=64, B=3, n_items=30,
+                           pooling="cls", task_attn_only=False),
+    "bf16_dh64_s128": small(dtype="bf16", d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, l_t=128, L=100, B=2, n_items=14,
+                            pooling="mean"),
+    # texts longer than one 128-row tile (Table 3 lists mean lengths of 147 and 271 tokens, Appendix D truncates at 512):
+    # several query tiles per sequence, a running maximum and sum over the key tiles, a ragged last tile; and histories
+    # of 200 positions through the causal task module
+    "bf16_dh64_t147": small(dtype="bf16", d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, l_t=147, L=6, B=2, n_items=8,
+                            n_layers=1, pooling="mean"),
+    "bf16_dh64_t271": small(dtype="bf16", d=128, n_heads=2, task_heads=2, d_ff=128, task_d_ff=128, l_t=271, L=6, B=2, n_items=8,
+                            n_layers=1, pooling="cls"),
+    "bf16_dh64_t512": small(dtype="bf16", d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, l_t=512, L=12, B=3, n_items=8,
+                            n_layers=1, pooling="mean"),
+    "bf16_dh64_L200": small(dtype="bf16", d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, l_t=8, L=200, B=2, n_items=30,
+                            n_layers=1, pooling="mean", task_attn_only=False),
 }
 
 
@@ -328,6 +350,12 @@ VARLEN = {
     # tensor-core attention: texts of 1..40 tokens in a 64-row tile, and 1..70 in a 96-row tile
     "bf16_mean_40": small(dtype="bf16", l_t=40, d=64, n_heads=2, d_ff=128, task_d_ff=128, n_items=30, pooling="mean"),
     "bf16_cls_70": small(dtype="bf16", l_t=70, d=64, n_heads=1, d_ff=64, task_d_ff=64, n_items=30, pooling="cls", B=2),
+    # heads of width 64 (tcgen05 attention): packed rows, one launch per length group, slots of 32, 64 and 128 rows
+    "bf16_dh64_var40": small(dtype="bf16", l_t=40, d=128, n_heads=2, task_heads=2, d_ff=128, task_d_ff=128, n_items=30, pooling="mean"),
+    "bf16_dh64_var128": small(dtype="bf16", l_t=128, d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, n_items=24, pooling="cls", B=3),
+    # texts of 1..300 tokens: the three short groups, and a last group that mixes 97..128-row texts with multi-tile ones
+    "bf16_dh64_var300": small(dtype="bf16", l_t=300, d=64, n_heads=1, task_heads=1, d_ff=64, task_d_ff=64, n_items=16, n_layers=1,
+                              pooling="mean", B=2, L=8),
     # several ragged encoder passes of 7 items, each with its own packed layout
     "f32_cls_micro_batches": small(l_t=9, pooling="cls", n_items=60, B=6, L=16),
 }
