@@ -70,7 +70,9 @@ enum { GRAM_MULTI_TABLE = 0, GRAM_MULTI_PSEUDO_TARGET = 1 };
  * attention, erf-GELU feed-forward), pooled to one d-vector per item.
  * CF (Section 3.1): task = KT: x_n = E[b,n] + pos[n] + resp[r_{n-1}], task_layers
  * causal layers (attention only when task_attn_only != 0), a linear head and
- * binary cross-entropy averaged over B*L predictions; task = NR: additive
+ * binary cross-entropy averaged over B*L predictions; task = NR: task_layers
+ * self-attention layers (not causal) over the clicked items of a user (Appendix D
+ * uses one; 0 = none), then additive
  * attention (width d_a) over the first L - n_cand encodings, dot-product scores
  * with the n_cand candidates, softmax cross-entropy on candidate 0 averaged
  * over B.  A context with n_layers == 0 and task == GRAM_TASK_NONE serves only
@@ -132,8 +134,8 @@ const char* gram_last_error(const gram_ctx* ctx);
  * tok_emb[vocab,d] pos_emb[l_t,d] emb_ln_g[d] emb_ln_b[d], then per layer
  * wqkv[3d,d] bqkv[3d] wo[d,d] bo[d] ln1_g ln1_b w1[d_ff,d] b1[d_ff] w2[d,d_ff]
  * b2[d] ln2_g ln2_b, then for GRAM_POOL_ADDITIVE pool_wa[d_a,d] pool_ba[d_a] pool_qa[d_a]; for KT: pos[L,d] resp[3,d], the layers (attention-only
- * layers hold wqkv bqkv wo bo), head_w[d] head_b[1]; for NR: wa[d_a,d] ba[d_a]
- * qa[d_a].  Rows 0..d-1 of wqkv produce Q, the next d K, the last d V; head h
+ * layers hold wqkv bqkv wo bo), head_w[d] head_b[1]; for NR: the task_layers
+ * layers, then wa[d_a,d] ba[d_a] qa[d_a].  Rows 0..d-1 of wqkv produce Q, the next d K, the last d V; head h
  * owns columns h*d/n_heads .. of each. */
 gram_status gram_param_count(const gram_ctx* ctx, int module, size_t* n);
 gram_status gram_set_params(gram_ctx* ctx, int module, const float* h_params, size_t n);

@@ -189,6 +189,123 @@ __device__ __forceinline__ void mma_mn_mn(uint32_t tmem_d, uint32_t sa, uint32_t
            (accumulate || k > 0) ? 1u : 0u);
 }
 
+// ---- register-resident softmax blocks for tiles whose rows look at no more than W = 32 or 64 score columns ----
+// (slots of up to 64 rows: a warp's 32 rows then share one window of W columns starting at cb)
+
+// 16 bytes of zeros into every 16-byte piece of row r of a 128 x 128 bf16 tile (two halves) outside columns [cb, cb + W)
+template <int W>
+__device__ __forceinline__ void zero_outside(uint32_t buf, int r, int cb) {
+#pragma unroll
+  for (int piece = 0; piece < 16; ++piece) {
+    const int col = piece * 8;
+    if (col < cb || col >= cb + W) sts128(swz(buf + (uint32_t)(piece >> 3) * TILE_BYTES, r, piece & 7), 0u, 0u, 0u, 0u);
+  }
+}
+// 32 packed bf16 pairs... the 16 words pk (32 columns from column c0) into row r of such a tile
+__device__ __forceinline__ void store_block32(uint32_t buf, int r, int c0, const uint32_t (&pk)[16]) {
+  const int piece0 = c0 >> 3;
+#pragma unroll
+  for (int c4 = 0; c4 < 4; ++c4) {
+    const int piece = piece0 + c4;
+    sts128(swz(buf + (uint32_t)(piece >> 3) * TILE_BYTES, r, piece & 7), pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
+  }
+}
+
+// Forward: the scores of this thread's row in columns [cb, cb + W) of S (tensor memory) -> probabilities exp2(c s - c max)
+// in the probability tile (zeros outside [lo, hi) and outside the window); returns the row maximum and the sum.
+template <int W, bool full>
+__device__ __forceinline__ void fwd_block_m(uint32_t s_addr, uint32_t pb, int r, int cb, int l0, int h0, float c, float& mx_out,
+                                            float& sum_out) {
+  constexpr int NB = W / 32;
+  uint32_t v[NB][32];
+#pragma unroll
+  for (int i = 0; i < NB; ++i) tc_ld32_issue(s_addr + (uint32_t)(cb + 32 * i), v[i]);
+#pragma unroll
+  for (int i = 0; i < NB; ++i) tc_ld32_wait(v[i]);
+  float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};          // four chains: the reductions are latency-bound otherwise
+#pragma unroll
+  for (int i = 0; i < NB; ++i)
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+      if (full || (32 * i + e >= l0 && 32 * i + e < h0)) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(v[i][e]));
+  const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+  const float mc = (mx == -INFINITY) ? 0.f : mx * c;
+  float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+      const int k0 = 32 * i + e;
+      const float p0 = (full || (k0 >= l0 && k0 < h0)) ? ex2(fmaf(__uint_as_float(v[i][e]), c, -mc)) : 0.f;
+      const float p1 = (full || (k0 + 1 >= l0 && k0 + 1 < h0)) ? ex2(fmaf(__uint_as_float(v[i][e + 1]), c, -mc)) : 0.f;
+      s4[(e >> 1) & 3] += p0 + p1;
+      pk[e >> 1] = pack_bf16x2(p0, p1);
+    }
+    store_block32(pb, r, cb + 32 * i, pk);
+  }
+  zero_outside<W>(pb, r, cb);
+  mx_out = mx;
+  sum_out = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+}
+// the unmasked variant when every row of the warp sees the whole window (equal-length sequences that fill their slots,
+// no causal mask): the per-element range tests are then not even fetched
+template <int W>
+__device__ __forceinline__ void fwd_block(uint32_t s_addr, uint32_t pb, int r, int cb, int lo, int hi, float c, float& mx_out,
+                                          float& sum_out) {
+  const int l0 = lo - cb, h0 = hi - cb;
+  if (__all_sync(0xffffffffu, l0 == 0 && h0 == W)) fwd_block_m<W, true>(s_addr, pb, r, cb, l0, h0, c, mx_out, sum_out);
+  else fwd_block_m<W, false>(s_addr, pb, r, cb, l0, h0, c, mx_out, sum_out);
+}
+
+// Backward: S and dP of this thread's row in columns [cb, cb + W) -> P = exp2(c S - lse) and dS = P (dP - delta) scale, bf16,
+// into the two tiles (zeros outside).  own_delta: delta is the row's sum of P dP (single key tile), else delta_in.
+template <int W, bool full>
+__device__ __forceinline__ void bwd_block_m(uint32_t lane_base, uint32_t pbuf, uint32_t dsbuf, int r, int cb, int l0, int h0, float c,
+                                            float lse2, float scale, bool own_delta, float delta_in) {
+  constexpr int NB = W / 32;
+  uint32_t v[NB][32], w[NB][32];
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
+    tc_ld32_issue(lane_base + (uint32_t)(cb + 32 * i), v[i]);
+    tc_ld32_issue(lane_base + 128u + (uint32_t)(cb + 32 * i), w[i]);
+  }
+#pragma unroll
+  for (int i = 0; i < NB; ++i) { tc_ld32_wait(v[i]); tc_ld32_wait(w[i]); }
+  float d4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < NB; ++i)
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const int k0 = 32 * i + e;
+      const float p = (full || (k0 >= l0 && k0 < h0)) ? ex2(fmaf(__uint_as_float(v[i][e]), c, -lse2)) : 0.f;
+      v[i][e] = __float_as_uint(p);
+      d4[e & 3] = fmaf(p, __uint_as_float(w[i][e]), d4[e & 3]);
+    }
+  const float delta = own_delta ? (d4[0] + d4[1]) + (d4[2] + d4[3]) : delta_in;
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
+    uint32_t pk[16], dk[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+      const float p0 = __uint_as_float(v[i][e]), p1 = __uint_as_float(v[i][e + 1]);
+      pk[e >> 1] = pack_bf16x2(p0, p1);
+      dk[e >> 1] = pack_bf16x2(p0 * scale * (__uint_as_float(w[i][e]) - delta), p1 * scale * (__uint_as_float(w[i][e + 1]) - delta));
+    }
+    store_block32(pbuf, r, cb + 32 * i, pk);
+    store_block32(dsbuf, r, cb + 32 * i, dk);
+  }
+  zero_outside<W>(pbuf, r, cb);
+  zero_outside<W>(dsbuf, r, cb);
+}
+template <int W>
+__device__ __forceinline__ void bwd_block(uint32_t lane_base, uint32_t pbuf, uint32_t dsbuf, int r, int cb, int lo, int hi, float c,
+                                          float lse2, float scale, bool own_delta, float delta_in) {
+  const int l0 = lo - cb, h0 = hi - cb;
+  if (__all_sync(0xffffffffu, l0 == 0 && h0 == W)) bwd_block_m<W, true>(lane_base, pbuf, dsbuf, r, cb, l0, h0, c, lse2, scale, own_delta, delta_in);
+  else bwd_block_m<W, false>(lane_base, pbuf, dsbuf, r, cb, l0, h0, c, lse2, scale, own_delta, delta_in);
+}
+
 struct Shared {
   uint32_t tiles;            // shared-memory address of the first stage (1024-byte aligned)
   uint32_t pbuf;             // the softmax groups' probability tiles
@@ -200,9 +317,11 @@ struct Shared {
 // ============================================================================================
 // forward
 // barriers: full[s], empty[s] per stage; per softmax group g: s_full[g] (scores in tensor memory),
-// p_full[g] (probabilities in shared memory, 128 arrivals), pv_done[g] (output accumulator complete)
+// p_full[g] (probabilities in shared memory, one arrival per warp), pv_done[g] (output accumulator complete)
 // tensor memory: S_g at columns 128 g, O_g at columns 256 + 64 g
 // ============================================================================================
+// WM: 32 or 64: short mode with slots of up to 32 / 64 rows (a row's scores fit a register-resident window); 128: the rest
+template <int WM>
 __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_qkv, AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -222,7 +341,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < FWD_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int g = 0; g < 2; ++g) { mbar_init(sfull_bar(g), 1); mbar_init(pfull_bar(g), 128); mbar_init(pvdone_bar(g), 1); }
+    for (int g = 0; g < 2; ++g) { mbar_init(sfull_bar(g), 1); mbar_init(pfull_bar(g), 4); mbar_init(pvdone_bar(g), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -312,11 +431,18 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
       for (int j = 0; j < x.nk && !failed; ++j, ++k) {
         int lo, hi;
         key_range(a, ri, j, lo, hi);
+        if (!mbar_wait(sfull_bar(g), k & 1u, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        if constexpr (WM <= 64) {
+          // one key tile and a window of at most 64 columns per row: everything stays in registers
+          float mx, sum;
+          fwd_block<WM>(s_addr, pb, r, WM * ((quarter * 32) / WM), lo, hi, a.c, mx, sum);
+          m_run = mx;
+          l_run = sum;
+        } else {
         // the 32-column blocks some row of this warp needs
         const int wlo = __reduce_min_sync(0xffffffffu, hi > lo ? lo : TQ), whi = __reduce_max_sync(0xffffffffu, hi > lo ? hi : 0);
         const int q0 = wlo >> 5, q1 = (whi + 31) >> 5;     // blocks [q0, q1)
-        if (!mbar_wait(sfull_bar(g), k & 1u, abort_flag)) { failed = true; break; }
-        tc_fence_after();
         float mx = -INFINITY;
         for (int q = q0; q < q1; ++q) {
           uint32_t v[32];
@@ -374,26 +500,32 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
         }
         l_run = l_run * alpha + sum;
         m_run = m_new;
+        }
         tc_fence_before();
         fence_proxy_async_smem();
-        mbar_arrive(pfull_bar(g));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pfull_bar(g));      // one arrival per warp: 128 would serialise on the barrier word
       }
       if (failed) break;
       // ---- the item's output: O / l, bf16, through this warp's rows of the probability tile, in whole rows ----
       if (!mbar_wait(pvdone_bar(g), (k - 1) & 1u, abort_flag)) { failed = true; break; }
       tc_fence_after();
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-#pragma unroll 1
-      for (int hblk = 0; hblk < 2; ++hblk) {
-        uint32_t v[32];
-        tc_ld32_issue(o_addr + 32u * hblk, v);
-        tc_ld32_wait(v);
+      {
+        uint32_t o[2][32];
+        tc_ld32_issue(o_addr, o[0]);
+        tc_ld32_issue(o_addr + 32u, o[1]);
+        tc_ld32_wait(o[0]);
+        tc_ld32_wait(o[1]);
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-          sts128(swz(pb, r, hblk * 4 + c4), pack_bf16x2(__uint_as_float(v[8 * c4]) * inv, __uint_as_float(v[8 * c4 + 1]) * inv),
-                 pack_bf16x2(__uint_as_float(v[8 * c4 + 2]) * inv, __uint_as_float(v[8 * c4 + 3]) * inv),
-                 pack_bf16x2(__uint_as_float(v[8 * c4 + 4]) * inv, __uint_as_float(v[8 * c4 + 5]) * inv),
-                 pack_bf16x2(__uint_as_float(v[8 * c4 + 6]) * inv, __uint_as_float(v[8 * c4 + 7]) * inv));
+        for (int hblk = 0; hblk < 2; ++hblk)
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4)
+            sts128(swz(pb, r, hblk * 4 + c4),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4]) * inv, __uint_as_float(o[hblk][8 * c4 + 1]) * inv),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 2]) * inv, __uint_as_float(o[hblk][8 * c4 + 3]) * inv),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 4]) * inv, __uint_as_float(o[hblk][8 * c4 + 5]) * inv),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 6]) * inv, __uint_as_float(o[hblk][8 * c4 + 7]) * inv));
       }
       tc_fence_before();
       if (a.lse && ri.valid) a.lse[(int64_t)x.h * a.T + ri.grow] = m_run * a.c + lg2(l_run);
@@ -448,7 +580,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
 //   mode 2: an item is a query tile and walks its key tiles: dQ.  Modes 1 and 2 read delta = dO . O per row from memory.
 // barriers: full[s], empty[s] (four arrivals: the MMA thread's commits for a step inside an item, the group's four warps
 // after the item's last step, because the results leave through the stage's own tiles); per group g: sdp_full, pds_full
-// (128 arrivals), out_full, out_free (128), csum (128).
+// (one arrival per warp), out_full, out_free, csum (one per warp).
 // tensor memory: S 0..127, dP 128..255, dV 256..319, dK 320..383, dQ 384..447
 // ============================================================================================
 constexpr int BWD_STAGES = 2;
@@ -489,6 +621,7 @@ __device__ __forceinline__ BwdItem bwd_item_of(const AttnBwdArgs& b, int64_t it)
   return y;
 }
 
+template <int WM>
 __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __grid_constant__ CUtensorMap tm_qkv,
                                                                      const __grid_constant__ CUtensorMap tm_do, AttnBwdArgs b) {
   const AttnArgs& a = b.f;
@@ -515,8 +648,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __gri
   if (threadIdx.x == 0) {
     for (int s = 0; s < BWD_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 4); }
     for (int g = 0; g < 2; ++g) {
-      mbar_init(sdp_bar(g), 1); mbar_init(pds_bar(g), 128); mbar_init(outfull_bar(g), 1); mbar_init(outfree_bar(g), 128);
-      mbar_init(csum_bar(g), 128);
+      mbar_init(sdp_bar(g), 1); mbar_init(pds_bar(g), 4); mbar_init(outfull_bar(g), 1); mbar_init(outfree_bar(g), 4);
+      mbar_init(csum_bar(g), 4);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -621,6 +754,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __gri
         float delta = (b.mode != 0 && ri.valid) ? b.delta[(int64_t)y.x.h * a.T + ri.grow] : 0.f;
         if (!mbar_wait(sdp_bar(g), k & 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
+        if constexpr (WM <= 64) {
+          bwd_block<WM>(lane_base, pbuf, dsbuf, r, WM * ((quarter * 32) / WM), lo, hi, a.c, lse2, b.scale, true, 0.f);
+        } else {
         // pass 1: P (bf16, to shared memory) and, in mode 0, delta = sum_j P dP
         float dsum = 0.f;
 #pragma unroll 1
@@ -683,9 +819,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __gri
           for (int c4 = 0; c4 < 4; ++c4)
             sts128(swz(half, r, (q & 1) * 4 + c4), pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
         }
+        }
         tc_fence_before();
         fence_proxy_async_smem();
-        mbar_arrive(pds_bar(g));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pds_bar(g));
       }
       if (failed) break;
       // ---- the item's results: bf16, through the (no longer read) tiles of the item's last stage, in whole rows ----
@@ -700,26 +838,29 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __gri
         if ((which == 0 && !want_q) || (which > 0 && !want_kv)) continue;
         const uint32_t tcol = which == 0 ? 384u : (which == 1 ? 320u : 256u);
         const uint32_t dst = st + (uint32_t)which * TILE_BYTES;
-#pragma unroll 1
+        uint32_t o[2][32];
+        tc_ld32_issue(lane_base + tcol, o[0]);
+        tc_ld32_issue(lane_base + tcol + 32u, o[1]);
+        tc_ld32_wait(o[0]);
+        tc_ld32_wait(o[1]);
+#pragma unroll
         for (int hblk = 0; hblk < 2; ++hblk) {
-          uint32_t v[32];
-          tc_ld32_issue(lane_base + tcol + 32u * hblk, v);
-          tc_ld32_wait(v);
           if (!ro.valid) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = 0u;
+            for (int e = 0; e < 32; ++e) o[hblk][e] = 0u;
           }
 #pragma unroll
           for (int c4 = 0; c4 < 4; ++c4)
-            sts128(swz(dst, r, hblk * 4 + c4), pack_bf16x2(__uint_as_float(v[8 * c4]), __uint_as_float(v[8 * c4 + 1])),
-                   pack_bf16x2(__uint_as_float(v[8 * c4 + 2]), __uint_as_float(v[8 * c4 + 3])),
-                   pack_bf16x2(__uint_as_float(v[8 * c4 + 4]), __uint_as_float(v[8 * c4 + 5])),
-                   pack_bf16x2(__uint_as_float(v[8 * c4 + 6]), __uint_as_float(v[8 * c4 + 7])));
+            sts128(swz(dst, r, hblk * 4 + c4),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4]), __uint_as_float(o[hblk][8 * c4 + 1])),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 2]), __uint_as_float(o[hblk][8 * c4 + 3])),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 4]), __uint_as_float(o[hblk][8 * c4 + 5])),
+                   pack_bf16x2(__uint_as_float(o[hblk][8 * c4 + 6]), __uint_as_float(o[hblk][8 * c4 + 7])));
         }
       }
       tc_fence_before();
-      mbar_arrive(outfree_bar(g));                     // tensor memory may take the next item's results
       __syncwarp();
+      if (lane == 0) mbar_arrive(outfree_bar(g));      // tensor memory may take the next item's results
       const int piece = lane & 7, sub = lane >> 3;
 #pragma unroll 1
       for (int which = 0; which < 3; ++which) {
@@ -752,7 +893,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_bwd_kernel(const __gri
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar(last_stage));      // this warp no longer touches the stage's tiles
       if (b.colpart) {
-        mbar_arrive(csum_bar(g));
+        if (lane == 0) mbar_arrive(csum_bar(g));       // after the __syncwarp above: this warp's partial sums are written
         if (!mbar_wait(csum_bar(g), (ki - 1) & 1u, abort_flag)) { failed = true; break; }
         // the four warps' sums in warp order: 192 columns, two per thread
         const int t2 = threadIdx.x - 64 - g * 128;            // 0..127 within the group
@@ -837,10 +978,14 @@ void plan_launch(AttnArgs& a, int64_t n_seq, int S, bool contiguous) {
 
 }  // namespace
 
-// GRAM_ATTN_TC=0 in the environment keeps the warp-level kernels (for comparisons)
+// Which sequences take these kernels: GRAM_ATTN_TC=1 in the environment: all (head width 64); GRAM_ATTN_TC=0: none;
+// unset: those the warp-level kernels cannot hold (more than 128 rows).  For short sequences the warp-level kernels, with
+// many small blocks per SM, hide memory latency better than one persistent block per SM does and are the faster ones
+// as measured on the knowledge-tracing workload.
 bool attention_tc_supported(int S, int d, int n_heads) {
-  static const bool on = []() { const char* v = getenv("GRAM_ATTN_TC"); return !(v && v[0] == '0'); }();
-  return on && S >= 1 && n_heads > 0 && d == n_heads * DH && get_encode_fn() != nullptr;
+  static const int mode = []() { const char* v = getenv("GRAM_ATTN_TC"); return !v ? 2 : (v[0] == '0' ? 0 : 1); }();
+  if (mode == 0 || !(S >= 1 && n_heads > 0 && d == n_heads * DH && get_encode_fn() != nullptr)) return false;
+  return mode == 1 || S > TQ;
 }
 
 gram_status attention_forward_tc(gram_ctx* ctx, const void* qkv, void* out, float* lse, int64_t rows, int64_t n_seq, int S, int d,
@@ -859,11 +1004,15 @@ gram_status attention_forward_tc(gram_ctx* ctx, const void* qkv, void* out, floa
     return gram_set_error(ctx, "attention: cuTensorMapEncodeTiled failed"), GRAM_ERR_CUDA;
   static bool attr_set = false;
   if (!attr_set) {
-    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_fwd_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
     attr_set = true;
   }
   const int grid = (int)(a.n_items < kNumSMs ? a.n_items : kNumSMs);
-  attn_tc_fwd_kernel<<<grid, ATT_THREADS, FWD_SMEM, st>>>(tm, a);
+  if (!a.long_mode && a.slot <= 32) attn_tc_fwd_kernel<32><<<grid, ATT_THREADS, FWD_SMEM, st>>>(tm, a);
+  else if (!a.long_mode && a.slot == 64) attn_tc_fwd_kernel<64><<<grid, ATT_THREADS, FWD_SMEM, st>>>(tm, a);
+  else attn_tc_fwd_kernel<128><<<grid, ATT_THREADS, FWD_SMEM, st>>>(tm, a);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }
@@ -898,13 +1047,17 @@ gram_status attention_backward_tc(gram_ctx* ctx, const void* qkv, const void* dc
     return gram_set_error(ctx, "attention: cuTensorMapEncodeTiled failed"), GRAM_ERR_CUDA;
   static bool attr_set = false;
   if (!attr_set) {
-    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_bwd_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
+    GRAM_CUDA(ctx, cudaFuncSetAttribute(attn_tc_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
     attr_set = true;
   }
   const int grid = (int)(a.n_items < kNumSMs ? a.n_items : kNumSMs);
   if (!a.long_mode) {
     b.mode = 0;
-    attn_tc_bwd_kernel<<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
+    if (a.slot <= 32) attn_tc_bwd_kernel<32><<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
+    else if (a.slot == 64) attn_tc_bwd_kernel<64><<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
+    else attn_tc_bwd_kernel<128><<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
   } else {
     if (!delta || !octx) return gram_set_error(ctx, "attention backward: long sequences need the forward output and a scratch row vector"), GRAM_ERR_ARG;
     int blocks = (int)((rows + 7) / 8);
@@ -913,9 +1066,9 @@ gram_status attention_backward_tc(gram_ctx* ctx, const void* qkv, const void* dc
     if (colpart)      // tiles a sequence does not have leave their rows unwritten
       GRAM_CUDA(ctx, cudaMemsetAsync(colpart + colpart_row0 * 3 * (int64_t)d, 0, (size_t)(n_seq * a.nq_max) * 3 * d * sizeof(float), st));
     b.mode = 1;
-    attn_tc_bwd_kernel<<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
+    attn_tc_bwd_kernel<128><<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
     b.mode = 2;
-    attn_tc_bwd_kernel<<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
+    attn_tc_bwd_kernel<128><<<grid, ATT_THREADS, BWD_SMEM, st>>>(tq, td, b);
   }
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;

@@ -347,18 +347,86 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
     }
     tc_fence_before();
     return true;
-  } else if constexpr (MODE == EPI_BIAS || MODE == EPI_GELU || MODE == EPI_RES) {
+  } else if constexpr (MODE == EPI_RES) {
+    // fp32 result = accumulator (+ bias) + residual (LayerNorm applied where it is read), plus an optional bf16 copy.
+    // The residual is 4 bytes per element from HBM, and eight warps per SM keep too few loads in flight to hide its
+    // latency if every 32-column block waits for its own: the loads of a block are therefore issued one block ahead,
+    // the first block's before the wait for the accumulator.
+    constexpr int NBLK = BN / PARTS / 32;
+    const int sub = lane >> 3, slot = lane & 7;
+    const int64_t rows_left = a.M - (row0 + sub);         // row rr*4 + sub exists iff rr*4 < rows_left
+    const int64_t step = 4 * a.ldc;
+    const int nbase = tn * BN + half * (BN / PARTS) + slot * 4;
+    const int64_t obase = (row0 + sub) * a.ldc + nbase;
+    float4 rnext[8];
+    auto load_res = [&](int blk, float4 (&dst)[8]) {
+      const bool col_ok = nbase + blk * 32 < a.N;
+      const float* rp = a.epi.res + obase + blk * 32;
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr)
+        dst[rr] = (col_ok && rr * 4 < rows_left) ? __ldcs(reinterpret_cast<const float4*>(rp + rr * step)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    load_res(0, rnext);
+    float mu_l = 0.f, rs_l = 1.f;
+    const bool ln = a.epi.res_mean != nullptr;
+    if (ln && row0 + lane < a.M) {
+      mu_l = a.epi.res_mean[row0 + lane];
+      rs_l = a.epi.res_rstd[row0 + lane];
+    }
+    if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+    tc_fence_after();
+#pragma unroll 1
+    for (int blk = 0; blk < NBLK; ++blk) {
+      float4 r4[8];
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr) r4[rr] = rnext[rr];
+      if (blk + 1 < NBLK) load_res(blk + 1, rnext);
+      uint32_t v[32];
+      tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / PARTS) + blk * 32), v);
+      tc_ld32_wait(v);
+      stage_write_row(stage, lane, v);
+      __syncwarp();
+      const int n = nbase + blk * 32;
+      if (n < a.N) {
+        float b4[4] = {0.f, 0.f, 0.f, 0.f}, g4[4] = {0.f, 0.f, 0.f, 0.f}, be4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (a.epi.bias) ld4(a.epi.bias + n, b4);
+        if (ln) {
+          ld4(a.epi.res_gamma + n, g4);
+          ld4(a.epi.res_beta + n, be4);
+        }
+        CT* cp = Cs + obase + blk * 32;
+        bf16* qp = a.epi.copy_out ? reinterpret_cast<bf16*>(a.epi.copy_out) + obase + blk * 32 : nullptr;
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr) {
+          const int rl = rr * 4 + sub;
+          const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
+          if (rr * 4 < rows_left) {
+            const float4 t = stage_read(stage, rl, slot);
+            float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
+            if (ln) {
+              x[0] += (r4[rr].x - mu) * rs * g4[0] + be4[0];
+              x[1] += (r4[rr].y - mu) * rs * g4[1] + be4[1];
+              x[2] += (r4[rr].z - mu) * rs * g4[2] + be4[2];
+              x[3] += (r4[rr].w - mu) * rs * g4[3] + be4[3];
+            } else {
+              x[0] += r4[rr].x; x[1] += r4[rr].y; x[2] += r4[rr].z; x[3] += r4[rr].w;
+            }
+            st4(cp, x);
+            if (qp) st4(qp, x);
+          }
+          cp += step;
+          if (qp) qp += step;
+        }
+      }
+      __syncwarp();
+    }
+    tc_fence_before();
+    return true;
+  } else if constexpr (MODE == EPI_BIAS || MODE == EPI_GELU) {
     if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
     tc_fence_after();
     const int sub = lane >> 3, slot = lane & 7;
     const int64_t rows_left = a.M - (row0 + sub);         // row rr*4 + sub exists iff rr*4 < rows_left
-    float mu_l = 0.f, rs_l = 1.f;
-    if constexpr (MODE == EPI_RES) {
-      if (a.epi.res_mean && row0 + lane < a.M) {
-        mu_l = a.epi.res_mean[row0 + lane];
-        rs_l = a.epi.res_rstd[row0 + lane];
-      }
-    }
 #pragma unroll 1
     for (int c0 = half * (BN / PARTS); c0 < (half + 1) * (BN / PARTS); c0 += 32) {
       uint32_t v[32];
@@ -404,41 +472,6 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
             }
             cp += step;
             pp += step;
-          }
-        } else {
-          float g4[4] = {0.f, 0.f, 0.f, 0.f}, be4[4] = {0.f, 0.f, 0.f, 0.f};
-          const bool ln = a.epi.res_mean != nullptr;
-          if (ln) {
-            ld4(a.epi.res_gamma + n, g4);
-            ld4(a.epi.res_beta + n, be4);
-          }
-          const float* rp = a.epi.res + o0;
-          float4 r4[8];
-#pragma unroll
-          for (int rr = 0; rr < 8; ++rr)                  // all residual loads first
-            r4[rr] = (rr * 4 < rows_left) ? *reinterpret_cast<const float4*>(rp + rr * step) : make_float4(0.f, 0.f, 0.f, 0.f);
-          CT* cp = Cs + o0;
-          bf16* qp = a.epi.copy_out ? reinterpret_cast<bf16*>(a.epi.copy_out) + o0 : nullptr;
-#pragma unroll
-          for (int rr = 0; rr < 8; ++rr) {
-            const int rl = rr * 4 + sub;
-            const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
-            if (rr * 4 < rows_left) {
-              const float4 t = stage_read(stage, rl, slot);
-              float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
-              if (ln) {
-                x[0] += (r4[rr].x - mu) * rs * g4[0] + be4[0];
-                x[1] += (r4[rr].y - mu) * rs * g4[1] + be4[1];
-                x[2] += (r4[rr].z - mu) * rs * g4[2] + be4[2];
-                x[3] += (r4[rr].w - mu) * rs * g4[3] + be4[3];
-              } else {
-                x[0] += r4[rr].x; x[1] += r4[rr].y; x[2] += r4[rr].z; x[3] += r4[rr].w;
-              }
-              st4(cp, x);
-              if (qp) st4(qp, x);
-            }
-            cp += step;
-            if (qp) qp += step;
           }
         }
       }

@@ -853,6 +853,81 @@ __global__ void nr_reduce_kernel(const float* __restrict__ part, int B, int d_a,
   else loss[0] = a * invB;
 }
 
+// ---------------------------------------------------------------------------- NR task: the clicked items as packed sequences
+// One block.  User b's clicked slots (the history positions whose label is not negative) become sequence b of a packed
+// layout: seq_len[b] = their number, seq_off = its exclusive prefix sum, rows[seq_off[b] + k] = position of the k-th clicked
+// slot, pos2row[position] = its packed row (-1 for empty slots and candidates).  rows[r] = -1 for the unused tail r >= total.
+__global__ void __launch_bounds__(1024) nr_layout_kernel(const int32_t* __restrict__ labels, int B, int L, int n_hist,
+                                                         int32_t* __restrict__ seq_len, int32_t* __restrict__ seq_off,
+                                                         int32_t* __restrict__ rows, int32_t* __restrict__ pos2row) {
+  __shared__ int32_t total;
+  if (threadIdx.x == 0) total = 0;
+  __syncthreads();
+  for (int b = 0; b < B; ++b) {                  // users in order: a few dozen to a few hundred per batch
+    const int32_t base = total;
+    __syncthreads();
+    int32_t placed = 0;
+    for (int n0 = 0; n0 < L; n0 += 1024) {
+      const int n = n0 + (int)threadIdx.x;
+      const bool hist = n < n_hist, clicked = hist && (!labels || labels[(int64_t)b * L + n] >= 0);
+      // rank of this slot among the clicked ones of the user: block-wide count of clicked slots before it
+      __shared__ int32_t wsum[32];
+      const uint32_t vote = __ballot_sync(0xffffffffu, clicked);
+      const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+      if (lane == 0) wsum[warp] = __popc(vote);
+      __syncthreads();
+      int32_t before = placed;
+      for (int w = 0; w < warp; ++w) before += wsum[w];
+      int32_t all = 0;
+      for (int w = 0; w < 32; ++w) all += wsum[w];
+      const int32_t rank = before + __popc(vote & ((1u << lane) - 1u));
+      if (n < L) pos2row[(int64_t)b * L + n] = clicked ? base + rank : -1;
+      if (clicked) rows[base + rank] = b * L + n;
+      placed += all;
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      seq_len[b] = placed;
+      seq_off[b] = base;
+      total = base + placed;
+    }
+    __syncthreads();
+  }
+  const int32_t t = total;
+  if (threadIdx.x == 0) seq_off[B] = t;
+  for (int64_t r = t + threadIdx.x; r < (int64_t)B * n_hist; r += blockDim.x) rows[r] = -1;
+}
+
+// out[r, :] = src[rows[r], :] (zero rows where rows[r] < 0), fp32, and an operand-typed copy when out_b is given
+template <typename T>
+__global__ void nr_pack_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows, int64_t n, int d,
+                               float* __restrict__ out, T* __restrict__ out_b) {
+  const int64_t r = blockIdx.x;
+  const int32_t p = rows[r];
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = p >= 0 ? src[(int64_t)p * d + c] : 0.f;
+    out[r * d + c] = v;
+    if (out_b) stf(out_b + r * d + c, v);
+  }
+}
+
+// out[p, :] = y(pos2row[p], :) where the position has a packed row, else other[p, :]; y is a view of the residual stream
+__global__ void nr_select_kernel(StreamRef y, const int32_t* __restrict__ pos2row, const float* __restrict__ other, int64_t P, int d,
+                                 float* __restrict__ out) {
+  const int64_t p = blockIdx.x;
+  const int32_t r = pos2row[p];
+  if (r < 0) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) out[p * d + c] = other[p * d + c];
+    return;
+  }
+  const bool ln = y.mean != nullptr;
+  const float mu = ln ? y.mean[r] : 0.f, rs = ln ? y.rstd[r] : 1.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = y.z[(int64_t)r * d + c];
+    out[p * d + c] = ln ? (v - mu) * rs * y.gamma[c] + y.beta[c] : v;
+  }
+}
+
 // ---------------------------------------------------------------------------- element-wise
 __global__ void f32_to_bf16_kernel(const float* __restrict__ in, bf16* __restrict__ out, size_t n) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
@@ -1297,6 +1372,31 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
     nr_user_kernel<T><<<B, 256, smem, st>>>(E, (const T*)pre, qa, dE, (T*)dpre, scratch, L, n_cand, d, d_a, 1.f / (float)B, labels);
   });
   nr_reduce_kernel<<<ceil_div(d_a + 1, 256), 256, 0, st>>>(scratch, B, d_a, 1.f / (float)B, dqa, loss);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+
+gram_status nr_layout(gram_ctx* ctx, const int32_t* labels, int B, int L, int n_hist, int32_t* seq_len, int32_t* seq_off,
+                      int32_t* rows, int32_t* pos2row, cudaStream_t st) {
+  if (B == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 12.0 * (double)B * L, 1, st);
+  nr_layout_kernel<<<1, 1024, 0, st>>>(labels, B, L, n_hist, seq_len, seq_off, rows, pos2row);
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status nr_pack(gram_ctx* ctx, int dtype, const float* src, const int32_t* rows, int64_t n, int d, float* out, void* out_b,
+                    cudaStream_t st) {
+  if (n == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, (double)n * d * (8.0 + (out_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), 1, st);
+  DISPATCH_T(dtype, nr_pack_kernel<T><<<(unsigned)n, d >= 256 ? 256 : 64, 0, st>>>(src, rows, n, d, out, (T*)out_b));
+  GRAM_LAUNCH_CHECK(ctx);
+  return GRAM_OK;
+}
+gram_status nr_select(gram_ctx* ctx, const StreamRef& y, const int32_t* pos2row, const float* other, int64_t P, int d, float* out,
+                      cudaStream_t st) {
+  if (P == 0) return GRAM_OK;
+  ProfScope prof(ctx, GRAM_K_TASK_HEAD, 8.0 * (double)P * d, 1, st);
+  nr_select_kernel<<<(unsigned)P, d >= 256 ? 256 : 64, 0, st>>>(y, pos2row, other, P, d, out);
   GRAM_LAUNCH_CHECK(ctx);
   return GRAM_OK;
 }

@@ -138,6 +138,18 @@ gram_status nr_user(gram_ctx* ctx, int dtype, const float* E, const void* pre, c
                     float* dqa, float* loss, float* scratch, const int32_t* labels, int B, int L, int n_cand, int d, int d_a,
                     cudaStream_t st);
 
+// News task with self-attention layers over the clicked items (Appendix D): the clicked history slots of every user as
+// packed sequences.  nr_layout: seq_len [B], seq_off [B + 1], rows [B * n_hist] (position of each packed row, -1 in the
+// unused tail), pos2row [B * L] (packed row of each position, -1 for empty slots and candidates); labels may be null (every
+// slot clicked).  nr_pack: out[r] = src[rows[r]] or a zero row, fp32 plus an operand-typed copy (out_b may be null).
+// nr_select: out[p] = y[pos2row[p]] where that is a row, else other[p].
+gram_status nr_layout(gram_ctx* ctx, const int32_t* labels, int B, int L, int n_hist, int32_t* seq_len, int32_t* seq_off,
+                      int32_t* rows, int32_t* pos2row, cudaStream_t st);
+gram_status nr_pack(gram_ctx* ctx, int dtype, const float* src, const int32_t* rows, int64_t n, int d, float* out, void* out_b,
+                    cudaStream_t st);
+gram_status nr_select(gram_ctx* ctx, const StreamRef& y, const int32_t* pos2row, const float* other, int64_t P, int d, float* out,
+                      cudaStream_t st);
+
 // element-wise helpers
 gram_status convert_f32_to_bf16(gram_ctx* ctx, const float* in, bf16* out, size_t n, cudaStream_t st);
 gram_status convert_to_f32(gram_ctx* ctx, int dtype, const void* in, float* out, size_t n, cudaStream_t st);

@@ -123,6 +123,9 @@ struct Model {
   Stack tk;
   float* tx = nullptr;               // task input stream, fp32
   void *txb = nullptr, *pre = nullptr, *dpre = nullptr;
+  // news task with self-attention layers over the clicked items: their packed layout, and the encodings after the layers
+  int32_t *nr_len = nullptr, *nr_off = nullptr, *nr_rows = nullptr, *nr_pos2row = nullptr;
+  float *nr_E2 = nullptr, *nr_dE2 = nullptr;
   // step buffers
   int32_t* item_tokens = nullptr;
   int32_t *ids = nullptr, *labels = nullptr, *unique = nullptr, *inverse = nullptr, *perm = nullptr, *seg_off = nullptr,
@@ -235,6 +238,18 @@ void layout_buffers(Model* m, Arena& a) {
     } else {
       m->pre = a.take((size_t)P * c.d_a * esz);
       m->dpre = a.take((size_t)P * c.d_a * esz);
+      if (c.task_layers > 0) {
+        const size_t Th = (size_t)m->tk.cap;
+        m->tx = (float*)a.take(Th * d * 4);
+        m->txb = a.take(Th * d * esz);
+        stack_buffers(a, m->tk, esz);
+        m->nr_len = (int32_t*)a.take((size_t)c.B_max * 4);
+        m->nr_off = (int32_t*)a.take(((size_t)c.B_max + 1) * 4);
+        m->nr_rows = (int32_t*)a.take(Th * 4);
+        m->nr_pos2row = (int32_t*)a.take((size_t)P * 4);
+        m->nr_E2 = (float*)a.take((size_t)P * d * 4);
+        m->nr_dE2 = (float*)a.take((size_t)P * d * 4);
+      }
     }
   }
   m->ids = (int32_t*)a.take((size_t)P * 4);
@@ -654,6 +669,26 @@ gram_status task_forward_backward(Model* m, const EncodingSource& src, const int
   if (c.task == GRAM_TASK_NR) {
     if (src.index || src.rows_bf16 || !dE) return gram_set_error(ctx, "the news task reads materialised fp32 encodings"), GRAM_ERR_ARG;
     const float* E = (const float*)src.rows;
+    const float* E_in = E;
+    float* dE_out = dE;
+    const int n_hist = c.L - c.n_cand;
+    const int64_t Th = (int64_t)B * n_hist;
+    if (c.task_layers > 0) {
+      // the clicked items of every user pass through the self-attention layers as one packed sequence per user; the rows
+      // after the last clicked item are zero rows that no sequence owns, so the layers run on B * n_hist rows whatever
+      // the number of clicks, and nothing has to be read back
+      GRAM_TRY(nr_layout(ctx, labels, B, c.L, n_hist, m->nr_len, m->nr_off, m->nr_rows, m->nr_pos2row, st));
+      GRAM_TRY(nr_pack(ctx, m->dtype, E_in, m->nr_rows, Th, c.d, m->tx, m->txb, st));
+      m->tk.seq_len = m->nr_len; m->tk.seq_off = m->nr_off; m->tk.packed_rows = Th; m->tk.grouped = false;
+      StreamRef x;
+      x.z = m->tx;
+      StreamRef y;
+      const void* y_b = nullptr;
+      GRAM_TRY(stack_forward(m, m->task, m->tk, x, m->txb, B, n_hist, st, &y, &y_b));
+      GRAM_TRY(nr_select(ctx, y, m->nr_pos2row, E_in, P, c.d, m->nr_E2, st));
+      E = m->nr_E2;
+      dE = m->nr_dE2;
+    }
     const void* Eb = E;                  // fp32 contexts: the stream is its own operand
     if (m->dtype == GRAM_BF16) {
       GRAM_TRY(convert_f32_to_bf16(ctx, E, (bf16*)m->Eb, (size_t)P * c.d, st));
@@ -669,6 +704,17 @@ gram_status task_forward_backward(Model* m, const EncodingSource& src, const int
     e = GemmEpilogue();
     e.accumulate = 1;                    // dE already holds the direct part
     GRAM_TRY(mm_dx(m, m->dpre, W(m, m->task, m->t_wa), dE, true, P, c.d_a, c.d, e, st));
+    if (c.task_layers > 0) {
+      // back through the layers: the gradient rows of the clicked items, packed; then every position takes the layers'
+      // input gradient where it has a packed row and the direct gradient (candidates; zeros at empty slots) elsewhere
+      void* dy_b = m->tk.attn_only ? m->tk.dzb : nullptr;
+      GRAM_TRY(nr_pack(ctx, m->dtype, dE, m->nr_rows, Th, c.d, m->tk.curf, dy_b, st));
+      float* dx = nullptr;
+      GRAM_TRY(stack_backward(m, m->task, m->tk, m->txb, B, n_hist, st, &dx));
+      StreamRef dxr;
+      dxr.z = dx;
+      GRAM_TRY(nr_select(ctx, dxr, m->nr_pos2row, dE, P, c.d, dE_out, st));
+    }
     return GRAM_OK;
   }
   return gram_set_error(ctx, "the context has no task module"), GRAM_ERR_ARG;
@@ -798,6 +844,13 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
     m->t_headb = at; at += 1;
   } else if (c.task == GRAM_TASK_NR) {
     if (c.d_a <= 0 || c.n_cand <= 0 || c.n_cand >= c.L) return gram_set_error(ctx, "bad task shape"), GRAM_ERR_ARG;
+    if (c.task_layers > 0) {             // self-attention layers over the clicked items, ahead of the additive attention
+      if (c.task_heads <= 0 || c.d % c.task_heads) return gram_set_error(ctx, "bad task shape"), GRAM_ERR_ARG;
+      m->tk.d = c.d; m->tk.heads = c.task_heads; m->tk.d_ff = c.task_d_ff; m->tk.n_layers = c.task_layers;
+      m->tk.attn_only = c.task_attn_only ? 1 : 0; m->tk.causal = 0;
+      m->tk.off.resize(c.task_layers);
+      for (int l = 0; l < c.task_layers; ++l) at = layer_layout(&m->tk.off[l], at, c.d, c.task_d_ff, m->tk.attn_only);
+    }
     m->t_wa = at; at += (size_t)c.d_a * c.d;
     m->t_ba = at; at += c.d_a;
     m->t_qa = at; at += c.d_a;
@@ -810,7 +863,7 @@ gram_status model_create(gram_ctx* ctx, const gram_config* cfg, Model** out) {
   if (mb > c.n_items) mb = c.n_items;
   m->mb = (int32_t)mb;
   m->enc.cap = (int64_t)m->mb * c.l_t;
-  m->tk.cap = P;
+  m->tk.cap = c.task == GRAM_TASK_NR ? (int64_t)c.B_max * (c.L - c.n_cand) : P;
   m->cls_tail = c.n_layers > 0 && c.pooling == GRAM_POOL_CLS && c.l_t > 1;
   if (m->cls_tail) {
     m->tail.d = c.d; m->tail.heads = c.n_heads; m->tail.d_ff = c.d_ff; m->tail.n_layers = 1;

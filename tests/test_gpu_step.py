@@ -27,6 +27,13 @@ CASES = {
     "cls_full_task": small(pooling="cls", task_attn_only=False, task_layers=2),
     "odd_sizes": small(n_items=23, l_t=5, d=24, n_heads=3, d_ff=40, B=3, L=7, task_heads=2),
     "nr": small(task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls"),
+    # the news task with one self-attention layer over the clicked items (Appendix D), attention only and with the whole layer
+    "nr_mhsa": small(task="nr", task_layers=1, task_heads=2, task_attn_only=True, n_cand=3, L=9, d_a=16, pooling="cls"),
+    "nr_mhsa_full": small(task="nr", task_layers=1, task_heads=2, task_attn_only=False, n_cand=3, L=9, d_a=16, pooling="cls"),
+    "bf16_nr_mhsa": small(dtype="bf16", task="nr", task_layers=1, task_heads=2, task_attn_only=True, n_cand=3, L=9, d_a=16,
+                          pooling="cls", d=64, d_ff=128),
+    "bf16_nr_mhsa_dh64": small(dtype="bf16", task="nr", task_layers=1, task_heads=2, task_attn_only=False, task_d_ff=128, n_cand=4,
+                               L=24, B=5, d_a=16, pooling="cls", d=128, d_ff=128, l_t=16),
     "tiny_bf16": synth.config("tiny").replace(dtype="bf16"),
     "bf16_cls_full": small(dtype="bf16", pooling="cls", task_attn_only=False, d=64, d_ff=128, task_d_ff=128),
     "bf16_nr": small(dtype="bf16", task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls", d=64, d_ff=128),
@@ -562,7 +569,7 @@ def test_additive_attention_pooling(name, var_len):
     assert np.abs(gce["pool_qa"]).max() > 0 and np.abs(gce["pool_wa"]).max() > 0
 
 
-@pytest.mark.parametrize("name", ["nr", "bf16_nr"])
+@pytest.mark.parametrize("name", ["nr", "bf16_nr", "nr_mhsa", "nr_mhsa_full", "bf16_nr_mhsa"])
 def test_click_histories_with_empty_slots(name):
     """NR: history slots with label -1 hold no click: they take no part in the user vector and get zero gradient rows."""
     shape = CASES[name]
@@ -584,3 +591,20 @@ def test_click_histories_with_empty_slots(name):
     assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
     full = orc.e2e_step(shape, ce, tk, toks, ids, np.zeros_like(lab))
     assert abs(full["loss"] - want["loss"]) > 1e-6                                  # the mask matters
+
+
+def test_tcgen05_attention_on_short_sequences_too():
+    """Sequences of up to 128 rows take the warp-level attention kernels by default (they are the faster ones there); the
+    tcgen05 kernels serve them as well when GRAM_ATTN_TC=1.  The choice is read once per process, so the cases with heads of
+    width 64 are run again in a child process with the switch set: slots of 8 to 128 rows, packed rows, causal tiles."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, GRAM_ATTN_TC="1")
+    sel = "bf16_dh64_s16 or bf16_dh64_s24 or bf16_dh64_s64 or bf16_dh64_s128 or bf16_dh64_var40 or bf16_dh64_var128 or bf16_long_seq"
+    out = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_step.py"), "-m", "gpu", "-q", "-x",
+                          "-k", f"({sel}) and not tcgen05_attention_on_short"], cwd=root, env=env, capture_output=True, text=True,
+                         timeout=1200)
+    assert out.returncode == 0, out.stdout[-3000:] + out.stderr[-1000:]
+    assert " passed" in out.stdout and "failed" not in out.stdout
