@@ -88,7 +88,7 @@ def gemm_traffic_per_row():
     """DRAM bytes per token row of the forward qkv product from the committed ncu summary; None when gemm.cu has
     changed since the counters were taken."""
     import hashlib
-    prof = os.path.join(ROOT, "profiles", "gemm_tc2_fwd_qkv_shape.md")
+    prof = os.path.join(ROOT, "profiles", "gemm_call_sites_65536_rows.md")
     src = os.path.join(ROOT, "paper_2204_04179_b200", "csrc", "gemm.cu")
     if not (os.path.exists(prof) and os.path.exists(src)):
         return None
@@ -529,6 +529,15 @@ def run_gram(args, shape):
     kinds = g.profile_read()
     sites = g.profile_dump()
     g.profile(False)
+    light_sites = None
+    if multistep and shape.K > 1:
+        # one more window, with the K-1 steps that run no encoder pass instrumented on their own: where a light step's time goes
+        g.profile(True)
+        for k in range(args.warmup, args.warmup + shape.K - 1):
+            run.step(k, dist)
+        light_sites = g.profile_dump()
+        g.profile(False)
+        run.step(args.warmup + shape.K - 1, dist)
 
     if rank != 0:
         run.close()
@@ -591,6 +600,8 @@ def run_gram(args, shape):
     }
     if multistep:
         line["multistep"] = {"K": shape.K, "windows_timed": args.steps // shape.K, "variant": args.multistep_variant,
+                             "light_step_call_sites": {t: {"ms_per_step": v["ms"] / (shape.K - 1), "launches_per_step": v["launches"] / (shape.K - 1)}
+                                                       for t, v in (light_sites or {}).items()},
                              "per_step": [{"k": i % shape.K, "ms": r.ms_total, "touched": r.n_touched,
                                            "encoder_pass": r.encoder_pass, "n_encoded": r.n_encoded} for i, r in enumerate(reports)]}
     batches0 = run.batches[0]

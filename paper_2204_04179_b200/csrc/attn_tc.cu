@@ -201,7 +201,7 @@ __device__ __forceinline__ void zero_outside(uint32_t buf, int r, int cb) {
     if (col < cb || col >= cb + W) sts128(swz(buf + (uint32_t)(piece >> 3) * TILE_BYTES, r, piece & 7), 0u, 0u, 0u, 0u);
   }
 }
-// 32 packed bf16 pairs... the 16 words pk (32 columns from column c0) into row r of such a tile
+// the 16 words pk (32 bf16 columns from column c0) into row r of such a tile
 __device__ __forceinline__ void store_block32(uint32_t buf, int r, int c0, const uint32_t (&pk)[16]) {
   const int piece0 = c0 >> 3;
 #pragma unroll
@@ -305,14 +305,6 @@ __device__ __forceinline__ void bwd_block(uint32_t lane_base, uint32_t pbuf, uin
   if (__all_sync(0xffffffffu, l0 == 0 && h0 == W)) bwd_block_m<W, true>(lane_base, pbuf, dsbuf, r, cb, l0, h0, c, lse2, scale, own_delta, delta_in);
   else bwd_block_m<W, false>(lane_base, pbuf, dsbuf, r, cb, l0, h0, c, lse2, scale, own_delta, delta_in);
 }
-
-struct Shared {
-  uint32_t tiles;            // shared-memory address of the first stage (1024-byte aligned)
-  uint32_t pbuf;             // the softmax groups' probability tiles
-  uint32_t bar0;             // first barrier
-  uint32_t* tmem_slot;
-  volatile int* abort_flag;
-};
 
 // ============================================================================================
 // forward

@@ -710,7 +710,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
 // moves 32 KB through shared memory instead of 48 KB, which is what bounds the single-CTA kernel.
 // Protocol: each CTA's TMA loads signal the leader's "full" barrier (two arrivals with their byte
 // counts); the leader's commits arrive on the "empty" and "accumulator full" barriers of both CTAs
-// (one commit per CTA, no multicast); the epilogue warps of both CTAs arrive on the leader's
+// (one plain commit per CTA); the epilogue warps of both CTAs arrive on the leader's
 // "accumulator empty" barrier.  Every wait is bounded as in the single-CTA kernel; the CTAs meet at a
 // cluster barrier before they exit so that neither releases shared or tensor memory the other may
 // still touch.
@@ -1054,10 +1054,11 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
       const int64_t row0 = (int64_t)tm * 2 * BM + (int64_t)rank * BM + q * 32;
       if constexpr (TS) {
         constexpr int NB = 32 / EW;               // blocks of 32 columns per warp
-        if (!epilogue_tile_ts<MODE, NB>(a, &tmC, &tmP, (int32_t)row0, tn * BN + half * (NB * 32), half * (NB * 32), q, lane,
+        const bool ok = epilogue_tile_ts<MODE, NB>(a, &tmC, &tmP, (int32_t)row0, tn * BN + half * (NB * 32), half * (NB * 32), q, lane,
                                     tiles + STAGES * Cfg::STAGE_BYTES + (uint32_t)(ew * WARP_BYTES), tmem_base, buf, tfull_bar(buf),
                                     (uint32_t)((it >> 1) & 1), abort_flag, map_to_cta(tempty_bar(buf), 0), ld_bar(ew),
-                                    (uint32_t)(it & 1))) {
+                                    (uint32_t)(it & 1));
+        if (!ok) {
           failed = true;
           break;
         }
