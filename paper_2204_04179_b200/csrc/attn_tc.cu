@@ -971,13 +971,14 @@ void plan_launch(AttnArgs& a, int64_t n_seq, int S, bool contiguous) {
 }  // namespace
 
 // Which sequences take these kernels: GRAM_ATTN_TC=1 in the environment: all (head width 64); GRAM_ATTN_TC=0: none;
-// unset: those the warp-level kernels cannot hold (more than 128 rows).  For short sequences the warp-level kernels, with
-// many small blocks per SM, hide memory latency better than one persistent block per SM does and are the faster ones
-// as measured on the knowledge-tracing workload.
+// unset: sequences of more than 64 rows.  Up to 64 rows the warp-level kernels keep several small blocks per SM resident
+// and hide memory latency by occupancy, which one persistent block per SM does not (measured on the knowledge-tracing
+// encoder: 5.9 + 16.2 ms per step against 6.9 + 19.0 ms); from 65 rows on their one-sequence tile fills an SM with a
+// single block, and beyond 128 rows they cannot hold a sequence at all.
 bool attention_tc_supported(int S, int d, int n_heads) {
   static const int mode = []() { const char* v = getenv("GRAM_ATTN_TC"); return !v ? 2 : (v[0] == '0' ? 0 : 1); }();
   if (mode == 0 || !(S >= 1 && n_heads > 0 && d == n_heads * DH && get_encode_fn() != nullptr)) return false;
-  return mode == 1 || S > TQ;
+  return mode == 1 || S > 64;
 }
 
 gram_status attention_forward_tc(gram_ctx* ctx, const void* qkv, void* out, float* lse, int64_t rows, int64_t n_seq, int S, int d,
