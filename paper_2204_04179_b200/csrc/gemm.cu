@@ -298,7 +298,8 @@ template <int BN> struct TcCfg {
 //   EPI_BIAS  (+ bias), bf16 or fp32 out
 //   EPI_GELU  + bias, GELU, saved derivative, both bf16
 //   EPI_RES   (+ bias) + fp32 residual (LayerNorm on the fly when res_mean is set), fp32 out (+ bf16 copy)
-enum { EPI_GENERAL = 0, EPI_DG = 1, EPI_BIAS = 2, EPI_GELU = 3, EPI_RES = 4 };
+//   EPI_RES_TS  the same without the bf16 copy, residual in and result out by bulk tensor copies (pair kernel)
+enum { EPI_GENERAL = 0, EPI_DG = 1, EPI_BIAS = 2, EPI_GELU = 3, EPI_RES = 4, EPI_RES_TS = 5 };
 
 template <int BN, typename CT, int MODE, int PARTS = 2>
 __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t row0, int tn, int half, int q, int lane,
@@ -387,36 +388,38 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, CT* Cs, int64_t r
       stage_write_row(stage, lane, v);
       __syncwarp();
       const int n = nbase + blk * 32;
-      if (n < a.N) {
-        float b4[4] = {0.f, 0.f, 0.f, 0.f}, g4[4] = {0.f, 0.f, 0.f, 0.f}, be4[4] = {0.f, 0.f, 0.f, 0.f};
+      const bool col_ok = n < a.N;                          // lanes of a warp may differ here when N is not a multiple of 32
+      float b4[4] = {0.f, 0.f, 0.f, 0.f}, g4[4] = {0.f, 0.f, 0.f, 0.f}, be4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (col_ok) {
         if (a.epi.bias) ld4(a.epi.bias + n, b4);
         if (ln) {
           ld4(a.epi.res_gamma + n, g4);
           ld4(a.epi.res_beta + n, be4);
         }
-        CT* cp = Cs + obase + blk * 32;
-        bf16* qp = a.epi.copy_out ? reinterpret_cast<bf16*>(a.epi.copy_out) + obase + blk * 32 : nullptr;
+      }
+      CT* cp = Cs + obase + blk * 32;
+      bf16* qp = a.epi.copy_out ? reinterpret_cast<bf16*>(a.epi.copy_out) + obase + blk * 32 : nullptr;
 #pragma unroll
-        for (int rr = 0; rr < 8; ++rr) {
-          const int rl = rr * 4 + sub;
-          const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
-          if (rr * 4 < rows_left) {
-            const float4 t = stage_read(stage, rl, slot);
-            float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
-            if (ln) {
-              x[0] += (r4[rr].x - mu) * rs * g4[0] + be4[0];
-              x[1] += (r4[rr].y - mu) * rs * g4[1] + be4[1];
-              x[2] += (r4[rr].z - mu) * rs * g4[2] + be4[2];
-              x[3] += (r4[rr].w - mu) * rs * g4[3] + be4[3];
-            } else {
-              x[0] += r4[rr].x; x[1] += r4[rr].y; x[2] += r4[rr].z; x[3] += r4[rr].w;
-            }
-            st4(cp, x);
-            if (qp) st4(qp, x);
+      for (int rr = 0; rr < 8; ++rr) {
+        const int rl = rr * 4 + sub;
+        // every lane takes part in the shuffles, whatever its columns
+        const float mu = __shfl_sync(0xffffffffu, mu_l, rl), rs = __shfl_sync(0xffffffffu, rs_l, rl);
+        if (col_ok && rr * 4 < rows_left) {
+          const float4 t = stage_read(stage, rl, slot);
+          float x[4] = {t.x + b4[0], t.y + b4[1], t.z + b4[2], t.w + b4[3]};
+          if (ln) {
+            x[0] += (r4[rr].x - mu) * rs * g4[0] + be4[0];
+            x[1] += (r4[rr].y - mu) * rs * g4[1] + be4[1];
+            x[2] += (r4[rr].z - mu) * rs * g4[2] + be4[2];
+            x[3] += (r4[rr].w - mu) * rs * g4[3] + be4[3];
+          } else {
+            x[0] += r4[rr].x; x[1] += r4[rr].y; x[2] += r4[rr].z; x[3] += r4[rr].w;
           }
-          cp += step;
-          if (qp) qp += step;
+          st4(cp, x);
+          if (qp) st4(qp, x);
         }
+        cp += step;
+        if (qp) qp += step;
       }
       __syncwarp();
     }
@@ -878,8 +881,112 @@ __device__ __forceinline__ bool epilogue_tile_ts(const TcArgs& a, const CUtensor
   return true;
 }
 
+// Epilogue of the pair kernel for the fp32 residual products (EPI_RES_TS): result = accumulator (+ bias) + residual,
+// the residual being the fp32 stream or LayerNorm of it applied where it is read.  One warp owns rows row0 .. row0+31
+// and four blocks of 32 columns from global column col0.  The residual is 4 bytes per element from HBM and the result
+// 4 bytes back: both travel as 32-row x 32-column boxes (128-byte rows, 128-byte swizzle) by bulk tensor copies, so the
+// warp issues no global load or store of its own and many boxes are in flight per SM.  A thread keeps its own row: 32
+// accumulators from tensor memory, its row of the residual box from shared memory, the sum written back in place,
+// and lane 0 hands the box to a bulk tensor store.  Three boxes per warp rotate (block k of the warp's running count
+// uses box k % 3 and load barrier k % 3): the loads of a tile's first two blocks are issued before the wait for the
+// accumulator, that of block b + 2 after the store of block b has been committed and the store before it has read its box.
+// sbuf: 12 KB, 1024-byte aligned, private to the warp; nb: the warp's running block count.
+__device__ __forceinline__ bool epilogue_tile_res(const TcArgs& a, const CUtensorMap* tmC, const CUtensorMap* tmR, int32_t row0,
+                                                  int32_t col0, int c_local, int q, int lane, uint32_t sbuf, uint32_t tmem_base,
+                                                  int buf, uint32_t tfull_addr, uint32_t parity, volatile int* abort_flag,
+                                                  uint32_t tempty_remote, uint32_t ld_bar0, uint32_t& nb) {
+  int nv = 0;                                               // blocks of this warp that lie inside the matrix
+  if (row0 < a.M) {
+    nv = (a.N - col0 + 31) / 32;
+    nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
+  }
+  auto request = [&](int b) {                               // residual box of block b of this tile -> box (nb + b) % 3
+    const uint32_t k = nb + (uint32_t)b;
+    const uint32_t bar = ld_bar0 + 8u * (k % 3u);
+    mbar_expect_tx(bar, 4096);
+    tma_load_2d(sbuf + (k % 3u) * 4096u, tmR, col0 + 32 * b, row0, bar);
+  };
+  if (lane == 0 && nv > 0) {
+    bulk_wait_read_but_one();                               // every store but the latest has read its box
+    request(0);
+    if (nv > 1) request(1);
+  }
+  const bool ln = a.epi.res_mean != nullptr;
+  float mu = 0.f, rs = 1.f;
+  if (ln && row0 + lane < a.M) {
+    mu = a.epi.res_mean[row0 + lane];
+    rs = a.epi.res_rstd[row0 + lane];
+  }
+  if (!mbar_wait(tfull_addr, parity, abort_flag)) return false;
+  tc_fence_after();
+  if (nv == 0) {
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive_remote(tempty_remote);
+    return true;
+  }
+  const uint32_t swz = (uint32_t)(lane & 7);
+#pragma unroll 1
+  for (int b = 0; b < nv; ++b) {
+    const uint32_t k = nb + (uint32_t)b;
+    const uint32_t box = sbuf + (k % 3u) * 4096u, srow = box + (uint32_t)lane * 128u;
+    uint32_t v[32];
+    tc_ld32_issue(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c_local + b * 32), v);
+    tc_ld32_wait(v);
+    if (b == nv - 1) {                                      // every value of this tile is in registers now
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(tempty_remote);
+    }
+    if (!mbar_wait(ld_bar0 + 8u * (k % 3u), (k / 3u) & 1u, abort_flag)) return false;
+    const int n = col0 + b * 32;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint32_t addr = srow + ((((uint32_t)c) ^ swz) << 4);
+      const uint4 ru = lds128(addr);
+      float x[4] = {__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]), __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3])};
+      const float r[4] = {__uint_as_float(ru.x), __uint_as_float(ru.y), __uint_as_float(ru.z), __uint_as_float(ru.w)};
+      if (n + 4 * c < a.N) {                                // N is a multiple of 8: a piece of four columns is in or out
+        if (a.epi.bias) {
+          const float4 b4 = __ldg(reinterpret_cast<const float4*>(a.epi.bias + n + 4 * c));
+          x[0] += b4.x; x[1] += b4.y; x[2] += b4.z; x[3] += b4.w;
+        }
+        if (ln) {
+          const float4 g4 = __ldg(reinterpret_cast<const float4*>(a.epi.res_gamma + n + 4 * c));
+          const float4 e4 = __ldg(reinterpret_cast<const float4*>(a.epi.res_beta + n + 4 * c));
+          x[0] += (r[0] - mu) * rs * g4.x + e4.x;
+          x[1] += (r[1] - mu) * rs * g4.y + e4.y;
+          x[2] += (r[2] - mu) * rs * g4.z + e4.z;
+          x[3] += (r[3] - mu) * rs * g4.w + e4.w;
+        } else {
+          x[0] += r[0]; x[1] += r[1]; x[2] += r[2]; x[3] += r[3];
+        }
+      }
+      sts128(addr, __float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      tma_store_2d(tmC, box, n, row0);
+      bulk_commit();
+      if (b + 2 < nv) {
+        bulk_wait_read_but_one();                           // the store of block b - 1 has read the box that block b + 2 takes
+        request(b + 2);
+      }
+    }
+    __syncwarp();
+  }
+  nb += (uint32_t)nv;
+  return true;
+}
+
 // EW epilogue warps per CTA: 8 (two per TMEM lane quarter) or, for the light epilogues whose register use allows
 // it, 16 (four per quarter, 64 columns each) with one pipeline stage fewer
+// bytes of private shared memory per epilogue warp: one 4 KB store box, two for the GELU epilogue (value and derivative),
+// three fp32 boxes for the residual epilogue
+template <typename CT, int MODE> constexpr int warp_bytes() {
+  return (sizeof(CT) == 4 && MODE == EPI_RES_TS) ? 12288 : ((sizeof(CT) == 2 && MODE == EPI_GELU) ? 8192 : 4096);
+}
 template <int EW, int WARP_BYTES = 4096> struct Tc2Cfg {
   static constexpr int BN = 256;                       // columns of the pair's tile
   static constexpr int A_BYTES = BM * BK * 2;          // this CTA's 128 rows of A
@@ -899,8 +1006,9 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
                                                                   const __grid_constant__ CUtensorMap tmB,
                                                                   const __grid_constant__ CUtensorMap tmC,
                                                                   const __grid_constant__ CUtensorMap tmP, TcArgs a) {
-  constexpr bool TS = sizeof(CT) == 2 && ((EW == 16 && MODE == EPI_DG) || MODE == EPI_BIAS || MODE == EPI_GELU);
-  constexpr int WARP_BYTES = (TS && MODE == EPI_GELU) ? 8192 : 4096;
+  constexpr bool RS = sizeof(CT) == 4 && MODE == EPI_RES_TS;       // fp32 residual epilogue through bulk tensor copies
+  constexpr bool TS = RS || (sizeof(CT) == 2 && ((EW == 16 && MODE == EPI_DG) || MODE == EPI_BIAS || MODE == EPI_GELU));
+  constexpr int WARP_BYTES = warp_bytes<CT, MODE>();
   using Cfg = Tc2Cfg<EW, WARP_BYTES>;
   constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -916,7 +1024,7 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };  // used in the leader
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  auto ld_bar = [&](int w) { return bar0 + 8u * (2 * STAGES + 6 + w); };      // one per epilogue warp (EPI_DG loads)
+  auto ld_bar = [&](int w) { return bar0 + 8u * (2 * STAGES + 6 + w); };      // one per epilogue warp (EPI_DG loads), three for EPI_RES_TS
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -931,7 +1039,7 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
       mbar_init(tempty_bar(b), 2 * EW);          // one arrival per epilogue warp of either CTA
     }
     if (TS) {
-      for (int w = 0; w < EW; ++w) mbar_init(ld_bar(w), 1);
+      for (int w = 0; w < (RS ? 3 * EW : EW); ++w) mbar_init(ld_bar(w), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1046,13 +1154,21 @@ __global__ void __launch_bounds__(64 + 32 * EW, 1) gemm_tc2_kernel(const __grid_
     float* stage = epi_stage + ew * (32 * STAGE_LD);
     CT* C = reinterpret_cast<CT*>(a.C);
     int64_t it = 0;
+    uint32_t res_blocks = 0;                      // EPI_RES_TS: this warp's running count of 32-column blocks
     for (int64_t t = cluster_id; t < total && !failed; t += n_clusters, ++it) {
       const int split = (int)(t / ((int64_t)a.n_tiles_m * a.n_tiles_n));
       const int64_t r = t - (int64_t)split * a.n_tiles_m * a.n_tiles_n;
       const int tm = (int)(r / a.n_tiles_n), tn = (int)(r % a.n_tiles_n);
       const int buf = (int)(it & 1);
       const int64_t row0 = (int64_t)tm * 2 * BM + (int64_t)rank * BM + q * 32;
-      if constexpr (TS) {
+      if constexpr (RS) {
+        if (!epilogue_tile_res(a, &tmC, &tmP, (int32_t)row0, tn * BN + half * 128, half * 128, q, lane,
+                               tiles + STAGES * Cfg::STAGE_BYTES + (uint32_t)(ew * WARP_BYTES), tmem_base, buf, tfull_bar(buf),
+                               (uint32_t)((it >> 1) & 1), abort_flag, map_to_cta(tempty_bar(buf), 0), ld_bar(3 * ew), res_blocks)) {
+          failed = true;
+          break;
+        }
+      } else if constexpr (TS) {
         constexpr int NB = 32 / EW;               // blocks of 32 columns per warp
         const bool ok = epilogue_tile_ts<MODE, NB>(a, &tmC, &tmP, (int32_t)row0, tn * BN + half * (NB * 32), half * (NB * 32), q, lane,
                                     tiles + STAGES * Cfg::STAGE_BYTES + (uint32_t)(ew * WARP_BYTES), tmem_base, buf, tfull_bar(buf),
@@ -1139,7 +1255,7 @@ cudaError_t launch_tc_major(bool a_k, bool b_k, const CUtensorMap& ma, const CUt
 template <bool A_K, bool B_K, typename CT, int MODE = EPI_GENERAL, int EW = EPI_WARPS>
 cudaError_t launch_tc2(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& args, int grid, cudaStream_t st,
                        const CUtensorMap* mc = nullptr, const CUtensorMap* mp = nullptr) {
-  using Tc2 = Tc2Cfg<EW, (sizeof(CT) == 2 && MODE == EPI_GELU) ? 8192 : 4096>;
+  using Tc2 = Tc2Cfg<EW, warp_bytes<CT, MODE>()>;
   auto kern = gemm_tc2_kernel<A_K, B_K, CT, MODE, EW>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -1174,6 +1290,11 @@ cudaError_t launch_tc2_major(bool a_k, bool b_k, const CUtensorMap& ma, const CU
 
 static bool pair_enabled_env() {
   static const bool on = []() { const char* v = getenv("GRAM_GEMM_PAIR"); return !(v && v[0] == '0'); }();
+  return on;
+}
+// GRAM_GEMM_RES_TS=0 in the environment keeps the register path of the fp32 residual epilogue (for comparisons)
+static bool res_ts_env() {
+  static const bool on = []() { const char* v = getenv("GRAM_GEMM_RES_TS"); return !(v && v[0] == '0'); }();
   return on;
 }
 bool gemm_fused_colsum(int dtype, int64_t M, int N) {
@@ -1300,10 +1421,20 @@ gram_status gemm_launch(gram_ctx* ctx, GemmWorkspace* ws, int dtype, const void*
     if (ts_ok && aux) ts_ok = make_map(&mp, aux, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, 32);
     const CUtensorMap* pc = &mc;
     const CUtensorMap* pp = aux ? &mp : &mc;
+    // the fp32 residual products with a short reduction (K <= 1024: the output projection of attention), where the epilogue's
+    // memory traffic outlasts the main loop: result and residual as fp32 boxes of 32 rows x 32 columns through bulk tensor
+    // copies (no bf16 copy on this path).  With longer K the register path keeps six pipeline stages instead of four and
+    // is the faster one (measured: 1279 against 1175 TFLOP/s at K = 3072).
+    CUtensorMap mcf, mrf;
+    const bool rs_ok = m_res && !e.copy_out && K <= 1024 && res_ts_env() && M < (int64_t)1 << 31 && (uintptr_t)e.res % 16 == 0 &&
+                       make_map_f32(&mcf, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 32, 32) &&
+                       make_map_f32(&mrf, e.res, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 32, 32);
     if (e.colsum_part && !(dg_only && ts_ok))
       return gram_set_error(ctx, "gemm: column-sum partials need the GELU-derivative variant with bulk stores"), GRAM_ERR_UNSUPPORTED;
     if (dg_only && ts_ok) err = launch_tc2<true, false, bf16, EPI_DG, 16>(ma, mb, args, grid, st, pc, pp);
     else if (m_gelu && ts_ok) err = launch_tc2<true, true, bf16, EPI_GELU, 8>(ma, mb, args, grid, st, pc, pp);
+    else if (m_res && rs_ok && b_kmajor) err = launch_tc2<true, true, float, EPI_RES_TS>(ma, mb, args, grid, st, &mcf, &mrf);
+    else if (m_res && rs_ok && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES_TS>(ma, mb, args, grid, st, &mcf, &mrf);
     else if (m_res && b_kmajor) err = launch_tc2<true, true, float, EPI_RES>(ma, mb, args, grid, st);
     else if (m_res && !b_kmajor) err = launch_tc2<true, false, float, EPI_RES>(ma, mb, args, grid, st);
     else if (m_bias && a_kmajor && b_kmajor && ts_ok) err = launch_tc2<true, true, bf16, EPI_BIAS, 8>(ma, mb, args, grid, st, pc, pp);

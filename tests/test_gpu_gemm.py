@@ -62,7 +62,7 @@ def _erf_gelu(v):
 
 
 # (M, N, K): full 256 x 256 pair tiles, ragged rows and columns, a small single-CTA shape, a wide N
-EPI_SHAPES = [(512, 768, 768), (1000, 768, 3072), (296, 3072, 768), (136, 200, 72), (2048, 2304, 768), (264, 264, 64)]
+EPI_SHAPES = [(512, 768, 768), (1000, 768, 3072), (296, 3072, 768), (136, 200, 72), (2048, 2304, 768), (264, 264, 64), (520, 1032, 128), (1288, 1096, 192)]
 
 
 @pytest.mark.parametrize("M,N,K", EPI_SHAPES)
