@@ -1114,7 +1114,12 @@ gram_status layernorm_backward(gram_ctx* ctx, int dtype, const float* dy, const 
   if (d > 1024 || (d & 3)) return gram_set_error(ctx, "LayerNorm: d must be a multiple of 4 and at most 1024"), GRAM_ERR_UNSUPPORTED;
   int cap = (int)(kRedScratchBytes / ((size_t)3 * d * sizeof(float)));
   if (cap > kNumSMs * 8) cap = kNumSMs * 8;
-  const int blocks = grid_for(rows * 32, 256, cap);
+  // at least sixteen rows per warp where the row count allows it: a block's fixed work (clearing and writing 3 d partial
+  // sums, which the reduction kernels then read) is otherwise most of a call on a few ten thousand rows
+  int64_t want = (rows + 127) / 128;
+  if (want < kNumSMs) want = kNumSMs;
+  if (want > cap) want = cap;
+  const int blocks = grid_for(rows * 32, 256, (int)want);
   const int nq = d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : d <= 768 ? 6 : 8;   // float4 per lane: the kernel's NQ
   const size_t smem = (size_t)4 * d * sizeof(float) + (dcol ? (size_t)8 * nq * 32 * sizeof(float4) : 0);
   ProfScope prof(ctx, GRAM_K_LAYERNORM, (double)rows * d * (12.0 + (dz_b ? (dtype == GRAM_BF16 ? 2.0 : 4.0) : 0.0)), dcol ? 3 : 2, st, "ln_bwd");

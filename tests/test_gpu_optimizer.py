@@ -1,4 +1,4 @@
-"""Adam with the Noam scheme (Section A) on the GPU against the oracle: the update kernel element by element, and
+"""Adam with the Noam scheme (Appendix D) on the GPU against the oracle: the update kernel element by element, and
 whole training steps through gram_step."""
 import numpy as np
 import pytest

@@ -608,3 +608,37 @@ def test_tcgen05_attention_on_short_sequences_too():
                          timeout=1200)
     assert out.returncode == 0, out.stdout[-3000:] + out.stderr[-1000:]
     assert " passed" in out.stdout and "failed" not in out.stdout
+
+
+@pytest.mark.parametrize("K", [1, 2])
+def test_deferred_update_and_device_gradient_buffers(K):
+    """defer_update: gram_step leaves the gradients in place and applies nothing; the device gradient buffers seen through
+    gram_grads_device are the ones gram_get_grads copies; gram_optimizer_step then applies the configured update, and
+    the result equals a context that updates inside the step (what a data-parallel trainer relies on between the two)."""
+    from paper_2204_04179_b200 import dist as gdist
+    shape = small(d=64, d_ff=128, task_d_ff=128, n_items=50, B=4, L=10, K=K, pooling="cls")
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=8)
+    kw = dict(K=K, lr_task=0.05, lr_ce=0.02, optimizer=binding.GRAM_OPT_ADAM, ce_micro_batch=16)
+    a = gh.make_ctx(shape, ce, tk, toks, **kw)
+    b = gh.make_ctx(shape, ce, tk, toks, defer_update=1, **kw)
+    if K > 1:
+        a.cache_fill(); b.cache_fill()
+    for step in range(2 * K):
+        ids, lab = synth.batch(shape, 8, step=step)
+        i_d, l_d = torch.from_numpy(ids).to(DEV), torch.from_numpy(lab).to(DEV)
+        ra = a.step(i_d, l_d, shape.B)
+        before = [b.get_params(m) for m in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK)]
+        rb = b.step(i_d, l_d, shape.B)
+        assert ra.loss == rb.loss and ra.encoder_pass == rb.encoder_pass
+        for m, p0 in zip((binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK), before):
+            assert np.array_equal(b.get_params(m), p0)                      # nothing applied yet
+        tens = gdist.gradient_tensors(b)
+        assert np.array_equal(tens[0].cpu().numpy(), b.get_grads(binding.GRAM_MODULE_CE))
+        assert np.array_equal(tens[1].cpu().numpy(), b.get_grads(binding.GRAM_MODULE_TASK))
+        assert gdist.allreduce_grads(b, gdist.n_predictions(shape, lab), None) == shape.B * shape.L     # one rank: unchanged
+        if rb.encoder_pass:
+            b.optimizer_step(binding.GRAM_MODULE_CE)
+        b.optimizer_step(binding.GRAM_MODULE_TASK)
+        for m in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK):
+            assert np.array_equal(a.get_params(m), b.get_params(m))
+    a.close(); b.close()

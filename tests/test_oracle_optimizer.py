@@ -1,4 +1,4 @@
-"""Pins for the oracle's optimiser (Adam with the Noam learning-rate scheme, Section A of the paper).
+"""Pins for the oracle's optimiser (Adam with the Noam learning-rate scheme, Appendix D of the paper).
 
 None of them re-types the oracle's formula: the Noam curve is checked at values that follow from its definition by
 hand, the Adam update against torch.optim.Adam (a library routine, constant rate) and against the closed form of the
