@@ -642,3 +642,34 @@ def test_deferred_update_and_device_gradient_buffers(K):
         for m in (binding.GRAM_MODULE_CE, binding.GRAM_MODULE_TASK):
             assert np.array_equal(a.get_params(m), b.get_params(m))
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_multistep_window_of_the_news_task(dtype):
+    """Multi-step GRAM with the news task module: the materialised gather from the cache (widened from bf16 in one pass in
+    bf16 contexts), K = 2 steps into the table, one encoder pass; losses, gradients, updated task parameters and the refreshed
+    cache against Algorithm 1 stepped by the oracle from the cache values the device holds."""
+    shape = small(dtype=dtype, task="nr", task_layers=0, n_cand=3, L=9, d_a=16, pooling="cls", d=64, d_ff=128, n_items=50, B=4, K=2)
+    ce, tk, toks, _, _ = gh.make_inputs(shape, seed=23)
+    lr = 0.05
+    batches = []
+    for k in range(2):
+        ids, lab = synth.batch(shape, 23, step=k)
+        batches.append((ids, np.zeros_like(lab)))
+    g = gh.make_ctx(shape, ce, tk, toks, K=2, lr_task=lr, ce_micro_batch=16)
+    g.cache_fill()
+    _, _, cache0 = g.get_window(want_table=False, want_touched=False)
+    want = orc.multistep_window(shape, ce, tk, toks, batches, cache0.astype(np.float64), lr_task=lr, cache_bf16=(dtype == "bf16"))
+    reps = [g.step(torch.from_numpy(i).to(DEV), torch.from_numpy(l).to(DEV), shape.B) for i, l in batches]
+    tol = TOL[dtype]
+    for k in range(2):
+        assert abs(reps[k].loss - want["losses"][k]) <= tol * abs(want["losses"][k])
+    assert [r.encoder_pass for r in reps] == [0, 1] and reps[-1].n_touched == len(want["items"])
+    gce, gtk = gh.gpu_grads(g, shape)
+    e1, n1 = gh.worst_rel_err(gce, want["grad_ce"])
+    e2, n2 = gh.worst_rel_err(gtk, want["grad_task_last"])
+    print(dtype, "worst CE", e1, n1, "worst task", e2, n2)
+    assert e1 <= tol and e2 <= tol, (e1, n1, e2, n2)
+    _, _, cache = g.get_window(want_table=False, want_touched=False)
+    assert gh.rel_err(cache, want["cache"]) <= tol
+    g.close()
