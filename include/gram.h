@@ -77,6 +77,9 @@ enum { GRAM_MULTI_TABLE = 0, GRAM_MULTI_PSEUDO_TARGET = 1 };
  * with the n_cand candidates, softmax cross-entropy on candidate 0 averaged
  * over B.  A context with n_layers == 0 and task == GRAM_TASK_NONE serves only
  * the index and accumulation calls.
+ * Texts and histories longer than 128 rows need dtype = GRAM_BF16 with heads of
+ * width 64 (d / n_heads, d / task_heads); other contexts return
+ * GRAM_ERR_UNSUPPORTED from the attention of such a sequence.
  * dtype = GRAM_BF16: matrix products and attention take bf16 operands with fp32
  * accumulation; the residual stream, LayerNorm statistics, encodings,
  * parameters and their gradients stay fp32.  GRAM_F32: everything fp32. */
@@ -252,9 +255,14 @@ gram_status gram_encoder_backward(gram_ctx* ctx, const float* d_G, const int32_t
  * context.  K > 1: encodings come from the cache (gram_cache_fill first), the
  * sums go to the table, and every K-th call runs the encoder forward and
  * backward over the touched items in micro-batches, refreshes their cache
- * rows and clears the window.  Task parameters take an SGD step of lr_task,
- * encoder parameters one of lr_ce after an encoder pass.  Synchronises; fills
- * *report (may be NULL). */
+ * rows and clears the window.  Task parameters take the configured update of
+ * rate lr_task, encoder parameters one of lr_ce after an encoder pass (none of
+ * it with defer_update).  Synchronises; fills *report (may be NULL).
+ * A batch with an item ID outside [0, n_items) returns GRAM_ERR_ID_RANGE and
+ * leaves parameters, optimiser state, table, touched bits, cache and the
+ * position in the window exactly as they were.  Host waits per call: K = 1:
+ * one after the dedup (U sizes the encoder pass) and one at the end; K > 1: one
+ * at the end, plus one on the K-th step for the number of touched items. */
 gram_status gram_step(gram_ctx* ctx, const int32_t* d_ids, const int32_t* d_labels, int32_t B,
                       gram_step_report* report, gram_stream stream);
 /* The same with HOST buffers: copies ids and labels to the device, runs the
