@@ -306,6 +306,27 @@ __device__ __forceinline__ void bwd_block(uint32_t lane_base, uint32_t pbuf, uin
   else bwd_block_m<W, false>(lane_base, pbuf, dsbuf, r, cb, l0, h0, c, lse2, scale, own_delta, delta_in);
 }
 
+// ---- pieces of the general softmax path (windows of up to 128 columns, several key tiles): 32 columns at a time ----
+// FULL: every row of the warp sees all 32 columns (no range tests)
+template <bool FULL>
+__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], int c0, int lo, int hi, float (&m4)[4]) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e)
+    if (FULL || (c0 + e >= lo && c0 + e < hi)) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(v[e]));
+}
+// probabilities exp2(c s - off) of 32 columns, packed to bf16 in pk; their sum goes to s4
+template <bool FULL>
+__device__ __forceinline__ void chunk_exp(const uint32_t (&v)[32], int c0, int lo, int hi, float c, float off, uint32_t (&pk)[16],
+                                          float (&s4)[4]) {
+#pragma unroll
+  for (int e = 0; e < 32; e += 2) {
+    const float p0 = (FULL || (c0 + e >= lo && c0 + e < hi)) ? ex2(fmaf(__uint_as_float(v[e]), c, -off)) : 0.f;
+    const float p1 = (FULL || (c0 + e + 1 >= lo && c0 + e + 1 < hi)) ? ex2(fmaf(__uint_as_float(v[e + 1]), c, -off)) : 0.f;
+    s4[(e >> 1) & 3] += p0 + p1;
+    pk[e >> 1] = pack_bf16x2(p0, p1);
+  }
+}
+
 // ============================================================================================
 // forward
 // barriers: full[s], empty[s] per stage; per softmax group g: s_full[g] (scores in tensor memory),
@@ -435,17 +456,17 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
         // the 32-column blocks some row of this warp needs
         const int wlo = __reduce_min_sync(0xffffffffu, hi > lo ? lo : TQ), whi = __reduce_max_sync(0xffffffffu, hi > lo ? hi : 0);
         const int q0 = wlo >> 5, q1 = (whi + 31) >> 5;     // blocks [q0, q1)
-        float mx = -INFINITY;
+        // the whole window visible to every row of the warp (inner key tiles of long sequences): no per-element tests
+        const bool full = __all_sync(0xffffffffu, lo == 0 && hi == TQ);
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         for (int q = q0; q < q1; ++q) {
           uint32_t v[32];
           tc_ld32_issue(s_addr + 32u * q, v);
           tc_ld32_wait(v);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int cidx = 32 * q + e;
-            if (cidx >= lo && cidx < hi) mx = fmaxf(mx, __uint_as_float(v[e]));
-          }
+          if (full) chunk_max<true>(v, 32 * q, lo, hi, m4);
+          else chunk_max<false>(v, 32 * q, lo, hi, m4);
         }
+        const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         const float m_new = fmaxf(m_run, mx);
         const float mc = (m_new == -INFINITY) ? 0.f : m_new * a.c;
         const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run * a.c - mc);
@@ -465,7 +486,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
           }
           tc_st_wait();
         }
-        float sum = 0.f;
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
         for (int q = 0; q < 4; ++q) {
           uint32_t pk[16];
@@ -473,14 +494,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
             uint32_t v[32];
             tc_ld32_issue(s_addr + 32u * q, v);
             tc_ld32_wait(v);
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const int cidx = 32 * q + e;
-              const float p0 = (cidx >= lo && cidx < hi) ? ex2(fmaf(__uint_as_float(v[e]), a.c, -mc)) : 0.f;
-              const float p1 = (cidx + 1 >= lo && cidx + 1 < hi) ? ex2(fmaf(__uint_as_float(v[e + 1]), a.c, -mc)) : 0.f;
-              sum += p0 + p1;
-              pk[e >> 1] = pack_bf16x2(p0, p1);
-            }
+            if (full) chunk_exp<true>(v, 32 * q, lo, hi, a.c, mc, pk, s4);
+            else chunk_exp<false>(v, 32 * q, lo, hi, a.c, mc, pk, s4);
           } else {
 #pragma unroll
             for (int e = 0; e < 16; ++e) pk[e] = 0u;
@@ -490,6 +505,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) attn_tc_fwd_kernel(const __gri
           for (int c4 = 0; c4 < 4; ++c4)
             sts128(swz(half, r, (q & 1) * 4 + c4), pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
         }
+        const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
         l_run = l_run * alpha + sum;
         m_run = m_new;
         }
